@@ -77,6 +77,8 @@ def validate(level, parent, cu):
     B = len(cu) - 1
     if cu[0] != 0:
         raise BadHierarchy("cu_seqlens[0] != 0")
+    if np.any(np.diff(cu) < 0) or int(cu[B]) != len(level):
+        raise BadHierarchy("cu_seqlens not monotone or not ending at the token count")
     for b in range(B):
         s0, s1 = int(cu[b]), int(cu[b + 1])
         if s1 < s0:
