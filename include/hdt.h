@@ -1,0 +1,180 @@
+/*
+ * libhdt — hierarchical sparse attention of the Hierarchical Document Transformer (HDT)
+ * for NVIDIA B200 (sm_100a).  C ABI; no C++ or framework types cross this boundary.
+ *
+ * The operation (paper, section "Hierarchical Document Transformer", paragraph
+ * "Hierarchical Attention", and Algorithm 1 in the appendix): tokens are laid out in document
+ * order with anchor tokens ([DOC], one [SEC] per section, one [SENT] per sentence).  Every
+ * token attends to its parent, its siblings (same parent, itself included) and its children;
+ * all other query-key pairs are masked with -inf before the row softmax:
+ *
+ *     A = Q K^T * softmax_scale,   S = softmax(A masked),   O = S V,
+ *     LSE_i = log sum_{j unmasked} exp(A_ij).
+ *
+ * The mask is the same for all heads and differs per sequence.
+ *
+ * Calling sequence:  hdt_build_index  (once per batch of documents; the index is valid for all
+ * layers, heads, forward and backward)  ->  hdt_attn_fwd / hdt_attn_bwd  (any number of times)
+ * ->  hdt_index_destroy.
+ *
+ * Conventions
+ *  - "device" pointers are CUDA device memory of the current device, owned by the caller.
+ *    The library never allocates or frees device memory; scratch comes in caller workspaces.
+ *  - Q, K, V, O, dO, dQ, dK, dV: packed token-major [total_tokens, heads, head_dim],
+ *    contiguous, 16-byte aligned, element type given by hdt_dtype_t.
+ *    LSE: float [heads, total_tokens], natural logarithm, softmax_scale included.
+ *  - Structure: level[i] in {0 root/[DOC], 1 [SEC], 2 [SENT], 3 regular token, deeper levels
+ *    allowed, -1 PAD}; parent[i] = index of the parent token relative to the start of its own
+ *    sequence, -1 for the root and for PAD; cu_seqlens[batch+1] cumulative sequence offsets
+ *    (cu_seqlens[0] = 0, cu_seqlens[batch] = total_tokens).  Preconditions, checked on the
+ *    device by hdt_build_index: the first token of a sequence is its only root (level 0);
+ *    0 <= parent[i] < i (sequence-relative); level[i] = level[parent[i]] + 1; tokens are in
+ *    document (pre-)order, i.e. a node whose children are all childless is directly followed
+ *    by those children; PAD only as a suffix of a sequence.
+ *    PAD rows produce O = 0, LSE = -inf and zero gradients.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  hdt_attn_fwd/bwd are
+ *    asynchronous on it.  hdt_build_index enqueues its kernels on it and then waits for them,
+ *    because it returns the sizes the attention calls need.
+ *  - Every function returns an hdt_status_t (HDT_OK = 0, errors negative); nothing throws,
+ *    aborts or traps the device.  hdt_last_error() gives a thread-local message.
+ */
+#ifndef HDT_H_
+#define HDT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HDT_OK = 0,
+    HDT_ERR_INVALID_ARG = -1,   /* null pointer, negative size, misaligned buffer            */
+    HDT_ERR_BAD_HIERARCHY = -2, /* structure arrays violate a precondition                    */
+    HDT_ERR_UNSUPPORTED = -3,   /* head_dim / dtype / size outside what the kernels cover     */
+    HDT_ERR_WORKSPACE = -4,     /* workspace too small                                        */
+    HDT_ERR_CUDA = -5,          /* a CUDA runtime call failed; see hdt_last_error()           */
+    HDT_ERR_TIMEOUT = -6        /* a bounded device-side wait ran out                         */
+} hdt_status_t;
+
+typedef enum { HDT_F32 = 0, HDT_BF16 = 1 } hdt_dtype_t;
+
+#define HDT_MAX_STAGES 16
+
+typedef struct {
+    int32_t block_m;    /* max rows per row block, 1..128; 0 = default 128                     */
+    int32_t max_stages; /* max hierarchy height handled, 1..HDT_MAX_STAGES; 0 = default 4
+                           ([DOC]/[SEC]/[SENT]/token documents need 3)                        */
+    int32_t reserved[6];
+} hdt_index_params_t;
+
+typedef struct hdt_index hdt_index_t; /* opaque host object; views into the caller's workspace */
+
+/*
+ * One stage of the index, device pointers into the index workspace (read-only).
+ * The index decomposes the mask into "families" {node} + its children, each of which is a
+ * contiguous range of a compacted token array; stage s handles the families whose members are
+ * all childless after the children handled by stages < s have been removed.  This replaces the
+ * per-tile emptiness test and the level sort of keys of the paper's Algorithm 1 (the "sort K, V"
+ * and "compute mask / if non-zero" steps): a row block's non-empty tiles are exactly its key
+ * span [a, b).
+ */
+typedef struct {
+    int32_t n;               /* elements in this stage's array                                */
+    int32_t n_blocks;        /* row blocks                                                    */
+    const int32_t *tok;      /* [n]   global token id of element e                            */
+    const int32_t *par;      /* [n]   index in this array of e's parent, -1 root / PAD        */
+    const int32_t *rng;      /* [n,2] key range [lo,hi) of row e in this array; (0,0) = none  */
+    const int32_t *up;       /* [n]   index of e in the next stage's array, -1 if removed     */
+    const int32_t *scu;      /* [batch+1] sequence offsets in this array                      */
+    const int32_t *blocks;   /* [n_blocks,5] r0, r1, a, b, flags (HDT_BLK_*)                  */
+    const int32_t *queue;    /* [n_blocks] block ids, cost (r1-r0)*(b-a) descending, id asc.  */
+} hdt_stage_view_t;
+
+#define HDT_BLK_SELF 1  /* key span inside the row block                                      */
+#define HDT_BLK_DENSE 2 /* every row's range equals the span: no in-tile masking needed       */
+#define HDT_BLK_CARRY 4 /* some row also has a partial result from a later stage              */
+#define HDT_BLK_EMPTY 8 /* no row has a key in this stage                                     */
+
+/*
+ * Bytes of device workspace hdt_build_index needs (host computation, no CUDA call).
+ * Returns 0 for invalid arguments.
+ */
+size_t hdt_index_workspace_bytes(int32_t batch, int32_t total_tokens,
+                                 const hdt_index_params_t *params /* NULL = defaults */);
+
+/*
+ * Build the index of one batch on the device (Algorithm 1's mask test and key ordering, done
+ * once per batch instead of per tile and per call).
+ *   level      device int8  [total_tokens]
+ *   parent     device int32 [total_tokens]
+ *   cu_seqlens device int32 [batch+1]
+ *   workspace  device, >= hdt_index_workspace_bytes(...), 256-byte aligned; must stay allocated
+ *              and untouched until hdt_index_destroy
+ *   out        receives a host object (free with hdt_index_destroy)
+ * Waits for the stream before returning.  Errors: HDT_ERR_BAD_HIERARCHY when a precondition on
+ * the structure arrays fails or the hierarchy needs more than max_stages stages (no index is
+ * returned), HDT_ERR_WORKSPACE, HDT_ERR_INVALID_ARG, HDT_ERR_CUDA.
+ */
+int hdt_build_index(const int8_t *level, const int32_t *parent, const int32_t *cu_seqlens,
+                    int32_t batch, int32_t total_tokens, const hdt_index_params_t *params,
+                    void *workspace, size_t workspace_bytes, void *stream, hdt_index_t **out);
+
+/* Totals of a built index: stages, unmasked pairs per head, visited pairs (sum of block rows x span). */
+int hdt_index_info(const hdt_index_t *index, int32_t *n_stages, int64_t *nnz_pairs,
+                   int64_t *visited_pairs);
+
+/* Device views of stage `stage` (0 <= stage < n_stages) for inspection and parity tests. */
+int hdt_index_export(const hdt_index_t *index, int32_t stage, hdt_stage_view_t *view);
+
+/* Frees the host object only. */
+int hdt_index_destroy(hdt_index_t *index);
+
+/*
+ * Bytes of device workspace for hdt_attn_fwd (bwd = 0) or hdt_attn_bwd (bwd = 1) with this
+ * index: partial results of the stages above stage 0, and delta = rowsum(dO o O) for backward.
+ */
+size_t hdt_attn_workspace_bytes(const hdt_index_t *index, int32_t heads, int32_t head_dim,
+                                int32_t dtype, int32_t bwd);
+
+/*
+ * Forward pass (hierarchical attention equation; Algorithm 1 without its per-tile HBM
+ * round trips): O and LSE for every token and head.
+ *   q, k, v   device [total_tokens, heads, head_dim] of `dtype`
+ *   o         device, same shape and dtype (written)
+ *   lse       device float [heads, total_tokens] (written)
+ *   softmax_scale <= 0 selects 1/sqrt(head_dim)
+ *   workspace device, >= hdt_attn_workspace_bytes(index, heads, head_dim, dtype, 0), 256-byte
+ *             aligned; contents are scratch
+ * head_dim must be 64 or 128.  Asynchronous on `stream`.
+ */
+int hdt_attn_fwd(const hdt_index_t *index, const void *q, const void *k, const void *v, void *o,
+                 float *lse, int32_t heads, int32_t head_dim, int32_t dtype, float softmax_scale,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Backward pass.  The paper prints no backward; this is the derivative of the forward map:
+ *   delta_i = sum_c dO_ic O_ic;  P_ij = exp(A_ij - LSE_i);  dV = P^T dO;  dP = dO V^T;
+ *   dS = P o (dP - delta);  dQ = scale dS K;  dK = scale dS^T Q        (unmasked pairs only).
+ *   o, lse    the forward results for the same q, k, v
+ *   d_o       device, gradient of the loss w.r.t. O
+ *   dq, dk, dv device, written (same shape and dtype as q)
+ *   workspace device, >= hdt_attn_workspace_bytes(..., 1), 256-byte aligned
+ * Asynchronous on `stream`.
+ */
+int hdt_attn_bwd(const hdt_index_t *index, const void *q, const void *k, const void *v,
+                 const void *o, const float *lse, const void *d_o, void *dq, void *dk, void *dv,
+                 int32_t heads, int32_t head_dim, int32_t dtype, float softmax_scale,
+                 void *workspace, size_t workspace_bytes, void *stream);
+
+/* Thread-local text of the last error returned on this thread ("" if none). */
+const char *hdt_last_error(void);
+
+/* Number of kernel launches the library has issued in this process (for benchmarks). */
+int64_t hdt_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HDT_H_ */

@@ -1,0 +1,206 @@
+"""ctypes binding of libhdt.so.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import re
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIBPATH = os.path.join(_HERE, "libhdt.so")
+_HEADER = os.path.join(_HERE, "..", "include", "hdt.h")
+_lib = None
+
+HDT_F32, HDT_BF16 = 0, 1
+HDT_MAX_STAGES = 16
+_DTYPES = {torch.float32: HDT_F32, torch.bfloat16: HDT_BF16}
+
+
+class HdtError(RuntimeError):
+    def __init__(self, code, msg):
+        super().__init__(f"libhdt error {code}: {msg}")
+        self.code = code
+
+
+class _Params(C.Structure):
+    _fields_ = [("block_m", C.c_int32), ("max_stages", C.c_int32), ("reserved", C.c_int32 * 6)]
+
+
+class _StageView(C.Structure):
+    _fields_ = [("n", C.c_int32), ("n_blocks", C.c_int32)] + \
+               [(nm, C.c_void_p) for nm in ("tok", "par", "rng", "up", "scu", "blocks", "queue")]
+
+
+def lib():
+    """Load libhdt.so; raises if it has not been built (python -m paper_2407_08330_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIBPATH):
+            raise HdtError(-5, f"{_LIBPATH} is missing: build it with `python paper_2407_08330_b200/build.py` "
+                               "(there is no fallback path)")
+        L = C.CDLL(_LIBPATH)
+        L.hdt_index_workspace_bytes.restype = C.c_size_t
+        L.hdt_index_workspace_bytes.argtypes = [C.c_int32, C.c_int32, C.c_void_p]
+        L.hdt_build_index.restype = C.c_int
+        L.hdt_build_index.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
+                                      C.c_void_p, C.c_size_t, C.c_void_p, C.POINTER(C.c_void_p)]
+        L.hdt_index_info.restype = C.c_int
+        L.hdt_index_info.argtypes = [C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.hdt_index_export.restype = C.c_int
+        L.hdt_index_export.argtypes = [C.c_void_p, C.c_int32, C.POINTER(_StageView)]
+        L.hdt_index_destroy.restype = C.c_int
+        L.hdt_index_destroy.argtypes = [C.c_void_p]
+        L.hdt_attn_workspace_bytes.restype = C.c_size_t
+        L.hdt_attn_workspace_bytes.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]
+        L.hdt_attn_fwd.restype = C.c_int
+        L.hdt_attn_fwd.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_int32, C.c_int32, C.c_float,
+                                                      C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hdt_attn_bwd.restype = C.c_int
+        L.hdt_attn_bwd.argtypes = [C.c_void_p] * 10 + [C.c_int32, C.c_int32, C.c_int32, C.c_float,
+                                                       C.c_void_p, C.c_size_t, C.c_void_p]
+        L.hdt_last_error.restype = C.c_char_p
+        L.hdt_launch_count.restype = C.c_int64
+        _lib = L
+    return _lib
+
+
+def declared_symbols():
+    """Names of every function include/hdt.h declares."""
+    txt = open(_HEADER).read()
+    txt = re.sub(r"/\*.*?\*/", "", txt, flags=re.S)
+    return sorted(set(re.findall(r"\b(hdt_[a-z0-9_]+)\s*\(", txt)))
+
+
+def exported_symbols():
+    """(declared, missing): declared functions and those libhdt.so does not export."""
+    L = lib()
+    names = declared_symbols()
+    return names, [n for n in names if not hasattr(L, n)]
+
+
+def _check(rc):
+    if rc != 0:
+        raise HdtError(rc, lib().hdt_last_error().decode())
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else C.c_void_p(0)
+
+
+def _stream():
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _params(block_m, max_stages):
+    p = _Params()
+    p.block_m, p.max_stages = int(block_m), int(max_stages)
+    return p
+
+
+def hdt_index_workspace_bytes(batch, total_tokens, block_m=0, max_stages=0) -> int:
+    p = _params(block_m, max_stages)
+    return int(lib().hdt_index_workspace_bytes(batch, total_tokens, C.cast(C.byref(p), C.c_void_p)))
+
+
+class HdtIndex:
+    """Owner of a built index: the opaque handle plus the device workspace it points into."""
+
+    def __init__(self, handle, workspace, batch, total_tokens):
+        self._h, self._ws = handle, workspace
+        self.batch, self.total_tokens = batch, total_tokens
+        ns, nnz, vis = C.c_int32(), C.c_int64(), C.c_int64()
+        _check(lib().hdt_index_info(self._h, C.byref(ns), C.byref(nnz), C.byref(vis)))
+        self.n_stages, self.nnz, self.visited = ns.value, nnz.value, vis.value
+
+    @property
+    def handle(self):
+        return self._h
+
+    def export(self, stage):
+        """Device arrays of one stage copied to host numpy arrays (parity tests, inspection)."""
+        import numpy as np
+        v = _StageView()
+        _check(lib().hdt_index_export(self._h, stage, C.byref(v)))
+        base = self._ws.data_ptr()
+
+        def arr(ptr, count):
+            off = (ptr - base) // 4
+            return self._ws.view(torch.int32)[off:off + count].cpu().numpy().copy()
+        B = self.batch
+        return dict(n=v.n, n_blocks=v.n_blocks, tok=arr(v.tok, v.n), par=arr(v.par, v.n),
+                    rng=arr(v.rng, 2 * v.n).reshape(-1, 2), up=arr(v.up, v.n), scu=arr(v.scu, B + 1),
+                    blocks=arr(v.blocks, 5 * v.n_blocks).reshape(-1, 5), queue=arr(v.queue, v.n_blocks))
+
+    def close(self):
+        if self._h is not None:
+            lib().hdt_index_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def hdt_build_index(level, parent, cu_seqlens, block_m=0, max_stages=0, workspace=None) -> HdtIndex:
+    """level int8[T], parent int32[T], cu_seqlens int32[B+1]: CUDA tensors."""
+    assert level.is_cuda and parent.is_cuda and cu_seqlens.is_cuda
+    assert level.dtype == torch.int8 and parent.dtype == torch.int32 and cu_seqlens.dtype == torch.int32
+    level, parent, cu_seqlens = level.contiguous(), parent.contiguous(), cu_seqlens.contiguous()
+    T, B = level.numel(), cu_seqlens.numel() - 1
+    p = _params(block_m, max_stages)
+    need = int(lib().hdt_index_workspace_bytes(B, T, C.cast(C.byref(p), C.c_void_p)))
+    if need == 0:
+        raise HdtError(-1, "invalid index parameters")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=level.device)
+    h = C.c_void_p()
+    _check(lib().hdt_build_index(_ptr(level), _ptr(parent), _ptr(cu_seqlens), B, T, C.cast(C.byref(p), C.c_void_p),
+                                 _ptr(workspace), workspace.numel(), _stream(), C.byref(h)))
+    return HdtIndex(h, workspace, B, T)
+
+
+def hdt_attn_workspace_bytes(index: HdtIndex, heads, head_dim, dtype, bwd) -> int:
+    return int(lib().hdt_attn_workspace_bytes(index.handle, heads, head_dim, _DTYPES[dtype], int(bwd)))
+
+
+def _ws(index, heads, head_dim, dtype, bwd, device, workspace):
+    need = hdt_attn_workspace_bytes(index, heads, head_dim, dtype, bwd)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
+    return workspace, need
+
+
+def hdt_attn_fwd(index: HdtIndex, q, k, v, softmax_scale=0.0, out=None, lse=None, workspace=None):
+    """q, k, v: CUDA [T, H, d] float32 or bfloat16, contiguous.  Returns (O, LSE [H, T])."""
+    T, H, d = q.shape
+    assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and q.dtype == k.dtype == v.dtype
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((H, T), dtype=torch.float32, device=q.device) if lse is None else lse
+    workspace, need = _ws(index, H, d, q.dtype, 0, q.device, workspace)
+    _check(lib().hdt_attn_fwd(index.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), H, d,
+                              _DTYPES[q.dtype], float(softmax_scale), _ptr(workspace), workspace.numel(),
+                              _stream()))
+    return o, lse
+
+
+def hdt_attn_bwd(index: HdtIndex, q, k, v, o, lse, d_o, softmax_scale=0.0, dq=None, dk=None, dv=None,
+                 workspace=None):
+    """Returns (dQ, dK, dV) with the shape and dtype of q."""
+    T, H, d = q.shape
+    for t in (q, k, v, o, d_o):
+        assert t.is_contiguous() and t.dtype == q.dtype
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(q) if dk is None else dk
+    dv = torch.empty_like(q) if dv is None else dv
+    workspace, need = _ws(index, H, d, q.dtype, 1, q.device, workspace)
+    _check(lib().hdt_attn_bwd(index.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(d_o),
+                              _ptr(dq), _ptr(dk), _ptr(dv), H, d, _DTYPES[q.dtype], float(softmax_scale),
+                              _ptr(workspace), workspace.numel(), _stream()))
+    return dq, dk, dv
+
+
+def hdt_launch_count() -> int:
+    return int(lib().hdt_launch_count())

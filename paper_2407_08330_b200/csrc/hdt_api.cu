@@ -1,0 +1,150 @@
+// C-ABI entry points of the attention passes, error text, launch counter.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+
+#include "hdt_internal.cuh"
+
+namespace hdt {
+
+static thread_local char g_err[512] = "";
+std::atomic<long long> g_launches{0};
+
+int set_error(int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+static size_t al256(size_t x) { return (x + 255) & ~size_t(255); }
+
+struct AttnLayout {
+    size_t delta;                       // bwd only
+    size_t part[HDT_MAX_STAGES][4];     // fwd: o, lse;  bwd: dq, dk, dv
+    size_t total;
+};
+
+static AttnLayout attn_layout(const hdt_index *ix, int H, int D, int bwd) {
+    AttnLayout L{};
+    size_t o = 0;
+    if (bwd) { L.delta = o; o += al256(sizeof(float) * (size_t)H * ix->total_tokens); }
+    for (int s = 1; s < ix->n_stages; ++s) {
+        const size_t n = (size_t)ix->desc[s].n;
+        const int cnt = bwd ? 3 : 1;
+        for (int c = 0; c < cnt; ++c) { L.part[s][c] = o; o += al256(sizeof(float) * n * H * D); }
+        if (!bwd) { L.part[s][1] = o; o += al256(sizeof(float) * n * H); }
+    }
+    L.total = o;
+    return L;
+}
+
+static int check_common(const hdt_index *ix, int H, int D, int dtype, const void *ws, size_t ws_bytes,
+                        size_t need, const char *fn) {
+    if (!ix) return set_error(HDT_ERR_INVALID_ARG, "%s: null index", fn);
+    if (H <= 0) return set_error(HDT_ERR_INVALID_ARG, "%s: heads must be positive", fn);
+    if (D != 64 && D != 128) return set_error(HDT_ERR_UNSUPPORTED, "%s: head_dim %d not supported (64 or 128)", fn, D);
+    if (dtype != HDT_F32 && dtype != HDT_BF16) return set_error(HDT_ERR_UNSUPPORTED, "%s: unknown dtype %d", fn, dtype);
+    if (need > 0 && (!ws || ws_bytes < need))
+        return set_error(HDT_ERR_WORKSPACE, "%s: workspace %zu < required %zu", fn, ws_bytes, need);
+    if (need > 0 && ((uintptr_t)ws & 255) != 0)
+        return set_error(HDT_ERR_INVALID_ARG, "%s: workspace must be 256-byte aligned", fn);
+    return HDT_OK;
+}
+
+static bool misaligned(const void *p) { return ((uintptr_t)p & 15) != 0; }
+
+}  // namespace hdt
+
+using namespace hdt;
+
+extern "C" const char *hdt_last_error(void) { return g_err; }
+extern "C" int64_t hdt_launch_count(void) { return (int64_t)g_launches.load(); }
+
+extern "C" size_t hdt_attn_workspace_bytes(const hdt_index_t *ix, int32_t heads, int32_t head_dim,
+                                           int32_t dtype, int32_t bwd) {
+    (void)dtype;
+    if (!ix || heads <= 0 || head_dim <= 0) return 0;
+    return attn_layout(ix, heads, head_dim, bwd).total;
+}
+
+extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k, const void *v, void *o,
+                            float *lse, int32_t heads, int32_t head_dim, int32_t dtype, float softmax_scale,
+                            void *workspace, size_t workspace_bytes, void *stream) {
+    if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: null index");
+    const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 0);
+    int rc = check_common(ix, heads, head_dim, dtype, workspace, workspace_bytes, L.total, "hdt_attn_fwd");
+    if (rc) return rc;
+    if (ix->total_tokens == 0) return HDT_OK;
+    if (!q || !k || !v || !o || !lse) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: null tensor pointer");
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(o))
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: tensors must be 16-byte aligned");
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = (char *)workspace;
+    for (int s = ix->n_stages - 1; s >= 0; --s) {
+        const StagePtrs &P = ix->st[s];
+        FwdStageArgs a{};
+        a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
+        a.tok = s ? P.tok : nullptr;
+        a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
+        a.q = q; a.k = k; a.v = v;
+        a.scale_log2 = scale * 1.4426950408889634f;
+        if (s + 1 < ix->n_stages) {
+            a.carry_o = (const float *)(ws + L.part[s + 1][0]);
+            a.carry_lse = (const float *)(ws + L.part[s + 1][1]);
+        }
+        if (s == 0) { a.o = o; a.lse = lse; }
+        else { a.part_o = (float *)(ws + L.part[s][0]); a.part_lse = (float *)(ws + L.part[s][1]); }
+        rc = launch_fwd_simt(a, head_dim, dtype, st);
+        if (rc) return rc;
+    }
+    return HDT_OK;
+}
+
+extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k, const void *v, const void *o,
+                            const float *lse, const void *d_o, void *dq, void *dk, void *dv, int32_t heads,
+                            int32_t head_dim, int32_t dtype, float softmax_scale, void *workspace,
+                            size_t workspace_bytes, void *stream) {
+    if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_bwd: null index");
+    const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 1);
+    int rc = check_common(ix, heads, head_dim, dtype, workspace, workspace_bytes, L.total, "hdt_attn_bwd");
+    if (rc) return rc;
+    if (ix->total_tokens == 0) return HDT_OK;
+    if (!q || !k || !v || !o || !lse || !d_o || !dq || !dk || !dv)
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_bwd: null tensor pointer");
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(o) || misaligned(d_o) || misaligned(dq) ||
+        misaligned(dk) || misaligned(dv))
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_bwd: tensors must be 16-byte aligned");
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = (char *)workspace;
+    float *delta = (float *)(ws + L.delta);
+    rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
+    if (rc) return rc;
+    for (int s = ix->n_stages - 1; s >= 0; --s) {
+        const StagePtrs &P = ix->st[s];
+        BwdStageArgs a{};
+        a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
+        a.tok = s ? P.tok : nullptr;
+        a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
+        a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = delta;
+        a.scale = scale;
+        a.scale_log2 = scale * 1.4426950408889634f;
+        if (s + 1 < ix->n_stages) {
+            a.carry_dq = (const float *)(ws + L.part[s + 1][0]);
+            a.carry_dk = (const float *)(ws + L.part[s + 1][1]);
+            a.carry_dv = (const float *)(ws + L.part[s + 1][2]);
+        }
+        if (s == 0) { a.dq = dq; a.dk = dk; a.dv = dv; }
+        else {
+            a.part_dq = (float *)(ws + L.part[s][0]);
+            a.part_dk = (float *)(ws + L.part[s][1]);
+            a.part_dv = (float *)(ws + L.part[s][2]);
+        }
+        rc = launch_bwd_simt(a, head_dim, dtype, st);
+        if (rc) return rc;
+    }
+    return HDT_OK;
+}

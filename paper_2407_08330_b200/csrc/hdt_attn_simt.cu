@@ -1,0 +1,427 @@
+// FP32 SIMT attention kernels over the staged family index.
+//
+// These are the exact-arithmetic path: fp32 inputs (where tensor cores have no fp32-input
+// mode accurate to 1e-4) and the small compacted stages above stage 0 (a few percent of the
+// tokens).  One CTA handles one (row block, head); a row is owned by G = D/16 adjacent lanes,
+// each holding 16 of the D dimensions; keys/values of the block's span are staged through
+// shared memory in chunks and every row walks only its own key range [lo, hi).
+#include <cuda_bf16.h>
+
+#include "hdt_internal.cuh"
+
+namespace hdt {
+
+static constexpr int KC = 32;        // keys per shared-memory chunk
+static constexpr int NTHREADS = 512;
+
+template <bool BF16>
+__device__ __forceinline__ float4 load4(const void *base, size_t elem) {
+    if constexpr (BF16) {
+        const uint2 u = *reinterpret_cast<const uint2 *>(reinterpret_cast<const __nv_bfloat16 *>(base) + elem);
+        float4 r;
+        r.x = __uint_as_float(u.x << 16);
+        r.y = __uint_as_float(u.x & 0xffff0000u);
+        r.z = __uint_as_float(u.y << 16);
+        r.w = __uint_as_float(u.y & 0xffff0000u);
+        return r;
+    } else {
+        return *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(base) + elem);
+    }
+}
+
+template <bool BF16>
+__device__ __forceinline__ void store4(void *base, size_t elem, float4 v) {
+    if constexpr (BF16) {
+        __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+        uint2 u;
+        u.x = *reinterpret_cast<uint32_t *>(&a);
+        u.y = *reinterpret_cast<uint32_t *>(&b);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(base) + elem) = u;
+    } else {
+        *reinterpret_cast<float4 *>(reinterpret_cast<float *>(base) + elem) = v;
+    }
+}
+
+__device__ __forceinline__ float dot4(float4 a, float4 b, float acc) {
+    acc = fmaf(a.x, b.x, acc);
+    acc = fmaf(a.y, b.y, acc);
+    acc = fmaf(a.z, b.z, acc);
+    acc = fmaf(a.w, b.w, acc);
+    return acc;
+}
+__device__ __forceinline__ void axpy4(float4 &y, float a, float4 x) {
+    y.x = fmaf(a, x.x, y.x);
+    y.y = fmaf(a, x.y, y.y);
+    y.z = fmaf(a, x.z, y.z);
+    y.w = fmaf(a, x.w, y.w);
+}
+__device__ __forceinline__ void scale4(float4 &y, float a) { y.x *= a; y.y *= a; y.z *= a; y.w *= a; }
+
+template <int G>
+__device__ __forceinline__ float group_sum(float x) {
+    x += __shfl_xor_sync(0xffffffffu, x, 1);
+    x += __shfl_xor_sync(0xffffffffu, x, 2);
+    if constexpr (G == 8) x += __shfl_xor_sync(0xffffffffu, x, 4);
+    return x;
+}
+
+// Stage `rows` [c0, c0+KC) of a [*, H, D] tensor (through tok) into smem as fp32, zero past `end`.
+template <int D, bool BF16>
+__device__ __forceinline__ void stage_rows(float4 *dst, const void *src, const int *tok, int c0, int end,
+                                           int H, int h) {
+    constexpr int U = D / 4;
+    for (int idx = threadIdx.x; idx < KC * U; idx += NTHREADS) {
+        const int r = idx / U, u = idx % U;
+        const int e = c0 + r;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (e < end) {
+            const int t = tok ? tok[e] : e;
+            v = load4<BF16>(src, ((size_t)t * H + h) * D + 4 * u);
+        }
+        dst[idx] = v;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// forward
+// ---------------------------------------------------------------------------------------------
+template <int D, bool BF16>
+__global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
+    constexpr int G = D / 16, U = D / 4, RP = NTHREADS / G;
+    __shared__ float4 sK[KC * U];
+    __shared__ float4 sV[KC * U];
+    const int blk = a.queue[blockIdx.x], h = blockIdx.y, H = a.H;
+    const int *rec = a.blocks + 5 * (size_t)blk;
+    const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3];
+    const int g = threadIdx.x % G, rl = threadIdx.x / G;
+    const float NEG = -INFINITY;
+
+    for (int p0 = r0; p0 < r1; p0 += RP) {
+        const int row = p0 + rl;
+        const bool inb = row < r1;
+        int lo = 0, hi = 0, trow = 0;
+        float4 q[4], o[4];
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { q[t] = make_float4(0, 0, 0, 0); o[t] = make_float4(0, 0, 0, 0); }
+        if (inb) {
+            lo = a.rng[2 * row];
+            hi = a.rng[2 * row + 1];
+            trow = a.tok ? a.tok[row] : row;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) q[t] = load4<BF16>(a.q, ((size_t)trow * H + h) * D + 4 * (g + G * t));
+        }
+        float m = NEG, l = 0.f;
+        for (int c0 = ka; c0 < kb; c0 += KC) {
+            __syncthreads();
+            stage_rows<D, BF16>(sK, a.k, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16>(sV, a.v, a.tok, c0, kb, H, h);
+            __syncthreads();
+            const int jlo = max(lo, c0), jhi = min(hi, c0 + KC);
+            const bool has = jhi > jlo;
+            const int wlo = __reduce_min_sync(0xffffffffu, has ? jlo : 0x7fffffff);
+            const int whi = __reduce_max_sync(0xffffffffu, has ? jhi : (int)0x80000000);
+            for (int j0 = wlo; j0 < whi; j0 += 8) {
+                float s[8];
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj) {
+                    const int j = j0 + jj;
+                    s[jj] = NEG;
+                    if (j < whi) {
+                        const float4 *kr = sK + (j - c0) * U;
+                        float acc = 0.f;
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) acc = dot4(q[t], kr[g + G * t], acc);
+                        acc = group_sum<G>(acc);
+                        if (j >= jlo && j < jhi) s[jj] = acc * a.scale_log2;
+                    }
+                }
+                float mx = s[0];
+#pragma unroll
+                for (int jj = 1; jj < 8; ++jj) mx = fmaxf(mx, s[jj]);
+                const float mn = fmaxf(m, mx);
+                if (mn > NEG) {
+                    const float alpha = exp2f(m - mn);
+                    l *= alpha;
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) scale4(o[t], alpha);
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) {
+                        const int j = j0 + jj;
+                        if (j < whi) {
+                            const float p = exp2f(s[jj] - mn);
+                            l += p;
+                            const float4 *vr = sV + (j - c0) * U;
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) axpy4(o[t], p, vr[g + G * t]);
+                        }
+                    }
+                    m = mn;
+                }
+            }
+        }
+        if (!inb) continue;
+        // own partial result, natural-log LSE
+        float lse = NEG;
+        if (l > 0.f) {
+            const float inv = 1.f / l;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) scale4(o[t], inv);
+            lse = (m + log2f(l)) * 0.6931471805599453f;
+        }
+        // merge the partial result of the later stages
+        if (a.carry_o != nullptr) {
+            const int u = a.up[row];
+            if (u >= 0) {
+                const float lc = a.carry_lse[(size_t)u * H + h];
+                if (lc > NEG) {
+                    const float mx = fmaxf(lse, lc);
+                    const float e0 = (lse > NEG) ? __expf(lse - mx) : 0.f, e1 = __expf(lc - mx);
+                    const float tot = e0 + e1;
+                    const float w0 = e0 / tot, w1 = e1 / tot;
+                    const float4 *oc = reinterpret_cast<const float4 *>(a.carry_o + ((size_t)u * H + h) * D);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        scale4(o[t], w0);
+                        axpy4(o[t], w1, oc[g + G * t]);
+                    }
+                    lse = mx + __logf(tot);
+                }
+            }
+        }
+        if (a.part_o != nullptr) {
+            float4 *po = reinterpret_cast<float4 *>(a.part_o + ((size_t)row * H + h) * D);
+#pragma unroll
+            for (int t = 0; t < 4; ++t) po[g + G * t] = o[t];
+            if (g == 0) a.part_lse[(size_t)row * H + h] = lse;
+        } else {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) store4<BF16>(a.o, ((size_t)trow * H + h) * D + 4 * (g + G * t), o[t]);
+            if (g == 0) a.lse[(size_t)h * a.T + trow] = lse;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// backward: phase A rows -> dQ, phase B keys -> dK, dV (the family ranges are symmetric, so the
+// same blocks serve as key blocks)
+// ---------------------------------------------------------------------------------------------
+template <int D, bool BF16>
+__global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
+    constexpr int G = D / 16, U = D / 4, RP = NTHREADS / G;
+    __shared__ float4 sA[KC * U];  // K (phase A) / Q (phase B)
+    __shared__ float4 sB[KC * U];  // V (phase A) / dO (phase B)
+    __shared__ float sL[KC], sDl[KC];
+    const int blk = a.queue[blockIdx.x], h = blockIdx.y, H = a.H;
+    const int *rec = a.blocks + 5 * (size_t)blk;
+    const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3];
+    const int g = threadIdx.x % G, rl = threadIdx.x / G;
+    const float LOG2E = 1.4426950408889634f;
+
+    for (int p0 = r0; p0 < r1; p0 += RP) {
+        const int row = p0 + rl;
+        const bool inb = row < r1;
+        int lo = 0, hi = 0, trow = 0;
+        if (inb) {
+            lo = a.rng[2 * row];
+            hi = a.rng[2 * row + 1];
+            trow = a.tok ? a.tok[row] : row;
+        }
+        const bool live = hi > lo;
+        // ---------------- phase A: this element as a query row ----------------
+        float4 x[4], y[4], acc[4];  // q, dO, dq
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            x[t] = y[t] = acc[t] = make_float4(0, 0, 0, 0);
+            if (live) {
+                x[t] = load4<BF16>(a.q, ((size_t)trow * H + h) * D + 4 * (g + G * t));
+                y[t] = load4<BF16>(a.d_o, ((size_t)trow * H + h) * D + 4 * (g + G * t));
+            }
+        }
+        float lse2 = 0.f, dl = 0.f;
+        if (live) {
+            lse2 = a.lse[(size_t)h * a.T + trow] * LOG2E;
+            dl = a.delta[(size_t)h * a.T + trow];
+        }
+        for (int c0 = ka; c0 < kb; c0 += KC) {
+            __syncthreads();
+            stage_rows<D, BF16>(sA, a.k, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16>(sB, a.v, a.tok, c0, kb, H, h);
+            __syncthreads();
+            const int jlo = max(lo, c0), jhi = min(hi, c0 + KC);
+            const bool has = jhi > jlo;
+            const int wlo = __reduce_min_sync(0xffffffffu, has ? jlo : 0x7fffffff);
+            const int whi = __reduce_max_sync(0xffffffffu, has ? jhi : (int)0x80000000);
+            for (int j = wlo; j < whi; ++j) {
+                const float4 *kr = sA + (j - c0) * U, *vr = sB + (j - c0) * U;
+                float s = 0.f, dp = 0.f;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    s = dot4(x[t], kr[g + G * t], s);
+                    dp = dot4(y[t], vr[g + G * t], dp);
+                }
+                s = group_sum<G>(s);
+                dp = group_sum<G>(dp);
+                if (j >= jlo && j < jhi) {
+                    const float p = exp2f(s * a.scale_log2 - lse2);
+                    const float ds = p * (dp - dl);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) axpy4(acc[t], ds, kr[g + G * t]);
+                }
+            }
+        }
+        if (inb) {
+            const int u = (a.carry_dq != nullptr) ? a.up[row] : -1;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                scale4(acc[t], a.scale);
+                if (u >= 0) {
+                    const float4 c = reinterpret_cast<const float4 *>(a.carry_dq + ((size_t)u * H + h) * D)[g + G * t];
+                    acc[t].x += c.x; acc[t].y += c.y; acc[t].z += c.z; acc[t].w += c.w;
+                }
+                if (a.part_dq != nullptr)
+                    reinterpret_cast<float4 *>(a.part_dq + ((size_t)row * H + h) * D)[g + G * t] = acc[t];
+                else
+                    store4<BF16>(a.dq, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc[t]);
+            }
+        }
+        // ---------------- phase B: this element as a key ----------------
+        float4 acc2[4];  // x = k, y = v, acc = dk, acc2 = dv
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            x[t] = y[t] = acc[t] = acc2[t] = make_float4(0, 0, 0, 0);
+            if (live) {
+                x[t] = load4<BF16>(a.k, ((size_t)trow * H + h) * D + 4 * (g + G * t));
+                y[t] = load4<BF16>(a.v, ((size_t)trow * H + h) * D + 4 * (g + G * t));
+            }
+        }
+        for (int c0 = ka; c0 < kb; c0 += KC) {
+            __syncthreads();
+            stage_rows<D, BF16>(sA, a.q, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16>(sB, a.d_o, a.tok, c0, kb, H, h);
+            if (threadIdx.x < KC) {
+                const int e = c0 + threadIdx.x;
+                float L = 0.f, dlt = 0.f;
+                if (e < kb) {
+                    const int t = a.tok ? a.tok[e] : e;
+                    L = a.lse[(size_t)h * a.T + t] * LOG2E;
+                    dlt = a.delta[(size_t)h * a.T + t];
+                }
+                sL[threadIdx.x] = L;
+                sDl[threadIdx.x] = dlt;
+            }
+            __syncthreads();
+            const int jlo = max(lo, c0), jhi = min(hi, c0 + KC);
+            const bool has = jhi > jlo;
+            const int wlo = __reduce_min_sync(0xffffffffu, has ? jlo : 0x7fffffff);
+            const int whi = __reduce_max_sync(0xffffffffu, has ? jhi : (int)0x80000000);
+            for (int i = wlo; i < whi; ++i) {
+                const float4 *qr = sA + (i - c0) * U, *dor = sB + (i - c0) * U;
+                float s = 0.f, dp = 0.f;
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    s = dot4(x[t], qr[g + G * t], s);
+                    dp = dot4(y[t], dor[g + G * t], dp);
+                }
+                s = group_sum<G>(s);
+                dp = group_sum<G>(dp);
+                if (i >= jlo && i < jhi) {
+                    const float p = exp2f(s * a.scale_log2 - sL[i - c0]);
+                    const float ds = p * (dp - sDl[i - c0]);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        axpy4(acc[t], ds, qr[g + G * t]);
+                        axpy4(acc2[t], p, dor[g + G * t]);
+                    }
+                }
+            }
+        }
+        if (inb) {
+            const int u = (a.carry_dk != nullptr) ? a.up[row] : -1;
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                scale4(acc[t], a.scale);
+                if (u >= 0) {
+                    const float4 c = reinterpret_cast<const float4 *>(a.carry_dk + ((size_t)u * H + h) * D)[g + G * t];
+                    const float4 c2 = reinterpret_cast<const float4 *>(a.carry_dv + ((size_t)u * H + h) * D)[g + G * t];
+                    acc[t].x += c.x; acc[t].y += c.y; acc[t].z += c.z; acc[t].w += c.w;
+                    acc2[t].x += c2.x; acc2[t].y += c2.y; acc2[t].z += c2.z; acc2[t].w += c2.w;
+                }
+                if (a.part_dk != nullptr) {
+                    reinterpret_cast<float4 *>(a.part_dk + ((size_t)row * H + h) * D)[g + G * t] = acc[t];
+                    reinterpret_cast<float4 *>(a.part_dv + ((size_t)row * H + h) * D)[g + G * t] = acc2[t];
+                } else {
+                    store4<BF16>(a.dk, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc[t]);
+                    store4<BF16>(a.dv, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc2[t]);
+                }
+            }
+        }
+    }
+}
+
+// delta[h, t] = sum_c dO[t,h,c] * O[t,h,c]; one warp per (t, h).
+template <int D, bool BF16>
+__global__ void k_delta(const void *o, const void *d_o, float *delta, int T, int H) {
+    const int lane = threadIdx.x & 31;
+    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (w >= (long long)T * H) return;
+    const int t = (int)(w / H), h = (int)(w % H);
+    float acc = 0.f;
+    if (lane < D / 4) {
+        const float4 x = load4<BF16>(o, (size_t)w * D + 4 * lane);
+        const float4 y = load4<BF16>(d_o, (size_t)w * D + 4 * lane);
+        acc = dot4(x, y, 0.f);
+    }
+    for (int s = 16; s; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+    if (lane == 0) delta[(size_t)h * T + t] = acc;
+}
+
+template <int D, bool BF16>
+static int launch_fwd_t(const FwdStageArgs &a, cudaStream_t st) {
+    if (a.nb == 0) return HDT_OK;
+    dim3 grid(a.nb, a.H);
+    k_fwd_simt<D, BF16><<<grid, NTHREADS, 0, st>>>(a);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+template <int D, bool BF16>
+static int launch_bwd_t(const BwdStageArgs &a, cudaStream_t st) {
+    if (a.nb == 0) return HDT_OK;
+    dim3 grid(a.nb, a.H);
+    k_bwd_simt<D, BF16><<<grid, NTHREADS, 0, st>>>(a);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+
+int launch_fwd_simt(const FwdStageArgs &a, int D, int dtype, cudaStream_t st) {
+    if (D == 64) return dtype == HDT_BF16 ? launch_fwd_t<64, true>(a, st) : launch_fwd_t<64, false>(a, st);
+    if (D == 128) return dtype == HDT_BF16 ? launch_fwd_t<128, true>(a, st) : launch_fwd_t<128, false>(a, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
+}
+int launch_bwd_simt(const BwdStageArgs &a, int D, int dtype, cudaStream_t st) {
+    if (D == 64) return dtype == HDT_BF16 ? launch_bwd_t<64, true>(a, st) : launch_bwd_t<64, false>(a, st);
+    if (D == 128) return dtype == HDT_BF16 ? launch_bwd_t<128, true>(a, st) : launch_bwd_t<128, false>(a, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
+}
+
+int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int D, int dtype, cudaStream_t st) {
+    const long long rows = (long long)T * H;
+    if (rows == 0) return HDT_OK;
+    const int threads = 256;
+    const long long blocks = (rows * 32 + threads - 1) / threads;
+    if (D == 64) {
+        if (dtype == HDT_BF16) k_delta<64, true><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
+        else k_delta<64, false><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
+    } else if (D == 128) {
+        if (dtype == HDT_BF16) k_delta<128, true><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
+        else k_delta<128, false><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
+    } else {
+        return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
+    }
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+
+}  // namespace hdt

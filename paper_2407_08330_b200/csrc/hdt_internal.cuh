@@ -1,0 +1,92 @@
+// Internal declarations shared by the translation units of libhdt.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <atomic>
+
+#include "../../include/hdt.h"
+
+namespace hdt {
+
+// Device-resident header of an index (first bytes of the index workspace).
+struct StageDesc {
+    int n;         // elements of the stage array
+    int nb;        // row blocks
+    int has_next;  // a later stage exists
+    int pad;
+};
+
+struct DevHeader {
+    int status;              // hdt_status_t, first error wins
+    int err_pos;             // element / sequence where it was detected
+    long long nnz;           // unmasked pairs
+    long long visited;       // sum over blocks of rows x span
+    StageDesc st[HDT_MAX_STAGES + 1];
+};
+
+// Host-side pointers to one stage's arrays inside the workspace.
+struct StagePtrs {
+    int *tok, *par, *rng, *up, *scu, *blocks, *queue;
+};
+
+}  // namespace hdt
+
+struct hdt_index {
+    int batch, total_tokens, block_m, n_stages;
+    long long nnz, visited;
+    hdt::StageDesc desc[HDT_MAX_STAGES + 1];
+    hdt::StagePtrs st[HDT_MAX_STAGES];
+    void *workspace;
+    size_t workspace_bytes;
+};
+
+namespace hdt {
+
+int set_error(int code, const char *fmt, ...);
+extern std::atomic<long long> g_launches;
+inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+#define HDT_CUDA_CHECK(expr)                                                                  \
+    do {                                                                                      \
+        cudaError_t e_ = (expr);                                                              \
+        if (e_ != cudaSuccess)                                                                \
+            return hdt::set_error(HDT_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
+    } while (0)
+
+// SIMT attention launchers (hdt_attn_simt.cu).  One launch handles one stage.
+struct FwdStageArgs {
+    // stage view
+    int n, nb, H;
+    const int *tok;     // nullptr: identity (stage 0)
+    const int *rng, *up, *blocks, *queue;
+    const void *q, *k, *v;
+    float scale_log2;   // softmax_scale * log2(e)
+    // partial results of the next stage (nullptr if none): [n_up, H, D] and [n_up, H]
+    const float *carry_o, *carry_lse;
+    // outputs: final (stage 0) ...
+    void *o;            // dtype [T,H,D]
+    float *lse;         // [H,T]
+    int T;
+    // ... or this stage's partial results
+    float *part_o, *part_lse;
+};
+
+struct BwdStageArgs {
+    int n, nb, H, T;
+    const int *tok;
+    const int *rng, *up, *blocks, *queue;
+    const void *q, *k, *v, *d_o;
+    const float *lse;    // [H,T] final
+    const float *delta;  // [H,T]
+    float scale, scale_log2;
+    const float *carry_dq, *carry_dk, *carry_dv;  // [n_up,H,D] from the next stage, or nullptr
+    void *dq, *dk, *dv;                           // final dtype [T,H,D] (stage 0)
+    float *part_dq, *part_dk, *part_dv;           // [n,H,D] (stages above 0)
+};
+
+int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
+int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
+int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
+                 cudaStream_t st);
+
+}  // namespace hdt

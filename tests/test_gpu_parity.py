@@ -1,0 +1,226 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Index metadata bit-exact; fp32 attention <= 1e-4; bf16 attention max <= 2e-2 and
+mean <= 2e-3 (absolute errors on stored outputs against the fp64 oracle on bf16-rounded inputs)."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+from oracle import index_oracle as ix
+from gpu_util import check_close, dev_struct, dev_tensor, host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def P():
+    import paper_2407_08330_b200 as P
+    return P
+
+
+def assert_index_equal(P, b, block_m=128, max_stages=8):
+    want = ix.build(b.level, b.parent, b.cu_seqlens, block_m)
+    idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=max_stages)
+    assert idx.n_stages == len(want.stages)
+    assert idx.nnz == want.nnz and idx.visited == want.visited
+    for s, st in enumerate(want.stages):
+        got = idx.export(s)
+        assert got["n"] == st.n and got["n_blocks"] == len(st.blocks), s
+        for name in ("tok", "par", "rng", "up", "scu", "blocks", "queue"):
+            assert np.array_equal(got[name], getattr(st, name)), (s, name)
+    return idx
+
+
+# ------------------------------------------------------------------------------------------
+# index
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("block_m", [128, 16, 5])
+def test_index_small_documents(P, block_m):
+    for seed in range(10):
+        b = gen.small_random_batch(seed, n_seqs=4, max_len=400)
+        assert_index_equal(P, b, block_m)
+
+
+def test_index_generic_trees_and_degenerate(P):
+    rng = np.random.default_rng(2)
+    seqs = [gen.layout_tree(gen.random_tree(rng, int(rng.integers(1, 7)), 5)) for _ in range(30)]
+    seqs.append((np.array([0], np.int8), np.array([-1], np.int32)))
+    seqs.append((np.array([0, -1, -1], np.int8), np.array([-1, -1, -1], np.int32)))
+    seqs.append((np.array([-1, -1], np.int8), np.array([-1, -1], np.int32)))
+    seqs.append((np.zeros(0, np.int8), np.zeros(0, np.int32)))
+    seqs.append(gen.layout([[300, 2], [1]]))
+    b = gen.pack(seqs)
+    for bm in (128, 7):
+        assert_index_equal(P, b, bm, max_stages=8)
+    # empty batch and batch of one empty sequence
+    assert_index_equal(P, gen.pack([]))
+    assert_index_equal(P, gen.pack([(np.zeros(0, np.int8), np.zeros(0, np.int32))]))
+
+
+@pytest.mark.parametrize("c", [1, 2, 3, 4, 5])
+def test_index_configs(P, c):
+    b = gen.make_hierarchy(c)
+    idx = assert_index_equal(P, b, 128, max_stages=4)
+    assert idx.n_stages == 3
+
+
+def test_index_rejects_bad_hierarchies(P):
+    lv, pa = gen.layout([[2, 1], [1]])
+    cu = np.array([0, 10], np.int32)
+
+    def build(lv, pa, cu, **kw):
+        return P.hdt_build_index(torch.from_numpy(np.asarray(lv, np.int8)).cuda(),
+                                 torch.from_numpy(np.asarray(pa, np.int32)).cuda(),
+                                 torch.from_numpy(np.asarray(cu, np.int32)).cuda(), **kw)
+    cases = []
+    bad = pa.copy(); bad[3] = 5; cases.append((lv, bad, cu))            # parent after the token
+    bad = pa.copy(); bad[6] = 2; cases.append((lv, bad, cu))            # not in document order
+    badl = lv.copy(); badl[3] = 2; cases.append((badl, pa, cu))         # level jump
+    badl = lv.copy(); badl[0] = 1; cases.append((badl, pa, cu))         # no root
+    lvp = lv.copy(); lvp[4] = -1; pap = pa.copy(); pap[4] = -1; cases.append((lvp, pap, cu))  # PAD inside
+    cases.append((lv, pa, np.array([0, 4, 3, 10], np.int32)))           # non-monotone offsets
+    cases.append((lv, pa, np.array([0, 9], np.int32)))                  # offsets do not end at T
+    for lv_, pa_, cu_ in cases:
+        with pytest.raises(P.HdtError) as e:
+            build(lv_, pa_, cu_)
+        assert e.value.code == -2
+        with pytest.raises(ix.BadHierarchy):
+            ix.build(lv_, pa_, cu_)
+    # deeper than max_stages
+    deep = gen.layout_tree([[[[[[]]]]]])
+    with pytest.raises(P.HdtError) as e:
+        build(deep[0], deep[1], np.array([0, len(deep[0])], np.int32), max_stages=2)
+    assert e.value.code == -2
+    # the context is still usable afterwards
+    assert_index_equal(P, gen.make_hierarchy(1))
+
+
+# ------------------------------------------------------------------------------------------
+# attention, small cases compared element by element
+# ------------------------------------------------------------------------------------------
+def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
+    t = gen.make_tensors(seed, b.total_tokens, H, d, dtype)
+    idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=8)
+    q, k, v, do = (dev_tensor(t[n], dtype) for n in ("q", "k", "v", "do"))
+    o, lse = P.hdt_attn_fwd(idx, q, k, v, softmax_scale=scale)
+    sc = scale if scale > 0 else None
+    o_ref, lse_ref = oracle.forward(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], scale=sc)
+    check_close(host(o), o_ref, dtype, "O")
+    check_close(host(lse), lse_ref, "f32" if dtype == "f32" else "bf16", "LSE")
+    if bwd:
+        dq, dk, dv = P.hdt_attn_bwd(idx, q, k, v, o, lse, do, softmax_scale=scale)
+        # the oracle differentiates its own forward; the GPU uses its stored (rounded) O for delta
+        dq_r, dk_r, dv_r = oracle.backward(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], t["do"], scale=sc)
+        check_close(host(dq), dq_r, dtype, "dQ")
+        check_close(host(dk), dk_r, dtype, "dK")
+        check_close(host(dv), dv_r, dtype, "dV")
+    torch.cuda.synchronize()
+
+
+def test_config1_fp32_forward(P):
+    b = gen.make_hierarchy(1)
+    run_case(P, b, 1, 64, "f32", 0, bwd=True)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("d", [64, 128])
+def test_small_documents(P, dtype, d):
+    for seed in range(3):
+        b = gen.small_random_batch(100 + seed, n_seqs=4, max_len=500, K=(0, 40))
+        run_case(P, b, 3, d, dtype, 7 + seed)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_ragged_long_families_and_padding(P, dtype):
+    # sentences longer than a row block, a 1-token document, PAD-only and empty sequences
+    seqs = [gen.layout([[300, 2], [1, 131, 0]]), gen.layout([[7] * 40]),
+            (np.array([0], np.int8), np.array([-1], np.int32)),
+            (np.array([-1, -1, -1], np.int8), np.array([-1, -1, -1], np.int32)),
+            (np.zeros(0, np.int8), np.zeros(0, np.int32)),
+            gen.fit(*gen.layout([[5, 6], [7]]), 64, pad=True)]
+    b = gen.pack(seqs)
+    run_case(P, b, 2, 64, dtype, 11)
+    run_case(P, b, 2, 128, dtype, 12, block_m=32)
+    run_case(P, b, 1, 64, dtype, 13, block_m=128, scale=0.2)
+
+
+def test_generic_depth_trees(P):
+    rng = np.random.default_rng(4)
+    seqs = [gen.layout_tree(gen.random_tree(rng, int(rng.integers(2, 7)), 6, p_leaf=0.4)) for _ in range(12)]
+    b = gen.pack(seqs)
+    run_case(P, b, 2, 64, "f32", 21)
+    run_case(P, b, 2, 64, "bf16", 22)
+
+
+def test_forward_is_deterministic_and_guard_bands_untouched(P):
+    b = gen.small_random_batch(55, n_seqs=3, max_len=300)
+    T, H, d = b.total_tokens, 2, 64
+    t = gen.make_tensors(5, T, H, d, "bf16")
+    idx = P.hdt_build_index(*dev_struct(b))
+    q, k, v = (dev_tensor(t[n], "bf16") for n in ("q", "k", "v"))
+    big = torch.full((T + 2, H, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+    o1, lse1 = P.hdt_attn_fwd(idx, q, k, v, out=big[1:T + 1])
+    o2, lse2 = P.hdt_attn_fwd(idx, q, k, v)
+    assert torch.equal(o1, o2) and torch.equal(lse1, lse2)
+    assert torch.isnan(big[0]).all() and torch.isnan(big[T + 1]).all()
+
+
+def test_argument_errors(P):
+    b = gen.make_hierarchy(1)
+    idx = P.hdt_build_index(*dev_struct(b))
+    q = torch.zeros((57, 1, 32), device="cuda")
+    with pytest.raises(P.HdtError) as e:
+        P.hdt_attn_fwd(idx, q, q, q)
+    assert e.value.code == -3
+    q = torch.zeros((57, 1, 64), device="cuda")
+    with pytest.raises(P.HdtError) as e:
+        P.hdt_attn_fwd(idx, q, q, q, workspace=torch.empty(256, dtype=torch.uint8, device="cuda")[:16])
+    assert e.value.code == -4
+
+
+# ------------------------------------------------------------------------------------------
+# full-size configurations: sampled rows / keys against the oracle, properties everywhere
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("c", [2, 3, 4, 5])
+def test_full_size_config_sampled(P, c):
+    cfg = gen.CONFIGS[c]
+    b = gen.make_hierarchy(c)
+    T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
+    t = gen.make_tensors(cfg.tensor_seed, T, H, d, cfg.dtype)
+    idx = P.hdt_build_index(*dev_struct(b), max_stages=4)
+    q, k, v, do = (dev_tensor(t[n], cfg.dtype) for n in ("q", "k", "v", "do"))
+    o, lse = P.hdt_attn_fwd(idx, q, k, v)
+    rng = np.random.default_rng(c)
+    real = np.flatnonzero(b.level >= 0)
+    anchors = np.flatnonzero((b.level >= 0) & (b.level < 3))
+    n_s = 24 if c == 5 else 48
+    sample = np.unique(np.concatenate([rng.choice(real, n_s, replace=False),
+                                       rng.choice(anchors, 12, replace=False),
+                                       b.cu_seqlens[:-1], b.cu_seqlens[1:] - 1])).astype(np.int32)
+    o_r, lse_r, dq_r = oracle.rows(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], sample,
+                                   do=t["do"] if cfg.backward else None)
+    check_close(host(o[sample.astype(np.int64)]), o_r, cfg.dtype, "O")
+    check_close(host(lse[:, sample.astype(np.int64)]).T, lse_r, cfg.dtype, "LSE")
+    # properties at full size: PAD rows are zero / -inf, real rows finite
+    pad = torch.from_numpy(b.level < 0).cuda()
+    assert torch.isfinite(o.float()).all()
+    if pad.any():
+        assert (o[pad] == 0).all() and torch.isneginf(lse[:, pad]).all()
+    assert torch.isfinite(lse[:, ~pad]).all()
+    if cfg.backward:
+        dq, dk, dv = P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
+        check_close(host(dq[sample.astype(np.int64)]), dq_r, cfg.dtype, "dQ")
+        cols = sample[:: 4 if c == 5 else 2]
+        dk_r, dv_r = oracle.cols(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], t["do"], cols)
+        check_close(host(dk[cols.astype(np.int64)]), dk_r, cfg.dtype, "dK")
+        check_close(host(dv[cols.astype(np.int64)]), dv_r, cfg.dtype, "dV")
+        for g in (dq, dk, dv):
+            assert torch.isfinite(g.float()).all()
+            if pad.any():
+                assert (g[pad] == 0).all()
+        # sum_j dS_ij = 0  =>  sum over tokens of dK = scale * sum_i (sum_j dS_ij ...) has no closed form,
+        # but sum over rows of dV equals sum_i dO_i (columns of S^T sum rows of S = 1) per head
+        tot_dv = dv.float().sum(0)
+        tot_do = do.float()[~pad].sum(0)
+        assert torch.allclose(tot_dv, tot_do, atol=2.0 if cfg.dtype == "bf16" else 1e-2, rtol=2e-2)
