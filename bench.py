@@ -1,0 +1,417 @@
+#!/usr/bin/env python
+"""Benchmark of the HDT hierarchical-attention hot path on B200.
+
+One step = hdt_build_index + hdt_attn_fwd + hdt_attn_bwd over one batch of synthetic
+hierarchical documents (default workload: batch 4 x 8192 tokens, 12 heads x 64, bf16, the shape
+of the paper's single-layer efficiency protocol).  Prints ONE JSON line on rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--impl reference]
+
+N > 1 (under torch.distributed.run): every rank runs an independent replica of the batch; there
+is no collective on the data path (the path does not shard inside a sequence).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+METRIC = "HDT attention fwd+bwd effective TFLOP/s (unmasked pairs) and % of bf16 peak; tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM traffic (read + write bytes per launch) of the dominant kernel from the ncu captures
+# summarised under profiles/; keyed by (config, profile id).  None = not captured.
+NCU_TRAFFIC = {}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def workload(c):
+    cfg = gen.CONFIGS[c]
+    b = gen.make_hierarchy(c)
+    return cfg, b
+
+
+def flops_per_step(nnz, H, d, backward):
+    return (4 + (10 if backward else 0)) * d * nnz * H
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    REASONS = {0x1: "gpu_idle", 0x2: "applications_clocks_setting", 0x4: "sw_power_cap", 0x8: "hw_slowdown",
+               0x10: "sync_boost", 0x20: "sw_thermal_slowdown", 0x40: "hw_thermal_slowdown",
+               0x80: "hw_power_brake_slowdown", 0x100: "display_clock_setting"}
+
+    def __init__(self, torch_dev):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._h = None
+        try:
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(torch_dev).uuid)
+                self._h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+                idx = int(vis.split(",")[torch_dev]) if vis and vis.split(",")[0].isdigit() else torch_dev
+                self._h = pynvml.nvmlDeviceGetHandleByIndex(idx)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self._h = None
+        self._t = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) if hasattr(
+                    nv, "nvmlDeviceGetCurrentClocksEventReasons") else int(
+                    nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if bits & bit and name != "gpu_idle":
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(0.05)
+
+    def __enter__(self):
+        if self._h is not None:
+            self._t.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        if self._h is not None:
+            self._t.join(timeout=2)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
+        return {"sm_mhz": int(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(c, cfg, b, heads=None, seqs=None):
+    """Sub-batch of the workload for the oracle: the listed sequences and the first `heads` heads."""
+    seqs = list(range(b.batch)) if seqs is None else seqs
+    parts = [(b.level[b.cu_seqlens[s]:b.cu_seqlens[s + 1]], b.parent[b.cu_seqlens[s]:b.cu_seqlens[s + 1]])
+             for s in seqs]
+    sub = gen.pack(parts)
+    H = cfg.heads if heads is None else heads
+    t = gen.make_tensors(cfg.tensor_seed, sub.total_tokens, H, cfg.head_dim, cfg.dtype)
+    return sub, t, H
+
+
+def oracle_step(sub, t, backward):
+    import oracle
+    t0 = time.perf_counter()
+    oracle.forward(sub.level, sub.parent, sub.cu_seqlens, t["q"], t["k"], t["v"])
+    if backward:
+        oracle.backward(sub.level, sub.parent, sub.cu_seqlens, t["q"], t["k"], t["v"], t["do"])
+    return time.perf_counter() - t0
+
+
+def oracle_nnz(sub):
+    ch = np.zeros(sub.total_tokens, np.int64)
+    nnz = 0
+    for s in range(sub.batch):
+        lo, hi = sub.cu_seqlens[s], sub.cu_seqlens[s + 1]
+        pa = sub.parent[lo:hi]
+        real = sub.level[lo:hi] >= 0
+        if not real.any():
+            continue
+        c = np.bincount(pa[pa >= 0], minlength=hi - lo)
+        heads = np.flatnonzero(c > 0)
+        nnz += int(((1 + c[heads]) ** 2).sum()) - int((heads != 0).sum()) if real.sum() > 1 else 1
+    return nnz
+
+
+CPU_SAMPLES = {2: dict(seqs=None, heads=None), 3: dict(seqs=None, heads=None),
+               4: dict(seqs=[0, 1], heads=4), 5: dict(seqs=[0], heads=2), 1: dict(seqs=None, heads=None)}
+
+
+def cpu_baseline(c, cfg, b):
+    import oracle
+    spec = CPU_SAMPLES[c]
+    sub, t, H = oracle_sample(c, cfg, b, spec["heads"], spec["seqs"])
+    dt = oracle_step(sub, t, cfg.backward)
+    fl = flops_per_step(oracle_nnz(sub), H, cfg.head_dim, cfg.backward)
+    return {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"{sub.batch} of {b.batch} sequences ({sub.total_tokens} tokens), {H} of {cfg.heads} heads, "
+                      f"forward{'+backward' if cfg.backward else ''} once, {dt:.2f} s",
+            "tokens_per_s": sub.real_tokens / dt * (H / cfg.heads)}
+
+
+def run_reference(args):
+    """The oracle as the reference arm: each step is a bounded sample of the workload."""
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    c = args.config
+    cfg, b = workload(c)
+    total = args.steps + args.warmup
+    budget = 90.0 / max(total, 1)
+    # probe with one head of sequence 0 to size the sample
+    sub, t, _ = oracle_sample(c, cfg, b, 1, [0])
+    t1 = oracle_step(sub, t, cfg.backward)
+    heads = int(max(1, min(cfg.heads, budget // max(t1, 1e-3))))
+    sub, t, H = oracle_sample(c, cfg, b, heads, [0])
+    for _ in range(args.warmup):
+        oracle_step(sub, t, cfg.backward)
+    times = [oracle_step(sub, t, cfg.backward) for _ in range(args.steps)]
+    dt = float(np.mean(times))
+    fl = flops_per_step(oracle_nnz(sub), H, cfg.head_dim, cfg.backward)
+    val = fl / dt / 1e12
+    sample = (f"sequence 0 of {b.batch} ({sub.total_tokens} tokens), {H} of {cfg.heads} heads, "
+              f"forward{'+backward' if cfg.backward else ''} per step")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": cfg.name, "description": cfg.description, "heads": cfg.heads,
+                       "head_dim": cfg.head_dim, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "tokens_per_s": sub.real_tokens / dt * (H / cfg.heads), "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU arm
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5])
+    ap.add_argument("--impl", default="hdt", choices=["hdt", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    args.warmup = max(args.warmup, 3)
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2407_08330_b200 as P
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    c = args.config
+    cfg, b = workload(c)
+    T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
+    tdt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+    t = gen.make_tensors(cfg.tensor_seed + rank, T, H, d, cfg.dtype)
+
+    def pin(x, dt=None):
+        h = torch.from_numpy(np.ascontiguousarray(x))
+        if dt is not None:
+            h = h.to(dt)
+        return h.pin_memory()
+
+    h_level, h_parent, h_cu = pin(b.level), pin(b.parent), pin(b.cu_seqlens)
+    h_q, h_k, h_v, h_do = (pin(t[n], tdt) for n in ("q", "k", "v", "do"))
+    del t
+    level, parent, cu = h_level.to(dev), h_parent.to(dev), h_cu.to(dev)
+    q, k, v, do = h_q.to(dev), h_k.to(dev), h_v.to(dev), h_do.to(dev)
+    o = torch.empty_like(q)
+    lse = torch.empty((H, T), dtype=torch.float32, device=dev)
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
+    ws_index = torch.empty(P.hdt_index_workspace_bytes(b.batch, T, 0, 4), dtype=torch.uint8, device=dev)
+    idx0 = P.hdt_build_index(level, parent, cu, max_stages=4, workspace=ws_index)
+    nnz = idx0.nnz
+    ws_f = torch.empty(max(256, P.hdt_attn_workspace_bytes(idx0, H, d, tdt, 0)), dtype=torch.uint8, device=dev)
+    ws_b = torch.empty(max(256, P.hdt_attn_workspace_bytes(idx0, H, d, tdt, 1)), dtype=torch.uint8, device=dev)
+    visited, n_stages = idx0.visited, idx0.n_stages
+    del idx0
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
+
+    def step():
+        idx = P.hdt_build_index(level, parent, cu, max_stages=4, workspace=ws_index)
+        P.hdt_attn_fwd(idx, q, k, v, out=o, lse=lse, workspace=ws_f)
+        if cfg.backward:
+            P.hdt_attn_bwd(idx, q, k, v, o, lse, do, dq=dq, dk=dk, dv=dv, workspace=ws_b)
+        idx.close()
+
+    def timed(fn, steps):
+        """Per-step CUDA events on the launch stream, L2 flushed (untimed) before every step."""
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for a, z in ev:
+            flush.zero_()
+            a.record()
+            fn()
+            z.record()
+        torch.cuda.synchronize()
+        return [a.elapsed_time(z) for a, z in ev]
+
+    for _ in range(args.warmup):
+        flush.zero_()
+        step()
+    barrier()
+    l0 = P.hdt_launch_count()
+    with ClockSampler(local) as clk:
+        w0 = time.perf_counter()
+        times = timed(step, args.steps)
+        barrier()
+        wall = time.perf_counter() - w0
+    launches = P.hdt_launch_count() - l0
+    ms = float(np.sum(times)) / args.steps
+    if world > 1:
+        tm = torch.tensor([ms], device=dev)
+        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+        ms = float(tm.item())
+
+    # phase split and per-kernel device times (library-side CUDA events on the launch stream)
+    L = P.lib()
+    import ctypes as C
+    L.hdt_profile_enable(1)
+    for i in range(6):
+        L.hdt_profile_read(i, None, None, 1)
+    for _ in range(2):
+        flush.zero_()
+        step()
+    for i in range(6):
+        L.hdt_profile_read(i, None, None, 1)
+    timed(step, args.steps)
+    kern = {}
+    for i in range(6):
+        n_, ms_ = C.c_int64(), C.c_double()
+        L.hdt_profile_read(i, C.byref(n_), C.byref(ms_), 1)
+        L.hdt_profile_name.restype = C.c_char_p
+        if n_.value:
+            kern[L.hdt_profile_name(i).decode()] = {"launches_per_step": n_.value / args.steps,
+                                                    "ms_per_step": ms_.value / args.steps}
+    L.hdt_profile_enable(0)
+
+    # end-to-end through the public API with host buffers (pinned): H2D of all inputs, D2H of all results
+    e2e = None
+    if not args.no_e2e:
+        ho, hdq, hdk, hdv = (torch.empty_like(h_q).pin_memory() for _ in range(4))
+        hlse = torch.empty((H, T), dtype=torch.float32).pin_memory()
+
+        def step_e2e():
+            level.copy_(h_level, non_blocking=True); parent.copy_(h_parent, non_blocking=True)
+            cu.copy_(h_cu, non_blocking=True)
+            q.copy_(h_q, non_blocking=True); k.copy_(h_k, non_blocking=True); v.copy_(h_v, non_blocking=True)
+            if cfg.backward:
+                do.copy_(h_do, non_blocking=True)
+            step()
+            ho.copy_(o, non_blocking=True); hlse.copy_(lse, non_blocking=True)
+            if cfg.backward:
+                hdq.copy_(dq, non_blocking=True); hdk.copy_(dk, non_blocking=True); hdv.copy_(dv, non_blocking=True)
+
+        for _ in range(2):
+            step_e2e()
+        barrier()
+        n_e = max(3, min(args.steps, 10))
+        w0 = time.perf_counter()
+        for _ in range(n_e):
+            step_e2e()
+        barrier()
+        e_ms = (time.perf_counter() - w0) / n_e * 1e3
+        if world > 1:
+            tm = torch.tensor([e_ms], device=dev)
+            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
+            e_ms = float(tm.item())
+        esz = q.element_size()
+        n_in = 3 + (1 if cfg.backward else 0)
+        n_out = 1 + (3 if cfg.backward else 0)
+        e2e = {"value": flops_per_step(nnz, H, d, cfg.backward) * world / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+               "h2d_bytes_per_step": n_in * T * H * d * esz + T * 5 + (b.batch + 1) * 4,
+               "d2h_bytes_per_step": n_out * T * H * d * esz + H * T * 4, "ms_per_step": e_ms}
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    pk = peaks()
+    fl = flops_per_step(nnz, H, d, cfg.backward)
+    value = fl * world / (ms * 1e-3) / 1e12
+    real = b.real_tokens
+    esz = 2 if cfg.dtype == "bf16" else 4
+    alg_bytes = {"k_fwd_stage0": (4 * d * esz + 4) * real * H,
+                 "k_bwd_stage0": (7 * d * esz + 8) * real * H,
+                 "k_delta": (2 * d * esz + 4) * real * H}
+    dom = max((kk for kk in kern if kk in alg_bytes), key=lambda kk: kern[kk]["ms_per_step"], default=None)
+    roofline = None
+    if dom:
+        dur = kern[dom]["ms_per_step"] / kern[dom]["launches_per_step"] * 1e-3
+        ach = alg_bytes[dom] / dur / 1e9
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / pk["hbm_gbs"], "traffic": NCU_TRAFFIC.get((c, dom)),
+                    "peak_source": pk["_source"], "algorithmic_bytes_per_launch": alg_bytes[dom],
+                    "kernel_ms": dur * 1e3}
+        for kk in kern:
+            if kk in alg_bytes:
+                kd = kern[kk]["ms_per_step"] / kern[kk]["launches_per_step"] * 1e-3
+                kern[kk]["achieved_gbs"] = alg_bytes[kk] / kd / 1e9
+                kern[kk]["frac_of_hbm_peak"] = kern[kk]["achieved_gbs"] / pk["hbm_gbs"]
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
+        "config": {"workload": cfg.name, "description": cfg.description, "batch": b.batch, "total_tokens": T,
+                   "real_tokens": real, "heads": H, "head_dim": d, "nnz_pairs_per_head": nnz,
+                   "visited_pairs_per_head": visited, "stages": n_stages,
+                   "step": "hdt_build_index + hdt_attn_fwd" + (" + hdt_attn_bwd" if cfg.backward else ""),
+                   "l2": "flushed between timed steps (256 MiB write, untimed)", "parallelism": f"replicas x{world}"},
+        "pct_bf16_peak": 100.0 * value / world / pk["bf16_tflops"],
+        "tokens_per_s": real * world / (ms * 1e-3),
+        "wall_ms_per_step_incl_flush": wall / args.steps * 1e3,
+        "kernels": kern, "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches),
+        "clocks": clk.summary(),
+    }
+    if not args.no_cpu_baseline and world >= 1:
+        line["cpu_baseline"] = cpu_baseline(c, cfg, b)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -174,6 +174,18 @@ const char *hdt_last_error(void);
 /* Number of kernel launches the library has issued in this process (for benchmarks). */
 int64_t hdt_launch_count(void);
 
+/*
+ * Optional per-kernel timing for benchmarks (no counterpart in the paper).  When enabled, the
+ * library brackets its launches with CUDA events on the launch stream.  Kernel ids:
+ * 0 index build (all its kernels), 1 forward stage 0, 2 forward upper stages, 3 delta,
+ * 4 backward stage 0, 5 backward upper stages.  hdt_profile_read waits for the recorded events,
+ * returns the number of bracketed launches and their summed device time in milliseconds since
+ * the last reset, and clears them when reset != 0.
+ */
+int hdt_profile_enable(int32_t on);
+const char *hdt_profile_name(int32_t id);
+int hdt_profile_read(int32_t id, int64_t *launches, double *total_ms, int32_t reset);
+
 #ifdef __cplusplus
 }
 #endif

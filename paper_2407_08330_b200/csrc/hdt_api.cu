@@ -2,6 +2,8 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <mutex>
+#include <vector>
 
 #include "hdt_internal.cuh"
 
@@ -16,6 +18,32 @@ int set_error(int code, const char *fmt, ...) {
     vsnprintf(g_err, sizeof(g_err), fmt, ap);
     va_end(ap);
     return code;
+}
+
+// ---- optional event timing -------------------------------------------------------------------
+struct ProfRec { int id; cudaEvent_t a, b; };
+static std::mutex g_prof_mu;
+static bool g_prof_on = false;
+static std::vector<ProfRec> g_prof_recs;      // recorded since the last read
+static std::vector<ProfRec> g_prof_pool;      // created, free
+static double g_prof_ms[PROF_COUNT];
+static long long g_prof_n[PROF_COUNT];
+
+ProfScope::ProfScope(int id, cudaStream_t s) : slot(-1), st(s) {
+    if (!g_prof_on) return;
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    ProfRec r;
+    if (!g_prof_pool.empty()) { r = g_prof_pool.back(); g_prof_pool.pop_back(); }
+    else if (cudaEventCreate(&r.a) != cudaSuccess || cudaEventCreate(&r.b) != cudaSuccess) return;
+    r.id = id;
+    cudaEventRecord(r.a, st);
+    g_prof_recs.push_back(r);
+    slot = (int)g_prof_recs.size() - 1;
+}
+ProfScope::~ProfScope() {
+    if (slot < 0) return;
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    cudaEventRecord(g_prof_recs[slot].b, st);
 }
 
 static size_t al256(size_t x) { return (x + 255) & ~size_t(255); }
@@ -62,6 +90,36 @@ using namespace hdt;
 extern "C" const char *hdt_last_error(void) { return g_err; }
 extern "C" int64_t hdt_launch_count(void) { return (int64_t)g_launches.load(); }
 
+extern "C" int hdt_profile_enable(int32_t on) {
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    g_prof_on = on != 0;
+    return HDT_OK;
+}
+
+extern "C" const char *hdt_profile_name(int32_t id) {
+    static const char *names[PROF_COUNT] = {"index_build(all kernels)", "k_fwd_stage0", "k_fwd_upper_stages",
+                                            "k_delta", "k_bwd_stage0", "k_bwd_upper_stages"};
+    return (id >= 0 && id < PROF_COUNT) ? names[id] : "";
+}
+
+extern "C" int hdt_profile_read(int32_t id, int64_t *launches, double *total_ms, int32_t reset) {
+    if (id < 0 || id >= PROF_COUNT) return set_error(HDT_ERR_INVALID_ARG, "hdt_profile_read: bad id %d", id);
+    std::lock_guard<std::mutex> lk(g_prof_mu);
+    for (ProfRec &r : g_prof_recs) {   // fold finished records into the totals
+        HDT_CUDA_CHECK(cudaEventSynchronize(r.b));
+        float ms = 0.f;
+        HDT_CUDA_CHECK(cudaEventElapsedTime(&ms, r.a, r.b));
+        g_prof_ms[r.id] += ms;
+        g_prof_n[r.id] += 1;
+        g_prof_pool.push_back(r);
+    }
+    g_prof_recs.clear();
+    if (launches) *launches = g_prof_n[id];
+    if (total_ms) *total_ms = g_prof_ms[id];
+    if (reset) { g_prof_n[id] = 0; g_prof_ms[id] = 0.0; }
+    return HDT_OK;
+}
+
 extern "C" size_t hdt_attn_workspace_bytes(const hdt_index_t *ix, int32_t heads, int32_t head_dim,
                                            int32_t dtype, int32_t bwd) {
     (void)dtype;
@@ -97,7 +155,10 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         }
         if (s == 0) { a.o = o; a.lse = lse; }
         else { a.part_o = (float *)(ws + L.part[s][0]); a.part_lse = (float *)(ws + L.part[s][1]); }
-        rc = launch_fwd_simt(a, head_dim, dtype, st);
+        {
+            ProfScope ps(s == 0 ? PROF_FWD_STAGE0 : PROF_FWD_UPPER, st);
+            rc = launch_fwd_simt(a, head_dim, dtype, st);
+        }
         if (rc) return rc;
     }
     return HDT_OK;
@@ -121,7 +182,10 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     cudaStream_t st = (cudaStream_t)stream;
     char *ws = (char *)workspace;
     float *delta = (float *)(ws + L.delta);
-    rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
+    {
+        ProfScope ps(PROF_DELTA, st);
+        rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
+    }
     if (rc) return rc;
     for (int s = ix->n_stages - 1; s >= 0; --s) {
         const StagePtrs &P = ix->st[s];
@@ -143,7 +207,10 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             a.part_dk = (float *)(ws + L.part[s][1]);
             a.part_dv = (float *)(ws + L.part[s][2]);
         }
-        rc = launch_bwd_simt(a, head_dim, dtype, st);
+        {
+            ProfScope ps(s == 0 ? PROF_BWD_STAGE0 : PROF_BWD_UPPER, st);
+            rc = launch_bwd_simt(a, head_dim, dtype, st);
+        }
         if (rc) return rc;
     }
     return HDT_OK;

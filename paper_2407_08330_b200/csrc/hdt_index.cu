@@ -463,6 +463,8 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         }                                                                              \
     } while (0)
 
+    {
+    ProfScope ps(PROF_INDEX, st);
     HDT_BUILD_CHECK(cudaMemsetAsync(hdr, 0, sizeof(DevHeader), st));
     const int nel = max(T, B + 1);
     const int g_el = (nel + 255) / 256;
@@ -503,6 +505,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         count_launch(4);
     }
     HDT_BUILD_CHECK(cudaGetLastError());
+    }
     DevHeader h;
     HDT_BUILD_CHECK(cudaMemcpyAsync(&h, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, st));
     HDT_BUILD_CHECK(cudaStreamSynchronize(st));

@@ -46,6 +46,16 @@ int set_error(int code, const char *fmt, ...);
 extern std::atomic<long long> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
+// Optional per-kernel timing with CUDA events on the launch stream (off by default).
+enum ProfId { PROF_INDEX = 0, PROF_FWD_STAGE0, PROF_FWD_UPPER, PROF_DELTA, PROF_BWD_STAGE0, PROF_BWD_UPPER,
+              PROF_COUNT };
+struct ProfScope {
+    int slot;
+    cudaStream_t st;
+    ProfScope(int id, cudaStream_t st);
+    ~ProfScope();
+};
+
 #define HDT_CUDA_CHECK(expr)                                                                  \
     do {                                                                                      \
         cudaError_t e_ = (expr);                                                              \
