@@ -186,6 +186,24 @@ int hdt_profile_enable(int32_t on);
 const char *hdt_profile_name(int32_t id);
 int hdt_profile_read(int32_t id, int64_t *launches, double *total_ms, int32_t reset);
 
+/*
+ * Waits for `stream`, then returns and clears the first failure a kernel of this library
+ * recorded on the device: HDT_ERR_TIMEOUT when a bounded wait (on a TMA or tensor-core
+ * completion barrier) ran out; results of that call are then undefined.  HDT_OK if none.
+ * (No counterpart in the paper.)
+ */
+int hdt_device_status(void *stream);
+
+/*
+ * Test hook for the tensor-core primitives (no counterpart in the paper): C[128,N] = A * B on
+ * one CTA with TMA-staged, 128-byte-swizzled operands and tcgen05.mma.
+ *   a  device bf16 [128, K] (a_mn = 0) or [K, 128] (a_mn = 1)
+ *   b  device bf16 [N, K] (b_mn = 0, C = A B^T) or [K, N] (b_mn = 1, C = A B)
+ *   c  device float [128, N];  N, K multiples of 16 in 16..128.  Waits for the result.
+ */
+int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
+                   void *stream);
+
 #ifdef __cplusplus
 }
 #endif

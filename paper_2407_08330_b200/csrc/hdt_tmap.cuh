@@ -1,0 +1,43 @@
+// Host side: TMA tensor maps for [T, H, D] bf16 tensors (D innermost), box = (64, 1, box_rows),
+// 128-byte swizzle.  cuTensorMapEncodeTiled is fetched through the runtime, so libcuda is not
+// linked.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "hdt_internal.cuh"
+
+namespace hdt {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// base: device pointer, 16-byte aligned; D: inner extent (elements, D * 2 bytes a multiple of 16).
+inline int make_tmap_bf16(CUtensorMap *tm, const void *base, int D, int H, long long T, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return set_error(HDT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)(T > 0 ? T : 1)};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)D * 2 * (cuuint64_t)H};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return set_error(HDT_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+    return HDT_OK;
+}
+
+}  // namespace hdt
