@@ -187,6 +187,12 @@ const char *hdt_profile_name(int32_t id);
 int hdt_profile_read(int32_t id, int64_t *launches, double *total_ms, int32_t reset);
 
 /*
+ * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
+ * through the fp32 SIMT kernels instead of the tensor-core kernels (A/B comparisons, tests).
+ */
+int hdt_set_option(const char *name, int32_t value);
+
+/*
  * Waits for `stream`, then returns and clears the first failure a kernel of this library
  * recorded on the device: HDT_ERR_TIMEOUT when a bounded wait (on a TMA or tensor-core
  * completion barrier) ran out; results of that call are then undefined.  HDT_OK if none.

@@ -202,5 +202,16 @@ def hdt_attn_bwd(index: HdtIndex, q, k, v, o, lse, d_o, softmax_scale=0.0, dq=No
     return dq, dk, dv
 
 
+def hdt_set_option(name: str, value: int) -> None:
+    lib().hdt_set_option.restype = C.c_int
+    _check(lib().hdt_set_option(C.c_char_p(name.encode()), C.c_int32(int(value))))
+
+
+def hdt_device_status() -> None:
+    """Wait for the current stream and raise if a kernel recorded a device-side failure."""
+    lib().hdt_device_status.restype = C.c_int
+    _check(lib().hdt_device_status(_stream()))
+
+
 def hdt_launch_count() -> int:
     return int(lib().hdt_launch_count())

@@ -2,6 +2,7 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstring>
 #include <mutex>
 #include <vector>
 
@@ -46,6 +47,18 @@ ProfScope::~ProfScope() {
     cudaEventRecord(g_prof_recs[slot].b, st);
 }
 
+// ---- device-side failure word -------------------------------------------------------------------
+__device__ int g_device_status = 0;  // first failure recorded by a kernel (hdt_status_t), 0 = none
+
+int *device_status_ptr() {
+    int *p = nullptr;
+    if (cudaGetSymbolAddress((void **)&p, g_device_status) != cudaSuccess) {
+        set_error(HDT_ERR_CUDA, "cudaGetSymbolAddress(g_device_status) failed");
+        return nullptr;
+    }
+    return p;
+}
+
 static size_t al256(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct AttnLayout {
@@ -87,8 +100,28 @@ static bool misaligned(const void *p) { return ((uintptr_t)p & 15) != 0; }
 
 using namespace hdt;
 
+static int g_force_simt = 0;
+
+extern "C" int hdt_set_option(const char *name, int32_t value) {
+    if (name && std::strcmp(name, "force_simt") == 0) { g_force_simt = value; return HDT_OK; }
+    return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
+}
+
 extern "C" const char *hdt_last_error(void) { return g_err; }
 extern "C" int64_t hdt_launch_count(void) { return (int64_t)g_launches.load(); }
+
+// Waits for `stream`, then returns and clears the first failure recorded by a kernel.
+extern "C" int hdt_device_status(void *stream) {
+    HDT_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
+    int h = 0;
+    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)));
+    if (h != 0) {
+        const int zero = 0;
+        HDT_CUDA_CHECK(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)));
+        return set_error(h, "a kernel recorded device-side failure %d (a bounded wait ran out)", h);
+    }
+    return HDT_OK;
+}
 
 extern "C" int hdt_profile_enable(int32_t on) {
     std::lock_guard<std::mutex> lk(g_prof_mu);
@@ -141,6 +174,8 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
     cudaStream_t st = (cudaStream_t)stream;
     char *ws = (char *)workspace;
+    int *status = device_status_ptr();
+    if (!status) return HDT_ERR_CUDA;
     for (int s = ix->n_stages - 1; s >= 0; --s) {
         const StagePtrs &P = ix->st[s];
         FwdStageArgs a{};
@@ -155,9 +190,11 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         }
         if (s == 0) { a.o = o; a.lse = lse; }
         else { a.part_o = (float *)(ws + L.part[s][0]); a.part_lse = (float *)(ws + L.part[s][1]); }
+        a.status = status;
         {
             ProfScope ps(s == 0 ? PROF_FWD_STAGE0 : PROF_FWD_UPPER, st);
-            rc = launch_fwd_simt(a, head_dim, dtype, st);
+            if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
+            else rc = launch_fwd_simt(a, head_dim, dtype, st);
         }
         if (rc) return rc;
     }

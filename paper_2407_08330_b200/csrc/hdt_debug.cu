@@ -9,8 +9,6 @@
 namespace hdt {
 using namespace sm100;
 
-__device__ int g_device_status = 0;  // first device-side failure (hdt_status_t), 0 = none
-
 struct DebugGemmArgs {
     int N, K, a_mn, b_mn;
     float *c;  // [128, N]
@@ -90,8 +88,8 @@ extern "C" int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N,
     if (rc) return rc;
     rc = make_tmap_bf16(&tb, b, b_mn ? N : K, 1, b_mn ? K : N, 128);
     if (rc) return rc;
-    int *status;
-    HDT_CUDA_CHECK(cudaGetSymbolAddress((void **)&status, g_device_status));
+    int *status = device_status_ptr();
+    if (!status) return HDT_ERR_CUDA;
     DebugGemmArgs g{N, K, a_mn, b_mn, c, status};
     const int smem = 4 * 16384 + 1024 + 64;
     HDT_CUDA_CHECK(cudaFuncSetAttribute(k_debug_gemm, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -101,16 +99,3 @@ extern "C" int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N,
     return hdt_device_status(stream);
 }
 
-// Waits for `stream`, then returns and clears the first failure recorded by a kernel of this
-// library (HDT_ERR_TIMEOUT when a bounded device-side wait ran out), HDT_OK if none.
-extern "C" int hdt_device_status(void *stream) {
-    HDT_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
-    int h = 0;
-    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)));
-    if (h != 0) {
-        const int zero = 0;
-        HDT_CUDA_CHECK(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)));
-        return set_error(h, "a kernel recorded device-side failure %d (bounded wait ran out)", h);
-    }
-    return HDT_OK;
-}

@@ -43,6 +43,7 @@ struct hdt_index {
 namespace hdt {
 
 int set_error(int code, const char *fmt, ...);
+int *device_status_ptr();  // device address of the failure word kernels report into
 extern std::atomic<long long> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
@@ -79,6 +80,7 @@ struct FwdStageArgs {
     int T;
     // ... or this stage's partial results
     float *part_o, *part_lse;
+    int *status;        // device failure word
 };
 
 struct BwdStageArgs {
@@ -95,6 +97,8 @@ struct BwdStageArgs {
 };
 
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
+// Tensor-core (TMA + tcgen05) stage-0 kernels for bf16 (hdt_attn_tc.cu).
+int launch_fwd_tc(const FwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
                  cudaStream_t st);

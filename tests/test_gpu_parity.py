@@ -100,6 +100,16 @@ def test_index_rejects_bad_hierarchies(P):
 # attention, small cases compared element by element
 # ------------------------------------------------------------------------------------------
 def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
+    """bf16 runs twice: tensor-core stage-0 kernels, then the SIMT kernels on every stage."""
+    for force_simt in ((0, 1) if dtype == "bf16" else (0,)):
+        P.hdt_set_option("force_simt", force_simt)
+        try:
+            _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale)
+        finally:
+            P.hdt_set_option("force_simt", 0)
+
+
+def _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale):
     t = gen.make_tensors(seed, b.total_tokens, H, d, dtype)
     idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=8)
     q, k, v, do = (dev_tensor(t[n], dtype) for n in ("q", "k", "v", "do"))
@@ -115,7 +125,7 @@ def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
         check_close(host(dq), dq_r, dtype, "dQ")
         check_close(host(dk), dk_r, dtype, "dK")
         check_close(host(dv), dv_r, dtype, "dV")
-    torch.cuda.synchronize()
+    P.hdt_device_status()
 
 
 def test_config1_fp32_forward(P):
@@ -221,6 +231,7 @@ def test_full_size_config_sampled(P, c):
                 assert (g[pad] == 0).all()
         # sum_j dS_ij = 0  =>  sum over tokens of dK = scale * sum_i (sum_j dS_ij ...) has no closed form,
         # but sum over rows of dV equals sum_i dO_i (columns of S^T sum rows of S = 1) per head
+        P.hdt_device_status()
         tot_dv = dv.float().sum(0)
         tot_do = do.float()[~pad].sum(0)
         assert torch.allclose(tot_dv, tot_do, atol=2.0 if cfg.dtype == "bf16" else 1e-2, rtol=2e-2)
