@@ -219,6 +219,8 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     cudaStream_t st = (cudaStream_t)stream;
     char *ws = (char *)workspace;
     float *delta = (float *)(ws + L.delta);
+    int *status = device_status_ptr();
+    if (!status) return HDT_ERR_CUDA;
     {
         ProfScope ps(PROF_DELTA, st);
         rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
@@ -244,9 +246,11 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             a.part_dk = (float *)(ws + L.part[s][1]);
             a.part_dv = (float *)(ws + L.part[s][2]);
         }
+        a.status = status;
         {
             ProfScope ps(s == 0 ? PROF_BWD_STAGE0 : PROF_BWD_UPPER, st);
-            rc = launch_bwd_simt(a, head_dim, dtype, st);
+            if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
+            else rc = launch_bwd_simt(a, head_dim, dtype, st);
         }
         if (rc) return rc;
     }

@@ -1,0 +1,340 @@
+// Tensor-core backward for stage 0 in bf16 (TMA + tcgen05/TMEM).
+//
+// One CTA (256 threads) per (row block, head).  A "tile pass" takes a query-side tile (Q, dO of
+// 128 token rows with their LSE and delta) and a key-side tile (K, V of 128 token rows):
+//   MMA   S = Q K^T, dP = dO V^T                                   -> TMEM
+//   rows  P = exp2(S*c - LSE) on the columns inside the row's family range, dS = P o (dP - delta);
+//         P and dS (bf16) -> shared memory, one sub-tile per 64 keys
+//   MMA   dQ += dS K  |  dV += P^T dO, dK += dS^T Q                 -> TMEM
+// Thread t handles row t % 128 (its TMEM lane) and the column half t / 128.
+// A block whose key span lies inside its own rows (the usual case: blocks are packed from whole
+// families) needs one pass with both tiles equal to the block; at D = 64 that pass produces dQ,
+// dK and dV together (5 MMAs).  Otherwise the block first walks its key span as a query block
+// (dQ), then walks the same span as a key block (dK, dV); the family ranges are symmetric, so the
+// same index serves both.
+#include <cuda_bf16.h>
+
+#include "hdt_internal.cuh"
+#include "hdt_sm100.cuh"
+#include "hdt_tmap.cuh"
+
+namespace hdt {
+using namespace sm100;
+
+static constexpr int SUB = 16384;
+static constexpr long long WAIT_CYCLES = 400000000LL;
+__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
+
+template <int D>
+struct BwdSmem {
+    static constexpr int NSUB = D / 64;
+    uint8_t *sQ, *sDO, *sK, *sV, *sP, *sDS;
+    uint64_t *bar_tma, *bar_mma;
+    uint32_t *slot;
+    volatile int *abort_flag;
+};
+
+template <int D>
+__global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensorMap tm_q,
+                                                const __grid_constant__ CUtensorMap tm_k,
+                                                const __grid_constant__ CUtensorMap tm_v,
+                                                const __grid_constant__ CUtensorMap tm_do, const BwdStageArgs a) {
+    constexpr int NSUB = D / 64;
+    // TMEM columns: S and dP per pass; accumulators.  At D = 128 dQ and dK share columns (they are
+    // never live together there, the fused pass exists only at D = 64).
+    constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_DK = (D == 64) ? 320 : 256, TM_DV = 384, TM_COLS = 512;
+    constexpr bool FUSE = (D == 64);
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = sm, *sDO = sQ + NSUB * SUB, *sK = sDO + NSUB * SUB, *sV = sK + NSUB * SUB;
+    uint8_t *sP = sV + NSUB * SUB, *sDS = sP + 2 * SUB;
+    uint64_t *bar_tma = (uint64_t *)(sDS + 2 * SUB);
+    uint64_t *bar_mma = bar_tma + 1;
+    uint32_t *slot = (uint32_t *)(bar_mma + 1);
+    volatile int *abort_flag = (volatile int *)(slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, hf = tid >> 7;
+    const int blk = a.queue[blockIdx.x], h = blockIdx.y, H = a.H;
+    const int *rec = a.blocks + 5 * (size_t)blk;
+    const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3], fl = rec[4];
+    const int nrows = r1 - r0;
+    const float LOG2E = 1.4426950408889634f;
+
+    if (tid == 0) {
+        mbar_init(bar_tma, 1);
+        mbar_init(bar_mma, 1);
+        *abort_flag = (*a.status != 0);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    const bool empty = (fl & HDT_BLK_EMPTY) != 0;
+    const bool self = (fl & HDT_BLK_SELF) != 0;
+    uint32_t ph_tma = 0, ph_mma = 0;
+    bool ok = true;
+
+    // One tile pass.  q_row0 / k_row0: first token row of the query-side / key-side tile;
+    // q_end / k_end: end of the valid rows of each side.
+    auto tile_pass = [&](int q_row0, int q_end, int k_row0, int k_end, bool want_dq, bool want_dkdv, bool acc_q,
+                         bool acc_kv) {
+        const int nq = min(128, q_end - q_row0), nk = min(128, k_end - k_row0);
+        const int Nc = (nk + 15) & ~15, Kr = (nq + 15) & ~15;
+        if (tid == 0 && !*abort_flag) {
+            tc_fence_after();
+            const uint32_t idesc = idesc_bf16(Nc, false, false);
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
+                mma_ss(tmem + TM_S, smem_desc(smem_u32(sQ) + off, 0, 1024), smem_desc(smem_u32(sK) + off, 0, 1024), idesc,
+                       kk > 0);
+            }
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
+                mma_ss(tmem + TM_DP, smem_desc(smem_u32(sDO) + off, 0, 1024), smem_desc(smem_u32(sV) + off, 0, 1024), idesc,
+                       kk > 0);
+            }
+            mma_commit(bar_mma);
+        }
+        // row statistics of this thread's query-side row while the MMAs run
+        const int e = q_row0 + rl;
+        const bool inq = e < q_end;
+        int lo = 0, hi = 0;
+        float lse2 = 0.f, dl = 0.f;
+        if (inq) {
+            lo = a.rng[2 * e];
+            hi = a.rng[2 * e + 1];
+            if (hi > lo) {
+                lse2 = a.lse[(size_t)h * a.T + e] * LOG2E;
+                dl = a.delta[(size_t)h * a.T + e];
+            }
+        }
+        const int jl = max(lo - k_row0, 0), jh = min(hi - k_row0, nk);
+        const bool has = inq && jh > jl;
+        ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+        ph_mma ^= 1;
+        tc_fence_after();
+#pragma unroll
+        for (int sl = 0; sl < 2; ++sl) {
+            const int s0 = 64 * hf + 32 * sl;
+            if (s0 >= Nc) continue;  // same decision in the whole warp (hf, Nc uniform)
+            const bool mine = has && jl < s0 + 32 && jh > s0;
+            uint32_t pp[16], pd[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) { pp[j] = 0u; pd[j] = 0u; }
+            if (__any_sync(0xffffffffu, mine)) {
+                uint32_t rs[32], rd[32];
+                tmem_ld32(tmem + TM_S + lane_base + s0, rs);
+                tmem_ld32(tmem + TM_DP + lane_base + s0, rd);
+                tmem_wait_ld();
+                if (mine) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float p0 = 0.f, p1 = 0.f, d0 = 0.f, d1 = 0.f;
+                        if (s0 + j >= jl && s0 + j < jh) {
+                            p0 = exp2f(fmaf(__uint_as_float(rs[j]), a.scale_log2, -lse2));
+                            d0 = p0 * (__uint_as_float(rd[j]) - dl);
+                        }
+                        if (s0 + j + 1 >= jl && s0 + j + 1 < jh) {
+                            p1 = exp2f(fmaf(__uint_as_float(rs[j + 1]), a.scale_log2, -lse2));
+                            d1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
+                        }
+                        pp[j >> 1] = pack_bf16(p0, p1);
+                        pd[j >> 1] = pack_bf16(d0, d1);
+                    }
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                const uint32_t off = hf * SUB + swz(rl, sl * 4 + c);
+                *reinterpret_cast<uint4 *>(sP + off) = make_uint4(pp[4 * c], pp[4 * c + 1], pp[4 * c + 2], pp[4 * c + 3]);
+                *reinterpret_cast<uint4 *>(sDS + off) = make_uint4(pd[4 * c], pd[4 * c + 1], pd[4 * c + 2], pd[4 * c + 3]);
+            }
+        }
+        fence_proxy_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0 && !*abort_flag) {
+            tc_fence_after();
+            const uint32_t idesc_kv = idesc_bf16(D, true, true);   // A = P^T / dS^T, B = dO / Q (both MN-major)
+            const uint32_t idesc_q = idesc_bf16(D, false, true);   // A = dS (K-major), B = K (MN-major)
+            if (want_dkdv) {
+                for (int kk = 0; kk < Kr / 16; ++kk) {
+                    const uint64_t ap = smem_desc(smem_u32(sP) + kk * 2048, SUB, 1024);
+                    const uint64_t bdo = smem_desc(smem_u32(sDO) + kk * 2048, SUB, 1024);
+                    mma_ss(tmem + TM_DV, ap, bdo, idesc_kv, acc_kv || kk > 0);
+                }
+                for (int kk = 0; kk < Kr / 16; ++kk) {
+                    const uint64_t ads = smem_desc(smem_u32(sDS) + kk * 2048, SUB, 1024);
+                    const uint64_t bq = smem_desc(smem_u32(sQ) + kk * 2048, SUB, 1024);
+                    mma_ss(tmem + TM_DK, ads, bq, idesc_kv, acc_kv || kk > 0);
+                }
+            }
+            if (want_dq) {
+                for (int kk = 0; kk < Nc / 16; ++kk) {
+                    const uint64_t ads = smem_desc(smem_u32(sDS) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024);
+                    const uint64_t bk = smem_desc(smem_u32(sK) + kk * 2048, SUB, 1024);
+                    mma_ss(tmem + TM_DQ, ads, bk, idesc_q, acc_q || kk > 0);
+                }
+            }
+            mma_commit(bar_mma);
+        }
+        ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+        ph_mma ^= 1;
+        tc_fence_after();
+    };
+
+    auto load = [&](bool q_side, int row0_q, bool k_side, int row0_k) {
+        if (tid == 0 && !*abort_flag) {
+            mbar_expect_tx(bar_tma, (uint32_t)((q_side ? 2 * NSUB : 0) + (k_side ? 2 * NSUB : 0)) * SUB);
+            for (int s = 0; s < NSUB; ++s) {
+                if (q_side) {
+                    tma_load_3d(sQ + s * SUB, &tm_q, 64 * s, h, row0_q, bar_tma);
+                    tma_load_3d(sDO + s * SUB, &tm_do, 64 * s, h, row0_q, bar_tma);
+                }
+                if (k_side) {
+                    tma_load_3d(sK + s * SUB, &tm_k, 64 * s, h, row0_k, bar_tma);
+                    tma_load_3d(sV + s * SUB, &tm_v, 64 * s, h, row0_k, bar_tma);
+                }
+            }
+        }
+        ok = mbar_wait(bar_tma, ph_tma, abort_flag, WAIT_CYCLES) && ok;
+        ph_tma ^= 1;
+    };
+
+    // Read an accumulator (this thread's row, its half of the D columns), scale, add the partial
+    // gradient of the upper stages, stage as bf16 into `dst` (NSUB swizzled sub-tiles).
+    auto drain = [&](uint32_t tm_col, bool have, float scale, const float *carry, uint8_t *dst) {
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl) {
+            const int c0 = hf * (D / 2) + 32 * sl;
+            uint32_t r[32];
+            if (have) {
+                tmem_ld32(tmem + tm_col + lane_base + c0, r);
+                tmem_wait_ld();
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
+            }
+            uint32_t pk[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                float x0 = __uint_as_float(r[j]) * scale, x1 = __uint_as_float(r[j + 1]) * scale;
+                if (carry != nullptr) {
+                    const float2 c = *reinterpret_cast<const float2 *>(carry + c0 + j);
+                    x0 += c.x;
+                    x1 += c.y;
+                }
+                pk[j >> 1] = pack_bf16(x0, x1);
+            }
+            uint8_t *d = dst + (c0 >> 6) * SUB;
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4 *>(d + swz(rl, ((c0 & 63) >> 3) + c)) =
+                    make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+        }
+    };
+    auto copy_out = [&](const uint8_t *src, void *dst_g) {
+        __nv_bfloat16 *g = reinterpret_cast<__nv_bfloat16 *>(dst_g);
+        for (int idx = tid; idx < NSUB * 128 * 8; idx += 256) {
+            const int t = idx >> 10, rem = idx & 1023, r = rem >> 3, c = rem & 7;
+            if (r < nrows) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(src + t * SUB + swz(r, c));
+                *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + r) * H + h) * D + t * 64 + c * 8) = v;
+            }
+        }
+    };
+
+    const bool run = !empty && !dead;
+    const int row = r0 + rl;
+    const bool inb = row < r1;
+    const float *cq = nullptr, *ck = nullptr, *cv = nullptr;
+    if (inb && a.carry_dq != nullptr) {
+        const int u = a.up[row];
+        if (u >= 0) {
+            cq = a.carry_dq + ((size_t)u * H + h) * D;
+            ck = a.carry_dk + ((size_t)u * H + h) * D;
+            cv = a.carry_dv + ((size_t)u * H + h) * D;
+        }
+    }
+
+    if (run && self && FUSE) {
+        load(true, r0, true, r0);
+        tile_pass(r0, r1, r0, r1, true, true, false, false);
+        if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+        drain(TM_DQ, true, a.scale, cq, sP);
+        drain(TM_DK, true, a.scale, ck, sDS);
+        drain(TM_DV, true, 1.f, cv, sQ);
+    } else {
+        if (run) {
+            // this block as query rows: dQ over the key span
+            load(true, r0, false, 0);
+            for (int c0 = ka; c0 < kb; c0 += 128) {
+                load(false, 0, true, c0);
+                tile_pass(r0, r1, c0, kb, true, false, c0 > ka, false);
+            }
+        }
+        drain(TM_DQ, run, a.scale, cq, sP);
+        // dQ leaves now: the second walk reuses sP and (at D = 128) the dQ columns of TMEM
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        copy_out(sP, a.dq);
+        __syncthreads();
+        if (run) {
+            // this block as keys: dK, dV over the same span taken as query rows
+            load(false, 0, true, r0);
+            for (int c0 = ka; c0 < kb; c0 += 128) {
+                load(true, c0, false, 0);
+                tile_pass(c0, kb, r0, r1, false, true, false, c0 > ka);
+            }
+            if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+        }
+        drain(TM_DK, run, a.scale, ck, sDS);
+        drain(TM_DV, run, 1.f, cv, sQ);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (run && self && FUSE) copy_out(sP, a.dq);   // same decision in every thread
+    copy_out(sDS, a.dk);
+    copy_out(sQ, a.dv);
+    if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
+template <int D>
+static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
+    CUtensorMap tq, tk, tv, tdo;
+    int rc = make_tmap_bf16(&tq, a.q, D, a.H, a.T, 128);
+    if (rc) return rc;
+    rc = make_tmap_bf16(&tk, a.k, D, a.H, a.T, 128);
+    if (rc) return rc;
+    rc = make_tmap_bf16(&tv, a.v, D, a.H, a.T, 128);
+    if (rc) return rc;
+    rc = make_tmap_bf16(&tdo, a.d_o, D, a.H, a.T, 128);
+    if (rc) return rc;
+    constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64;
+    static bool attr = false;
+    if (!attr) {
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr = true;
+    }
+    dim3 grid(a.nb, a.H);
+    k_bwd_tc<D><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, a);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+
+int launch_bwd_tc(const BwdStageArgs &a, int D, cudaStream_t st) {
+    if (a.nb == 0) return HDT_OK;
+    if (D == 64) return launch_bwd_tc_t<64>(a, st);
+    if (D == 128) return launch_bwd_tc_t<128>(a, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
+}
+
+}  // namespace hdt

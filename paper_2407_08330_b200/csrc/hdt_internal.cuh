@@ -94,11 +94,13 @@ struct BwdStageArgs {
     const float *carry_dq, *carry_dk, *carry_dv;  // [n_up,H,D] from the next stage, or nullptr
     void *dq, *dk, *dv;                           // final dtype [T,H,D] (stage 0)
     float *part_dq, *part_dk, *part_dv;           // [n,H,D] (stages above 0)
+    int *status;                                  // device failure word
 };
 
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 // Tensor-core (TMA + tcgen05) stage-0 kernels for bf16 (hdt_attn_tc.cu).
 int launch_fwd_tc(const FwdStageArgs &a, int head_dim, cudaStream_t st);
+int launch_bwd_tc(const BwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
                  cudaStream_t st);
