@@ -187,6 +187,32 @@ const char *hdt_profile_name(int32_t id);
 int hdt_profile_read(int32_t id, int64_t *launches, double *total_ms, int32_t reset);
 
 /*
+ * Forward pass without a caller workspace (the paper has no counterpart; this is an addition for
+ * embedding the library).  Same inputs, outputs and results as hdt_attn_fwd, but the partial
+ * results of the upper stages are kept in a fixed array inside the library instead of a
+ * workspace.  It is meant for callers that are not allowed to allocate device memory at the point
+ * of the call: code running inside a memory pool that has already handed out all of its budget, a
+ * plug-in whose host owns every allocation, or a latency-critical loop where cudaMalloc (which
+ * synchronises the device) must not appear.  The call itself performs no cudaMalloc, cudaFree or
+ * other allocating call.
+ *  - Limit: hdt_attn_workspace_bytes(index, heads, head_dim, dtype, 0) must not exceed
+ *    hdt_attn_fwd_static_max_bytes() (8 MiB, enough for about 2 000 anchor tokens x 16 heads x
+ *    head_dim 64); larger batches get HDT_ERR_WORKSPACE and a message that says so.  The array
+ *    occupies that much memory on every GPU that loads the library, until the process exits.
+ *  - The first call on each device looks up the array's device address (a CUDA runtime query);
+ *    make that first call outside any stream capture.
+ *  - All calls share the one array.  It keeps whatever the last call left, which is harmless:
+ *    each call overwrites every entry before reading it, so nothing needs clearing.  Two calls
+ *    that overlap on the GPU (different streams, or different threads) race on it and corrupt
+ *    each other's results: serialise them.
+ * The structure arrays and the index still come from hdt_build_index and its workspace.
+ */
+size_t hdt_attn_fwd_static_max_bytes(void);
+int hdt_attn_fwd_static(const hdt_index_t *index, const void *q, const void *k, const void *v, void *o,
+                        float *lse, int32_t heads, int32_t head_dim, int32_t dtype, float softmax_scale,
+                        void *stream);
+
+/*
  * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
  * through the fp32 SIMT kernels instead of the tensor-core kernels (A/B comparisons, tests).
  */

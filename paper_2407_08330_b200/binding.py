@@ -202,6 +202,28 @@ def hdt_attn_bwd(index: HdtIndex, q, k, v, o, lse, d_o, softmax_scale=0.0, dq=No
     return dq, dk, dv
 
 
+def hdt_attn_fwd_static_max_bytes() -> int:
+    lib().hdt_attn_fwd_static_max_bytes.restype = C.c_size_t
+    return int(lib().hdt_attn_fwd_static_max_bytes())
+
+
+def hdt_attn_fwd_static(index: HdtIndex, q, k, v, softmax_scale=0.0, out=None, lse=None):
+    """Forward pass for callers that may not allocate device memory during the call: the scratch
+    for the upper stages' partial results is a fixed array inside the library, so nothing is
+    allocated here as long as `out` and `lse` are passed in.  Raises HdtError (-4) when the batch
+    needs more scratch than hdt_attn_fwd_static_max_bytes().  Calls must not overlap on the GPU."""
+    T, H, d = q.shape
+    assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous() and q.dtype == k.dtype == v.dtype
+    o = torch.empty_like(q) if out is None else out
+    lse = torch.empty((H, T), dtype=torch.float32, device=q.device) if lse is None else lse
+    f = lib().hdt_attn_fwd_static
+    f.restype = C.c_int
+    f.argtypes = [C.c_void_p] * 6 + [C.c_int32, C.c_int32, C.c_int32, C.c_float, C.c_void_p]
+    _check(f(index.handle, _ptr(q), _ptr(k), _ptr(v), _ptr(o), _ptr(lse), H, d, _DTYPES[q.dtype],
+             float(softmax_scale), _stream()))
+    return o, lse
+
+
 def hdt_set_option(name: str, value: int) -> None:
     lib().hdt_set_option.restype = C.c_int
     _check(lib().hdt_set_option(C.c_char_p(name.encode()), C.c_int32(int(value))))

@@ -256,3 +256,78 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     }
     return HDT_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Forward pass for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------------
+// The partial results of the upper stages normally live in a workspace the caller allocates.
+// Here they live in this fixed array, which every GPU that loads the library holds until the
+// process exits.  In host code the name `g_fwd_scratch` is only a handle: the device address
+// comes from cudaGetSymbolAddress, once per device, with that device current.
+#define HDT_FWD_STATIC_SCRATCH_BYTES (8u << 20)
+static __device__ __align__(256) unsigned char g_fwd_scratch[HDT_FWD_STATIC_SCRATCH_BYTES];
+
+static void *g_fwd_scratch_ptr[64];   // device address of g_fwd_scratch, per device ordinal
+static std::mutex g_fwd_scratch_mu;
+
+extern "C" size_t hdt_attn_fwd_static_max_bytes(void) { return (size_t)HDT_FWD_STATIC_SCRATCH_BYTES; }
+
+extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const void *k, const void *v, void *o,
+                                   float *lse, int32_t heads, int32_t head_dim, int32_t dtype,
+                                   float softmax_scale, void *stream) {
+    if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd_static: null index");
+    const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 0);
+    if (L.total > (size_t)HDT_FWD_STATIC_SCRATCH_BYTES)
+        return set_error(HDT_ERR_WORKSPACE,
+                         "hdt_attn_fwd_static: this batch needs %zu bytes of scratch, the built-in array holds %zu; "
+                         "use hdt_attn_fwd with a caller workspace",
+                         L.total, (size_t)HDT_FWD_STATIC_SCRATCH_BYTES);
+    int dev = -1;
+    HDT_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return set_error(HDT_ERR_UNSUPPORTED, "hdt_attn_fwd_static: device ordinal %d", dev);
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_fwd_scratch_mu);
+        if (!g_fwd_scratch_ptr[dev]) {   // first call on this device: resolve the array's device address
+            void *p = nullptr;
+            HDT_CUDA_CHECK(cudaGetSymbolAddress(&p, g_fwd_scratch));
+            g_fwd_scratch_ptr[dev] = p;
+        }
+        scratch = g_fwd_scratch_ptr[dev];
+    }
+    int rc = check_common(ix, heads, head_dim, dtype, scratch, (size_t)HDT_FWD_STATIC_SCRATCH_BYTES, L.total,
+                          "hdt_attn_fwd_static");
+    if (rc) return rc;
+    if (ix->total_tokens == 0) return HDT_OK;
+    if (!q || !k || !v || !o || !lse)
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd_static: null tensor pointer");
+    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(o))
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd_static: tensors must be 16-byte aligned");
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = (char *)scratch;
+    int *status = device_status_ptr();
+    if (!status) return HDT_ERR_CUDA;
+    // Every partial result a stage reads was written by the stage above it in this same call, so
+    // nothing in the array has to start at zero; what the previous call left is overwritten.
+    for (int s = ix->n_stages - 1; s >= 0; --s) {
+        const StagePtrs &P = ix->st[s];
+        FwdStageArgs a{};
+        a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
+        a.tok = s ? P.tok : nullptr;
+        a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
+        a.q = q; a.k = k; a.v = v;
+        a.scale_log2 = scale * 1.4426950408889634f;
+        if (s + 1 < ix->n_stages) {
+            a.carry_o = (const float *)(ws + L.part[s + 1][0]);
+            a.carry_lse = (const float *)(ws + L.part[s + 1][1]);
+        }
+        if (s == 0) { a.o = o; a.lse = lse; }
+        else { a.part_o = (float *)(ws + L.part[s][0]); a.part_lse = (float *)(ws + L.part[s][1]); }
+        a.status = status;
+        if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
+        else rc = launch_fwd_simt(a, head_dim, dtype, st);
+        if (rc) return rc;
+    }
+    return HDT_OK;
+}
