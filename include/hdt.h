@@ -90,6 +90,9 @@ typedef struct {
     const int32_t *scu;      /* [batch+1] sequence offsets in this array                      */
     const int32_t *blocks;   /* [n_blocks,5] r0, r1, a, b, flags (HDT_BLK_*)                  */
     const int32_t *queue;    /* [n_blocks] block ids, cost (r1-r0)*(b-a) descending, id asc.  */
+    const int32_t *queue_split; /* [n_blocks] the same order inside two groups: first the n_fused
+                                blocks that are SELF and not EMPTY, then all others             */
+    int32_t n_fused;
 } hdt_stage_view_t;
 
 #define HDT_BLK_SELF 1  /* key span inside the row block                                      */

@@ -34,6 +34,8 @@ Per stage s the index holds, for the compacted array A_s of n_s elements:
                       bit2 CARRY some row has up>=0 (a partial result comes from stage s+1)
                       bit3 EMPTY no row has a key in this stage
   queue         block ids sorted by cost (r1-r0)*(b-a) descending, ties by id ascending
+  queue_split   the same ids: first the n_fused blocks that are SELF and not EMPTY, then the others,
+                each group in queue order
 Totals: nnz = sum over stages and rows of hi-lo (= number of unmasked pairs of the batch),
 visited = sum over blocks of (r1-r0)*(b-a).
 """
@@ -59,6 +61,8 @@ class Stage:
     scu: np.ndarray      # int32 [B+1]
     blocks: np.ndarray   # int32 [nb,5]
     queue: np.ndarray    # int32 [nb]
+    queue_split: np.ndarray = None   # int32 [nb]: SELF non-EMPTY blocks first, each group in queue order
+    n_fused: int = 0
 
 
 @dataclass
@@ -222,7 +226,10 @@ def build(level, parent, cu, block_m: int = 128, max_stages: int = 32) -> Index:
         cost = (blocks[:, 1] - blocks[:, 0]).astype(np.int64) * (blocks[:, 3] - blocks[:, 2]).astype(np.int64)
         queue = np.asarray(sorted(range(len(blocks)), key=lambda i: (-int(cost[i]), i)), np.int32)
 
-        stages.append(Stage(n, tok.copy(), par.copy(), rng, up, scu.copy(), blocks, queue))
+        elig = [bool(f & F_SELF) and not (f & F_EMPTY) for f in blocks[:, 4]] if len(blocks) else []
+        queue_split = np.asarray([i for i in queue if elig[i]] + [i for i in queue if not elig[i]], np.int32)
+        stages.append(Stage(n, tok.copy(), par.copy(), rng, up, scu.copy(), blocks, queue, queue_split,
+                            int(sum(elig))))
 
         if not has_next:
             break

@@ -29,7 +29,8 @@ class _Params(C.Structure):
 
 class _StageView(C.Structure):
     _fields_ = [("n", C.c_int32), ("n_blocks", C.c_int32)] + \
-               [(nm, C.c_void_p) for nm in ("tok", "par", "rng", "up", "scu", "blocks", "queue")]
+               [(nm, C.c_void_p) for nm in ("tok", "par", "rng", "up", "scu", "blocks", "queue", "queue_split")] + \
+               [("n_fused", C.c_int32)]
 
 
 def lib():
@@ -130,7 +131,8 @@ class HdtIndex:
         B = self.batch
         return dict(n=v.n, n_blocks=v.n_blocks, tok=arr(v.tok, v.n), par=arr(v.par, v.n),
                     rng=arr(v.rng, 2 * v.n).reshape(-1, 2), up=arr(v.up, v.n), scu=arr(v.scu, B + 1),
-                    blocks=arr(v.blocks, 5 * v.n_blocks).reshape(-1, 5), queue=arr(v.queue, v.n_blocks))
+                    blocks=arr(v.blocks, 5 * v.n_blocks).reshape(-1, 5), queue=arr(v.queue, v.n_blocks),
+                    queue_split=arr(v.queue_split, v.n_blocks), n_fused=int(v.n_fused))
 
     def close(self):
         if self._h is not None:

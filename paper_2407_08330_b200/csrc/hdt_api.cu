@@ -101,9 +101,11 @@ static bool misaligned(const void *p) { return ((uintptr_t)p & 15) != 0; }
 using namespace hdt;
 
 static int g_force_simt = 0;
+static int g_no_persistent = 0;
 
 extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "force_simt") == 0) { g_force_simt = value; return HDT_OK; }
+    if (name && std::strcmp(name, "no_persistent") == 0) { g_no_persistent = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 
@@ -182,6 +184,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
         a.tok = s ? P.tok : nullptr;
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
+        a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
         a.q = q; a.k = k; a.v = v;
         a.scale_log2 = scale * 1.4426950408889634f;
         if (s + 1 < ix->n_stages) {
@@ -232,6 +235,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
         a.tok = s ? P.tok : nullptr;
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
+        a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
         a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = delta;
         a.scale = scale;
         a.scale_log2 = scale * 1.4426950408889634f;
@@ -247,6 +251,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             a.part_dv = (float *)(ws + L.part[s][2]);
         }
         a.status = status;
+        a.no_persistent = g_no_persistent;
         {
             ProfScope ps(s == 0 ? PROF_BWD_STAGE0 : PROF_BWD_UPPER, st);
             if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
@@ -316,6 +321,7 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
         a.tok = s ? P.tok : nullptr;
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
+        a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
         a.q = q; a.k = k; a.v = v;
         a.scale_log2 = scale * 1.4426950408889634f;
         if (s + 1 < ix->n_stages) {

@@ -26,15 +26,6 @@ static constexpr long long WAIT_CYCLES = 400000000LL;
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
 template <int D>
-struct BwdSmem {
-    static constexpr int NSUB = D / 64;
-    uint8_t *sQ, *sDO, *sK, *sV, *sP, *sDS;
-    uint64_t *bar_tma, *bar_mma;
-    uint32_t *slot;
-    volatile int *abort_flag;
-};
-
-template <int D>
 __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensorMap tm_q,
                                                 const __grid_constant__ CUtensorMap tm_k,
                                                 const __grid_constant__ CUtensorMap tm_v,
@@ -54,7 +45,9 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     volatile int *abort_flag = (volatile int *)(slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, hf = tid >> 7;
-    const int blk = a.queue[blockIdx.x], h = blockIdx.y, H = a.H;
+    // rest_only: take the blocks after the first n_fused entries of queue_split
+    const int blk = a.rest_only ? a.queue_split[a.n_fused + blockIdx.x] : a.queue[blockIdx.x];
+    const int h = blockIdx.y, H = a.H;
     const int *rec = a.blocks + 5 * (size_t)blk;
     const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3], fl = rec[4];
     const int nrows = r1 - r0;
@@ -306,6 +299,248 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Persistent, software-pipelined backward for blocks that are SELF and not EMPTY at D = 64.
+// One CTA of 512 threads per SM walks its share of the (block, head) items (queue_split order,
+// longest first, round-robin over CTAs).  Inputs are double-buffered: while item i is computed
+// the TMA loads of item i+1 are in flight or done and those of item i+2 start as soon as item i's
+// output MMAs have finished.  S/dP of item i+1 are issued together with the output MMAs of item i,
+// so they run while the CTA drains dQ/dK/dV of item i.
+// Thread t: row t % 128 (TMEM lane), column quarter t / 128.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUtensorMap tm_q,
+                                                     const __grid_constant__ CUtensorMap tm_k,
+                                                     const __grid_constant__ CUtensorMap tm_v,
+                                                     const __grid_constant__ CUtensorMap tm_do, const BwdStageArgs a) {
+    constexpr int D = 64;
+    constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_DK = 320, TM_DV = 384, TM_COLS = 512;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sIn = sm;                    // 2 stages x {Q, dO, K, V}
+    uint8_t *sP = sm + 8 * SUB;           // 2 sub-tiles; later staging of dQ (sub-tile 0), dK (sub-tile 1)
+    uint8_t *sDS = sP + 2 * SUB;          // 2 sub-tiles; later staging of dV (sub-tile 0)
+    uint64_t *bar_tma = (uint64_t *)(sDS + 2 * SUB);   // [2]
+    uint64_t *bar_a = bar_tma + 2, *bar_b = bar_tma + 3;
+    uint32_t *slot = (uint32_t *)(bar_tma + 4);
+    volatile int *abort_flag = (volatile int *)(slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, qt = tid >> 7;
+    const int H = a.H, G = gridDim.x;
+    const int n_items = a.n_fused * H;
+    const int my_count = ((int)blockIdx.x < n_items) ? (n_items - (int)blockIdx.x + G - 1) / G : 0;
+    const float LOG2E = 1.4426950408889634f;
+
+    if (tid == 0) {
+        mbar_init(&bar_tma[0], 1);
+        mbar_init(&bar_tma[1], 1);
+        mbar_init(bar_a, 1);
+        mbar_init(bar_b, 1);
+        *abort_flag = (*a.status != 0);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    bool ok = true;
+
+    auto item_of = [&](int i, int &blk, int &h) {
+        const int item = (int)blockIdx.x + i * G;
+        blk = a.queue_split[item / H];
+        h = item % H;
+    };
+    auto issue_tma = [&](int i) {       // thread 0
+        int blk, h;
+        item_of(i, blk, h);
+        const int r0 = a.blocks[5 * (size_t)blk];
+        uint8_t *st = sIn + (i & 1) * 4 * SUB;
+        uint64_t *bar = &bar_tma[i & 1];
+        mbar_expect_tx(bar, 4 * SUB);
+        tma_load_3d(st, &tm_q, 0, h, r0, bar);
+        tma_load_3d(st + SUB, &tm_do, 0, h, r0, bar);
+        tma_load_3d(st + 2 * SUB, &tm_k, 0, h, r0, bar);
+        tma_load_3d(st + 3 * SUB, &tm_v, 0, h, r0, bar);
+    };
+    auto issue_sdp = [&](int i, int Nc) {   // thread 0, inputs of item i have landed
+        const uint32_t st = smem_u32(sIn + (i & 1) * 4 * SUB);
+        const uint32_t idesc = idesc_bf16(Nc, false, false);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss(tmem + TM_S, smem_desc(st + kk * 32, 0, 1024), smem_desc(st + 2 * SUB + kk * 32, 0, 1024), idesc, kk > 0);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss(tmem + TM_DP, smem_desc(st + SUB + kk * 32, 0, 1024), smem_desc(st + 3 * SUB + kk * 32, 0, 1024), idesc,
+                   kk > 0);
+        mma_commit(bar_a);
+    };
+    auto rows16 = [&](int blk) {
+        const int n = a.blocks[5 * (size_t)blk + 1] - a.blocks[5 * (size_t)blk];
+        return (n + 15) & ~15;
+    };
+
+    if (!dead && my_count > 0) {
+        if (tid == 0) {
+            issue_tma(0);
+            if (my_count > 1) issue_tma(1);
+            ok = mbar_wait(&bar_tma[0], 0, abort_flag, WAIT_CYCLES) && ok;
+            if (!*abort_flag) {
+                int blk, h;
+                item_of(0, blk, h);
+                tc_fence_after();
+                issue_sdp(0, rows16(blk));
+            }
+        }
+        for (int it = 0; it < my_count; ++it) {
+            int blk, h;
+            item_of(it, blk, h);
+            const int *rec = a.blocks + 5 * (size_t)blk;
+            const int r0 = rec[0], r1 = rec[1];
+            const int nrows = r1 - r0, Nc = (nrows + 15) & ~15;
+            const int row = r0 + rl;
+            const bool inb = row < r1;
+            int lo = 0, hi = 0;
+            float lse2 = 0.f, dl = 0.f;
+            const float *cq = nullptr, *ck = nullptr, *cv = nullptr;
+            if (inb) {
+                lo = a.rng[2 * row];
+                hi = a.rng[2 * row + 1];
+                if (hi > lo) {
+                    lse2 = a.lse[(size_t)h * a.T + row] * LOG2E;
+                    dl = a.delta[(size_t)h * a.T + row];
+                }
+                if (a.carry_dq != nullptr) {
+                    const int u = a.up[row];
+                    if (u >= 0) {
+                        cq = a.carry_dq + ((size_t)u * H + h) * D;
+                        ck = a.carry_dk + ((size_t)u * H + h) * D;
+                        cv = a.carry_dv + ((size_t)u * H + h) * D;
+                    }
+                }
+            }
+            const int jl = max(lo - r0, 0), jh = min(hi - r0, nrows);
+            const bool has = inb && jh > jl;
+            uint8_t *st = sIn + (it & 1) * 4 * SUB;
+
+            ok = mbar_wait(bar_a, it & 1, abort_flag, WAIT_CYCLES) && ok;   // S, dP of this item
+            tc_fence_after();
+            // ---- P and dS of this thread's 32 columns, in two halves of 16 ----
+            if (32 * qt < Nc) {
+#pragma unroll
+                for (int hh = 0; hh < 2; ++hh) {
+                    const int s0 = 32 * qt + 16 * hh;
+                    const bool mine = has && jl < s0 + 16 && jh > s0;
+                    uint32_t pp[8], pd[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { pp[j] = 0u; pd[j] = 0u; }
+                    if (__any_sync(0xffffffffu, mine)) {
+                        uint32_t rs[16], rd[16];
+                        tmem_ld16(tmem + TM_S + lane_base + s0, rs);
+                        tmem_ld16(tmem + TM_DP + lane_base + s0, rd);
+                        tmem_wait_ld();
+                        if (mine) {
+#pragma unroll
+                            for (int j = 0; j < 16; j += 2) {
+                                float p0 = 0.f, p1 = 0.f, d0 = 0.f, d1 = 0.f;
+                                if (s0 + j >= jl && s0 + j < jh) {
+                                    p0 = exp2f(fmaf(__uint_as_float(rs[j]), a.scale_log2, -lse2));
+                                    d0 = p0 * (__uint_as_float(rd[j]) - dl);
+                                }
+                                if (s0 + j + 1 >= jl && s0 + j + 1 < jh) {
+                                    p1 = exp2f(fmaf(__uint_as_float(rs[j + 1]), a.scale_log2, -lse2));
+                                    d1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
+                                }
+                                pp[j >> 1] = pack_bf16(p0, p1);
+                                pd[j >> 1] = pack_bf16(d0, d1);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int c = 0; c < 2; ++c) {
+                        const uint32_t off = (qt >> 1) * SUB + swz(rl, (qt & 1) * 4 + hh * 2 + c);
+                        *reinterpret_cast<uint4 *>(sP + off) = make_uint4(pp[4 * c], pp[4 * c + 1], pp[4 * c + 2], pp[4 * c + 3]);
+                        *reinterpret_cast<uint4 *>(sDS + off) = make_uint4(pd[4 * c], pd[4 * c + 1], pd[4 * c + 2], pd[4 * c + 3]);
+                    }
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0 && !*abort_flag) {
+                tc_fence_after();
+                const uint32_t sb = smem_u32(st);
+                const uint32_t idesc_kv = idesc_bf16(D, true, true), idesc_q = idesc_bf16(D, false, true);
+                for (int kk = 0; kk < Nc / 16; ++kk)   // dV = P^T dO
+                    mma_ss(tmem + TM_DV, smem_desc(smem_u32(sP) + kk * 2048, SUB, 1024),
+                           smem_desc(sb + SUB + kk * 2048, SUB, 1024), idesc_kv, kk > 0);
+                for (int kk = 0; kk < Nc / 16; ++kk)   // dK = dS^T Q
+                    mma_ss(tmem + TM_DK, smem_desc(smem_u32(sDS) + kk * 2048, SUB, 1024),
+                           smem_desc(sb + kk * 2048, SUB, 1024), idesc_kv, kk > 0);
+                for (int kk = 0; kk < Nc / 16; ++kk)   // dQ = dS K
+                    mma_ss(tmem + TM_DQ, smem_desc(smem_u32(sDS) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024),
+                           smem_desc(sb + 2 * SUB + kk * 2048, SUB, 1024), idesc_q, kk > 0);
+                mma_commit(bar_b);
+                if (it + 1 < my_count) {               // S, dP of the next item run during this item's drain
+                    ok = mbar_wait(&bar_tma[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag, WAIT_CYCLES) && ok;
+                    if (!*abort_flag) {
+                        int blk2, h2;
+                        item_of(it + 1, blk2, h2);
+                        tc_fence_after();
+                        issue_sdp(it + 1, rows16(blk2));
+                    }
+                }
+            }
+            ok = mbar_wait(bar_b, it & 1, abort_flag, WAIT_CYCLES) && ok;   // dQ, dK, dV of this item
+            tc_fence_after();
+            if (tid == 0 && it + 2 < my_count && !*abort_flag) issue_tma(it + 2);   // this stage is free again
+            // ---- drain: 16 columns of each gradient per thread, staged as bf16 ----
+#pragma unroll
+            for (int t = 0; t < 3; ++t) {
+                const uint32_t col = (t == 0) ? TM_DQ : (t == 1) ? TM_DK : TM_DV;
+                const float sc = (t == 2) ? 1.f : a.scale;
+                const float *cy = (t == 0) ? cq : (t == 1) ? ck : cv;
+                uint8_t *dst = (t == 0) ? sP : (t == 1) ? (sP + SUB) : sDS;
+                uint32_t r[16];
+                tmem_ld16(tmem + col + lane_base + 16 * qt, r);
+                tmem_wait_ld();
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 16; j += 2) {
+                    float x0 = __uint_as_float(r[j]) * sc, x1 = __uint_as_float(r[j + 1]) * sc;
+                    if (cy != nullptr) {
+                        const float2 c = *reinterpret_cast<const float2 *>(cy + 16 * qt + j);
+                        x0 += c.x;
+                        x1 += c.y;
+                    }
+                    pk[j >> 1] = pack_bf16(x0, x1);
+                }
+                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
+            tc_fence_before();
+            __syncthreads();
+            // ---- coalesced stores: 3 tensors x 128 rows x 8 chunks ----
+            for (int idx = tid; idx < 3 * 1024; idx += 512) {
+                const int t = idx >> 10, rem = idx & 1023, r = rem >> 3, c = rem & 7;
+                if (r < nrows) {
+                    const uint8_t *src = (t == 0) ? sP : (t == 1) ? (sP + SUB) : sDS;
+                    __nv_bfloat16 *g = reinterpret_cast<__nv_bfloat16 *>((t == 0) ? a.dq : (t == 1) ? a.dk : a.dv);
+                    const uint4 v = *reinterpret_cast<const uint4 *>(src + swz(r, c));
+                    *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + r) * H + h) * D + c * 8) = v;
+                }
+            }
+            __syncthreads();   // staging is read out before the next item's P / dS are written
+        }
+    }
+    if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
 template <int D>
 static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     CUtensorMap tq, tk, tv, tdo;
@@ -323,10 +558,34 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attr = true;
     }
-    dim3 grid(a.nb, a.H);
-    k_bwd_tc<D><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, a);
-    count_launch();
-    HDT_CUDA_CHECK(cudaGetLastError());
+    BwdStageArgs b = a;
+    b.rest_only = 0;
+    int n_general = a.nb;
+    if (D == 64 && a.n_fused > 0 && !a.no_persistent) {
+        constexpr int smem_p = 12 * SUB + 1024 + 64;
+        static bool attr_p = false;
+        static int n_sm = 0;
+        if (!attr_p) {
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            int dev = 0;
+            HDT_CUDA_CHECK(cudaGetDevice(&dev));
+            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+            attr_p = true;
+        }
+        const long long items = (long long)a.n_fused * a.H;
+        const int grid_p = (int)(items < n_sm ? items : n_sm);
+        k_bwd_tc_p<<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, a);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+        b.rest_only = 1;
+        n_general = a.nb - a.n_fused;
+    }
+    if (n_general > 0) {
+        dim3 grid(n_general, a.H);
+        k_bwd_tc<D><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, b);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+    }
     return HDT_OK;
 }
 

@@ -20,7 +20,7 @@ static constexpr int CHUNK = 1024;  // elements per CTA in the element-wise kern
 
 struct Layout {
     size_t header, cnt, nlc, pre, keep, fpos, blocksum, bstart, seqcount, cost, stage0, stage_stride;
-    size_t s_tok, s_par, s_rng, s_up, s_scu, s_blocks, s_queue;  // offsets inside a stage
+    size_t s_tok, s_par, s_rng, s_up, s_scu, s_blocks, s_queue, s_queue2;  // offsets inside a stage
     size_t total;
     int capnb, nchunk;
 };
@@ -51,6 +51,7 @@ static Layout make_layout(int B, int T, int bm, int max_stages) {
     L.s_scu = s; s += al(sizeof(int) * (size_t)(B + 1));
     L.s_blocks = s; s += al(sizeof(int) * 5 * (size_t)L.capnb);
     L.s_queue = s; s += al(sizeof(int) * (size_t)L.capnb);
+    L.s_queue2 = s; s += al(sizeof(int) * (size_t)L.capnb);
     L.stage_stride = s;
     L.total = o + s * (size_t)max_stages;
     return L;
@@ -386,18 +387,30 @@ __global__ void k_blocks(DevHeader *hdr, int s, int bm, int B, const int *__rest
     if (lane == 0 && vis) atomicAdd((unsigned long long *)&hdr->visited, (unsigned long long)vis);
 }
 
-// Rank sort: queue[rank] = block id, cost descending, id ascending.
-__global__ void k_queue(const DevHeader *hdr, int s, const long long *__restrict__ cost, int *queue) {
+// Rank sort: queue[rank] = block id, cost descending, id ascending.  queue_split: the same order
+// inside two groups, blocks that are SELF and not EMPTY first (n_fused of them), then the others.
+__global__ void k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost,
+                        const int *__restrict__ blocks, int *queue, int *queue_split) {
     const int nb = hdr->st[s].nb;
+    int mine = 0;
     for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nb; i += gridDim.x * blockDim.x) {
         const long long ci = cost[i];
-        int rank = 0;
+        const int fi = blocks[5 * i + 4];
+        const int ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
+        int rank = 0, rank2 = 0;
         for (int j = 0; j < nb; ++j) {
             const long long cj = cost[j];
-            rank += (cj > ci) || (cj == ci && j < i);
+            const int fj = blocks[5 * j + 4];
+            const int ej = ((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0;
+            const int before = (cj > ci) || (cj == ci && j < i);
+            rank += before;
+            rank2 += (ej > ei) || (ej == ei && before);
         }
         queue[rank] = i;
+        queue_split[rank2] = i;
+        mine += ei;
     }
+    if (mine) atomicAdd(&hdr->st[s].n_fused, mine);
 }
 
 }  // namespace hdt
@@ -452,7 +465,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         char *base = ws + L.stage0 + L.stage_stride * (size_t)s;
         ix->st[s] = StagePtrs{(int *)(base + L.s_tok), (int *)(base + L.s_par), (int *)(base + L.s_rng),
                               (int *)(base + L.s_up), (int *)(base + L.s_scu), (int *)(base + L.s_blocks),
-                              (int *)(base + L.s_queue)};
+                              (int *)(base + L.s_queue), (int *)(base + L.s_queue2)};
     }
 #define HDT_BUILD_CHECK(expr)                                                          \
     do {                                                                               \
@@ -499,7 +512,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             int maxlen_smem = kSmemCap;  // sequences longer than this walk through global memory
             k_walk<<<B, 256, kSmemCap, st>>>(hdr, s, bm, P.scu, fpos, bstart, seqcount, maxlen_smem);
             k_blocks<<<B, 256, 0, st>>>(hdr, s, bm, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost);
-            k_queue<<<max(1, min(L.capnb / 128 + 1, 148 * 4)), 128, 0, st>>>(hdr, s, cost, P.queue);
+            k_queue<<<max(1, min(L.capnb / 128 + 1, 148 * 4)), 128, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
             count_launch(3);
         }
         count_launch(4);
@@ -548,6 +561,8 @@ extern "C" int hdt_index_export(const hdt_index_t *ix, int32_t stage, hdt_stage_
     v->n_blocks = ix->desc[stage].nb;
     v->tok = P.tok; v->par = P.par; v->rng = P.rng; v->up = P.up; v->scu = P.scu;
     v->blocks = P.blocks; v->queue = P.queue;
+    v->queue_split = P.queue_split;
+    v->n_fused = ix->desc[stage].n_fused;
     return HDT_OK;
 }
 

@@ -13,7 +13,7 @@ struct StageDesc {
     int n;         // elements of the stage array
     int nb;        // row blocks
     int has_next;  // a later stage exists
-    int pad;
+    int n_fused;   // blocks that are SELF and not EMPTY (first n_fused entries of queue_split)
 };
 
 struct DevHeader {
@@ -26,7 +26,7 @@ struct DevHeader {
 
 // Host-side pointers to one stage's arrays inside the workspace.
 struct StagePtrs {
-    int *tok, *par, *rng, *up, *scu, *blocks, *queue;
+    int *tok, *par, *rng, *up, *scu, *blocks, *queue, *queue_split;
 };
 
 }  // namespace hdt
@@ -70,6 +70,8 @@ struct FwdStageArgs {
     int n, nb, H;
     const int *tok;     // nullptr: identity (stage 0)
     const int *rng, *up, *blocks, *queue;
+    const int *queue_split;  // SELF non-EMPTY blocks first (n_fused of them), then the rest
+    int n_fused;
     const void *q, *k, *v;
     float scale_log2;   // softmax_scale * log2(e)
     // partial results of the next stage (nullptr if none): [n_up, H, D] and [n_up, H]
@@ -81,12 +83,16 @@ struct FwdStageArgs {
     // ... or this stage's partial results
     float *part_o, *part_lse;
     int *status;        // device failure word
+    int rest_only;      // general kernel: only blocks after the first n_fused
+    int no_persistent;  // option: do not use the persistent kernels
 };
 
 struct BwdStageArgs {
     int n, nb, H, T;
     const int *tok;
     const int *rng, *up, *blocks, *queue;
+    const int *queue_split;
+    int n_fused;
     const void *q, *k, *v, *d_o;
     const float *lse;    // [H,T] final
     const float *delta;  // [H,T]
@@ -95,6 +101,8 @@ struct BwdStageArgs {
     void *dq, *dk, *dv;                           // final dtype [T,H,D] (stage 0)
     float *part_dq, *part_dk, *part_dv;           // [n,H,D] (stages above 0)
     int *status;                                  // device failure word
+    int rest_only;                                // general kernel: only blocks after the first n_fused
+    int no_persistent;                            // option: do not use the persistent kernels
 };
 
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);

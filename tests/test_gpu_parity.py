@@ -27,8 +27,9 @@ def assert_index_equal(P, b, block_m=128, max_stages=8):
     for s, st in enumerate(want.stages):
         got = idx.export(s)
         assert got["n"] == st.n and got["n_blocks"] == len(st.blocks), s
-        for name in ("tok", "par", "rng", "up", "scu", "blocks", "queue"):
+        for name in ("tok", "par", "rng", "up", "scu", "blocks", "queue", "queue_split"):
             assert np.array_equal(got[name], getattr(st, name)), (s, name)
+        assert got["n_fused"] == st.n_fused
     return idx
 
 
@@ -100,13 +101,17 @@ def test_index_rejects_bad_hierarchies(P):
 # attention, small cases compared element by element
 # ------------------------------------------------------------------------------------------
 def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
-    """bf16 runs twice: tensor-core stage-0 kernels, then the SIMT kernels on every stage."""
-    for force_simt in ((0, 1) if dtype == "bf16" else (0,)):
-        P.hdt_set_option("force_simt", force_simt)
+    """bf16 runs three times: persistent + general tensor-core kernels, general tensor-core kernels
+    only, SIMT kernels on every stage."""
+    opts = ({}, {"no_persistent": 1}, {"force_simt": 1}) if dtype == "bf16" else ({},)
+    for opt in opts:
+        for k_, v_ in opt.items():
+            P.hdt_set_option(k_, v_)
         try:
             _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale)
         finally:
-            P.hdt_set_option("force_simt", 0)
+            for k_ in opt:
+                P.hdt_set_option(k_, 0)
 
 
 def _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale):

@@ -49,6 +49,11 @@ def check_structure(b, idx, block_m):
         assert sorted(q.tolist()) == list(range(len(st.blocks)))
         for x, y in zip(q[:-1], q[1:]):
             assert (cost[x], -x) >= (cost[y], -y)
+        elig = [(f & ix.F_SELF) and not (f & ix.F_EMPTY) for f in st.blocks[:, 4]]
+        assert st.n_fused == sum(bool(x) for x in elig)
+        assert all(elig[i] for i in st.queue_split[:st.n_fused])
+        assert not any(elig[i] for i in st.queue_split[st.n_fused:])
+        assert sorted(st.queue_split.tolist()) == list(range(len(st.blocks)))
         # up / tok maps
         if si + 1 < len(idx.stages):
             nx = idx.stages[si + 1]
