@@ -239,6 +239,15 @@ int hdt_device_status(void *stream);
 int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
                    void *stream);
 
+/*
+ * Diagnostics (no counterpart in the paper): SM clock cycles that CTA 0 of the persistent backward
+ * kernel spent in each of its phases since the last call (out16[0..11]: prefetch issue, wait for
+ * S/dP, P/dS arithmetic, barrier, rest of the MMA issue, wait for dQ/dK/dV, drain, barrier, stores,
+ * loop end, issue of the output MMAs, wait for the next item's TMA), out16[12] = items processed.
+ * Synchronises the device and resets the counters.
+ */
+int hdt_debug_bwd_phase_cycles(int64_t *out16);
+
 #ifdef __cplusplus
 }
 #endif

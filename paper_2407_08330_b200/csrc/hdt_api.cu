@@ -178,7 +178,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
     char *ws = (char *)workspace;
     int *status = device_status_ptr();
     if (!status) return HDT_ERR_CUDA;
-    for (int s = ix->n_stages - 1; s >= 0; --s) {
+    for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
         const StagePtrs &P = ix->st[s];
         FwdStageArgs a{};
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
@@ -187,12 +187,15 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
         a.q = q; a.k = k; a.v = v;
         a.scale_log2 = scale * 1.4426950408889634f;
-        if (s + 1 < ix->n_stages) {
-            a.carry_o = (const float *)(ws + L.part[s + 1][0]);
-            a.carry_lse = (const float *)(ws + L.part[s + 1][1]);
+        if (s > 0) {   // partial results the stages below left for this stage's elements
+            a.carry_o = (const float *)(ws + L.part[s][0]);
+            a.carry_lse = (const float *)(ws + L.part[s][1]);
         }
-        if (s == 0) { a.o = o; a.lse = lse; }
-        else { a.part_o = (float *)(ws + L.part[s][0]); a.part_lse = (float *)(ws + L.part[s][1]); }
+        if (s + 1 < ix->n_stages) {   // where this stage leaves its own for the next one
+            a.part_o = (float *)(ws + L.part[s + 1][0]);
+            a.part_lse = (float *)(ws + L.part[s + 1][1]);
+        }
+        a.o = o; a.lse = lse;
         a.status = status;
         {
             ProfScope ps(s == 0 ? PROF_FWD_STAGE0 : PROF_FWD_UPPER, st);
@@ -229,7 +232,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
     }
     if (rc) return rc;
-    for (int s = ix->n_stages - 1; s >= 0; --s) {
+    for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
         const StagePtrs &P = ix->st[s];
         BwdStageArgs a{};
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
@@ -239,17 +242,17 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = delta;
         a.scale = scale;
         a.scale_log2 = scale * 1.4426950408889634f;
+        if (s > 0) {
+            a.carry_dq = (const float *)(ws + L.part[s][0]);
+            a.carry_dk = (const float *)(ws + L.part[s][1]);
+            a.carry_dv = (const float *)(ws + L.part[s][2]);
+        }
         if (s + 1 < ix->n_stages) {
-            a.carry_dq = (const float *)(ws + L.part[s + 1][0]);
-            a.carry_dk = (const float *)(ws + L.part[s + 1][1]);
-            a.carry_dv = (const float *)(ws + L.part[s + 1][2]);
+            a.part_dq = (float *)(ws + L.part[s + 1][0]);
+            a.part_dk = (float *)(ws + L.part[s + 1][1]);
+            a.part_dv = (float *)(ws + L.part[s + 1][2]);
         }
-        if (s == 0) { a.dq = dq; a.dk = dk; a.dv = dv; }
-        else {
-            a.part_dq = (float *)(ws + L.part[s][0]);
-            a.part_dk = (float *)(ws + L.part[s][1]);
-            a.part_dv = (float *)(ws + L.part[s][2]);
-        }
+        a.dq = dq; a.dk = dk; a.dv = dv;
         a.status = status;
         a.no_persistent = g_no_persistent;
         {
@@ -313,9 +316,9 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
     char *ws = (char *)scratch;
     int *status = device_status_ptr();
     if (!status) return HDT_ERR_CUDA;
-    // Every partial result a stage reads was written by the stage above it in this same call, so
+    // Every partial result a stage reads was written by the stage below it in this same call, so
     // nothing in the array has to start at zero; what the previous call left is overwritten.
-    for (int s = ix->n_stages - 1; s >= 0; --s) {
+    for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
         const StagePtrs &P = ix->st[s];
         FwdStageArgs a{};
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
@@ -324,12 +327,15 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
         a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
         a.q = q; a.k = k; a.v = v;
         a.scale_log2 = scale * 1.4426950408889634f;
-        if (s + 1 < ix->n_stages) {
-            a.carry_o = (const float *)(ws + L.part[s + 1][0]);
-            a.carry_lse = (const float *)(ws + L.part[s + 1][1]);
+        if (s > 0) {   // partial results the stages below left for this stage's elements
+            a.carry_o = (const float *)(ws + L.part[s][0]);
+            a.carry_lse = (const float *)(ws + L.part[s][1]);
         }
-        if (s == 0) { a.o = o; a.lse = lse; }
-        else { a.part_o = (float *)(ws + L.part[s][0]); a.part_lse = (float *)(ws + L.part[s][1]); }
+        if (s + 1 < ix->n_stages) {   // where this stage leaves its own for the next one
+            a.part_o = (float *)(ws + L.part[s + 1][0]);
+            a.part_lse = (float *)(ws + L.part[s + 1][1]);
+        }
+        a.o = o; a.lse = lse;
         a.status = status;
         if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
         else rc = launch_fwd_simt(a, head_dim, dtype, st);

@@ -168,36 +168,35 @@ __global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
             for (int t = 0; t < 4; ++t) scale4(o[t], inv);
             lse = (m + log2f(l)) * 0.6931471805599453f;
         }
-        // merge the partial result of the later stages
+        // merge the partial result the stages below left for this element (same index)
         if (a.carry_o != nullptr) {
-            const int u = a.up[row];
-            if (u >= 0) {
-                const float lc = a.carry_lse[(size_t)u * H + h];
-                if (lc > NEG) {
-                    const float mx = fmaxf(lse, lc);
-                    const float e0 = (lse > NEG) ? __expf(lse - mx) : 0.f, e1 = __expf(lc - mx);
-                    const float tot = e0 + e1;
-                    const float w0 = e0 / tot, w1 = e1 / tot;
-                    const float4 *oc = reinterpret_cast<const float4 *>(a.carry_o + ((size_t)u * H + h) * D);
+            const float lc = a.carry_lse[(size_t)row * H + h];
+            if (lc > NEG) {
+                const float mx = fmaxf(lse, lc);
+                const float e0 = (lse > NEG) ? __expf(lse - mx) : 0.f, e1 = __expf(lc - mx);
+                const float tot = e0 + e1;
+                const float w0 = e0 / tot, w1 = e1 / tot;
+                const float4 *oc = reinterpret_cast<const float4 *>(a.carry_o + ((size_t)row * H + h) * D);
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        scale4(o[t], w0);
-                        axpy4(o[t], w1, oc[g + G * t]);
-                    }
-                    lse = mx + __logf(tot);
+                for (int t = 0; t < 4; ++t) {
+                    scale4(o[t], w0);
+                    axpy4(o[t], w1, oc[g + G * t]);
                 }
+                lse = mx + __logf(tot);
             }
         }
-        if (a.part_o != nullptr) {
-            float4 *po = reinterpret_cast<float4 *>(a.part_o + ((size_t)row * H + h) * D);
+        // hand the merged partial to the next stage if the element lives on there ...
+        const int u = (a.part_o != nullptr) ? a.up[row] : -1;
+        if (u >= 0) {
+            float4 *po = reinterpret_cast<float4 *>(a.part_o + ((size_t)u * H + h) * D);
 #pragma unroll
             for (int t = 0; t < 4; ++t) po[g + G * t] = o[t];
-            if (g == 0) a.part_lse[(size_t)row * H + h] = lse;
-        } else {
-#pragma unroll
-            for (int t = 0; t < 4; ++t) store4<BF16>(a.o, ((size_t)trow * H + h) * D + 4 * (g + G * t), o[t]);
-            if (g == 0) a.lse[(size_t)h * a.T + trow] = lse;
+            if (g == 0) a.part_lse[(size_t)u * H + h] = lse;
         }
+        // ... and write the result so far; a later stage overwrites it with the complete one
+#pragma unroll
+        for (int t = 0; t < 4; ++t) store4<BF16>(a.o, ((size_t)trow * H + h) * D + 4 * (g + G * t), o[t]);
+        if (g == 0) a.lse[(size_t)h * a.T + trow] = lse;
     }
 }
 
@@ -270,18 +269,16 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
             }
         }
         if (inb) {
-            const int u = (a.carry_dq != nullptr) ? a.up[row] : -1;
+            const int u = (a.part_dq != nullptr) ? a.up[row] : -1;
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 scale4(acc[t], a.scale);
-                if (u >= 0) {
-                    const float4 c = reinterpret_cast<const float4 *>(a.carry_dq + ((size_t)u * H + h) * D)[g + G * t];
+                if (a.carry_dq != nullptr) {   // partial gradient from the stages below (same index)
+                    const float4 c = reinterpret_cast<const float4 *>(a.carry_dq + ((size_t)row * H + h) * D)[g + G * t];
                     acc[t].x += c.x; acc[t].y += c.y; acc[t].z += c.z; acc[t].w += c.w;
                 }
-                if (a.part_dq != nullptr)
-                    reinterpret_cast<float4 *>(a.part_dq + ((size_t)row * H + h) * D)[g + G * t] = acc[t];
-                else
-                    store4<BF16>(a.dq, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc[t]);
+                if (u >= 0) reinterpret_cast<float4 *>(a.part_dq + ((size_t)u * H + h) * D)[g + G * t] = acc[t];
+                store4<BF16>(a.dq, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc[t]);
             }
         }
         // ---------------- phase B: this element as a key ----------------
@@ -336,23 +333,22 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
             }
         }
         if (inb) {
-            const int u = (a.carry_dk != nullptr) ? a.up[row] : -1;
+            const int u = (a.part_dk != nullptr) ? a.up[row] : -1;
 #pragma unroll
             for (int t = 0; t < 4; ++t) {
                 scale4(acc[t], a.scale);
-                if (u >= 0) {
-                    const float4 c = reinterpret_cast<const float4 *>(a.carry_dk + ((size_t)u * H + h) * D)[g + G * t];
-                    const float4 c2 = reinterpret_cast<const float4 *>(a.carry_dv + ((size_t)u * H + h) * D)[g + G * t];
+                if (a.carry_dk != nullptr) {
+                    const float4 c = reinterpret_cast<const float4 *>(a.carry_dk + ((size_t)row * H + h) * D)[g + G * t];
+                    const float4 c2 = reinterpret_cast<const float4 *>(a.carry_dv + ((size_t)row * H + h) * D)[g + G * t];
                     acc[t].x += c.x; acc[t].y += c.y; acc[t].z += c.z; acc[t].w += c.w;
                     acc2[t].x += c2.x; acc2[t].y += c2.y; acc2[t].z += c2.z; acc2[t].w += c2.w;
                 }
-                if (a.part_dk != nullptr) {
-                    reinterpret_cast<float4 *>(a.part_dk + ((size_t)row * H + h) * D)[g + G * t] = acc[t];
-                    reinterpret_cast<float4 *>(a.part_dv + ((size_t)row * H + h) * D)[g + G * t] = acc2[t];
-                } else {
-                    store4<BF16>(a.dk, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc[t]);
-                    store4<BF16>(a.dv, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc2[t]);
+                if (u >= 0) {
+                    reinterpret_cast<float4 *>(a.part_dk + ((size_t)u * H + h) * D)[g + G * t] = acc[t];
+                    reinterpret_cast<float4 *>(a.part_dv + ((size_t)u * H + h) * D)[g + G * t] = acc2[t];
                 }
+                store4<BF16>(a.dk, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc[t]);
+                store4<BF16>(a.dv, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc2[t]);
             }
         }
     }

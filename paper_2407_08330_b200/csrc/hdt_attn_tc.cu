@@ -6,7 +6,8 @@
 //   MMA   S = Q K^T                       ->  TMEM columns [0, 128)
 //   rows  tcgen05.ld S, mask columns outside [lo, hi), online softmax, P (bf16) -> shared memory
 //   MMA   O (+)= P V                      ->  TMEM columns [128, 128 + D)
-//   rows  tcgen05.ld O, 1/l, merge the partial result of the upper stages, store O and LSE
+//   rows  tcgen05.ld O, 1/l, store O and LSE; rows that also belong to the next stage leave their
+//         fp32 partial (O, LSE) in its buffer, and that stage writes their final result
 // Blocks are packed from whole families, so nearly every block has a single key chunk equal to
 // its own rows (Q, K, V are the same 128 token rows); long families loop over key chunks with
 // the running maximum and a rescale of O in TMEM.  Two CTAs fit on an SM at D = 64 (80 KB of
@@ -190,23 +191,16 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
     }
     if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
 
-    // ---- epilogue: normalise, merge the upper stages' partial result, stage O, store ----
-    float lse = NEG, w0 = 0.f, w1 = 0.f;
+    // ---- epilogue: normalise; rows that live on in the next stage also leave their fp32 partial
+    // result (O, LSE) there, the next stage completes and overwrites them; stage O, store ----
+    float lse = NEG, w0 = 0.f;
     if (l > 0.f) { w0 = 1.f / l; lse = (m + log2f(l)) * LN2; }
-    const float *oc = nullptr;
-    if (inb && a.carry_o != nullptr) {
+    float *po = nullptr;
+    if (inb && a.part_o != nullptr) {
         const int u = a.up[row];
         if (u >= 0) {
-            const float lc = a.carry_lse[(size_t)u * H + h];
-            if (lc > NEG) {
-                const float mxx = fmaxf(lse, lc);
-                const float e0 = (lse > NEG) ? __expf(lse - mxx) : 0.f, e1 = __expf(lc - mxx);
-                const float tot = e0 + e1;
-                w0 *= e0 / tot;
-                w1 = e1 / tot;
-                lse = mxx + __logf(tot);
-                oc = a.carry_o + ((size_t)u * H + h) * D;
-            }
+            po = a.part_o + ((size_t)u * H + h) * D;
+            a.part_lse[(size_t)u * H + h] = lse;
         }
     }
 #pragma unroll
@@ -219,18 +213,17 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 #pragma unroll
             for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
+        float x[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) x[j] = (w0 > 0.f) ? __uint_as_float(r[j]) * w0 : 0.f;
+        if (po != nullptr) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4 *>(po + 32 * k + j) = make_float4(x[j], x[j + 1], x[j + 2], x[j + 3]);
+        }
         uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-            float x0 = (w0 > 0.f) ? __uint_as_float(r[j]) * w0 : 0.f;
-            float x1 = (w0 > 0.f) ? __uint_as_float(r[j + 1]) * w0 : 0.f;
-            if (oc != nullptr) {
-                const float2 c = *reinterpret_cast<const float2 *>(oc + 32 * k + j);
-                x0 = fmaf(w1, c.x, x0);
-                x1 = fmaf(w1, c.y, x1);
-            }
-            pk[j >> 1] = pack_bf16(x0, x1);
-        }
+        for (int j = 0; j < 16; ++j) pk[j] = pack_bf16(x[2 * j], x[2 * j + 1]);
         uint8_t *dst = sQ + (k >> 1) * SUB;
 #pragma unroll
         for (int c = 0; c < 4; ++c)

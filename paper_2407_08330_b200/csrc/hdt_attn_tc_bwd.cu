@@ -200,9 +200,10 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         ph_tma ^= 1;
     };
 
-    // Read an accumulator (this thread's row, its half of the D columns), scale, add the partial
-    // gradient of the upper stages, stage as bf16 into `dst` (NSUB swizzled sub-tiles).
-    auto drain = [&](uint32_t tm_col, bool have, float scale, const float *carry, uint8_t *dst) {
+    // Read an accumulator (this thread's row, its half of the D columns), scale, stage as bf16 into
+    // `dst` (NSUB swizzled sub-tiles); rows that live on in the next stage also leave the fp32
+    // values in that stage's buffer (`part`), which completes and overwrites them.
+    auto drain = [&](uint32_t tm_col, bool have, float scale, float *part, uint8_t *dst) {
 #pragma unroll
         for (int sl = 0; sl < D / 64; ++sl) {
             const int c0 = hf * (D / 2) + 32 * sl;
@@ -217,12 +218,8 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
             uint32_t pk[16];
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-                float x0 = __uint_as_float(r[j]) * scale, x1 = __uint_as_float(r[j + 1]) * scale;
-                if (carry != nullptr) {
-                    const float2 c = *reinterpret_cast<const float2 *>(carry + c0 + j);
-                    x0 += c.x;
-                    x1 += c.y;
-                }
+                const float x0 = __uint_as_float(r[j]) * scale, x1 = __uint_as_float(r[j + 1]) * scale;
+                if (part != nullptr) *reinterpret_cast<float2 *>(part + c0 + j) = make_float2(x0, x1);
                 pk[j >> 1] = pack_bf16(x0, x1);
             }
             uint8_t *d = dst + (c0 >> 6) * SUB;
@@ -246,13 +243,13 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     const bool run = !empty && !dead;
     const int row = r0 + rl;
     const bool inb = row < r1;
-    const float *cq = nullptr, *ck = nullptr, *cv = nullptr;
-    if (inb && a.carry_dq != nullptr) {
+    float *cq = nullptr, *ck = nullptr, *cv = nullptr;
+    if (inb && a.part_dq != nullptr) {
         const int u = a.up[row];
         if (u >= 0) {
-            cq = a.carry_dq + ((size_t)u * H + h) * D;
-            ck = a.carry_dk + ((size_t)u * H + h) * D;
-            cv = a.carry_dv + ((size_t)u * H + h) * D;
+            cq = a.part_dq + ((size_t)u * H + h) * D;
+            ck = a.part_dk + ((size_t)u * H + h) * D;
+            cv = a.part_dv + ((size_t)u * H + h) * D;
         }
     }
 
@@ -300,6 +297,17 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
 }
 
 
+// Cycle counts per phase of k_bwd_tc_p, accumulated by thread 0 of CTA 0 (diagnostics).
+__device__ long long g_bwd_phase_cycles[16];
+#define HDT_STAMP(i)                                        \
+    do {                                                    \
+        if (stamp) {                                        \
+            const long long now_ = clock64();               \
+            ph_acc[i] += now_ - t_last;                     \
+            t_last = now_;                                  \
+        }                                                   \
+    } while (0)
+
 // ---------------------------------------------------------------------------------------------
 // Persistent, software-pipelined backward for blocks that are SELF and not EMPTY at D = 64.
 // One CTA of 512 threads per SM walks its share of the (block, head) items (queue_split order,
@@ -315,6 +323,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                                                      const __grid_constant__ CUtensorMap tm_do, const BwdStageArgs a) {
     constexpr int D = 64;
     constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_DK = 320, TM_DV = 384, TM_COLS = 512;
+    constexpr int STG = 128 * 144;        // bytes of one staged output tile (rows padded to 144 bytes)
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sIn = sm;                    // 2 stages x {Q, dO, K, V}
@@ -334,8 +343,8 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     if (tid == 0) {
         mbar_init(&bar_tma[0], 1);
         mbar_init(&bar_tma[1], 1);
-        mbar_init(bar_a, 1);
-        mbar_init(bar_b, 1);
+        mbar_init(bar_a, 2);   // S and dP are issued by two threads
+        mbar_init(bar_b, 3);   // dV, dK, dQ by three
         *abort_flag = (*a.status != 0);
         fence_mbar_init();
     }
@@ -347,86 +356,100 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const bool dead = (*abort_flag != 0);
     bool ok = true;
+    // MMAs are issued by lane 0 of warps 0, 1, 2 in parallel: a single thread needs about 100 cycles
+    // per small MMA (descriptor arithmetic), three chains issued side by side hide that
+    const bool issuer = ((tid & 31) == 0) && warp < 3;
 
-    auto item_of = [&](int i, int &blk, int &h) {
-        const int item = (int)blockIdx.x + i * G;
-        blk = a.queue_split[item / H];
-        h = item % H;
+    // Item i of this CTA: block, head, rows.  Descriptors are fetched two items ahead and the row
+    // statistics one item ahead, so that no global-memory latency sits between two items.
+    struct Desc { int r0, r1, h; };
+    auto load_blk = [&](int i) { return a.queue_split[((int)blockIdx.x + i * G) / H]; };
+    auto load_rec = [&](int i, int blk) {
+        Desc d;
+        d.h = ((int)blockIdx.x + i * G) % H;
+        d.r0 = a.blocks[5 * (size_t)blk];
+        d.r1 = a.blocks[5 * (size_t)blk + 1];
+        return d;
     };
-    auto issue_tma = [&](int i) {       // thread 0
-        int blk, h;
-        item_of(i, blk, h);
-        const int r0 = a.blocks[5 * (size_t)blk];
+    auto load_desc = [&](int i) { return load_rec(i, load_blk(i)); };
+    struct RowStat { int lo, hi, up; float lse2, dl; };
+    auto load_stat = [&](const Desc &d) {
+        RowStat r{0, 0, -1, 0.f, 0.f};
+        const int row = d.r0 + rl;
+        if (row < d.r1) {
+            r.lo = a.rng[2 * row];
+            r.hi = a.rng[2 * row + 1];
+            r.lse2 = a.lse[(size_t)d.h * a.T + row];   // natural log; scaled where it is used
+            r.dl = a.delta[(size_t)d.h * a.T + row];
+            if (a.part_dq != nullptr) r.up = a.up[row];
+        }
+        return r;
+    };
+    auto issue_tma = [&](int i, const Desc &d) {       // thread 0
         uint8_t *st = sIn + (i & 1) * 4 * SUB;
         uint64_t *bar = &bar_tma[i & 1];
         mbar_expect_tx(bar, 4 * SUB);
-        tma_load_3d(st, &tm_q, 0, h, r0, bar);
-        tma_load_3d(st + SUB, &tm_do, 0, h, r0, bar);
-        tma_load_3d(st + 2 * SUB, &tm_k, 0, h, r0, bar);
-        tma_load_3d(st + 3 * SUB, &tm_v, 0, h, r0, bar);
+        tma_load_3d(st, &tm_q, 0, d.h, d.r0, bar);
+        tma_load_3d(st + SUB, &tm_do, 0, d.h, d.r0, bar);
+        tma_load_3d(st + 2 * SUB, &tm_k, 0, d.h, d.r0, bar);
+        tma_load_3d(st + 3 * SUB, &tm_v, 0, d.h, d.r0, bar);
     };
-    auto issue_sdp = [&](int i, int Nc) {   // thread 0, inputs of item i have landed
+    auto issue_sdp = [&](int i, int Nc) {   // warps 0 (S) and 1 (dP), lane 0; inputs of item i have landed
         const uint32_t st = smem_u32(sIn + (i & 1) * 4 * SUB);
         const uint32_t idesc = idesc_bf16(Nc, false, false);
+        const uint32_t a_off = (warp == 0) ? 0u : (uint32_t)SUB, b_off = (warp == 0) ? 2u * SUB : 3u * SUB;
+        const uint32_t col = (warp == 0) ? TM_S : TM_DP;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk)
-            mma_ss(tmem + TM_S, smem_desc(st + kk * 32, 0, 1024), smem_desc(st + 2 * SUB + kk * 32, 0, 1024), idesc, kk > 0);
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk)
-            mma_ss(tmem + TM_DP, smem_desc(st + SUB + kk * 32, 0, 1024), smem_desc(st + 3 * SUB + kk * 32, 0, 1024), idesc,
-                   kk > 0);
+            mma_ss(tmem + col, smem_desc(st + a_off + kk * 32, 0, 1024), smem_desc(st + b_off + kk * 32, 0, 1024), idesc, kk > 0);
         mma_commit(bar_a);
-    };
-    auto rows16 = [&](int blk) {
-        const int n = a.blocks[5 * (size_t)blk + 1] - a.blocks[5 * (size_t)blk];
-        return (n + 15) & ~15;
     };
 
     if (!dead && my_count > 0) {
+        Desc dc = load_desc(0), dn = dc, dn2 = dc;
+        if (my_count > 1) dn = load_desc(1);
+        int blk2 = (my_count > 2) ? load_blk(2) : 0;   // block id of item it+2, fetched one iteration ahead
+        RowStat rc = load_stat(dc), rn = rc;
         if (tid == 0) {
-            issue_tma(0);
-            if (my_count > 1) issue_tma(1);
+            issue_tma(0, dc);
+            if (my_count > 1) issue_tma(1, dn);
+        }
+        if (issuer && warp < 2) {
             ok = mbar_wait(&bar_tma[0], 0, abort_flag, WAIT_CYCLES) && ok;
             if (!*abort_flag) {
-                int blk, h;
-                item_of(0, blk, h);
                 tc_fence_after();
-                issue_sdp(0, rows16(blk));
+                issue_sdp(0, (dc.r1 - dc.r0 + 15) & ~15);
             }
         }
+        const bool stamp = (tid == 0 && blockIdx.x == 0);
+        long long ph_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+        long long t_last = clock64();
         for (int it = 0; it < my_count; ++it) {
-            int blk, h;
-            item_of(it, blk, h);
-            const int *rec = a.blocks + 5 * (size_t)blk;
-            const int r0 = rec[0], r1 = rec[1];
+            HDT_STAMP(9);
+            // prefetch: descriptor of item it+2, row statistics of item it+1
+            if (it + 2 < my_count) dn2 = load_rec(it + 2, blk2);
+            if (it + 3 < my_count) blk2 = load_blk(it + 3);
+            if (it + 1 < my_count) rn = load_stat(dn);
+            const int r0 = dc.r0, r1 = dc.r1, h = dc.h;
             const int nrows = r1 - r0, Nc = (nrows + 15) & ~15;
-            const int row = r0 + rl;
-            const bool inb = row < r1;
-            int lo = 0, hi = 0;
-            float lse2 = 0.f, dl = 0.f;
-            const float *cq = nullptr, *ck = nullptr, *cv = nullptr;
-            if (inb) {
-                lo = a.rng[2 * row];
-                hi = a.rng[2 * row + 1];
-                if (hi > lo) {
-                    lse2 = a.lse[(size_t)h * a.T + row] * LOG2E;
-                    dl = a.delta[(size_t)h * a.T + row];
-                }
-                if (a.carry_dq != nullptr) {
-                    const int u = a.up[row];
-                    if (u >= 0) {
-                        cq = a.carry_dq + ((size_t)u * H + h) * D;
-                        ck = a.carry_dk + ((size_t)u * H + h) * D;
-                        cv = a.carry_dv + ((size_t)u * H + h) * D;
-                    }
-                }
+            const bool inb = r0 + rl < r1;
+            const float lse2 = rc.lse2 * LOG2E, dl = rc.dl;
+            float *cq = nullptr, *ck = nullptr, *cv = nullptr;
+            if (rc.up >= 0) {   // this row lives on in the next stage: its fp32 gradients go there too
+                cq = a.part_dq + ((size_t)rc.up * H + h) * D;
+                ck = a.part_dk + ((size_t)rc.up * H + h) * D;
+                cv = a.part_dv + ((size_t)rc.up * H + h) * D;
             }
-            const int jl = max(lo - r0, 0), jh = min(hi - r0, nrows);
+            const int jl = max(rc.lo - r0, 0), jh = min(rc.hi - r0, nrows);
             const bool has = inb && jh > jl;
             uint8_t *st = sIn + (it & 1) * 4 * SUB;
 
-            ok = mbar_wait(bar_a, it & 1, abort_flag, WAIT_CYCLES) && ok;   // S, dP of this item
+            HDT_STAMP(0);
+            // S, dP of this item: warp 0 polls the mbarrier, the other warps sleep at the CTA barrier
+            if (warp == 0) ok = mbar_wait(bar_a, it & 1, abort_flag, WAIT_CYCLES) && ok;
+            __syncthreads();   // also: the previous item's staged gradients have been stored
             tc_fence_after();
+            HDT_STAMP(1);
             // ---- P and dS of this thread's 32 columns, in two halves of 16 ----
             if (32 * qt < Nc) {
 #pragma unroll
@@ -468,71 +491,95 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             }
             fence_proxy_async_smem();
             tc_fence_before();
+            HDT_STAMP(2);
             __syncthreads();
-            if (tid == 0 && !*abort_flag) {
+            HDT_STAMP(3);
+            if (issuer && !*abort_flag) {
                 tc_fence_after();
+                // descriptors differ only in the start address: add (bytes >> 4) to the low word
                 const uint32_t sb = smem_u32(st);
-                const uint32_t idesc_kv = idesc_bf16(D, true, true), idesc_q = idesc_bf16(D, false, true);
-                for (int kk = 0; kk < Nc / 16; ++kk)   // dV = P^T dO
-                    mma_ss(tmem + TM_DV, smem_desc(smem_u32(sP) + kk * 2048, SUB, 1024),
-                           smem_desc(sb + SUB + kk * 2048, SUB, 1024), idesc_kv, kk > 0);
-                for (int kk = 0; kk < Nc / 16; ++kk)   // dK = dS^T Q
-                    mma_ss(tmem + TM_DK, smem_desc(smem_u32(sDS) + kk * 2048, SUB, 1024),
-                           smem_desc(sb + kk * 2048, SUB, 1024), idesc_kv, kk > 0);
-                for (int kk = 0; kk < Nc / 16; ++kk)   // dQ = dS K
-                    mma_ss(tmem + TM_DQ, smem_desc(smem_u32(sDS) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024),
-                           smem_desc(sb + 2 * SUB + kk * 2048, SUB, 1024), idesc_q, kk > 0);
+                const int nk = Nc / 16;
+                if (warp == 0) {          // dV = P^T dO
+                    const uint32_t idesc = idesc_bf16(D, true, true);
+                    const uint64_t da = smem_desc(smem_u32(sP), SUB, 1024), db = smem_desc(sb + SUB, SUB, 1024);
+                    for (int kk = 0; kk < nk; ++kk)
+                        mma_ss(tmem + TM_DV, da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc, kk > 0);
+                } else if (warp == 1) {   // dK = dS^T Q
+                    const uint32_t idesc = idesc_bf16(D, true, true);
+                    const uint64_t da = smem_desc(smem_u32(sDS), SUB, 1024), db = smem_desc(sb, SUB, 1024);
+                    for (int kk = 0; kk < nk; ++kk)
+                        mma_ss(tmem + TM_DK, da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc, kk > 0);
+                } else {                  // dQ = dS K
+                    const uint32_t idesc = idesc_bf16(D, false, true);
+                    const uint64_t da = smem_desc(smem_u32(sDS), 0, 1024), db = smem_desc(sb + 2 * SUB, SUB, 1024);
+                    for (int kk = 0; kk < nk; ++kk)
+                        mma_ss(tmem + TM_DQ, da + (uint64_t)((kk / 4) * (SUB >> 4) + (kk % 4) * 2),
+                               db + (uint64_t)(kk * 128), idesc, kk > 0);
+                }
                 mma_commit(bar_b);
-                if (it + 1 < my_count) {               // S, dP of the next item run during this item's drain
+                HDT_STAMP(10);
+                if (warp < 2 && it + 1 < my_count) {   // S, dP of the next item run during this item's drain
                     ok = mbar_wait(&bar_tma[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag, WAIT_CYCLES) && ok;
+                    HDT_STAMP(11);
                     if (!*abort_flag) {
-                        int blk2, h2;
-                        item_of(it + 1, blk2, h2);
                         tc_fence_after();
-                        issue_sdp(it + 1, rows16(blk2));
+                        issue_sdp(it + 1, (dn.r1 - dn.r0 + 15) & ~15);
                     }
                 }
             }
-            ok = mbar_wait(bar_b, it & 1, abort_flag, WAIT_CYCLES) && ok;   // dQ, dK, dV of this item
+            HDT_STAMP(4);
+            if (warp == 0) ok = mbar_wait(bar_b, it & 1, abort_flag, WAIT_CYCLES) && ok;   // dQ, dK, dV of this item
+            __syncthreads();
             tc_fence_after();
-            if (tid == 0 && it + 2 < my_count && !*abort_flag) issue_tma(it + 2);   // this stage is free again
+            HDT_STAMP(5);
+            if (tid == 0 && it + 2 < my_count && !*abort_flag) issue_tma(it + 2, dn2);   // this stage is free again
             // ---- drain: 16 columns of each gradient per thread, staged as bf16 ----
 #pragma unroll
             for (int t = 0; t < 3; ++t) {
                 const uint32_t col = (t == 0) ? TM_DQ : (t == 1) ? TM_DK : TM_DV;
                 const float sc = (t == 2) ? 1.f : a.scale;
-                const float *cy = (t == 0) ? cq : (t == 1) ? ck : cv;
-                uint8_t *dst = (t == 0) ? sP : (t == 1) ? (sP + SUB) : sDS;
+                float *cy = (t == 0) ? cq : (t == 1) ? ck : cv;
+                uint8_t *dst = sP + t * STG;    // staging: 128 rows x 144 bytes per tensor
                 uint32_t r[16];
                 tmem_ld16(tmem + col + lane_base + 16 * qt, r);
                 tmem_wait_ld();
+                float x[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) x[j] = __uint_as_float(r[j]) * sc;
+                if (cy != nullptr) {   // rows that also exist in the next stage (a few per block)
+                    float4 *c4 = reinterpret_cast<float4 *>(cy + 16 * qt);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) c4[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+                }
                 uint32_t pk[8];
 #pragma unroll
-                for (int j = 0; j < 16; j += 2) {
-                    float x0 = __uint_as_float(r[j]) * sc, x1 = __uint_as_float(r[j + 1]) * sc;
-                    if (cy != nullptr) {
-                        const float2 c = *reinterpret_cast<const float2 *>(cy + 16 * qt + j);
-                        x0 += c.x;
-                        x1 += c.y;
-                    }
-                    pk[j >> 1] = pack_bf16(x0, x1);
-                }
-                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                for (int j = 0; j < 8; ++j) pk[j] = pack_bf16(x[2 * j], x[2 * j + 1]);
+                *reinterpret_cast<uint4 *>(dst + rl * 144 + qt * 32) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(dst + rl * 144 + qt * 32 + 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
             tc_fence_before();
+            HDT_STAMP(6);
             __syncthreads();
-            // ---- coalesced stores: 3 tensors x 128 rows x 8 chunks ----
-            for (int idx = tid; idx < 3 * 1024; idx += 512) {
-                const int t = idx >> 10, rem = idx & 1023, r = rem >> 3, c = rem & 7;
-                if (r < nrows) {
-                    const uint8_t *src = (t == 0) ? sP : (t == 1) ? (sP + SUB) : sDS;
+            HDT_STAMP(7);
+            // ---- coalesced stores: thread -> rows tid/8 and tid/8 + 64, 16-byte chunk tid%8, 3 tensors ----
+            {
+                const int rA = tid >> 3, c = tid & 7;
+#pragma unroll
+                for (int t = 0; t < 3; ++t) {
                     __nv_bfloat16 *g = reinterpret_cast<__nv_bfloat16 *>((t == 0) ? a.dq : (t == 1) ? a.dk : a.dv);
-                    const uint4 v = *reinterpret_cast<const uint4 *>(src + swz(r, c));
-                    *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + r) * H + h) * D + c * 8) = v;
+                    uint4 v0, v1;
+                    if (rA < nrows) v0 = *reinterpret_cast<const uint4 *>(sP + t * STG + rA * 144 + c * 16);
+                    if (rA + 64 < nrows) v1 = *reinterpret_cast<const uint4 *>(sP + t * STG + (rA + 64) * 144 + c * 16);
+                    if (rA < nrows) *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + rA) * H + h) * D + c * 8) = v0;
+                    if (rA + 64 < nrows) *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + rA + 64) * H + h) * D + c * 8) = v1;
                 }
             }
-            __syncthreads();   // staging is read out before the next item's P / dS are written
+            HDT_STAMP(8);
+            dc = dn; dn = dn2; rc = rn;
+        }
+        if (stamp) {
+            for (int i = 0; i < 12; ++i) g_bwd_phase_cycles[i] += ph_acc[i];
+            g_bwd_phase_cycles[12] += my_count;
         }
     }
     if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
@@ -586,6 +633,15 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
     }
+    return HDT_OK;
+}
+
+// Diagnostics: cycles CTA 0 of the persistent backward spent per phase since the last call
+// (10 phases, then the item count); resets the counters.
+int read_bwd_phase_cycles(long long *out16) {
+    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out16, g_bwd_phase_cycles, sizeof(long long) * 16));
+    long long zero[16] = {0};
+    HDT_CUDA_CHECK(cudaMemcpyToSymbol(g_bwd_phase_cycles, zero, sizeof(zero)));
     return HDT_OK;
 }
 

@@ -74,13 +74,16 @@ struct FwdStageArgs {
     int n_fused;
     const void *q, *k, *v;
     float scale_log2;   // softmax_scale * log2(e)
-    // partial results of the next stage (nullptr if none): [n_up, H, D] and [n_up, H]
+    // Stages run bottom-up.  carry_*: partial results the stages below left for this stage's
+    // elements, indexed by element ([n, H, D] and [n, H]); nullptr for stage 0.
     const float *carry_o, *carry_lse;
-    // outputs: final (stage 0) ...
+    // Every stage writes its merged result to the caller's tensors (later stages overwrite the
+    // rows they complete) ...
     void *o;            // dtype [T,H,D]
     float *lse;         // [H,T]
     int T;
-    // ... or this stage's partial results
+    // ... and, for elements that live on in the next stage, to that stage's buffers at up[e]
+    // ([n_next, H, D] and [n_next, H]); nullptr for the last stage.
     float *part_o, *part_lse;
     int *status;        // device failure word
     int rest_only;      // general kernel: only blocks after the first n_fused
@@ -97,9 +100,9 @@ struct BwdStageArgs {
     const float *lse;    // [H,T] final
     const float *delta;  // [H,T]
     float scale, scale_log2;
-    const float *carry_dq, *carry_dk, *carry_dv;  // [n_up,H,D] from the next stage, or nullptr
-    void *dq, *dk, *dv;                           // final dtype [T,H,D] (stage 0)
-    float *part_dq, *part_dk, *part_dv;           // [n,H,D] (stages above 0)
+    const float *carry_dq, *carry_dk, *carry_dv;  // [n,H,D] partials from the stages below, or nullptr
+    void *dq, *dk, *dv;                           // dtype [T,H,D], written by every stage
+    float *part_dq, *part_dk, *part_dv;           // [n_next,H,D] next stage's buffers (at up[e]), or nullptr
     int *status;                                  // device failure word
     int rest_only;                                // general kernel: only blocks after the first n_fused
     int no_persistent;                            // option: do not use the persistent kernels
@@ -109,6 +112,7 @@ int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t
 // Tensor-core (TMA + tcgen05) stage-0 kernels for bf16 (hdt_attn_tc.cu).
 int launch_fwd_tc(const FwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_bwd_tc(const BwdStageArgs &a, int head_dim, cudaStream_t st);
+int read_bwd_phase_cycles(long long *out16);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
                  cudaStream_t st);
