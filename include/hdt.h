@@ -66,7 +66,10 @@ typedef struct {
     int32_t block_m;    /* max rows per row block, 1..128; 0 = default 128                     */
     int32_t max_stages; /* max hierarchy height handled, 1..HDT_MAX_STAGES; 0 = default 4
                            ([DOC]/[SEC]/[SENT]/token documents need 3)                        */
-    int32_t reserved[6];
+    int32_t block_m_upper; /* max rows per row block in the stages above 0 (their arrays are a
+                           few percent of the tokens: smaller blocks give their kernels more
+                           CTAs), 1..128; 0 = default 32                                      */
+    int32_t reserved[5];
 } hdt_index_params_t;
 
 typedef struct hdt_index hdt_index_t; /* opaque host object; views into the caller's workspace */

@@ -26,8 +26,8 @@ Per stage s the index holds, for the compacted array A_s of n_s elements:
                 (q, q+1+c); child of head q: (q, q+1+c), c = number of children of q.
   up[e]         index of e in A_{s+1}, -1 if removed (or no next stage)
   scu[b]        start of sequence b in A_s (cumulative, B+1 entries)
-  blocks        rows (r0, r1, a, b, flags): row blocks of at most block_m consecutive elements of
-                one sequence, packed greedily and cut at family boundaries when a family fits
+  blocks        rows (r0, r1, a, b, flags): row blocks of at most block_m (stage 0) or block_m_upper
+                (stages above 0) consecutive elements of one sequence, packed greedily and cut at family boundaries when a family fits
                 in a block; [a,b) = hull of the rows' key ranges (a=b=r0 if none);
                 flags bit0 SELF  a>=r0 and b<=r1 (block needs no key outside itself)
                       bit1 DENSE every row's range is exactly [a,b)
@@ -108,7 +108,7 @@ def validate(level, parent, cu):
                     raise BadHierarchy("level must be parent's level + 1")
 
 
-def build(level, parent, cu, block_m: int = 128, max_stages: int = 32) -> Index:
+def build(level, parent, cu, block_m: int = 128, max_stages: int = 32, block_m_upper: int = 32) -> Index:
     level = np.asarray(level, np.int8)
     parent = np.asarray(parent, np.int32)
     cu = np.asarray(cu, np.int32)
@@ -192,8 +192,9 @@ def build(level, parent, cu, block_m: int = 128, max_stages: int = 32) -> Index:
         blocks = []
         for b in range(B):
             pos, end_seq = int(scu[b]), int(scu[b + 1])
+            bm = block_m if s == 0 else block_m_upper    # stages above 0 use their own block size
             while pos < end_seq:
-                end = min(pos + block_m, end_seq)
+                end = min(pos + bm, end_seq)
                 if end < end_seq and uid[end] >= 0 and uid[end] == uid[end - 1] and uid[end] > pos:
                     end = int(uid[end])
                 a, bb, any_key, dense, carry = None, None, False, True, False

@@ -24,7 +24,8 @@ class HdtError(RuntimeError):
 
 
 class _Params(C.Structure):
-    _fields_ = [("block_m", C.c_int32), ("max_stages", C.c_int32), ("reserved", C.c_int32 * 6)]
+    _fields_ = [("block_m", C.c_int32), ("max_stages", C.c_int32), ("block_m_upper", C.c_int32),
+                ("reserved", C.c_int32 * 5)]
 
 
 class _StageView(C.Structure):
@@ -93,14 +94,14 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def _params(block_m, max_stages):
+def _params(block_m, max_stages, block_m_upper=0):
     p = _Params()
-    p.block_m, p.max_stages = int(block_m), int(max_stages)
+    p.block_m, p.max_stages, p.block_m_upper = int(block_m), int(max_stages), int(block_m_upper)
     return p
 
 
-def hdt_index_workspace_bytes(batch, total_tokens, block_m=0, max_stages=0) -> int:
-    p = _params(block_m, max_stages)
+def hdt_index_workspace_bytes(batch, total_tokens, block_m=0, max_stages=0, block_m_upper=0) -> int:
+    p = _params(block_m, max_stages, block_m_upper)
     return int(lib().hdt_index_workspace_bytes(batch, total_tokens, C.cast(C.byref(p), C.c_void_p)))
 
 
@@ -146,13 +147,14 @@ class HdtIndex:
             pass
 
 
-def hdt_build_index(level, parent, cu_seqlens, block_m=0, max_stages=0, workspace=None) -> HdtIndex:
+def hdt_build_index(level, parent, cu_seqlens, block_m=0, max_stages=0, workspace=None,
+                    block_m_upper=0) -> HdtIndex:
     """level int8[T], parent int32[T], cu_seqlens int32[B+1]: CUDA tensors."""
     assert level.is_cuda and parent.is_cuda and cu_seqlens.is_cuda
     assert level.dtype == torch.int8 and parent.dtype == torch.int32 and cu_seqlens.dtype == torch.int32
     level, parent, cu_seqlens = level.contiguous(), parent.contiguous(), cu_seqlens.contiguous()
     T, B = level.numel(), cu_seqlens.numel() - 1
-    p = _params(block_m, max_stages)
+    p = _params(block_m, max_stages, block_m_upper)
     need = int(lib().hdt_index_workspace_bytes(B, T, C.cast(C.byref(p), C.c_void_p)))
     if need == 0:
         raise HdtError(-1, "invalid index parameters")

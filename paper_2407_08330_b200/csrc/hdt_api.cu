@@ -185,6 +185,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.tok = s ? P.tok : nullptr;
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
         a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
+        a.block_rows = s ? ix->block_m_upper : ix->block_m;
         a.q = q; a.k = k; a.v = v;
         a.scale_log2 = scale * 1.4426950408889634f;
         if (s > 0) {   // partial results the stages below left for this stage's elements
@@ -239,6 +240,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.tok = s ? P.tok : nullptr;
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
         a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
+        a.block_rows = s ? ix->block_m_upper : ix->block_m;
         a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = delta;
         a.scale = scale;
         a.scale_log2 = scale * 1.4426950408889634f;
@@ -325,6 +327,7 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
         a.tok = s ? P.tok : nullptr;
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
         a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
+        a.block_rows = s ? ix->block_m_upper : ix->block_m;
         a.q = q; a.k = k; a.v = v;
         a.scale_log2 = scale * 1.4426950408889634f;
         if (s > 0) {   // partial results the stages below left for this stage's elements

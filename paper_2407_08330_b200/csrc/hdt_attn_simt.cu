@@ -12,7 +12,6 @@
 namespace hdt {
 
 static constexpr int KC = 32;        // keys per shared-memory chunk
-static constexpr int NTHREADS = 512;
 
 template <bool BF16>
 __device__ __forceinline__ float4 load4(const void *base, size_t elem) {
@@ -66,7 +65,7 @@ __device__ __forceinline__ float group_sum(float x) {
 }
 
 // Stage `rows` [c0, c0+KC) of a [*, H, D] tensor (through tok) into smem as fp32, zero past `end`.
-template <int D, bool BF16>
+template <int D, bool BF16, int NTHREADS>
 __device__ __forceinline__ void stage_rows(float4 *dst, const void *src, const int *tok, int c0, int end,
                                            int H, int h) {
     constexpr int U = D / 4;
@@ -85,7 +84,7 @@ __device__ __forceinline__ void stage_rows(float4 *dst, const void *src, const i
 // ---------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------
-template <int D, bool BF16>
+template <int D, bool BF16, int NTHREADS>
 __global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
     constexpr int G = D / 16, U = D / 4, RP = NTHREADS / G;
     __shared__ float4 sK[KC * U];
@@ -113,8 +112,8 @@ __global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
         float m = NEG, l = 0.f;
         for (int c0 = ka; c0 < kb; c0 += KC) {
             __syncthreads();
-            stage_rows<D, BF16>(sK, a.k, a.tok, c0, kb, H, h);
-            stage_rows<D, BF16>(sV, a.v, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16, NTHREADS>(sK, a.k, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16, NTHREADS>(sV, a.v, a.tok, c0, kb, H, h);
             __syncthreads();
             const int jlo = max(lo, c0), jhi = min(hi, c0 + KC);
             const bool has = jhi > jlo;
@@ -204,7 +203,7 @@ __global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
 // backward: phase A rows -> dQ, phase B keys -> dK, dV (the family ranges are symmetric, so the
 // same blocks serve as key blocks)
 // ---------------------------------------------------------------------------------------------
-template <int D, bool BF16>
+template <int D, bool BF16, int NTHREADS>
 __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
     constexpr int G = D / 16, U = D / 4, RP = NTHREADS / G;
     __shared__ float4 sA[KC * U];  // K (phase A) / Q (phase B)
@@ -243,8 +242,8 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
         }
         for (int c0 = ka; c0 < kb; c0 += KC) {
             __syncthreads();
-            stage_rows<D, BF16>(sA, a.k, a.tok, c0, kb, H, h);
-            stage_rows<D, BF16>(sB, a.v, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16, NTHREADS>(sA, a.k, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16, NTHREADS>(sB, a.v, a.tok, c0, kb, H, h);
             __syncthreads();
             const int jlo = max(lo, c0), jhi = min(hi, c0 + KC);
             const bool has = jhi > jlo;
@@ -293,9 +292,9 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
         }
         for (int c0 = ka; c0 < kb; c0 += KC) {
             __syncthreads();
-            stage_rows<D, BF16>(sA, a.q, a.tok, c0, kb, H, h);
-            stage_rows<D, BF16>(sB, a.d_o, a.tok, c0, kb, H, h);
-            if (threadIdx.x < KC) {
+            stage_rows<D, BF16, NTHREADS>(sA, a.q, a.tok, c0, kb, H, h);
+            stage_rows<D, BF16, NTHREADS>(sB, a.d_o, a.tok, c0, kb, H, h);
+            if (threadIdx.x < KC) {   // KC <= NTHREADS
                 const int e = c0 + threadIdx.x;
                 float L = 0.f, dlt = 0.f;
                 if (e < kb) {
@@ -354,28 +353,47 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
     }
 }
 
-// delta[h, t] = sum_c dO[t,h,c] * O[t,h,c]; one warp per (t, h).
+// delta[h, t] = sum_c dO[t,h,c] * O[t,h,c].  A (token, head) row is read by LPR adjacent lanes with
+// one 16-byte load each per tensor (8 bf16 or 4 fp32 values), so a warp covers 32 / LPR rows.
 template <int D, bool BF16>
-__global__ void k_delta(const void *o, const void *d_o, float *delta, int T, int H) {
-    const int lane = threadIdx.x & 31;
-    const long long w = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    if (w >= (long long)T * H) return;
-    const int t = (int)(w / H), h = (int)(w % H);
+__global__ void __launch_bounds__(256) k_delta(const void *o, const void *d_o, float *delta, int T, int H) {
+    constexpr int VPL = BF16 ? 8 : 4;          // values per lane
+    constexpr int LPR = D / VPL;               // lanes per row: 8 (bf16, D=64) ... 32 (fp32, D=128)
+    const long long gtid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long row = gtid / LPR;
+    const int sub = (int)(gtid % LPR);
     float acc = 0.f;
-    if (lane < D / 4) {
-        const float4 x = load4<BF16>(o, (size_t)w * D + 4 * lane);
-        const float4 y = load4<BF16>(d_o, (size_t)w * D + 4 * lane);
-        acc = dot4(x, y, 0.f);
+    if (row < (long long)T * H) {
+        if constexpr (BF16) {
+            const uint4 x = *reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(o) + row * D + sub * 8);
+            const uint4 y = *reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(d_o) + row * D + sub * 8);
+            const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                acc = fmaf(__uint_as_float(xs[i] << 16), __uint_as_float(ys[i] << 16), acc);
+                acc = fmaf(__uint_as_float(xs[i] & 0xffff0000u), __uint_as_float(ys[i] & 0xffff0000u), acc);
+            }
+        } else {
+            const float4 x = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(o) + row * D + sub * 4);
+            const float4 y = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(d_o) + row * D + sub * 4);
+            acc = dot4(x, y, 0.f);
+        }
     }
-    for (int s = 16; s; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
-    if (lane == 0) delta[(size_t)h * T + t] = acc;
+#pragma unroll
+    for (int s = LPR / 2; s; s >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, s);
+    if (sub == 0 && row < (long long)T * H) {
+        const int t = (int)(row / H), h = (int)(row % H);
+        delta[(size_t)h * T + t] = acc;
+    }
 }
 
+// Small row blocks (the stages above 0) run with 128-thread CTAs so that several fit on an SM.
 template <int D, bool BF16>
 static int launch_fwd_t(const FwdStageArgs &a, cudaStream_t st) {
     if (a.nb == 0) return HDT_OK;
     dim3 grid(a.nb, a.H);
-    k_fwd_simt<D, BF16><<<grid, NTHREADS, 0, st>>>(a);
+    if (a.block_rows <= 32) k_fwd_simt<D, BF16, 128><<<grid, 128, 0, st>>>(a);
+    else k_fwd_simt<D, BF16, 512><<<grid, 512, 0, st>>>(a);
     count_launch();
     HDT_CUDA_CHECK(cudaGetLastError());
     return HDT_OK;
@@ -384,7 +402,8 @@ template <int D, bool BF16>
 static int launch_bwd_t(const BwdStageArgs &a, cudaStream_t st) {
     if (a.nb == 0) return HDT_OK;
     dim3 grid(a.nb, a.H);
-    k_bwd_simt<D, BF16><<<grid, NTHREADS, 0, st>>>(a);
+    if (a.block_rows <= 32) k_bwd_simt<D, BF16, 128><<<grid, 128, 0, st>>>(a);
+    else k_bwd_simt<D, BF16, 512><<<grid, 512, 0, st>>>(a);
     count_launch();
     HDT_CUDA_CHECK(cudaGetLastError());
     return HDT_OK;
@@ -401,17 +420,21 @@ int launch_bwd_simt(const BwdStageArgs &a, int D, int dtype, cudaStream_t st) {
     return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
 }
 
+template <int D, bool BF16>
+static void launch_delta_t(const void *o, const void *d_o, float *delta, int T, int H, cudaStream_t st) {
+    constexpr int LPR = D / (BF16 ? 8 : 4);
+    const long long threads = (long long)T * H * LPR;
+    k_delta<D, BF16><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(o, d_o, delta, T, H);
+}
+
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int D, int dtype, cudaStream_t st) {
-    const long long rows = (long long)T * H;
-    if (rows == 0) return HDT_OK;
-    const int threads = 256;
-    const long long blocks = (rows * 32 + threads - 1) / threads;
+    if ((long long)T * H == 0) return HDT_OK;
     if (D == 64) {
-        if (dtype == HDT_BF16) k_delta<64, true><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
-        else k_delta<64, false><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
+        if (dtype == HDT_BF16) launch_delta_t<64, true>(o, d_o, delta, T, H, st);
+        else launch_delta_t<64, false>(o, d_o, delta, T, H, st);
     } else if (D == 128) {
-        if (dtype == HDT_BF16) k_delta<128, true><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
-        else k_delta<128, false><<<(unsigned)blocks, threads, 0, st>>>(o, d_o, delta, T, H);
+        if (dtype == HDT_BF16) launch_delta_t<128, true>(o, d_o, delta, T, H, st);
+        else launch_delta_t<128, false>(o, d_o, delta, T, H, st);
     } else {
         return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
     }

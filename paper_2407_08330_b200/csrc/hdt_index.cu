@@ -27,7 +27,7 @@ struct Layout {
 
 static size_t al(size_t x) { return (x + 255) & ~size_t(255); }
 
-static Layout make_layout(int B, int T, int bm, int max_stages) {
+static Layout make_layout(int B, int T, int bm, int max_stages) {   // bm: the smaller of the two block sizes
     Layout L;
     L.capnb = 2 * (T / bm + 1) + 4 * B + 2;
     L.nchunk = (T + CHUNK - 1) / CHUNK + 1;
@@ -66,7 +66,7 @@ __device__ __forceinline__ void dev_fail(DevHeader *h, int code, int pos) {
 // ---------------------------------------------------------------------------------------------
 __global__ void k_init(const int8_t *__restrict__ level, const int32_t *__restrict__ parent,
                        const int32_t *__restrict__ cu, int B, int T, int max_level, DevHeader *hdr,
-                       int *tok, int *par, int *scu, int *cnt, int *nlc) {
+                       int *tok, int *par, int *scu, int *cnt) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i <= B) {
         const int c = cu[i];
@@ -107,8 +107,7 @@ __global__ void k_init(const int8_t *__restrict__ level, const int32_t *__restri
     if (!ok) { dev_fail(hdr, HDT_ERR_BAD_HIERARCHY, i); gp = -1; }
     tok[i] = i;
     par[i] = gp;
-    cnt[i] = 0;
-    nlc[i] = 0;
+    if (gp >= 0) atomicAdd(&cnt[gp], 1);   // cnt and nlc were zeroed with the header
 }
 
 __global__ void k_count(const DevHeader *hdr, int s, const int *__restrict__ par, int *cnt) {
@@ -275,7 +274,7 @@ __global__ void k_compact(const DevHeader *hdr, int s, int B, const int *__restr
 // (0 for heads and for elements in no family, capped at 255 >= block_m).
 __global__ void k_walk(const DevHeader *hdr, int s, int bm, const int *__restrict__ scu,
                        const uint8_t *__restrict__ fpos, int *bstart, int *seqcount, int smem_cap) {
-    extern __shared__ uint8_t s_fp[];
+    extern __shared__ __align__(16) uint8_t s_fp[];
     const int n = hdr->st[s].n;
     const int b = blockIdx.x;
     if (s > 0 && n == 0) { if (threadIdx.x == 0) seqcount[b] = 0; return; }
@@ -294,12 +293,18 @@ __global__ void k_walk(const DevHeader *hdr, int s, int bm, const int *__restric
     }
     __syncthreads();
     off = s_red[0];
-    const bool in_smem = len <= smem_cap;
-    if (in_smem)
-        for (int i = threadIdx.x; i < len; i += blockDim.x) s_fp[i] = fpos[s0 + i];
+    // stage fpos[a0 .. s1) from the 16-byte boundary a0 <= s0 with vector loads
+    const int a0 = s0 & ~15, skew = s0 - a0;
+    const bool in_smem = len + 32 <= smem_cap;
+    if (in_smem) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(fpos + a0);
+        uint4 *dst = reinterpret_cast<uint4 *>(s_fp);
+        const int nv = (skew + len + 15) >> 4;   // the workspace array is padded to 256 bytes: no overrun
+        for (int i = threadIdx.x; i < nv; i += blockDim.x) dst[i] = src[i];
+    }
     __syncthreads();
     if (threadIdx.x != 0) return;
-    const uint8_t *fp = in_smem ? s_fp : (fpos + s0);
+    const uint8_t *fp = in_smem ? (s_fp + skew) : (fpos + s0);
     int pos = 0, cntb = 0;
     while (pos < len) {
         int end = min(pos + bm, len);
@@ -348,10 +353,10 @@ __global__ void k_blocks(DevHeader *hdr, int s, int bm, int B, const int *__rest
     off = s_red[0][0];
     base = s_red[1][0];
     const int nb_seq = seqcount[b], s1 = scu[b + 1];
-    if (b == B - 1 && threadIdx.x == 0) hdr->st[s].nb = base + nb_seq;
+    if (b == B - 1 && threadIdx.x == 0 && blockIdx.y == 0) hdr->st[s].nb = base + nb_seq;
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
     long long vis = 0;
-    for (int i = w; i < nb_seq; i += nw) {
+    for (int i = blockIdx.y * nw + w; i < nb_seq; i += nw * gridDim.y) {   // grid.y CTAs share a sequence
         const int r0 = bstart[off + i];
         const int r1 = (i + 1 < nb_seq) ? bstart[off + i + 1] : s1;
         int a = INT_MAX, bb = INT_MIN, carry = 0;
@@ -389,63 +394,294 @@ __global__ void k_blocks(DevHeader *hdr, int s, int bm, int B, const int *__rest
 
 // Rank sort: queue[rank] = block id, cost descending, id ascending.  queue_split: the same order
 // inside two groups, blocks that are SELF and not EMPTY first (n_fused of them), then the others.
-__global__ void k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost,
-                        const int *__restrict__ blocks, int *queue, int *queue_split) {
+__global__ void __launch_bounds__(256)
+k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost, const int *__restrict__ blocks, int *queue,
+        int *queue_split) {
+    // sort key of a block: (cost << 1 | eligible); tiles of keys go through shared memory
+    __shared__ long long s_key[1024];
     const int nb = hdr->st[s].nb;
+    const int ntile = (nb + 1023) / 1024;
     int mine = 0;
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < nb; i += gridDim.x * blockDim.x) {
-        const long long ci = cost[i];
-        const int fi = blocks[5 * i + 4];
-        const int ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
-        int rank = 0, rank2 = 0;
-        for (int j = 0; j < nb; ++j) {
-            const long long cj = cost[j];
-            const int fj = blocks[5 * j + 4];
-            const int ej = ((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0;
-            const int before = (cj > ci) || (cj == ci && j < i);
-            rank += before;
-            rank2 += (ej > ei) || (ej == ei && before);
+    for (int i0 = blockIdx.x * blockDim.x; i0 < nb; i0 += gridDim.x * blockDim.x) {   // same trip count in the CTA
+        const int i = i0 + threadIdx.x;
+        long long ci = 0;
+        int ei = 0;
+        if (i < nb) {
+            ci = cost[i];
+            const int fi = blocks[5 * i + 4];
+            ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
         }
-        queue[rank] = i;
-        queue_split[rank2] = i;
-        mine += ei;
+        int rank = 0, rank2 = 0;
+        for (int tl = 0; tl < ntile; ++tl) {
+            __syncthreads();
+            for (int j = threadIdx.x; j < 1024; j += blockDim.x) {
+                const int jj = tl * 1024 + j;
+                if (jj < nb) {
+                    const int fj = blocks[5 * jj + 4];
+                    s_key[j] = (cost[jj] << 1) | (((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0);
+                }
+            }
+            __syncthreads();
+            const int lim = min(1024, nb - tl * 1024);
+            if (i < nb) {
+                for (int j = 0; j < lim; ++j) {
+                    const long long kj = s_key[j];
+                    const long long cj = kj >> 1;
+                    const int ej = (int)(kj & 1);
+                    const int before = (cj > ci) || (cj == ci && tl * 1024 + j < i);
+                    rank += before;
+                    rank2 += (ej > ei) || (ej == ei && before);
+                }
+            }
+        }
+        if (i < nb) {
+            queue[rank] = i;
+            queue_split[rank2] = i;
+            mine += ei;
+        }
     }
     if (mine) atomicAdd(&hdr->st[s].n_fused, mine);
+}
+
+// ---------------------------------------------------------------------------------------------
+// All stages above 0 in one CTA.  Their arrays are a few percent of the tokens, so a single CTA
+// with block-wide barriers between the steps replaces eight launches per stage.
+// ---------------------------------------------------------------------------------------------
+struct UpperArgs {
+    StagePtrs st[HDT_MAX_STAGES];
+    int max_stages, B, bm;
+    int *cnt, *nlc, *pre, *bstart, *seqcount;
+    uint8_t *keep, *fpos;
+    long long *cost;
+};
+
+static constexpr int UT = 1024;      // threads of the fused kernel
+static constexpr int UMAXB = 1024;   // sequences it handles (per-sequence offsets live in shared memory)
+
+__global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const UpperArgs u) {
+    __shared__ int s_off[UMAXB], s_base[UMAXB];
+    __shared__ int s_w[32];
+    __shared__ int s_carry, s_flag;
+    __shared__ long long s_ll[32];
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    const int B = u.B, bm = u.bm;
+    for (int s = 1; s < u.max_stages; ++s) {
+        const int n = hdr->st[s].n;      // written by the previous stage, same value in every thread
+        if (n == 0) break;
+        const StagePtrs P = u.st[s];
+        const bool last = (s + 1 == u.max_stages);
+        const StagePtrs N = u.st[last ? s : s + 1];
+        // children counts (cnt, nlc are zero for [0, n))
+        for (int e = t; e < n; e += UT) { const int p = P.par[e]; if (p >= 0) atomicAdd(&u.cnt[p], 1); }
+        if (t == 0) { s_flag = 0; s_carry = 0; }
+        __syncthreads();
+        for (int e = t; e < n; e += UT) { const int p = P.par[e]; if (p >= 0 && u.cnt[e] > 0) atomicAdd(&u.nlc[p], 1); }
+        __syncthreads();
+        // ranges, keep flags
+        long long deg = 0;
+        for (int e = t; e < n; e += UT) {
+            const int p = P.par[e], c = u.cnt[e];
+            const bool head = (c > 0 && u.nlc[e] == 0);
+            int lo = 0, hi = 0, fp = 0, kp = 1;
+            if (head) {
+                lo = (p < 0) ? e : e + 1;
+                hi = e + 1 + c;
+            } else if (p >= 0) {
+                const int cp = u.cnt[p];
+                if (cp > 0 && u.nlc[p] == 0) {
+                    if (!(p < e && e <= p + cp)) dev_fail(hdr, HDT_ERR_BAD_HIERARCHY, e);
+                    lo = p; hi = p + 1 + cp; fp = min(e - p, 255); kp = 0;
+                }
+            }
+            P.rng[2 * e] = lo;
+            P.rng[2 * e + 1] = hi;
+            u.keep[e] = (uint8_t)kp;
+            u.fpos[e] = (uint8_t)fp;
+            deg += hi - lo;
+            if (kp && p >= 0) s_flag = 1;
+        }
+        for (int o = 16; o; o >>= 1) deg += __shfl_xor_sync(0xffffffffu, deg, o);
+        if (lane == 0) s_ll[w] = deg;
+        __syncthreads();
+        if (t == 0) {
+            long long d = 0;
+            for (int i = 0; i < UT / 32; ++i) d += s_ll[i];
+            if (d) atomicAdd((unsigned long long *)&hdr->nnz, (unsigned long long)d);
+            hdr->st[s].has_next = s_flag;
+        }
+        const int has_next = s_flag;
+        // exclusive scan of keep[] in chunks of UT
+        for (int base = 0; base < n; base += UT) {
+            const int e = base + t;
+            const int kp = (e < n) ? u.keep[e] : 0;
+            int v = kp;
+            for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
+            if (lane == 31) s_w[w] = v;
+            __syncthreads();
+            if (w == 0) {
+                int x = s_w[lane];
+                for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
+                s_w[lane] = x;
+            }
+            __syncthreads();
+            const int excl = s_carry + (w ? s_w[w - 1] : 0) + v - kp;
+            if (e < n) {
+                u.pre[e] = excl;
+                const int up = (kp && has_next) ? excl : -1;
+                P.up[e] = up;
+                if (up >= 0 && !last) N.tok[up] = P.tok[e];
+            }
+            __syncthreads();
+            if (t == 0) s_carry += s_w[31];
+            __syncthreads();
+        }
+        const int n2 = has_next ? s_carry : 0;
+        if (t == 0) hdr->st[s + 1].n = n2;
+        // next stage's parents and sequence offsets; clear cnt / nlc for it
+        if (!last) {
+            for (int e = t; e < n; e += UT) {
+                const int up = P.up[e];
+                if (up >= 0) { const int p = P.par[e]; N.par[up] = (p >= 0) ? u.pre[p] : -1; }
+            }
+            for (int b = t; b <= B; b += UT) {
+                const int x = P.scu[b];
+                N.scu[b] = (n2 > 0) ? ((x < n) ? u.pre[x] : n2) : 0;
+            }
+        }
+        __syncthreads();   // every cnt / nlc / pre read of this stage is done
+        for (int e = t; e < max(n2, 0); e += UT) { u.cnt[e] = 0; u.nlc[e] = 0; }
+        // per-sequence capacity offsets, greedy walk (one lane per sequence)
+        for (int b = t; b < B; b += UT) {
+            int off = 0;
+            for (int c = 0; c < b; ++c) off += 2 * ((P.scu[c + 1] - P.scu[c] + bm - 1) / bm) + 2;
+            s_off[b] = off;
+        }
+        __syncthreads();
+        for (int b = w; b < B; b += UT / 32) {
+            if (lane == 0) {
+                const int s0 = P.scu[b], len = P.scu[b + 1] - s0, off = s_off[b];
+                int pos = 0, cntb = 0;
+                while (pos < len) {
+                    int end = min(pos + bm, len);
+                    if (end < len) {
+                        const int f = u.fpos[s0 + end];
+                        if (f >= 1 && f < end - pos) end -= f;
+                    }
+                    u.bstart[off + cntb] = s0 + pos;
+                    ++cntb;
+                    pos = end;
+                }
+                u.seqcount[b] = cntb;
+            }
+        }
+        __syncthreads();
+        for (int b = t; b < B; b += UT) {
+            int base = 0;
+            for (int c = 0; c < b; ++c) base += u.seqcount[c];
+            s_base[b] = base;
+            if (b == B - 1) hdr->st[s].nb = base + u.seqcount[b];
+        }
+        __syncthreads();
+        // block records, one warp per block
+        long long vis = 0;
+        for (int b = 0; b < B; ++b) {
+            const int nb_seq = u.seqcount[b], off = s_off[b], base = s_base[b], s1 = P.scu[b + 1];
+            for (int i = w; i < nb_seq; i += UT / 32) {
+                const int r0 = u.bstart[off + i];
+                const int r1 = (i + 1 < nb_seq) ? u.bstart[off + i + 1] : s1;
+                int a = 0x7fffffff, bb = (int)0x80000000, carry = 0;
+                for (int e = r0 + lane; e < r1; e += 32) {
+                    const int lo = P.rng[2 * e], hi = P.rng[2 * e + 1];
+                    if (hi > lo) { a = min(a, lo); bb = max(bb, hi); }
+                    if (P.up[e] >= 0) carry = 1;
+                }
+                for (int o = 16; o; o >>= 1) {
+                    a = min(a, __shfl_xor_sync(0xffffffffu, a, o));
+                    bb = max(bb, __shfl_xor_sync(0xffffffffu, bb, o));
+                    carry |= __shfl_xor_sync(0xffffffffu, carry, o);
+                }
+                const bool any = bb > a;
+                if (!any) { a = r0; bb = r0; }
+                int dense = 1;
+                for (int e = r0 + lane; e < r1; e += 32)
+                    if (P.rng[2 * e] != a || P.rng[2 * e + 1] != bb) dense = 0;
+                for (int o = 16; o; o >>= 1) dense &= __shfl_xor_sync(0xffffffffu, dense, o);
+                if (lane == 0) {
+                    int fl = 0;
+                    if (a >= r0 && bb <= r1) fl |= HDT_BLK_SELF;
+                    if (dense && any) fl |= HDT_BLK_DENSE;
+                    if (carry) fl |= HDT_BLK_CARRY;
+                    if (!any) fl |= HDT_BLK_EMPTY;
+                    int *rec = P.blocks + 5 * (size_t)(base + i);
+                    rec[0] = r0; rec[1] = r1; rec[2] = a; rec[3] = bb; rec[4] = fl;
+                    const long long c = (long long)(r1 - r0) * (long long)(bb - a);
+                    u.cost[base + i] = c;
+                    vis += c;
+                }
+            }
+        }
+        if (lane == 0 && vis) atomicAdd((unsigned long long *)&hdr->visited, (unsigned long long)vis);
+        __syncthreads();
+        // queues
+        const int nb = (B > 0) ? s_base[B - 1] + u.seqcount[B - 1] : 0;
+        int mine = 0;
+        for (int i = t; i < nb; i += UT) {
+            const long long ci = u.cost[i];
+            const int fi = P.blocks[5 * i + 4];
+            const int ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
+            int rank = 0, rank2 = 0;
+            for (int j = 0; j < nb; ++j) {
+                const long long cj = u.cost[j];
+                const int fj = P.blocks[5 * j + 4];
+                const int ej = ((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0;
+                const int before = (cj > ci) || (cj == ci && j < i);
+                rank += before;
+                rank2 += (ej > ei) || (ej == ei && before);
+            }
+            P.queue[rank] = i;
+            P.queue_split[rank2] = i;
+            mine += ei;
+        }
+        if (mine) atomicAdd(&hdr->st[s].n_fused, mine);
+        __syncthreads();   // hdr->st[s+1].n and everything else is visible before the next stage reads it
+    }
 }
 
 }  // namespace hdt
 
 using namespace hdt;
 
-static void norm_params(const hdt_index_params_t *p, int &bm, int &ms) {
+static void norm_params(const hdt_index_params_t *p, int &bm, int &ms, int &bmu) {
     bm = (p && p->block_m) ? p->block_m : 128;
     ms = (p && p->max_stages) ? p->max_stages : 4;
+    bmu = (p && p->block_m_upper) ? p->block_m_upper : 32;
 }
 
 extern "C" size_t hdt_index_workspace_bytes(int32_t batch, int32_t total_tokens,
                                             const hdt_index_params_t *params) {
-    int bm, ms;
-    norm_params(params, bm, ms);
-    if (batch < 0 || total_tokens < 0 || bm < 1 || bm > 128 || ms < 1 || ms > HDT_MAX_STAGES) return 0;
-    return make_layout(batch, total_tokens, bm, ms).total;
+    int bm, ms, bmu;
+    norm_params(params, bm, ms, bmu);
+    if (batch < 0 || total_tokens < 0 || bm < 1 || bm > 128 || bmu < 1 || bmu > 128 || ms < 1 || ms > HDT_MAX_STAGES)
+        return 0;
+    return make_layout(batch, total_tokens, min(bm, bmu), ms).total;
 }
 
 extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const int32_t *cu_seqlens,
                                int32_t batch, int32_t total_tokens, const hdt_index_params_t *params,
                                void *workspace, size_t workspace_bytes, void *stream, hdt_index_t **out) {
     if (out) *out = nullptr;
-    int bm, ms;
-    norm_params(params, bm, ms);
+    int bm, ms, bmu;
+    norm_params(params, bm, ms, bmu);
     if (!out || !cu_seqlens || !workspace || batch < 0 || total_tokens < 0 ||
         (total_tokens > 0 && (!level || !parent)))
         return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: null pointer or negative size");
-    if (bm < 1 || bm > 128 || ms < 1 || ms > HDT_MAX_STAGES)
-        return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: block_m must be 1..128, max_stages 1..%d",
+    if (bm < 1 || bm > 128 || bmu < 1 || bmu > 128 || ms < 1 || ms > HDT_MAX_STAGES)
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: block_m, block_m_upper must be 1..128, max_stages 1..%d",
                          HDT_MAX_STAGES);
     if (((uintptr_t)workspace & 255) != 0)
         return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: workspace must be 256-byte aligned");
     const int B = batch, T = total_tokens;
-    const Layout L = make_layout(B, T, bm, ms);
+    const Layout L = make_layout(B, T, min(bm, bmu), ms);
     if (workspace_bytes < L.total)
         return set_error(HDT_ERR_WORKSPACE, "hdt_build_index: workspace %zu < required %zu", workspace_bytes,
                          L.total);
@@ -459,7 +695,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     long long *cost = (long long *)(ws + L.cost);
 
     hdt_index *ix = new hdt_index();
-    ix->batch = B; ix->total_tokens = T; ix->block_m = bm; ix->n_stages = 0;
+    ix->batch = B; ix->total_tokens = T; ix->block_m = bm; ix->block_m_upper = bmu; ix->n_stages = 0;
     ix->workspace = workspace; ix->workspace_bytes = workspace_bytes;
     for (int s = 0; s < ms; ++s) {
         char *base = ws + L.stage0 + L.stage_stride * (size_t)s;
@@ -478,26 +714,34 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
 
     {
     ProfScope ps(PROF_INDEX, st);
-    HDT_BUILD_CHECK(cudaMemsetAsync(hdr, 0, sizeof(DevHeader), st));
+    // header, cnt and nlc are adjacent in the workspace: one memset clears all three
+    HDT_BUILD_CHECK(cudaMemsetAsync(ws + L.header, 0, L.pre - L.header, st));
     const int nel = max(T, B + 1);
     const int g_el = (nel + 255) / 256;
     const int g_chunk = max(1, (T + CHUNK - 1) / CHUNK);
     const int g_stride = max(1, min((T + 255) / 256, 148 * 8));
     static const int kSmemCap = 200 * 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
-        attr_set = true;
-    }
+    HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
     k_init<<<g_el, 256, 0, st>>>(level, parent, cu_seqlens, B, T, HDT_MAX_STAGES * 8, hdr, ix->st[0].tok,
-                                 ix->st[0].par, ix->st[0].scu, cnt, nlc);
+                                 ix->st[0].par, ix->st[0].scu, cnt);
     count_launch();
+    const bool fused_upper = (B <= UMAXB);
     for (int s = 0; s < ms; ++s) {
+        if (s >= 1 && fused_upper) {
+            UpperArgs u;
+            for (int i = 0; i < HDT_MAX_STAGES; ++i) u.st[i] = ix->st[i < ms ? i : ms - 1];
+            u.max_stages = ms; u.B = B; u.bm = bmu;
+            u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.bstart = bstart; u.seqcount = seqcount;
+            u.keep = keep; u.fpos = fpos; u.cost = cost;
+            k_upper_stages<<<1, UT, 0, st>>>(hdr, u);
+            count_launch();
+            break;
+        }
         const StagePtrs &P = ix->st[s];
         // the last possible stage writes its (unused) next-stage arrays into its own up/pre scratch
         const StagePtrs &N = ix->st[(s + 1 < ms) ? s + 1 : s];
         const bool last = (s + 1 == ms);
-        k_count<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt);
+        if (s >= 1) { k_count<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt); count_launch(); }
         k_nlc<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt, nlc);
         k_ranges<<<g_chunk, CHUNK, 0, st>>>(hdr, s, s == 0 ? level : nullptr, P.par, cnt, nlc, P.rng, keep,
                                             fpos, blocksum);
@@ -510,12 +754,14 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         }
         if (B > 0) {
             int maxlen_smem = kSmemCap;  // sequences longer than this walk through global memory
-            k_walk<<<B, 256, kSmemCap, st>>>(hdr, s, bm, P.scu, fpos, bstart, seqcount, maxlen_smem);
-            k_blocks<<<B, 256, 0, st>>>(hdr, s, bm, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost);
-            k_queue<<<max(1, min(L.capnb / 128 + 1, 148 * 4)), 128, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
+            const int bms = (s == 0) ? bm : bmu;
+            k_walk<<<B, 256, kSmemCap, st>>>(hdr, s, bms, P.scu, fpos, bstart, seqcount, maxlen_smem);
+            const int gy = max(1, min(64, 2048 / max(B, 1)));   // enough CTAs to spread a few long sequences
+            k_blocks<<<dim3(B, gy), 256, 0, st>>>(hdr, s, bms, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost);
+            k_queue<<<max(1, min(L.capnb / 256 + 1, 148 * 4)), 256, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
             count_launch(3);
         }
-        count_launch(4);
+        count_launch(3);
     }
     HDT_BUILD_CHECK(cudaGetLastError());
     }

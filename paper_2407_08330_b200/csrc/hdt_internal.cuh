@@ -32,7 +32,7 @@ struct StagePtrs {
 }  // namespace hdt
 
 struct hdt_index {
-    int batch, total_tokens, block_m, n_stages;
+    int batch, total_tokens, block_m, block_m_upper, n_stages;
     long long nnz, visited;
     hdt::StageDesc desc[HDT_MAX_STAGES + 1];
     hdt::StagePtrs st[HDT_MAX_STAGES];
@@ -88,6 +88,7 @@ struct FwdStageArgs {
     int *status;        // device failure word
     int rest_only;      // general kernel: only blocks after the first n_fused
     int no_persistent;  // option: do not use the persistent kernels
+    int block_rows;     // max rows of a block in this stage
 };
 
 struct BwdStageArgs {
@@ -106,6 +107,7 @@ struct BwdStageArgs {
     int *status;                                  // device failure word
     int rest_only;                                // general kernel: only blocks after the first n_fused
     int no_persistent;                            // option: do not use the persistent kernels
+    int block_rows;                               // max rows of a block in this stage
 };
 
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);

@@ -19,9 +19,9 @@ def P():
     return P
 
 
-def assert_index_equal(P, b, block_m=128, max_stages=8):
-    want = ix.build(b.level, b.parent, b.cu_seqlens, block_m)
-    idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=max_stages)
+def assert_index_equal(P, b, block_m=128, max_stages=8, block_m_upper=32):
+    want = ix.build(b.level, b.parent, b.cu_seqlens, block_m, block_m_upper=block_m_upper)
+    idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=max_stages, block_m_upper=block_m_upper)
     assert idx.n_stages == len(want.stages)
     assert idx.nnz == want.nnz and idx.visited == want.visited
     for s, st in enumerate(want.stages):
@@ -41,6 +41,7 @@ def test_index_small_documents(P, block_m):
     for seed in range(10):
         b = gen.small_random_batch(seed, n_seqs=4, max_len=400)
         assert_index_equal(P, b, block_m)
+        assert_index_equal(P, b, 128, block_m_upper=block_m)
 
 
 def test_index_generic_trees_and_degenerate(P):
@@ -57,6 +58,13 @@ def test_index_generic_trees_and_degenerate(P):
     # empty batch and batch of one empty sequence
     assert_index_equal(P, gen.pack([]))
     assert_index_equal(P, gen.pack([(np.zeros(0, np.int8), np.zeros(0, np.int32))]))
+
+
+def test_index_many_sequences(P):
+    """More sequences than the single-CTA upper-stage builder takes: the per-stage kernels run."""
+    rng = np.random.default_rng(12)
+    seqs = [gen.gen_fill(rng, int(rng.integers(3, 40)), (1, 3), (1, 3), (0, 6))[:2] for _ in range(1100)]
+    assert_index_equal(P, gen.pack(seqs), 128, max_stages=4)
 
 
 @pytest.mark.parametrize("c", [1, 2, 3, 4, 5])

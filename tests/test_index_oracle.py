@@ -69,9 +69,11 @@ def check_structure(b, idx, block_m):
 def test_documents(block_m):
     for seed in range(12):
         b = gen.small_random_batch(seed, n_seqs=3, max_len=160)
-        idx = ix.build(b.level, b.parent, b.cu_seqlens, block_m)
+        idx = ix.build(b.level, b.parent, b.cu_seqlens, block_m, block_m_upper=block_m)
         check_structure(b, idx, block_m)
         assert len(idx.stages) <= 3
+        idx = ix.build(b.level, b.parent, b.cu_seqlens, 128, block_m_upper=block_m)
+        check_structure(b, idx, 128)
 
 
 def test_three_stages_on_config1_and_family_alignment():
@@ -104,7 +106,7 @@ def test_generic_trees_and_degenerate_documents():
     seqs.append(gen.layout([[300, 2], [1]]))                                        # family longer than a block
     b = gen.pack(seqs)
     for bm in (128, 7):
-        idx = ix.build(b.level, b.parent, b.cu_seqlens, bm)
+        idx = ix.build(b.level, b.parent, b.cu_seqlens, bm, block_m_upper=bm)
         check_structure(b, idx, bm)
 
 
