@@ -250,6 +250,10 @@ int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N, int32_t K,
  * Synchronises the device and resets the counters.
  */
 int hdt_debug_bwd_phase_cycles(int64_t *out16);
+/* The same for the persistent forward kernel: out16[0..11] = prefetch issue, wait for S, row maximum,
+ * barriers (max exchange), P arithmetic and stores, barrier, MMA issue, wait for O, drain, loop top,
+ * barrier, output stores; out16[12] = items processed. */
+int hdt_debug_fwd_phase_cycles(int64_t *out16);
 
 #ifdef __cplusplus
 }

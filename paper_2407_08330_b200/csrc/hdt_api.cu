@@ -198,6 +198,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         }
         a.o = o; a.lse = lse;
         a.status = status;
+        a.no_persistent = g_no_persistent;
         {
             ProfScope ps(s == 0 ? PROF_FWD_STAGE0 : PROF_FWD_UPPER, st);
             if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
@@ -340,6 +341,7 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
         }
         a.o = o; a.lse = lse;
         a.status = status;
+        a.no_persistent = g_no_persistent;
         if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
         else rc = launch_fwd_simt(a, head_dim, dtype, st);
         if (rc) return rc;

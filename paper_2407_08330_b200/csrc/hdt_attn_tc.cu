@@ -28,25 +28,31 @@ static constexpr long long WAIT_CYCLES = 400000000LL;  // ~0.2 s: bound of every
 // byte offset of 16-byte chunk c (0..7) of row r inside a swizzled sub-tile
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
-template <int D>
+// SINGLE = true: the block has one key chunk (SELF blocks).  Q and K are dead once S is computed and
+// S is dead once P is written, so P reuses the Q/K tiles and O reuses S's TMEM columns: 48 KB of
+// shared memory and 128 TMEM columns per CTA at D = 64, four CTAs per SM.
+template <int D, bool SINGLE>
 __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensorMap tm_q,
                                                 const __grid_constant__ CUtensorMap tm_k,
                                                 const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
     constexpr int NSUB = D / 64;
-    constexpr uint32_t TM_S = 0, TM_O = 128, TM_COLS = 256;
+    constexpr uint32_t TM_S = 0, TM_O = SINGLE ? 0 : 128, TM_COLS = SINGLE ? 128 : 256;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = sm;                       // NSUB sub-tiles; reused to stage O
     uint8_t *sK = sQ + NSUB * SUB;
     uint8_t *sV = sK + NSUB * SUB;
-    uint8_t *sP = sV + NSUB * SUB;          // 2 sub-tiles (128 keys)
-    uint64_t *bar_tma = (uint64_t *)(sP + 2 * SUB);
+    uint8_t *sP = SINGLE ? sQ : sV + NSUB * SUB;   // 2 sub-tiles (128 keys)
+    uint64_t *bar_tma = (uint64_t *)((SINGLE ? sV + NSUB * SUB : sP + 2 * SUB));
     uint64_t *bar_mma = bar_tma + 1;
     uint32_t *slot = (uint32_t *)(bar_mma + 1);
     volatile int *abort_flag = (volatile int *)(slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int blk = a.queue[blockIdx.x], h = blockIdx.y, H = a.H;
+    // SINGLE: the first n_fused entries of queue_split; rest_only: the blocks after them
+    const int blk = SINGLE ? a.queue_split[blockIdx.x]
+                           : (a.rest_only ? a.queue_split[a.n_fused + blockIdx.x] : a.queue[blockIdx.x]);
+    const int h = blockIdx.y, H = a.H;
     const int *rec = a.blocks + 5 * (size_t)blk;
     const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3], fl = rec[4];
     const float NEG = -INFINITY, LN2 = 0.6931471805599453f;
@@ -247,6 +253,269 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
+
+// Cycle counts per phase of k_fwd_tc_p, accumulated by thread 0 of CTA 0 (diagnostics).
+__device__ long long g_fwd_phase_cycles[16];
+#define HDT_STAMP(i)                                        \
+    do {                                                    \
+        if (stamp) {                                        \
+            const long long now_ = clock64();               \
+            ph_acc[i] += now_ - t_last;                     \
+            t_last = now_;                                  \
+        }                                                   \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// Persistent, software-pipelined forward for blocks that are SELF and not EMPTY at D = 64.
+// One CTA of 512 threads per SM walks its share of the (block, head) items in queue_split order.
+// Q/K/V of the next two items are in flight or resident (double-buffered TMA); S of item i+1 is
+// issued together with O = P V of item i and runs while the CTA drains O.
+// Thread t: row t % 128 (TMEM lane), column quarter t / 128; the four threads of a row exchange
+// their partial row maximum and row sum through shared memory.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(512, 1) k_fwd_tc_p(const __grid_constant__ CUtensorMap tm_q,
+                                                     const __grid_constant__ CUtensorMap tm_k,
+                                                     const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
+    constexpr int D = 64;
+    constexpr uint32_t TM_S = 0, TM_O = 128, TM_COLS = 256;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sIn = sm;                    // 2 stages x {Q, K, V}
+    uint8_t *sP = sm + 6 * SUB;           // 2 sub-tiles; reused to stage O (rows padded to 144 bytes) once P V is done
+    float *s_red = (float *)(sP + 2 * SUB);              // [4][128] partial row max, then partial row sums
+    uint64_t *bar_tma = (uint64_t *)(s_red + 4 * 128);   // [2]
+    uint64_t *bar_s = bar_tma + 2, *bar_o = bar_tma + 3;
+    uint32_t *slot = (uint32_t *)(bar_tma + 4);
+    volatile int *abort_flag = (volatile int *)(slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, qt = tid >> 7;
+    const int H = a.H, G = gridDim.x;
+    const int n_items = a.n_fused * H;
+    const int my_count = ((int)blockIdx.x < n_items) ? (n_items - (int)blockIdx.x + G - 1) / G : 0;
+    const float NEG = -INFINITY, LN2 = 0.6931471805599453f;
+
+    if (tid == 0) {
+        mbar_init(&bar_tma[0], 1);
+        mbar_init(&bar_tma[1], 1);
+        mbar_init(bar_s, 1);
+        mbar_init(bar_o, 1);
+        *abort_flag = (*a.status != 0);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    bool ok = true;
+
+    struct Desc { int r0, r1, h; };
+    auto load_blk = [&](int i) { return a.queue_split[((int)blockIdx.x + i * G) / H]; };
+    auto load_rec = [&](int i, int blk) {
+        Desc d;
+        d.h = ((int)blockIdx.x + i * G) % H;
+        d.r0 = a.blocks[5 * (size_t)blk];
+        d.r1 = a.blocks[5 * (size_t)blk + 1];
+        return d;
+    };
+    struct RowStat { int lo, hi, up; };
+    auto load_stat = [&](const Desc &d) {
+        RowStat r{0, 0, -1};
+        const int row = d.r0 + rl;
+        if (row < d.r1) {
+            r.lo = a.rng[2 * row];
+            r.hi = a.rng[2 * row + 1];
+            if (a.part_o != nullptr) r.up = a.up[row];
+        }
+        return r;
+    };
+    auto issue_tma = [&](int i, const Desc &d) {       // thread 0
+        uint8_t *st = sIn + (i & 1) * 3 * SUB;
+        uint64_t *bar = &bar_tma[i & 1];
+        mbar_expect_tx(bar, 3 * SUB);
+        tma_load_3d(st, &tm_q, 0, d.h, d.r0, bar);
+        tma_load_3d(st + SUB, &tm_k, 0, d.h, d.r0, bar);
+        tma_load_3d(st + 2 * SUB, &tm_v, 0, d.h, d.r0, bar);
+    };
+    auto issue_s = [&](int i, int Nc) {   // one thread; inputs of item i have landed
+        const uint32_t st = smem_u32(sIn + (i & 1) * 3 * SUB);
+        const uint32_t idesc = idesc_bf16(Nc, false, false);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss(tmem + TM_S, smem_desc(st + kk * 32, 0, 1024), smem_desc(st + SUB + kk * 32, 0, 1024), idesc, kk > 0);
+        mma_commit(bar_s);
+    };
+
+    if (!dead && my_count > 0) {
+        Desc dc = load_rec(0, load_blk(0)), dn = dc, dn2 = dc;
+        if (my_count > 1) dn = load_rec(1, load_blk(1));
+        int blk2 = (my_count > 2) ? load_blk(2) : 0;
+        RowStat rc = load_stat(dc), rn = rc;
+        if (tid == 0) {
+            issue_tma(0, dc);
+            if (my_count > 1) issue_tma(1, dn);
+            ok = mbar_wait(&bar_tma[0], 0, abort_flag, WAIT_CYCLES) && ok;
+            if (!*abort_flag) {
+                tc_fence_after();
+                issue_s(0, (dc.r1 - dc.r0 + 15) & ~15);
+            }
+        }
+        const bool stamp = (tid == 0 && blockIdx.x == 0);
+        long long ph_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
+        long long t_last = clock64();
+        for (int it = 0; it < my_count; ++it) {
+            HDT_STAMP(9);
+            if (it + 2 < my_count) dn2 = load_rec(it + 2, blk2);
+            if (it + 3 < my_count) blk2 = load_blk(it + 3);
+            if (it + 1 < my_count) rn = load_stat(dn);
+            const int r0 = dc.r0, r1 = dc.r1, h = dc.h;
+            const int nrows = r1 - r0, Nc = (nrows + 15) & ~15;
+            const bool inb = r0 + rl < r1;
+            const int jl = max(rc.lo - r0, 0), jh = min(rc.hi - r0, nrows);
+            const bool has = inb && jh > jl;
+            uint8_t *st = sIn + (it & 1) * 3 * SUB;
+
+            HDT_STAMP(0);
+            if (warp == 0) ok = mbar_wait(bar_s, it & 1, abort_flag, WAIT_CYCLES) && ok;   // S of this item
+            __syncthreads();   // also: the previous item's staged O has been stored
+            tc_fence_after();
+            HDT_STAMP(1);
+            // ---- this thread's 32 columns of S, kept in registers across both passes ----
+            const int s0 = 32 * qt;
+            const bool active = s0 < Nc;                       // same in the whole warp
+            const bool mine = has && jl < s0 + 32 && jh > s0;
+            uint32_t sv[32];
+            bool loaded = false;
+            float mx = NEG;
+            if (active && __any_sync(0xffffffffu, mine)) {
+                tmem_ld32(tmem + TM_S + lane_base + s0, sv);
+                tmem_wait_ld();
+                loaded = true;
+                if (mine) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (s0 + j >= jl && s0 + j < jh) mx = fmaxf(mx, __uint_as_float(sv[j]));
+                }
+            }
+            s_red[qt * 128 + rl] = mx;
+            HDT_STAMP(2);
+            __syncthreads();
+            const float mrow = fmaxf(fmaxf(s_red[rl], s_red[128 + rl]), fmaxf(s_red[256 + rl], s_red[384 + rl])) * a.scale_log2;
+            __syncthreads();   // every thread has read the maxima before the sums overwrite them
+            HDT_STAMP(3);
+            float lsum = 0.f;
+            if (active) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[j] = 0u;
+                if (loaded && mine) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float p0 = 0.f, p1 = 0.f;
+                        if (s0 + j >= jl && s0 + j < jh) p0 = exp2f(fmaf(__uint_as_float(sv[j]), a.scale_log2, -mrow));
+                        if (s0 + j + 1 >= jl && s0 + j + 1 < jh) p1 = exp2f(fmaf(__uint_as_float(sv[j + 1]), a.scale_log2, -mrow));
+                        const uint32_t u = pack_bf16(p0, p1);
+                        lsum += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
+                        pk[j >> 1] = u;
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<uint4 *>(sP + (qt >> 1) * SUB + swz(rl, (qt & 1) * 4 + c)) =
+                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            }
+            s_red[qt * 128 + rl] = lsum;
+            fence_proxy_async_smem();
+            tc_fence_before();
+            HDT_STAMP(4);
+            __syncthreads();
+            HDT_STAMP(5);
+            if ((tid & 31) == 0 && warp < 2 && !*abort_flag) {
+                tc_fence_after();
+                if (warp == 0) {   // O = P V
+                    const uint32_t idesc = idesc_bf16(D, false, true);
+                    const uint64_t da = smem_desc(smem_u32(sP), 0, 1024), db = smem_desc(smem_u32(st) + 2 * SUB, SUB, 1024);
+                    const int nk = Nc / 16;
+                    for (int kk = 0; kk < nk; ++kk)
+                        mma_ss(tmem + TM_O, da + (uint64_t)((kk / 4) * (SUB >> 4) + (kk % 4) * 2), db + (uint64_t)(kk * 128),
+                               idesc, kk > 0);
+                    mma_commit(bar_o);
+                } else if (it + 1 < my_count) {   // S of the next item runs during this item's drain
+                    ok = mbar_wait(&bar_tma[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag, WAIT_CYCLES) && ok;
+                    if (!*abort_flag) {
+                        tc_fence_after();
+                        issue_s(it + 1, (dn.r1 - dn.r0 + 15) & ~15);
+                    }
+                }
+            }
+            const float l = s_red[rl] + s_red[128 + rl] + s_red[256 + rl] + s_red[384 + rl];
+            HDT_STAMP(6);
+            if (warp == 0) ok = mbar_wait(bar_o, it & 1, abort_flag, WAIT_CYCLES) && ok;   // O of this item
+            __syncthreads();
+            tc_fence_after();
+            HDT_STAMP(7);
+            if (tid == 0 && it + 2 < my_count && !*abort_flag) issue_tma(it + 2, dn2);   // this stage is free again
+            // ---- drain: 16 columns of O per thread ----
+            {
+                float lse = NEG, w0 = 0.f;
+                if (l > 0.f) { w0 = 1.f / l; lse = (mrow + log2f(l)) * LN2; }
+                uint32_t r[16];
+                tmem_ld16(tmem + TM_O + lane_base + 16 * qt, r);
+                tmem_wait_ld();
+                float x[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) x[j] = (w0 > 0.f) ? __uint_as_float(r[j]) * w0 : 0.f;
+                if (rc.up >= 0) {   // this row lives on in the next stage: leave its fp32 partial there
+                    float4 *po = reinterpret_cast<float4 *>(a.part_o + ((size_t)rc.up * H + h) * D + 16 * qt);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) po[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+                    if (qt == 0) a.part_lse[(size_t)rc.up * H + h] = lse;
+                }
+                if (qt == 0 && inb) a.lse[(size_t)h * a.T + r0 + rl] = lse;
+                uint32_t pk[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) pk[j] = pack_bf16(x[2 * j], x[2 * j + 1]);
+                *reinterpret_cast<uint4 *>(sP + rl * 144 + qt * 32) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(sP + rl * 144 + qt * 32 + 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+            }
+            tc_fence_before();
+            HDT_STAMP(8);
+            __syncthreads();
+            HDT_STAMP(10);
+            // ---- coalesced stores: thread -> rows tid/8 and tid/8 + 64, 16-byte chunk tid%8 ----
+            {
+                const int rA = tid >> 3, c = tid & 7;
+                __nv_bfloat16 *g = reinterpret_cast<__nv_bfloat16 *>(a.o);
+                uint4 v0, v1;
+                if (rA < nrows) v0 = *reinterpret_cast<const uint4 *>(sP + rA * 144 + c * 16);
+                if (rA + 64 < nrows) v1 = *reinterpret_cast<const uint4 *>(sP + (rA + 64) * 144 + c * 16);
+                if (rA < nrows) *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + rA) * H + h) * D + c * 8) = v0;
+                if (rA + 64 < nrows) *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + rA + 64) * H + h) * D + c * 8) = v1;
+            }
+            HDT_STAMP(11);
+            dc = dn; dn = dn2; rc = rn;
+        }
+        if (stamp) {
+            for (int i = 0; i < 12; ++i) g_fwd_phase_cycles[i] += ph_acc[i];
+            g_fwd_phase_cycles[12] += my_count;
+        }
+    }
+    if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
+// Diagnostics: cycles CTA 0 of the persistent forward spent per phase since the last call.
+int read_fwd_phase_cycles(long long *out16) {
+    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out16, g_fwd_phase_cycles, sizeof(long long) * 16));
+    long long zero[16] = {0};
+    HDT_CUDA_CHECK(cudaMemcpyToSymbol(g_fwd_phase_cycles, zero, sizeof(zero)));
+    return HDT_OK;
+}
+
 template <int D>
 static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     CUtensorMap tq, tk, tv;
@@ -257,15 +526,40 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     rc = make_tmap_bf16(&tv, a.v, D, a.H, a.T, 128);
     if (rc) return rc;
     constexpr int smem = (3 * (D / 64) + 2) * SUB + 1024 + 64;
+    constexpr int smem_1 = 3 * (D / 64) * SUB + 1024 + 64;
     static bool attr = false;
     if (!attr) {
-        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                            8 * SUB + 4 * 128 * 4 + 1024 + 64));
         attr = true;
     }
-    dim3 grid(a.nb, a.H);
-    k_fwd_tc<D><<<grid, 128, smem, st>>>(tq, tk, tv, a);
-    count_launch();
-    HDT_CUDA_CHECK(cudaGetLastError());
+    FwdStageArgs b = a;
+    b.rest_only = 0;
+    int n_general = a.nb;
+    if (a.n_fused > 0 && a.no_persistent != 1) {
+        if (D == 64 && a.no_persistent == 2) {   // option: the persistent single-CTA-per-SM kernel
+            constexpr int smem_p = 8 * SUB + 4 * 128 * 4 + 1024 + 64;
+            int dev = 0, n_sm = 0;
+            HDT_CUDA_CHECK(cudaGetDevice(&dev));
+            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+            const long long items = (long long)a.n_fused * a.H;
+            k_fwd_tc_p<<<(int)(items < n_sm ? items : n_sm), 512, smem_p, st>>>(tq, tk, tv, a);
+        } else {
+            k_fwd_tc<D, true><<<dim3(a.n_fused, a.H), 128, smem_1, st>>>(tq, tk, tv, a);
+        }
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+        b.rest_only = 1;
+        n_general = a.nb - a.n_fused;
+    }
+    if (n_general > 0) {
+        dim3 grid(n_general, a.H);
+        k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+    }
     return HDT_OK;
 }
 

@@ -103,6 +103,12 @@ extern "C" int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N,
 // Diagnostics (no counterpart in the paper): SM cycles that CTA 0 of the persistent backward kernel
 // spent in each of its phases since the last call (out16[0..11]) and the items it processed (out16[12]).
 // Waits for the device.
+extern "C" int hdt_debug_fwd_phase_cycles(int64_t *out16) {
+    if (!out16) return set_error(HDT_ERR_INVALID_ARG, "hdt_debug_fwd_phase_cycles: null pointer");
+    HDT_CUDA_CHECK(cudaDeviceSynchronize());
+    return read_fwd_phase_cycles((long long *)out16);
+}
+
 extern "C" int hdt_debug_bwd_phase_cycles(int64_t *out16) {
     if (!out16) return set_error(HDT_ERR_INVALID_ARG, "hdt_debug_bwd_phase_cycles: null pointer");
     HDT_CUDA_CHECK(cudaDeviceSynchronize());

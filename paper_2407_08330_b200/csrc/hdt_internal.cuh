@@ -115,6 +115,7 @@ int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t
 int launch_fwd_tc(const FwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_bwd_tc(const BwdStageArgs &a, int head_dim, cudaStream_t st);
 int read_bwd_phase_cycles(long long *out16);
+int read_fwd_phase_cycles(long long *out16);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
                  cudaStream_t st);

@@ -111,7 +111,8 @@ def test_index_rejects_bad_hierarchies(P):
 def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
     """bf16 runs three times: persistent + general tensor-core kernels, general tensor-core kernels
     only, SIMT kernels on every stage."""
-    opts = ({}, {"no_persistent": 1}, {"force_simt": 1}) if dtype == "bf16" else ({},)
+    # default kernels; general tensor-core kernels only; persistent forward; SIMT everywhere
+    opts = ({}, {"no_persistent": 1}, {"no_persistent": 2}, {"force_simt": 1}) if dtype == "bf16" else ({},)
     for opt in opts:
         for k_, v_ in opt.items():
             P.hdt_set_option(k_, v_)
