@@ -202,7 +202,7 @@ int hdt_profile_read(int32_t id, int64_t *launches, double *total_ms, int32_t re
  * synchronises the device) must not appear.  The call itself performs no cudaMalloc, cudaFree or
  * other allocating call.
  *  - Limit: hdt_attn_workspace_bytes(index, heads, head_dim, dtype, 0) must not exceed
- *    hdt_attn_fwd_static_max_bytes() (8 MiB, enough for about 2 000 anchor tokens x 16 heads x
+ *    hdt_attn_fwd_static_max_bytes() (8 MiB, enough for about 1 000 anchor tokens x 16 heads x
  *    head_dim 64); larger batches get HDT_ERR_WORKSPACE and a message that says so.  The array
  *    occupies that much memory on every GPU that loads the library, until the process exits.
  *  - The first call on each device looks up the array's device address (a CUDA runtime query);
@@ -220,7 +220,10 @@ int hdt_attn_fwd_static(const hdt_index_t *index, const void *q, const void *k, 
 
 /*
  * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
- * through the fp32 SIMT kernels instead of the tensor-core kernels (A/B comparisons, tests).
+ * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
+ * general tensor-core kernels, = 2 the persistent forward kernel; "no_overlap" = 1 runs the stages
+ * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream
+ * (A/B comparisons, tests).
  */
 int hdt_set_option(const char *name, int32_t value);
 

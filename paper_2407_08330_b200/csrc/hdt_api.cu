@@ -59,11 +59,33 @@ int *device_status_ptr() {
     return p;
 }
 
+// ---- side stream: the stages above 0 run beside stage 0 -------------------------------------------
+// One non-blocking stream and two events per host thread and device, created on first use.
+struct Side { cudaStream_t s; cudaEvent_t fork, join; bool ready; };
+static thread_local Side g_side[64];
+static int g_no_overlap = 0;
+
+static int get_side(Side **out) {
+    int dev = -1;
+    HDT_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return set_error(HDT_ERR_UNSUPPORTED, "device ordinal %d", dev);
+    Side &sd = g_side[dev];
+    if (!sd.ready) {
+        HDT_CUDA_CHECK(cudaStreamCreateWithFlags(&sd.s, cudaStreamNonBlocking));
+        HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.fork, cudaEventDisableTiming));
+        HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join, cudaEventDisableTiming));
+        sd.ready = true;
+    }
+    *out = &sd;
+    return HDT_OK;
+}
+
 static size_t al256(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct AttnLayout {
     size_t delta;                       // bwd only
-    size_t part[HDT_MAX_STAGES][4];     // fwd: o, lse;  bwd: dq, dk, dv
+    size_t part[HDT_MAX_STAGES][4];     // partials handed from stage s-1 to stage s.  fwd: o, lse;  bwd: dq, dk, dv
+    size_t own[HDT_MAX_STAGES][4];      // own partials of stage s when it is computed beside stage 0
     size_t total;
 };
 
@@ -76,6 +98,8 @@ static AttnLayout attn_layout(const hdt_index *ix, int H, int D, int bwd) {
         const int cnt = bwd ? 3 : 1;
         for (int c = 0; c < cnt; ++c) { L.part[s][c] = o; o += al256(sizeof(float) * n * H * D); }
         if (!bwd) { L.part[s][1] = o; o += al256(sizeof(float) * n * H); }
+        for (int c = 0; c < cnt; ++c) { L.own[s][c] = o; o += al256(sizeof(float) * n * H * D); }
+        if (!bwd) { L.own[s][1] = o; o += al256(sizeof(float) * n * H); }
     }
     L.total = o;
     return L;
@@ -106,6 +130,7 @@ static int g_no_persistent = 0;
 extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "force_simt") == 0) { g_force_simt = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_persistent") == 0) { g_no_persistent = value; return HDT_OK; }
+    if (name && std::strcmp(name, "no_overlap") == 0) { g_no_overlap = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 
@@ -178,7 +203,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
     char *ws = (char *)workspace;
     int *status = device_status_ptr();
     if (!status) return HDT_ERR_CUDA;
-    for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
+    auto stage_args = [&](int s) {
         const StagePtrs &P = ix->st[s];
         FwdStageArgs a{};
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
@@ -199,9 +224,36 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.o = o; a.lse = lse;
         a.status = status;
         a.no_persistent = g_no_persistent;
+        return a;
+    };
+    // The stages above 0 do not depend on stage 0 until their results are merged: compute them on
+    // the side stream while stage 0 runs, then finish each with an element-wise merge.
+    const bool overlap = ix->n_stages > 1 && !g_no_overlap;
+    Side *sd = nullptr;
+    if (overlap) {
+        rc = get_side(&sd);
+        if (rc) return rc;
+        HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
+        HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+        for (int s = 1; s < ix->n_stages; ++s) {
+            FwdStageArgs a = stage_args(s);
+            a.own_o = (float *)(ws + L.own[s][0]);
+            a.own_lse = (float *)(ws + L.own[s][1]);
+            rc = launch_fwd_simt(a, head_dim, dtype, sd->s);
+            if (rc) return rc;
+        }
+        HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+    }
+    for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
+        FwdStageArgs a = stage_args(s);
+        if (s == 1 && overlap) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         {
             ProfScope ps(s == 0 ? PROF_FWD_STAGE0 : PROF_FWD_UPPER, st);
-            if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
+            if (s > 0 && overlap) {
+                a.own_o = (float *)(ws + L.own[s][0]);
+                a.own_lse = (float *)(ws + L.own[s][1]);
+                rc = launch_merge_fwd(a, head_dim, dtype, st);
+            } else if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
             else rc = launch_fwd_simt(a, head_dim, dtype, st);
         }
         if (rc) return rc;
@@ -234,7 +286,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
     }
     if (rc) return rc;
-    for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
+    auto stage_args = [&](int s) {
         const StagePtrs &P = ix->st[s];
         BwdStageArgs a{};
         a.n = ix->desc[s].n; a.nb = ix->desc[s].nb; a.H = heads; a.T = ix->total_tokens;
@@ -258,9 +310,36 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.dq = dq; a.dk = dk; a.dv = dv;
         a.status = status;
         a.no_persistent = g_no_persistent;
+        return a;
+    };
+    const bool overlap = ix->n_stages > 1 && !g_no_overlap;
+    Side *sd = nullptr;
+    if (overlap) {   // delta is ready: the upper stages' own gradients are computed beside stage 0
+        rc = get_side(&sd);
+        if (rc) return rc;
+        HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
+        HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+        for (int s = 1; s < ix->n_stages; ++s) {
+            BwdStageArgs a = stage_args(s);
+            a.own_dq = (float *)(ws + L.own[s][0]);
+            a.own_dk = (float *)(ws + L.own[s][1]);
+            a.own_dv = (float *)(ws + L.own[s][2]);
+            rc = launch_bwd_simt(a, head_dim, dtype, sd->s);
+            if (rc) return rc;
+        }
+        HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+    }
+    for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
+        BwdStageArgs a = stage_args(s);
+        if (s == 1 && overlap) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         {
             ProfScope ps(s == 0 ? PROF_BWD_STAGE0 : PROF_BWD_UPPER, st);
-            if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
+            if (s > 0 && overlap) {
+                a.own_dq = (float *)(ws + L.own[s][0]);
+                a.own_dk = (float *)(ws + L.own[s][1]);
+                a.own_dv = (float *)(ws + L.own[s][2]);
+                rc = launch_merge_bwd(a, head_dim, dtype, st);
+            } else if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
             else rc = launch_bwd_simt(a, head_dim, dtype, st);
         }
         if (rc) return rc;

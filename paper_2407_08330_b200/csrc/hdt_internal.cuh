@@ -85,6 +85,9 @@ struct FwdStageArgs {
     // ... and, for elements that live on in the next stage, to that stage's buffers at up[e]
     // ([n_next, H, D] and [n_next, H]); nullptr for the last stage.
     float *part_o, *part_lse;
+    // own_*: when set, the kernel only writes its own partial result per element ([n,H,D], [n,H])
+    // and does no merging or final write (the stage runs beside stage 0; merge_fwd finishes it)
+    float *own_o, *own_lse;
     int *status;        // device failure word
     int rest_only;      // general kernel: only blocks after the first n_fused
     int no_persistent;  // option: do not use the persistent kernels
@@ -104,6 +107,7 @@ struct BwdStageArgs {
     const float *carry_dq, *carry_dk, *carry_dv;  // [n,H,D] partials from the stages below, or nullptr
     void *dq, *dk, *dv;                           // dtype [T,H,D], written by every stage
     float *part_dq, *part_dk, *part_dv;           // [n_next,H,D] next stage's buffers (at up[e]), or nullptr
+    float *own_dq, *own_dk, *own_dv;              // when set: own gradients only, [n,H,D] (see FwdStageArgs)
     int *status;                                  // device failure word
     int rest_only;                                // general kernel: only blocks after the first n_fused
     int no_persistent;                            // option: do not use the persistent kernels
@@ -119,5 +123,9 @@ int read_fwd_phase_cycles(long long *out16);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
                  cudaStream_t st);
+// Element-wise completion of a stage that was computed beside stage 0: own partial (own_*) merged
+// with the partial from below (carry_*), handed on (part_*) and written to the caller's tensors.
+int launch_merge_fwd(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
+int launch_merge_bwd(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 
 }  // namespace hdt

@@ -112,7 +112,9 @@ def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
     """bf16 runs three times: persistent + general tensor-core kernels, general tensor-core kernels
     only, SIMT kernels on every stage."""
     # default kernels; general tensor-core kernels only; persistent forward; SIMT everywhere
-    opts = ({}, {"no_persistent": 1}, {"no_persistent": 2}, {"force_simt": 1}) if dtype == "bf16" else ({},)
+    # (fp32 runs with and without the side-stream overlap of the upper stages)
+    opts = (({}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2}, {"force_simt": 1})
+            if dtype == "bf16" else ({}, {"no_overlap": 1}))
     for opt in opts:
         for k_, v_ in opt.items():
             P.hdt_set_option(k_, v_)
