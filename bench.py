@@ -32,7 +32,11 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 
 # DRAM traffic (read + write bytes per launch) of the dominant kernel from the ncu captures
 # summarised under profiles/; keyed by (config, profile id).  None = not captured.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/k_bwd_tc_p_and_k_fwd_tc_c3_b4_L8192.md
+    (3, "k_bwd_stage0"): 349.7e6,
+    (3, "k_fwd_stage0"): 182.8e6,
+}
 
 
 def peaks():
@@ -98,7 +102,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            self._stop.wait(0.05)
+            self._stop.wait(0.002)
 
     def __enter__(self):
         if self._h is not None:
