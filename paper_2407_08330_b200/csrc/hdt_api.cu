@@ -61,11 +61,10 @@ int *device_status_ptr() {
 
 // ---- side stream: the stages above 0 run beside stage 0 -------------------------------------------
 // One non-blocking stream and two events per host thread and device, created on first use.
-struct Side { cudaStream_t s; cudaEvent_t fork, join; bool ready; };
 static thread_local Side g_side[64];
-static int g_no_overlap = 0;
+int g_no_overlap = 0;
 
-static int get_side(Side **out) {
+int get_side(Side **out) {
     int dev = -1;
     HDT_CUDA_CHECK(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return set_error(HDT_ERR_UNSUPPORTED, "device ordinal %d", dev);

@@ -20,6 +20,7 @@ static constexpr int CHUNK = 1024;  // elements per CTA in the element-wise kern
 
 struct Layout {
     size_t header, cnt, nlc, pre, keep, fpos, blocksum, bstart, seqcount, cost, stage0, stage_stride;
+    size_t fpos2, bstart2, seqcount2, cost2;   // second set for the upper stages, built beside stage 0's blocks
     size_t s_tok, s_par, s_rng, s_up, s_scu, s_blocks, s_queue, s_queue2;  // offsets inside a stage
     size_t total;
     int capnb, nchunk;
@@ -42,6 +43,10 @@ static Layout make_layout(int B, int T, int bm, int max_stages) {   // bm: the s
     L.bstart = o; o += al(sizeof(int) * (size_t)L.capnb);
     L.seqcount = o; o += al(sizeof(int) * (size_t)(B + 1));
     L.cost = o; o += al(sizeof(long long) * (size_t)L.capnb);
+    L.fpos2 = o; o += al((size_t)T);
+    L.bstart2 = o; o += al(sizeof(int) * (size_t)L.capnb);
+    L.seqcount2 = o; o += al(sizeof(int) * (size_t)(B + 1));
+    L.cost2 = o; o += al(sizeof(long long) * (size_t)L.capnb);
     L.stage0 = o;
     size_t s = 0;
     L.s_tok = s; s += al(sizeof(int) * (size_t)T);
@@ -726,15 +731,24 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
                                  ix->st[0].par, ix->st[0].scu, cnt);
     count_launch();
     const bool fused_upper = (B <= UMAXB);
+    // The upper stages only need stage 0's compaction; with their own scratch they are built on the
+    // side stream while stage 0's blocks and queues are built on the caller's stream.
+    Side *sd = nullptr;
+    if (fused_upper && ms > 1 && !g_no_overlap && get_side(&sd) != HDT_OK) sd = nullptr;
+    auto launch_upper = [&](cudaStream_t s_) {
+        UpperArgs u;
+        for (int i = 0; i < HDT_MAX_STAGES; ++i) u.st[i] = ix->st[i < ms ? i : ms - 1];
+        u.max_stages = ms; u.B = B; u.bm = bmu;
+        u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.keep = keep;
+        u.bstart = (int *)(ws + L.bstart2); u.seqcount = (int *)(ws + L.seqcount2);
+        u.fpos = (uint8_t *)(ws + L.fpos2); u.cost = (long long *)(ws + L.cost2);
+        k_upper_stages<<<1, UT, 0, s_>>>(hdr, u);
+        count_launch();
+    };
     for (int s = 0; s < ms; ++s) {
         if (s >= 1 && fused_upper) {
-            UpperArgs u;
-            for (int i = 0; i < HDT_MAX_STAGES; ++i) u.st[i] = ix->st[i < ms ? i : ms - 1];
-            u.max_stages = ms; u.B = B; u.bm = bmu;
-            u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.bstart = bstart; u.seqcount = seqcount;
-            u.keep = keep; u.fpos = fpos; u.cost = cost;
-            k_upper_stages<<<1, UT, 0, st>>>(hdr, u);
-            count_launch();
+            if (sd) HDT_BUILD_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
+            else launch_upper(st);
             break;
         }
         const StagePtrs &P = ix->st[s];
@@ -751,6 +765,12 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         if (!last) {
             k_compact<<<g_stride, 256, 0, st>>>(hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc);
             count_launch();
+            if (s == 0 && sd) {   // fork: the upper stages start now
+                HDT_BUILD_CHECK(cudaEventRecord(sd->fork, st));
+                HDT_BUILD_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+                launch_upper(sd->s);
+                HDT_BUILD_CHECK(cudaEventRecord(sd->join, sd->s));
+            }
         }
         if (B > 0) {
             int maxlen_smem = kSmemCap;  // sequences longer than this walk through global memory

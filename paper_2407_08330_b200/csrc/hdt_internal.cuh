@@ -64,6 +64,12 @@ struct ProfScope {
             return hdt::set_error(HDT_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
     } while (0)
 
+// Side stream (one per host thread and device, created on first use): work that does not depend
+// on the main kernel of a call runs beside it.  fork / join are events for the two hand-overs.
+struct Side { cudaStream_t s; cudaEvent_t fork, join; bool ready; };
+int get_side(Side **out);
+extern int g_no_overlap;   // option "no_overlap"
+
 // SIMT attention launchers (hdt_attn_simt.cu).  One launch handles one stage.
 struct FwdStageArgs {
     // stage view
