@@ -317,13 +317,19 @@ __device__ long long g_bwd_phase_cycles[16];
 // so they run while the CTA drains dQ/dK/dV of item i.
 // Thread t: row t % 128 (TMEM lane), column quarter t / 128.
 // ---------------------------------------------------------------------------------------------
+// Output tiles leave through TMA stores.  A block has 1..128 rows and a store box has a fixed
+// number of rows, so each gradient tensor gets seven maps with boxes of 64, 32, ..., 1 rows and a
+// tile is stored as the binary decomposition of its row count.
+struct StoreMaps { CUtensorMap m[3][7]; };
+
 __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
                                                      const __grid_constant__ CUtensorMap tm_v,
-                                                     const __grid_constant__ CUtensorMap tm_do, const BwdStageArgs a) {
+                                                     const __grid_constant__ CUtensorMap tm_do,
+                                                     const __grid_constant__ StoreMaps sm_out, const BwdStageArgs a) {
     constexpr int D = 64;
     constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_DK = 320, TM_DV = 384, TM_COLS = 512;
-    constexpr int STG = 128 * 144;        // bytes of one staged output tile (rows padded to 144 bytes)
+    constexpr int STG = SUB;              // one staged output tile: [128 x 64] bf16, swizzled like the inputs
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sIn = sm;                    // 2 stages x {Q, dO, K, V}
@@ -359,6 +365,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     // MMAs are issued by lane 0 of warps 0, 1, 2 in parallel: a single thread needs about 100 cycles
     // per small MMA (descriptor arithmetic), three chains issued side by side hide that
     const bool issuer = ((tid & 31) == 0) && warp < 3;
+    const bool store_thread = ((tid & 15) == 0) && tid < 384;   // 24 threads, one per (tensor, box slot)
 
     // Item i of this CTA: block, head, rows.  Descriptors are fetched two items ahead and the row
     // statistics one item ahead, so that no global-memory latency sits between two items.
@@ -447,7 +454,8 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             HDT_STAMP(0);
             // S, dP of this item: warp 0 polls the mbarrier, the other warps sleep at the CTA barrier
             if (warp == 0) ok = mbar_wait(bar_a, it & 1, abort_flag, WAIT_CYCLES) && ok;
-            __syncthreads();   // also: the previous item's staged gradients have been stored
+            if (store_thread) bulk_wait_read();   // the previous item's staged gradients have left shared memory
+            __syncthreads();
             tc_fence_after();
             HDT_STAMP(1);
             // ---- P and dS of this thread's 32 columns, in two halves of 16 ----
@@ -554,25 +562,24 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                 uint32_t pk[8];
 #pragma unroll
                 for (int j = 0; j < 8; ++j) pk[j] = pack_bf16(x[2 * j], x[2 * j + 1]);
-                *reinterpret_cast<uint4 *>(dst + rl * 144 + qt * 32) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                *reinterpret_cast<uint4 *>(dst + rl * 144 + qt * 32 + 16) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
+                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
             }
+            fence_proxy_async_smem();
             tc_fence_before();
             HDT_STAMP(6);
             __syncthreads();
             HDT_STAMP(7);
-            // ---- coalesced stores: thread -> rows tid/8 and tid/8 + 64, 16-byte chunk tid%8, 3 tensors ----
-            {
-                const int rA = tid >> 3, c = tid & 7;
-#pragma unroll
-                for (int t = 0; t < 3; ++t) {
-                    __nv_bfloat16 *g = reinterpret_cast<__nv_bfloat16 *>((t == 0) ? a.dq : (t == 1) ? a.dk : a.dv);
-                    uint4 v0, v1;
-                    if (rA < nrows) v0 = *reinterpret_cast<const uint4 *>(sP + t * STG + rA * 144 + c * 16);
-                    if (rA + 64 < nrows) v1 = *reinterpret_cast<const uint4 *>(sP + t * STG + (rA + 64) * 144 + c * 16);
-                    if (rA < nrows) *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + rA) * H + h) * D + c * 8) = v0;
-                    if (rA + 64 < nrows) *reinterpret_cast<uint4 *>(g + ((size_t)(r0 + rA + 64) * H + h) * D + c * 8) = v1;
-                }
+            // ---- TMA stores: rows [0, nrows) of each staged tile as boxes of 64, 64, 32, ..., 1 rows;
+            // 24 (tensor, box) slots, one per store thread ----
+            if (store_thread) {
+                const int t = (tid >> 4) >> 3, slot = (tid >> 4) & 7;
+                int rows, off, b;
+                if (slot < 2) { b = 0; rows = 64; off = 64 * slot; }
+                else { b = slot - 1; rows = 64 >> b; off = nrows & ~(2 * rows - 1); }
+                const bool use = (slot < 2) ? (nrows >= 64 * (slot + 1)) : ((nrows & rows) != 0);
+                if (use) tma_store_3d(&sm_out.m[t][b], 0, h, r0 + off, sP + t * STG + off * 128);
+                bulk_commit();
             }
             HDT_STAMP(8);
             dc = dn; dn = dn2; rc = rn;
@@ -583,6 +590,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
         }
     }
     if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+    if (store_thread) bulk_wait_read();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
@@ -621,7 +629,14 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
         }
         const long long items = (long long)a.n_fused * a.H;
         const int grid_p = (int)(items < n_sm ? items : n_sm);
-        k_bwd_tc_p<<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, a);
+        StoreMaps outs;
+        void *outp[3] = {a.dq, a.dk, a.dv};
+        for (int t = 0; t < 3; ++t)
+            for (int b = 0; b < 7; ++b) {
+                rc = make_tmap_bf16(&outs.m[t][b], outp[t], D, a.H, a.T, 64 >> b);
+                if (rc) return rc;
+            }
+        k_bwd_tc_p<<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, a);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
         b.rest_only = 1;

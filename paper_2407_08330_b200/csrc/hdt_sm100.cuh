@@ -61,6 +61,14 @@ __device__ __forceinline__ void tma_load_3d(void *dst, const CUtensorMap *tm, in
         : "memory");
 }
 
+// 3-D tiled store of a shared-memory box (same swizzled format as the loads) to global memory;
+// completion is tracked per thread in bulk groups (bulk_commit / bulk_wait_read).
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap *tm, int x, int y, int z, const void *src) {
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(tm), "r"(x), "r"(y),
+                 "r"(z), "r"(smem_u32(src))
+                 : "memory");
+}
+
 // Bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned) from shared to global
 // memory; completion is tracked per thread in bulk groups.
 __device__ __forceinline__ void bulk_store(void *gdst, const void *ssrc, uint32_t bytes) {
