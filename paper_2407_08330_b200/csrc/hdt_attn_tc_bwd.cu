@@ -31,10 +31,11 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
                                                 const __grid_constant__ CUtensorMap tm_v,
                                                 const __grid_constant__ CUtensorMap tm_do, const BwdStageArgs a) {
     constexpr int NSUB = D / 64;
-    // TMEM columns: S and dP per pass; accumulators.  At D = 128 dQ and dK share columns (they are
-    // never live together there, the fused pass exists only at D = 64).
-    constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_DK = (D == 64) ? 320 : 256, TM_DV = 384, TM_COLS = 512;
-    constexpr bool FUSE = (D == 64);
+    // TMEM columns: S and dP per pass (0..255); accumulators.  D = 64: dQ 256, dK 320, dV 384.
+    // D = 128 (3 x 128 accumulator columns do not fit beside S and dP): a fused pass puts dV and dK
+    // over S and dP, which are dead once P and dS are written; the two-walk path keeps dQ, then
+    // dK, in columns 256.. and dV in 384.. while S and dP are rewritten per chunk.
+    constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_COLS = 512;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = sm, *sDO = sQ + NSUB * SUB, *sK = sDO + NSUB * SUB, *sV = sK + NSUB * SUB;
@@ -68,6 +69,9 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     const bool dead = (*abort_flag != 0);
     const bool empty = (fl & HDT_BLK_EMPTY) != 0;
     const bool self = (fl & HDT_BLK_SELF) != 0;
+    const bool fused = self && !empty && !dead;   // one pass yields dQ, dK and dV
+    const uint32_t TM_DK = (D == 64) ? 320u : (fused ? 128u : 256u);
+    const uint32_t TM_DV = (D == 64) ? 384u : (fused ? 0u : 384u);
     uint32_t ph_tma = 0, ph_mma = 0;
     bool ok = true;
 
@@ -253,7 +257,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         }
     }
 
-    if (run && self && FUSE) {
+    if (fused) {
         load(true, r0, true, r0);
         tile_pass(r0, r1, r0, r1, true, true, false, false);
         if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
@@ -290,7 +294,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     }
     tc_fence_before();
     __syncthreads();
-    if (run && self && FUSE) copy_out(sP, a.dq);   // same decision in every thread
+    if (fused) copy_out(sP, a.dq);   // same decision in every thread
     copy_out(sDS, a.dk);
     copy_out(sQ, a.dv);
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
