@@ -326,6 +326,7 @@ __device__ long long g_bwd_phase_cycles[16];
 // tile is stored as the binary decomposition of its row count.
 struct StoreMaps { CUtensorMap m[3][7]; };
 
+template <bool SPLIT>
 __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
                                                      const __grid_constant__ CUtensorMap tm_v,
@@ -346,8 +347,6 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
 
     const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, qt = tid >> 7;
     const int H = a.H, G = gridDim.x;
-    const int n_items = a.n_fused * H;
-    const int my_count = ((int)blockIdx.x < n_items) ? (n_items - (int)blockIdx.x + G - 1) / G : 0;
     const float LOG2E = 1.4426950408889634f;
 
     if (tid == 0) {
@@ -371,42 +370,119 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     const bool issuer = ((tid & 31) == 0) && warp < 3;
     const bool store_thread = ((tid & 15) == 0) && tid < 384;   // 24 threads, one per (tensor, box slot)
 
-    // Item i of this CTA: block, head, rows.  Descriptors are fetched two items ahead and the row
-    // statistics one item ahead, so that no global-memory latency sits between two items.
-    struct Desc { int r0, r1, h; };
-    auto load_blk = [&](int i) { return a.queue_split[((int)blockIdx.x + i * G) / H]; };
-    auto load_rec = [&](int i, int blk) {
-        Desc d;
-        d.h = ((int)blockIdx.x + i * G) % H;
-        d.r0 = a.blocks[5 * (size_t)blk];
-        d.r1 = a.blocks[5 * (size_t)blk + 1];
-        return d;
+    // ---- work stream of this CTA ----------------------------------------------------------------
+    // A unit is a (block, head); this CTA takes units blockIdx.x, + gridDim.x, ... of its group of
+    // queue_split (mode 0: the first n_fused blocks, SELF and not EMPTY; mode 1: the others).
+    // A SELF block is one item (both tiles = the block, all three gradients).  A block of a split
+    // family is 2 x chunks items: first as query rows over its key span (dQ accumulates in TMEM),
+    // then as keys over the same span taken as query rows (dK, dV accumulate).  EMPTY blocks are
+    // written as zeros on the spot.  Block ids are fetched two units ahead, records one unit ahead,
+    // items two ahead and row statistics one ahead: no global-memory latency between two items.
+    constexpr bool split = SPLIT;
+    const int unit_base = split ? a.n_fused : 0;
+    const int n_units = (split ? (a.nb - a.n_fused) : a.n_fused) * H;
+    struct UB { int blk, h; };
+    struct Unit { int valid, r0, r1, ka, kb, h, empty; };
+    struct Item { int valid, q0, qe, k0, ke, h, r0, nrows, flags, up; };
+    constexpr int F_DQ = 1, F_DKDV = 2, F_ACC = 4, F_LAST = 8;
+    int unit_next = (int)blockIdx.x;
+    auto fetch_ub = [&]() {
+        UB x{-1, 0};
+        const int u = unit_next;
+        unit_next += G;
+        if (u < n_units) { x.blk = a.queue_split[unit_base + u / H]; x.h = u % H; }
+        return x;
     };
-    auto load_desc = [&](int i) { return load_rec(i, load_blk(i)); };
-    struct RowStat { int lo, hi, up; float lse2, dl; };
-    auto load_stat = [&](const Desc &d) {
-        RowStat r{0, 0, -1, 0.f, 0.f};
-        const int row = d.r0 + rl;
-        if (row < d.r1) {
+    auto fetch_unit = [&](const UB &x) {
+        Unit v{0, 0, 0, 0, 0, x.h, 1};
+        if (x.blk >= 0) {
+            const int *rec = a.blocks + 5 * (size_t)x.blk;
+            v.valid = 1; v.r0 = rec[0]; v.r1 = rec[1]; v.ka = rec[2]; v.kb = rec[3];
+            v.empty = (rec[4] & HDT_BLK_EMPTY) ? 1 : 0;
+        }
+        return v;
+    };
+    auto block_up = [&](const Unit &v) {   // next-stage index of this thread's row of the block
+        return (v.valid && a.part_dq != nullptr && v.r0 + rl < v.r1) ? a.up[v.r0 + rl] : -1;
+    };
+    UB nn = fetch_ub();
+    Unit cur = fetch_unit(nn);
+    nn = fetch_ub();
+    Unit nxt = fetch_unit(nn);
+    nn = fetch_ub();
+    int up_cur = block_up(cur);
+    int role = 0, chunk = 0;
+    auto write_empty = [&](const Unit &v, int up) {   // zero gradients of an EMPTY block, this thread's share
+        if (v.r0 + rl < v.r1) {
+            const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+            const size_t e = ((size_t)(v.r0 + rl) * H + v.h) * D + 16 * qt;
+            __nv_bfloat16 *g[3] = {(__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv};
+            float *pt[3] = {a.part_dq, a.part_dk, a.part_dv};
+#pragma unroll
+            for (int t = 0; t < 3; ++t) {
+                *reinterpret_cast<uint4 *>(g[t] + e) = z;
+                *reinterpret_cast<uint4 *>(g[t] + e + 8) = z;
+                if (up >= 0) {
+                    float4 *c4 = reinterpret_cast<float4 *>(pt[t] + ((size_t)up * H + v.h) * D + 16 * qt);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) c4[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+    };
+    auto next_item = [&]() {
+        Item x{0, 0, 0, 0, 0, 0, 0, 0, 0, -1};
+        while (cur.valid) {
+            if (cur.empty) {
+                if (role == 0) write_empty(cur, up_cur);
+                role = 2;
+            }
+            if (role < 2) {
+                x.valid = 1; x.h = cur.h; x.r0 = cur.r0; x.nrows = cur.r1 - cur.r0; x.up = up_cur;
+                if (!split) {
+                    x.q0 = cur.r0; x.qe = cur.r1; x.k0 = cur.r0; x.ke = cur.r1;
+                    x.flags = F_DQ | F_DKDV | F_LAST;
+                    role = 2;
+                } else {
+                    const int nch = (cur.kb - cur.ka + 127) >> 7, c0 = cur.ka + 128 * chunk;
+                    if (role == 0) { x.q0 = cur.r0; x.qe = cur.r1; x.k0 = c0; x.ke = cur.kb; }
+                    else { x.q0 = c0; x.qe = cur.kb; x.k0 = cur.r0; x.ke = cur.r1; }
+                    x.flags = (role == 0 ? F_DQ : F_DKDV) | (chunk > 0 ? F_ACC : 0) | (chunk == nch - 1 ? F_LAST : 0);
+                    if (++chunk == nch) { chunk = 0; ++role; }
+                }
+                return x;
+            }
+            cur = nxt;                 // next unit; its record was fetched one unit ago
+            up_cur = block_up(cur);
+            nxt = fetch_unit(nn);
+            nn = fetch_ub();
+            role = 0; chunk = 0;
+        }
+        return x;
+    };
+    struct RowStat { int lo, hi; float lse2, dl; };
+    auto load_stat = [&](const Item &d) {
+        RowStat r{0, 0, 0.f, 0.f};
+        const int row = d.q0 + rl;
+        if (d.valid && row < d.qe) {
             r.lo = a.rng[2 * row];
             r.hi = a.rng[2 * row + 1];
             r.lse2 = a.lse[(size_t)d.h * a.T + row];   // natural log; scaled where it is used
             r.dl = a.delta[(size_t)d.h * a.T + row];
-            if (a.part_dq != nullptr) r.up = a.up[row];
         }
         return r;
     };
-    auto issue_tma = [&](int i, const Desc &d) {       // thread 0
-        uint8_t *st = sIn + (i & 1) * 4 * SUB;
-        uint64_t *bar = &bar_tma[i & 1];
+    auto issue_tma = [&](int n, const Item &d) {       // thread 0
+        uint8_t *st = sIn + (n & 1) * 4 * SUB;
+        uint64_t *bar = &bar_tma[n & 1];
         mbar_expect_tx(bar, 4 * SUB);
-        tma_load_3d(st, &tm_q, 0, d.h, d.r0, bar);
-        tma_load_3d(st + SUB, &tm_do, 0, d.h, d.r0, bar);
-        tma_load_3d(st + 2 * SUB, &tm_k, 0, d.h, d.r0, bar);
-        tma_load_3d(st + 3 * SUB, &tm_v, 0, d.h, d.r0, bar);
+        tma_load_3d(st, &tm_q, 0, d.h, d.q0, bar);
+        tma_load_3d(st + SUB, &tm_do, 0, d.h, d.q0, bar);
+        tma_load_3d(st + 2 * SUB, &tm_k, 0, d.h, d.k0, bar);
+        tma_load_3d(st + 3 * SUB, &tm_v, 0, d.h, d.k0, bar);
     };
-    auto issue_sdp = [&](int i, int Nc) {   // warps 0 (S) and 1 (dP), lane 0; inputs of item i have landed
-        const uint32_t st = smem_u32(sIn + (i & 1) * 4 * SUB);
+    auto issue_sdp = [&](int n, int Nc) {   // warps 0 (S) and 1 (dP), lane 0; inputs of item n have landed
+        const uint32_t st = smem_u32(sIn + (n & 1) * 4 * SUB);
         const uint32_t idesc = idesc_bf16(Nc, false, false);
         const uint32_t a_off = (warp == 0) ? 0u : (uint32_t)SUB, b_off = (warp == 0) ? 2u * SUB : 3u * SUB;
         const uint32_t col = (warp == 0) ? TM_S : TM_DP;
@@ -415,44 +491,37 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             mma_ss(tmem + col, smem_desc(st + a_off + kk * 32, 0, 1024), smem_desc(st + b_off + kk * 32, 0, 1024), idesc, kk > 0);
         mma_commit(bar_a);
     };
+    auto keys16 = [&](const Item &d) { return (min(128, d.ke - d.k0) + 15) & ~15; };
 
-    if (!dead && my_count > 0) {
-        Desc dc = load_desc(0), dn = dc, dn2 = dc;
-        if (my_count > 1) dn = load_desc(1);
-        int blk2 = (my_count > 2) ? load_blk(2) : 0;   // block id of item it+2, fetched one iteration ahead
-        RowStat rc = load_stat(dc), rn = rc;
-        if (tid == 0) {
-            issue_tma(0, dc);
-            if (my_count > 1) issue_tma(1, dn);
+    if (!dead && n_units > 0) {
+        Item d0 = next_item(), d1 = next_item(), d2 = next_item();
+        RowStat rc = load_stat(d0), rn = rc;
+        if (tid == 0 && d0.valid) {
+            issue_tma(0, d0);
+            if (d1.valid) issue_tma(1, d1);
         }
-        if (issuer && warp < 2) {
+        if (issuer && warp < 2 && d0.valid) {
             ok = mbar_wait(&bar_tma[0], 0, abort_flag, WAIT_CYCLES) && ok;
             if (!*abort_flag) {
                 tc_fence_after();
-                issue_sdp(0, (dc.r1 - dc.r0 + 15) & ~15);
+                issue_sdp(0, keys16(d0));
             }
         }
         const bool stamp = (tid == 0 && blockIdx.x == 0);
         long long ph_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
         long long t_last = clock64();
-        for (int it = 0; it < my_count; ++it) {
+        int it = 0;
+        for (; d0.valid; ++it) {
             HDT_STAMP(9);
-            // prefetch: descriptor of item it+2, row statistics of item it+1
-            if (it + 2 < my_count) dn2 = load_rec(it + 2, blk2);
-            if (it + 3 < my_count) blk2 = load_blk(it + 3);
-            if (it + 1 < my_count) rn = load_stat(dn);
-            const int r0 = dc.r0, r1 = dc.r1, h = dc.h;
-            const int nrows = r1 - r0, Nc = (nrows + 15) & ~15;
-            const bool inb = r0 + rl < r1;
+            rn = load_stat(d1);   // row statistics of the next item
+            const int h = d0.h, k0 = d0.k0;
+            const int nq = min(128, d0.qe - d0.q0), nk = min(128, d0.ke - k0);
+            const int Nc = (nk + 15) & ~15, Kr = (nq + 15) & ~15;
+            const bool inq = d0.q0 + rl < d0.qe;
             const float lse2 = rc.lse2 * LOG2E, dl = rc.dl;
-            float *cq = nullptr, *ck = nullptr, *cv = nullptr;
-            if (rc.up >= 0) {   // this row lives on in the next stage: its fp32 gradients go there too
-                cq = a.part_dq + ((size_t)rc.up * H + h) * D;
-                ck = a.part_dk + ((size_t)rc.up * H + h) * D;
-                cv = a.part_dv + ((size_t)rc.up * H + h) * D;
-            }
-            const int jl = max(rc.lo - r0, 0), jh = min(rc.hi - r0, nrows);
-            const bool has = inb && jh > jl;
+            const int jl = max(rc.lo - k0, 0), jh = min(rc.hi - k0, nk);
+            const bool has = inq && jh > jl;
+            const int flags = SPLIT ? d0.flags : (F_DQ | F_DKDV | F_LAST);   // constant for self-contained blocks
             uint8_t *st = sIn + (it & 1) * 4 * SUB;
 
             HDT_STAMP(0);
@@ -479,17 +548,17 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                         if (mine) {
 #pragma unroll
                             for (int j = 0; j < 16; j += 2) {
-                                float p0 = 0.f, p1 = 0.f, d0 = 0.f, d1 = 0.f;
+                                float p0 = 0.f, p1 = 0.f, e0 = 0.f, e1 = 0.f;
                                 if (s0 + j >= jl && s0 + j < jh) {
                                     p0 = exp2f(fmaf(__uint_as_float(rs[j]), a.scale_log2, -lse2));
-                                    d0 = p0 * (__uint_as_float(rd[j]) - dl);
+                                    e0 = p0 * (__uint_as_float(rd[j]) - dl);
                                 }
                                 if (s0 + j + 1 >= jl && s0 + j + 1 < jh) {
                                     p1 = exp2f(fmaf(__uint_as_float(rs[j + 1]), a.scale_log2, -lse2));
-                                    d1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
+                                    e1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
                                 }
                                 pp[j >> 1] = pack_bf16(p0, p1);
-                                pd[j >> 1] = pack_bf16(d0, d1);
+                                pd[j >> 1] = pack_bf16(e0, e1);
                             }
                         }
                     }
@@ -510,87 +579,92 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                 tc_fence_after();
                 // descriptors differ only in the start address: add (bytes >> 4) to the low word
                 const uint32_t sb = smem_u32(st);
-                const int nk = Nc / 16;
-                if (warp == 0) {          // dV = P^T dO
+                const uint32_t acc = (flags & F_ACC) ? 1u : 0u;
+                if (warp == 0 && (flags & F_DKDV)) {          // dV (+)= P^T dO, contraction over the query rows
                     const uint32_t idesc = idesc_bf16(D, true, true);
                     const uint64_t da = smem_desc(smem_u32(sP), SUB, 1024), db = smem_desc(sb + SUB, SUB, 1024);
-                    for (int kk = 0; kk < nk; ++kk)
-                        mma_ss(tmem + TM_DV, da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc, kk > 0);
-                } else if (warp == 1) {   // dK = dS^T Q
+                    for (int kk = 0; kk < Kr / 16; ++kk)
+                        mma_ss(tmem + TM_DV, da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc, acc | (kk > 0));
+                } else if (warp == 1 && (flags & F_DKDV)) {   // dK (+)= dS^T Q
                     const uint32_t idesc = idesc_bf16(D, true, true);
                     const uint64_t da = smem_desc(smem_u32(sDS), SUB, 1024), db = smem_desc(sb, SUB, 1024);
-                    for (int kk = 0; kk < nk; ++kk)
-                        mma_ss(tmem + TM_DK, da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc, kk > 0);
-                } else {                  // dQ = dS K
+                    for (int kk = 0; kk < Kr / 16; ++kk)
+                        mma_ss(tmem + TM_DK, da + (uint64_t)(kk * 128), db + (uint64_t)(kk * 128), idesc, acc | (kk > 0));
+                } else if (warp == 2 && (flags & F_DQ)) {     // dQ (+)= dS K, contraction over the keys
                     const uint32_t idesc = idesc_bf16(D, false, true);
                     const uint64_t da = smem_desc(smem_u32(sDS), 0, 1024), db = smem_desc(sb + 2 * SUB, SUB, 1024);
-                    for (int kk = 0; kk < nk; ++kk)
+                    for (int kk = 0; kk < Nc / 16; ++kk)
                         mma_ss(tmem + TM_DQ, da + (uint64_t)((kk / 4) * (SUB >> 4) + (kk % 4) * 2),
-                               db + (uint64_t)(kk * 128), idesc, kk > 0);
+                               db + (uint64_t)(kk * 128), idesc, acc | (kk > 0));
                 }
-                mma_commit(bar_b);
+                mma_commit(bar_b);   // every issuer arrives, with or without MMAs of its own
                 HDT_STAMP(10);
-                if (warp < 2 && it + 1 < my_count) {   // S, dP of the next item run during this item's drain
+                if (warp < 2 && d1.valid) {   // S, dP of the next item run during this item's drain
                     ok = mbar_wait(&bar_tma[(it + 1) & 1], ((it + 1) >> 1) & 1, abort_flag, WAIT_CYCLES) && ok;
                     HDT_STAMP(11);
                     if (!*abort_flag) {
                         tc_fence_after();
-                        issue_sdp(it + 1, (dn.r1 - dn.r0 + 15) & ~15);
+                        issue_sdp(it + 1, keys16(d1));
                     }
                 }
             }
             HDT_STAMP(4);
-            if (warp == 0) ok = mbar_wait(bar_b, it & 1, abort_flag, WAIT_CYCLES) && ok;   // dQ, dK, dV of this item
+            if (warp == 0) ok = mbar_wait(bar_b, it & 1, abort_flag, WAIT_CYCLES) && ok;   // this item's output MMAs
             __syncthreads();
             tc_fence_after();
             HDT_STAMP(5);
-            if (tid == 0 && it + 2 < my_count && !*abort_flag) issue_tma(it + 2, dn2);   // this stage is free again
-            // ---- drain: 16 columns of each gradient per thread, staged as bf16 ----
+            if (tid == 0 && d2.valid && !*abort_flag) issue_tma(it + 2, d2);   // this stage is free again
+            if (flags & F_LAST) {
+                // ---- drain: 16 columns of each finished gradient per thread, staged as bf16 ----
+                const int r0 = d0.r0, nrows = d0.nrows;
 #pragma unroll
-            for (int t = 0; t < 3; ++t) {
-                const uint32_t col = (t == 0) ? TM_DQ : (t == 1) ? TM_DK : TM_DV;
-                const float sc = (t == 2) ? 1.f : a.scale;
-                float *cy = (t == 0) ? cq : (t == 1) ? ck : cv;
-                uint8_t *dst = sP + t * STG;    // staging: 128 rows x 144 bytes per tensor
-                uint32_t r[16];
-                tmem_ld16(tmem + col + lane_base + 16 * qt, r);
-                tmem_wait_ld();
-                float x[16];
+                for (int t = 0; t < 3; ++t) {
+                    if (!(flags & (t == 0 ? F_DQ : F_DKDV))) continue;   // same in every thread
+                    const uint32_t col = (t == 0) ? TM_DQ : (t == 1) ? TM_DK : TM_DV;
+                    const float sc = (t == 2) ? 1.f : a.scale;
+                    uint8_t *dst = sP + t * STG;    // staging: one swizzled [128 x 64] tile per tensor
+                    uint32_t r[16];
+                    tmem_ld16(tmem + col + lane_base + 16 * qt, r);
+                    tmem_wait_ld();
+                    float x[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) x[j] = __uint_as_float(r[j]) * sc;
-                if (cy != nullptr) {   // rows that also exist in the next stage (a few per block)
-                    float4 *c4 = reinterpret_cast<float4 *>(cy + 16 * qt);
+                    for (int j = 0; j < 16; ++j) x[j] = __uint_as_float(r[j]) * sc;
+                    if (d0.up >= 0) {   // this row lives on in the next stage: its fp32 gradients go there too
+                        float *base = (t == 0) ? a.part_dq : (t == 1) ? a.part_dk : a.part_dv;
+                        float4 *c4 = reinterpret_cast<float4 *>(base + ((size_t)d0.up * H + h) * D + 16 * qt);
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) c4[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+                        for (int j = 0; j < 4; ++j) c4[j] = make_float4(x[4 * j], x[4 * j + 1], x[4 * j + 2], x[4 * j + 3]);
+                    }
+                    uint32_t pk[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) pk[j] = pack_bf16(x[2 * j], x[2 * j + 1]);
+                    *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+                    *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
                 }
-                uint32_t pk[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j) pk[j] = pack_bf16(x[2 * j], x[2 * j + 1]);
-                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
-                *reinterpret_cast<uint4 *>(dst + swz(rl, 2 * qt + 1)) = make_uint4(pk[4], pk[5], pk[6], pk[7]);
-            }
-            fence_proxy_async_smem();
-            tc_fence_before();
-            HDT_STAMP(6);
-            __syncthreads();
-            HDT_STAMP(7);
-            // ---- TMA stores: rows [0, nrows) of each staged tile as boxes of 64, 64, 32, ..., 1 rows;
-            // 24 (tensor, box) slots, one per store thread ----
-            if (store_thread) {
-                const int t = (tid >> 4) >> 3, slot = (tid >> 4) & 7;
-                int rows, off, b;
-                if (slot < 2) { b = 0; rows = 64; off = 64 * slot; }
-                else { b = slot - 1; rows = 64 >> b; off = nrows & ~(2 * rows - 1); }
-                const bool use = (slot < 2) ? (nrows >= 64 * (slot + 1)) : ((nrows & rows) != 0);
-                if (use) tma_store_3d(&sm_out.m[t][b], 0, h, r0 + off, sP + t * STG + off * 128);
-                bulk_commit();
+                fence_proxy_async_smem();
+                tc_fence_before();
+                HDT_STAMP(6);
+                __syncthreads();
+                HDT_STAMP(7);
+                // ---- TMA stores: rows [0, nrows) of each staged tile as boxes of 64, 64, 32, ..., 1 rows;
+                // 24 (tensor, box) slots, one per store thread ----
+                if (store_thread) {
+                    const int t = (tid >> 4) >> 3, slot = (tid >> 4) & 7;
+                    int rows, off, b;
+                    if (slot < 2) { b = 0; rows = 64; off = 64 * slot; }
+                    else { b = slot - 1; rows = 64 >> b; off = nrows & ~(2 * rows - 1); }
+                    bool use = (slot < 2) ? (nrows >= 64 * (slot + 1)) : ((nrows & rows) != 0);
+                    use = use && (flags & (t == 0 ? F_DQ : F_DKDV));
+                    if (use) tma_store_3d(&sm_out.m[t][b], 0, h, r0 + off, sP + t * STG + off * 128);
+                    bulk_commit();
+                }
             }
             HDT_STAMP(8);
-            dc = dn; dn = dn2; rc = rn;
+            d0 = d1; d1 = d2; d2 = next_item(); rc = rn;
         }
         if (stamp) {
             for (int i = 0; i < 12; ++i) g_bwd_phase_cycles[i] += ph_acc[i];
-            g_bwd_phase_cycles[12] += my_count;
+            g_bwd_phase_cycles[12] += it;
         }
     }
     if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
@@ -620,31 +694,39 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     BwdStageArgs b = a;
     b.rest_only = 0;
     int n_general = a.nb;
-    if (D == 64 && a.n_fused > 0 && !a.no_persistent) {
+    if (D == 64 && a.nb > 0 && !a.no_persistent) {
+        // the persistent kernel takes everything: first the blocks of split families (longest first),
+        // then the self-contained blocks
         constexpr int smem_p = 12 * SUB + 1024 + 64;
         static bool attr_p = false;
         static int n_sm = 0;
         if (!attr_p) {
-            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
             int dev = 0;
             HDT_CUDA_CHECK(cudaGetDevice(&dev));
             HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
             attr_p = true;
         }
-        const long long items = (long long)a.n_fused * a.H;
-        const int grid_p = (int)(items < n_sm ? items : n_sm);
         StoreMaps outs;
         void *outp[3] = {a.dq, a.dk, a.dv};
         for (int t = 0; t < 3; ++t)
-            for (int b = 0; b < 7; ++b) {
-                rc = make_tmap_bf16(&outs.m[t][b], outp[t], D, a.H, a.T, 64 >> b);
+            for (int bx = 0; bx < 7; ++bx) {
+                rc = make_tmap_bf16(&outs.m[t][bx], outp[t], D, a.H, a.T, 64 >> bx);
                 if (rc) return rc;
             }
-        k_bwd_tc_p<<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, a);
-        count_launch();
-        HDT_CUDA_CHECK(cudaGetLastError());
-        b.rest_only = 1;
-        n_general = a.nb - a.n_fused;
+        for (int mode = 1; mode >= 0; --mode) {
+            const long long units = (long long)(mode ? a.nb - a.n_fused : a.n_fused) * a.H;
+            if (units == 0) continue;
+            BwdStageArgs c = a;
+            c.rest_only = mode;
+            const int grid_p = (int)(units < n_sm ? units : n_sm);
+            if (mode) k_bwd_tc_p<true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
+            else k_bwd_tc_p<false><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
+            count_launch();
+            HDT_CUDA_CHECK(cudaGetLastError());
+        }
+        n_general = 0;
     }
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
@@ -656,7 +738,7 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
 }
 
 // Diagnostics: cycles CTA 0 of the persistent backward spent per phase since the last call
-// (10 phases, then the item count); resets the counters.
+// (12 phases, then the item count); resets the counters.
 int read_bwd_phase_cycles(long long *out16) {
     HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out16, g_bwd_phase_cycles, sizeof(long long) * 16));
     long long zero[16] = {0};
