@@ -254,6 +254,226 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 }
 
 
+// ---------------------------------------------------------------------------------------------
+// Looping forward for SELF, non-EMPTY blocks: the single-chunk layout above (P over Q/K, O over
+// S), but each CTA stays resident and walks items blockIdx.x, + gridDim.x, ... (queue_split order
+// x heads), with 4 (D = 64) or 2 (D = 128) CTAs per SM.  TMEM and barriers are set up once; Q and
+// K of the next item are fetched as soon as P V of the current one has finished (P, which lives
+// in the Q/K tiles, is dead then), V of the next item once the staged O has left the V tile.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUtensorMap tm_q,
+                                                     const __grid_constant__ CUtensorMap tm_k,
+                                                     const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
+    constexpr int NSUB = D / 64;
+    constexpr uint32_t TM_COLS = 128;   // S, then O over it
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = sm, *sK = sQ + NSUB * SUB, *sV = sK + NSUB * SUB;
+    uint8_t *sP = sQ;                   // P (2 sub-tiles) over Q (and K at D = 64)
+    uint64_t *bar_qk = (uint64_t *)(sV + NSUB * SUB);
+    uint64_t *bar_v = bar_qk + 1, *bar_mma = bar_qk + 2;
+    uint32_t *slot = (uint32_t *)(bar_qk + 3);
+    volatile int *abort_flag = (volatile int *)(slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int H = a.H, G = gridDim.x;
+    const int n_items = a.n_fused * H;
+    const float NEG = -INFINITY, LN2 = 0.6931471805599453f;
+
+    if (tid == 0) {
+        mbar_init(bar_qk, 1);
+        mbar_init(bar_v, 1);
+        mbar_init(bar_mma, 1);
+        *abort_flag = (*a.status != 0);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    bool ok = true;
+
+    struct Desc { int r0, r1, ka, kb, h; };
+    auto load_desc = [&](int item) {
+        Desc d{0, 0, 0, 0, 0};
+        if (item < n_items) {
+            const int *rec = a.blocks + 5 * (size_t)a.queue_split[item / H];
+            d.r0 = rec[0]; d.r1 = rec[1]; d.ka = rec[2]; d.kb = rec[3]; d.h = item % H;
+        }
+        return d;
+    };
+    auto issue_qk = [&](const Desc &d) {   // thread 0
+        mbar_expect_tx(bar_qk, (uint32_t)(2 * NSUB) * SUB);
+        for (int s = 0; s < NSUB; ++s) {
+            tma_load_3d(sQ + s * SUB, &tm_q, 64 * s, d.h, d.r0, bar_qk);
+            tma_load_3d(sK + s * SUB, &tm_k, 64 * s, d.h, d.ka, bar_qk);
+        }
+    };
+    auto issue_v = [&](const Desc &d) {    // thread 0
+        mbar_expect_tx(bar_v, (uint32_t)NSUB * SUB);
+        for (int s = 0; s < NSUB; ++s) tma_load_3d(sV + s * SUB, &tm_v, 64 * s, d.h, d.ka, bar_v);
+    };
+
+    if (!dead && (int)blockIdx.x < n_items) {
+        Desc dc = load_desc((int)blockIdx.x), dn = load_desc((int)blockIdx.x + G);
+        if (tid == 0) { issue_qk(dc); issue_v(dc); }
+        uint32_t ph = 0;           // phase of bar_qk and bar_v (one completion of each per item)
+        uint32_t ph_mma = 0;
+        for (int item = (int)blockIdx.x; item < n_items; item += G) {
+            const Desc dn2 = load_desc(item + 2 * G);   // needed two iterations from now
+            const int r0 = dc.r0, r1 = dc.r1, ka = dc.ka, kb = dc.kb, h = dc.h;
+            const bool have_next = item + G < n_items;
+            const int row = r0 + tid;
+            const bool inb = row < r1;
+            int lo = 0, hi = 0, up = -1;
+            if (inb) {
+                lo = a.rng[2 * row];
+                hi = a.rng[2 * row + 1];
+                if (a.part_o != nullptr) up = a.up[row];
+            }
+            const int nvalid = min(128, kb - ka), Nc = (nvalid + 15) & ~15;
+
+            ok = mbar_wait(bar_qk, ph, abort_flag, WAIT_CYCLES) && ok;
+            if (tid == 0 && !*abort_flag) {
+                tc_fence_after();
+                const uint32_t idesc = idesc_bf16(Nc, false, false);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
+                    mma_ss(tmem, smem_desc(smem_u32(sQ) + off, 0, 1024), smem_desc(smem_u32(sK) + off, 0, 1024), idesc, kk > 0);
+                }
+                mma_commit(bar_mma);
+            }
+            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            ph_mma ^= 1;
+            tc_fence_after();
+
+            // ---- masked softmax of this row (one chunk: no running maximum needed) ----
+            const int jl = max(lo - ka, 0), jh = min(hi - ka, nvalid);
+            const bool has = inb && jh > jl;
+            const int nsl = (Nc + 31) >> 5;
+            float mx = NEG;
+            for (int k = 0; k < nsl; ++k) {
+                const int s0 = 32 * k;
+                const bool mine = has && jl < s0 + 32 && jh > s0;
+                if (__any_sync(0xffffffffu, mine)) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem + lane_base + s0, r);
+                    tmem_wait_ld();
+                    if (mine) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (s0 + j >= jl && s0 + j < jh) mx = fmaxf(mx, __uint_as_float(r[j]));
+                    }
+                }
+            }
+            const float m = mx * a.scale_log2;
+            float l = 0.f;
+            for (int k = 0; k < nsl; ++k) {
+                const int s0 = 32 * k;
+                const bool mine = has && jl < s0 + 32 && jh > s0;
+                uint32_t pk[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[j] = 0u;
+                if (__any_sync(0xffffffffu, mine)) {
+                    uint32_t r[32];
+                    tmem_ld32(tmem + lane_base + s0, r);
+                    tmem_wait_ld();
+                    if (mine) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            float p0 = 0.f, p1 = 0.f;
+                            if (s0 + j >= jl && s0 + j < jh) p0 = exp2f(fmaf(__uint_as_float(r[j]), a.scale_log2, -m));
+                            if (s0 + j + 1 >= jl && s0 + j + 1 < jh) p1 = exp2f(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m));
+                            const uint32_t u = pack_bf16(p0, p1);   // the row sum uses the rounded values the MMA sees
+                            l += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
+                            pk[j >> 1] = u;
+                        }
+                    }
+                }
+                uint8_t *dst = sP + (k >> 1) * SUB;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<uint4 *>(dst + swz(tid, (k & 1) * 4 + c)) =
+                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            ok = mbar_wait(bar_v, ph, abort_flag, WAIT_CYCLES) && ok;
+            ph ^= 1;
+            if (tid == 0 && !*abort_flag) {
+                tc_fence_after();
+                const uint32_t idesc = idesc_bf16(D, false, true);
+                for (int kk = 0; kk < Nc / 16; ++kk)
+                    mma_ss(tmem, smem_desc(smem_u32(sP) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024),
+                           smem_desc(smem_u32(sV) + kk * 2048, SUB, 1024), idesc, kk > 0);
+                mma_commit(bar_mma);
+            }
+            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            ph_mma ^= 1;
+            tc_fence_after();
+            if (tid == 0 && have_next && !*abort_flag) issue_qk(dn);   // P is dead: Q, K of the next item
+
+            // ---- drain O, stage it (bf16) in the V tile, store ----
+            float lse = NEG, w0 = 0.f;
+            if (l > 0.f) { w0 = 1.f / l; lse = (m + log2f(l)) * LN2; }
+            float *po = nullptr;
+            if (up >= 0) {
+                po = a.part_o + ((size_t)up * H + h) * D;
+                a.part_lse[(size_t)up * H + h] = lse;
+            }
+#pragma unroll
+            for (int k = 0; k < D / 32; ++k) {
+                uint32_t r[32];
+                tmem_ld32(tmem + lane_base + 32 * k, r);
+                tmem_wait_ld();
+                float x[32];
+#pragma unroll
+                for (int j = 0; j < 32; ++j) x[j] = (w0 > 0.f) ? __uint_as_float(r[j]) * w0 : 0.f;
+                if (po != nullptr) {
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4)
+                        *reinterpret_cast<float4 *>(po + 32 * k + j) = make_float4(x[j], x[j + 1], x[j + 2], x[j + 3]);
+                }
+                uint32_t pk[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) pk[j] = pack_bf16(x[2 * j], x[2 * j + 1]);
+                uint8_t *dst = sV + (k >> 1) * SUB;
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    *reinterpret_cast<uint4 *>(dst + swz(tid, (k & 1) * 4 + c)) =
+                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            }
+            if (inb) a.lse[(size_t)h * a.T + row] = lse;
+            tc_fence_before();
+            __syncthreads();
+            {
+                __nv_bfloat16 *og = reinterpret_cast<__nv_bfloat16 *>(a.o);
+                const int nrows = r1 - r0;
+                for (int idx = tid; idx < NSUB * 128 * 8; idx += 128) {
+                    const int t = idx >> 10, rem = idx & 1023, r = rem >> 3, c = rem & 7;
+                    if (r < nrows) {
+                        const uint4 v = *reinterpret_cast<const uint4 *>(sV + t * SUB + swz(r, c));
+                        *reinterpret_cast<uint4 *>(og + ((size_t)(r0 + r) * H + h) * D + t * 64 + c * 8) = v;
+                    }
+                }
+            }
+            __syncthreads();   // the staged O has been read: the V tile may be overwritten
+            if (tid == 0 && have_next && !*abort_flag) issue_v(dn);
+            dc = dn; dn = dn2;
+        }
+    }
+    if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
 // Cycle counts per phase of k_fwd_tc_p, accumulated by thread 0 of CTA 0 (diagnostics).
 __device__ long long g_fwd_phase_cycles[16];
 #define HDT_STAMP(i)                                        \
@@ -531,6 +751,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     if (!attr) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             8 * SUB + 4 * 128 * 4 + 1024 + 64));
         attr = true;
@@ -546,8 +767,15 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
             HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
             const long long items = (long long)a.n_fused * a.H;
             k_fwd_tc_p<<<(int)(items < n_sm ? items : n_sm), 512, smem_p, st>>>(tq, tk, tv, a);
-        } else {
+        } else if (a.no_persistent == 3) {       // option: one CTA per (block, head), no loop
             k_fwd_tc<D, true><<<dim3(a.n_fused, a.H), 128, smem_1, st>>>(tq, tk, tv, a);
+        } else {
+            int dev = 0, n_sm = 0;
+            HDT_CUDA_CHECK(cudaGetDevice(&dev));
+            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+            const long long items = (long long)a.n_fused * a.H;
+            const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
+            k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
         }
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());

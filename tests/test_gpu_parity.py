@@ -113,7 +113,7 @@ def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
     only, SIMT kernels on every stage."""
     # default kernels; general tensor-core kernels only; persistent forward; SIMT everywhere
     # (fp32 runs with and without the side-stream overlap of the upper stages)
-    opts = (({}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2}, {"force_simt": 1})
+    opts = (({}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2}, {"no_persistent": 3}, {"force_simt": 1})
             if dtype == "bf16" else ({}, {"no_overlap": 1}))
     for opt in opts:
         for k_, v_ in opt.items():
