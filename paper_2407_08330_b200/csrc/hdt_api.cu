@@ -228,31 +228,43 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
     // The stages above 0 do not depend on stage 0 until their results are merged: compute them on
     // the side stream while stage 0 runs, then finish each with an element-wise merge.
     const bool overlap = ix->n_stages > 1 && !g_no_overlap;
-    Side *sd = nullptr;
     if (overlap) {
+        Side *sd = nullptr;
         rc = get_side(&sd);
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
+        {   // stage 0 first, so that nothing delays its launch
+            FwdStageArgs a = stage_args(0);
+            ProfScope ps(PROF_FWD_STAGE0, st);
+            if (dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
+            else rc = launch_fwd_simt(a, head_dim, dtype, st);
+            if (rc) return rc;
+        }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+        ChainArgs c{};
+        c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 1;
+        c.tok1 = ix->st[1].tok;
         for (int s = 1; s < ix->n_stages; ++s) {
             FwdStageArgs a = stage_args(s);
             a.own_o = (float *)(ws + L.own[s][0]);
             a.own_lse = (float *)(ws + L.own[s][1]);
+            c.up[s] = ix->st[s].up; c.own[s][0] = a.own_o; c.own_lse[s] = a.own_lse;
             rc = launch_fwd_simt(a, head_dim, dtype, sd->s);
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+        HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
+        c.base[0] = (const float *)(ws + L.part[1][0]);
+        c.base_lse = (const float *)(ws + L.part[1][1]);
+        c.out[0] = o; c.lse = lse;
+        ProfScope ps(PROF_FWD_UPPER, st);
+        return launch_chain_merge(c, head_dim, dtype, st);
     }
     for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
         FwdStageArgs a = stage_args(s);
-        if (s == 1 && overlap) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         {
             ProfScope ps(s == 0 ? PROF_FWD_STAGE0 : PROF_FWD_UPPER, st);
-            if (s > 0 && overlap) {
-                a.own_o = (float *)(ws + L.own[s][0]);
-                a.own_lse = (float *)(ws + L.own[s][1]);
-                rc = launch_merge_fwd(a, head_dim, dtype, st);
-            } else if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
+            if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
             else rc = launch_fwd_simt(a, head_dim, dtype, st);
         }
         if (rc) return rc;
@@ -312,33 +324,44 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         return a;
     };
     const bool overlap = ix->n_stages > 1 && !g_no_overlap;
-    Side *sd = nullptr;
     if (overlap) {   // delta is ready: the upper stages' own gradients are computed beside stage 0
+        Side *sd = nullptr;
         rc = get_side(&sd);
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
+        {
+            BwdStageArgs a = stage_args(0);
+            ProfScope ps(PROF_BWD_STAGE0, st);
+            if (dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
+            else rc = launch_bwd_simt(a, head_dim, dtype, st);
+            if (rc) return rc;
+        }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+        ChainArgs c{};
+        c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 3;
+        c.tok1 = ix->st[1].tok;
         for (int s = 1; s < ix->n_stages; ++s) {
             BwdStageArgs a = stage_args(s);
             a.own_dq = (float *)(ws + L.own[s][0]);
             a.own_dk = (float *)(ws + L.own[s][1]);
             a.own_dv = (float *)(ws + L.own[s][2]);
+            c.up[s] = ix->st[s].up;
+            c.own[s][0] = a.own_dq; c.own[s][1] = a.own_dk; c.own[s][2] = a.own_dv;
             rc = launch_bwd_simt(a, head_dim, dtype, sd->s);
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+        HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
+        for (int k = 0; k < 3; ++k) c.base[k] = (const float *)(ws + L.part[1][k]);
+        c.out[0] = dq; c.out[1] = dk; c.out[2] = dv;
+        ProfScope ps(PROF_BWD_UPPER, st);
+        return launch_chain_merge(c, head_dim, dtype, st);
     }
     for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
         BwdStageArgs a = stage_args(s);
-        if (s == 1 && overlap) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         {
             ProfScope ps(s == 0 ? PROF_BWD_STAGE0 : PROF_BWD_UPPER, st);
-            if (s > 0 && overlap) {
-                a.own_dq = (float *)(ws + L.own[s][0]);
-                a.own_dk = (float *)(ws + L.own[s][1]);
-                a.own_dv = (float *)(ws + L.own[s][2]);
-                rc = launch_merge_bwd(a, head_dim, dtype, st);
-            } else if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
+            if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
             else rc = launch_bwd_simt(a, head_dim, dtype, st);
         }
         if (rc) return rc;

@@ -484,6 +484,68 @@ static int launch_merge_any(const FwdStageArgs *f, const BwdStageArgs *b, int D,
 int launch_merge_fwd(const FwdStageArgs &a, int D, int dtype, cudaStream_t st) { return launch_merge_any(&a, nullptr, D, dtype, st); }
 int launch_merge_bwd(const BwdStageArgs &a, int D, int dtype, cudaStream_t st) { return launch_merge_any(nullptr, &a, D, dtype, st); }
 
+template <int D, bool BF16>
+__global__ void __launch_bounds__(256) k_chain_merge(const ChainArgs c) {
+    constexpr int U = D / 4;
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long rowh = gid / U;           // stage-1 element * H + head
+    const int u4 = (int)(gid % U);
+    if (rowh >= (long long)c.n1 * c.H) return;
+    const int e1 = (int)(rowh / c.H), h = (int)(rowh % c.H);
+    const int t = c.tok1[e1];
+    const float NEG = -INFINITY;
+    if (c.nt == 1) {   // forward: log-sum-exp merge
+        float lse = c.base_lse[rowh];
+        float4 o = reinterpret_cast<const float4 *>(c.base[0] + rowh * D)[u4];
+        int e = e1;
+        for (int s = 1; s < c.n_stages; ++s) {
+            const size_t r = (size_t)e * c.H + h;
+            const float lc = c.own_lse[s][r];
+            if (lc > NEG) {
+                const float mx = fmaxf(lse, lc);
+                const float w0 = (lse > NEG) ? __expf(lse - mx) : 0.f, w1 = __expf(lc - mx);
+                const float tot = w0 + w1;
+                const float4 oc = reinterpret_cast<const float4 *>(c.own[s][0] + r * D)[u4];
+                scale4(o, w0 / tot);
+                axpy4(o, w1 / tot, oc);
+                lse = mx + __logf(tot);
+            }
+            e = c.up[s][e];
+            if (e < 0) break;
+        }
+        store4<BF16>(c.out[0], ((size_t)t * c.H + h) * D + 4 * u4, o);
+        if (u4 == 0) c.lse[(size_t)h * c.T + t] = lse;
+    } else {           // backward: sums
+#pragma unroll
+        for (int k = 0; k < 3; ++k) {
+            float4 x = reinterpret_cast<const float4 *>(c.base[k] + rowh * D)[u4];
+            int e = e1;
+            for (int s = 1; s < c.n_stages; ++s) {
+                const float4 y = reinterpret_cast<const float4 *>(c.own[s][k] + ((size_t)e * c.H + h) * D)[u4];
+                x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
+                e = c.up[s][e];
+                if (e < 0) break;
+            }
+            store4<BF16>(c.out[k], ((size_t)t * c.H + h) * D + 4 * u4, x);
+        }
+    }
+}
+
+template <int D, bool BF16>
+static int launch_chain_t(const ChainArgs &c, cudaStream_t st) {
+    const long long threads = (long long)c.n1 * c.H * (D / 4);
+    if (threads == 0) return HDT_OK;
+    k_chain_merge<D, BF16><<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(c);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+int launch_chain_merge(const ChainArgs &c, int D, int dtype, cudaStream_t st) {
+    if (D == 64) return dtype == HDT_BF16 ? launch_chain_t<64, true>(c, st) : launch_chain_t<64, false>(c, st);
+    if (D == 128) return dtype == HDT_BF16 ? launch_chain_t<128, true>(c, st) : launch_chain_t<128, false>(c, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
+}
+
 // Small row blocks (the stages above 0) run with 128-thread CTAs so that several fit on an SM.
 template <int D, bool BF16>
 static int launch_fwd_t(const FwdStageArgs &a, cudaStream_t st) {

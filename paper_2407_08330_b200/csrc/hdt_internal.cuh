@@ -133,5 +133,20 @@ int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int
 // with the partial from below (carry_*), handed on (part_*) and written to the caller's tensors.
 int launch_merge_fwd(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_merge_bwd(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
+// One launch that completes every token of stage 1 (= every token that lives in a stage above 0):
+// stage 0's partial merged with the own partials of all upper stages the token belongs to, found
+// by following the `up` maps.  nt = 1 tensor (forward: O with LSE) or 3 (backward: dQ, dK, dV).
+struct ChainArgs {
+    int n1, H, T, n_stages, nt;
+    const int *tok1;
+    const int *up[HDT_MAX_STAGES];           // up[s]: stage s -> stage s+1
+    const float *own[HDT_MAX_STAGES][3];     // own[s][t], s >= 1
+    const float *own_lse[HDT_MAX_STAGES];    // forward only
+    const float *base[3];                    // stage 0's partials for stage 1's elements
+    const float *base_lse;
+    void *out[3];
+    float *lse;
+};
+int launch_chain_merge(const ChainArgs &c, int head_dim, int dtype, cudaStream_t st);
 
 }  // namespace hdt
