@@ -233,13 +233,6 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         rc = get_side(&sd);
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
-        {   // stage 0 first, so that nothing delays its launch
-            FwdStageArgs a = stage_args(0);
-            ProfScope ps(PROF_FWD_STAGE0, st);
-            if (dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
-            else rc = launch_fwd_simt(a, head_dim, dtype, st);
-            if (rc) return rc;
-        }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 1;
@@ -253,6 +246,14 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+        {   // stage 0 after the small side kernels are queued: they take their SM share first (the
+            // stage-0 kernel would otherwise fill every SM and push them behind itself)
+            FwdStageArgs a = stage_args(0);
+            ProfScope ps(PROF_FWD_STAGE0, st);
+            if (dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
+            else rc = launch_fwd_simt(a, head_dim, dtype, st);
+            if (rc) return rc;
+        }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         c.base[0] = (const float *)(ws + L.part[1][0]);
         c.base_lse = (const float *)(ws + L.part[1][1]);
@@ -329,13 +330,6 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         rc = get_side(&sd);
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
-        {
-            BwdStageArgs a = stage_args(0);
-            ProfScope ps(PROF_BWD_STAGE0, st);
-            if (dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
-            else rc = launch_bwd_simt(a, head_dim, dtype, st);
-            if (rc) return rc;
-        }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 3;
@@ -351,6 +345,13 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+        {
+            BwdStageArgs a = stage_args(0);
+            ProfScope ps(PROF_BWD_STAGE0, st);
+            if (dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
+            else rc = launch_bwd_simt(a, head_dim, dtype, st);
+            if (rc) return rc;
+        }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         for (int k = 0; k < 3; ++k) c.base[k] = (const float *)(ws + L.part[1][k]);
         c.out[0] = dq; c.out[1] = dk; c.out[2] = dv;
