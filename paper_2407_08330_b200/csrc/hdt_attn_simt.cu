@@ -408,82 +408,9 @@ __global__ void __launch_bounds__(256) k_delta(const void *o, const void *d_o, f
 }
 
 // ---------------------------------------------------------------------------------------------
-// Completion of a stage above 0 that was computed beside stage 0 (one thread per 4 values).
+// Completion of the tokens that live in stages above 0, after those stages were computed beside
+// stage 0 (one thread per 4 values of a (stage-1 element, head)).
 // ---------------------------------------------------------------------------------------------
-template <int D, bool BF16>
-__global__ void __launch_bounds__(256) k_merge_fwd(const FwdStageArgs a) {
-    constexpr int U = D / 4;
-    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long rowh = gid / U;           // element * H + head
-    const int u4 = (int)(gid % U);
-    if (rowh >= (long long)a.n * a.H) return;
-    const int e = (int)(rowh / a.H), h = (int)(rowh % a.H);
-    const float NEG = -INFINITY;
-    float lse = a.own_lse[rowh];
-    float4 o = reinterpret_cast<const float4 *>(a.own_o + rowh * D)[u4];
-    const float lc = a.carry_lse[rowh];
-    if (lc > NEG) {
-        const float mx = fmaxf(lse, lc);
-        const float e0 = (lse > NEG) ? __expf(lse - mx) : 0.f, e1 = __expf(lc - mx);
-        const float tot = e0 + e1;
-        const float4 oc = reinterpret_cast<const float4 *>(a.carry_o + rowh * D)[u4];
-        scale4(o, e0 / tot);
-        axpy4(o, e1 / tot, oc);
-        lse = mx + __logf(tot);
-    }
-    const int up = (a.part_o != nullptr) ? a.up[e] : -1;
-    if (up >= 0) {
-        reinterpret_cast<float4 *>(a.part_o + ((size_t)up * a.H + h) * D)[u4] = o;
-        if (u4 == 0) a.part_lse[(size_t)up * a.H + h] = lse;
-    }
-    const int t = a.tok[e];
-    store4<BF16>(a.o, ((size_t)t * a.H + h) * D + 4 * u4, o);
-    if (u4 == 0) a.lse[(size_t)h * a.T + t] = lse;
-}
-
-template <int D, bool BF16>
-__global__ void __launch_bounds__(256) k_merge_bwd(const BwdStageArgs a) {
-    constexpr int U = D / 4;
-    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const long long rowh = gid / U;
-    const int u4 = (int)(gid % U);
-    if (rowh >= (long long)a.n * a.H) return;
-    const int e = (int)(rowh / a.H), h = (int)(rowh % a.H);
-    const int up = (a.part_dq != nullptr) ? a.up[e] : -1;
-    const int t = a.tok[e];
-    const float *own[3] = {a.own_dq, a.own_dk, a.own_dv};
-    const float *car[3] = {a.carry_dq, a.carry_dk, a.carry_dv};
-    float *part[3] = {a.part_dq, a.part_dk, a.part_dv};
-    void *fin[3] = {a.dq, a.dk, a.dv};
-#pragma unroll
-    for (int c = 0; c < 3; ++c) {
-        float4 x = reinterpret_cast<const float4 *>(own[c] + rowh * D)[u4];
-        const float4 y = reinterpret_cast<const float4 *>(car[c] + rowh * D)[u4];
-        x.x += y.x; x.y += y.y; x.z += y.z; x.w += y.w;
-        if (up >= 0) reinterpret_cast<float4 *>(part[c] + ((size_t)up * a.H + h) * D)[u4] = x;
-        store4<BF16>(fin[c], ((size_t)t * a.H + h) * D + 4 * u4, x);
-    }
-}
-
-template <int D, bool BF16>
-static int launch_merge_t(const FwdStageArgs *f, const BwdStageArgs *b, cudaStream_t st) {
-    const long long threads = (long long)(f ? f->n : b->n) * (f ? f->H : b->H) * (D / 4);
-    if (threads == 0) return HDT_OK;
-    const unsigned grid = (unsigned)((threads + 255) / 256);
-    if (f) k_merge_fwd<D, BF16><<<grid, 256, 0, st>>>(*f);
-    else k_merge_bwd<D, BF16><<<grid, 256, 0, st>>>(*b);
-    count_launch();
-    HDT_CUDA_CHECK(cudaGetLastError());
-    return HDT_OK;
-}
-static int launch_merge_any(const FwdStageArgs *f, const BwdStageArgs *b, int D, int dtype, cudaStream_t st) {
-    if (D == 64) return dtype == HDT_BF16 ? launch_merge_t<64, true>(f, b, st) : launch_merge_t<64, false>(f, b, st);
-    if (D == 128) return dtype == HDT_BF16 ? launch_merge_t<128, true>(f, b, st) : launch_merge_t<128, false>(f, b, st);
-    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
-}
-int launch_merge_fwd(const FwdStageArgs &a, int D, int dtype, cudaStream_t st) { return launch_merge_any(&a, nullptr, D, dtype, st); }
-int launch_merge_bwd(const BwdStageArgs &a, int D, int dtype, cudaStream_t st) { return launch_merge_any(nullptr, &a, D, dtype, st); }
-
 template <int D, bool BF16>
 __global__ void __launch_bounds__(256) k_chain_merge(const ChainArgs c) {
     constexpr int U = D / 4;

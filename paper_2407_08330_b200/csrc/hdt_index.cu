@@ -785,9 +785,13 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     }
     HDT_BUILD_CHECK(cudaGetLastError());
     }
-    DevHeader h;
-    HDT_BUILD_CHECK(cudaMemcpyAsync(&h, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, st));
+    // the header comes back through a pinned host buffer (one per host thread, allocated once):
+    // a copy to pageable memory would be staged by the driver
+    static thread_local DevHeader *h_pinned = nullptr;
+    if (!h_pinned) HDT_BUILD_CHECK(cudaMallocHost((void **)&h_pinned, sizeof(DevHeader)));
+    HDT_BUILD_CHECK(cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, st));
     HDT_BUILD_CHECK(cudaStreamSynchronize(st));
+    const DevHeader h = *h_pinned;
 #undef HDT_BUILD_CHECK
     if (h.status != 0) {
         delete ix;

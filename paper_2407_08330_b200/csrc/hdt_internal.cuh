@@ -129,10 +129,6 @@ int read_fwd_phase_cycles(long long *out16);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
                  cudaStream_t st);
-// Element-wise completion of a stage that was computed beside stage 0: own partial (own_*) merged
-// with the partial from below (carry_*), handed on (part_*) and written to the caller's tensors.
-int launch_merge_fwd(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
-int launch_merge_bwd(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 // One launch that completes every token of stage 1 (= every token that lives in a stage above 0):
 // stage 0's partial merged with the own partials of all upper stages the token belongs to, found
 // by following the `up` maps.  nt = 1 tensor (forward: O with LSE) or 3 (backward: dQ, dK, dV).
