@@ -237,6 +237,9 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
+    # everything runs on an explicit stream (the legacy default stream cannot be captured into the
+    # CUDA graph hdt_build_index replays)
+    torch.cuda.set_stream(torch.cuda.Stream(device=dev))
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 

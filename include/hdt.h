@@ -222,8 +222,9 @@ int hdt_attn_fwd_static(const hdt_index_t *index, const void *q, const void *k, 
  * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
  * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
  * general tensor-core kernels, = 2 the persistent forward kernel; "no_overlap" = 1 runs the stages
- * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream
- * (A/B comparisons, tests).
+ * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream;
+ * "no_graph" = 1 makes hdt_build_index launch its kernels one by one instead of replaying a cached
+ * CUDA graph (A/B comparisons, tests).
  */
 int hdt_set_option(const char *name, int32_t value);
 

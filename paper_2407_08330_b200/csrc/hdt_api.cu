@@ -63,6 +63,7 @@ int *device_status_ptr() {
 // One non-blocking stream and two events per host thread and device, created on first use.
 static thread_local Side g_side[64];
 int g_no_overlap = 0;
+int g_no_graph = 0;
 
 int get_side(Side **out) {
     int dev = -1;
@@ -130,6 +131,7 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "force_simt") == 0) { g_force_simt = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_persistent") == 0) { g_no_persistent = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_overlap") == 0) { g_no_overlap = value; return HDT_OK; }
+    if (name && std::strcmp(name, "no_graph") == 0) { g_no_graph = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 

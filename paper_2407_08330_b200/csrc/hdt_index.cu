@@ -11,6 +11,7 @@
 //   blocks    per block key span, flags, cost
 //   queue     rank sort by cost (longest first)
 #include <cstdio>
+#include <cstring>
 
 #include "hdt_internal.cuh"
 
@@ -717,73 +718,117 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         }                                                                              \
     } while (0)
 
-    {
-    ProfScope ps(PROF_INDEX, st);
-    // header, cnt and nlc are adjacent in the workspace: one memset clears all three
-    HDT_BUILD_CHECK(cudaMemsetAsync(ws + L.header, 0, L.pre - L.header, st));
     const int nel = max(T, B + 1);
     const int g_el = (nel + 255) / 256;
     const int g_chunk = max(1, (T + CHUNK - 1) / CHUNK);
     const int g_stride = max(1, min((T + 255) / 256, 148 * 8));
     static const int kSmemCap = 200 * 1024;
     HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
-    k_init<<<g_el, 256, 0, st>>>(level, parent, cu_seqlens, B, T, HDT_MAX_STAGES * 8, hdr, ix->st[0].tok,
-                                 ix->st[0].par, ix->st[0].scu, cnt);
-    count_launch();
     const bool fused_upper = (B <= UMAXB);
     // The upper stages only need stage 0's compaction; with their own scratch they are built on the
     // side stream while stage 0's blocks and queues are built on the caller's stream.
     Side *sd = nullptr;
     if (fused_upper && ms > 1 && !g_no_overlap && get_side(&sd) != HDT_OK) sd = nullptr;
-    auto launch_upper = [&](cudaStream_t s_) {
-        UpperArgs u;
-        for (int i = 0; i < HDT_MAX_STAGES; ++i) u.st[i] = ix->st[i < ms ? i : ms - 1];
-        u.max_stages = ms; u.B = B; u.bm = bmu;
-        u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.keep = keep;
-        u.bstart = (int *)(ws + L.bstart2); u.seqcount = (int *)(ws + L.seqcount2);
-        u.fpos = (uint8_t *)(ws + L.fpos2); u.cost = (long long *)(ws + L.cost2);
-        k_upper_stages<<<1, UT, 0, s_>>>(hdr, u);
-        count_launch();
-    };
-    for (int s = 0; s < ms; ++s) {
-        if (s >= 1 && fused_upper) {
-            if (sd) HDT_BUILD_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
-            else launch_upper(st);
-            break;
-        }
-        const StagePtrs &P = ix->st[s];
-        // the last possible stage writes its (unused) next-stage arrays into its own up/pre scratch
-        const StagePtrs &N = ix->st[(s + 1 < ms) ? s + 1 : s];
-        const bool last = (s + 1 == ms);
-        if (s >= 1) { k_count<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt); count_launch(); }
-        k_nlc<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt, nlc);
-        k_ranges<<<g_chunk, CHUNK, 0, st>>>(hdr, s, s == 0 ? level : nullptr, P.par, cnt, nlc, P.rng, keep,
-                                            fpos, blocksum);
-        // tok2 of the last possible stage is never read: point it at scratch (pre is rewritten first)
-        k_scan<<<g_chunk, CHUNK, 0, st>>>(hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
-                                          last ? cnt : N.tok);
-        if (!last) {
-            k_compact<<<g_stride, 256, 0, st>>>(hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc);
-            count_launch();
-            if (s == 0 && sd) {   // fork: the upper stages start now
-                HDT_BUILD_CHECK(cudaEventRecord(sd->fork, st));
-                HDT_BUILD_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
-                launch_upper(sd->s);
-                HDT_BUILD_CHECK(cudaEventRecord(sd->join, sd->s));
+
+    // Everything the build enqueues; returns the first CUDA error.  Called directly or under
+    // stream capture (see below).
+    int n_launched = 0;
+    auto enqueue_all = [&]() -> cudaError_t {
+        cudaError_t e;
+#define HDT_ENQ(expr) do { e = (expr); if (e != cudaSuccess) return e; } while (0)
+        // header, cnt and nlc are adjacent in the workspace: one memset clears all three
+        HDT_ENQ(cudaMemsetAsync(ws + L.header, 0, L.pre - L.header, st));
+        k_init<<<g_el, 256, 0, st>>>(level, parent, cu_seqlens, B, T, HDT_MAX_STAGES * 8, hdr, ix->st[0].tok,
+                                     ix->st[0].par, ix->st[0].scu, cnt);
+        ++n_launched;
+        auto launch_upper = [&](cudaStream_t s_) {
+            UpperArgs u;
+            for (int i = 0; i < HDT_MAX_STAGES; ++i) u.st[i] = ix->st[i < ms ? i : ms - 1];
+            u.max_stages = ms; u.B = B; u.bm = bmu;
+            u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.keep = keep;
+            u.bstart = (int *)(ws + L.bstart2); u.seqcount = (int *)(ws + L.seqcount2);
+            u.fpos = (uint8_t *)(ws + L.fpos2); u.cost = (long long *)(ws + L.cost2);
+            k_upper_stages<<<1, UT, 0, s_>>>(hdr, u);
+            ++n_launched;
+        };
+        for (int s = 0; s < ms; ++s) {
+            if (s >= 1 && fused_upper) {
+                if (sd) HDT_ENQ(cudaStreamWaitEvent(st, sd->join, 0));
+                else launch_upper(st);
+                break;
+            }
+            const StagePtrs &P = ix->st[s];
+            // the last possible stage writes its (unused) next-stage arrays into its own up/pre scratch
+            const StagePtrs &N = ix->st[(s + 1 < ms) ? s + 1 : s];
+            const bool last = (s + 1 == ms);
+            if (s >= 1) { k_count<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt); ++n_launched; }
+            k_nlc<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt, nlc);
+            k_ranges<<<g_chunk, CHUNK, 0, st>>>(hdr, s, s == 0 ? level : nullptr, P.par, cnt, nlc, P.rng, keep,
+                                                fpos, blocksum);
+            // tok2 of the last possible stage is never read: point it at scratch (pre is rewritten first)
+            k_scan<<<g_chunk, CHUNK, 0, st>>>(hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
+                                              last ? cnt : N.tok);
+            n_launched += 3;
+            if (!last) {
+                k_compact<<<g_stride, 256, 0, st>>>(hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc);
+                ++n_launched;
+                if (s == 0 && sd) {   // fork: the upper stages start now
+                    HDT_ENQ(cudaEventRecord(sd->fork, st));
+                    HDT_ENQ(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+                    launch_upper(sd->s);
+                    HDT_ENQ(cudaEventRecord(sd->join, sd->s));
+                }
+            }
+            if (B > 0) {
+                int maxlen_smem = kSmemCap;  // sequences longer than this walk through global memory
+                const int bms = (s == 0) ? bm : bmu;
+                k_walk<<<B, 256, kSmemCap, st>>>(hdr, s, bms, P.scu, fpos, bstart, seqcount, maxlen_smem);
+                const int gy = max(1, min(64, 2048 / max(B, 1)));   // enough CTAs to spread a few long sequences
+                k_blocks<<<dim3(B, gy), 256, 0, st>>>(hdr, s, bms, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost);
+                k_queue<<<max(1, min(L.capnb / 256 + 1, 148 * 4)), 256, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
+                n_launched += 3;
             }
         }
-        if (B > 0) {
-            int maxlen_smem = kSmemCap;  // sequences longer than this walk through global memory
-            const int bms = (s == 0) ? bm : bmu;
-            k_walk<<<B, 256, kSmemCap, st>>>(hdr, s, bms, P.scu, fpos, bstart, seqcount, maxlen_smem);
-            const int gy = max(1, min(64, 2048 / max(B, 1)));   // enough CTAs to spread a few long sequences
-            k_blocks<<<dim3(B, gy), 256, 0, st>>>(hdr, s, bms, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost);
-            k_queue<<<max(1, min(L.capnb / 256 + 1, 148 * 4)), 256, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
-            count_launch(3);
+        return cudaGetLastError();
+#undef HDT_ENQ
+    };
+
+    {
+        ProfScope ps(PROF_INDEX, st);
+        // The build is a dozen tiny kernels: launching them one by one is slower than running them.
+        // They are captured once into a CUDA graph, which is replayed while the same buffers, sizes
+        // and parameters come back (one cached graph per host thread).
+        struct GraphKey { const void *a, *b, *c, *w; int B, T, bm, ms, bmu, ov; };
+        struct GraphCache { GraphKey key; cudaGraphExec_t exec; int launches; bool valid; };
+        static thread_local GraphCache cache{};
+        const GraphKey key{level, parent, cu_seqlens, workspace, B, T, bm, ms, bmu, sd ? 1 : 0};
+        bool done = false;
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        // (the legacy and per-thread default streams cannot be captured)
+        const bool capturable = st != nullptr && st != cudaStreamLegacy && st != cudaStreamPerThread;
+        if (!g_no_graph && capturable && cudaStreamIsCapturing(st, &cap) == cudaSuccess &&
+            cap == cudaStreamCaptureStatusNone) {
+            if (cache.valid && std::memcmp(&cache.key, &key, sizeof(key)) == 0) {
+                if (cudaGraphLaunch(cache.exec, st) == cudaSuccess) { done = true; count_launch(cache.launches); }
+            } else if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
+                const cudaError_t e = enqueue_all();
+                cudaGraph_t g = nullptr;
+                const cudaError_t e2 = cudaStreamEndCapture(st, &g);
+                cudaGraphExec_t exec = nullptr;
+                if (e == cudaSuccess && e2 == cudaSuccess && g && cudaGraphInstantiate(&exec, g, 0) == cudaSuccess) {
+                    if (cache.valid) cudaGraphExecDestroy(cache.exec);
+                    cache = GraphCache{key, exec, n_launched, true};
+                    if (cudaGraphLaunch(exec, st) == cudaSuccess) { done = true; count_launch(n_launched); }
+                }
+                if (g) cudaGraphDestroy(g);
+                if (!done) (void)cudaGetLastError();   // fall back to direct launches below
+            }
         }
-        count_launch(3);
-    }
-    HDT_BUILD_CHECK(cudaGetLastError());
+        if (!done) {
+            n_launched = 0;
+            HDT_BUILD_CHECK(enqueue_all());
+            count_launch(n_launched);
+        }
     }
     // the header comes back through a pinned host buffer (one per host thread, allocated once):
     // a copy to pageable memory would be staged by the driver

@@ -69,6 +69,7 @@ struct ProfScope {
 struct Side { cudaStream_t s; cudaEvent_t fork, join; bool ready; };
 int get_side(Side **out);
 extern int g_no_overlap;   // option "no_overlap"
+extern int g_no_graph;     // option "no_graph"
 
 // SIMT attention launchers (hdt_attn_simt.cu).  One launch handles one stage.
 struct FwdStageArgs {

@@ -60,6 +60,32 @@ def test_index_generic_trees_and_degenerate(P):
     assert_index_equal(P, gen.pack([(np.zeros(0, np.int8), np.zeros(0, np.int32))]))
 
 
+def test_index_graph_replay_with_new_contents(P):
+    """hdt_build_index replays a cached CUDA graph while buffers and sizes repeat: the second build
+    reuses every buffer of the first with another hierarchy of the same size written into them."""
+    rng = np.random.default_rng(3)
+    batches = [gen.pack([gen.gen_fill(rng, 700, (2, 6), (2, 9), (3, 30)) for _ in range(3)]) for _ in range(3)]
+    lv, pa, cu = dev_struct(batches[0])
+    ws = torch.empty(P.hdt_index_workspace_bytes(3, 2100, 0, 4), dtype=torch.uint8, device="cuda")
+    for no_graph in (0, 1):
+        P.hdt_set_option("no_graph", no_graph)
+        try:
+          with torch.cuda.stream(torch.cuda.Stream()):      # the default stream cannot be captured
+            for b in batches:
+                lv.copy_(torch.from_numpy(b.level).cuda()); pa.copy_(torch.from_numpy(b.parent).cuda())
+                cu.copy_(torch.from_numpy(b.cu_seqlens).cuda())
+                idx = P.hdt_build_index(lv, pa, cu, max_stages=4, workspace=ws)
+                want = ix.build(b.level, b.parent, b.cu_seqlens, 128)
+                assert idx.nnz == want.nnz and idx.n_stages == len(want.stages)
+                for s_, st in enumerate(want.stages):
+                    got = idx.export(s_)
+                    for name in ("rng", "up", "blocks", "queue", "queue_split"):
+                        assert np.array_equal(got[name], getattr(st, name)), (s_, name)
+            torch.cuda.current_stream().synchronize()
+        finally:
+            P.hdt_set_option("no_graph", 0)
+
+
 def test_index_many_sequences(P):
     """More sequences than the single-CTA upper-stage builder takes: the per-stage kernels run."""
     rng = np.random.default_rng(12)
