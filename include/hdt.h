@@ -219,6 +219,25 @@ int hdt_attn_fwd_static(const hdt_index_t *index, const void *q, const void *k, 
                         void *stream);
 
 /*
+ * Hierarchical positional encoding (paper, paragraph "Hierarchical Positional Encoding", the
+ * positional-encoding equation): HPE(p, 2k) = sum_l sin(w_k p^l), HPE(p, 2k+1) = sum_l cos(w_k p^l),
+ * w_k = 10000^(-2k/d_model), l = 1..n_levels, where p^l is the number (from 1) of the token's
+ * level-l ancestor (or of the token itself) among its siblings, and 0 on levels deeper than the
+ * token's own.  The root has p = 0 on every level; PAD tokens get 0 (accumulate = 0) or are left
+ * unchanged (accumulate = 1).
+ *   index              built from the same level / parent / cu_seqlens (its stages give the
+ *                      sibling numbers)
+ *   x                  device [total_tokens, d_model] of `dtype`; overwritten (accumulate = 0) or
+ *                      incremented (accumulate = 1: token embeddings + HPE, as the encoder input)
+ *   workspace          device, >= hdt_hpe_workspace_bytes(index, n_levels), 256-byte aligned
+ * d_model must be even.  Asynchronous on `stream`.
+ */
+size_t hdt_hpe_workspace_bytes(const hdt_index_t *index, int32_t n_levels);
+int hdt_hpe(const hdt_index_t *index, const int8_t *level, const int32_t *parent, const int32_t *cu_seqlens,
+            int32_t n_levels, int32_t d_model, int32_t dtype, int32_t accumulate, void *x, void *workspace,
+            size_t workspace_bytes, void *stream);
+
+/*
  * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
  * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
  * general tensor-core kernels, = 2 the persistent forward kernel; "no_overlap" = 1 runs the stages

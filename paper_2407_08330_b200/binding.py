@@ -228,6 +228,26 @@ def hdt_attn_fwd_static(index: HdtIndex, q, k, v, softmax_scale=0.0, out=None, l
     return o, lse
 
 
+def hdt_hpe(index: HdtIndex, level, parent, cu_seqlens, d_model, n_levels=3, dtype=torch.float32, x=None,
+            accumulate=False, workspace=None):
+    """Hierarchical positional encoding [T, d_model]; with `x` and accumulate=True it is added to x."""
+    L = lib()
+    L.hdt_hpe_workspace_bytes.restype = C.c_size_t
+    L.hdt_hpe_workspace_bytes.argtypes = [C.c_void_p, C.c_int32]
+    L.hdt_hpe.restype = C.c_int
+    L.hdt_hpe.argtypes = [C.c_void_p] * 4 + [C.c_int32] * 4 + [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+    T = level.numel()
+    if x is None:
+        x = torch.empty((T, d_model), dtype=dtype, device=level.device)
+    assert x.is_contiguous() and x.shape == (T, d_model)
+    need = int(L.hdt_hpe_workspace_bytes(index.handle, n_levels))
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=level.device)
+    _check(L.hdt_hpe(index.handle, _ptr(level), _ptr(parent), _ptr(cu_seqlens), n_levels, d_model, _DTYPES[x.dtype],
+                     int(bool(accumulate)), _ptr(x), _ptr(workspace), workspace.numel(), _stream()))
+    return x
+
+
 def hdt_set_option(name: str, value: int) -> None:
     lib().hdt_set_option.restype = C.c_int
     _check(lib().hdt_set_option(C.c_char_p(name.encode()), C.c_int32(int(value))))

@@ -1,0 +1,45 @@
+"""GPU parity of hdt_hpe against the fp64 oracle (fp32 <= 1e-4, bf16 within bf16 rounding)."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+from gpu_util import dev_struct
+from oracle import hpe_oracle as ho
+
+pytestmark = pytest.mark.gpu
+
+
+def run(P, b, d_model, n_levels, dtype, max_stages=8):
+    lv, pa, cu = dev_struct(b)
+    idx = P.hdt_build_index(lv, pa, cu, max_stages=max_stages)
+    want = ho.hpe(b.level, b.parent, b.cu_seqlens, d_model, n_levels)
+    got = P.hdt_hpe(idx, lv, pa, cu, d_model, n_levels, dtype=dtype).float().cpu().numpy().astype(np.float64)
+    tol = 1e-4 if dtype == torch.float32 else 2e-2
+    assert np.abs(got - want).max() <= tol
+    # accumulate: x + HPE
+    x0 = torch.randn((b.total_tokens, d_model), device="cuda").to(dtype)
+    x = x0.clone()
+    P.hdt_hpe(idx, lv, pa, cu, d_model, n_levels, x=x, accumulate=True)
+    pad = torch.from_numpy(b.level < 0).cuda()
+    assert torch.equal(x[pad], x0[pad])
+    err = np.abs(x.float().cpu().numpy() - (x0.float().cpu().numpy() + want))
+    assert err.max() <= (1e-4 if dtype == torch.float32 else 6e-2)
+    P.hdt_device_status()
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_hpe_small_and_generic(dtype):
+    import paper_2407_08330_b200 as P
+    for seed in range(3):
+        run(P, gen.small_random_batch(seed, n_seqs=4, max_len=400, K=(0, 40)), 64, 3, dtype)
+    rng = np.random.default_rng(4)
+    b = gen.pack([gen.layout_tree(gen.random_tree(rng, int(rng.integers(2, 7)), 5)) for _ in range(10)])
+    run(P, b, 96, 6, dtype)
+    run(P, b, 6, 2, dtype)          # fewer levels than the trees have: deeper levels are ignored
+
+
+def test_hpe_config_sizes():
+    import paper_2407_08330_b200 as P
+    run(P, gen.make_hierarchy(1), 768, 3, torch.float32)
+    run(P, gen.make_hierarchy(5), 768, 3, torch.float32, max_stages=4)   # sibling numbers up to ~1000
