@@ -222,6 +222,7 @@ def main():
     ap.add_argument("--impl", default="hdt", choices=["hdt", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-hpe", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -371,12 +372,38 @@ def main():
                "h2d_bytes_per_step": n_in * T * H * d * esz + T * 5 + (b.batch + 1) * 4,
                "d2h_bytes_per_step": n_out * T * H * d * esz + H * T * 4, "ms_per_step": e_ms}
 
+    # the step before the path, timed alone on the same batch: hierarchical positional encoding
+    # added to a resident [T, heads*head_dim] embedding (read + write of x, p-vectors from the index)
+    hpe = None
+    if rank == 0 and not args.no_hpe:
+        d_model = H * d
+        x = torch.zeros((T, d_model), dtype=tdt, device=dev)
+        idx = P.hdt_build_index(level, parent, cu, max_stages=4, workspace=ws_index)
+        ws_h = torch.empty(max(256, P.hdt_hpe_workspace_bytes(idx, 3)), dtype=torch.uint8, device=dev)
+
+        def step_hpe():
+            P.hdt_hpe(idx, level, parent, cu, d_model, n_levels=3, x=x, accumulate=True, workspace=ws_h)
+
+        for _ in range(3):
+            step_hpe()
+        l1 = P.hdt_launch_count()
+        th = timed(step_hpe, args.steps)
+        hpe_ms = float(np.mean(th))
+        hpe_bytes = 2 * T * d_model * x.element_size() + T * 5
+        hpe = {"ms": hpe_ms, "algorithmic_bytes": hpe_bytes, "achieved_gbs": hpe_bytes / (hpe_ms * 1e-3) / 1e9,
+               "launches": (P.hdt_launch_count() - l1) // args.steps, "d_model": d_model, "levels": 3,
+               "mode": "x += HPE(p)"}
+        idx.close()
+        del x, ws_h
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     pk = peaks()
+    if hpe:
+        hpe["frac_of_hbm_peak"] = hpe["achieved_gbs"] / pk["hbm_gbs"]
     fl = flops_per_step(nnz, H, d, cfg.backward)
     value = fl * world / (ms * 1e-3) / 1e12
     real = b.real_tokens
@@ -413,6 +440,8 @@ def main():
         "kernels": kern, "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches),
         "clocks": clk.summary(),
     }
+    if hpe:
+        line["next_rows"] = {"hpe": hpe}
     if not args.no_cpu_baseline and world >= 1:
         line["cpu_baseline"] = cpu_baseline(c, cfg, b)
     print(json.dumps(line))

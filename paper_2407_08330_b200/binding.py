@@ -228,6 +228,13 @@ def hdt_attn_fwd_static(index: HdtIndex, q, k, v, softmax_scale=0.0, out=None, l
     return o, lse
 
 
+def hdt_hpe_workspace_bytes(index: HdtIndex, n_levels=3) -> int:
+    L = lib()
+    L.hdt_hpe_workspace_bytes.restype = C.c_size_t
+    L.hdt_hpe_workspace_bytes.argtypes = [C.c_void_p, C.c_int32]
+    return int(L.hdt_hpe_workspace_bytes(index.handle, n_levels))
+
+
 def hdt_hpe(index: HdtIndex, level, parent, cu_seqlens, d_model, n_levels=3, dtype=torch.float32, x=None,
             accumulate=False, workspace=None):
     """Hierarchical positional encoding [T, d_model]; with `x` and accumulate=True it is added to x."""
