@@ -124,6 +124,23 @@ def gen_fill(rng, L, S, M, K):
     return fit(lv, pa, L, pad=False) + (doc,)
 
 
+def gen_pseudo(rng, L, K, per_section=32):
+    """Flat text: sentences of U{K} tokens are drawn until the document reaches L and grouped into
+    pseudo-sections of exactly `per_section` consecutive sentences (the last one may be shorter);
+    cut at L."""
+    sents = []
+    total = 1
+    while total < L:
+        if len(sents) % per_section == 0:
+            total += 1                      # the [SEC] anchor of a new pseudo-section
+        k = _u(rng, K)
+        sents.append(k)
+        total += 1 + k
+    doc = [sents[i:i + per_section] for i in range(0, len(sents), per_section)]
+    lv, pa = layout(doc)
+    return fit(lv, pa, L, pad=False) + (doc,)
+
+
 def zipf_len(rng, a=1.5, cap=1024, clip=False) -> int:
     k = int(rng.zipf(a))
     if clip:
@@ -224,6 +241,10 @@ CONFIGS = {
               "16 packed documents, lengths U{512..16384}, same generator as c3, head_dim 128"),
     5: Config("c5_skew_2x32768", 12, 64, "bf16", True, 1005, 2005,
               "2 documents of 32768: one section with 60% of tokens, Zipf(1.5) sentences capped 1024, 200 small sections"),
+    # not one of the five headline configurations: flat text cut into pseudo-sections of 32 sentences
+    # (the paper's setting for inputs without document structure), shape of config 3 otherwise
+    6: Config("c6_pseudo32_b4_L8192", 12, 64, "bf16", True, 1006, 2006,
+              "4 flat documents of 8192 tokens; pseudo-sections of 32 sentences, tokens U{5..60}"),
 }
 
 
@@ -243,6 +264,8 @@ def make_hierarchy(c: int, clip: bool = False) -> Batch:
         return pack([gen_fill(rng, L, (4, 24), (3, 20), (5, 60)) for L in lens])
     if c == 5:
         return pack([gen_skew(rng, 32768, clip=clip) for _ in range(2)])
+    if c == 6:
+        return pack([gen_pseudo(rng, 8192, (5, 60)) for _ in range(4)])
     raise KeyError(c)
 
 

@@ -66,9 +66,9 @@ typedef struct {
     int32_t block_m;    /* max rows per row block, 1..128; 0 = default 128                     */
     int32_t max_stages; /* max hierarchy height handled, 1..HDT_MAX_STAGES; 0 = default 4
                            ([DOC]/[SEC]/[SENT]/token documents need 3)                        */
-    int32_t block_m_upper; /* max rows per row block in the stages above 0 (their arrays are a
-                           few percent of the tokens: smaller blocks give their kernels more
-                           CTAs), 1..128; 0 = default 32                                      */
+    int32_t block_m_upper; /* max rows per row block in the stages above 0, 1..128; 0 = default
+                           128 (whole families per block for the tensor-core kernels; the fp32
+                           SIMT kernels of those stages get more CTAs from smaller blocks)    */
     int32_t reserved[5];
 } hdt_index_params_t;
 
@@ -240,7 +240,9 @@ int hdt_hpe(const hdt_index_t *index, const int8_t *level, const int32_t *parent
 /*
  * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
  * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
- * general tensor-core kernels, = 2 the persistent forward kernel; "no_overlap" = 1 runs the stages
+ * general tensor-core kernels, = 2 the persistent forward kernel, = 3 the forward kernel with one CTA
+ * per (block, head); "simt_upper" = 1 computes the stages above 0 of bf16 calls on the fp32 SIMT
+ * kernels instead of the gathering tensor-core kernels; "no_overlap" = 1 runs the stages
  * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream;
  * "no_graph" = 1 makes hdt_build_index launch its kernels one by one instead of replaying a cached
  * CUDA graph (A/B comparisons, tests).

@@ -108,7 +108,7 @@ def validate(level, parent, cu):
                     raise BadHierarchy("level must be parent's level + 1")
 
 
-def build(level, parent, cu, block_m: int = 128, max_stages: int = 32, block_m_upper: int = 32) -> Index:
+def build(level, parent, cu, block_m: int = 128, max_stages: int = 32, block_m_upper: int = 128) -> Index:
     level = np.asarray(level, np.int8)
     parent = np.asarray(parent, np.int32)
     cu = np.asarray(cu, np.int32)

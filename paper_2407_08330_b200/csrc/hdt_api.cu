@@ -60,7 +60,9 @@ int *device_status_ptr() {
 }
 
 // ---- side stream: the stages above 0 run beside stage 0 -------------------------------------------
-// One non-blocking stream and two events per host thread and device, created on first use.
+// Two non-blocking streams (odd and even stages: their kernels are independent and should all
+// be resident before stage 0 fills the SMs) and three events per host thread and device, created
+// on first use.
 static thread_local Side g_side[64];
 int g_no_overlap = 0;
 int g_no_graph = 0;
@@ -72,8 +74,10 @@ int get_side(Side **out) {
     Side &sd = g_side[dev];
     if (!sd.ready) {
         HDT_CUDA_CHECK(cudaStreamCreateWithFlags(&sd.s, cudaStreamNonBlocking));
+        HDT_CUDA_CHECK(cudaStreamCreateWithFlags(&sd.s2, cudaStreamNonBlocking));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.fork, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join, cudaEventDisableTiming));
+        HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join2, cudaEventDisableTiming));
         sd.ready = true;
     }
     *out = &sd;
@@ -126,10 +130,12 @@ using namespace hdt;
 
 static int g_force_simt = 0;
 static int g_no_persistent = 0;
+static int g_simt_upper = 0;
 
 extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "force_simt") == 0) { g_force_simt = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_persistent") == 0) { g_no_persistent = value; return HDT_OK; }
+    if (name && std::strcmp(name, "simt_upper") == 0) { g_simt_upper = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_overlap") == 0) { g_no_overlap = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_graph") == 0) { g_no_graph = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
@@ -236,6 +242,12 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+        const bool two = ix->n_stages > 2;
+        if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
+        // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
+        // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
+        // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
+        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3;
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 1;
         c.tok1 = ix->st[1].tok;
@@ -244,10 +256,13 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
             a.own_o = (float *)(ws + L.own[s][0]);
             a.own_lse = (float *)(ws + L.own[s][1]);
             c.up[s] = ix->st[s].up; c.own[s][0] = a.own_o; c.own_lse[s] = a.own_lse;
-            rc = launch_fwd_simt(a, head_dim, dtype, sd->s);
+            cudaStream_t ss = (s & 1) ? sd->s : sd->s2;
+            if (tc_upper) rc = launch_fwd_tc_upper(a, head_dim, ss);
+            else rc = launch_fwd_simt(a, head_dim, dtype, ss);
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+        if (two) HDT_CUDA_CHECK(cudaEventRecord(sd->join2, sd->s2));
         {   // stage 0 after the small side kernels are queued: they take their SM share first (the
             // stage-0 kernel would otherwise fill every SM and push them behind itself)
             FwdStageArgs a = stage_args(0);
@@ -257,6 +272,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
+        if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
         c.base[0] = (const float *)(ws + L.part[1][0]);
         c.base_lse = (const float *)(ws + L.part[1][1]);
         c.out[0] = o; c.lse = lse;
@@ -333,6 +349,12 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
+        const bool two = ix->n_stages > 2;
+        if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
+        // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
+        // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
+        // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
+        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3;
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 3;
         c.tok1 = ix->st[1].tok;
@@ -343,10 +365,13 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             a.own_dv = (float *)(ws + L.own[s][2]);
             c.up[s] = ix->st[s].up;
             c.own[s][0] = a.own_dq; c.own[s][1] = a.own_dk; c.own[s][2] = a.own_dv;
-            rc = launch_bwd_simt(a, head_dim, dtype, sd->s);
+            cudaStream_t ss = (s & 1) ? sd->s : sd->s2;
+            if (tc_upper) rc = launch_bwd_tc_upper(a, head_dim, ss);
+            else rc = launch_bwd_simt(a, head_dim, dtype, ss);
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
+        if (two) HDT_CUDA_CHECK(cudaEventRecord(sd->join2, sd->s2));
         {
             BwdStageArgs a = stage_args(0);
             ProfScope ps(PROF_BWD_STAGE0, st);
@@ -355,6 +380,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
+        if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
         for (int k = 0; k < 3; ++k) c.base[k] = (const float *)(ws + L.part[1][k]);
         c.out[0] = dq; c.out[1] = dk; c.out[2] = dv;
         ProfScope ps(PROF_BWD_UPPER, st);

@@ -28,10 +28,45 @@ static constexpr long long WAIT_CYCLES = 400000000LL;  // ~0.2 s: bound of every
 // byte offset of 16-byte chunk c (0..7) of row r inside a swizzled sub-tile
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
-// SINGLE = true: the block has one key chunk (SELF blocks).  Q and K are dead once S is computed and
-// S is dead once P is written, so P reuses the Q/K tiles and O reuses S's TMEM columns: 48 KB of
-// shared memory and 128 TMEM columns per CTA at D = 64, four CTAs per SM.
-template <int D, bool SINGLE>
+// Stages above 0: elements [row0, row0 + 128) of the stage are token rows tok[e] of [T, H, D] bf16
+// tensors.  The threads copy them (head h) into D / 64 swizzled sub-tiles per tensor, the layout
+// the TMA loads of stage 0 produce; elements at or beyond `end` become zero rows.  Thread t owns
+// 16-byte chunk t % 8 of rows t / 8, t / 8 + NT / 8, ...; all indices are loaded first, then all
+// rows of all NTEN tensors, then everything is stored, so that the loads overlap.
+template <int D, int NT, int NTEN>
+__device__ __forceinline__ void gather_tiles(uint8_t *const (&dst)[NTEN], const void *const (&src)[NTEN],
+                                             const int *__restrict__ tok, int row0, int end, int H, int h, int tid) {
+    constexpr int RPP = NT / 8, NP = 128 / RPP, NSUB = D / 64;
+    const int c = tid & 7, rr = tid >> 3;
+    int tk[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const int e = row0 + rr + p * RPP;
+        tk[p] = e < end ? tok[e] : -1;
+    }
+#pragma unroll
+    for (int t = 0; t < NSUB; ++t) {
+        uint4 v[NTEN][NP];
+#pragma unroll
+        for (int x = 0; x < NTEN; ++x) {
+            const __nv_bfloat16 *g = reinterpret_cast<const __nv_bfloat16 *>(src[x]);
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                v[x][p] = make_uint4(0u, 0u, 0u, 0u);
+                if (tk[p] >= 0) v[x][p] = *reinterpret_cast<const uint4 *>(g + ((size_t)tk[p] * H + h) * D + t * 64 + c * 8);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < NTEN; ++x)
+#pragma unroll
+            for (int p = 0; p < NP; ++p) *reinterpret_cast<uint4 *>(dst[x] + t * SUB + swz(rr + p * RPP, c)) = v[x][p];
+    }
+}
+
+// GATHER = true (with SINGLE = false): a stage above 0 computed beside stage 0.  Rows are gathered
+// through the stage's tok map by the threads instead of TMA, and the kernel leaves only the
+// stage's own partial result per element (fp32 O, LSE, indexed by element) for the chain merge.
+template <int D, bool SINGLE, bool GATHER = false>
 __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensorMap tm_q,
                                                 const __grid_constant__ CUtensorMap tm_k,
                                                 const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
@@ -85,16 +120,29 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             const int nvalid = min(128, kb - c0);
             const int Nc = (nvalid + 15) & ~15;
             const bool first = (c0 == ka);
-            if (tid == 0 && !*abort_flag) {   // after a failed wait nothing new is issued
-                mbar_expect_tx(bar_tma, (uint32_t)((first ? NSUB : 0) + 2 * NSUB) * SUB);
-                for (int s = 0; s < NSUB; ++s) {
-                    if (first) tma_load_3d(sQ + s * SUB, &tm_q, 64 * s, h, r0, bar_tma);
-                    tma_load_3d(sK + s * SUB, &tm_k, 64 * s, h, c0, bar_tma);
-                    tma_load_3d(sV + s * SUB, &tm_v, 64 * s, h, c0, bar_tma);
+            if constexpr (GATHER) {
+                if (first) {
+                    uint8_t *const dq_[1] = {sQ};
+                    const void *const sq_[1] = {a.q};
+                    gather_tiles<D, 128, 1>(dq_, sq_, a.tok, r0, r1, H, h, tid);
                 }
+                uint8_t *const dkv[2] = {sK, sV};
+                const void *const skv[2] = {a.k, a.v};
+                gather_tiles<D, 128, 2>(dkv, skv, a.tok, c0, kb, H, h, tid);
+                fence_proxy_async_smem();     // generic-proxy writes, read by the MMA
+                __syncthreads();
+            } else {
+                if (tid == 0 && !*abort_flag) {   // after a failed wait nothing new is issued
+                    mbar_expect_tx(bar_tma, (uint32_t)((first ? NSUB : 0) + 2 * NSUB) * SUB);
+                    for (int s = 0; s < NSUB; ++s) {
+                        if (first) tma_load_3d(sQ + s * SUB, &tm_q, 64 * s, h, r0, bar_tma);
+                        tma_load_3d(sK + s * SUB, &tm_k, 64 * s, h, c0, bar_tma);
+                        tma_load_3d(sV + s * SUB, &tm_v, 64 * s, h, c0, bar_tma);
+                    }
+                }
+                ok = mbar_wait(bar_tma, ph_tma, abort_flag, WAIT_CYCLES) && ok;
+                ph_tma ^= 1;
             }
-            ok = mbar_wait(bar_tma, ph_tma, abort_flag, WAIT_CYCLES) && ok;
-            ph_tma ^= 1;
             if (tid == 0 && !*abort_flag) {
                 tc_fence_after();
                 const uint32_t idesc = idesc_bf16(Nc, false, false);
@@ -201,6 +249,36 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
     // result (O, LSE) there, the next stage completes and overwrites them; stage O, store ----
     float lse = NEG, w0 = 0.f;
     if (l > 0.f) { w0 = 1.f / l; lse = (m + log2f(l)) * LN2; }
+    if constexpr (GATHER) {
+        float *own = inb ? a.own_o + ((size_t)row * H + h) * D : nullptr;
+#pragma unroll
+        for (int k = 0; k < D / 32; ++k) {
+            uint32_t r[32];
+            if (!empty && !dead) {      // uniform in the CTA
+                tmem_ld32(tmem + TM_O + lane_base + 32 * k, r);
+                tmem_wait_ld();
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
+            }
+            if (own != nullptr) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    float4 x;
+                    x.x = (w0 > 0.f) ? __uint_as_float(r[j]) * w0 : 0.f;
+                    x.y = (w0 > 0.f) ? __uint_as_float(r[j + 1]) * w0 : 0.f;
+                    x.z = (w0 > 0.f) ? __uint_as_float(r[j + 2]) * w0 : 0.f;
+                    x.w = (w0 > 0.f) ? __uint_as_float(r[j + 3]) * w0 : 0.f;
+                    *reinterpret_cast<float4 *>(own + 32 * k + j) = x;
+                }
+            }
+        }
+        if (inb) a.own_lse[(size_t)row * H + h] = lse;
+        tc_fence_before();
+        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+        return;
+    }
     float *po = nullptr;
     if (inb && a.part_o != nullptr) {
         const int u = a.up[row];
@@ -789,6 +867,35 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         HDT_CUDA_CHECK(cudaGetLastError());
     }
     return HDT_OK;
+}
+
+// A stage above 0 in own-partial mode (a.tok and a.own_* set): one CTA per (block, head).
+template <int D>
+static int launch_fwd_tc_upper_t(const FwdStageArgs &a, cudaStream_t st) {
+    CUtensorMap tq;     // the gathering kernel takes no tensor map; the parameter slots get a valid one
+    int rc = make_tmap_bf16(&tq, a.q, D, a.H, a.T, 128);
+    if (rc) return rc;
+    constexpr int smem = (3 * (D / 64) + 2) * SUB + 1024 + 64;
+    static bool attr = false;
+    if (!attr) {
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr = true;
+    }
+    FwdStageArgs b = a;
+    b.rest_only = 0;
+    k_fwd_tc<D, false, true><<<dim3(a.nb, a.H), 128, smem, st>>>(tq, tq, tq, b);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+
+int launch_fwd_tc_upper(const FwdStageArgs &a, int D, cudaStream_t st) {
+    if (a.nb == 0) return HDT_OK;
+    if (a.tok == nullptr || a.own_o == nullptr || a.own_lse == nullptr)
+        return set_error(HDT_ERR_INVALID_ARG, "launch_fwd_tc_upper: needs a tok map and own-partial buffers");
+    if (D == 64) return launch_fwd_tc_upper_t<64>(a, st);
+    if (D == 128) return launch_fwd_tc_upper_t<128>(a, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
 }
 
 int launch_fwd_tc(const FwdStageArgs &a, int D, cudaStream_t st) {

@@ -25,7 +25,45 @@ static constexpr int SUB = 16384;
 static constexpr long long WAIT_CYCLES = 400000000LL;
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
-template <int D>
+// Stages above 0: elements [row0, row0 + 128) of the stage are token rows tok[e] of [T, H, D] bf16
+// tensors.  The threads copy them (head h) into D / 64 swizzled sub-tiles per tensor, the layout
+// the TMA loads of stage 0 produce; elements at or beyond `end` become zero rows.  Thread t owns
+// 16-byte chunk t % 8 of rows t / 8, t / 8 + NT / 8, ...; all indices are loaded first, then all
+// rows of all NTEN tensors, then everything is stored, so that the loads overlap.
+template <int D, int NT, int NTEN>
+__device__ __forceinline__ void gather_tiles(uint8_t *const (&dst)[NTEN], const void *const (&src)[NTEN],
+                                             const int *__restrict__ tok, int row0, int end, int H, int h, int tid) {
+    constexpr int RPP = NT / 8, NP = 128 / RPP, NSUB = D / 64;
+    const int c = tid & 7, rr = tid >> 3;
+    int tk[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const int e = row0 + rr + p * RPP;
+        tk[p] = e < end ? tok[e] : -1;
+    }
+#pragma unroll
+    for (int t = 0; t < NSUB; ++t) {
+        uint4 v[NTEN][NP];
+#pragma unroll
+        for (int x = 0; x < NTEN; ++x) {
+            const __nv_bfloat16 *g = reinterpret_cast<const __nv_bfloat16 *>(src[x]);
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                v[x][p] = make_uint4(0u, 0u, 0u, 0u);
+                if (tk[p] >= 0) v[x][p] = *reinterpret_cast<const uint4 *>(g + ((size_t)tk[p] * H + h) * D + t * 64 + c * 8);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < NTEN; ++x)
+#pragma unroll
+            for (int p = 0; p < NP; ++p) *reinterpret_cast<uint4 *>(dst[x] + t * SUB + swz(rr + p * RPP, c)) = v[x][p];
+    }
+}
+
+// GATHER = true: a stage above 0 computed beside stage 0.  Rows (and their LSE / delta) are fetched
+// through the stage's tok map by the threads instead of TMA, and the kernel leaves only the stage's
+// own gradients per element (fp32, indexed by element) for the chain merge.
+template <int D, bool GATHER = false>
 __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensorMap tm_q,
                                                 const __grid_constant__ CUtensorMap tm_k,
                                                 const __grid_constant__ CUtensorMap tm_v,
@@ -107,8 +145,9 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
             lo = a.rng[2 * e];
             hi = a.rng[2 * e + 1];
             if (hi > lo) {
-                lse2 = a.lse[(size_t)h * a.T + e] * LOG2E;
-                dl = a.delta[(size_t)h * a.T + e];
+                const int tk = GATHER ? a.tok[e] : e;
+                lse2 = a.lse[(size_t)h * a.T + tk] * LOG2E;
+                dl = a.delta[(size_t)h * a.T + tk];
             }
         }
         const int jl = max(lo - k_row0, 0), jh = min(hi - k_row0, nk);
@@ -187,6 +226,27 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     };
 
     auto load = [&](bool q_side, int row0_q, bool k_side, int row0_k) {
+        if constexpr (GATHER) {
+            if (q_side && k_side && row0_q == row0_k) {
+                uint8_t *const d4[4] = {sQ, sDO, sK, sV};
+                const void *const s4[4] = {a.q, a.d_o, a.k, a.v};
+                gather_tiles<D, 256, 4>(d4, s4, a.tok, row0_q, a.n, H, h, tid);
+            } else {
+                if (q_side) {
+                    uint8_t *const d2[2] = {sQ, sDO};
+                    const void *const s2[2] = {a.q, a.d_o};
+                    gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_q, a.n, H, h, tid);
+                }
+                if (k_side) {
+                    uint8_t *const d2[2] = {sK, sV};
+                    const void *const s2[2] = {a.k, a.v};
+                    gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_k, a.n, H, h, tid);
+                }
+            }
+            fence_proxy_async_smem();     // generic-proxy writes, read by the MMAs
+            __syncthreads();
+            return;
+        }
         if (tid == 0 && !*abort_flag) {
             mbar_expect_tx(bar_tma, (uint32_t)((q_side ? 2 * NSUB : 0) + (k_side ? 2 * NSUB : 0)) * SUB);
             for (int s = 0; s < NSUB; ++s) {
@@ -248,7 +308,13 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     const int row = r0 + rl;
     const bool inb = row < r1;
     float *cq = nullptr, *ck = nullptr, *cv = nullptr;
-    if (inb && a.part_dq != nullptr) {
+    if constexpr (GATHER) {
+        if (inb) {      // the drains write the own gradients here; the staged bf16 copies are not used
+            cq = a.own_dq + ((size_t)row * H + h) * D;
+            ck = a.own_dk + ((size_t)row * H + h) * D;
+            cv = a.own_dv + ((size_t)row * H + h) * D;
+        }
+    } else if (inb && a.part_dq != nullptr) {
         const int u = a.up[row];
         if (u >= 0) {
             cq = a.part_dq + ((size_t)u * H + h) * D;
@@ -278,7 +344,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
-        copy_out(sP, a.dq);
+        if constexpr (!GATHER) copy_out(sP, a.dq);
         __syncthreads();
         if (run) {
             // this block as keys: dK, dV over the same span taken as query rows
@@ -294,9 +360,11 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     }
     tc_fence_before();
     __syncthreads();
-    if (fused) copy_out(sP, a.dq);   // same decision in every thread
-    copy_out(sDS, a.dk);
-    copy_out(sQ, a.dv);
+    if constexpr (!GATHER) {
+        if (fused) copy_out(sP, a.dq);   // same decision in every thread
+        copy_out(sDS, a.dk);
+        copy_out(sQ, a.dv);
+    }
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
@@ -744,6 +812,35 @@ int read_bwd_phase_cycles(long long *out16) {
     long long zero[16] = {0};
     HDT_CUDA_CHECK(cudaMemcpyToSymbol(g_bwd_phase_cycles, zero, sizeof(zero)));
     return HDT_OK;
+}
+
+// A stage above 0 in own-gradient mode (a.tok and a.own_* set): one CTA per (block, head).
+template <int D>
+static int launch_bwd_tc_upper_t(const BwdStageArgs &a, cudaStream_t st) {
+    CUtensorMap tq;     // the gathering kernel takes no tensor map; the parameter slots get a valid one
+    int rc = make_tmap_bf16(&tq, a.q, D, a.H, a.T, 128);
+    if (rc) return rc;
+    constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64;
+    static bool attr = false;
+    if (!attr) {
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr = true;
+    }
+    BwdStageArgs b = a;
+    b.rest_only = 0;
+    k_bwd_tc<D, true><<<dim3(a.nb, a.H), 256, smem, st>>>(tq, tq, tq, tq, b);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+
+int launch_bwd_tc_upper(const BwdStageArgs &a, int D, cudaStream_t st) {
+    if (a.nb == 0) return HDT_OK;
+    if (a.tok == nullptr || a.own_dq == nullptr || a.own_dk == nullptr || a.own_dv == nullptr)
+        return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_upper: needs a tok map and own-gradient buffers");
+    if (D == 64) return launch_bwd_tc_upper_t<64>(a, st);
+    if (D == 128) return launch_bwd_tc_upper_t<128>(a, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
 }
 
 int launch_bwd_tc(const BwdStageArgs &a, int D, cudaStream_t st) {

@@ -660,7 +660,7 @@ using namespace hdt;
 static void norm_params(const hdt_index_params_t *p, int &bm, int &ms, int &bmu) {
     bm = (p && p->block_m) ? p->block_m : 128;
     ms = (p && p->max_stages) ? p->max_stages : 4;
-    bmu = (p && p->block_m_upper) ? p->block_m_upper : 32;
+    bmu = (p && p->block_m_upper) ? p->block_m_upper : 128;
 }
 
 extern "C" size_t hdt_index_workspace_bytes(int32_t batch, int32_t total_tokens,

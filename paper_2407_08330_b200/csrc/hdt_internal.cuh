@@ -66,7 +66,7 @@ struct ProfScope {
 
 // Side stream (one per host thread and device, created on first use): work that does not depend
 // on the main kernel of a call runs beside it.  fork / join are events for the two hand-overs.
-struct Side { cudaStream_t s; cudaEvent_t fork, join; bool ready; };
+struct Side { cudaStream_t s, s2; cudaEvent_t fork, join, join2; bool ready; };
 int get_side(Side **out);
 extern int g_no_overlap;   // option "no_overlap"
 extern int g_no_graph;     // option "no_graph"
@@ -125,6 +125,9 @@ int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t
 // Tensor-core (TMA + tcgen05) stage-0 kernels for bf16 (hdt_attn_tc.cu).
 int launch_fwd_tc(const FwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_bwd_tc(const BwdStageArgs &a, int head_dim, cudaStream_t st);
+// Stages above 0 in own-partial mode on the tensor-core kernels (rows gathered through tok).
+int launch_fwd_tc_upper(const FwdStageArgs &a, int head_dim, cudaStream_t st);
+int launch_bwd_tc_upper(const BwdStageArgs &a, int head_dim, cudaStream_t st);
 int read_bwd_phase_cycles(long long *out16);
 int read_fwd_phase_cycles(long long *out16);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);

@@ -19,7 +19,7 @@ def P():
     return P
 
 
-def assert_index_equal(P, b, block_m=128, max_stages=8, block_m_upper=32):
+def assert_index_equal(P, b, block_m=128, max_stages=8, block_m_upper=128):
     want = ix.build(b.level, b.parent, b.cu_seqlens, block_m, block_m_upper=block_m_upper)
     idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=max_stages, block_m_upper=block_m_upper)
     assert idx.n_stages == len(want.stages)
@@ -93,7 +93,7 @@ def test_index_many_sequences(P):
     assert_index_equal(P, gen.pack(seqs), 128, max_stages=4)
 
 
-@pytest.mark.parametrize("c", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("c", [1, 2, 3, 4, 5, 6])
 def test_index_configs(P, c):
     b = gen.make_hierarchy(c)
     idx = assert_index_equal(P, b, 128, max_stages=4)
@@ -139,21 +139,25 @@ def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
     only, SIMT kernels on every stage."""
     # default kernels; general tensor-core kernels only; persistent forward; SIMT everywhere
     # (fp32 runs with and without the side-stream overlap of the upper stages)
-    opts = (({}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2}, {"no_persistent": 3}, {"force_simt": 1})
+    # (the upper stages of bf16 runs: gathering tensor-core kernels with 128- and 32-row blocks, SIMT)
+    opts = (({}, {"_block_m_upper": 32}, {"simt_upper": 1}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2},
+             {"no_persistent": 3}, {"force_simt": 1})
             if dtype == "bf16" else ({}, {"no_overlap": 1}))
     for opt in opts:
+        opt = dict(opt)
+        bmu = opt.pop("_block_m_upper", 0)
         for k_, v_ in opt.items():
             P.hdt_set_option(k_, v_)
         try:
-            _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale)
+            _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale, bmu)
         finally:
             for k_ in opt:
                 P.hdt_set_option(k_, 0)
 
 
-def _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale):
+def _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale, block_m_upper=0):
     t = gen.make_tensors(seed, b.total_tokens, H, d, dtype)
-    idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=8)
+    idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=8, block_m_upper=block_m_upper)
     q, k, v, do = (dev_tensor(t[n], dtype) for n in ("q", "k", "v", "do"))
     o, lse = P.hdt_attn_fwd(idx, q, k, v, softmax_scale=scale)
     sc = scale if scale > 0 else None
@@ -234,7 +238,7 @@ def test_argument_errors(P):
 # ------------------------------------------------------------------------------------------
 # full-size configurations: sampled rows / keys against the oracle, properties everywhere
 # ------------------------------------------------------------------------------------------
-@pytest.mark.parametrize("c", [2, 3, 4, 5])
+@pytest.mark.parametrize("c", [2, 3, 4, 5, 6])
 def test_full_size_config_sampled(P, c):
     cfg = gen.CONFIGS[c]
     b = gen.make_hierarchy(c)
