@@ -135,40 +135,43 @@ def oracle_sample(c, cfg, b, heads=None, seqs=None):
     return sub, t, H
 
 
-def oracle_step(sub, t, backward):
+def oracle_step(sub, t, backward, directions=7):
     import oracle
     t0 = time.perf_counter()
-    oracle.forward(sub.level, sub.parent, sub.cu_seqlens, t["q"], t["k"], t["v"])
+    oracle.forward(sub.level, sub.parent, sub.cu_seqlens, t["q"], t["k"], t["v"], directions=directions)
     if backward:
-        oracle.backward(sub.level, sub.parent, sub.cu_seqlens, t["q"], t["k"], t["v"], t["do"])
+        oracle.backward(sub.level, sub.parent, sub.cu_seqlens, t["q"], t["k"], t["v"], t["do"], directions=directions)
     return time.perf_counter() - t0
 
 
-def oracle_nnz(sub):
-    ch = np.zeros(sub.total_tokens, np.int64)
+def oracle_nnz(sub, directions=7):
+    """Unmasked pairs of the batch from counts alone: the diagonal, one entry per non-root token
+    for each of the child->parent and parent->child groups, c (c - 1) sibling entries per family
+    of c children."""
     nnz = 0
     for s in range(sub.batch):
         lo, hi = sub.cu_seqlens[s], sub.cu_seqlens[s + 1]
         pa = sub.parent[lo:hi]
         real = sub.level[lo:hi] >= 0
-        if not real.any():
-            continue
-        c = np.bincount(pa[pa >= 0], minlength=hi - lo)
-        heads = np.flatnonzero(c > 0)
-        nnz += int(((1 + c[heads]) ** 2).sum()) - int((heads != 0).sum()) if real.sum() > 1 else 1
+        c = np.bincount(pa[(pa >= 0) & real], minlength=hi - lo).astype(np.int64)
+        non_root = int(((pa >= 0) & real).sum())
+        nnz += int(real.sum()) + non_root * (bool(directions & 1) + bool(directions & 4))
+        if directions & 2:
+            nnz += int((c * (c - 1)).sum())
     return nnz
 
 
 CPU_SAMPLES = {2: dict(seqs=None, heads=None), 3: dict(seqs=None, heads=None),
-               4: dict(seqs=[0, 1], heads=4), 5: dict(seqs=[0], heads=2), 1: dict(seqs=None, heads=None)}
+               4: dict(seqs=[0, 1], heads=4), 5: dict(seqs=[0], heads=2), 1: dict(seqs=None, heads=None),
+               6: dict(seqs=None, heads=None), 7: dict(seqs=None, heads=None)}
 
 
-def cpu_baseline(c, cfg, b):
+def cpu_baseline(c, cfg, b, directions=7):
     import oracle
     spec = CPU_SAMPLES[c]
     sub, t, H = oracle_sample(c, cfg, b, spec["heads"], spec["seqs"])
-    dt = oracle_step(sub, t, cfg.backward)
-    fl = flops_per_step(oracle_nnz(sub), H, cfg.head_dim, cfg.backward)
+    dt = oracle_step(sub, t, cfg.backward, directions)
+    fl = flops_per_step(oracle_nnz(sub, directions), H, cfg.head_dim, cfg.backward)
     return {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.threads(), "kind": "oracle",
             "sample": f"{sub.batch} of {b.batch} sequences ({sub.total_tokens} tokens), {H} of {cfg.heads} heads, "
                       f"forward{'+backward' if cfg.backward else ''} once, {dt:.2f} s",
@@ -187,14 +190,15 @@ def run_reference(args):
     budget = 90.0 / max(total, 1)
     # probe with one head of sequence 0 to size the sample
     sub, t, _ = oracle_sample(c, cfg, b, 1, [0])
-    t1 = oracle_step(sub, t, cfg.backward)
+    dirs = args.directions
+    t1 = oracle_step(sub, t, cfg.backward, dirs)
     heads = int(max(1, min(cfg.heads, budget // max(t1, 1e-3))))
     sub, t, H = oracle_sample(c, cfg, b, heads, [0])
     for _ in range(args.warmup):
-        oracle_step(sub, t, cfg.backward)
-    times = [oracle_step(sub, t, cfg.backward) for _ in range(args.steps)]
+        oracle_step(sub, t, cfg.backward, dirs)
+    times = [oracle_step(sub, t, cfg.backward, dirs) for _ in range(args.steps)]
     dt = float(np.mean(times))
-    fl = flops_per_step(oracle_nnz(sub), H, cfg.head_dim, cfg.backward)
+    fl = flops_per_step(oracle_nnz(sub, dirs), H, cfg.head_dim, cfg.backward)
     val = fl / dt / 1e12
     sample = (f"sequence 0 of {b.batch} ({sub.total_tokens} tokens), {H} of {cfg.heads} heads, "
               f"forward{'+backward' if cfg.backward else ''} per step")
@@ -218,7 +222,9 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5, 6])
+    ap.add_argument("--config", type=int, default=3, choices=[1, 2, 3, 4, 5, 6, 7])
+    ap.add_argument("--directions", type=int, default=7, choices=range(8),
+                    help="bits 1|2|4 keep the child->parent, sibling, parent->child entries (7 = full rule)")
     ap.add_argument("--impl", default="hdt", choices=["hdt", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -269,8 +275,9 @@ def main():
     o = torch.empty_like(q)
     lse = torch.empty((H, T), dtype=torch.float32, device=dev)
     dq, dk, dv = torch.empty_like(q), torch.empty_like(q), torch.empty_like(q)
-    ws_index = torch.empty(P.hdt_index_workspace_bytes(b.batch, T, 0, 4), dtype=torch.uint8, device=dev)
-    idx0 = P.hdt_build_index(level, parent, cu, max_stages=4, workspace=ws_index)
+    max_st = 24 if c == 7 else 4      # expression trees reach depth 20
+    ws_index = torch.empty(P.hdt_index_workspace_bytes(b.batch, T, 0, max_st), dtype=torch.uint8, device=dev)
+    idx0 = P.hdt_build_index(level, parent, cu, max_stages=max_st, workspace=ws_index, directions=args.directions)
     nnz = idx0.nnz
     ws_f = torch.empty(max(256, P.hdt_attn_workspace_bytes(idx0, H, d, tdt, 0)), dtype=torch.uint8, device=dev)
     ws_b = torch.empty(max(256, P.hdt_attn_workspace_bytes(idx0, H, d, tdt, 1)), dtype=torch.uint8, device=dev)
@@ -279,7 +286,7 @@ def main():
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > 126 MB L2
 
     def step():
-        idx = P.hdt_build_index(level, parent, cu, max_stages=4, workspace=ws_index)
+        idx = P.hdt_build_index(level, parent, cu, max_stages=max_st, workspace=ws_index, directions=args.directions)
         P.hdt_attn_fwd(idx, q, k, v, out=o, lse=lse, workspace=ws_f)
         if cfg.backward:
             P.hdt_attn_bwd(idx, q, k, v, o, lse, do, dq=dq, dk=dk, dv=dv, workspace=ws_b)
@@ -378,7 +385,7 @@ def main():
     if rank == 0 and not args.no_hpe:
         d_model = H * d
         x = torch.zeros((T, d_model), dtype=tdt, device=dev)
-        idx = P.hdt_build_index(level, parent, cu, max_stages=4, workspace=ws_index)
+        idx = P.hdt_build_index(level, parent, cu, max_stages=max_st, workspace=ws_index, directions=args.directions)
         ws_h = torch.empty(max(256, P.hdt_hpe_workspace_bytes(idx, 3)), dtype=torch.uint8, device=dev)
 
         def step_hpe():
@@ -431,7 +438,7 @@ def main():
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": cfg.name, "description": cfg.description, "batch": b.batch, "total_tokens": T,
                    "real_tokens": real, "heads": H, "head_dim": d, "nnz_pairs_per_head": nnz,
-                   "visited_pairs_per_head": visited, "stages": n_stages,
+                   "visited_pairs_per_head": visited, "stages": n_stages, "directions": args.directions,
                    "step": "hdt_build_index + hdt_attn_fwd" + (" + hdt_attn_bwd" if cfg.backward else ""),
                    "l2": "flushed between timed steps (256 MiB write, untimed)", "parallelism": f"replicas x{world}"},
         "pct_bf16_peak": 100.0 * value / world / pk["bf16_tflops"],
@@ -443,7 +450,7 @@ def main():
     if hpe:
         line["next_rows"] = {"hpe": hpe}
     if not args.no_cpu_baseline and world >= 1:
-        line["cpu_baseline"] = cpu_baseline(c, cfg, b)
+        line["cpu_baseline"] = cpu_baseline(c, cfg, b, args.directions)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

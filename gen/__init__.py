@@ -179,6 +179,28 @@ def random_tree(rng, max_depth: int, max_children: int, p_leaf: float = 0.3):
     return t
 
 
+def listops_tree(rng, max_depth: int = 20, max_args: int = 5, max_len: int = 512, p_nest: float = 0.25):
+    """Nested-list expression tree shaped like a ListOps sample: every operator has 2..max_args
+    operands, an operand is a number (leaf) or, with probability p_nest and while depth and length
+    allow, another operator; at most max_depth operator levels and max_len tokens.  The root of
+    the list is the outermost operator."""
+    budget = [max_len - 1]
+
+    def op(depth):
+        n_args = int(rng.integers(2, max_args + 1))
+        kids = []
+        for _ in range(n_args):
+            if budget[0] <= 0:
+                break
+            budget[0] -= 1
+            if depth + 1 < max_depth and budget[0] >= 3 and rng.random() < p_nest:
+                kids.append(op(depth + 1))
+            else:
+                kids.append([])
+        return kids
+    return op(0)
+
+
 # ----------------------------------------------------------------------------
 # batches
 # ----------------------------------------------------------------------------
@@ -245,6 +267,10 @@ CONFIGS = {
     # (the paper's setting for inputs without document structure), shape of config 3 otherwise
     6: Config("c6_pseudo32_b4_L8192", 12, 64, "bf16", True, 1006, 2006,
               "4 flat documents of 8192 tokens; pseudo-sections of 32 sentences, tokens U{5..60}"),
+    # ListOps-shaped expression trees (depth <= 20, 2..5 operands, <= 512 tokens), batch 200,
+    # feature dimension 128 as 2 heads x 64; used with the directed mask variants
+    7: Config("c7_listops_b200_d20", 2, 64, "bf16", True, 1007, 2007,
+              "200 expression trees: operators with 2..5 operands, nesting probability 0.45, depth <= 20, <= 512 tokens"),
 }
 
 
@@ -266,6 +292,8 @@ def make_hierarchy(c: int, clip: bool = False) -> Batch:
         return pack([gen_skew(rng, 32768, clip=clip) for _ in range(2)])
     if c == 6:
         return pack([gen_pseudo(rng, 8192, (5, 60)) for _ in range(4)])
+    if c == 7:
+        return pack([layout_tree(listops_tree(rng, 20, 5, 512, 0.45)) for _ in range(200)])
     raise KeyError(c)
 
 

@@ -60,7 +60,7 @@ typedef enum {
 
 typedef enum { HDT_F32 = 0, HDT_BF16 = 1 } hdt_dtype_t;
 
-#define HDT_MAX_STAGES 16
+#define HDT_MAX_STAGES 24
 
 typedef struct {
     int32_t block_m;    /* max rows per row block, 1..128; 0 = default 128                     */
@@ -69,7 +69,13 @@ typedef struct {
     int32_t block_m_upper; /* max rows per row block in the stages above 0, 1..128; 0 = default
                            128 (whole families per block for the tensor-core kernels; the fp32
                            SIMT kernels of those stages get more CTAs from smaller blocks)    */
-    int32_t reserved[5];
+    int32_t mask_off;   /* directed variants of the rule (paper, "Mathematical Reasoning Tasks": the
+                           ListOps attention patterns): bit 0 switches OFF a token attending to its
+                           parent, bit 1 to its other siblings, bit 2 to its children; the diagonal
+                           always stays.  0 = the full parent/sibling/child rule.  The family
+                           ranges of the index do not change; nnz counts the remaining pairs and
+                           the attention kernels drop the switched-off entries inside each range */
+    int32_t reserved[4];
 } hdt_index_params_t;
 
 typedef struct hdt_index hdt_index_t; /* opaque host object; views into the caller's workspace */

@@ -62,20 +62,35 @@ def _inputs(*xs):
     return [None if x is None else np.ascontiguousarray(x, dt) for x in xs], int(f32)
 
 
+class _Directions:
+    """Sets the oracle's direction bits (1 = child attends parent, 2 = siblings attend each other,
+    4 = parent attends children; the diagonal always stays) for the calls inside the block."""
+
+    def __init__(self, bits):
+        self.bits = 7 if bits is None else int(bits)
+
+    def __enter__(self):
+        lib().hdt_oracle_set_directions(ctypes.c_int(self.bits))
+
+    def __exit__(self, *a):
+        lib().hdt_oracle_set_directions(ctypes.c_int(7))
+
+
 def default_scale(d: int) -> float:
     return 1.0 / float(np.sqrt(d))
 
 
-def mask(level, parent, cu, b: int) -> np.ndarray:
+def mask(level, parent, cu, b: int, directions=None) -> np.ndarray:
     """Dense 0/1 mask (uint8 [n, n]) of sequence b from the parent/sibling/child rule."""
     level, parent, cu = _struct(level, parent, cu)
     n = int(cu[b + 1] - cu[b])
     out = np.zeros((n, n), np.uint8)
-    lib().hdt_oracle_mask(_p(level), _p(parent), _p(cu), ctypes.c_int(b), _p(out))
+    with _Directions(directions):
+        lib().hdt_oracle_mask(_p(level), _p(parent), _p(cu), ctypes.c_int(b), _p(out))
     return out
 
 
-def forward(level, parent, cu, q, k, v, scale=None):
+def forward(level, parent, cu, q, k, v, scale=None, directions=None):
     """O fp64 [T,H,d] and LSE fp64 [H,T] of masked softmax attention."""
     level, parent, cu = _struct(level, parent, cu)
     (q, k, v), f32 = _inputs(q, k, v)
@@ -83,14 +98,15 @@ def forward(level, parent, cu, q, k, v, scale=None):
     scale = default_scale(d) if scale is None else scale
     o = np.zeros((T, H, d), np.float64)
     lse = np.full((H, T), -np.inf, np.float64)
-    rc = lib().hdt_oracle_fwd(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
-                              ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v),
-                              ctypes.c_int(f32), ctypes.c_double(scale), _p(o), _p(lse))
+    with _Directions(directions):
+        rc = lib().hdt_oracle_fwd(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
+                                  ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v),
+                                  ctypes.c_int(f32), ctypes.c_double(scale), _p(o), _p(lse))
     assert rc == 0
     return o, lse
 
 
-def backward(level, parent, cu, q, k, v, do, scale=None):
+def backward(level, parent, cu, q, k, v, do, scale=None, directions=None):
     """dQ, dK, dV fp64 [T,H,d]."""
     level, parent, cu = _struct(level, parent, cu)
     (q, k, v, do), f32 = _inputs(q, k, v, do)
@@ -99,14 +115,15 @@ def backward(level, parent, cu, q, k, v, do, scale=None):
     dq = np.zeros((T, H, d), np.float64)
     dk = np.zeros((T, H, d), np.float64)
     dv = np.zeros((T, H, d), np.float64)
-    rc = lib().hdt_oracle_bwd(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
-                              ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v), _p(do),
-                              ctypes.c_int(f32), ctypes.c_double(scale), _p(dq), _p(dk), _p(dv))
+    with _Directions(directions):
+        rc = lib().hdt_oracle_bwd(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
+                                  ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v), _p(do),
+                                  ctypes.c_int(f32), ctypes.c_double(scale), _p(dq), _p(dk), _p(dv))
     assert rc == 0
     return dq, dk, dv
 
 
-def rows(level, parent, cu, q, k, v, rows, do=None, scale=None):
+def rows(level, parent, cu, q, k, v, rows, do=None, scale=None, directions=None):
     """Sampled rows (global token ids): O [r,H,d], LSE [r,H] and, with do, dQ [r,H,d]."""
     level, parent, cu = _struct(level, parent, cu)
     (q, k, v, do), f32 = _inputs(q, k, v, do)
@@ -116,15 +133,16 @@ def rows(level, parent, cu, q, k, v, rows, do=None, scale=None):
     o = np.zeros((len(rows), H, d), np.float64)
     lse = np.zeros((len(rows), H), np.float64)
     dq = np.zeros((len(rows), H, d), np.float64) if do is not None else None
-    rc = lib().hdt_oracle_rows(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
-                               ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v), _p(do),
-                               ctypes.c_int(f32), ctypes.c_double(scale), _p(rows),
-                               ctypes.c_int(len(rows)), _p(o), _p(lse), _p(dq))
+    with _Directions(directions):
+        rc = lib().hdt_oracle_rows(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
+                                   ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v), _p(do),
+                                   ctypes.c_int(f32), ctypes.c_double(scale), _p(rows),
+                                   ctypes.c_int(len(rows)), _p(o), _p(lse), _p(dq))
     assert rc == 0
     return o, lse, dq
 
 
-def cols(level, parent, cu, q, k, v, do, cols, scale=None):
+def cols(level, parent, cu, q, k, v, do, cols, scale=None, directions=None):
     """Sampled keys (global token ids): dK, dV [c,H,d]."""
     level, parent, cu = _struct(level, parent, cu)
     (q, k, v, do), f32 = _inputs(q, k, v, do)
@@ -133,15 +151,16 @@ def cols(level, parent, cu, q, k, v, do, cols, scale=None):
     cols = np.ascontiguousarray(cols, np.int32)
     dk = np.zeros((len(cols), H, d), np.float64)
     dv = np.zeros((len(cols), H, d), np.float64)
-    rc = lib().hdt_oracle_cols(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
-                               ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v), _p(do),
-                               ctypes.c_int(f32), ctypes.c_double(scale), _p(cols),
-                               ctypes.c_int(len(cols)), _p(dk), _p(dv))
+    with _Directions(directions):
+        rc = lib().hdt_oracle_cols(_p(level), _p(parent), _p(cu), ctypes.c_int(len(cu) - 1),
+                                   ctypes.c_int(H), ctypes.c_int(d), _p(q), _p(k), _p(v), _p(do),
+                                   ctypes.c_int(f32), ctypes.c_double(scale), _p(cols),
+                                   ctypes.c_int(len(cols)), _p(dk), _p(dv))
     assert rc == 0
     return dk, dv
 
 
-def probs(level, parent, cu, q, k, b: int, h: int, scale=None) -> np.ndarray:
+def probs(level, parent, cu, q, k, b: int, h: int, scale=None, directions=None) -> np.ndarray:
     """Dense softmax matrix S fp64 [n, n] of sequence b, head h."""
     level, parent, cu = _struct(level, parent, cu)
     (q, k), f32 = _inputs(q, k)
@@ -149,8 +168,9 @@ def probs(level, parent, cu, q, k, b: int, h: int, scale=None) -> np.ndarray:
     scale = default_scale(d) if scale is None else scale
     n = int(cu[b + 1] - cu[b])
     S = np.zeros((n, n), np.float64)
-    rc = lib().hdt_oracle_probs(_p(level), _p(parent), _p(cu), ctypes.c_int(b), ctypes.c_int(H),
-                                ctypes.c_int(d), _p(q), _p(k), ctypes.c_int(f32),
-                                ctypes.c_double(scale), ctypes.c_int(h), _p(S))
+    with _Directions(directions):
+        rc = lib().hdt_oracle_probs(_p(level), _p(parent), _p(cu), ctypes.c_int(b), ctypes.c_int(H),
+                                    ctypes.c_int(d), _p(q), _p(k), ctypes.c_int(f32),
+                                    ctypes.c_double(scale), ctypes.c_int(h), _p(S))
     assert rc == 0
     return S

@@ -46,13 +46,26 @@ static inline double ld(const void *p, size_t idx, int f32) {
     return f32 ? (double)((const float *)p)[idx] : ((const double *)p)[idx];
 }
 
+/*
+ * Directed variants of the rule (paper, "Mathematical Reasoning Tasks": the ListOps attention
+ * patterns).  Three groups of entries can be switched off: a token attending to its parent
+ * (bit 0; the variant where operands do not attend to their operators clears it), a token
+ * attending to its other siblings (bit 1; the variant where operands do not attend to each
+ * other clears it as well), a token attending to its children (bit 2).  The diagonal always
+ * stays.  7 = the full rule of the section "Hierarchical Attention"; every function below uses
+ * the value set here.
+ */
+static int g_directions = 7;
+void hdt_oracle_set_directions(int bits) { g_directions = bits & 7; }
+
 /* Parent / sibling / child rule on sequence-relative indices i, j. */
 static int mask_rule(const int8_t *lv, const int32_t *pa, int i, int j) {
     if (lv[i] < 0 || lv[j] < 0) return 0;                 /* PAD */
     if (i == j) return 1;                                 /* a token is its own sibling */
-    if (pa[i] == j) return 1;                             /* j is the parent of i */
-    if (pa[j] == i) return 1;                             /* j is a child of i */
-    if (pa[i] >= 0 && pa[i] == pa[j] && lv[i] == lv[j]) return 1; /* siblings */
+    if (pa[i] == j) return (g_directions & 1) != 0;       /* j is the parent of i */
+    if (pa[j] == i) return (g_directions & 4) != 0;       /* j is a child of i */
+    if (pa[i] >= 0 && pa[i] == pa[j] && lv[i] == lv[j])   /* siblings */
+        return (g_directions & 2) != 0;
     return 0;
 }
 

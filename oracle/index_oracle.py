@@ -36,7 +36,8 @@ Per stage s the index holds, for the compacted array A_s of n_s elements:
   queue         block ids sorted by cost (r1-r0)*(b-a) descending, ties by id ascending
   queue_split   the same ids: first the n_fused blocks that are SELF and not EMPTY, then the others,
                 each group in queue order
-Totals: nnz = sum over stages and rows of hi-lo (= number of unmasked pairs of the batch),
+Totals: nnz = sum over stages and rows of the allowed keys in [lo, hi) (all of them under the full
+rule: hi-lo; = number of unmasked pairs of the batch),
 visited = sum over blocks of (r1-r0)*(b-a).
 """
 from __future__ import annotations
@@ -108,7 +109,30 @@ def validate(level, parent, cu):
                     raise BadHierarchy("level must be parent's level + 1")
 
 
-def build(level, parent, cu, block_m: int = 128, max_stages: int = 32, block_m_upper: int = 128) -> Index:
+def pair_allowed(e: int, j: int, lo: int, directions: int) -> bool:
+    """Direction bits on one entry (row e, key j) of a stage whose row range starts at lo.
+    A row whose range starts at or after itself is the head of its family (the keys after it are
+    its children); otherwise lo is the row's parent and the other keys are its siblings.
+    Bits: 1 = a token attends to its parent, 2 = to its other siblings, 4 = to its children; the
+    diagonal always stays (paper, "Mathematical Reasoning Tasks": the ListOps attention patterns)."""
+    if j == e:
+        return True
+    if lo >= e:
+        return bool(directions & 4)
+    return bool(directions & (1 if j == lo else 2))
+
+
+def row_pairs(e: int, lo: int, hi: int, directions: int) -> int:
+    """Number of allowed keys of row e with range [lo, hi)."""
+    if hi <= lo:
+        return 0
+    if lo >= e:
+        return (1 if lo == e else 0) + ((hi - e - 1) if directions & 4 else 0)
+    return 1 + (1 if directions & 1 else 0) + ((hi - lo - 2) if directions & 2 else 0)
+
+
+def build(level, parent, cu, block_m: int = 128, max_stages: int = 32, block_m_upper: int = 128,
+          directions: int = 7) -> Index:
     level = np.asarray(level, np.int8)
     parent = np.asarray(parent, np.int32)
     cu = np.asarray(cu, np.int32)
@@ -170,7 +194,7 @@ def build(level, parent, cu, block_m: int = 128, max_stages: int = 32, block_m_u
                     raise BadHierarchy("children of a node must follow it in document order")
                 rng[e] = (p, p + 1 + c)
                 uid[e] = p
-        nnz += int((rng[:, 1] - rng[:, 0]).sum())
+        nnz += sum(row_pairs(e, int(rng[e, 0]), int(rng[e, 1]), directions) for e in range(n))
 
         # removal for the next stage
         keep = np.zeros(n, bool)
@@ -245,12 +269,13 @@ def build(level, parent, cu, block_m: int = 128, max_stages: int = 32, block_m_u
     return Index(stages, nnz, visited)
 
 
-def pairs_of(index: Index, T: int) -> np.ndarray:
+def pairs_of(index: Index, T: int, directions: int = 7) -> np.ndarray:
     """Count matrix [T,T] of how often each (query token, key token) pair is covered."""
     C = np.zeros((T, T), np.int32)
     for st in index.stages:
         for e in range(st.n):
             lo, hi = st.rng[e]
             for j in range(lo, hi):
-                C[st.tok[e], st.tok[j]] += 1
+                if pair_allowed(e, j, int(lo), directions):
+                    C[st.tok[e], st.tok[j]] += 1
     return C

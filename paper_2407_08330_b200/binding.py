@@ -13,7 +13,7 @@ _HEADER = os.path.join(_HERE, "..", "include", "hdt.h")
 _lib = None
 
 HDT_F32, HDT_BF16 = 0, 1
-HDT_MAX_STAGES = 16
+HDT_MAX_STAGES = 24
 _DTYPES = {torch.float32: HDT_F32, torch.bfloat16: HDT_BF16}
 
 
@@ -25,7 +25,7 @@ class HdtError(RuntimeError):
 
 class _Params(C.Structure):
     _fields_ = [("block_m", C.c_int32), ("max_stages", C.c_int32), ("block_m_upper", C.c_int32),
-                ("reserved", C.c_int32 * 5)]
+                ("mask_off", C.c_int32), ("reserved", C.c_int32 * 4)]
 
 
 class _StageView(C.Structure):
@@ -94,9 +94,10 @@ def _stream():
     return C.c_void_p(torch.cuda.current_stream().cuda_stream)
 
 
-def _params(block_m, max_stages, block_m_upper=0):
+def _params(block_m, max_stages, block_m_upper=0, directions=7):
     p = _Params()
     p.block_m, p.max_stages, p.block_m_upper = int(block_m), int(max_stages), int(block_m_upper)
+    p.mask_off = (~int(directions)) & 7
     return p
 
 
@@ -148,13 +149,14 @@ class HdtIndex:
 
 
 def hdt_build_index(level, parent, cu_seqlens, block_m=0, max_stages=0, workspace=None,
-                    block_m_upper=0) -> HdtIndex:
-    """level int8[T], parent int32[T], cu_seqlens int32[B+1]: CUDA tensors."""
+                    block_m_upper=0, directions=7) -> HdtIndex:
+    """level int8[T], parent int32[T], cu_seqlens int32[B+1]: CUDA tensors.  directions: bits
+    1 | 2 | 4 keep the child->parent, sibling<->sibling, parent->child entries (7 = full rule)."""
     assert level.is_cuda and parent.is_cuda and cu_seqlens.is_cuda
     assert level.dtype == torch.int8 and parent.dtype == torch.int32 and cu_seqlens.dtype == torch.int32
     level, parent, cu_seqlens = level.contiguous(), parent.contiguous(), cu_seqlens.contiguous()
     T, B = level.numel(), cu_seqlens.numel() - 1
-    p = _params(block_m, max_stages, block_m_upper)
+    p = _params(block_m, max_stages, block_m_upper, directions)
     need = int(lib().hdt_index_workspace_bytes(B, T, C.cast(C.byref(p), C.c_void_p)))
     if need == 0:
         raise HdtError(-1, "invalid index parameters")

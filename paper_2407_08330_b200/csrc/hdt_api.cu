@@ -231,6 +231,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.o = o; a.lse = lse;
         a.status = status;
         a.no_persistent = g_no_persistent;
+        a.dirs = ix->directions;
         return a;
     };
     // The stages above 0 do not depend on stage 0 until their results are merged: compute them on
@@ -247,7 +248,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
         // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
         // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
-        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3;
+        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3 && ix->directions == 7;
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 1;
         c.tok1 = ix->st[1].tok;
@@ -340,6 +341,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.dq = dq; a.dk = dk; a.dv = dv;
         a.status = status;
         a.no_persistent = g_no_persistent;
+        a.dirs = ix->directions;
         return a;
     };
     const bool overlap = ix->n_stages > 1 && !g_no_overlap;
@@ -354,7 +356,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
         // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
         // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
-        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3;
+        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3 && ix->directions == 7;
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 3;
         c.tok1 = ix->st[1].tok;
@@ -472,6 +474,7 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
         a.o = o; a.lse = lse;
         a.status = status;
         a.no_persistent = g_no_persistent;
+        a.dirs = ix->directions;
         if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
         else rc = launch_fwd_simt(a, head_dim, dtype, st);
         if (rc) return rc;

@@ -131,7 +131,7 @@ __global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
 #pragma unroll
                         for (int t = 0; t < 4; ++t) acc = dot4(q[t], kr[g + G * t], acc);
                         acc = group_sum<G>(acc);
-                        if (j >= jlo && j < jhi) s[jj] = acc * a.scale_log2;
+                        if (j >= jlo && j < jhi && (a.dirs == 7 || dir_ok(row, j, lo, a.dirs))) s[jj] = acc * a.scale_log2;
                     }
                 }
                 float mx = s[0];
@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
                 }
                 s = group_sum<G>(s);
                 dp = group_sum<G>(dp);
-                if (j >= jlo && j < jhi) {
+                if (j >= jlo && j < jhi && (a.dirs == 7 || dir_ok(row, j, lo, a.dirs))) {
                     const float p = exp2f(s * a.scale_log2 - lse2);
                     const float ds = p * (dp - dl);
 #pragma unroll
@@ -333,7 +333,7 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
                 }
                 s = group_sum<G>(s);
                 dp = group_sum<G>(dp);
-                if (i >= jlo && i < jhi) {
+                if (i >= jlo && i < jhi && (a.dirs == 7 || dir_ok_key(row, i, lo, a.dirs))) {
                     const float p = exp2f(s * a.scale_log2 - sL[i - c0]);
                     const float ds = p * (dp - sDl[i - c0]);
 #pragma unroll

@@ -66,7 +66,9 @@ __device__ __forceinline__ void gather_tiles(uint8_t *const (&dst)[NTEN], const 
 // GATHER = true (with SINGLE = false): a stage above 0 computed beside stage 0.  Rows are gathered
 // through the stage's tok map by the threads instead of TMA, and the kernel leaves only the
 // stage's own partial result per element (fp32 O, LSE, indexed by element) for the chain merge.
-template <int D, bool SINGLE, bool GATHER = false>
+// DIRS = true: the index carries direction bits other than 7; entries of the row range that the
+// bits switch off are masked as well (dir_ok).
+template <int D, bool SINGLE, bool GATHER = false, bool DIRS = false>
 __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensorMap tm_q,
                                                 const __grid_constant__ CUtensorMap tm_k,
                                                 const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
@@ -162,6 +164,11 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             const int jl = max(lo - c0, 0), jh = min(hi - c0, nvalid);
             const bool has = inb && jh > jl;
             const int nsl = (Nc + 31) >> 5;
+            // direction bits: column of the row itself, of its parent (none for a head row), and
+            // whether the parent entry / every other entry of the range is kept
+            const int c_self = row - c0, c_head = (lo < row) ? lo - c0 : -0x40000000;
+            const bool keep_head = (a.dirs & 1) != 0, keep_rest = (a.dirs & ((lo >= row) ? 4 : 2)) != 0;
+            auto kept = [&](int c) { return !DIRS || c == c_self || (c == c_head ? keep_head : keep_rest); };
             float mx = NEG;
             for (int k = 0; k < nsl; ++k) {
                 const int s0 = 32 * k;
@@ -173,7 +180,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                     if (mine) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (s0 + j >= jl && s0 + j < jh) mx = fmaxf(mx, __uint_as_float(r[j]));
+                            if (s0 + j >= jl && s0 + j < jh && kept(s0 + j)) mx = fmaxf(mx, __uint_as_float(r[j]));
                     }
                 }
             }
@@ -194,8 +201,9 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
                             float p0 = 0.f, p1 = 0.f;
-                            if (s0 + j >= jl && s0 + j < jh) p0 = exp2f(fmaf(__uint_as_float(r[j]), a.scale_log2, -m_new));
-                            if (s0 + j + 1 >= jl && s0 + j + 1 < jh)
+                            if (s0 + j >= jl && s0 + j < jh && kept(s0 + j))
+                                p0 = exp2f(fmaf(__uint_as_float(r[j]), a.scale_log2, -m_new));
+                            if (s0 + j + 1 >= jl && s0 + j + 1 < jh && kept(s0 + j + 1))
                                 p1 = exp2f(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m_new));
                             // the row sum uses the bf16-rounded probabilities the MMA will see
                             const uint32_t u = pack_bf16(p0, p1);
@@ -837,6 +845,17 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     FwdStageArgs b = a;
     b.rest_only = 0;
     int n_general = a.nb;
+    if (a.dirs != 7) {   // direction bits: every block through the general kernel that applies them
+        static bool attr_d = false;
+        if (!attr_d) {
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attr_d = true;
+        }
+        k_fwd_tc<D, false, false, true><<<dim3(a.nb, a.H), 128, smem, st>>>(tq, tk, tv, b);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+        return HDT_OK;
+    }
     if (a.n_fused > 0 && a.no_persistent != 1) {
         if (D == 64 && a.no_persistent == 2) {   // option: the persistent single-CTA-per-SM kernel
             constexpr int smem_p = 8 * SUB + 4 * 128 * 4 + 1024 + 64;

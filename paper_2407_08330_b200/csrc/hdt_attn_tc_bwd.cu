@@ -63,7 +63,9 @@ __device__ __forceinline__ void gather_tiles(uint8_t *const (&dst)[NTEN], const 
 // GATHER = true: a stage above 0 computed beside stage 0.  Rows (and their LSE / delta) are fetched
 // through the stage's tok map by the threads instead of TMA, and the kernel leaves only the stage's
 // own gradients per element (fp32, indexed by element) for the chain merge.
-template <int D, bool GATHER = false>
+// DIRS = true: the index carries direction bits other than 7; entries of the row range that the
+// bits switch off are masked as well (dir_ok).
+template <int D, bool GATHER = false, bool DIRS = false>
 __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensorMap tm_q,
                                                 const __grid_constant__ CUtensorMap tm_k,
                                                 const __grid_constant__ CUtensorMap tm_v,
@@ -152,6 +154,11 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         }
         const int jl = max(lo - k_row0, 0), jh = min(hi - k_row0, nk);
         const bool has = inq && jh > jl;
+        // direction bits: column of the row itself, of its parent (none for a head row), and
+        // whether the parent entry / every other entry of the range is kept
+        const int c_self = e - k_row0, c_head = (lo < e) ? lo - k_row0 : -0x40000000;
+        const bool keep_head = (a.dirs & 1) != 0, keep_rest = (a.dirs & ((lo >= e) ? 4 : 2)) != 0;
+        auto kept = [&](int c) { return !DIRS || c == c_self || (c == c_head ? keep_head : keep_rest); };
         ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
         ph_mma ^= 1;
         tc_fence_after();
@@ -172,11 +179,11 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
                         float p0 = 0.f, p1 = 0.f, d0 = 0.f, d1 = 0.f;
-                        if (s0 + j >= jl && s0 + j < jh) {
+                        if (s0 + j >= jl && s0 + j < jh && kept(s0 + j)) {
                             p0 = exp2f(fmaf(__uint_as_float(rs[j]), a.scale_log2, -lse2));
                             d0 = p0 * (__uint_as_float(rd[j]) - dl);
                         }
-                        if (s0 + j + 1 >= jl && s0 + j + 1 < jh) {
+                        if (s0 + j + 1 >= jl && s0 + j + 1 < jh && kept(s0 + j + 1)) {
                             p1 = exp2f(fmaf(__uint_as_float(rs[j + 1]), a.scale_log2, -lse2));
                             d1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
                         }
@@ -762,6 +769,17 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     BwdStageArgs b = a;
     b.rest_only = 0;
     int n_general = a.nb;
+    if (a.dirs != 7) {   // direction bits: every block through the general kernel that applies them
+        static bool attr_d = false;
+        if (!attr_d) {
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+            attr_d = true;
+        }
+        k_bwd_tc<D, false, true><<<dim3(a.nb, a.H), 256, smem, st>>>(tq, tk, tv, tdo, b);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+        return HDT_OK;
+    }
     if (D == 64 && a.nb > 0 && !a.no_persistent) {
         // the persistent kernel takes everything: first the blocks of split families (longest first),
         // then the self-contained blocks

@@ -134,10 +134,20 @@ __global__ void k_nlc(const DevHeader *hdr, int s, const int *__restrict__ par,
 }
 
 // One CTA per CHUNK elements (needed for the per-chunk keep counts).
+// Keys of row e with range [lo, hi) that the direction bits keep.  A row whose range starts at or
+// after itself is the head of its family (the keys after it are its children); otherwise lo is
+// the row's parent and the remaining keys are its siblings.  dirs: 1 = child -> parent,
+// 2 = sibling <-> sibling, 4 = parent -> child; the diagonal always stays.
+__device__ __forceinline__ int row_pairs(int e, int lo, int hi, int dirs) {
+    if (hi <= lo) return 0;
+    if (lo >= e) return (lo == e ? 1 : 0) + ((dirs & 4) ? hi - e - 1 : 0);
+    return 1 + ((dirs & 1) ? 1 : 0) + ((dirs & 2) ? hi - lo - 2 : 0);
+}
+
 __global__ void __launch_bounds__(CHUNK)
 k_ranges(DevHeader *hdr, int s, const int8_t *__restrict__ level /* stage 0 only */,
          const int *__restrict__ par, const int *__restrict__ cnt, const int *__restrict__ nlc,
-         int *rng, uint8_t *keep, uint8_t *fpos, int *blocksum) {
+         int *rng, uint8_t *keep, uint8_t *fpos, int *blocksum, int dirs) {
     const int n = hdr->st[s].n;
     const int e = blockIdx.x * CHUNK + threadIdx.x;
     int kp = 0;
@@ -165,7 +175,7 @@ k_ranges(DevHeader *hdr, int s, const int8_t *__restrict__ level /* stage 0 only
         rng[2 * e + 1] = hi;
         keep[e] = (uint8_t)kp;
         fpos[e] = (uint8_t)fp;
-        deg = hi - lo;
+        deg = row_pairs(e, lo, hi, dirs);
         if (kp && p >= 0) hdr->st[s].has_next = 1;  // same value from every writer
     }
     // CTA reductions: keep count and nnz
@@ -455,7 +465,7 @@ k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost, const int *__
 // ---------------------------------------------------------------------------------------------
 struct UpperArgs {
     StagePtrs st[HDT_MAX_STAGES];
-    int max_stages, B, bm;
+    int max_stages, B, bm, dirs;
     int *cnt, *nlc, *pre, *bstart, *seqcount;
     uint8_t *keep, *fpos;
     long long *cost;
@@ -503,7 +513,7 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
             P.rng[2 * e + 1] = hi;
             u.keep[e] = (uint8_t)kp;
             u.fpos[e] = (uint8_t)fp;
-            deg += hi - lo;
+            deg += row_pairs(e, lo, hi, u.dirs);
             if (kp && p >= 0) s_flag = 1;
         }
         for (int o = 16; o; o >>= 1) deg += __shfl_xor_sync(0xffffffffu, deg, o);
@@ -657,6 +667,8 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
 
 using namespace hdt;
 
+static int norm_dirs(const hdt_index_params_t *p) { return p ? (~p->mask_off) & 7 : 7; }
+
 static void norm_params(const hdt_index_params_t *p, int &bm, int &ms, int &bmu) {
     bm = (p && p->block_m) ? p->block_m : 128;
     ms = (p && p->max_stages) ? p->max_stages : 4;
@@ -678,12 +690,15 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     if (out) *out = nullptr;
     int bm, ms, bmu;
     norm_params(params, bm, ms, bmu);
+    const int dirs = norm_dirs(params);
     if (!out || !cu_seqlens || !workspace || batch < 0 || total_tokens < 0 ||
         (total_tokens > 0 && (!level || !parent)))
         return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: null pointer or negative size");
     if (bm < 1 || bm > 128 || bmu < 1 || bmu > 128 || ms < 1 || ms > HDT_MAX_STAGES)
         return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: block_m, block_m_upper must be 1..128, max_stages 1..%d",
                          HDT_MAX_STAGES);
+    if (params && (params->mask_off & ~7))
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: mask_off has bits outside 0..7");
     if (((uintptr_t)workspace & 255) != 0)
         return set_error(HDT_ERR_INVALID_ARG, "hdt_build_index: workspace must be 256-byte aligned");
     const int B = batch, T = total_tokens;
@@ -702,6 +717,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
 
     hdt_index *ix = new hdt_index();
     ix->batch = B; ix->total_tokens = T; ix->block_m = bm; ix->block_m_upper = bmu; ix->n_stages = 0;
+    ix->directions = dirs;
     ix->workspace = workspace; ix->workspace_bytes = workspace_bytes;
     for (int s = 0; s < ms; ++s) {
         char *base = ws + L.stage0 + L.stage_stride * (size_t)s;
@@ -724,7 +740,10 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     const int g_stride = max(1, min((T + 255) / 256, 148 * 8));
     static const int kSmemCap = 200 * 1024;
     HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
-    const bool fused_upper = (B <= UMAXB);
+    // One CTA builds all stages above 0 when they are small (documents: a few percent of the
+    // tokens, up to 3-4 stages).  A caller that allows many stages expects deep trees, whose upper
+    // stages hold most of the elements: those go through the per-stage kernels.
+    const bool fused_upper = (B <= UMAXB) && ms <= 8;
     // The upper stages only need stage 0's compaction; with their own scratch they are built on the
     // side stream while stage 0's blocks and queues are built on the caller's stream.
     Side *sd = nullptr;
@@ -744,7 +763,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         auto launch_upper = [&](cudaStream_t s_) {
             UpperArgs u;
             for (int i = 0; i < HDT_MAX_STAGES; ++i) u.st[i] = ix->st[i < ms ? i : ms - 1];
-            u.max_stages = ms; u.B = B; u.bm = bmu;
+            u.max_stages = ms; u.B = B; u.bm = bmu; u.dirs = dirs;
             u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.keep = keep;
             u.bstart = (int *)(ws + L.bstart2); u.seqcount = (int *)(ws + L.seqcount2);
             u.fpos = (uint8_t *)(ws + L.fpos2); u.cost = (long long *)(ws + L.cost2);
@@ -764,7 +783,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             if (s >= 1) { k_count<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt); ++n_launched; }
             k_nlc<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt, nlc);
             k_ranges<<<g_chunk, CHUNK, 0, st>>>(hdr, s, s == 0 ? level : nullptr, P.par, cnt, nlc, P.rng, keep,
-                                                fpos, blocksum);
+                                                fpos, blocksum, dirs);
             // tok2 of the last possible stage is never read: point it at scratch (pre is rewritten first)
             k_scan<<<g_chunk, CHUNK, 0, st>>>(hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
                                               last ? cnt : N.tok);
@@ -798,10 +817,10 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         // The build is a dozen tiny kernels: launching them one by one is slower than running them.
         // They are captured once into a CUDA graph, which is replayed while the same buffers, sizes
         // and parameters come back (one cached graph per host thread).
-        struct GraphKey { const void *a, *b, *c, *w; int B, T, bm, ms, bmu, ov; };
+        struct GraphKey { const void *a, *b, *c, *w; int B, T, bm, ms, bmu, ov, dirs; };
         struct GraphCache { GraphKey key; cudaGraphExec_t exec; int launches; bool valid; };
         static thread_local GraphCache cache{};
-        const GraphKey key{level, parent, cu_seqlens, workspace, B, T, bm, ms, bmu, sd ? 1 : 0};
+        const GraphKey key{level, parent, cu_seqlens, workspace, B, T, bm, ms, bmu, sd ? 1 : 0, dirs};
         bool done = false;
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         // (the legacy and per-thread default streams cannot be captured)

@@ -33,6 +33,7 @@ struct StagePtrs {
 
 struct hdt_index {
     int batch, total_tokens, block_m, block_m_upper, n_stages;
+    int directions;   // bits 1 | 2 | 4: child->parent, sibling<->sibling, parent->child entries kept (7 = full rule)
     long long nnz, visited;
     hdt::StageDesc desc[HDT_MAX_STAGES + 1];
     hdt::StagePtrs st[HDT_MAX_STAGES];
@@ -71,6 +72,23 @@ int get_side(Side **out);
 extern int g_no_overlap;   // option "no_overlap"
 extern int g_no_graph;     // option "no_graph"
 
+// Direction bits inside a row range (paper, "Mathematical Reasoning Tasks": the ListOps attention
+// patterns).  Row e of a stage has the key range [lo, hi).  If the range starts at or after e, e is
+// the head of the family and the keys after it are its children; otherwise lo is e's parent and
+// the other keys are its siblings.  dirs: 1 = child -> parent, 2 = sibling <-> sibling,
+// 4 = parent -> child entries are kept; the diagonal always is.
+__host__ __device__ __forceinline__ bool dir_ok(int e, int j, int lo, int dirs) {
+    if (j == e) return true;
+    if (lo >= e) return (dirs & 4) != 0;
+    return (dirs & (j == lo ? 1 : 2)) != 0;
+}
+// The same entry seen from the key: key element `key` has the range [lo, hi), query i lies in it.
+__host__ __device__ __forceinline__ bool dir_ok_key(int key, int i, int lo, int dirs) {
+    if (i == key) return true;
+    if (lo >= key) return (dirs & 1) != 0;            // i is a child of the head `key`
+    return (dirs & (i == lo ? 4 : 2)) != 0;           // i is key's parent, or a sibling
+}
+
 // SIMT attention launchers (hdt_attn_simt.cu).  One launch handles one stage.
 struct FwdStageArgs {
     // stage view
@@ -99,6 +117,7 @@ struct FwdStageArgs {
     int rest_only;      // general kernel: only blocks after the first n_fused
     int no_persistent;  // option: do not use the persistent kernels
     int block_rows;     // max rows of a block in this stage
+    int dirs;           // direction bits kept (7 = full rule), see dir_ok
 };
 
 struct BwdStageArgs {
@@ -119,6 +138,7 @@ struct BwdStageArgs {
     int rest_only;                                // general kernel: only blocks after the first n_fused
     int no_persistent;                            // option: do not use the persistent kernels
     int block_rows;                               // max rows of a block in this stage
+    int dirs;                                     // direction bits kept (7 = full rule), see dir_ok
 };
 
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
