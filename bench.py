@@ -403,6 +403,37 @@ def main():
         idx.close()
         del x, ws_h
 
+    # the step after the path, timed alone: 256 decoder rows per document cross-attending to a level
+    # subset of this batch's encoder rows (forward + backward), for the three subsets of the paper
+    cross = None
+    if rank == 0 and not args.no_hpe and cfg.backward:
+        nq = 256
+        cuq = torch.arange(0, (b.batch + 1) * nq, nq, dtype=torch.int32, device=dev)
+        Tq = b.batch * nq
+        gq = torch.Generator(device="cpu").manual_seed(cfg.tensor_seed + 77)
+        xq, xdo = (torch.randn((Tq, H, d), generator=gq).to(tdt).to(dev) for _ in range(2))
+        xo = torch.empty_like(xq); xlse = torch.empty((H, Tq), dtype=torch.float32, device=dev)
+        xdq = torch.empty_like(xq)
+        ws_x = torch.empty(P.hdt_cross_workspace_bytes(b.batch, T, Tq, H, 1), dtype=torch.uint8, device=dev)
+        cross = {"decoder_rows": Tq, "subsets": {}}
+        for name, mask in (("[SEC]", 2), ("[SEC]+[SENT]", 6), ("[SEC]+[SENT]+tokens", 14)):
+            n_keys = int(sum(int((b.level == l).sum()) for l in range(4) if (mask >> l) & 1))
+
+            def step_x():
+                P.hdt_cross_attn_fwd(level, cu, cuq, mask, xq, k, v, out=xo, lse=xlse, workspace=ws_x)
+                P.hdt_cross_attn_bwd(level, cu, cuq, mask, xq, k, v, xo, xlse, xdo, dq=xdq, dk=dk, dv=dv, workspace=ws_x)
+
+            n_x = 3 if mask == 14 else args.steps
+            for _ in range(2):
+                step_x()
+            x_ms = float(np.mean(timed(step_x, n_x)))
+            pairs = sum(nq * int(((b.level[b.cu_seqlens[s]:b.cu_seqlens[s + 1]] >= 0) &
+                                  (((mask >> np.maximum(b.level[b.cu_seqlens[s]:b.cu_seqlens[s + 1]], 0)) & 1) == 1)).sum())
+                        for s in range(b.batch))
+            cross["subsets"][name] = {"chosen_keys": n_keys, "ms_fwd_bwd": x_ms,
+                                      "tflops": 14 * d * pairs * H / (x_ms * 1e-3) / 1e12}
+        del xq, xdo, xo, xlse, xdq, ws_x
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -449,6 +480,8 @@ def main():
     }
     if hpe:
         line["next_rows"] = {"hpe": hpe}
+        if cross:
+            line["next_rows"]["cross_attention"] = cross
     if not args.no_cpu_baseline and world >= 1:
         line["cpu_baseline"] = cpu_baseline(c, cfg, b, args.directions)
     print(json.dumps(line))

@@ -244,6 +244,36 @@ int hdt_hpe(const hdt_index_t *index, const int8_t *level, const int32_t *parent
             size_t workspace_bytes, void *stream);
 
 /*
+ * Decoder cross-attention to a level subset of the encoder tokens (paper, paragraph "Results on
+ * FacetSum (Encoder-Decoder Models)": the decoder attends only to [SEC] anchors, to [SEC] and [SENT]
+ * anchors, or to every token of the encoder output; the decoder's cross-attention sub-layer of the
+ * paragraph "Hierarchical Encoder and Decoder Stacks").  For document b the decoder rows
+ * cu_seqlens_q[b] .. cu_seqlens_q[b+1] attend to the encoder tokens of the same document whose level
+ * l has bit l set in level_mask (PAD, level -1, is never chosen):
+ *     O = softmax(Q Ks^T * scale) Vs,   LSE_i = log sum_j exp(A_ij).
+ * A decoder row of a document without a chosen token gets O = 0 and LSE = -inf.
+ *   level              device int8 [total_tokens]; cu_seqlens_k / cu_seqlens_q device int32 [batch+1]
+ *   q, o, d_o, dq      device [total_q, heads, head_dim] of `dtype`, 16-byte aligned
+ *   k, v, dk, dv       device [total_tokens, heads, head_dim]; dk, dv are written for every encoder
+ *                      row (zero outside the subset)
+ *   lse                device float [heads, total_q]
+ *   workspace          device, >= hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, bwd),
+ *                      256-byte aligned; holds the list of chosen tokens, rebuilt by every call
+ * head_dim 64 or 128; softmax_scale <= 0 means 1/sqrt(head_dim).  Asynchronous on `stream`, no
+ * host wait.  The chosen rows are read in place through the list (no gathered copy of K, V).
+ */
+size_t hdt_cross_workspace_bytes(int32_t batch, int32_t total_tokens, int32_t total_q, int32_t heads, int32_t bwd);
+int hdt_cross_attn_fwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q, int32_t batch,
+                       int32_t total_tokens, int32_t total_q, int32_t level_mask, const void *q, const void *k,
+                       const void *v, void *o, float *lse, int32_t heads, int32_t head_dim, int32_t dtype,
+                       float softmax_scale, void *workspace, size_t workspace_bytes, void *stream);
+int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q, int32_t batch,
+                       int32_t total_tokens, int32_t total_q, int32_t level_mask, const void *q, const void *k,
+                       const void *v, const void *o, const float *lse, const void *d_o, void *dq, void *dk, void *dv,
+                       int32_t heads, int32_t head_dim, int32_t dtype, float softmax_scale, void *workspace,
+                       size_t workspace_bytes, void *stream);
+
+/*
  * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
  * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
  * general tensor-core kernels, = 2 the persistent forward kernel, = 3 the forward kernel with one CTA

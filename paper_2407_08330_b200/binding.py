@@ -257,6 +257,65 @@ def hdt_hpe(index: HdtIndex, level, parent, cu_seqlens, d_model, n_levels=3, dty
     return x
 
 
+def hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, bwd) -> int:
+    L = lib()
+    L.hdt_cross_workspace_bytes.restype = C.c_size_t
+    L.hdt_cross_workspace_bytes.argtypes = [C.c_int32] * 5
+    return int(L.hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, int(bwd)))
+
+
+def _cross_common(level, cu_seqlens_k, cu_seqlens_q, q, k):
+    assert level.dtype == torch.int8 and cu_seqlens_k.dtype == torch.int32 and cu_seqlens_q.dtype == torch.int32
+    Tq, H, d = q.shape
+    T, B = k.shape[0], cu_seqlens_k.numel() - 1
+    assert cu_seqlens_q.numel() == B + 1 and level.numel() == T
+    return B, T, Tq, H, d
+
+
+def hdt_cross_attn_fwd(level, cu_seqlens_k, cu_seqlens_q, level_mask, q, k, v, softmax_scale=0.0, out=None, lse=None,
+                       workspace=None):
+    """Decoder rows q [Tq,H,d] attend to the encoder rows of k, v [T,H,d] whose level bit is set in
+    level_mask.  Returns (O [Tq,H,d], LSE [H,Tq])."""
+    L = lib()
+    L.hdt_cross_attn_fwd.restype = C.c_int
+    L.hdt_cross_attn_fwd.argtypes = [C.c_void_p] * 3 + [C.c_int32] * 4 + [C.c_void_p] * 5 + [C.c_int32] * 3 + \
+                                    [C.c_float, C.c_void_p, C.c_size_t, C.c_void_p]
+    B, T, Tq, H, d = _cross_common(level, cu_seqlens_k, cu_seqlens_q, q, k)
+    assert q.is_contiguous() and k.is_contiguous() and v.is_contiguous()
+    if out is None:
+        out = torch.empty_like(q)
+    if lse is None:
+        lse = torch.empty((H, Tq), dtype=torch.float32, device=q.device)
+    need = hdt_cross_workspace_bytes(B, T, Tq, H, 0)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    _check(L.hdt_cross_attn_fwd(_ptr(level), _ptr(cu_seqlens_k), _ptr(cu_seqlens_q), B, T, Tq, int(level_mask), _ptr(q),
+                                _ptr(k), _ptr(v), _ptr(out), _ptr(lse), H, d, _DTYPES[q.dtype], float(softmax_scale),
+                                _ptr(workspace), workspace.numel(), _stream()))
+    return out, lse
+
+
+def hdt_cross_attn_bwd(level, cu_seqlens_k, cu_seqlens_q, level_mask, q, k, v, o, lse, do, softmax_scale=0.0, dq=None,
+                       dk=None, dv=None, workspace=None):
+    """Gradients (dQ [Tq,H,d], dK, dV [T,H,d]) of hdt_cross_attn_fwd."""
+    L = lib()
+    L.hdt_cross_attn_bwd.restype = C.c_int
+    L.hdt_cross_attn_bwd.argtypes = [C.c_void_p] * 3 + [C.c_int32] * 4 + [C.c_void_p] * 9 + [C.c_int32] * 3 + \
+                                    [C.c_float, C.c_void_p, C.c_size_t, C.c_void_p]
+    B, T, Tq, H, d = _cross_common(level, cu_seqlens_k, cu_seqlens_q, q, k)
+    assert all(x.is_contiguous() for x in (q, k, v, o, do))
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    need = hdt_cross_workspace_bytes(B, T, Tq, H, 1)
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
+    _check(L.hdt_cross_attn_bwd(_ptr(level), _ptr(cu_seqlens_k), _ptr(cu_seqlens_q), B, T, Tq, int(level_mask), _ptr(q),
+                                _ptr(k), _ptr(v), _ptr(o), _ptr(lse), _ptr(do), _ptr(dq), _ptr(dk), _ptr(dv), H, d,
+                                _DTYPES[q.dtype], float(softmax_scale), _ptr(workspace), workspace.numel(), _stream()))
+    return dq, dk, dv
+
+
 def hdt_set_option(name: str, value: int) -> None:
     lib().hdt_set_option.restype = C.c_int
     _check(lib().hdt_set_option(C.c_char_p(name.encode()), C.c_int32(int(value))))

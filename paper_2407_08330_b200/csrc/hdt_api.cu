@@ -232,6 +232,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.status = status;
         a.no_persistent = g_no_persistent;
         a.dirs = ix->directions;
+        a.tok_rows = a.tok;
         return a;
     };
     // The stages above 0 do not depend on stage 0 until their results are merged: compute them on
@@ -342,6 +343,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.status = status;
         a.no_persistent = g_no_persistent;
         a.dirs = ix->directions;
+        a.tok_rows = a.tok;
         return a;
     };
     const bool overlap = ix->n_stages > 1 && !g_no_overlap;
@@ -475,6 +477,7 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
         a.status = status;
         a.no_persistent = g_no_persistent;
         a.dirs = ix->directions;
+        a.tok_rows = a.tok;
         if (s == 0 && dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
         else rc = launch_fwd_simt(a, head_dim, dtype, st);
         if (rc) return rc;

@@ -105,7 +105,7 @@ __global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
         if (inb) {
             lo = a.rng[2 * row];
             hi = a.rng[2 * row + 1];
-            trow = a.tok ? a.tok[row] : row;
+            trow = a.tok_rows ? a.tok_rows[row] : row;
 #pragma unroll
             for (int t = 0; t < 4; ++t) q[t] = load4<BF16>(a.q, ((size_t)trow * H + h) * D + 4 * (g + G * t));
         }
@@ -229,11 +229,12 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
         if (inb) {
             lo = a.rng[2 * row];
             hi = a.rng[2 * row + 1];
-            trow = a.tok ? a.tok[row] : row;
+            trow = a.tok_rows ? a.tok_rows[row] : row;
         }
         const bool live = hi > lo;
         // ---------------- phase A: this element as a query row ----------------
         float4 x[4], y[4], acc[4];  // q, dO, dq
+        if (a.phases != 2) {   // same decision in the whole grid
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
             x[t] = y[t] = acc[t] = make_float4(0, 0, 0, 0);
@@ -293,6 +294,8 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
                 store4<BF16>(a.dq, ((size_t)trow * H + h) * D + 4 * (g + G * t), acc[t]);
             }
         }
+        }
+        if (a.phases == 1) continue;
         // ---------------- phase B: this element as a key ----------------
         float4 acc2[4];  // x = k, y = v, acc = dk, acc2 = dv
 #pragma unroll

@@ -1,0 +1,257 @@
+// Decoder cross-attention to a level subset of the encoder tokens (paper, paragraph "Results on
+// FacetSum (Encoder-Decoder Models)": the decoder attends only to [SEC] anchors, to [SEC] and
+// [SENT] anchors, or to all tokens of the encoder output; decoder of the paragraph "Hierarchical
+// Encoder and Decoder Stacks").  Within the chosen subset it is plain softmax attention between
+// the decoder rows of a document and the chosen encoder rows of the same document.
+//
+// The chosen rows are never copied: an ordered list `sel` of their token indices is built per call
+// (count, scan, fill: three small kernels, no host wait) and the fp32 SIMT attention kernels of the
+// hierarchical path read K and V through it.  Those kernels take any (row blocks, per-row key
+// range, key map) description, so the forward is one launch over blocks of decoder rows whose key
+// range is the document's slice of `sel`, and the backward two launches: decoder-row blocks for
+// dQ, blocks of chosen keys (walking the document's decoder rows) for dK and dV, which are
+// scattered to the encoder rows; rows outside the subset are zeroed first.
+// Block slots are assigned without a scan: document b owns the slots from start / 32 + b on,
+// unused slots stay empty (r0 == r1).
+#include <cuda_bf16.h>
+
+#include "hdt_internal.cuh"
+
+namespace hdt {
+
+constexpr int XR = 32;      // rows per block (the 128-thread SIMT kernels take 32 rows per pass)
+
+struct CrossLayout {
+    size_t cnt, cu_sel, sel, rngq, rngk, blocks_q, blocks_k, queue, delta, total;
+    int nbq, nbk;
+    size_t zero_bytes;      // cnt .. queue is cleared at the start of every call
+};
+
+static size_t al256c(size_t v) { return (v + 255) & ~size_t(255); }
+
+static CrossLayout cross_layout(int B, int T, int Tq, int H, int bwd) {
+    CrossLayout L{};
+    L.nbq = Tq / XR + B + 1;
+    L.nbk = T / XR + B + 1;
+    size_t o = 0;
+    L.cnt = o; o += al256c(sizeof(int) * (size_t)(B + 1));
+    L.cu_sel = o; o += al256c(sizeof(int) * (size_t)(B + 2));
+    L.blocks_q = o; o += al256c(sizeof(int) * 5 * (size_t)L.nbq);
+    L.blocks_k = o; o += al256c(sizeof(int) * 5 * (size_t)L.nbk);
+    L.zero_bytes = o;
+    L.sel = o; o += al256c(sizeof(int) * (size_t)max(T, 1));
+    L.rngq = o; o += al256c(sizeof(int) * 2 * (size_t)max(Tq, 1));
+    L.rngk = o; o += al256c(sizeof(int) * 2 * (size_t)max(T, 1));
+    L.queue = o; o += al256c(sizeof(int) * (size_t)max(L.nbq, L.nbk));
+    L.delta = o; if (bwd) o += al256c(sizeof(float) * (size_t)H * max(Tq, 1));
+    L.total = o + 256;
+    return L;
+}
+
+__device__ __forceinline__ int chosen(const int8_t *level, int i, int level_mask) {
+    const int lv = level[i];
+    return (lv >= 0 && lv < 31 && ((level_mask >> lv) & 1)) ? 1 : 0;
+}
+
+// cnt[b] = chosen tokens of document b
+__global__ void k_cross_count(const int8_t *__restrict__ level, const int32_t *__restrict__ cu_k, int level_mask,
+                              int *cnt) {
+    const int b = blockIdx.x;
+    int c = 0;
+    for (int i = cu_k[b] + threadIdx.x; i < cu_k[b + 1]; i += blockDim.x) c += chosen(level, i, level_mask);
+    for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(&cnt[b], c);
+}
+
+// cu_sel = exclusive scan of cnt (one CTA); queue = identity
+__global__ void __launch_bounds__(1024) k_cross_scan(const int *__restrict__ cnt, int B, int *cu_sel, int *queue, int nq) {
+    __shared__ int s_w[32];
+    __shared__ int s_carry;
+    const int t = threadIdx.x, lane = t & 31, w = t >> 5;
+    if (t == 0) s_carry = 0;
+    __syncthreads();
+    for (int base = 0; base < B; base += 1024) {
+        const int b = base + t;
+        const int c = (b < B) ? cnt[b] : 0;
+        int v = c;
+        for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
+        if (lane == 31) s_w[w] = v;
+        __syncthreads();
+        if (w == 0) {
+            int x = s_w[lane];
+            for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(0xffffffffu, x, o); if (lane >= o) x += y; }
+            s_w[lane] = x;
+        }
+        __syncthreads();
+        if (b < B) cu_sel[b] = s_carry + (w ? s_w[w - 1] : 0) + v - c;
+        __syncthreads();
+        if (t == 0) s_carry += s_w[31];
+        __syncthreads();
+    }
+    if (t == 0) cu_sel[B] = s_carry;
+    for (int i = t; i < nq; i += 1024) queue[i] = i;
+}
+
+// Document b: ordered list of its chosen tokens, the key range of its decoder rows, the row range of
+// its chosen keys, and the block records of both sides.
+__global__ void __launch_bounds__(256) k_cross_fill(const int8_t *__restrict__ level, const int32_t *__restrict__ cu_k,
+                                                    const int32_t *__restrict__ cu_q, int level_mask,
+                                                    const int *__restrict__ cu_sel, int *sel, int *rngq, int *rngk,
+                                                    int *blocks_q, int *blocks_k) {
+    __shared__ int s_w[8];
+    __shared__ int s_carry;
+    const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, w = t >> 5;
+    const int k0 = cu_k[b], k1 = cu_k[b + 1], q0 = cu_q[b], q1 = cu_q[b + 1], s0 = cu_sel[b], s1 = cu_sel[b + 1];
+    if (t == 0) s_carry = 0;
+    __syncthreads();
+    for (int base = k0; base < k1; base += 256) {
+        const int i = base + t;
+        const int f = (i < k1) ? chosen(level, i, level_mask) : 0;
+        int v = f;
+        for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
+        if (lane == 31) s_w[w] = v;
+        __syncthreads();
+        int before = s_carry;
+        for (int j = 0; j < w; ++j) before += s_w[j];
+        if (f) {
+            const int pos = s0 + before + v - 1;
+            sel[pos] = i;
+            rngk[2 * pos] = q0;
+            rngk[2 * pos + 1] = q1;
+        }
+        __syncthreads();
+        if (t == 0) { int tot = 0; for (int j = 0; j < 8; ++j) tot += s_w[j]; s_carry += tot; }
+        __syncthreads();
+    }
+    for (int r = q0 + t; r < q1; r += 256) { rngq[2 * r] = s0; rngq[2 * r + 1] = s1; }
+    const int live = (s1 > s0 && q1 > q0) ? 0 : HDT_BLK_EMPTY;
+    const int slot_q = q0 / XR + b, nbq = (q1 - q0 + XR - 1) / XR;
+    for (int j = t; j < nbq; j += 256) {
+        int *rec = blocks_q + 5 * (size_t)(slot_q + j);
+        rec[0] = q0 + j * XR; rec[1] = min(q1, q0 + (j + 1) * XR); rec[2] = s0; rec[3] = s1; rec[4] = live;
+    }
+    const int slot_k = s0 / XR + b, nbk = (s1 - s0 + XR - 1) / XR;
+    for (int j = t; j < nbk; j += 256) {
+        int *rec = blocks_k + 5 * (size_t)(slot_k + j);
+        rec[0] = s0 + j * XR; rec[1] = min(s1, s0 + (j + 1) * XR); rec[2] = q0; rec[3] = q1; rec[4] = live;
+    }
+}
+
+static int cross_build(const CrossLayout &L, char *ws, const int8_t *level, const int32_t *cu_k, const int32_t *cu_q,
+                       int B, int level_mask, cudaStream_t st) {
+    HDT_CUDA_CHECK(cudaMemsetAsync(ws, 0, L.zero_bytes, st));
+    if (B > 0) {
+        k_cross_count<<<B, 256, 0, st>>>(level, cu_k, level_mask, (int *)(ws + L.cnt));
+        k_cross_scan<<<1, 1024, 0, st>>>((const int *)(ws + L.cnt), B, (int *)(ws + L.cu_sel), (int *)(ws + L.queue),
+                                         max(L.nbq, L.nbk));
+        k_cross_fill<<<B, 256, 0, st>>>(level, cu_k, cu_q, level_mask, (const int *)(ws + L.cu_sel), (int *)(ws + L.sel),
+                                        (int *)(ws + L.rngq), (int *)(ws + L.rngk), (int *)(ws + L.blocks_q),
+                                        (int *)(ws + L.blocks_k));
+        count_launch(3);
+    }
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+
+static int cross_check(const void *level, const void *cu_k, const void *cu_q, int B, int T, int Tq, int H, int D,
+                       int dtype, int level_mask, const void *ws, size_t ws_bytes, size_t need, const char *who) {
+    if (B < 0 || T < 0 || Tq < 0 || H < 1) return set_error(HDT_ERR_INVALID_ARG, "%s: negative size or no head", who);
+    if (D != 64 && D != 128) return set_error(HDT_ERR_UNSUPPORTED, "%s: head_dim %d not supported (64 or 128)", who, D);
+    if (dtype != HDT_F32 && dtype != HDT_BF16) return set_error(HDT_ERR_UNSUPPORTED, "%s: unknown dtype %d", who, dtype);
+    if (level_mask < 0) return set_error(HDT_ERR_INVALID_ARG, "%s: level_mask must be a set of level bits 0..30", who);
+    if (!cu_k || !cu_q || (T > 0 && !level)) return set_error(HDT_ERR_INVALID_ARG, "%s: null structure pointer", who);
+    if (!ws || ws_bytes < need) return set_error(HDT_ERR_WORKSPACE, "%s: workspace %zu < required %zu", who, ws_bytes, need);
+    if ((uintptr_t)ws & 255) return set_error(HDT_ERR_INVALID_ARG, "%s: workspace must be 256-byte aligned", who);
+    return HDT_OK;
+}
+
+}  // namespace hdt
+
+using namespace hdt;
+
+extern "C" size_t hdt_cross_workspace_bytes(int32_t batch, int32_t total_tokens, int32_t total_q, int32_t heads,
+                                            int32_t bwd) {
+    if (batch < 0 || total_tokens < 0 || total_q < 0 || heads < 1) return 0;
+    return cross_layout(batch, total_tokens, total_q, heads, bwd).total;
+}
+
+extern "C" int hdt_cross_attn_fwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q,
+                                  int32_t batch, int32_t total_tokens, int32_t total_q, int32_t level_mask,
+                                  const void *q, const void *k, const void *v, void *o, float *lse, int32_t heads,
+                                  int32_t head_dim, int32_t dtype, float softmax_scale, void *workspace,
+                                  size_t workspace_bytes, void *stream) {
+    const CrossLayout L = cross_layout(max(batch, 0), max(total_tokens, 0), max(total_q, 0), max(heads, 1), 0);
+    int rc = cross_check(level, cu_seqlens_k, cu_seqlens_q, batch, total_tokens, total_q, heads, head_dim, dtype,
+                         level_mask, workspace, workspace_bytes, L.total, "hdt_cross_attn_fwd");
+    if (rc) return rc;
+    if (total_q == 0) return HDT_OK;
+    if (!q || !o || !lse || (total_tokens > 0 && (!k || !v)))
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_cross_attn_fwd: null tensor pointer");
+    cudaStream_t st = (cudaStream_t)stream;
+    char *ws = (char *)workspace;
+    rc = cross_build(L, ws, level, cu_seqlens_k, cu_seqlens_q, batch, level_mask, st);
+    if (rc) return rc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    FwdStageArgs a{};
+    a.n = total_q; a.nb = L.nbq; a.H = heads; a.T = total_q;
+    a.tok = (const int *)(ws + L.sel);      // keys through the list of chosen tokens
+    a.tok_rows = nullptr;                   // decoder rows in place
+    a.rng = (const int *)(ws + L.rngq); a.blocks = (const int *)(ws + L.blocks_q);
+    a.queue = (const int *)(ws + L.queue); a.queue_split = a.queue;
+    a.q = q; a.k = k; a.v = v; a.o = o; a.lse = lse;
+    a.scale_log2 = scale * 1.4426950408889634f;
+    a.status = device_status_ptr();
+    a.block_rows = XR; a.dirs = 7;
+    return launch_fwd_simt(a, head_dim, dtype, st);
+}
+
+extern "C" int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q,
+                                  int32_t batch, int32_t total_tokens, int32_t total_q, int32_t level_mask,
+                                  const void *q, const void *k, const void *v, const void *o, const float *lse,
+                                  const void *d_o, void *dq, void *dk, void *dv, int32_t heads, int32_t head_dim,
+                                  int32_t dtype, float softmax_scale, void *workspace, size_t workspace_bytes,
+                                  void *stream) {
+    const CrossLayout L = cross_layout(max(batch, 0), max(total_tokens, 0), max(total_q, 0), max(heads, 1), 1);
+    int rc = cross_check(level, cu_seqlens_k, cu_seqlens_q, batch, total_tokens, total_q, heads, head_dim, dtype,
+                         level_mask, workspace, workspace_bytes, L.total, "hdt_cross_attn_bwd");
+    if (rc) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t esz = dtype == HDT_BF16 ? 2 : 4;
+    if (total_tokens > 0) {
+        if (!dk || !dv) return set_error(HDT_ERR_INVALID_ARG, "hdt_cross_attn_bwd: null tensor pointer");
+        // encoder rows outside the subset (and of documents without decoder rows) get zero gradients
+        HDT_CUDA_CHECK(cudaMemsetAsync(dk, 0, (size_t)total_tokens * heads * head_dim * esz, st));
+        HDT_CUDA_CHECK(cudaMemsetAsync(dv, 0, (size_t)total_tokens * heads * head_dim * esz, st));
+    }
+    if (total_q == 0) return HDT_OK;
+    if (!q || !o || !lse || !d_o || !dq || (total_tokens > 0 && (!k || !v)))
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_cross_attn_bwd: null tensor pointer");
+    char *ws = (char *)workspace;
+    rc = cross_build(L, ws, level, cu_seqlens_k, cu_seqlens_q, batch, level_mask, st);
+    if (rc) return rc;
+    float *delta = (float *)(ws + L.delta);
+    rc = launch_delta(o, d_o, delta, total_q, heads, head_dim, dtype, st);
+    if (rc) return rc;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    BwdStageArgs a{};
+    a.H = heads; a.T = total_q;
+    a.queue = (const int *)(ws + L.queue); a.queue_split = a.queue;
+    a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = delta;
+    a.scale = scale; a.scale_log2 = scale * 1.4426950408889634f;
+    a.dq = dq; a.dk = dk; a.dv = dv;
+    a.status = device_status_ptr();
+    a.block_rows = XR; a.dirs = 7;
+    // decoder rows as queries: dQ
+    BwdStageArgs aq = a;
+    aq.n = total_q; aq.nb = L.nbq; aq.phases = 1;
+    aq.tok = (const int *)(ws + L.sel); aq.tok_rows = nullptr;
+    aq.rng = (const int *)(ws + L.rngq); aq.blocks = (const int *)(ws + L.blocks_q);
+    rc = launch_bwd_simt(aq, head_dim, dtype, st);
+    if (rc) return rc;
+    // chosen encoder rows as keys: dK, dV, scattered to their token rows
+    BwdStageArgs ak = a;
+    ak.n = total_tokens; ak.nb = L.nbk; ak.phases = 2;
+    ak.tok = nullptr; ak.tok_rows = (const int *)(ws + L.sel);
+    ak.rng = (const int *)(ws + L.rngk); ak.blocks = (const int *)(ws + L.blocks_k);
+    return launch_bwd_simt(ak, head_dim, dtype, st);
+}

@@ -118,6 +118,7 @@ struct FwdStageArgs {
     int no_persistent;  // option: do not use the persistent kernels
     int block_rows;     // max rows of a block in this stage
     int dirs;           // direction bits kept (7 = full rule), see dir_ok
+    const int *tok_rows;  // SIMT kernels: token map of the block rows (nullptr: identity); `tok` maps the keys
 };
 
 struct BwdStageArgs {
@@ -139,6 +140,8 @@ struct BwdStageArgs {
     int no_persistent;                            // option: do not use the persistent kernels
     int block_rows;                               // max rows of a block in this stage
     int dirs;                                     // direction bits kept (7 = full rule), see dir_ok
+    const int *tok_rows;                          // SIMT kernel: token map of the block rows (nullptr: identity); `tok` maps the walked span
+    int phases;                                   // SIMT kernel: 0 = both, 1 = rows as queries only (dQ), 2 = rows as keys only (dK, dV)
 };
 
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);

@@ -1,0 +1,86 @@
+"""GPU parity of hdt_cross_attn_fwd / hdt_cross_attn_bwd (decoder rows attending to a level subset of
+the encoder tokens) against the fp64 oracle: fp32 <= 1e-4, bf16 max <= 2e-2 and mean <= 2e-3."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+from oracle import cross_oracle as co
+from gpu_util import check_close, dev_tensor, host
+
+pytestmark = pytest.mark.gpu
+
+DOC, SEC, SENT, TOK = 1, 2, 4, 8
+
+
+def case(b, nq, H, d, dtype, seed):
+    rng = np.random.default_rng(seed)
+    cu_q = np.concatenate([[0], np.cumsum(nq)]).astype(np.int32)
+    Tq = int(cu_q[-1])
+    f = gen.round_bf16 if dtype == "bf16" else (lambda x: x)
+    qd, do = (f(rng.standard_normal((Tq, H, d)).astype(np.float32)) for _ in range(2))
+    k, v = (f(rng.standard_normal((b.total_tokens, H, d)).astype(np.float32)) for _ in range(2))
+    if dtype == "bf16":
+        do = do * 0.125      # gradients of order one: the absolute bf16 tolerance is stated for that range
+    return cu_q, qd, k, v, do
+
+
+def run(P, b, nq, mask, H, d, dtype, seed):
+    cu_q, qd, k, v, do = case(b, nq, H, d, dtype, seed)
+    lv = torch.from_numpy(b.level).cuda()
+    cuk = torch.from_numpy(b.cu_seqlens).cuda()
+    cuq = torch.from_numpy(cu_q).cuda()
+    tq, tk, tv, tdo = (dev_tensor(x, dtype) for x in (qd, k, v, do))
+    o, lse = P.hdt_cross_attn_fwd(lv, cuk, cuq, mask, tq, tk, tv)
+    o_r, lse_r = co.forward(b.level, b.cu_seqlens, mask, cu_q, qd, k, v)
+    check_close(host(o), o_r, dtype, "O")
+    check_close(host(lse), lse_r, "f32" if dtype == "f32" else "bf16", "LSE")
+    dq = torch.full_like(tq, float("nan")); dk = torch.full_like(tk, float("nan")); dv = torch.full_like(tv, float("nan"))
+    P.hdt_cross_attn_bwd(lv, cuk, cuq, mask, tq, tk, tv, o, lse, tdo, dq=dq, dk=dk, dv=dv)
+    dq_r, dk_r, dv_r = co.backward(b.level, b.cu_seqlens, mask, cu_q, qd, k, v, do)
+    check_close(host(dq), dq_r, dtype, "dQ")
+    check_close(host(dk), dk_r, dtype, "dK")
+    check_close(host(dv), dv_r, dtype, "dV")
+    P.hdt_device_status()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mask", [SEC, SEC | SENT, SEC | SENT | TOK, DOC | SEC | SENT | TOK])
+def test_cross_attention_small(mask, dtype):
+    import paper_2407_08330_b200 as P
+    b = gen.small_random_batch(61, n_seqs=5, max_len=400, K=(0, 25))
+    run(P, b, [70, 0, 33, 1, 129], mask, 2, 64, dtype, 3)           # a document without decoder rows, ragged blocks
+
+
+def test_cross_attention_edge_cases():
+    import paper_2407_08330_b200 as P
+    # a document whose subset is empty (only its root), PAD tails, head_dim 128
+    b = gen.small_random_batch(62, n_seqs=3, pad_to=200, max_len=150)
+    lone = gen.pack([(np.array([0], np.int8), np.array([-1], np.int32))] + [
+        (b.level[b.cu_seqlens[s]:b.cu_seqlens[s + 1]], b.parent[b.cu_seqlens[s]:b.cu_seqlens[s + 1]]) for s in range(b.batch)])
+    run(P, lone, [5, 40, 7, 64], SEC | SENT, 3, 128, "f32", 4)
+    run(P, lone, [5, 40, 7, 64], SEC | SENT, 3, 128, "bf16", 5)
+    run(P, lone, [0, 0, 0, 0], SEC, 1, 64, "f32", 6)                # no decoder rows at all: dK = dV = 0
+
+
+def test_cross_attention_config3_anchor_subsets():
+    """Encoder side of configuration 3 (4 x 8192 tokens), 256 decoder rows per document, attending
+    to the [SEC] and [SENT] anchors: sampled decoder rows and keys against the oracle."""
+    import paper_2407_08330_b200 as P
+    b = gen.make_hierarchy(3)
+    H, d = 12, 64
+    cu_q, qd, k, v, do = case(b, [256] * 4, H, d, "bf16", 7)
+    lv = torch.from_numpy(b.level).cuda(); cuk = torch.from_numpy(b.cu_seqlens).cuda(); cuq = torch.from_numpy(cu_q).cuda()
+    tq, tk, tv, tdo = (dev_tensor(x, "bf16") for x in (qd, k, v, do))
+    o, lse = P.hdt_cross_attn_fwd(lv, cuk, cuq, SEC | SENT, tq, tk, tv)
+    dq, dk, dv = P.hdt_cross_attn_bwd(lv, cuk, cuq, SEC | SENT, tq, tk, tv, o, lse, tdo)
+    P.hdt_device_status()
+    o_r, lse_r = co.forward(b.level, b.cu_seqlens, SEC | SENT, cu_q, qd, k, v)
+    dq_r, dk_r, dv_r = co.backward(b.level, b.cu_seqlens, SEC | SENT, cu_q, qd, k, v, do)
+    check_close(host(o), o_r, "bf16", "O")
+    check_close(host(lse), lse_r, "bf16", "LSE")
+    check_close(host(dq), dq_r, "bf16", "dQ")
+    check_close(host(dk), dk_r, "bf16", "dK")
+    check_close(host(dv), dv_r, "bf16", "dV")
+    regular = torch.from_numpy(b.level == 3).cuda()
+    assert (dk[regular] == 0).all() and (dv[regular] == 0).all()
