@@ -56,6 +56,22 @@ def workload(c):
     return cfg, b
 
 
+def max_over_ranks(x, dev):
+    """Largest value of x over the ranks of the default process group (x itself without one)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(flops_per_replica, world, ms):
+    """Whole-job effective TFLOP/s of `world` independent replicas that all finish within `ms`."""
+    return flops_per_replica * world / (ms * 1e-3) / 1e12
+
+
 def flops_per_step(nnz, H, d, backward):
     return (4 + (10 if backward else 0)) * d * nnz * H
 
@@ -315,10 +331,7 @@ def main():
         wall = time.perf_counter() - w0
     launches = P.hdt_launch_count() - l0
     ms = float(np.sum(times)) / args.steps
-    if world > 1:
-        tm = torch.tensor([ms], device=dev)
-        dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-        ms = float(tm.item())
+    ms = max_over_ranks(ms, dev)
 
     # phase split and per-kernel device times (library-side CUDA events on the launch stream)
     L = P.lib()
@@ -368,14 +381,11 @@ def main():
             step_e2e()
         barrier()
         e_ms = (time.perf_counter() - w0) / n_e * 1e3
-        if world > 1:
-            tm = torch.tensor([e_ms], device=dev)
-            dist.all_reduce(tm, op=dist.ReduceOp.MAX)
-            e_ms = float(tm.item())
+        e_ms = max_over_ranks(e_ms, dev)
         esz = q.element_size()
         n_in = 3 + (1 if cfg.backward else 0)
         n_out = 1 + (3 if cfg.backward else 0)
-        e2e = {"value": flops_per_step(nnz, H, d, cfg.backward) * world / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+        e2e = {"value": job_value(flops_per_step(nnz, H, d, cfg.backward), world, e_ms), "unit": "TFLOP/s",
                "h2d_bytes_per_step": n_in * T * H * d * esz + T * 5 + (b.batch + 1) * 4,
                "d2h_bytes_per_step": n_out * T * H * d * esz + H * T * 4, "ms_per_step": e_ms}
 
@@ -443,7 +453,7 @@ def main():
     if hpe:
         hpe["frac_of_hbm_peak"] = hpe["achieved_gbs"] / pk["hbm_gbs"]
     fl = flops_per_step(nnz, H, d, cfg.backward)
-    value = fl * world / (ms * 1e-3) / 1e12
+    value = job_value(fl, world, ms)
     real = b.real_tokens
     esz = 2 if cfg.dtype == "bf16" else 4
     alg_bytes = {"k_fwd_stage0": (4 * d * esz + 4) * real * H,
