@@ -168,11 +168,11 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             // whether the parent entry / every other entry of the range is kept
             const int c_self = row - c0, c_head = (lo < row) ? lo - c0 : -0x40000000;
             const bool keep_head = (a.dirs & 1) != 0, keep_rest = (a.dirs & ((lo >= row) ? 4 : 2)) != 0;
-            auto kept = [&](int c) { return !DIRS || c == c_self || (c == c_head ? keep_head : keep_rest); };
             float mx = NEG;
             for (int k = 0; k < nsl; ++k) {
                 const int s0 = 32 * k;
-                const bool mine = has && jl < s0 + 32 && jh > s0;
+                const uint32_t km = has ? keep_mask<DIRS>(s0, 32, jl, jh, c_self, c_head, keep_head, keep_rest) : 0u;
+                const bool mine = km != 0u;
                 if (__any_sync(0xffffffffu, mine)) {
                     uint32_t r[32];
                     tmem_ld32(tmem + TM_S + lane_base + s0, r);
@@ -180,7 +180,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                     if (mine) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (s0 + j >= jl && s0 + j < jh && kept(s0 + j)) mx = fmaxf(mx, __uint_as_float(r[j]));
+                            if (km & (1u << j)) mx = fmaxf(mx, __uint_as_float(r[j]));
                     }
                 }
             }
@@ -189,7 +189,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             float lsum = 0.f;
             for (int k = 0; k < nsl; ++k) {
                 const int s0 = 32 * k;
-                const bool mine = has && jl < s0 + 32 && jh > s0;
+                const uint32_t km = has ? keep_mask<DIRS>(s0, 32, jl, jh, c_self, c_head, keep_head, keep_rest) : 0u;
+                const bool mine = km != 0u;
                 uint32_t pk[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) pk[j] = 0u;
@@ -201,10 +202,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
                             float p0 = 0.f, p1 = 0.f;
-                            if (s0 + j >= jl && s0 + j < jh && kept(s0 + j))
-                                p0 = exp2f(fmaf(__uint_as_float(r[j]), a.scale_log2, -m_new));
-                            if (s0 + j + 1 >= jl && s0 + j + 1 < jh && kept(s0 + j + 1))
-                                p1 = exp2f(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m_new));
+                            if (km & (1u << j)) p0 = exp2f(fmaf(__uint_as_float(r[j]), a.scale_log2, -m_new));
+                            if (km & (2u << j)) p1 = exp2f(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m_new));
                             // the row sum uses the bf16-rounded probabilities the MMA will see
                             const uint32_t u = pack_bf16(p0, p1);
                             lsum += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
@@ -347,7 +346,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 // K of the next item are fetched as soon as P V of the current one has finished (P, which lives
 // in the Q/K tiles, is dead then), V of the next item once the staged O has left the V tile.
 // ---------------------------------------------------------------------------------------------
-template <int D>
+template <int D, bool DIRS = false>
 __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
                                                      const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
@@ -442,10 +441,14 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             const int jl = max(lo - ka, 0), jh = min(hi - ka, nvalid);
             const bool has = inb && jh > jl;
             const int nsl = (Nc + 31) >> 5;
+            // direction bits (DIRS instantiation): see dir_ok
+            const int c_self = row - ka, c_head = (lo < row) ? lo - ka : -0x40000000;
+            const bool keep_head = (a.dirs & 1) != 0, keep_rest = (a.dirs & ((lo >= row) ? 4 : 2)) != 0;
             float mx = NEG;
             for (int k = 0; k < nsl; ++k) {
                 const int s0 = 32 * k;
-                const bool mine = has && jl < s0 + 32 && jh > s0;
+                const uint32_t km = has ? keep_mask<DIRS>(s0, 32, jl, jh, c_self, c_head, keep_head, keep_rest) : 0u;
+                const bool mine = km != 0u;
                 if (__any_sync(0xffffffffu, mine)) {
                     uint32_t r[32];
                     tmem_ld32(tmem + lane_base + s0, r);
@@ -453,7 +456,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
                     if (mine) {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
-                            if (s0 + j >= jl && s0 + j < jh) mx = fmaxf(mx, __uint_as_float(r[j]));
+                            if (km & (1u << j)) mx = fmaxf(mx, __uint_as_float(r[j]));
                     }
                 }
             }
@@ -461,7 +464,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             float l = 0.f;
             for (int k = 0; k < nsl; ++k) {
                 const int s0 = 32 * k;
-                const bool mine = has && jl < s0 + 32 && jh > s0;
+                const uint32_t km = has ? keep_mask<DIRS>(s0, 32, jl, jh, c_self, c_head, keep_head, keep_rest) : 0u;
+                const bool mine = km != 0u;
                 uint32_t pk[16];
 #pragma unroll
                 for (int j = 0; j < 16; ++j) pk[j] = 0u;
@@ -473,8 +477,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
                             float p0 = 0.f, p1 = 0.f;
-                            if (s0 + j >= jl && s0 + j < jh) p0 = exp2f(fmaf(__uint_as_float(r[j]), a.scale_log2, -m));
-                            if (s0 + j + 1 >= jl && s0 + j + 1 < jh) p1 = exp2f(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m));
+                            if (km & (1u << j)) p0 = exp2f(fmaf(__uint_as_float(r[j]), a.scale_log2, -m));
+                            if (km & (2u << j)) p1 = exp2f(fmaf(__uint_as_float(r[j + 1]), a.scale_log2, -m));
                             const uint32_t u = pack_bf16(p0, p1);   // the row sum uses the rounded values the MMA sees
                             l += __uint_as_float(u << 16) + __uint_as_float(u & 0xffff0000u);
                             pk[j >> 1] = u;
@@ -838,6 +842,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             8 * SUB + 4 * 128 * 4 + 1024 + 64));
         attr = true;
@@ -845,26 +851,16 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     FwdStageArgs b = a;
     b.rest_only = 0;
     int n_general = a.nb;
-    if (a.dirs != 7) {   // direction bits: every block through the general kernel that applies them
-        static bool attr_d = false;
-        if (!attr_d) {
-            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            attr_d = true;
-        }
-        k_fwd_tc<D, false, false, true><<<dim3(a.nb, a.H), 128, smem, st>>>(tq, tk, tv, b);
-        count_launch();
-        HDT_CUDA_CHECK(cudaGetLastError());
-        return HDT_OK;
-    }
+    const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
     if (a.n_fused > 0 && a.no_persistent != 1) {
-        if (D == 64 && a.no_persistent == 2) {   // option: the persistent single-CTA-per-SM kernel
+        if (D == 64 && a.no_persistent == 2 && !dirs) {   // option: the persistent single-CTA-per-SM kernel
             constexpr int smem_p = 8 * SUB + 4 * 128 * 4 + 1024 + 64;
             int dev = 0, n_sm = 0;
             HDT_CUDA_CHECK(cudaGetDevice(&dev));
             HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
             const long long items = (long long)a.n_fused * a.H;
             k_fwd_tc_p<<<(int)(items < n_sm ? items : n_sm), 512, smem_p, st>>>(tq, tk, tv, a);
-        } else if (a.no_persistent == 3) {       // option: one CTA per (block, head), no loop
+        } else if (a.no_persistent == 3 && !dirs) {       // option: one CTA per (block, head), no loop
             k_fwd_tc<D, true><<<dim3(a.n_fused, a.H), 128, smem_1, st>>>(tq, tk, tv, a);
         } else {
             int dev = 0, n_sm = 0;
@@ -872,7 +868,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
             HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
             const long long items = (long long)a.n_fused * a.H;
             const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
-            k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
+            if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
+            else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
         }
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
@@ -881,7 +878,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     }
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
-        k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);
+        if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);
+        else k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
     }

@@ -158,7 +158,6 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         // whether the parent entry / every other entry of the range is kept
         const int c_self = e - k_row0, c_head = (lo < e) ? lo - k_row0 : -0x40000000;
         const bool keep_head = (a.dirs & 1) != 0, keep_rest = (a.dirs & ((lo >= e) ? 4 : 2)) != 0;
-        auto kept = [&](int c) { return !DIRS || c == c_self || (c == c_head ? keep_head : keep_rest); };
         ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
         ph_mma ^= 1;
         tc_fence_after();
@@ -166,7 +165,8 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         for (int sl = 0; sl < 2; ++sl) {
             const int s0 = 64 * hf + 32 * sl;
             if (s0 >= Nc) continue;  // same decision in the whole warp (hf, Nc uniform)
-            const bool mine = has && jl < s0 + 32 && jh > s0;
+            const uint32_t km = has ? keep_mask<DIRS>(s0, 32, jl, jh, c_self, c_head, keep_head, keep_rest) : 0u;
+            const bool mine = km != 0u;
             uint32_t pp[16], pd[16];
 #pragma unroll
             for (int j = 0; j < 16; ++j) { pp[j] = 0u; pd[j] = 0u; }
@@ -179,11 +179,11 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
 #pragma unroll
                     for (int j = 0; j < 32; j += 2) {
                         float p0 = 0.f, p1 = 0.f, d0 = 0.f, d1 = 0.f;
-                        if (s0 + j >= jl && s0 + j < jh && kept(s0 + j)) {
+                        if (km & (1u << j)) {
                             p0 = exp2f(fmaf(__uint_as_float(rs[j]), a.scale_log2, -lse2));
                             d0 = p0 * (__uint_as_float(rd[j]) - dl);
                         }
-                        if (s0 + j + 1 >= jl && s0 + j + 1 < jh && kept(s0 + j + 1)) {
+                        if (km & (2u << j)) {
                             p1 = exp2f(fmaf(__uint_as_float(rs[j + 1]), a.scale_log2, -lse2));
                             d1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
                         }
@@ -401,7 +401,7 @@ __device__ long long g_bwd_phase_cycles[16];
 // tile is stored as the binary decomposition of its row count.
 struct StoreMaps { CUtensorMap m[3][7]; };
 
-template <bool SPLIT>
+template <bool SPLIT, bool DIRS = false>
 __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
                                                      const __grid_constant__ CUtensorMap tm_v,
@@ -596,6 +596,10 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             const float lse2 = rc.lse2 * LOG2E, dl = rc.dl;
             const int jl = max(rc.lo - k0, 0), jh = min(rc.hi - k0, nk);
             const bool has = inq && jh > jl;
+            // direction bits (DIRS instantiations): see dir_ok
+            const int e_row = d0.q0 + rl;
+            const int c_self = e_row - k0, c_head = (rc.lo < e_row) ? rc.lo - k0 : -0x40000000;
+            const bool keep_head = (a.dirs & 1) != 0, keep_rest = (a.dirs & ((rc.lo >= e_row) ? 4 : 2)) != 0;
             const int flags = SPLIT ? d0.flags : (F_DQ | F_DKDV | F_LAST);   // constant for self-contained blocks
             uint8_t *st = sIn + (it & 1) * 4 * SUB;
 
@@ -611,7 +615,8 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
 #pragma unroll
                 for (int hh = 0; hh < 2; ++hh) {
                     const int s0 = 32 * qt + 16 * hh;
-                    const bool mine = has && jl < s0 + 16 && jh > s0;
+                    const uint32_t km = has ? keep_mask<DIRS>(s0, 16, jl, jh, c_self, c_head, keep_head, keep_rest) : 0u;
+                    const bool mine = km != 0u;
                     uint32_t pp[8], pd[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) { pp[j] = 0u; pd[j] = 0u; }
@@ -624,11 +629,11 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
 #pragma unroll
                             for (int j = 0; j < 16; j += 2) {
                                 float p0 = 0.f, p1 = 0.f, e0 = 0.f, e1 = 0.f;
-                                if (s0 + j >= jl && s0 + j < jh) {
+                                if (km & (1u << j)) {
                                     p0 = exp2f(fmaf(__uint_as_float(rs[j]), a.scale_log2, -lse2));
                                     e0 = p0 * (__uint_as_float(rd[j]) - dl);
                                 }
-                                if (s0 + j + 1 >= jl && s0 + j + 1 < jh) {
+                                if (km & (2u << j)) {
                                     p1 = exp2f(fmaf(__uint_as_float(rs[j + 1]), a.scale_log2, -lse2));
                                     e1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
                                 }
@@ -769,17 +774,7 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     BwdStageArgs b = a;
     b.rest_only = 0;
     int n_general = a.nb;
-    if (a.dirs != 7) {   // direction bits: every block through the general kernel that applies them
-        static bool attr_d = false;
-        if (!attr_d) {
-            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-            attr_d = true;
-        }
-        k_bwd_tc<D, false, true><<<dim3(a.nb, a.H), 256, smem, st>>>(tq, tk, tv, tdo, b);
-        count_launch();
-        HDT_CUDA_CHECK(cudaGetLastError());
-        return HDT_OK;
-    }
+    const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
     if (D == 64 && a.nb > 0 && !a.no_persistent) {
         // the persistent kernel takes everything: first the blocks of split families (longest first),
         // then the self-contained blocks
@@ -789,6 +784,8 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
         if (!attr_p) {
             HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
             HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
             int dev = 0;
             HDT_CUDA_CHECK(cudaGetDevice(&dev));
             HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
@@ -807,7 +804,10 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
             BwdStageArgs c = a;
             c.rest_only = mode;
             const int grid_p = (int)(units < n_sm ? units : n_sm);
-            if (mode) k_bwd_tc_p<true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
+            if (dirs) {
+                if (mode) k_bwd_tc_p<true, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
+                else k_bwd_tc_p<false, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
+            } else if (mode) k_bwd_tc_p<true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
             else k_bwd_tc_p<false><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
             count_launch();
             HDT_CUDA_CHECK(cudaGetLastError());
@@ -816,7 +816,14 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     }
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
-        k_bwd_tc<D><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, b);
+        if (dirs) {
+            static bool attr_d = false;
+            if (!attr_d) {
+                HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+                attr_d = true;
+            }
+            k_bwd_tc<D, false, true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, b);
+        } else k_bwd_tc<D><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, b);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
     }

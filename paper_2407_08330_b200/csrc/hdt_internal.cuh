@@ -89,6 +89,27 @@ __host__ __device__ __forceinline__ bool dir_ok_key(int key, int i, int lo, int 
     return (dirs & (i == lo ? 4 : 2)) != 0;           // i is key's parent, or a sibling
 }
 
+// Tensor-core kernels: bit j of the result says that column s0 + j (j < W <= 32) of a row's tile is
+// one of its kept entries: inside the row's range [jl, jh) (tile-relative) and, with direction
+// bits (DIRS), not switched off.  c_self / c_head: tile-relative columns of the row itself and of
+// its parent (far negative for a head row); keep_head / keep_rest: whether the parent entry / every
+// other entry of the range is kept (see dir_ok).
+template <bool DIRS>
+__device__ __forceinline__ uint32_t keep_mask(int s0, int W, int jl, int jh, int c_self, int c_head, bool keep_head,
+                                              bool keep_rest) {
+    const int lo = max(jl - s0, 0), hi = min(jh - s0, W);
+    if (hi <= lo) return 0u;
+    uint32_t m = (hi >= 32 ? 0xffffffffu : ((1u << hi) - 1u)) & ~((1u << lo) - 1u);
+    if constexpr (DIRS) {
+        uint32_t k = keep_rest ? 0xffffffffu : 0u;
+        const int cs = c_self - s0, ch = c_head - s0;
+        if (cs >= 0 && cs < 32) k |= 1u << cs;
+        if (ch >= 0 && ch < 32) k = keep_head ? (k | (1u << ch)) : (k & ~(1u << ch));
+        m &= k;
+    }
+    return m;
+}
+
 // SIMT attention launchers (hdt_attn_simt.cu).  One launch handles one stage.
 struct FwdStageArgs {
     // stage view

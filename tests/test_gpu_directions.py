@@ -68,7 +68,7 @@ def test_directed_attention_small(P, d, dtype):
 
 def test_directed_attention_general_and_simt_paths_bf16(P):
     b = small_batches()[0][1]
-    for opt in ({"no_overlap": 1}, {"force_simt": 1}):
+    for opt in ({"no_overlap": 1}, {"no_persistent": 1}, {"force_simt": 1}):
         for k_, v_ in opt.items():
             P.hdt_set_option(k_, v_)
         try:
