@@ -91,7 +91,8 @@ def _ptr(t):
 
 
 def _stream():
-    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+    # the raw handle of the current stream without building a torch.cuda.Stream object
+    return C.c_void_p(torch._C._cuda_getCurrentRawStream(torch.cuda.current_device()))
 
 
 def _params(block_m, max_stages, block_m_upper=0, directions=7):
@@ -112,9 +113,26 @@ class HdtIndex:
     def __init__(self, handle, workspace, batch, total_tokens):
         self._h, self._ws = handle, workspace
         self.batch, self.total_tokens = batch, total_tokens
-        ns, nnz, vis = C.c_int32(), C.c_int64(), C.c_int64()
-        _check(lib().hdt_index_info(self._h, C.byref(ns), C.byref(nnz), C.byref(vis)))
-        self.n_stages, self.nnz, self.visited = ns.value, nnz.value, vis.value
+        self._info = None
+
+    def _get_info(self):
+        if self._info is None:
+            ns, nnz, vis = C.c_int32(), C.c_int64(), C.c_int64()
+            _check(lib().hdt_index_info(self._h, C.byref(ns), C.byref(nnz), C.byref(vis)))
+            self._info = (ns.value, nnz.value, vis.value)
+        return self._info
+
+    @property
+    def n_stages(self):
+        return self._get_info()[0]
+
+    @property
+    def nnz(self):
+        return self._get_info()[1]
+
+    @property
+    def visited(self):
+        return self._get_info()[2]
 
     @property
     def handle(self):
@@ -173,10 +191,10 @@ def hdt_attn_workspace_bytes(index: HdtIndex, heads, head_dim, dtype, bwd) -> in
 
 
 def _ws(index, heads, head_dim, dtype, bwd, device, workspace):
+    if workspace is not None:      # the library checks the size itself
+        return workspace, None
     need = hdt_attn_workspace_bytes(index, heads, head_dim, dtype, bwd)
-    if workspace is None:
-        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=device)
-    return workspace, need
+    return torch.empty(max(need, 256), dtype=torch.uint8, device=device), need
 
 
 def hdt_attn_fwd(index: HdtIndex, q, k, v, softmax_scale=0.0, out=None, lse=None, workspace=None):
