@@ -5,7 +5,7 @@
 // the decoder rows of a document and the chosen encoder rows of the same document.
 //
 // The chosen rows are never copied: an ordered list `sel` of their token indices is built per call
-// (count, scan, fill: three small kernels, no host wait) and the fp32 SIMT attention kernels of the
+// (count, scan, fill: three small kernels, 32 CTAs per document, no host wait) and the fp32 SIMT attention kernels of the
 // hierarchical path read K and V through it.  Those kernels take any (row blocks, per-row key
 // range, key map) description, so the forward is one launch over blocks of decoder rows whose key
 // range is the document's slice of `sel`, and the backward two launches: decoder-row blocks for
@@ -20,9 +20,10 @@
 namespace hdt {
 
 constexpr int XR = 32;      // rows per block (the 128-thread SIMT kernels take 32 rows per pass)
+constexpr int XC = 32;      // CTAs (contiguous chunks) per document in the selection kernels
 
 struct CrossLayout {
-    size_t cnt, cu_sel, sel, rngq, rngk, blocks_q, blocks_k, queue, delta, total;
+    size_t cnt, cntc, cu_sel, sel, rngq, rngk, blocks_q, blocks_k, queue, delta, total;
     int nbq, nbk;
     size_t zero_bytes;      // cnt .. queue is cleared at the start of every call
 };
@@ -35,6 +36,7 @@ static CrossLayout cross_layout(int B, int T, int Tq, int H, int bwd) {
     L.nbk = T / XR + B + 1;
     size_t o = 0;
     L.cnt = o; o += al256c(sizeof(int) * (size_t)(B + 1));
+    L.cntc = o; o += al256c(sizeof(int) * (size_t)(B + 1) * XC);
     L.cu_sel = o; o += al256c(sizeof(int) * (size_t)(B + 2));
     L.blocks_q = o; o += al256c(sizeof(int) * 5 * (size_t)L.nbq);
     L.blocks_k = o; o += al256c(sizeof(int) * 5 * (size_t)L.nbk);
@@ -53,14 +55,24 @@ __device__ __forceinline__ int chosen(const int8_t *level, int i, int level_mask
     return (lv >= 0 && lv < 31 && ((level_mask >> lv) & 1)) ? 1 : 0;
 }
 
-// cnt[b] = chosen tokens of document b
+// cnt[b] = chosen tokens of document b; cntc[b][y] = those in its y-th chunk (XC equal chunks)
 __global__ void k_cross_count(const int8_t *__restrict__ level, const int32_t *__restrict__ cu_k, int level_mask,
-                              int *cnt) {
-    const int b = blockIdx.x;
+                              int *cnt, int *cntc) {
+    __shared__ int s_c;
+    const int b = blockIdx.x, y = blockIdx.y;
+    const int k0 = cu_k[b], k1 = cu_k[b + 1], cs = (k1 - k0 + XC - 1) / XC;
+    const int c0 = k0 + y * cs, c1 = min(k1, c0 + cs);
+    if (threadIdx.x == 0) s_c = 0;
+    __syncthreads();
     int c = 0;
-    for (int i = cu_k[b] + threadIdx.x; i < cu_k[b + 1]; i += blockDim.x) c += chosen(level, i, level_mask);
+    for (int i = c0 + threadIdx.x; i < c1; i += blockDim.x) c += chosen(level, i, level_mask);
     for (int o = 16; o; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-    if ((threadIdx.x & 31) == 0 && c) atomicAdd(&cnt[b], c);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(&s_c, c);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        cntc[b * XC + y] = s_c;
+        if (s_c) atomicAdd(&cnt[b], s_c);
+    }
 }
 
 // cu_sel = exclusive scan of cnt (one CTA); queue = identity
@@ -92,21 +104,26 @@ __global__ void __launch_bounds__(1024) k_cross_scan(const int *__restrict__ cnt
     for (int i = t; i < nq; i += 1024) queue[i] = i;
 }
 
-// Document b: ordered list of its chosen tokens, the key range of its decoder rows, the row range of
-// its chosen keys, and the block records of both sides.
+// Chunk y of document b: its part of the ordered list of chosen tokens and of their row ranges,
+// and its share of the document's decoder-row key ranges and of the block records of both sides.
 __global__ void __launch_bounds__(256) k_cross_fill(const int8_t *__restrict__ level, const int32_t *__restrict__ cu_k,
                                                     const int32_t *__restrict__ cu_q, int level_mask,
-                                                    const int *__restrict__ cu_sel, int *sel, int *rngq, int *rngk,
-                                                    int *blocks_q, int *blocks_k) {
+                                                    const int *__restrict__ cu_sel, const int *__restrict__ cntc, int *sel,
+                                                    int *rngq, int *rngk, int *blocks_q, int *blocks_k) {
     __shared__ int s_w[8];
     __shared__ int s_carry;
-    const int b = blockIdx.x, t = threadIdx.x, lane = t & 31, w = t >> 5;
+    const int b = blockIdx.x, y = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
     const int k0 = cu_k[b], k1 = cu_k[b + 1], q0 = cu_q[b], q1 = cu_q[b + 1], s0 = cu_sel[b], s1 = cu_sel[b + 1];
-    if (t == 0) s_carry = 0;
+    const int cs = (k1 - k0 + XC - 1) / XC, c0 = k0 + y * cs, c1 = min(k1, c0 + cs);
+    if (w == 0) {       // chosen tokens of the chunks before this one
+        int v = (lane < y) ? cntc[b * XC + lane] : 0;       // XC == 32: one lane per chunk
+        for (int o = 16; o; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) s_carry = v;
+    }
     __syncthreads();
-    for (int base = k0; base < k1; base += 256) {
+    for (int base = c0; base < c1; base += 256) {
         const int i = base + t;
-        const int f = (i < k1) ? chosen(level, i, level_mask) : 0;
+        const int f = (i < c1) ? chosen(level, i, level_mask) : 0;
         int v = f;
         for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
         if (lane == 31) s_w[w] = v;
@@ -123,15 +140,17 @@ __global__ void __launch_bounds__(256) k_cross_fill(const int8_t *__restrict__ l
         if (t == 0) { int tot = 0; for (int j = 0; j < 8; ++j) tot += s_w[j]; s_carry += tot; }
         __syncthreads();
     }
-    for (int r = q0 + t; r < q1; r += 256) { rngq[2 * r] = s0; rngq[2 * r + 1] = s1; }
+    // decoder rows and block records: spread over the document's chunks
+    const int nt = XC * 256, gt = y * 256 + t;
+    for (int r = q0 + gt; r < q1; r += nt) { rngq[2 * r] = s0; rngq[2 * r + 1] = s1; }
     const int live = (s1 > s0 && q1 > q0) ? 0 : HDT_BLK_EMPTY;
     const int slot_q = q0 / XR + b, nbq = (q1 - q0 + XR - 1) / XR;
-    for (int j = t; j < nbq; j += 256) {
+    for (int j = gt; j < nbq; j += nt) {
         int *rec = blocks_q + 5 * (size_t)(slot_q + j);
         rec[0] = q0 + j * XR; rec[1] = min(q1, q0 + (j + 1) * XR); rec[2] = s0; rec[3] = s1; rec[4] = live;
     }
     const int slot_k = s0 / XR + b, nbk = (s1 - s0 + XR - 1) / XR;
-    for (int j = t; j < nbk; j += 256) {
+    for (int j = gt; j < nbk; j += nt) {
         int *rec = blocks_k + 5 * (size_t)(slot_k + j);
         rec[0] = s0 + j * XR; rec[1] = min(s1, s0 + (j + 1) * XR); rec[2] = q0; rec[3] = q1; rec[4] = live;
     }
@@ -141,10 +160,12 @@ static int cross_build(const CrossLayout &L, char *ws, const int8_t *level, cons
                        int B, int level_mask, cudaStream_t st) {
     HDT_CUDA_CHECK(cudaMemsetAsync(ws, 0, L.zero_bytes, st));
     if (B > 0) {
-        k_cross_count<<<B, 256, 0, st>>>(level, cu_k, level_mask, (int *)(ws + L.cnt));
+        static_assert(XC == 32, "k_cross_fill sums the chunk counts with one lane per chunk");
+        k_cross_count<<<dim3(B, XC), 256, 0, st>>>(level, cu_k, level_mask, (int *)(ws + L.cnt), (int *)(ws + L.cntc));
         k_cross_scan<<<1, 1024, 0, st>>>((const int *)(ws + L.cnt), B, (int *)(ws + L.cu_sel), (int *)(ws + L.queue),
                                          max(L.nbq, L.nbk));
-        k_cross_fill<<<B, 256, 0, st>>>(level, cu_k, cu_q, level_mask, (const int *)(ws + L.cu_sel), (int *)(ws + L.sel),
+        k_cross_fill<<<dim3(B, XC), 256, 0, st>>>(level, cu_k, cu_q, level_mask, (const int *)(ws + L.cu_sel),
+                                                  (const int *)(ws + L.cntc), (int *)(ws + L.sel),
                                         (int *)(ws + L.rngq), (int *)(ws + L.rngk), (int *)(ws + L.blocks_q),
                                         (int *)(ws + L.blocks_k));
         count_launch(3);
