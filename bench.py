@@ -424,7 +424,8 @@ def main():
         xq, xdo = (torch.randn((Tq, H, d), generator=gq).to(tdt).to(dev) for _ in range(2))
         xo = torch.empty_like(xq); xlse = torch.empty((H, Tq), dtype=torch.float32, device=dev)
         xdq = torch.empty_like(xq)
-        ws_x = torch.empty(P.hdt_cross_workspace_bytes(b.batch, T, Tq, H, 1), dtype=torch.uint8, device=dev)
+        ws_x = torch.empty(max(P.hdt_cross_workspace_bytes(b.batch, T, Tq, H, d, tdt, w_) for w_ in (0, 1)),
+                           dtype=torch.uint8, device=dev)
         cross = {"decoder_rows": Tq, "subsets": {}}
         for name, mask in (("[SEC]", 2), ("[SEC]+[SENT]", 6), ("[SEC]+[SENT]+tokens", 14)):
             n_keys = int(sum(int((b.level == l).sum()) for l in range(4) if (mask >> l) & 1))
@@ -433,7 +434,7 @@ def main():
                 P.hdt_cross_attn_fwd(level, cu, cuq, mask, xq, k, v, out=xo, lse=xlse, workspace=ws_x)
                 P.hdt_cross_attn_bwd(level, cu, cuq, mask, xq, k, v, xo, xlse, xdo, dq=xdq, dk=dk, dv=dv, workspace=ws_x)
 
-            n_x = 3 if mask == 14 else args.steps
+            n_x = args.steps
             for _ in range(2):
                 step_x()
             x_ms = float(np.mean(timed(step_x, n_x)))

@@ -257,12 +257,15 @@ int hdt_hpe(const hdt_index_t *index, const int8_t *level, const int32_t *parent
  *   k, v, dk, dv       device [total_tokens, heads, head_dim]; dk, dv are written for every encoder
  *                      row (zero outside the subset)
  *   lse                device float [heads, total_q]
- *   workspace          device, >= hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, bwd),
- *                      256-byte aligned; holds the list of chosen tokens, rebuilt by every call
+ *   workspace          device, >= hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads,
+ *                      head_dim, dtype, bwd), 256-byte aligned; holds the list of chosen tokens,
+ *                      rebuilt by every call, and (bf16) fp32 results per element before they are
+ *                      converted
  * head_dim 64 or 128; softmax_scale <= 0 means 1/sqrt(head_dim).  Asynchronous on `stream`, no
  * host wait.  The chosen rows are read in place through the list (no gathered copy of K, V).
  */
-size_t hdt_cross_workspace_bytes(int32_t batch, int32_t total_tokens, int32_t total_q, int32_t heads, int32_t bwd);
+size_t hdt_cross_workspace_bytes(int32_t batch, int32_t total_tokens, int32_t total_q, int32_t heads,
+                                 int32_t head_dim, int32_t dtype, int32_t bwd);
 int hdt_cross_attn_fwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q, int32_t batch,
                        int32_t total_tokens, int32_t total_q, int32_t level_mask, const void *q, const void *k,
                        const void *v, void *o, float *lse, int32_t heads, int32_t head_dim, int32_t dtype,

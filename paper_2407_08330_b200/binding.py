@@ -275,11 +275,11 @@ def hdt_hpe(index: HdtIndex, level, parent, cu_seqlens, d_model, n_levels=3, dty
     return x
 
 
-def hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, bwd) -> int:
+def hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, head_dim, dtype, bwd) -> int:
     L = lib()
     L.hdt_cross_workspace_bytes.restype = C.c_size_t
-    L.hdt_cross_workspace_bytes.argtypes = [C.c_int32] * 5
-    return int(L.hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, int(bwd)))
+    L.hdt_cross_workspace_bytes.argtypes = [C.c_int32] * 7
+    return int(L.hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, head_dim, _DTYPES[dtype], int(bwd)))
 
 
 def _cross_common(level, cu_seqlens_k, cu_seqlens_q, q, k):
@@ -304,7 +304,7 @@ def hdt_cross_attn_fwd(level, cu_seqlens_k, cu_seqlens_q, level_mask, q, k, v, s
         out = torch.empty_like(q)
     if lse is None:
         lse = torch.empty((H, Tq), dtype=torch.float32, device=q.device)
-    need = hdt_cross_workspace_bytes(B, T, Tq, H, 0)
+    need = hdt_cross_workspace_bytes(B, T, Tq, H, d, q.dtype, 0)
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     _check(L.hdt_cross_attn_fwd(_ptr(level), _ptr(cu_seqlens_k), _ptr(cu_seqlens_q), B, T, Tq, int(level_mask), _ptr(q),
@@ -325,7 +325,7 @@ def hdt_cross_attn_bwd(level, cu_seqlens_k, cu_seqlens_q, level_mask, q, k, v, o
     dq = torch.empty_like(q) if dq is None else dq
     dk = torch.empty_like(k) if dk is None else dk
     dv = torch.empty_like(v) if dv is None else dv
-    need = hdt_cross_workspace_bytes(B, T, Tq, H, 1)
+    need = hdt_cross_workspace_bytes(B, T, Tq, H, d, q.dtype, 1)
     if workspace is None:
         workspace = torch.empty(need, dtype=torch.uint8, device=q.device)
     _check(L.hdt_cross_attn_bwd(_ptr(level), _ptr(cu_seqlens_k), _ptr(cu_seqlens_q), B, T, Tq, int(level_mask), _ptr(q),

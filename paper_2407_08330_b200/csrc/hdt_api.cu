@@ -128,7 +128,7 @@ static bool misaligned(const void *p) { return ((uintptr_t)p & 15) != 0; }
 
 using namespace hdt;
 
-static int g_force_simt = 0;
+namespace hdt { int g_force_simt = 0; }
 static int g_no_persistent = 0;
 static int g_simt_upper = 0;
 

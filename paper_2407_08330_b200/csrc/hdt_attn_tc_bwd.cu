@@ -234,20 +234,21 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
 
     auto load = [&](bool q_side, int row0_q, bool k_side, int row0_k) {
         if constexpr (GATHER) {
-            if (q_side && k_side && row0_q == row0_k) {
+            const int end_q = a.gather_end_q ? a.gather_end_q : a.n, end_k = a.gather_end_k ? a.gather_end_k : a.n;
+            if (q_side && k_side && row0_q == row0_k && end_q == end_k) {
                 uint8_t *const d4[4] = {sQ, sDO, sK, sV};
                 const void *const s4[4] = {a.q, a.d_o, a.k, a.v};
-                gather_tiles<D, 256, 4>(d4, s4, a.tok, row0_q, a.n, H, h, tid);
+                gather_tiles<D, 256, 4>(d4, s4, a.tok, row0_q, end_q, H, h, tid);
             } else {
                 if (q_side) {
                     uint8_t *const d2[2] = {sQ, sDO};
                     const void *const s2[2] = {a.q, a.d_o};
-                    gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_q, a.n, H, h, tid);
+                    gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_q, end_q, H, h, tid);
                 }
                 if (k_side) {
                     uint8_t *const d2[2] = {sK, sV};
                     const void *const s2[2] = {a.k, a.v};
-                    gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_k, a.n, H, h, tid);
+                    gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_k, end_k, H, h, tid);
                 }
             }
             fence_proxy_async_smem();     // generic-proxy writes, read by the MMAs
@@ -317,9 +318,11 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     float *cq = nullptr, *ck = nullptr, *cv = nullptr;
     if constexpr (GATHER) {
         if (inb) {      // the drains write the own gradients here; the staged bf16 copies are not used
-            cq = a.own_dq + ((size_t)row * H + h) * D;
-            ck = a.own_dk + ((size_t)row * H + h) * D;
-            cv = a.own_dv + ((size_t)row * H + h) * D;
+            if (a.phases != 2) cq = a.own_dq + ((size_t)row * H + h) * D;
+            if (a.phases != 1) {
+                ck = a.own_dk + ((size_t)row * H + h) * D;
+                cv = a.own_dv + ((size_t)row * H + h) * D;
+            }
         }
     } else if (inb && a.part_dq != nullptr) {
         const int u = a.up[row];
@@ -338,7 +341,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         drain(TM_DK, true, a.scale, ck, sDS);
         drain(TM_DV, true, 1.f, cv, sQ);
     } else {
-        if (run) {
+        if (run && (!GATHER || a.phases != 2)) {
             // this block as query rows: dQ over the key span
             load(true, r0, false, 0);
             for (int c0 = ka; c0 < kb; c0 += 128) {
@@ -353,7 +356,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         tc_fence_after();
         if constexpr (!GATHER) copy_out(sP, a.dq);
         __syncthreads();
-        if (run) {
+        if (run && (!GATHER || a.phases != 1)) {
             // this block as keys: dK, dV over the same span taken as query rows
             load(false, 0, true, r0);
             for (int c0 = ka; c0 < kb; c0 += 128) {

@@ -4,48 +4,66 @@
 // Encoder and Decoder Stacks").  Within the chosen subset it is plain softmax attention between
 // the decoder rows of a document and the chosen encoder rows of the same document.
 //
-// The chosen rows are never copied: an ordered list `sel` of their token indices is built per call
-// (count, scan, fill: three small kernels, 32 CTAs per document, no host wait) and the fp32 SIMT attention kernels of the
-// hierarchical path read K and V through it.  Those kernels take any (row blocks, per-row key
-// range, key map) description, so the forward is one launch over blocks of decoder rows whose key
-// range is the document's slice of `sel`, and the backward two launches: decoder-row blocks for
-// dQ, blocks of chosen keys (walking the document's decoder rows) for dK and dV, which are
-// scattered to the encoder rows; rows outside the subset are zeroed first.
-// Block slots are assigned without a scan: document b owns the slots from start / 32 + b on,
-// unused slots stay empty (r0 == r1).
+// The chosen rows are never copied.  Every call builds (count, scan, fill: three small kernels,
+// 32 CTAs per document, no host wait) one element space for both sides: elements 0 .. Tq-1 are
+// the decoder rows (token map = identity, into Q / dO / O), elements Tq .. Tq+ns-1 the chosen
+// encoder tokens in order (token map = their index, into K / V); a decoder row's key range is its
+// document's slice of the second part, a chosen token's range the document's decoder rows.  The
+// attention kernels of the hierarchical path take any (row blocks, per-row range, token map)
+// description, so they serve as they are:
+//   bf16  the gathering tcgen05 kernels (128-row blocks): forward over the decoder-row blocks;
+//         backward once over the decoder-row blocks (dQ) and once over the blocks of chosen
+//         tokens (dK, dV); they leave fp32 results per element, which small kernels convert and
+//         scatter to the caller's tensors;
+//   fp32  the SIMT kernels (32-row blocks), which write the caller's tensors directly.
+// Encoder rows outside the subset get zero dK, dV (cleared first).  Block slots are assigned
+// without a scan: document b owns the slots from start / rows_per_block + b on, unused slots stay
+// empty (r0 == r1).
 #include <cuda_bf16.h>
 
 #include "hdt_internal.cuh"
 
 namespace hdt {
 
-constexpr int XR = 32;      // rows per block (the 128-thread SIMT kernels take 32 rows per pass)
 constexpr int XC = 32;      // CTAs (contiguous chunks) per document in the selection kernels
 
 struct CrossLayout {
-    size_t cnt, cntc, cu_sel, sel, rngq, rngk, blocks_q, blocks_k, queue, delta, total;
-    int nbq, nbk;
-    size_t zero_bytes;      // cnt .. queue is cleared at the start of every call
+    size_t cnt, cntc, cu_sel, tokx, rngx, blocks_q, blocks_k, queue, delta, own[5], total;
+    int nbq, nbk, xr;
+    size_t zero_bytes;      // cnt .. tokx is cleared at the start of every call
 };
 
 static size_t al256c(size_t v) { return (v + 255) & ~size_t(255); }
 
-static CrossLayout cross_layout(int B, int T, int Tq, int H, int bwd) {
+// tc: bf16 on the tensor-core kernels (fp32 per-element results in the workspace)
+static CrossLayout cross_layout(int B, int T, int Tq, int H, int D, bool tc, int bwd) {
     CrossLayout L{};
-    L.nbq = Tq / XR + B + 1;
-    L.nbk = T / XR + B + 1;
+    L.xr = tc ? 128 : 32;
+    L.nbq = Tq / L.xr + B + 1;
+    L.nbk = T / L.xr + B + 1;
+    const size_t n = (size_t)Tq + T;
     size_t o = 0;
     L.cnt = o; o += al256c(sizeof(int) * (size_t)(B + 1));
     L.cntc = o; o += al256c(sizeof(int) * (size_t)(B + 1) * XC);
     L.cu_sel = o; o += al256c(sizeof(int) * (size_t)(B + 2));
     L.blocks_q = o; o += al256c(sizeof(int) * 5 * (size_t)L.nbq);
     L.blocks_k = o; o += al256c(sizeof(int) * 5 * (size_t)L.nbk);
+    L.tokx = o; o += al256c(sizeof(int) * max(n, (size_t)1));
     L.zero_bytes = o;
-    L.sel = o; o += al256c(sizeof(int) * (size_t)max(T, 1));
-    L.rngq = o; o += al256c(sizeof(int) * 2 * (size_t)max(Tq, 1));
-    L.rngk = o; o += al256c(sizeof(int) * 2 * (size_t)max(T, 1));
+    L.rngx = o; o += al256c(sizeof(int) * 2 * max(n, (size_t)1));
     L.queue = o; o += al256c(sizeof(int) * (size_t)max(L.nbq, L.nbk));
     L.delta = o; if (bwd) o += al256c(sizeof(float) * (size_t)H * max(Tq, 1));
+    if (tc) {
+        const size_t rq = sizeof(float) * (size_t)max(Tq, 1) * H, rk = sizeof(float) * (size_t)max(T, 1) * H;
+        if (!bwd) {
+            L.own[0] = o; o += al256c(rq * D);      // O
+            L.own[1] = o; o += al256c(rq);          // LSE
+        } else {
+            L.own[2] = o; o += al256c(rq * D);      // dQ
+            L.own[3] = o; o += al256c(rk * D);      // dK
+            L.own[4] = o; o += al256c(rk * D);      // dV
+        }
+    }
     L.total = o + 256;
     return L;
 }
@@ -104,12 +122,13 @@ __global__ void __launch_bounds__(1024) k_cross_scan(const int *__restrict__ cnt
     for (int i = t; i < nq; i += 1024) queue[i] = i;
 }
 
-// Chunk y of document b: its part of the ordered list of chosen tokens and of their row ranges,
-// and its share of the document's decoder-row key ranges and of the block records of both sides.
+// Chunk y of document b: its part of the ordered list of chosen tokens (elements KO + position, with
+// their row ranges) and its share of the document's decoder rows (elements = row numbers: token
+// map, key range) and of the block records of both sides.  xr = rows per block.
 __global__ void __launch_bounds__(256) k_cross_fill(const int8_t *__restrict__ level, const int32_t *__restrict__ cu_k,
                                                     const int32_t *__restrict__ cu_q, int level_mask,
-                                                    const int *__restrict__ cu_sel, const int *__restrict__ cntc, int *sel,
-                                                    int *rngq, int *rngk, int *blocks_q, int *blocks_k) {
+                                                    const int *__restrict__ cu_sel, const int *__restrict__ cntc, int KO,
+                                                    int xr, int *tokx, int *rngx, int *blocks_q, int *blocks_k) {
     __shared__ int s_w[8];
     __shared__ int s_carry;
     const int b = blockIdx.x, y = blockIdx.y, t = threadIdx.x, lane = t & 31, w = t >> 5;
@@ -131,10 +150,10 @@ __global__ void __launch_bounds__(256) k_cross_fill(const int8_t *__restrict__ l
         int before = s_carry;
         for (int j = 0; j < w; ++j) before += s_w[j];
         if (f) {
-            const int pos = s0 + before + v - 1;
-            sel[pos] = i;
-            rngk[2 * pos] = q0;
-            rngk[2 * pos + 1] = q1;
+            const int e = KO + s0 + before + v - 1;
+            tokx[e] = i;
+            rngx[2 * e] = q0;
+            rngx[2 * e + 1] = q1;
         }
         __syncthreads();
         if (t == 0) { int tot = 0; for (int j = 0; j < 8; ++j) tot += s_w[j]; s_carry += tot; }
@@ -142,22 +161,60 @@ __global__ void __launch_bounds__(256) k_cross_fill(const int8_t *__restrict__ l
     }
     // decoder rows and block records: spread over the document's chunks
     const int nt = XC * 256, gt = y * 256 + t;
-    for (int r = q0 + gt; r < q1; r += nt) { rngq[2 * r] = s0; rngq[2 * r + 1] = s1; }
+    for (int r = q0 + gt; r < q1; r += nt) { tokx[r] = r; rngx[2 * r] = KO + s0; rngx[2 * r + 1] = KO + s1; }
     const int live = (s1 > s0 && q1 > q0) ? 0 : HDT_BLK_EMPTY;
-    const int slot_q = q0 / XR + b, nbq = (q1 - q0 + XR - 1) / XR;
+    const int slot_q = q0 / xr + b, nbq = (q1 - q0 + xr - 1) / xr;
     for (int j = gt; j < nbq; j += nt) {
         int *rec = blocks_q + 5 * (size_t)(slot_q + j);
-        rec[0] = q0 + j * XR; rec[1] = min(q1, q0 + (j + 1) * XR); rec[2] = s0; rec[3] = s1; rec[4] = live;
+        rec[0] = q0 + j * xr; rec[1] = min(q1, q0 + (j + 1) * xr); rec[2] = KO + s0; rec[3] = KO + s1; rec[4] = live;
     }
-    const int slot_k = s0 / XR + b, nbk = (s1 - s0 + XR - 1) / XR;
+    const int slot_k = s0 / xr + b, nbk = (s1 - s0 + xr - 1) / xr;
     for (int j = gt; j < nbk; j += nt) {
         int *rec = blocks_k + 5 * (size_t)(slot_k + j);
-        rec[0] = s0 + j * XR; rec[1] = min(s1, s0 + (j + 1) * XR); rec[2] = q0; rec[3] = q1; rec[4] = live;
+        rec[0] = KO + s0 + j * xr; rec[1] = KO + min(s1, s0 + (j + 1) * xr); rec[2] = q0; rec[3] = q1; rec[4] = live;
     }
 }
 
+// fp32 per-element results [n, H, D] of the tensor-core kernels -> bf16 rows of the caller's tensor:
+// element e goes to row map[e] (e itself without a map); count: device counter of the elements, or
+// null for n.  One thread per 8 values.  lse_src [n, H] -> lse_dst [H, n_rows] on the side.
+template <int D>
+__global__ void k_cross_cvt(const float *__restrict__ src, __nv_bfloat16 *dst, const int *__restrict__ map, int n,
+                            const int *__restrict__ count, int H, const float *__restrict__ lse_src, float *lse_dst,
+                            int lse_rows) {
+    constexpr int G = D / 8;
+    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int m = count ? min(n, *count) : n;
+    const long long e = gid / ((long long)H * G);
+    if (e >= m) return;
+    const int h = (int)((gid / G) % H), g = (int)(gid % G);
+    const float4 *p = reinterpret_cast<const float4 *>(src + ((size_t)e * H + h) * D + 8 * g);
+    const float4 x = p[0], y = p[1];
+    const int row = map ? map[e] : (int)e;
+    uint4 out;
+    __nv_bfloat162 *o2 = reinterpret_cast<__nv_bfloat162 *>(&out);
+    o2[0] = __floats2bfloat162_rn(x.x, x.y); o2[1] = __floats2bfloat162_rn(x.z, x.w);
+    o2[2] = __floats2bfloat162_rn(y.x, y.y); o2[3] = __floats2bfloat162_rn(y.z, y.w);
+    *reinterpret_cast<uint4 *>(dst + ((size_t)row * H + h) * D + 8 * g) = out;
+    if (lse_src != nullptr && g == 0) lse_dst[(size_t)h * lse_rows + row] = lse_src[(size_t)e * H + h];
+}
+
+static int cross_cvt(const float *src, void *dst, const int *map, int n, const int *count, int H, int D,
+                     const float *lse_src, float *lse_dst, int lse_rows, cudaStream_t st) {
+    if (n == 0) return HDT_OK;
+    const long long threads = (long long)n * H * (D / 8);
+    const unsigned grid = (unsigned)((threads + 255) / 256);
+    if (D == 64) k_cross_cvt<64><<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, map, n, count, H, lse_src, lse_dst, lse_rows);
+    else k_cross_cvt<128><<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, map, n, count, H, lse_src, lse_dst, lse_rows);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+
 static int cross_build(const CrossLayout &L, char *ws, const int8_t *level, const int32_t *cu_k, const int32_t *cu_q,
-                       int B, int level_mask, cudaStream_t st) {
+                       int B, int Tq, int level_mask, cudaStream_t st) {
+    // the token map is cleared as a whole: tiles of the gathering kernels reach past the elements
+    // in use, and element 0 is a valid row of every tensor
     HDT_CUDA_CHECK(cudaMemsetAsync(ws, 0, L.zero_bytes, st));
     if (B > 0) {
         static_assert(XC == 32, "k_cross_fill sums the chunk counts with one lane per chunk");
@@ -165,9 +222,8 @@ static int cross_build(const CrossLayout &L, char *ws, const int8_t *level, cons
         k_cross_scan<<<1, 1024, 0, st>>>((const int *)(ws + L.cnt), B, (int *)(ws + L.cu_sel), (int *)(ws + L.queue),
                                          max(L.nbq, L.nbk));
         k_cross_fill<<<dim3(B, XC), 256, 0, st>>>(level, cu_k, cu_q, level_mask, (const int *)(ws + L.cu_sel),
-                                                  (const int *)(ws + L.cntc), (int *)(ws + L.sel),
-                                        (int *)(ws + L.rngq), (int *)(ws + L.rngk), (int *)(ws + L.blocks_q),
-                                        (int *)(ws + L.blocks_k));
+                                                  (const int *)(ws + L.cntc), Tq, L.xr, (int *)(ws + L.tokx),
+                                                  (int *)(ws + L.rngx), (int *)(ws + L.blocks_q), (int *)(ws + L.blocks_k));
         count_launch(3);
     }
     HDT_CUDA_CHECK(cudaGetLastError());
@@ -190,10 +246,13 @@ static int cross_check(const void *level, const void *cu_k, const void *cu_q, in
 
 using namespace hdt;
 
+static bool cross_tc(int dtype) { return dtype == HDT_BF16 && !g_force_simt; }
+
 extern "C" size_t hdt_cross_workspace_bytes(int32_t batch, int32_t total_tokens, int32_t total_q, int32_t heads,
-                                            int32_t bwd) {
-    if (batch < 0 || total_tokens < 0 || total_q < 0 || heads < 1) return 0;
-    return cross_layout(batch, total_tokens, total_q, heads, bwd).total;
+                                            int32_t head_dim, int32_t dtype, int32_t bwd) {
+    if (batch < 0 || total_tokens < 0 || total_q < 0 || heads < 1 || (head_dim != 64 && head_dim != 128)) return 0;
+    // sized for the tensor-core path whenever the dtype allows it (the larger of the two layouts)
+    return cross_layout(batch, total_tokens, total_q, heads, head_dim, dtype == HDT_BF16, bwd).total;
 }
 
 extern "C" int hdt_cross_attn_fwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q,
@@ -201,29 +260,36 @@ extern "C" int hdt_cross_attn_fwd(const int8_t *level, const int32_t *cu_seqlens
                                   const void *q, const void *k, const void *v, void *o, float *lse, int32_t heads,
                                   int32_t head_dim, int32_t dtype, float softmax_scale, void *workspace,
                                   size_t workspace_bytes, void *stream) {
-    const CrossLayout L = cross_layout(max(batch, 0), max(total_tokens, 0), max(total_q, 0), max(heads, 1), 0);
+    const size_t need = hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, head_dim, dtype, 0);
     int rc = cross_check(level, cu_seqlens_k, cu_seqlens_q, batch, total_tokens, total_q, heads, head_dim, dtype,
-                         level_mask, workspace, workspace_bytes, L.total, "hdt_cross_attn_fwd");
+                         level_mask, workspace, workspace_bytes, need, "hdt_cross_attn_fwd");
     if (rc) return rc;
     if (total_q == 0) return HDT_OK;
     if (!q || !o || !lse || (total_tokens > 0 && (!k || !v)))
         return set_error(HDT_ERR_INVALID_ARG, "hdt_cross_attn_fwd: null tensor pointer");
+    const bool tc = cross_tc(dtype);
+    const CrossLayout L = cross_layout(batch, total_tokens, total_q, heads, head_dim, tc, 0);
     cudaStream_t st = (cudaStream_t)stream;
     char *ws = (char *)workspace;
-    rc = cross_build(L, ws, level, cu_seqlens_k, cu_seqlens_q, batch, level_mask, st);
+    rc = cross_build(L, ws, level, cu_seqlens_k, cu_seqlens_q, batch, total_q, level_mask, st);
     if (rc) return rc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
     FwdStageArgs a{};
-    a.n = total_q; a.nb = L.nbq; a.H = heads; a.T = total_q;
-    a.tok = (const int *)(ws + L.sel);      // keys through the list of chosen tokens
-    a.tok_rows = nullptr;                   // decoder rows in place
-    a.rng = (const int *)(ws + L.rngq); a.blocks = (const int *)(ws + L.blocks_q);
+    a.n = total_q + total_tokens; a.nb = L.nbq; a.H = heads; a.T = total_q;
+    a.tok = (const int *)(ws + L.tokx);
+    a.tok_rows = a.tok;
+    a.rng = (const int *)(ws + L.rngx); a.blocks = (const int *)(ws + L.blocks_q);
     a.queue = (const int *)(ws + L.queue); a.queue_split = a.queue;
     a.q = q; a.k = k; a.v = v; a.o = o; a.lse = lse;
     a.scale_log2 = scale * 1.4426950408889634f;
     a.status = device_status_ptr();
-    a.block_rows = XR; a.dirs = 7;
-    return launch_fwd_simt(a, head_dim, dtype, st);
+    a.block_rows = L.xr; a.dirs = 7;
+    if (!tc) return launch_fwd_simt(a, head_dim, dtype, st);
+    a.own_o = (float *)(ws + L.own[0]);
+    a.own_lse = (float *)(ws + L.own[1]);
+    rc = launch_fwd_tc_upper(a, head_dim, st);
+    if (rc) return rc;
+    return cross_cvt(a.own_o, o, nullptr, total_q, nullptr, heads, head_dim, a.own_lse, lse, total_q, st);
 }
 
 extern "C" int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q,
@@ -232,9 +298,9 @@ extern "C" int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens
                                   const void *d_o, void *dq, void *dk, void *dv, int32_t heads, int32_t head_dim,
                                   int32_t dtype, float softmax_scale, void *workspace, size_t workspace_bytes,
                                   void *stream) {
-    const CrossLayout L = cross_layout(max(batch, 0), max(total_tokens, 0), max(total_q, 0), max(heads, 1), 1);
+    const size_t need = hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads, head_dim, dtype, 1);
     int rc = cross_check(level, cu_seqlens_k, cu_seqlens_q, batch, total_tokens, total_q, heads, head_dim, dtype,
-                         level_mask, workspace, workspace_bytes, L.total, "hdt_cross_attn_bwd");
+                         level_mask, workspace, workspace_bytes, need, "hdt_cross_attn_bwd");
     if (rc) return rc;
     cudaStream_t st = (cudaStream_t)stream;
     const size_t esz = dtype == HDT_BF16 ? 2 : 4;
@@ -247,32 +313,49 @@ extern "C" int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens
     if (total_q == 0) return HDT_OK;
     if (!q || !o || !lse || !d_o || !dq || (total_tokens > 0 && (!k || !v)))
         return set_error(HDT_ERR_INVALID_ARG, "hdt_cross_attn_bwd: null tensor pointer");
+    const bool tc = cross_tc(dtype);
+    const CrossLayout L = cross_layout(batch, total_tokens, total_q, heads, head_dim, tc, 1);
     char *ws = (char *)workspace;
-    rc = cross_build(L, ws, level, cu_seqlens_k, cu_seqlens_q, batch, level_mask, st);
+    rc = cross_build(L, ws, level, cu_seqlens_k, cu_seqlens_q, batch, total_q, level_mask, st);
     if (rc) return rc;
     float *delta = (float *)(ws + L.delta);
     rc = launch_delta(o, d_o, delta, total_q, heads, head_dim, dtype, st);
     if (rc) return rc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
+    const int KO = total_q;
     BwdStageArgs a{};
-    a.H = heads; a.T = total_q;
+    a.n = total_q + total_tokens; a.H = heads; a.T = total_q;
+    a.tok = (const int *)(ws + L.tokx); a.tok_rows = a.tok;
+    a.rng = (const int *)(ws + L.rngx);
     a.queue = (const int *)(ws + L.queue); a.queue_split = a.queue;
     a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = delta;
     a.scale = scale; a.scale_log2 = scale * 1.4426950408889634f;
     a.dq = dq; a.dk = dk; a.dv = dv;
     a.status = device_status_ptr();
-    a.block_rows = XR; a.dirs = 7;
-    // decoder rows as queries: dQ
-    BwdStageArgs aq = a;
-    aq.n = total_q; aq.nb = L.nbq; aq.phases = 1;
-    aq.tok = (const int *)(ws + L.sel); aq.tok_rows = nullptr;
-    aq.rng = (const int *)(ws + L.rngq); aq.blocks = (const int *)(ws + L.blocks_q);
-    rc = launch_bwd_simt(aq, head_dim, dtype, st);
+    a.block_rows = L.xr; a.dirs = 7;
+    a.gather_end_q = total_q;                       // Q, dO have total_q rows
+    a.gather_end_k = total_q + total_tokens;
+    BwdStageArgs aq = a, ak = a;
+    aq.nb = L.nbq; aq.phases = 1; aq.blocks = (const int *)(ws + L.blocks_q);   // decoder rows as queries: dQ
+    ak.nb = L.nbk; ak.phases = 2; ak.blocks = (const int *)(ws + L.blocks_k);   // chosen tokens as keys: dK, dV
+    if (!tc) {
+        rc = launch_bwd_simt(aq, head_dim, dtype, st);
+        if (rc) return rc;
+        return launch_bwd_simt(ak, head_dim, dtype, st);
+    }
+    float *own_dq = (float *)(ws + L.own[2]), *own_dk = (float *)(ws + L.own[3]), *own_dv = (float *)(ws + L.own[4]);
+    aq.own_dq = own_dq; aq.own_dk = own_dk; aq.own_dv = own_dv;           // only dQ is written (phases = 1)
+    // the chosen tokens are elements KO ..: their results land at position e - KO of the buffers
+    const size_t shift = (size_t)KO * heads * head_dim;
+    ak.own_dq = own_dq; ak.own_dk = own_dk - shift; ak.own_dv = own_dv - shift;
+    rc = launch_bwd_tc_upper(aq, head_dim, st);
     if (rc) return rc;
-    // chosen encoder rows as keys: dK, dV, scattered to their token rows
-    BwdStageArgs ak = a;
-    ak.n = total_tokens; ak.nb = L.nbk; ak.phases = 2;
-    ak.tok = nullptr; ak.tok_rows = (const int *)(ws + L.sel);
-    ak.rng = (const int *)(ws + L.rngk); ak.blocks = (const int *)(ws + L.blocks_k);
-    return launch_bwd_simt(ak, head_dim, dtype, st);
+    rc = launch_bwd_tc_upper(ak, head_dim, st);
+    if (rc) return rc;
+    rc = cross_cvt(own_dq, dq, nullptr, total_q, nullptr, heads, head_dim, nullptr, nullptr, 0, st);
+    if (rc) return rc;
+    const int *sel = (const int *)(ws + L.tokx) + KO, *ns = (const int *)(ws + L.cu_sel) + batch;
+    rc = cross_cvt(own_dk, dk, sel, total_tokens, ns, heads, head_dim, nullptr, nullptr, 0, st);
+    if (rc) return rc;
+    return cross_cvt(own_dv, dv, sel, total_tokens, ns, heads, head_dim, nullptr, nullptr, 0, st);
 }

@@ -70,6 +70,7 @@ struct ProfScope {
 struct Side { cudaStream_t s, s2; cudaEvent_t fork, join, join2; bool ready; };
 int get_side(Side **out);
 extern int g_no_overlap;   // option "no_overlap"
+extern int g_force_simt;   // option "force_simt"
 extern int g_no_graph;     // option "no_graph"
 
 // Direction bits inside a row range (paper, "Mathematical Reasoning Tasks": the ListOps attention
@@ -162,7 +163,8 @@ struct BwdStageArgs {
     int block_rows;                               // max rows of a block in this stage
     int dirs;                                     // direction bits kept (7 = full rule), see dir_ok
     const int *tok_rows;                          // SIMT kernel: token map of the block rows (nullptr: identity); `tok` maps the walked span
-    int phases;                                   // SIMT kernel: 0 = both, 1 = rows as queries only (dQ), 2 = rows as keys only (dK, dV)
+    int phases;                                   // 0 = both, 1 = rows as queries only (dQ), 2 = rows as keys only (dK, dV); SIMT and gathering kernels
+    int gather_end_q, gather_end_k;               // gathering kernel: elements at or beyond these read as zero rows on the Q/dO and the K/V side (0: n)
 };
 
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);

@@ -52,6 +52,17 @@ def test_cross_attention_small(mask, dtype):
     run(P, b, [70, 0, 33, 1, 129], mask, 2, 64, dtype, 3)           # a document without decoder rows, ragged blocks
 
 
+def test_cross_attention_bf16_on_the_simt_kernels_too():
+    import paper_2407_08330_b200 as P
+    b = gen.small_random_batch(63, n_seqs=3, max_len=300, K=(0, 20))
+    P.hdt_set_option("force_simt", 1)
+    try:
+        run(P, b, [40, 17, 130], SEC | SENT | TOK, 2, 64, "bf16", 8)
+    finally:
+        P.hdt_set_option("force_simt", 0)
+    run(P, b, [40, 17, 130], SEC | SENT | TOK, 2, 128, "bf16", 8)     # tensor-core path, head_dim 128, > 128 keys
+
+
 def test_cross_attention_edge_cases():
     import paper_2407_08330_b200 as P
     # a document whose subset is empty (only its root), PAD tails, head_dim 128
