@@ -245,6 +245,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-hpe", action="store_true")
+    ap.add_argument("--option", action="append", default=[], metavar="NAME=VALUE",
+                    help="library switch for A/B runs (hdt_set_option), e.g. no_persistent=4")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -271,6 +273,9 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    for kv in args.option:
+        name, _, val = kv.partition("=")
+        P.hdt_set_option(name, int(val))
     c = args.config
     cfg, b = workload(c)
     T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
@@ -481,6 +486,7 @@ def main():
         "config": {"workload": cfg.name, "description": cfg.description, "batch": b.batch, "total_tokens": T,
                    "real_tokens": real, "heads": H, "head_dim": d, "nnz_pairs_per_head": nnz,
                    "visited_pairs_per_head": visited, "stages": n_stages, "directions": args.directions,
+                   "options": args.option,
                    "step": "hdt_build_index + hdt_attn_fwd" + (" + hdt_attn_bwd" if cfg.backward else ""),
                    "l2": "flushed between timed steps (256 MiB write, untimed)", "parallelism": f"replicas x{world}"},
         "pct_bf16_peak": 100.0 * value / world / pk["bf16_tflops"],

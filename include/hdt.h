@@ -280,7 +280,7 @@ int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const i
  * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
  * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
  * general tensor-core kernels, = 2 the persistent forward kernel, = 3 the forward kernel with one CTA
- * per (block, head); "simt_upper" = 1 computes the stages above 0 of bf16 calls on the fp32 SIMT
+ * per (block, head), = 5 the looping backward kernel (the default at head_dim 128) at head_dim 64 too; "simt_upper" = 1 computes the stages above 0 of bf16 calls on the fp32 SIMT
  * kernels instead of the gathering tensor-core kernels; "no_overlap" = 1 runs the stages
  * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream;
  * "no_graph" = 1 makes hdt_build_index launch its kernels one by one instead of replaying a cached

@@ -379,6 +379,232 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
 }
 
 
+// ---------------------------------------------------------------------------------------------
+// Looping backward for SELF, non-EMPTY blocks at D = 128 (the persistent kernel below covers
+// D = 64): the fused pass of k_bwd_tc (S, dP; P, dS; dV, dK, dQ over the dead S / dP columns), but
+// the CTA stays resident (one per SM: 224 KB of shared memory, all of TMEM), walks the items
+// blockIdx.x, + gridDim.x, ... of queue_split x heads, and requests the four input tiles of the
+// next item as soon as the output MMAs of the current one have finished — the gradients are
+// staged in tiles of their own, so the loads fly while the CTA drains, stages and stores.
+// ---------------------------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ CUtensorMap tm_q,
+                                                        const __grid_constant__ CUtensorMap tm_k,
+                                                        const __grid_constant__ CUtensorMap tm_v,
+                                                        const __grid_constant__ CUtensorMap tm_do, const BwdStageArgs a) {
+    constexpr int NSUB = D / 64;
+    constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DV = 0, TM_DK = 128, TM_DQ = 256, TM_COLS = 512;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = sm, *sDO = sQ + NSUB * SUB, *sK = sDO + NSUB * SUB, *sV = sK + NSUB * SUB;
+    uint8_t *sP = sV + NSUB * SUB, *sDS = sP + 2 * SUB;     // P, dS; later staging of dQ, dK
+    uint8_t *sStg = sDS + 2 * SUB;                          // staging of dV
+    uint64_t *bar_in = (uint64_t *)(sStg + NSUB * SUB);
+    uint64_t *bar_mma = bar_in + 1;
+    uint32_t *slot = (uint32_t *)(bar_mma + 1);
+    volatile int *abort_flag = (volatile int *)(slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, hf = tid >> 7;
+    const int H = a.H, G = gridDim.x;
+    const float LOG2E = 1.4426950408889634f;
+    const int n_items = a.n_fused * H;
+
+    if (tid == 0) {
+        mbar_init(bar_in, 1);
+        mbar_init(bar_mma, 1);
+        *abort_flag = (*a.status != 0);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    bool ok = true;
+    uint32_t ph_mma = 0;
+
+    struct It { int valid, r0, r1, h; };
+    auto fetch = [&](int i) {
+        It x{0, 0, 0, 0};
+        if (i < n_items) {
+            const int *rec = a.blocks + 5 * (size_t)a.queue_split[i / H];
+            x.valid = 1; x.r0 = rec[0]; x.r1 = rec[1]; x.h = i % H;
+        }
+        return x;
+    };
+    auto issue_loads = [&](const It &d) {       // thread 0
+        mbar_expect_tx(bar_in, (uint32_t)(4 * NSUB) * SUB);
+        for (int s = 0; s < NSUB; ++s) {
+            tma_load_3d(sQ + s * SUB, &tm_q, 64 * s, d.h, d.r0, bar_in);
+            tma_load_3d(sDO + s * SUB, &tm_do, 64 * s, d.h, d.r0, bar_in);
+            tma_load_3d(sK + s * SUB, &tm_k, 64 * s, d.h, d.r0, bar_in);
+            tma_load_3d(sV + s * SUB, &tm_v, 64 * s, d.h, d.r0, bar_in);
+        }
+    };
+    struct RowStat { int lo, hi, up; float lse, dl; };
+    auto load_stat = [&](const It &d) {
+        RowStat r{0, 0, -1, 0.f, 0.f};
+        const int row = d.r0 + rl;
+        if (d.valid && row < d.r1) {
+            r.lo = a.rng[2 * row];
+            r.hi = a.rng[2 * row + 1];
+            r.lse = a.lse[(size_t)d.h * a.T + row];      // natural log; scaled where it is used
+            r.dl = a.delta[(size_t)d.h * a.T + row];
+            if (a.part_dq != nullptr) r.up = a.up[row];
+        }
+        return r;
+    };
+
+    if (!dead && n_items > 0) {
+        It d0 = fetch((int)blockIdx.x), d1 = fetch((int)blockIdx.x + G);
+        RowStat rc = load_stat(d0);
+        if (tid == 0 && d0.valid) issue_loads(d0);
+        for (int it = 0; d0.valid && !*abort_flag; ++it) {
+            const It d2 = fetch((int)blockIdx.x + (it + 2) * G);      // record two items ahead
+            const RowStat rn = load_stat(d1);                          // row statistics one item ahead
+            const int r0 = d0.r0, r1 = d0.r1, h = d0.h, nrows = r1 - r0;
+            const int Nc = (nrows + 15) & ~15;
+            ok = mbar_wait(bar_in, it & 1, abort_flag, WAIT_CYCLES) && ok;
+            if (tid == 0 && !*abort_flag) {
+                tc_fence_after();
+                const uint32_t idesc = idesc_bf16(Nc, false, false);
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
+                    mma_ss(tmem + TM_S, smem_desc(smem_u32(sQ) + off, 0, 1024), smem_desc(smem_u32(sK) + off, 0, 1024), idesc, kk > 0);
+                }
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
+                    mma_ss(tmem + TM_DP, smem_desc(smem_u32(sDO) + off, 0, 1024), smem_desc(smem_u32(sV) + off, 0, 1024), idesc, kk > 0);
+                }
+                mma_commit(bar_mma);
+            }
+            const bool inq = rl < nrows;
+            const float lse2 = rc.lse * LOG2E, dl = rc.dl;
+            const int jl = max(rc.lo - r0, 0), jh = min(rc.hi - r0, nrows);
+            const bool has = inq && jh > jl;
+            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            ph_mma ^= 1;
+            tc_fence_after();
+#pragma unroll
+            for (int sl = 0; sl < 2; ++sl) {
+                const int s0 = 64 * hf + 32 * sl;
+                if (s0 >= Nc) continue;      // same decision in the whole warp
+                const uint32_t km = has ? keep_mask<false>(s0, 32, jl, jh, 0, 0, false, false) : 0u;
+                const bool mine = km != 0u;
+                uint32_t pp[16], pd[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) { pp[j] = 0u; pd[j] = 0u; }
+                if (__any_sync(0xffffffffu, mine)) {
+                    uint32_t rs[32], rd[32];
+                    tmem_ld32(tmem + TM_S + lane_base + s0, rs);
+                    tmem_ld32(tmem + TM_DP + lane_base + s0, rd);
+                    tmem_wait_ld();
+                    if (mine) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            float p0 = 0.f, p1 = 0.f, e0 = 0.f, e1 = 0.f;
+                            if (km & (1u << j)) {
+                                p0 = exp2f(fmaf(__uint_as_float(rs[j]), a.scale_log2, -lse2));
+                                e0 = p0 * (__uint_as_float(rd[j]) - dl);
+                            }
+                            if (km & (2u << j)) {
+                                p1 = exp2f(fmaf(__uint_as_float(rs[j + 1]), a.scale_log2, -lse2));
+                                e1 = p1 * (__uint_as_float(rd[j + 1]) - dl);
+                            }
+                            pp[j >> 1] = pack_bf16(p0, p1);
+                            pd[j >> 1] = pack_bf16(e0, e1);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t off = hf * SUB + swz(rl, sl * 4 + c);
+                    *reinterpret_cast<uint4 *>(sP + off) = make_uint4(pp[4 * c], pp[4 * c + 1], pp[4 * c + 2], pp[4 * c + 3]);
+                    *reinterpret_cast<uint4 *>(sDS + off) = make_uint4(pd[4 * c], pd[4 * c + 1], pd[4 * c + 2], pd[4 * c + 3]);
+                }
+            }
+            fence_proxy_async_smem();
+            tc_fence_before();
+            __syncthreads();
+            if (tid == 0 && !*abort_flag) {
+                tc_fence_after();
+                const uint32_t idesc_kv = idesc_bf16(D, true, true);   // A = P^T / dS^T, B = dO / Q (both MN-major)
+                const uint32_t idesc_q = idesc_bf16(D, false, true);   // A = dS (K-major), B = K (MN-major)
+                for (int kk = 0; kk < Nc / 16; ++kk)
+                    mma_ss(tmem + TM_DV, smem_desc(smem_u32(sP) + kk * 2048, SUB, 1024), smem_desc(smem_u32(sDO) + kk * 2048, SUB, 1024),
+                           idesc_kv, kk > 0);
+                for (int kk = 0; kk < Nc / 16; ++kk)
+                    mma_ss(tmem + TM_DK, smem_desc(smem_u32(sDS) + kk * 2048, SUB, 1024), smem_desc(smem_u32(sQ) + kk * 2048, SUB, 1024),
+                           idesc_kv, kk > 0);
+                for (int kk = 0; kk < Nc / 16; ++kk)
+                    mma_ss(tmem + TM_DQ, smem_desc(smem_u32(sDS) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024),
+                           smem_desc(smem_u32(sK) + kk * 2048, SUB, 1024), idesc_q, kk > 0);
+                mma_commit(bar_mma);
+            }
+            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            ph_mma ^= 1;
+            tc_fence_after();
+            // the input tiles are free: the next item's loads fly during the drain and the stores
+            if (tid == 0 && d1.valid && !*abort_flag) issue_loads(d1);
+            // ---- drain: this thread's row, its half of the D columns of each gradient ----
+            {
+                const uint32_t cols[3] = {TM_DQ, TM_DK, TM_DV};
+                uint8_t *dsts[3] = {sP, sDS, sStg};
+                float *parts[3] = {a.part_dq, a.part_dk, a.part_dv};
+#pragma unroll
+                for (int t = 0; t < 3; ++t) {
+                    const float sc = (t == 2) ? 1.f : a.scale;
+                    float *part = (inq && rc.up >= 0) ? parts[t] + ((size_t)rc.up * H + h) * D : nullptr;
+#pragma unroll
+                    for (int sl = 0; sl < D / 64; ++sl) {
+                        const int c0 = hf * (D / 2) + 32 * sl;
+                        uint32_t r[32];
+                        tmem_ld32(tmem + cols[t] + lane_base + c0, r);
+                        tmem_wait_ld();
+                        uint32_t pk[16];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            const float x0 = __uint_as_float(r[j]) * sc, x1 = __uint_as_float(r[j + 1]) * sc;
+                            if (part != nullptr) *reinterpret_cast<float2 *>(part + c0 + j) = make_float2(x0, x1);
+                            pk[j >> 1] = pack_bf16(x0, x1);
+                        }
+                        uint8_t *d = dsts[t] + (c0 >> 6) * SUB;
+#pragma unroll
+                        for (int c = 0; c < 4; ++c)
+                            *reinterpret_cast<uint4 *>(d + swz(rl, ((c0 & 63) >> 3) + c)) =
+                                make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncthreads();
+            {
+                __nv_bfloat16 *g[3] = {(__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv};
+                const uint8_t *srcs[3] = {sP, sDS, sStg};
+#pragma unroll
+                for (int t = 0; t < 3; ++t)
+                    for (int idx = tid; idx < NSUB * 128 * 8; idx += 256) {
+                        const int u = idx >> 10, rem = idx & 1023, r = rem >> 3, c = rem & 7;
+                        if (r < nrows) {
+                            const uint4 v = *reinterpret_cast<const uint4 *>(srcs[t] + u * SUB + swz(r, c));
+                            *reinterpret_cast<uint4 *>(g[t] + ((size_t)(r0 + r) * H + h) * D + u * 64 + c * 8) = v;
+                        }
+                    }
+            }
+            __syncthreads();     // the staged tiles are read before the next item's P and dS overwrite them
+            d0 = d1; d1 = d2; rc = rn;
+        }
+    }
+    if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
 // Cycle counts per phase of k_bwd_tc_p, accumulated by thread 0 of CTA 0 (diagnostics).
 __device__ long long g_bwd_phase_cycles[16];
 #define HDT_STAMP(i)                                        \
@@ -778,7 +1004,7 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     b.rest_only = 0;
     int n_general = a.nb;
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
-    if (D == 64 && a.nb > 0 && !a.no_persistent) {
+    if (D == 64 && a.nb > 0 && !a.no_persistent) {   // (no_persistent == 5: the looping kernel below instead)
         // the persistent kernel takes everything: first the blocks of split families (longest first),
         // then the self-contained blocks
         constexpr int smem_p = 12 * SUB + 1024 + 64;
@@ -816,6 +1042,25 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
             HDT_CUDA_CHECK(cudaGetLastError());
         }
         n_general = 0;
+    }
+    if (((D == 128 && !a.no_persistent) || (D == 64 && a.no_persistent == 5)) && a.n_fused > 0 && !dirs) {
+        // self-contained blocks through the looping kernel, the rest through the general one
+        constexpr int smem_l = (4 * (D / 64) + 4 + (D / 64)) * SUB + 1024 + 64;
+        static bool attr_l = false;
+        static int n_sm_l = 0;
+        if (!attr_l) {
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_loop<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_l));
+            int dev = 0;
+            HDT_CUDA_CHECK(cudaGetDevice(&dev));
+            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm_l, cudaDevAttrMultiProcessorCount, dev));
+            attr_l = true;
+        }
+        const long long items = (long long)a.n_fused * a.H;
+        k_bwd_tc_loop<D><<<(int)(items < n_sm_l ? items : n_sm_l), 256, smem_l, st>>>(tq, tk, tv, tdo, a);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+        b.rest_only = 1;
+        n_general = a.nb - a.n_fused;
     }
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
