@@ -400,8 +400,8 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
     uint8_t *sP = sV + NSUB * SUB, *sDS = sP + 2 * SUB;     // P, dS; later staging of dQ, dK
     uint8_t *sStg = sDS + 2 * SUB;                          // staging of dV
     uint64_t *bar_in = (uint64_t *)(sStg + NSUB * SUB);
-    uint64_t *bar_mma = bar_in + 1;
-    uint32_t *slot = (uint32_t *)(bar_mma + 1);
+    uint64_t *bar_a = bar_in + 1, *bar_b = bar_in + 2;      // S and dP (two issuing threads); dV, dK, dQ (three)
+    uint32_t *slot = (uint32_t *)(bar_in + 3);
     volatile int *abort_flag = (volatile int *)(slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, hf = tid >> 7;
@@ -411,7 +411,8 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
 
     if (tid == 0) {
         mbar_init(bar_in, 1);
-        mbar_init(bar_mma, 1);
+        mbar_init(bar_a, 2);
+        mbar_init(bar_b, 3);
         *abort_flag = (*a.status != 0);
         fence_mbar_init();
     }
@@ -423,7 +424,8 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
     const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
     const bool dead = (*abort_flag != 0);
     bool ok = true;
-    uint32_t ph_mma = 0;
+    // MMAs are issued by lane 0 of warps 0, 1, 2 side by side (a thread needs about 100 cycles per MMA)
+    const bool issuer = ((tid & 31) == 0) && warp < 3;
 
     struct It { int valid, r0, r1, h; };
     auto fetch = [&](int i) {
@@ -467,27 +469,22 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
             const int r0 = d0.r0, r1 = d0.r1, h = d0.h, nrows = r1 - r0;
             const int Nc = (nrows + 15) & ~15;
             ok = mbar_wait(bar_in, it & 1, abort_flag, WAIT_CYCLES) && ok;
-            if (tid == 0 && !*abort_flag) {
+            if (issuer && warp < 2 && !*abort_flag) {      // warp 0: S = Q K^T, warp 1: dP = dO V^T
                 tc_fence_after();
                 const uint32_t idesc = idesc_bf16(Nc, false, false);
+                const uint32_t sa = smem_u32(warp == 0 ? sQ : sDO), sb = smem_u32(warp == 0 ? sK : sV);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
-                    mma_ss(tmem + TM_S, smem_desc(smem_u32(sQ) + off, 0, 1024), smem_desc(smem_u32(sK) + off, 0, 1024), idesc, kk > 0);
+                    mma_ss(tmem + (warp == 0 ? TM_S : TM_DP), smem_desc(sa + off, 0, 1024), smem_desc(sb + off, 0, 1024), idesc, kk > 0);
                 }
-#pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
-                    mma_ss(tmem + TM_DP, smem_desc(smem_u32(sDO) + off, 0, 1024), smem_desc(smem_u32(sV) + off, 0, 1024), idesc, kk > 0);
-                }
-                mma_commit(bar_mma);
+                mma_commit(bar_a);
             }
             const bool inq = rl < nrows;
             const float lse2 = rc.lse * LOG2E, dl = rc.dl;
             const int jl = max(rc.lo - r0, 0), jh = min(rc.hi - r0, nrows);
             const bool has = inq && jh > jl;
-            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
-            ph_mma ^= 1;
+            ok = mbar_wait(bar_a, it & 1, abort_flag, WAIT_CYCLES) && ok;
             tc_fence_after();
 #pragma unroll
             for (int sl = 0; sl < 2; ++sl) {
@@ -530,23 +527,26 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
             fence_proxy_async_smem();
             tc_fence_before();
             __syncthreads();
-            if (tid == 0 && !*abort_flag) {
+            if (issuer && !*abort_flag) {
                 tc_fence_after();
                 const uint32_t idesc_kv = idesc_bf16(D, true, true);   // A = P^T / dS^T, B = dO / Q (both MN-major)
                 const uint32_t idesc_q = idesc_bf16(D, false, true);   // A = dS (K-major), B = K (MN-major)
-                for (int kk = 0; kk < Nc / 16; ++kk)
-                    mma_ss(tmem + TM_DV, smem_desc(smem_u32(sP) + kk * 2048, SUB, 1024), smem_desc(smem_u32(sDO) + kk * 2048, SUB, 1024),
-                           idesc_kv, kk > 0);
-                for (int kk = 0; kk < Nc / 16; ++kk)
-                    mma_ss(tmem + TM_DK, smem_desc(smem_u32(sDS) + kk * 2048, SUB, 1024), smem_desc(smem_u32(sQ) + kk * 2048, SUB, 1024),
-                           idesc_kv, kk > 0);
-                for (int kk = 0; kk < Nc / 16; ++kk)
-                    mma_ss(tmem + TM_DQ, smem_desc(smem_u32(sDS) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024),
-                           smem_desc(smem_u32(sK) + kk * 2048, SUB, 1024), idesc_q, kk > 0);
-                mma_commit(bar_mma);
+                if (warp == 0) {
+                    for (int kk = 0; kk < Nc / 16; ++kk)
+                        mma_ss(tmem + TM_DV, smem_desc(smem_u32(sP) + kk * 2048, SUB, 1024),
+                               smem_desc(smem_u32(sDO) + kk * 2048, SUB, 1024), idesc_kv, kk > 0);
+                } else if (warp == 1) {
+                    for (int kk = 0; kk < Nc / 16; ++kk)
+                        mma_ss(tmem + TM_DK, smem_desc(smem_u32(sDS) + kk * 2048, SUB, 1024),
+                               smem_desc(smem_u32(sQ) + kk * 2048, SUB, 1024), idesc_kv, kk > 0);
+                } else {
+                    for (int kk = 0; kk < Nc / 16; ++kk)
+                        mma_ss(tmem + TM_DQ, smem_desc(smem_u32(sDS) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024),
+                               smem_desc(smem_u32(sK) + kk * 2048, SUB, 1024), idesc_q, kk > 0);
+                }
+                mma_commit(bar_b);
             }
-            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
-            ph_mma ^= 1;
+            ok = mbar_wait(bar_b, it & 1, abort_flag, WAIT_CYCLES) && ok;
             tc_fence_after();
             // the input tiles are free: the next item's loads fly during the drain and the stores
             if (tid == 0 && d1.valid && !*abort_flag) issue_loads(d1);
