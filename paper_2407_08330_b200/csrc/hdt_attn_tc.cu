@@ -74,15 +74,20 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                                                 const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
     constexpr int NSUB = D / 64;
     constexpr uint32_t TM_S = 0, TM_O = SINGLE ? 0 : 128, TM_COLS = SINGLE ? 128 : 256;
+    // PIPE: blocks that walk several key chunks with TMA loads keep two K tiles: K of chunk i + 1 is
+    // requested before S of chunk i is computed, V of chunk i + 1 as soon as P V of chunk i is done
+    constexpr bool PIPE = !SINGLE && !GATHER;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = sm;                       // NSUB sub-tiles; reused to stage O
     uint8_t *sK = sQ + NSUB * SUB;
     uint8_t *sV = sK + NSUB * SUB;
     uint8_t *sP = SINGLE ? sQ : sV + NSUB * SUB;   // 2 sub-tiles (128 keys)
-    uint64_t *bar_tma = (uint64_t *)((SINGLE ? sV + NSUB * SUB : sP + 2 * SUB));
+    uint8_t *sK1 = sP + 2 * SUB;            // PIPE only: the second K tile
+    uint64_t *bar_tma = (uint64_t *)((SINGLE ? sV + NSUB * SUB : sP + 2 * SUB + (PIPE ? NSUB * SUB : 0)));
     uint64_t *bar_mma = bar_tma + 1;
-    uint32_t *slot = (uint32_t *)(bar_mma + 1);
+    uint64_t *bar_k1 = bar_tma + 2, *bar_v = bar_tma + 3;   // PIPE only
+    uint32_t *slot = (uint32_t *)(bar_tma + 4);
     volatile int *abort_flag = (volatile int *)(slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5;
@@ -97,6 +102,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
     if (tid == 0) {
         mbar_init(bar_tma, 1);
         mbar_init(bar_mma, 1);
+        mbar_init(bar_k1, 1);
+        mbar_init(bar_v, 1);
         *abort_flag = (*a.status != 0);     // an earlier failure: do not wait for anything
         fence_mbar_init();
     }
@@ -133,6 +140,26 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                 gather_tiles<D, 128, 2>(dkv, skv, a.tok, c0, kb, H, h, tid);
                 fence_proxy_async_smem();     // generic-proxy writes, read by the MMA
                 __syncthreads();
+            } else if constexpr (PIPE) {
+                const int ci = (c0 - ka) >> 7;
+                if (tid == 0 && !*abort_flag) {   // after a failed wait nothing new is issued
+                    if (first) {
+                        mbar_expect_tx(bar_tma, (uint32_t)(2 * NSUB) * SUB);
+                        mbar_expect_tx(bar_v, (uint32_t)NSUB * SUB);
+                        for (int s = 0; s < NSUB; ++s) {
+                            tma_load_3d(sQ + s * SUB, &tm_q, 64 * s, h, r0, bar_tma);
+                            tma_load_3d(sK + s * SUB, &tm_k, 64 * s, h, c0, bar_tma);
+                            tma_load_3d(sV + s * SUB, &tm_v, 64 * s, h, c0, bar_v);
+                        }
+                    }
+                    if (c0 + 128 < kb) {          // K of the next chunk into the tile that S of the previous chunk has left
+                        uint64_t *bn = (ci & 1) ? bar_tma : bar_k1;
+                        uint8_t *kn = (ci & 1) ? sK : sK1;
+                        mbar_expect_tx(bn, (uint32_t)NSUB * SUB);
+                        for (int s = 0; s < NSUB; ++s) tma_load_3d(kn + s * SUB, &tm_k, 64 * s, h, c0 + 128, bn);
+                    }
+                }
+                ok = mbar_wait((ci & 1) ? bar_k1 : bar_tma, (ci >> 1) & 1, abort_flag, WAIT_CYCLES) && ok;
             } else {
                 if (tid == 0 && !*abort_flag) {   // after a failed wait nothing new is issued
                     mbar_expect_tx(bar_tma, (uint32_t)((first ? NSUB : 0) + 2 * NSUB) * SUB);
@@ -151,8 +178,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk / 4) * SUB + (kk % 4) * 32;
-                    mma_ss(tmem + TM_S, smem_desc(smem_u32(sQ) + off, 0, 1024), smem_desc(smem_u32(sK) + off, 0, 1024),
-                           idesc, kk > 0);
+                    const uint32_t kb_ = smem_u32((PIPE && (((c0 - ka) >> 7) & 1)) ? sK1 : sK);
+                    mma_ss(tmem + TM_S, smem_desc(smem_u32(sQ) + off, 0, 1024), smem_desc(kb_ + off, 0, 1024), idesc, kk > 0);
                 }
                 mma_commit(bar_mma);
             }
@@ -232,6 +259,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             }
             l = l * alpha + lsum;
             m = m_new;
+            if constexpr (PIPE) ok = mbar_wait(bar_v, ((c0 - ka) >> 7) & 1, abort_flag, WAIT_CYCLES) && ok;   // V of this chunk
             fence_proxy_async_smem();
             tc_fence_before();
             __syncthreads();
@@ -248,6 +276,12 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
             ph_mma ^= 1;
             tc_fence_after();
+            if constexpr (PIPE) {
+                if (tid == 0 && c0 + 128 < kb && !*abort_flag) {   // V of the next chunk: the tile is free now
+                    mbar_expect_tx(bar_v, (uint32_t)NSUB * SUB);
+                    for (int s = 0; s < NSUB; ++s) tma_load_3d(sV + s * SUB, &tm_v, 64 * s, h, c0 + 128, bar_v);
+                }
+            }
         }
     }
     if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
@@ -835,7 +869,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     if (rc) return rc;
     rc = make_tmap_bf16(&tv, a.v, D, a.H, a.T, 128);
     if (rc) return rc;
-    constexpr int smem = (3 * (D / 64) + 2) * SUB + 1024 + 64;
+    constexpr int smem = (4 * (D / 64) + 2) * SUB + 1024 + 64;     // general kernel: Q, two K tiles, V, P
     constexpr int smem_1 = 3 * (D / 64) * SUB + 1024 + 64;
     static bool attr = false;
     if (!attr) {
