@@ -366,24 +366,67 @@ def main():
         ho, hdq, hdk, hdv = (torch.empty_like(h_q).pin_memory() for _ in range(4))
         hlse = torch.empty((H, T), dtype=torch.float32).pin_memory()
 
-        def step_e2e():
-            level.copy_(h_level, non_blocking=True); parent.copy_(h_parent, non_blocking=True)
-            cu.copy_(h_cu, non_blocking=True)
-            q.copy_(h_q, non_blocking=True); k.copy_(h_k, non_blocking=True); v.copy_(h_v, non_blocking=True)
-            if cfg.backward:
-                do.copy_(h_do, non_blocking=True)
-            step()
-            ho.copy_(o, non_blocking=True); hlse.copy_(lse, non_blocking=True)
-            if cfg.backward:
-                hdq.copy_(dq, non_blocking=True); hdk.copy_(dk, non_blocking=True); hdv.copy_(dv, non_blocking=True)
+        # Two sets of device buffers and three streams: the copy-in of step i + 1 and the copy-out of
+        # step i - 1 run beside the compute of step i (PCIe carries both directions at once).  Every
+        # step still copies all of its inputs in and all of its results out inside the timed region.
+        cur = torch.cuda.current_stream()
+        s_in, s_out = torch.cuda.Stream(device=dev), torch.cuda.Stream(device=dev)
+        sets = [dict(level=level, parent=parent, cu=cu, q=q, k=k, v=v, do=do, o=o, lse=lse, dq=dq, dk=dk, dv=dv)]
+        sets.append({n: torch.empty_like(t_) for n, t_ in sets[0].items()})
+        ev_in = [torch.cuda.Event() for _ in range(2)]       # inputs of set j have arrived
+        ev_c = [torch.cuda.Event() for _ in range(2)]        # compute on set j is done
+        ev_out = [torch.cuda.Event() for _ in range(2)]      # results of set j have left
+        for e in ev_c + ev_out:
+            e.record(cur)
 
-        for _ in range(2):
-            step_e2e()
+        def copy_in(j):
+            S = sets[j]
+            s_in.wait_event(ev_c[j])                          # the step that last used set j is done with its inputs
+            with torch.cuda.stream(s_in):
+                S["level"].copy_(h_level, non_blocking=True); S["parent"].copy_(h_parent, non_blocking=True)
+                S["cu"].copy_(h_cu, non_blocking=True)
+                S["q"].copy_(h_q, non_blocking=True); S["k"].copy_(h_k, non_blocking=True); S["v"].copy_(h_v, non_blocking=True)
+                if cfg.backward:
+                    S["do"].copy_(h_do, non_blocking=True)
+                ev_in[j].record(s_in)
+
+        def compute(j):
+            S = sets[j]
+            cur.wait_event(ev_in[j])
+            cur.wait_event(ev_out[j])                         # the previous results of set j have been copied out
+            idx = P.hdt_build_index(S["level"], S["parent"], S["cu"], max_stages=max_st, workspace=ws_index,
+                                    directions=args.directions)
+            P.hdt_attn_fwd(idx, S["q"], S["k"], S["v"], out=S["o"], lse=S["lse"], workspace=ws_f)
+            if cfg.backward:
+                P.hdt_attn_bwd(idx, S["q"], S["k"], S["v"], S["o"], S["lse"], S["do"], dq=S["dq"], dk=S["dk"], dv=S["dv"],
+                               workspace=ws_b)
+            idx.close()
+            ev_c[j].record(cur)
+
+        def copy_out(j):
+            S = sets[j]
+            s_out.wait_event(ev_c[j])
+            with torch.cuda.stream(s_out):
+                ho.copy_(S["o"], non_blocking=True); hlse.copy_(S["lse"], non_blocking=True)
+                if cfg.backward:
+                    hdq.copy_(S["dq"], non_blocking=True); hdk.copy_(S["dk"], non_blocking=True)
+                    hdv.copy_(S["dv"], non_blocking=True)
+                ev_out[j].record(s_out)
+
+        def run_e2e(n):
+            copy_in(0)
+            for i in range(n):
+                if i + 1 < n:
+                    copy_in((i + 1) & 1)
+                compute(i & 1)
+                copy_out(i & 1)
+            s_out.synchronize()
+
+        run_e2e(3)
         barrier()
-        n_e = max(3, min(args.steps, 10))
+        n_e = max(4, min(args.steps, 10))
         w0 = time.perf_counter()
-        for _ in range(n_e):
-            step_e2e()
+        run_e2e(n_e)
         barrier()
         e_ms = (time.perf_counter() - w0) / n_e * 1e3
         e_ms = max_over_ranks(e_ms, dev)
@@ -392,7 +435,8 @@ def main():
         n_out = 1 + (3 if cfg.backward else 0)
         e2e = {"value": job_value(flops_per_step(nnz, H, d, cfg.backward), world, e_ms), "unit": "TFLOP/s",
                "h2d_bytes_per_step": n_in * T * H * d * esz + T * 5 + (b.batch + 1) * 4,
-               "d2h_bytes_per_step": n_out * T * H * d * esz + H * T * 4, "ms_per_step": e_ms}
+               "d2h_bytes_per_step": n_out * T * H * d * esz + H * T * 4, "ms_per_step": e_ms,
+               "pipeline": "copy-in of step i+1 and copy-out of step i-1 beside the compute of step i (two buffer sets)"}
 
     # the step before the path, timed alone on the same batch: hierarchical positional encoding
     # added to a resident [T, heads*head_dim] embedding (read + write of x, p-vectors from the index)
