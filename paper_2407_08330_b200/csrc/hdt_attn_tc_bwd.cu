@@ -627,7 +627,7 @@ __device__ long long g_bwd_phase_cycles[16];
 // ---------------------------------------------------------------------------------------------
 // Output tiles leave through TMA stores.  A block has 1..128 rows and a store box has a fixed
 // number of rows, so each gradient tensor gets seven maps with boxes of 64, 32, ..., 1 rows and a
-// tile is stored as the binary decomposition of its row count.
+// tile is stored as two (possibly overlapping) boxes of the largest size that fits.
 struct StoreMaps { CUtensorMap m[3][7]; };
 
 template <bool SPLIT, bool DIRS = false>
@@ -672,7 +672,8 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     // MMAs are issued by lane 0 of warps 0, 1, 2 in parallel: a single thread needs about 100 cycles
     // per small MMA (descriptor arithmetic), three chains issued side by side hide that
     const bool issuer = ((tid & 31) == 0) && warp < 3;
-    const bool store_thread = ((tid & 15) == 0) && tid < 384;   // 24 threads, one per (tensor, box slot)
+    // six store threads in six warps: (tensor, first / second box); the MMA-issuing warps 0..2 are left alone
+    const bool store_thread = ((tid & 31) == 0) && warp >= 4 && warp < 10;
 
     // ---- work stream of this CTA ----------------------------------------------------------------
     // A unit is a (block, head); this CTA takes units blockIdx.x, + gridDim.x, ... of its group of
@@ -955,16 +956,17 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                 HDT_STAMP(6);
                 __syncthreads();
                 HDT_STAMP(7);
-                // ---- TMA stores: rows [0, nrows) of each staged tile as boxes of 64, 64, 32, ..., 1 rows;
-                // 24 (tensor, box) slots, one per store thread ----
+                // ---- TMA stores: rows [0, nrows) of each staged tile as at most two boxes of b rows, b the
+                // largest power of two <= min(nrows, 64): [0, b) and [nrows - b, nrows).  Where the two
+                // overlap the same values are written twice.  (A TMA store request costs its thread and the
+                // TMA unit about 100 cycles: the binary decomposition of nrows took up to six per tensor.) ----
                 if (store_thread) {
-                    const int t = (tid >> 4) >> 3, slot = (tid >> 4) & 7;
-                    int rows, off, b;
-                    if (slot < 2) { b = 0; rows = 64; off = 64 * slot; }
-                    else { b = slot - 1; rows = 64 >> b; off = nrows & ~(2 * rows - 1); }
-                    bool use = (slot < 2) ? (nrows >= 64 * (slot + 1)) : ((nrows & rows) != 0);
-                    use = use && (flags & (t == 0 ? F_DQ : F_DKDV));
-                    if (use) tma_store_3d(&sm_out.m[t][b], 0, h, r0 + off, sP + t * STG + off * 128);
+                    const int t = (warp - 4) >> 1, second = (warp - 4) & 1;
+                    const int bx = max(__clz(nrows) - 25, 0);          // box of 64 >> bx rows: 64 for nrows >= 64
+                    const int b = 64 >> bx;
+                    const int off = second ? nrows - b : 0;
+                    const bool use = (flags & (t == 0 ? F_DQ : F_DKDV)) && (!second || nrows > b);
+                    if (use) tma_store_3d(&sm_out.m[t][bx], 0, h, r0 + off, sP + t * STG + off * 128);
                     bulk_commit();
                 }
             }
