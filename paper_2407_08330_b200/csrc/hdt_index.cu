@@ -410,53 +410,38 @@ __global__ void k_blocks(DevHeader *hdr, int s, int bm, int B, const int *__rest
 
 // Rank sort: queue[rank] = block id, cost descending, id ascending.  queue_split: the same order
 // inside two groups, blocks that are SELF and not EMPTY first (n_fused of them), then the others.
+// One warp per block: its lanes share the scan over all blocks and add up their counts.
 __global__ void __launch_bounds__(256)
 k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost, const int *__restrict__ blocks, int *queue,
         int *queue_split) {
-    // sort key of a block: (cost << 1 | eligible); tiles of keys go through shared memory
-    __shared__ long long s_key[1024];
     const int nb = hdr->st[s].nb;
-    const int ntile = (nb + 1023) / 1024;
+    const int lane = threadIdx.x & 31;
+    const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nw = (gridDim.x * blockDim.x) >> 5;
     int mine = 0;
-    for (int i0 = blockIdx.x * blockDim.x; i0 < nb; i0 += gridDim.x * blockDim.x) {   // same trip count in the CTA
-        const int i = i0 + threadIdx.x;
-        long long ci = 0;
-        int ei = 0;
-        if (i < nb) {
-            ci = cost[i];
-            const int fi = blocks[5 * i + 4];
-            ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
-        }
+    for (int i = gw; i < nb; i += nw) {
+        const long long ci = cost[i];
+        const int fi = blocks[5 * i + 4];
+        const int ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
         int rank = 0, rank2 = 0;
-        for (int tl = 0; tl < ntile; ++tl) {
-            __syncthreads();
-            for (int j = threadIdx.x; j < 1024; j += blockDim.x) {
-                const int jj = tl * 1024 + j;
-                if (jj < nb) {
-                    const int fj = blocks[5 * jj + 4];
-                    s_key[j] = (cost[jj] << 1) | (((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0);
-                }
-            }
-            __syncthreads();
-            const int lim = min(1024, nb - tl * 1024);
-            if (i < nb) {
-                for (int j = 0; j < lim; ++j) {
-                    const long long kj = s_key[j];
-                    const long long cj = kj >> 1;
-                    const int ej = (int)(kj & 1);
-                    const int before = (cj > ci) || (cj == ci && tl * 1024 + j < i);
-                    rank += before;
-                    rank2 += (ej > ei) || (ej == ei && before);
-                }
-            }
+        for (int j = lane; j < nb; j += 32) {
+            const long long cj = cost[j];
+            const int fj = blocks[5 * j + 4];
+            const int ej = ((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0;
+            const int before = (cj > ci) || (cj == ci && j < i);
+            rank += before;
+            rank2 += (ej > ei) || (ej == ei && before);
         }
-        if (i < nb) {
+        for (int o = 16; o; o >>= 1) {
+            rank += __shfl_xor_sync(0xffffffffu, rank, o);
+            rank2 += __shfl_xor_sync(0xffffffffu, rank2, o);
+        }
+        if (lane == 0) {
             queue[rank] = i;
             queue_split[rank2] = i;
             mine += ei;
         }
     }
-    if (mine) atomicAdd(&hdr->st[s].n_fused, mine);
+    if (lane == 0 && mine) atomicAdd(&hdr->st[s].n_fused, mine);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -473,9 +458,18 @@ struct UpperArgs {
 
 static constexpr int UT = 1024;      // threads of the fused kernel
 static constexpr int UMAXB = 1024;   // sequences it handles (per-sequence offsets live in shared memory)
+static constexpr int UCAP = 4096;    // elements of a stage whose scratch fits in shared memory
+static constexpr int USMEM = UCAP * (7 * 4 + 2);   // bytes of that scratch
 
 __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const UpperArgs u) {
-    __shared__ int s_off[UMAXB], s_base[UMAXB];
+    // Stages of at most UCAP elements keep their per-element scratch (parents, child counts, keep
+    // flags, prefix sums, ranges, next-stage indices) in shared memory: a dozen barrier-separated
+    // steps per stage would otherwise each pay a round trip to global memory.
+    extern __shared__ __align__(16) int s_dyn[];
+    int *s_par = s_dyn, *s_cnt = s_par + UCAP, *s_nlc = s_cnt + UCAP, *s_pre = s_nlc + UCAP, *s_up = s_pre + UCAP;
+    int *s_rng = s_up + UCAP;                                   // 2 * UCAP
+    uint8_t *s_keep = reinterpret_cast<uint8_t *>(s_rng + 2 * UCAP), *s_fpos = s_keep + UCAP;
+    __shared__ int s_off[UMAXB], s_base[UMAXB + 1], s_nbs[UMAXB], s_scu[UMAXB + 1];   // per sequence: block slots, first block, block count, offsets
     __shared__ int s_w[32];
     __shared__ int s_carry, s_flag;
     __shared__ long long s_ll[32];
@@ -487,32 +481,42 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         const StagePtrs P = u.st[s];
         const bool last = (s + 1 == u.max_stages);
         const StagePtrs N = u.st[last ? s : s + 1];
+        const bool small = n <= UCAP;
+        int *cnt = small ? s_cnt : u.cnt, *nlc = small ? s_nlc : u.nlc, *pre = small ? s_pre : u.pre;
+        uint8_t *keep = small ? s_keep : u.keep, *fpos = small ? s_fpos : u.fpos;
+        const int *par = small ? s_par : P.par;
+        const int *rngr = small ? s_rng : P.rng, *upr = small ? s_up : P.up;    // read-back of this stage's results
+        for (int b = t; b <= B; b += UT) s_scu[b] = P.scu[b];
+        if (small)
+            for (int e = t; e < n; e += UT) { s_par[e] = P.par[e]; s_cnt[e] = 0; s_nlc[e] = 0; }
+        __syncthreads();
         // children counts (cnt, nlc are zero for [0, n))
-        for (int e = t; e < n; e += UT) { const int p = P.par[e]; if (p >= 0) atomicAdd(&u.cnt[p], 1); }
+        for (int e = t; e < n; e += UT) { const int p = par[e]; if (p >= 0) atomicAdd(&cnt[p], 1); }
         if (t == 0) { s_flag = 0; s_carry = 0; }
         __syncthreads();
-        for (int e = t; e < n; e += UT) { const int p = P.par[e]; if (p >= 0 && u.cnt[e] > 0) atomicAdd(&u.nlc[p], 1); }
+        for (int e = t; e < n; e += UT) { const int p = par[e]; if (p >= 0 && cnt[e] > 0) atomicAdd(&nlc[p], 1); }
         __syncthreads();
         // ranges, keep flags
         long long deg = 0;
         for (int e = t; e < n; e += UT) {
-            const int p = P.par[e], c = u.cnt[e];
-            const bool head = (c > 0 && u.nlc[e] == 0);
+            const int p = par[e], c = cnt[e];
+            const bool head = (c > 0 && nlc[e] == 0);
             int lo = 0, hi = 0, fp = 0, kp = 1;
             if (head) {
                 lo = (p < 0) ? e : e + 1;
                 hi = e + 1 + c;
             } else if (p >= 0) {
-                const int cp = u.cnt[p];
-                if (cp > 0 && u.nlc[p] == 0) {
+                const int cp = cnt[p];
+                if (cp > 0 && nlc[p] == 0) {
                     if (!(p < e && e <= p + cp)) dev_fail(hdr, HDT_ERR_BAD_HIERARCHY, e);
                     lo = p; hi = p + 1 + cp; fp = min(e - p, 255); kp = 0;
                 }
             }
             P.rng[2 * e] = lo;
             P.rng[2 * e + 1] = hi;
-            u.keep[e] = (uint8_t)kp;
-            u.fpos[e] = (uint8_t)fp;
+            if (small) { s_rng[2 * e] = lo; s_rng[2 * e + 1] = hi; }
+            keep[e] = (uint8_t)kp;
+            fpos[e] = (uint8_t)fp;
             deg += row_pairs(e, lo, hi, u.dirs);
             if (kp && p >= 0) s_flag = 1;
         }
@@ -529,7 +533,7 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         // exclusive scan of keep[] in chunks of UT
         for (int base = 0; base < n; base += UT) {
             const int e = base + t;
-            const int kp = (e < n) ? u.keep[e] : 0;
+            const int kp = (e < n) ? keep[e] : 0;
             int v = kp;
             for (int o = 1; o < 32; o <<= 1) { const int x = __shfl_up_sync(0xffffffffu, v, o); if (lane >= o) v += x; }
             if (lane == 31) s_w[w] = v;
@@ -542,9 +546,10 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
             __syncthreads();
             const int excl = s_carry + (w ? s_w[w - 1] : 0) + v - kp;
             if (e < n) {
-                u.pre[e] = excl;
+                pre[e] = excl;
                 const int up = (kp && has_next) ? excl : -1;
                 P.up[e] = up;
+                if (small) s_up[e] = up;
                 if (up >= 0 && !last) N.tok[up] = P.tok[e];
             }
             __syncthreads();
@@ -556,31 +561,32 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         // next stage's parents and sequence offsets; clear cnt / nlc for it
         if (!last) {
             for (int e = t; e < n; e += UT) {
-                const int up = P.up[e];
-                if (up >= 0) { const int p = P.par[e]; N.par[up] = (p >= 0) ? u.pre[p] : -1; }
+                const int up = upr[e];
+                if (up >= 0) { const int p = par[e]; N.par[up] = (p >= 0) ? pre[p] : -1; }
             }
             for (int b = t; b <= B; b += UT) {
-                const int x = P.scu[b];
-                N.scu[b] = (n2 > 0) ? ((x < n) ? u.pre[x] : n2) : 0;
+                const int x = s_scu[b];
+                N.scu[b] = (n2 > 0) ? ((x < n) ? pre[x] : n2) : 0;
             }
         }
         __syncthreads();   // every cnt / nlc / pre read of this stage is done
-        for (int e = t; e < max(n2, 0); e += UT) { u.cnt[e] = 0; u.nlc[e] = 0; }
+        if (!small)
+            for (int e = t; e < max(n2, 0); e += UT) { u.cnt[e] = 0; u.nlc[e] = 0; }
         // per-sequence capacity offsets, greedy walk (one lane per sequence)
         for (int b = t; b < B; b += UT) {
             int off = 0;
-            for (int c = 0; c < b; ++c) off += 2 * ((P.scu[c + 1] - P.scu[c] + bm - 1) / bm) + 2;
+            for (int c = 0; c < b; ++c) off += 2 * ((s_scu[c + 1] - s_scu[c] + bm - 1) / bm) + 2;
             s_off[b] = off;
         }
         __syncthreads();
         for (int b = w; b < B; b += UT / 32) {
             if (lane == 0) {
-                const int s0 = P.scu[b], len = P.scu[b + 1] - s0, off = s_off[b];
+                const int s0 = s_scu[b], len = s_scu[b + 1] - s0, off = s_off[b];
                 int pos = 0, cntb = 0;
                 while (pos < len) {
                     int end = min(pos + bm, len);
                     if (end < len) {
-                        const int f = u.fpos[s0 + end];
+                        const int f = fpos[s0 + end];
                         if (f >= 1 && f < end - pos) end -= f;
                     }
                     u.bstart[off + cntb] = s0 + pos;
@@ -588,28 +594,34 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                     pos = end;
                 }
                 u.seqcount[b] = cntb;
+                s_nbs[b] = cntb;
             }
         }
         __syncthreads();
         for (int b = t; b < B; b += UT) {
             int base = 0;
-            for (int c = 0; c < b; ++c) base += u.seqcount[c];
+            for (int c = 0; c < b; ++c) base += s_nbs[c];
             s_base[b] = base;
-            if (b == B - 1) hdr->st[s].nb = base + u.seqcount[b];
+            if (b == B - 1) { hdr->st[s].nb = base + s_nbs[b]; s_base[B] = base + s_nbs[b]; }
         }
         __syncthreads();
-        // block records, one warp per block
+        // block records, one warp per block over all sequences (the block's sequence by bisection of s_base)
         long long vis = 0;
-        for (int b = 0; b < B; ++b) {
-            const int nb_seq = u.seqcount[b], off = s_off[b], base = s_base[b], s1 = P.scu[b + 1];
-            for (int i = w; i < nb_seq; i += UT / 32) {
+        {
+            const int nb_all = (B > 0) ? s_base[B] : 0;
+            for (int gb = w; gb < nb_all; gb += UT / 32) {
+                int lo_b = 0, hi_b = B;
+                while (hi_b - lo_b > 1) { const int mid = (lo_b + hi_b) >> 1; if (s_base[mid] <= gb) lo_b = mid; else hi_b = mid; }
+                // (the largest b with s_base[b] <= gb always owns blocks: an empty sequence has the base of its successor)
+                const int b = lo_b, i = gb - s_base[b];
+                const int nb_seq = s_nbs[b], off = s_off[b], base = s_base[b], s1 = s_scu[b + 1];
                 const int r0 = u.bstart[off + i];
                 const int r1 = (i + 1 < nb_seq) ? u.bstart[off + i + 1] : s1;
                 int a = 0x7fffffff, bb = (int)0x80000000, carry = 0;
                 for (int e = r0 + lane; e < r1; e += 32) {
-                    const int lo = P.rng[2 * e], hi = P.rng[2 * e + 1];
+                    const int lo = rngr[2 * e], hi = rngr[2 * e + 1];
                     if (hi > lo) { a = min(a, lo); bb = max(bb, hi); }
-                    if (P.up[e] >= 0) carry = 1;
+                    if (upr[e] >= 0) carry = 1;
                 }
                 for (int o = 16; o; o >>= 1) {
                     a = min(a, __shfl_xor_sync(0xffffffffu, a, o));
@@ -620,7 +632,7 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                 if (!any) { a = r0; bb = r0; }
                 int dense = 1;
                 for (int e = r0 + lane; e < r1; e += 32)
-                    if (P.rng[2 * e] != a || P.rng[2 * e + 1] != bb) dense = 0;
+                    if (rngr[2 * e] != a || rngr[2 * e + 1] != bb) dense = 0;
                 for (int o = 16; o; o >>= 1) dense &= __shfl_xor_sync(0xffffffffu, dense, o);
                 if (lane == 0) {
                     int fl = 0;
@@ -639,14 +651,14 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         if (lane == 0 && vis) atomicAdd((unsigned long long *)&hdr->visited, (unsigned long long)vis);
         __syncthreads();
         // queues
-        const int nb = (B > 0) ? s_base[B - 1] + u.seqcount[B - 1] : 0;
+        const int nb = (B > 0) ? s_base[B] : 0;
         int mine = 0;
-        for (int i = t; i < nb; i += UT) {
+        for (int i = w; i < nb; i += UT / 32) {      // one warp per block, lanes share the scan
             const long long ci = u.cost[i];
             const int fi = P.blocks[5 * i + 4];
             const int ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
             int rank = 0, rank2 = 0;
-            for (int j = 0; j < nb; ++j) {
+            for (int j = lane; j < nb; j += 32) {
                 const long long cj = u.cost[j];
                 const int fj = P.blocks[5 * j + 4];
                 const int ej = ((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0;
@@ -654,9 +666,15 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                 rank += before;
                 rank2 += (ej > ei) || (ej == ei && before);
             }
-            P.queue[rank] = i;
-            P.queue_split[rank2] = i;
-            mine += ei;
+            for (int o = 16; o; o >>= 1) {
+                rank += __shfl_xor_sync(0xffffffffu, rank, o);
+                rank2 += __shfl_xor_sync(0xffffffffu, rank2, o);
+            }
+            if (lane == 0) {
+                P.queue[rank] = i;
+                P.queue_split[rank2] = i;
+                mine += ei;
+            }
         }
         if (mine) atomicAdd(&hdr->st[s].n_fused, mine);
         __syncthreads();   // hdr->st[s+1].n and everything else is visible before the next stage reads it
@@ -740,6 +758,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     const int g_stride = max(1, min((T + 255) / 256, 148 * 8));
     static const int kSmemCap = 200 * 1024;
     HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
+    HDT_BUILD_CHECK(cudaFuncSetAttribute(k_upper_stages, cudaFuncAttributeMaxDynamicSharedMemorySize, USMEM));
     // One CTA builds all stages above 0 when they are small (documents: a few percent of the
     // tokens, up to 3-4 stages).  A caller that allows many stages expects deep trees, whose upper
     // stages hold most of the elements: those go through the per-stage kernels.
@@ -767,7 +786,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.keep = keep;
             u.bstart = (int *)(ws + L.bstart2); u.seqcount = (int *)(ws + L.seqcount2);
             u.fpos = (uint8_t *)(ws + L.fpos2); u.cost = (long long *)(ws + L.cost2);
-            k_upper_stages<<<1, UT, 0, s_>>>(hdr, u);
+            k_upper_stages<<<1, UT, USMEM, s_>>>(hdr, u);
             ++n_launched;
         };
         for (int s = 0; s < ms; ++s) {
@@ -804,7 +823,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
                 k_walk<<<B, 256, kSmemCap, st>>>(hdr, s, bms, P.scu, fpos, bstart, seqcount, maxlen_smem);
                 const int gy = max(1, min(64, 2048 / max(B, 1)));   // enough CTAs to spread a few long sequences
                 k_blocks<<<dim3(B, gy), 256, 0, st>>>(hdr, s, bms, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost);
-                k_queue<<<max(1, min(L.capnb / 256 + 1, 148 * 4)), 256, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
+                k_queue<<<max(1, min(L.capnb / 8 + 1, 148 * 4)), 256, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
                 n_launched += 3;
             }
         }
