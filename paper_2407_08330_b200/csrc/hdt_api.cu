@@ -244,7 +244,13 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
-        const bool two = ix->n_stages > 2;
+        const bool tc0 = dtype == HDT_BF16 && !g_force_simt;
+        // Stage 0's blocks that are not self-contained (split families, EMPTY blocks) have a kernel of
+        // their own.  Where the split families are the smaller part it runs on the second side stream beside the
+        // looping kernel (measured: a batch of padded documents gains 7 %); where split families
+        // dominate, one kernel after the other is faster (the skewed batch loses 3 % side by side).
+        const bool rest_beside = tc0 && 2 * (ix->desc[0].nb - ix->desc[0].n_fused - ix->desc[0].n_empty) <= ix->desc[0].nb;
+        const bool two = ix->n_stages > 2 || rest_beside;
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
         // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
         // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
@@ -263,13 +269,20 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
             else rc = launch_fwd_simt(a, head_dim, dtype, ss);
             if (rc) return rc;
         }
+        if (rest_beside) {
+            FwdStageArgs a = stage_args(0);
+            a.part = 2;
+            rc = launch_fwd_tc(a, head_dim, sd->s2);      // behind the (small) even stages, not behind stage 1
+            if (rc) return rc;
+        }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
         if (two) HDT_CUDA_CHECK(cudaEventRecord(sd->join2, sd->s2));
         {   // stage 0 after the small side kernels are queued: they take their SM share first (the
             // stage-0 kernel would otherwise fill every SM and push them behind itself)
             FwdStageArgs a = stage_args(0);
+            a.part = rest_beside ? 1 : 0;
             ProfScope ps(PROF_FWD_STAGE0, st);
-            if (dtype == HDT_BF16 && !g_force_simt) rc = launch_fwd_tc(a, head_dim, st);
+            if (tc0) rc = launch_fwd_tc(a, head_dim, st);
             else rc = launch_fwd_simt(a, head_dim, dtype, st);
             if (rc) return rc;
         }

@@ -886,7 +886,11 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     b.rest_only = 0;
     int n_general = a.nb;
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
-    if (a.n_fused > 0 && a.no_persistent != 1) {
+    const bool split_launch = a.no_persistent != 1;     // two kernels: self-contained blocks, the others
+    if (a.n_fused > 0 && split_launch && a.part == 2) {  // the caller launches the looping kernel separately
+        b.rest_only = 1;
+        n_general = a.nb - a.n_fused;
+    } else if (a.n_fused > 0 && split_launch) {
         if (D == 64 && a.no_persistent == 2 && !dirs) {   // option: the persistent single-CTA-per-SM kernel
             constexpr int smem_p = 8 * SUB + 4 * 128 * 4 + 1024 + 64;
             int dev = 0, n_sm = 0;
@@ -910,6 +914,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         b.rest_only = 1;
         n_general = a.nb - a.n_fused;
     }
+    if (a.part == 1 && split_launch) n_general = 0;     // the caller launches the other blocks separately
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
         if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);

@@ -417,7 +417,7 @@ k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost, const int *__
     const int nb = hdr->st[s].nb;
     const int lane = threadIdx.x & 31;
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nw = (gridDim.x * blockDim.x) >> 5;
-    int mine = 0;
+    int mine = 0, mine_empty = 0;
     for (int i = gw; i < nb; i += nw) {
         const long long ci = cost[i];
         const int fi = blocks[5 * i + 4];
@@ -439,9 +439,11 @@ k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost, const int *__
             queue[rank] = i;
             queue_split[rank2] = i;
             mine += ei;
+            mine_empty += (fi & HDT_BLK_EMPTY) ? 1 : 0;
         }
     }
     if (lane == 0 && mine) atomicAdd(&hdr->st[s].n_fused, mine);
+    if (lane == 0 && mine_empty) atomicAdd(&hdr->st[s].n_empty, mine_empty);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -652,7 +654,7 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         __syncthreads();
         // queues
         const int nb = (B > 0) ? s_base[B] : 0;
-        int mine = 0;
+        int mine = 0, mine_empty = 0;
         for (int i = w; i < nb; i += UT / 32) {      // one warp per block, lanes share the scan
             const long long ci = u.cost[i];
             const int fi = P.blocks[5 * i + 4];
@@ -674,9 +676,11 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                 P.queue[rank] = i;
                 P.queue_split[rank2] = i;
                 mine += ei;
+                mine_empty += (fi & HDT_BLK_EMPTY) ? 1 : 0;
             }
         }
         if (mine) atomicAdd(&hdr->st[s].n_fused, mine);
+        if (mine_empty) atomicAdd(&hdr->st[s].n_empty, mine_empty);
         __syncthreads();   // hdr->st[s+1].n and everything else is visible before the next stage reads it
     }
 }
@@ -836,10 +840,11 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         // The build is a dozen tiny kernels: launching them one by one is slower than running them.
         // They are captured once into a CUDA graph, which is replayed while the same buffers, sizes
         // and parameters come back (one cached graph per host thread).
-        struct GraphKey { const void *a, *b, *c, *w; int B, T, bm, ms, bmu, ov, dirs; };
+        struct GraphKey { const void *a, *b, *c, *w; int B, T, bm, ms, bmu, ov, dirs, pad; };   // no padding bytes: compared with memcmp
         struct GraphCache { GraphKey key; cudaGraphExec_t exec; int launches; bool valid; };
         static thread_local GraphCache cache{};
-        const GraphKey key{level, parent, cu_seqlens, workspace, B, T, bm, ms, bmu, sd ? 1 : 0, dirs};
+        const GraphKey key{level, parent, cu_seqlens, workspace, B, T, bm, ms, bmu, sd ? 1 : 0, dirs, 0};
+        static_assert(sizeof(GraphKey) == 4 * sizeof(void *) + 8 * sizeof(int), "GraphKey must not contain padding");
         bool done = false;
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         // (the legacy and per-thread default streams cannot be captured)

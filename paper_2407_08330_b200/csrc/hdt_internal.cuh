@@ -14,6 +14,7 @@ struct StageDesc {
     int nb;        // row blocks
     int has_next;  // a later stage exists
     int n_fused;   // blocks that are SELF and not EMPTY (first n_fused entries of queue_split)
+    int n_empty;   // EMPTY blocks (rows without any key in this stage: PAD, lone roots)
 };
 
 struct DevHeader {
@@ -141,6 +142,7 @@ struct FwdStageArgs {
     int block_rows;     // max rows of a block in this stage
     int dirs;           // direction bits kept (7 = full rule), see dir_ok
     const int *tok_rows;  // SIMT kernels: token map of the block rows (nullptr: identity); `tok` maps the keys
+    int part;             // launch_fwd_tc: 0 = all blocks, 1 = only the self-contained ones (looping kernel), 2 = only the others
 };
 
 struct BwdStageArgs {
