@@ -877,8 +877,19 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     // a copy to pageable memory would be staged by the driver
     static thread_local DevHeader *h_pinned = nullptr;
     if (!h_pinned) HDT_BUILD_CHECK(cudaMallocHost((void **)&h_pinned, sizeof(DevHeader)));
+    // The host watches the copy land instead of waiting in the driver: first and last word of the
+    // pinned buffer are set to a value the device never writes (status is 0 or negative, tail is 0)
+    // and polled; the copy is the last operation of the build on the stream, and its words arrive
+    // in order.  After a bounded number of polls the ordinary wait takes over.
+    const int kUnset = 0x7fffffff;
+    volatile int *p_status = &h_pinned->status, *p_tail = &h_pinned->tail;
+    *p_status = kUnset;
+    *p_tail = kUnset;
     HDT_BUILD_CHECK(cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, st));
-    HDT_BUILD_CHECK(cudaStreamSynchronize(st));
+    bool landed = false;
+    for (long long spin = 0; spin < 20000000LL && !landed; ++spin) landed = (*p_tail != kUnset && *p_status != kUnset);
+    if (!landed) HDT_BUILD_CHECK(cudaStreamSynchronize(st));
+    std::atomic_thread_fence(std::memory_order_acquire);
     const DevHeader h = *h_pinned;
 #undef HDT_BUILD_CHECK
     if (h.status != 0) {

@@ -23,6 +23,7 @@ struct DevHeader {
     long long nnz;           // unmasked pairs
     long long visited;       // sum over blocks of rows x span
     StageDesc st[HDT_MAX_STAGES + 1];
+    int tail;                // always 0 on the device: the last word of the header to arrive on the host
 };
 
 // Host-side pointers to one stage's arrays inside the workspace.
