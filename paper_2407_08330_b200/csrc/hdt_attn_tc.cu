@@ -901,9 +901,12 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         } else if (a.no_persistent == 3 && !dirs) {       // option: one CTA per (block, head), no loop
             k_fwd_tc<D, true><<<dim3(a.n_fused, a.H), 128, smem_1, st>>>(tq, tk, tv, a);
         } else {
-            int dev = 0, n_sm = 0;
-            HDT_CUDA_CHECK(cudaGetDevice(&dev));
-            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+            static int n_sm = 0;      // once per process (one process per GPU)
+            if (n_sm == 0) {
+                int dev = 0;
+                HDT_CUDA_CHECK(cudaGetDevice(&dev));
+                HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+            }
             const long long items = (long long)a.n_fused * a.H;
             const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
             if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);

@@ -761,8 +761,12 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     const int g_chunk = max(1, (T + CHUNK - 1) / CHUNK);
     const int g_stride = max(1, min((T + 255) / 256, 148 * 8));
     static const int kSmemCap = 200 * 1024;
-    HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
-    HDT_BUILD_CHECK(cudaFuncSetAttribute(k_upper_stages, cudaFuncAttributeMaxDynamicSharedMemorySize, USMEM));
+    static bool attr_done = false;     // once per process (one process per GPU)
+    if (!attr_done) {
+        HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
+        HDT_BUILD_CHECK(cudaFuncSetAttribute(k_upper_stages, cudaFuncAttributeMaxDynamicSharedMemorySize, USMEM));
+        attr_done = true;
+    }
     // One CTA builds all stages above 0 when they are small (documents: a few percent of the
     // tokens, up to 3-4 stages).  A caller that allows many stages expects deep trees, whose upper
     // stages hold most of the elements: those go through the per-stage kernels.
