@@ -506,8 +506,11 @@ def main():
     value = job_value(fl, world, ms)
     real = b.real_tokens
     esz = 2 if cfg.dtype == "bf16" else 4
+    # backward stage 0: q, k, v, dO in, dq, dk, dv out, lse and delta; without a delta pass (the
+    # kernel computes dO . O itself) it reads o instead of delta
+    fused_delta = cfg.backward and "k_delta" not in kern
     alg_bytes = {"k_fwd_stage0": (4 * d * esz + 4) * real * H,
-                 "k_bwd_stage0": (7 * d * esz + 8) * real * H,
+                 "k_bwd_stage0": ((8 * d * esz + 4) if fused_delta else (7 * d * esz + 8)) * real * H,
                  "k_delta": (2 * d * esz + 4) * real * H}
     dom = max((kk for kk in kern if kk in alg_bytes), key=lambda kk: kern[kk]["ms_per_step"], default=None)
     roofline = None

@@ -318,6 +318,13 @@ int hdt_debug_bwd_phase_cycles(int64_t *out16);
  * barriers (max exchange), P arithmetic and stores, barrier, MMA issue, wait for O, drain, loop top,
  * barrier, output stores; out16[12] = items processed. */
 int hdt_debug_fwd_phase_cycles(int64_t *out16);
+/* With option "phase_stamps" = 1 the transposed looping backward (head_dim 64) runs an instrumented
+ * instantiation: hdt_debug_bwd_phase_cycles then reports its phases (out16[0..11]: loop top, wait for
+ * the input tiles, issue of S^T/dP^T, wait for them, P^T/dS^T arithmetic, barrier, issue of the output
+ * MMAs, prefetch and wait for dV/dK/dQ, drain, barrier, store requests, loop end), and
+ * hdt_debug_bwd_timeline the last such launch per CTA (up to 512): out2048[4 c + 0..3] = global timer
+ * (ns) at entry, when the first input tiles had arrived, at the end of the item loop, and the SM. */
+int hdt_debug_bwd_timeline(int64_t *out2048);
 
 #ifdef __cplusplus
 }

@@ -66,6 +66,8 @@ int *device_status_ptr() {
 static thread_local Side g_side[64];
 int g_no_overlap = 0;
 int g_no_graph = 0;
+int g_phase_stamps = 0;
+static int g_no_fused_delta = 0;
 
 int get_side(Side **out) {
     int dev = -1;
@@ -138,6 +140,8 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "simt_upper") == 0) { g_simt_upper = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_overlap") == 0) { g_no_overlap = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_graph") == 0) { g_no_graph = value; return HDT_OK; }
+    if (name && std::strcmp(name, "phase_stamps") == 0) { g_phase_stamps = value; return HDT_OK; }
+    if (name && std::strcmp(name, "no_fused_delta") == 0) { g_no_fused_delta = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 
@@ -326,7 +330,18 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     float *delta = (float *)(ws + L.delta);
     int *status = device_status_ptr();
     if (!status) return HDT_ERR_CUDA;
-    {
+    const bool overlap = ix->n_stages > 1 && !g_no_overlap;
+    // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
+    // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
+    // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
+    const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3 && ix->directions == 7;
+    // No delta pass when every kernel of this call computes dO . O of its rows itself: stage 0
+    // entirely on the transposed looping kernel (head_dim 64, every block self-contained), the
+    // stages above it on the gathering tensor-core kernels.
+    const bool fused_delta = dtype == HDT_BF16 && !g_force_simt && head_dim == 64 && g_no_persistent == 0 &&
+                             !g_no_fused_delta && ix->directions == 7 && ix->desc[0].n_fused == ix->desc[0].nb &&
+                             ix->desc[0].nb > 0 && (ix->n_stages == 1 || (overlap && tc_upper));
+    if (!fused_delta) {
         ProfScope ps(PROF_DELTA, st);
         rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
     }
@@ -339,7 +354,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
         a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
         a.block_rows = s ? ix->block_m_upper : ix->block_m;
-        a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = delta;
+        a.q = q; a.k = k; a.v = v; a.d_o = d_o; a.lse = lse; a.delta = fused_delta ? nullptr : delta; a.o = o;
         a.scale = scale;
         a.scale_log2 = scale * 1.4426950408889634f;
         if (s > 0) {
@@ -359,7 +374,6 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.tok_rows = a.tok;
         return a;
     };
-    const bool overlap = ix->n_stages > 1 && !g_no_overlap;
     if (overlap) {   // delta is ready: the upper stages' own gradients are computed beside stage 0
         Side *sd = nullptr;
         rc = get_side(&sd);
@@ -368,10 +382,6 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
         const bool two = ix->n_stages > 2;
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
-        // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
-        // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
-        // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
-        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3 && ix->directions == 7;
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 3;
         c.tok1 = ix->st[1].tok;

@@ -149,7 +149,21 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
             if (hi > lo) {
                 const int tk = GATHER ? a.tok[e] : e;
                 lse2 = a.lse[(size_t)h * a.T + tk] * LOG2E;
-                dl = a.delta[(size_t)h * a.T + tk];
+                if (a.delta != nullptr) dl = a.delta[(size_t)h * a.T + tk];
+                else {      // no delta pass ran: dO . O of the row, here
+                    const uint4 *po = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.o) + ((size_t)tk * H + h) * D);
+                    const uint4 *pg = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.d_o) + ((size_t)tk * H + h) * D);
+#pragma unroll
+                    for (int c = 0; c < D / 8; ++c) {
+                        const uint4 x = po[c], y = pg[c];
+                        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
+#pragma unroll
+                        for (int w = 0; w < 4; ++w) {
+                            dl = fmaf(__uint_as_float(xs[w] << 16), __uint_as_float(ys[w] << 16), dl);
+                            dl = fmaf(__uint_as_float(xs[w] & 0xffff0000u), __uint_as_float(ys[w] & 0xffff0000u), dl);
+                        }
+                    }
+                }
             }
         }
         const int jl = max(lo - k_row0, 0), jh = min(hi - k_row0, nk);
@@ -625,10 +639,6 @@ __device__ long long g_bwd_phase_cycles[16];
 // so they run while the CTA drains dQ/dK/dV of item i.
 // Thread t: row t % 128 (TMEM lane), column quarter t / 128.
 // ---------------------------------------------------------------------------------------------
-// Output tiles leave through TMA stores.  A block has 1..128 rows and a store box has a fixed
-// number of rows, so each gradient tensor gets seven maps with boxes of 64, 32, ..., 1 rows and a
-// tile is stored as two (possibly overlapping) boxes of the largest size that fits.
-struct StoreMaps { CUtensorMap m[3][7]; };
 
 template <bool SPLIT, bool DIRS = false>
 __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUtensorMap tm_q,
@@ -1006,7 +1016,7 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     b.rest_only = 0;
     int n_general = a.nb;
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
-    if (D == 64 && a.nb > 0 && !a.no_persistent) {   // (no_persistent == 5: the looping kernel below instead)
+    if (D == 64 && a.nb > 0 && (!a.no_persistent || a.no_persistent == 4 || a.no_persistent == 6)) {   // (no_persistent == 5: the looping kernel below instead)
         // the persistent kernel takes everything: first the blocks of split families (longest first),
         // then the self-contained blocks
         constexpr int smem_p = 12 * SUB + 1024 + 64;
@@ -1032,6 +1042,11 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
         for (int mode = 1; mode >= 0; --mode) {
             const long long units = (long long)(mode ? a.nb - a.n_fused : a.n_fused) * a.H;
             if (units == 0) continue;
+            if (mode == 0 && a.no_persistent != 4) {     // (4: the persistent kernel takes these too)
+                rc = launch_bwd_tc_fused64(a, tq, tk, tv, tdo, outs, st);
+                if (rc) return rc;
+                continue;
+            }
             BwdStageArgs c = a;
             c.rest_only = mode;
             const int grid_p = (int)(units < n_sm ? units : n_sm);

@@ -112,5 +112,15 @@ extern "C" int hdt_debug_fwd_phase_cycles(int64_t *out16) {
 extern "C" int hdt_debug_bwd_phase_cycles(int64_t *out16) {
     if (!out16) return set_error(HDT_ERR_INVALID_ARG, "hdt_debug_bwd_phase_cycles: null pointer");
     HDT_CUDA_CHECK(cudaDeviceSynchronize());
-    return read_bwd_phase_cycles((long long *)out16);
+    const int rc = read_bwd_phase_cycles((long long *)out16);
+    return rc ? rc : read_bwd_t_phase_cycles((long long *)out16);
+}
+
+// Diagnostics: per CTA (up to 512) of the last instrumented transposed backward launch (option
+// "phase_stamps"): global timer at entry, when the first input tiles had arrived, at the end of its
+// item loop (ns), and the SM it ran on.  Waits for the device.
+extern "C" int hdt_debug_bwd_timeline(int64_t *out2048) {
+    if (!out2048) return hdt::set_error(HDT_ERR_INVALID_ARG, "hdt_debug_bwd_timeline: null pointer");
+    HDT_CUDA_CHECK(cudaDeviceSynchronize());
+    return hdt::read_bwd_t_timeline((long long *)out2048);
 }

@@ -74,6 +74,7 @@ int get_side(Side **out);
 extern int g_no_overlap;   // option "no_overlap"
 extern int g_force_simt;   // option "force_simt"
 extern int g_no_graph;     // option "no_graph"
+extern int g_phase_stamps; // option "phase_stamps": the transposed backward runs its instrumented instantiation
 
 // Direction bits inside a row range (paper, "Mathematical Reasoning Tasks": the ListOps attention
 // patterns).  Row e of a stage has the key range [lo, hi).  If the range starts at or after e, e is
@@ -154,7 +155,8 @@ struct BwdStageArgs {
     int n_fused;
     const void *q, *k, *v, *d_o;
     const float *lse;    // [H,T] final
-    const float *delta;  // [H,T]
+    const float *delta;  // [H,T]; nullptr: the kernels compute dO . O of their rows themselves (needs o)
+    const void *o;       // forward output, dtype [T,H,D]; read only when delta is nullptr
     float scale, scale_log2;
     const float *carry_dq, *carry_dk, *carry_dv;  // [n,H,D] partials from the stages below, or nullptr
     void *dq, *dk, *dv;                           // dtype [T,H,D], written by every stage
@@ -178,6 +180,8 @@ int launch_bwd_tc(const BwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_fwd_tc_upper(const FwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_bwd_tc_upper(const BwdStageArgs &a, int head_dim, cudaStream_t st);
 int read_bwd_phase_cycles(long long *out16);
+int read_bwd_t_phase_cycles(long long *out16);   // adds to out16
+int read_bwd_t_timeline(long long *out2048);     // per CTA of the last instrumented launch: entry, first tiles in, end (ns), SM
 int read_fwd_phase_cycles(long long *out16);
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,

@@ -40,4 +40,15 @@ inline int make_tmap_bf16(CUtensorMap *tm, const void *base, int D, int H, long 
     return HDT_OK;
 }
 
+// Output tiles of the persistent backward kernels leave through TMA stores.  A block has 1..128 rows
+// and a store box has a fixed number of rows, so each gradient tensor (dq, dk, dv) gets seven maps
+// with boxes of 64, 32, ..., 1 rows and a tile is stored as two (possibly overlapping) boxes of the
+// largest size that fits.
+struct StoreMaps { CUtensorMap m[3][7]; };
+
+// Self-contained (SELF, non-EMPTY) blocks of stage 0 at head_dim 64 through the transposed looping
+// backward (hdt_attn_tc_bwd_t.cu); the maps are those of q, k, v, dO with boxes of 128 rows.
+int launch_bwd_tc_fused64(const BwdStageArgs &a, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+                          const CUtensorMap &tdo, const StoreMaps &outs, cudaStream_t st);
+
 }  // namespace hdt
