@@ -75,7 +75,15 @@ typedef struct {
                            always stays.  0 = the full parent/sibling/child rule.  The family
                            ranges of the index do not change; nnz counts the remaining pairs and
                            the attention kernels drop the switched-off entries inside each range */
-    int32_t reserved[4];
+    int32_t deferred;   /* 0: hdt_build_index waits until the index is complete and reports structure
+                           errors itself.  1: it returns as soon as the work is queued on the stream;
+                           the first call that needs the counts of the index on the host
+                           (hdt_index_info, hdt_index_export, the workspace queries, the attention and
+                           positional-encoding calls) waits instead and returns the structure error,
+                           if any; every later call on that index returns it too.  hdt_attn_fwd on a
+                           bf16 index still in flight queues its stage-0 kernel first (the kernel
+                           reads the counts on the device) and waits only then                 */
+    int32_t reserved[3];
 } hdt_index_params_t;
 
 typedef struct hdt_index hdt_index_t; /* opaque host object; views into the caller's workspace */
@@ -125,9 +133,11 @@ size_t hdt_index_workspace_bytes(int32_t batch, int32_t total_tokens,
  *   workspace  device, >= hdt_index_workspace_bytes(...), 256-byte aligned; must stay allocated
  *              and untouched until hdt_index_destroy
  *   out        receives a host object (free with hdt_index_destroy)
- * Waits for the stream before returning.  Errors: HDT_ERR_BAD_HIERARCHY when a precondition on
- * the structure arrays fails or the hierarchy needs more than max_stages stages (no index is
- * returned), HDT_ERR_WORKSPACE, HDT_ERR_INVALID_ARG, HDT_ERR_CUDA.
+ * Waits for the stream before returning (unless params->deferred is set: see there).  Errors:
+ * HDT_ERR_BAD_HIERARCHY when a precondition on the structure arrays fails or the hierarchy needs
+ * more than max_stages stages (no index is returned; a deferred build returns the index and the
+ * error comes from the first call that uses it), HDT_ERR_WORKSPACE, HDT_ERR_INVALID_ARG,
+ * HDT_ERR_CUDA.
  */
 int hdt_build_index(const int8_t *level, const int32_t *parent, const int32_t *cu_seqlens,
                     int32_t batch, int32_t total_tokens, const hdt_index_params_t *params,

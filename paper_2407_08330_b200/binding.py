@@ -25,7 +25,7 @@ class HdtError(RuntimeError):
 
 class _Params(C.Structure):
     _fields_ = [("block_m", C.c_int32), ("max_stages", C.c_int32), ("block_m_upper", C.c_int32),
-                ("mask_off", C.c_int32), ("reserved", C.c_int32 * 4)]
+                ("mask_off", C.c_int32), ("deferred", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
 class _StageView(C.Structure):
@@ -95,10 +95,11 @@ def _stream():
     return C.c_void_p(torch._C._cuda_getCurrentRawStream(torch.cuda.current_device()))
 
 
-def _params(block_m, max_stages, block_m_upper=0, directions=7):
+def _params(block_m, max_stages, block_m_upper=0, directions=7, deferred=False):
     p = _Params()
     p.block_m, p.max_stages, p.block_m_upper = int(block_m), int(max_stages), int(block_m_upper)
     p.mask_off = (~int(directions)) & 7
+    p.deferred = 1 if deferred else 0
     return p
 
 
@@ -167,14 +168,16 @@ class HdtIndex:
 
 
 def hdt_build_index(level, parent, cu_seqlens, block_m=0, max_stages=0, workspace=None,
-                    block_m_upper=0, directions=7) -> HdtIndex:
+                    block_m_upper=0, directions=7, deferred=False) -> HdtIndex:
     """level int8[T], parent int32[T], cu_seqlens int32[B+1]: CUDA tensors.  directions: bits
-    1 | 2 | 4 keep the child->parent, sibling<->sibling, parent->child entries (7 = full rule)."""
+    1 | 2 | 4 keep the child->parent, sibling<->sibling, parent->child entries (7 = full rule).
+    deferred: return once the build is queued; the first call that needs the index's counts on the
+    host waits for it (and raises what the build found wrong with the structure arrays)."""
     assert level.is_cuda and parent.is_cuda and cu_seqlens.is_cuda
     assert level.dtype == torch.int8 and parent.dtype == torch.int32 and cu_seqlens.dtype == torch.int32
     level, parent, cu_seqlens = level.contiguous(), parent.contiguous(), cu_seqlens.contiguous()
     T, B = level.numel(), cu_seqlens.numel() - 1
-    p = _params(block_m, max_stages, block_m_upper, directions)
+    p = _params(block_m, max_stages, block_m_upper, directions, deferred)
     need = int(lib().hdt_index_workspace_bytes(B, T, C.cast(C.byref(p), C.c_void_p)))
     if need == 0:
         raise HdtError(-1, "invalid index parameters")

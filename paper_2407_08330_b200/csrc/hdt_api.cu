@@ -30,8 +30,8 @@ static std::vector<ProfRec> g_prof_pool;      // created, free
 static double g_prof_ms[PROF_COUNT];
 static long long g_prof_n[PROF_COUNT];
 
-ProfScope::ProfScope(int id, cudaStream_t s) : slot(-1), st(s) {
-    if (!g_prof_on) return;
+ProfScope::ProfScope(int id, cudaStream_t s, bool enabled) : slot(-1), st(s) {
+    if (!g_prof_on || !enabled) return;
     std::lock_guard<std::mutex> lk(g_prof_mu);
     ProfRec r;
     if (!g_prof_pool.empty()) { r = g_prof_pool.back(); g_prof_pool.pop_back(); }
@@ -195,6 +195,7 @@ extern "C" size_t hdt_attn_workspace_bytes(const hdt_index_t *ix, int32_t heads,
                                            int32_t dtype, int32_t bwd) {
     (void)dtype;
     if (!ix || heads <= 0 || head_dim <= 0) return 0;
+    if (index_ready(ix)) return 0;
     return attn_layout(ix, heads, head_dim, bwd).total;
 }
 
@@ -202,18 +203,54 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
                             float *lse, int32_t heads, int32_t head_dim, int32_t dtype, float softmax_scale,
                             void *workspace, size_t workspace_bytes, void *stream) {
     if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: null index");
-    const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 0);
-    int rc = check_common(ix, heads, head_dim, dtype, workspace, workspace_bytes, L.total, "hdt_attn_fwd");
+    int rc = check_common(ix, heads, head_dim, dtype, workspace, workspace_bytes, 0, "hdt_attn_fwd");
     if (rc) return rc;
-    if (ix->total_tokens == 0) return HDT_OK;
-    if (!q || !k || !v || !o || !lse) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: null tensor pointer");
-    if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(o))
-        return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: tensors must be 16-byte aligned");
+    if (ix->total_tokens > 0) {
+        if (!q || !k || !v || !o || !lse) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: null tensor pointer");
+        if (misaligned(q) || misaligned(k) || misaligned(v) || misaligned(o))
+            return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd: tensors must be 16-byte aligned");
+    }
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
     cudaStream_t st = (cudaStream_t)stream;
     char *ws = (char *)workspace;
     int *status = device_status_ptr();
     if (!status) return HDT_ERR_CUDA;
+    // A deferred index whose build is still in flight: the looping stage-0 kernel of bf16 calls is
+    // queued before the host waits for the counts (it reads them on the device), so the GPU goes
+    // from the build straight into the attention.  The stream is forked first: what the host
+    // launches on the side streams after its wait still runs beside that kernel, not behind it.
+    bool early = false;
+    if (ix->pending && ix->total_tokens > 0 && dtype == HDT_BF16 && !g_force_simt && g_no_persistent == 0 &&
+        !g_no_overlap && (workspace == nullptr || ((uintptr_t)workspace & 255) == 0)) {
+        Side *sd = nullptr;
+        rc = get_side(&sd);
+        if (rc) return rc;
+        HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
+        const StagePtrs &P = ix->st[0];
+        FwdStageArgs a{};
+        a.n = ix->total_tokens; a.H = heads; a.T = ix->total_tokens;
+        a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue; a.queue_split = P.queue_split;
+        a.block_rows = ix->block_m;
+        a.q = q; a.k = k; a.v = v;
+        a.scale_log2 = scale * 1.4426950408889634f;
+        a.part_o = (float *)ws;              // stage 1's partial results come first in the workspace
+        a.ws_bytes = workspace ? workspace_bytes : 0;
+        a.hdr = ix->hdr_dev;
+        a.o = o; a.lse = lse;
+        a.status = status;
+        a.dirs = ix->directions;
+        a.part = 1;
+        ProfScope ps(PROF_FWD_STAGE0, st);
+        rc = launch_fwd_tc(a, head_dim, st);
+        if (rc) return rc;
+        early = true;
+    }
+    rc = index_ready(ix);
+    if (rc) return rc;
+    const AttnLayout L = attn_layout(ix, heads, head_dim, 0);
+    rc = check_common(ix, heads, head_dim, dtype, workspace, workspace_bytes, L.total, "hdt_attn_fwd");
+    if (rc) return rc;
+    if (ix->total_tokens == 0) return HDT_OK;
     auto stage_args = [&](int s) {
         const StagePtrs &P = ix->st[s];
         FwdStageArgs a{};
@@ -241,19 +278,19 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
     };
     // The stages above 0 do not depend on stage 0 until their results are merged: compute them on
     // the side stream while stage 0 runs, then finish each with an element-wise merge.
-    const bool overlap = ix->n_stages > 1 && !g_no_overlap;
+    const bool overlap = (ix->n_stages > 1 && !g_no_overlap) || early;
     if (overlap) {
         Side *sd = nullptr;
         rc = get_side(&sd);
         if (rc) return rc;
-        HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
+        if (!early) HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
         const bool tc0 = dtype == HDT_BF16 && !g_force_simt;
         // Stage 0's blocks that are not self-contained (split families, EMPTY blocks) have a kernel of
         // their own.  Where the split families are the smaller part it runs on the second side stream beside the
         // looping kernel (measured: a batch of padded documents gains 7 %); where split families
         // dominate, one kernel after the other is faster (the skewed batch loses 3 % side by side).
-        const bool rest_beside = tc0 && 2 * (ix->desc[0].nb - ix->desc[0].n_fused - ix->desc[0].n_empty) <= ix->desc[0].nb;
+        const bool rest_beside = early || (tc0 && 2 * (ix->desc[0].nb - ix->desc[0].n_fused - ix->desc[0].n_empty) <= ix->desc[0].nb);
         const bool two = ix->n_stages > 2 || rest_beside;
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
         // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
@@ -276,6 +313,8 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         if (rest_beside) {
             FwdStageArgs a = stage_args(0);
             a.part = 2;
+            // (profiled with stage 0 when the looping kernel went ahead: the two make up the stage)
+            ProfScope ps(PROF_FWD_STAGE0, sd->s2, early && a.nb > a.n_fused);
             rc = launch_fwd_tc(a, head_dim, sd->s2);      // behind the (small) even stages, not behind stage 1
             if (rc) return rc;
         }
@@ -285,10 +324,16 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
             // stage-0 kernel would otherwise fill every SM and push them behind itself)
             FwdStageArgs a = stage_args(0);
             a.part = rest_beside ? 1 : 0;
-            ProfScope ps(PROF_FWD_STAGE0, st);
-            if (tc0) rc = launch_fwd_tc(a, head_dim, st);
-            else rc = launch_fwd_simt(a, head_dim, dtype, st);
-            if (rc) return rc;
+            if (!early) {                    // (early: already queued)
+                ProfScope ps(PROF_FWD_STAGE0, st);
+                if (tc0) rc = launch_fwd_tc(a, head_dim, st);
+                else rc = launch_fwd_simt(a, head_dim, dtype, st);
+                if (rc) return rc;
+            }
+        }
+        if (ix->n_stages == 1) {             // (early only) nothing to merge: wait for the other blocks' kernel
+            if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
+            return HDT_OK;
         }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
@@ -315,6 +360,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
                             int32_t head_dim, int32_t dtype, float softmax_scale, void *workspace,
                             size_t workspace_bytes, void *stream) {
     if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_bwd: null index");
+    if (const int rc0 = index_ready(ix)) return rc0;
     const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 1);
     int rc = check_common(ix, heads, head_dim, dtype, workspace, workspace_bytes, L.total, "hdt_attn_bwd");
     if (rc) return rc;
@@ -444,6 +490,7 @@ extern "C" int hdt_attn_fwd_static(const hdt_index_t *ix, const void *q, const v
                                    float *lse, int32_t heads, int32_t head_dim, int32_t dtype,
                                    float softmax_scale, void *stream) {
     if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_fwd_static: null index");
+    if (const int rc0 = index_ready(ix)) return rc0;
     const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 0);
     if (L.total > (size_t)HDT_FWD_STATIC_SCRATCH_BYTES)
         return set_error(HDT_ERR_WORKSPACE,

@@ -397,7 +397,26 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int H = a.H, G = gridDim.x;
-    const int n_items = a.n_fused * H;
+    // Counts not yet known to the host (the index build is still in flight when this kernel is
+    // queued): they are read from the index header, and the partial buffers of stage 1 are laid
+    // out from its element count the way the host does it (results, then LSE, 256-byte aligned).
+    int n_fused = a.n_fused;
+    float *part_o = a.part_o, *part_lse = a.part_lse;
+    if (a.hdr != nullptr) {
+        const DevHeader *hd = a.hdr;
+        n_fused = (hd->status == 0) ? hd->st[0].n_fused : 0;
+        const size_t n1 = (size_t)hd->st[1].n;
+        const size_t b_o = (sizeof(float) * n1 * H * D + 255) & ~size_t(255), b_l = (sizeof(float) * n1 * H + 255) & ~size_t(255);
+        if (n1 == 0) {
+            part_o = nullptr;
+            part_lse = nullptr;
+        } else if (part_o == nullptr || b_o + b_l > a.ws_bytes) {
+            n_fused = 0;            // the host finds the same after its wait and reports the workspace error
+        } else {
+            part_lse = reinterpret_cast<float *>(reinterpret_cast<char *>(part_o) + b_o);
+        }
+    }
+    const int n_items = n_fused * H;
     const float NEG = -INFINITY, LN2 = 0.6931471805599453f;
 
     if (tid == 0) {
@@ -452,7 +471,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             if (inb) {
                 lo = a.rng[2 * row];
                 hi = a.rng[2 * row + 1];
-                if (a.part_o != nullptr) up = a.up[row];
+                if (part_o != nullptr) up = a.up[row];
             }
             const int nvalid = min(128, kb - ka), Nc = (nvalid + 15) & ~15;
 
@@ -548,8 +567,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             if (l > 0.f) { w0 = 1.f / l; lse = (m + log2f(l)) * LN2; }
             float *po = nullptr;
             if (up >= 0) {
-                po = a.part_o + ((size_t)up * H + h) * D;
-                a.part_lse[(size_t)up * H + h] = lse;
+                po = part_o + ((size_t)up * H + h) * D;
+                part_lse[(size_t)up * H + h] = lse;
             }
 #pragma unroll
             for (int k = 0; k < D / 32; ++k) {
@@ -882,10 +901,24 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
                                             8 * SUB + 4 * 128 * 4 + 1024 + 64));
         attr = true;
     }
+    const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
+    if (a.hdr != nullptr) {          // counts on the device only: the looping kernel with all its CTAs
+        static int n_sm_e = 0;
+        if (n_sm_e == 0) {
+            int dev = 0;
+            HDT_CUDA_CHECK(cudaGetDevice(&dev));
+            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm_e, cudaDevAttrMultiProcessorCount, dev));
+        }
+        const int grid = n_sm_e * (D == 64 ? 4 : 2);
+        if (dirs) k_fwd_tc_loop<D, true><<<grid, 128, smem_1, st>>>(tq, tk, tv, a);
+        else k_fwd_tc_loop<D><<<grid, 128, smem_1, st>>>(tq, tk, tv, a);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+        return HDT_OK;
+    }
     FwdStageArgs b = a;
     b.rest_only = 0;
     int n_general = a.nb;
-    const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
     const bool split_launch = a.no_persistent != 1;     // two kernels: self-contained blocks, the others
     if (a.n_fused > 0 && split_launch && a.part == 2) {  // the caller launches the looping kernel separately
         b.rest_only = 1;
@@ -958,7 +991,7 @@ int launch_fwd_tc_upper(const FwdStageArgs &a, int D, cudaStream_t st) {
 }
 
 int launch_fwd_tc(const FwdStageArgs &a, int D, cudaStream_t st) {
-    if (a.nb == 0) return HDT_OK;
+    if (a.nb == 0 && a.hdr == nullptr) return HDT_OK;
     if (D == 64) return launch_fwd_tc_t<64>(a, st);
     if (D == 128) return launch_fwd_tc_t<128>(a, st);
     return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);

@@ -368,6 +368,7 @@ extern "C" int hdt_hpe(const hdt_index_t *ix, const int8_t *level, const int32_t
                        int32_t n_levels, int32_t d_model, int32_t dtype, int32_t accumulate, void *x,
                        void *workspace, size_t workspace_bytes, void *stream) {
     if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_hpe: null index");
+    if (const int rc0 = index_ready(ix)) return rc0;
     if (n_levels < 1 || n_levels > 32 || d_model < 2 || (d_model & 1))
         return set_error(HDT_ERR_INVALID_ARG, "hdt_hpe: n_levels must be 1..32, d_model even and positive");
     if (dtype != HDT_F32 && dtype != HDT_BF16) return set_error(HDT_ERR_UNSUPPORTED, "hdt_hpe: unknown dtype %d", dtype);

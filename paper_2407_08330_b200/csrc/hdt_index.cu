@@ -12,6 +12,9 @@
 //   queue     rank sort by cost (longest first)
 #include <cstdio>
 #include <cstring>
+#include <atomic>
+#include <mutex>
+#include <vector>
 
 #include "hdt_internal.cuh"
 
@@ -706,6 +709,30 @@ extern "C" size_t hdt_index_workspace_bytes(int32_t batch, int32_t total_tokens,
     return make_layout(batch, total_tokens, min(bm, bmu), ms).total;
 }
 
+// Pinned landing buffers for index headers: a small pool shared by all host threads (a deferred
+// index keeps its buffer until the header has been read).
+static const int kUnset = 0x7fffffff;
+static std::mutex g_pinned_mu;
+static std::vector<DevHeader *> g_pinned_free;
+static DevHeader *pinned_acquire() {
+    {
+        std::lock_guard<std::mutex> lk(g_pinned_mu);
+        if (!g_pinned_free.empty()) {
+            DevHeader *p = g_pinned_free.back();
+            g_pinned_free.pop_back();
+            return p;
+        }
+    }
+    DevHeader *p = nullptr;
+    if (cudaMallocHost((void **)&p, sizeof(DevHeader)) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
+    return p;
+}
+static void pinned_release(DevHeader *p) {
+    if (!p) return;
+    std::lock_guard<std::mutex> lk(g_pinned_mu);
+    g_pinned_free.push_back(p);
+}
+
 extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const int32_t *cu_seqlens,
                                int32_t batch, int32_t total_tokens, const hdt_index_params_t *params,
                                void *workspace, size_t workspace_bytes, void *stream, hdt_index_t **out) {
@@ -877,48 +904,95 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             count_launch(n_launched);
         }
     }
-    // the header comes back through a pinned host buffer (one per host thread, allocated once):
-    // a copy to pageable memory would be staged by the driver
-    static thread_local DevHeader *h_pinned = nullptr;
-    if (!h_pinned) HDT_BUILD_CHECK(cudaMallocHost((void **)&h_pinned, sizeof(DevHeader)));
-    // The host watches the copy land instead of waiting in the driver: first and last word of the
-    // pinned buffer are set to a value the device never writes (status is 0 or negative, tail is 0)
-    // and polled; the copy is the last operation of the build on the stream, and its words arrive
-    // in order.  After a bounded number of polls the ordinary wait takes over.
-    const int kUnset = 0x7fffffff;
-    volatile int *p_status = &h_pinned->status, *p_tail = &h_pinned->tail;
-    *p_status = kUnset;
-    *p_tail = kUnset;
-    HDT_BUILD_CHECK(cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, st));
-    bool landed = false;
-    for (long long spin = 0; spin < 20000000LL && !landed; ++spin) landed = (*p_tail != kUnset && *p_status != kUnset);
-    if (!landed) HDT_BUILD_CHECK(cudaStreamSynchronize(st));
-    std::atomic_thread_fence(std::memory_order_acquire);
-    const DevHeader h = *h_pinned;
+    // The header comes back through a pinned host buffer (a copy to pageable memory would be staged
+    // by the driver).  First and last word of the buffer are set to a value the device never writes
+    // (status is 0 or negative, tail is 0) so that the host can watch the copy land: it is the last
+    // operation of the build on the stream, and its words arrive in order.
+    DevHeader *h_pinned = pinned_acquire();
+    if (!h_pinned) {
+        delete ix;
+        return set_error(HDT_ERR_CUDA, "hdt_build_index: no pinned host memory for the index header");
+    }
+    h_pinned->status = kUnset;
+    h_pinned->tail = kUnset;
+    ix->h_pinned = h_pinned;
+    ix->hdr_dev = hdr;
+    ix->stream = st;
+    ix->max_stages = ms;
+    ix->pending = 1;
+    {
+        const cudaError_t e_ = cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, st);
+        if (e_ != cudaSuccess) {
+            pinned_release(h_pinned);
+            delete ix;
+            return set_error(HDT_ERR_CUDA, "cudaMemcpyAsync of the index header failed: %s", cudaGetErrorString(e_));
+        }
+    }
 #undef HDT_BUILD_CHECK
-    if (h.status != 0) {
-        delete ix;
-        return set_error(h.status, "hdt_build_index: structure arrays violate a precondition near element %d",
-                         h.err_pos);
+    if (!(params && params->deferred)) {
+        const int rc = index_ready(ix);
+        if (rc) {
+            delete ix;
+            return rc;
+        }
     }
-    int ns = 1;
-    while (ns < ms && h.st[ns].n > 0) ++ns;
-    if (h.st[ns - 1].has_next && ns == ms) {
-        delete ix;
-        return set_error(HDT_ERR_BAD_HIERARCHY,
-                         "hdt_build_index: hierarchy needs more than max_stages = %d stages", ms);
-    }
-    // a last stage that found "has_next" without one being built cannot happen below ms
-    ix->n_stages = ns;
-    ix->nnz = h.nnz;
-    ix->visited = h.visited;
-    for (int s = 0; s <= HDT_MAX_STAGES; ++s) ix->desc[s] = h.st[s];
     *out = ix;
     return HDT_OK;
 }
 
+namespace hdt {
+int index_ready(const hdt_index *cix) {
+    hdt_index *ix = const_cast<hdt_index *>(cix);
+    if (ix->pending) {
+        // The host watches the copy land instead of waiting in the driver; after a bounded number
+        // of polls the ordinary wait takes over.
+        DevHeader *hp = ix->h_pinned;
+        volatile int *p_status = &hp->status, *p_tail = &hp->tail;
+        bool landed = false;
+        for (long long spin = 0; spin < 20000000LL && !landed; ++spin) landed = (*p_tail != kUnset && *p_status != kUnset);
+        if (!landed) {
+            const cudaError_t e_ = cudaStreamSynchronize(ix->stream);
+            if (e_ != cudaSuccess) {
+                ix->pending = 0;
+                ix->failed = HDT_ERR_CUDA;
+                pinned_release(hp);
+                ix->h_pinned = nullptr;
+                return set_error(HDT_ERR_CUDA, "waiting for the index build failed: %s", cudaGetErrorString(e_));
+            }
+        }
+        std::atomic_thread_fence(std::memory_order_acquire);
+        const DevHeader h = *hp;
+        pinned_release(hp);
+        ix->h_pinned = nullptr;
+        ix->pending = 0;
+        ix->failed = h.status;
+        ix->err_pos = h.err_pos;
+        if (h.status == 0) {
+            int ns = 1;
+            while (ns < ix->max_stages && h.st[ns].n > 0) ++ns;
+            // (a last stage that found "has_next" without one being built cannot happen below max_stages)
+            if (h.st[ns - 1].has_next && ns == ix->max_stages) {
+                ix->failed = HDT_ERR_BAD_HIERARCHY;
+                ix->err_pos = -1;
+            } else {
+                ix->n_stages = ns;
+                ix->nnz = h.nnz;
+                ix->visited = h.visited;
+                for (int s = 0; s <= HDT_MAX_STAGES; ++s) ix->desc[s] = h.st[s];
+            }
+        }
+    }
+    if (ix->failed == 0) return HDT_OK;
+    if (ix->failed == HDT_ERR_BAD_HIERARCHY && ix->err_pos < 0)
+        return set_error(HDT_ERR_BAD_HIERARCHY, "hdt_build_index: hierarchy needs more than max_stages = %d stages",
+                         ix->max_stages);
+    return set_error(ix->failed, "hdt_build_index: structure arrays violate a precondition near element %d", ix->err_pos);
+}
+}  // namespace hdt
+
 extern "C" int hdt_index_info(const hdt_index_t *ix, int32_t *n_stages, int64_t *nnz, int64_t *visited) {
     if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_index_info: null index");
+    if (const int rc = index_ready(ix)) return rc;
     if (n_stages) *n_stages = ix->n_stages;
     if (nnz) *nnz = ix->nnz;
     if (visited) *visited = ix->visited;
@@ -927,6 +1001,7 @@ extern "C" int hdt_index_info(const hdt_index_t *ix, int32_t *n_stages, int64_t 
 
 extern "C" int hdt_index_export(const hdt_index_t *ix, int32_t stage, hdt_stage_view_t *v) {
     if (!ix || !v) return set_error(HDT_ERR_INVALID_ARG, "hdt_index_export: null argument");
+    if (const int rc = index_ready(ix)) return rc;
     if (stage < 0 || stage >= ix->n_stages)
         return set_error(HDT_ERR_INVALID_ARG, "hdt_index_export: stage %d outside [0,%d)", stage, ix->n_stages);
     const StagePtrs &P = ix->st[stage];
@@ -940,6 +1015,7 @@ extern "C" int hdt_index_export(const hdt_index_t *ix, int32_t stage, hdt_stage_
 }
 
 extern "C" int hdt_index_destroy(hdt_index_t *ix) {
+    if (ix && ix->pending) (void)index_ready(ix);     // the header copy must not land in a recycled buffer
     delete ix;
     return HDT_OK;
 }

@@ -41,11 +41,22 @@ struct hdt_index {
     hdt::StagePtrs st[HDT_MAX_STAGES];
     void *workspace;
     size_t workspace_bytes;
+    // Deferred build: the device header is on its way to h_pinned; hdt::index_ready() waits for it
+    // and fills n_stages, nnz, visited and desc.
+    int pending;                      // 1 until the header has been read
+    int failed;                       // hdt_status_t found in the header (or by its check), 0 = fine
+    int err_pos, max_stages;
+    hdt::DevHeader *h_pinned;         // pinned landing buffer (from a pool), nullptr once released
+    const hdt::DevHeader *hdr_dev;    // the header in the index workspace
+    cudaStream_t stream;              // stream of the build
 };
 
 namespace hdt {
 
 int set_error(int code, const char *fmt, ...);
+// Waits (if the build was deferred) until the counts of the index are on the host; returns the
+// structure error of the build, if any.
+int index_ready(const hdt_index *ix);
 int *device_status_ptr();  // device address of the failure word kernels report into
 extern std::atomic<long long> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
@@ -56,7 +67,7 @@ enum ProfId { PROF_INDEX = 0, PROF_FWD_STAGE0, PROF_FWD_UPPER, PROF_DELTA, PROF_
 struct ProfScope {
     int slot;
     cudaStream_t st;
-    ProfScope(int id, cudaStream_t st);
+    ProfScope(int id, cudaStream_t st, bool enabled = true);
     ~ProfScope();
 };
 
@@ -145,6 +156,8 @@ struct FwdStageArgs {
     int dirs;           // direction bits kept (7 = full rule), see dir_ok
     const int *tok_rows;  // SIMT kernels: token map of the block rows (nullptr: identity); `tok` maps the keys
     int part;             // launch_fwd_tc: 0 = all blocks, 1 = only the self-contained ones (looping kernel), 2 = only the others
+    const DevHeader *hdr; // set: the index build is still in flight; the looping kernel reads n_fused and stage 1's size here
+    size_t ws_bytes;      // with hdr: bytes behind part_o (the caller's workspace)
 };
 
 struct BwdStageArgs {
