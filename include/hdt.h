@@ -294,7 +294,13 @@ int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const i
  * kernels instead of the gathering tensor-core kernels; "no_overlap" = 1 runs the stages
  * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream;
  * "no_graph" = 1 makes hdt_build_index launch its kernels one by one instead of replaying a cached
- * CUDA graph (A/B comparisons, tests).
+ * CUDA graph (A/B comparisons, tests).  "no_persistent" = 4 keeps the self-contained blocks of a
+ * head_dim 64 backward on the persistent 512-thread kernel instead of the transposed looping one,
+ * = 6 gives the latter one CTA per SM; "no_fused_delta" = 1 runs the delta pass even where every
+ * backward kernel of the call could compute dO . O itself; "no_fold" bit 0 = 1 lets a merge
+ * kernel complete the elements of stage 1 in the forward instead of the stage-1 kernel itself, bit 2
+ * = 1 makes the backward's stage-1 kernel do it (off by default); "phase_stamps" = 1 selects the
+ * instrumented instantiation of the transposed looping backward (see hdt_debug_bwd_timeline).
  */
 int hdt_set_option(const char *name, int32_t value);
 

@@ -68,6 +68,7 @@ int g_no_overlap = 0;
 int g_no_graph = 0;
 int g_phase_stamps = 0;
 static int g_no_fused_delta = 0;
+static int g_no_fold = 0;
 
 int get_side(Side **out) {
     int dev = -1;
@@ -142,6 +143,7 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "no_graph") == 0) { g_no_graph = value; return HDT_OK; }
     if (name && std::strcmp(name, "phase_stamps") == 0) { g_phase_stamps = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_fused_delta") == 0) { g_no_fused_delta = value; return HDT_OK; }
+    if (name && std::strcmp(name, "no_fold") == 0) { g_no_fold = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 
@@ -300,11 +302,17 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 1;
         c.tok1 = ix->st[1].tok;
+        // On the gathering kernels stage 1 runs after stage 0 and completes its elements itself
+        // (its own result merged with stage 0's partial and stage 2's own); only stage 2 runs beside
+        // stage 0, and there is no merge kernel.
+        const bool fold = tc_upper && !(g_no_fold & 1) && ix->n_stages > 1;
+        FwdStageArgs a1{};
         for (int s = 1; s < ix->n_stages; ++s) {
             FwdStageArgs a = stage_args(s);
             a.own_o = (float *)(ws + L.own[s][0]);
             a.own_lse = (float *)(ws + L.own[s][1]);
             c.up[s] = ix->st[s].up; c.own[s][0] = a.own_o; c.own_lse[s] = a.own_lse;
+            if (fold && s == 1) { a1 = a; continue; }
             cudaStream_t ss = (s & 1) ? sd->s : sd->s2;
             if (tc_upper) rc = launch_fwd_tc_upper(a, head_dim, ss);
             else rc = launch_fwd_simt(a, head_dim, dtype, ss);
@@ -337,10 +345,16 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
+        ProfScope ps(PROF_FWD_UPPER, st);
+        if (fold) {
+            a1.final_merge = 1;
+            a1.own_o = nullptr; a1.own_lse = nullptr;
+            if (ix->n_stages > 2) { a1.next_own_o = c.own[2][0]; a1.next_own_lse = c.own_lse[2]; }
+            return launch_fwd_tc_upper(a1, head_dim, st);
+        }
         c.base[0] = (const float *)(ws + L.part[1][0]);
         c.base_lse = (const float *)(ws + L.part[1][1]);
         c.out[0] = o; c.lse = lse;
-        ProfScope ps(PROF_FWD_UPPER, st);
         return launch_chain_merge(c, head_dim, dtype, st);
     }
     for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first
@@ -431,6 +445,9 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 3;
         c.tok1 = ix->st[1].tok;
+        // (stage 1 on the gathering kernels: after stage 0, completing its elements itself; see hdt_attn_fwd)
+        const bool fold = tc_upper && (g_no_fold & 4);   // measured: no gain in the backward (the kernel is longer than the merge it saves); option only
+        BwdStageArgs a1{};
         for (int s = 1; s < ix->n_stages; ++s) {
             BwdStageArgs a = stage_args(s);
             a.own_dq = (float *)(ws + L.own[s][0]);
@@ -438,6 +455,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             a.own_dv = (float *)(ws + L.own[s][2]);
             c.up[s] = ix->st[s].up;
             c.own[s][0] = a.own_dq; c.own[s][1] = a.own_dk; c.own[s][2] = a.own_dv;
+            if (fold && s == 1) { a1 = a; continue; }
             cudaStream_t ss = (s & 1) ? sd->s : sd->s2;
             if (tc_upper) rc = launch_bwd_tc_upper(a, head_dim, ss);
             else rc = launch_bwd_simt(a, head_dim, dtype, ss);
@@ -454,9 +472,17 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
+        ProfScope ps(PROF_BWD_UPPER, st);
+        if (fold) {
+            a1.final_merge = 1;
+            a1.own_dq = nullptr; a1.own_dk = nullptr; a1.own_dv = nullptr;
+            if (ix->n_stages > 2) {
+                a1.next_own_dq = c.own[2][0]; a1.next_own_dk = c.own[2][1]; a1.next_own_dv = c.own[2][2];
+            }
+            return launch_bwd_tc_upper(a1, head_dim, st);
+        }
         for (int k = 0; k < 3; ++k) c.base[k] = (const float *)(ws + L.part[1][k]);
         c.out[0] = dq; c.out[1] = dk; c.out[2] = dv;
-        ProfScope ps(PROF_BWD_UPPER, st);
         return launch_chain_merge(c, head_dim, dtype, st);
     }
     for (int s = 0; s < ix->n_stages; ++s) {   // bottom-up: stage 0 first

@@ -291,6 +291,78 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
     float lse = NEG, w0 = 0.f;
     if (l > 0.f) { w0 = 1.f / l; lse = (m + log2f(l)) * LN2; }
     if constexpr (GATHER) {
+        if (a.final_merge) {
+            // log-sum-exp merge of the three partial results of the element: this stage's (in TMEM,
+            // unnormalised), stage 0's, stage 2's; straight to the token's row
+            float lb = NEG, lu = NEG;
+            const float *pb = nullptr, *pu = nullptr;
+            int tk = 0;
+            if (inb) {
+                tk = a.tok[row];
+                lb = a.carry_lse[(size_t)row * H + h];
+                pb = a.carry_o + ((size_t)row * H + h) * D;
+                if (a.next_own_o != nullptr) {
+                    const int e2 = a.up[row];
+                    if (e2 >= 0) {
+                        lu = a.next_own_lse[(size_t)e2 * H + h];
+                        pu = a.next_own_o + ((size_t)e2 * H + h) * D;
+                    }
+                }
+            }
+            const float mx = fmaxf(fmaxf(lse, lb), lu);
+            float wo = 0.f, wb = 0.f, wu = 0.f, lse_f = NEG;
+            if (mx > NEG) {
+                wo = (lse > NEG) ? __expf(lse - mx) : 0.f;
+                wb = (lb > NEG) ? __expf(lb - mx) : 0.f;
+                wu = (lu > NEG) ? __expf(lu - mx) : 0.f;
+                const float tot = wo + wb + wu, inv = 1.f / tot;
+                wo *= inv * w0; wb *= inv; wu *= inv;        // (w0 normalises this stage's accumulator)
+                lse_f = mx + __logf(tot);
+            }
+            __nv_bfloat16 *og = reinterpret_cast<__nv_bfloat16 *>(a.o) + ((size_t)tk * H + h) * D;
+#pragma unroll
+            for (int k = 0; k < D / 32; ++k) {
+                uint32_t r[32];
+                if (!empty && !dead) {      // uniform in the CTA
+                    tmem_ld32(tmem + TM_O + lane_base + 32 * k, r);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] = 0u;
+                }
+                if (inb) {
+                    float x[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) x[j] = (wo > 0.f) ? __uint_as_float(r[j]) * wo : 0.f;
+                    if (wb > 0.f) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 y = *reinterpret_cast<const float4 *>(pb + 32 * k + j);
+                            x[j] = fmaf(wb, y.x, x[j]); x[j + 1] = fmaf(wb, y.y, x[j + 1]);
+                            x[j + 2] = fmaf(wb, y.z, x[j + 2]); x[j + 3] = fmaf(wb, y.w, x[j + 3]);
+                        }
+                    }
+                    if (wu > 0.f) {
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 y = *reinterpret_cast<const float4 *>(pu + 32 * k + j);
+                            x[j] = fmaf(wu, y.x, x[j]); x[j + 1] = fmaf(wu, y.y, x[j + 1]);
+                            x[j + 2] = fmaf(wu, y.z, x[j + 2]); x[j + 3] = fmaf(wu, y.w, x[j + 3]);
+                        }
+                    }
+#pragma unroll
+                    for (int c = 0; c < 4; ++c)
+                        *reinterpret_cast<uint4 *>(og + 32 * k + 8 * c) =
+                            make_uint4(pack_bf16(x[8 * c], x[8 * c + 1]), pack_bf16(x[8 * c + 2], x[8 * c + 3]),
+                                       pack_bf16(x[8 * c + 4], x[8 * c + 5]), pack_bf16(x[8 * c + 6], x[8 * c + 7]));
+                }
+            }
+            if (inb) a.lse[(size_t)h * a.T + tk] = lse_f;
+            tc_fence_before();
+            __syncthreads();
+            if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+            return;
+        }
         float *own = inb ? a.own_o + ((size_t)row * H + h) * D : nullptr;
 #pragma unroll
         for (int k = 0; k < D / 32; ++k) {
@@ -983,8 +1055,9 @@ static int launch_fwd_tc_upper_t(const FwdStageArgs &a, cudaStream_t st) {
 
 int launch_fwd_tc_upper(const FwdStageArgs &a, int D, cudaStream_t st) {
     if (a.nb == 0) return HDT_OK;
-    if (a.tok == nullptr || a.own_o == nullptr || a.own_lse == nullptr)
-        return set_error(HDT_ERR_INVALID_ARG, "launch_fwd_tc_upper: needs a tok map and own-partial buffers");
+    if (a.tok == nullptr || (!a.final_merge && (a.own_o == nullptr || a.own_lse == nullptr)) ||
+        (a.final_merge && (a.carry_o == nullptr || a.carry_lse == nullptr)))
+        return set_error(HDT_ERR_INVALID_ARG, "launch_fwd_tc_upper: needs a tok map and own-partial (or carry) buffers");
     if (D == 64) return launch_fwd_tc_upper_t<64>(a, st);
     if (D == 128) return launch_fwd_tc_upper_t<128>(a, st);
     return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);

@@ -315,6 +315,45 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
                     make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
         }
     };
+    // final_merge (gathering kernel, stage 1 after stage 0): the accumulator plus stage 0's partial
+    // (`base`) plus stage 2's own gradient (`next`, may be nullptr) go straight to the token's row.
+    auto drain_final = [&](uint32_t tm_col, bool have, float scale, const float *base, const float *next,
+                           __nv_bfloat16 *out) {
+#pragma unroll
+        for (int sl = 0; sl < D / 64; ++sl) {
+            const int c0 = hf * (D / 2) + 32 * sl;
+            uint32_t r[32];
+            if (have) {
+                tmem_ld32(tmem + tm_col + lane_base + c0, r);
+                tmem_wait_ld();
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) r[j] = 0u;
+            }
+            if (out == nullptr) continue;
+            float x[32];
+#pragma unroll
+            for (int j = 0; j < 32; j += 4) {
+                const float4 y = *reinterpret_cast<const float4 *>(base + c0 + j);
+                x[j] = fmaf(__uint_as_float(r[j]), scale, y.x);
+                x[j + 1] = fmaf(__uint_as_float(r[j + 1]), scale, y.y);
+                x[j + 2] = fmaf(__uint_as_float(r[j + 2]), scale, y.z);
+                x[j + 3] = fmaf(__uint_as_float(r[j + 3]), scale, y.w);
+            }
+            if (next != nullptr) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float4 y = *reinterpret_cast<const float4 *>(next + c0 + j);
+                    x[j] += y.x; x[j + 1] += y.y; x[j + 2] += y.z; x[j + 3] += y.w;
+                }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+                *reinterpret_cast<uint4 *>(out + c0 + 8 * c) =
+                    make_uint4(pack_bf16(x[8 * c], x[8 * c + 1]), pack_bf16(x[8 * c + 2], x[8 * c + 3]),
+                               pack_bf16(x[8 * c + 4], x[8 * c + 5]), pack_bf16(x[8 * c + 6], x[8 * c + 7]));
+        }
+    };
     auto copy_out = [&](const uint8_t *src, void *dst_g) {
         __nv_bfloat16 *g = reinterpret_cast<__nv_bfloat16 *>(dst_g);
         for (int idx = tid; idx < NSUB * 128 * 8; idx += 256) {
@@ -331,7 +370,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     const bool inb = row < r1;
     float *cq = nullptr, *ck = nullptr, *cv = nullptr;
     if constexpr (GATHER) {
-        if (inb) {      // the drains write the own gradients here; the staged bf16 copies are not used
+        if (inb && !a.final_merge) {      // the drains write the own gradients here; the staged bf16 copies are not used
             if (a.phases != 2) cq = a.own_dq + ((size_t)row * H + h) * D;
             if (a.phases != 1) {
                 ck = a.own_dk + ((size_t)row * H + h) * D;
@@ -347,13 +386,41 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         }
     }
 
+    // final_merge: where this row's three gradients go and what is added to them
+    const bool fin = GATHER && a.final_merge;
+    const float *fb[3] = {nullptr, nullptr, nullptr}, *fn[3] = {nullptr, nullptr, nullptr};
+    __nv_bfloat16 *fo[3] = {nullptr, nullptr, nullptr};
+    if constexpr (GATHER) {
+        if (fin && inb) {
+            const size_t tk = (size_t)a.tok[row];
+            const size_t ob = ((size_t)row * H + h) * D;
+            fb[0] = a.carry_dq + ob; fb[1] = a.carry_dk + ob; fb[2] = a.carry_dv + ob;
+            fo[0] = reinterpret_cast<__nv_bfloat16 *>(a.dq) + (tk * H + h) * D;
+            fo[1] = reinterpret_cast<__nv_bfloat16 *>(a.dk) + (tk * H + h) * D;
+            fo[2] = reinterpret_cast<__nv_bfloat16 *>(a.dv) + (tk * H + h) * D;
+            if (a.next_own_dq != nullptr) {
+                const int e2 = a.up[row];
+                if (e2 >= 0) {
+                    const size_t on = ((size_t)e2 * H + h) * D;
+                    fn[0] = a.next_own_dq + on; fn[1] = a.next_own_dk + on; fn[2] = a.next_own_dv + on;
+                }
+            }
+        }
+    }
+
     if (fused) {
         load(true, r0, true, r0);
         tile_pass(r0, r1, r0, r1, true, true, false, false);
         if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
-        drain(TM_DQ, true, a.scale, cq, sP);
-        drain(TM_DK, true, a.scale, ck, sDS);
-        drain(TM_DV, true, 1.f, cv, sQ);
+        if (fin) {
+            drain_final(TM_DQ, true, a.scale, fb[0], fn[0], fo[0]);
+            drain_final(TM_DK, true, a.scale, fb[1], fn[1], fo[1]);
+            drain_final(TM_DV, true, 1.f, fb[2], fn[2], fo[2]);
+        } else {
+            drain(TM_DQ, true, a.scale, cq, sP);
+            drain(TM_DK, true, a.scale, ck, sDS);
+            drain(TM_DV, true, 1.f, cv, sQ);
+        }
     } else {
         if (run && (!GATHER || a.phases != 2)) {
             // this block as query rows: dQ over the key span
@@ -363,7 +430,8 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
                 tile_pass(r0, r1, c0, kb, true, false, c0 > ka, false);
             }
         }
-        drain(TM_DQ, run, a.scale, cq, sP);
+        if (fin) drain_final(TM_DQ, run, a.scale, fb[0], fn[0], fo[0]);
+        else drain(TM_DQ, run, a.scale, cq, sP);
         // dQ leaves now: the second walk reuses sP and (at D = 128) the dQ columns of TMEM
         tc_fence_before();
         __syncthreads();
@@ -379,8 +447,13 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
             }
             if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
         }
-        drain(TM_DK, run, a.scale, ck, sDS);
-        drain(TM_DV, run, 1.f, cv, sQ);
+        if (fin) {
+            drain_final(TM_DK, run, a.scale, fb[1], fn[1], fo[1]);
+            drain_final(TM_DV, run, 1.f, fb[2], fn[2], fo[2]);
+        } else {
+            drain(TM_DK, run, a.scale, ck, sDS);
+            drain(TM_DV, run, 1.f, cv, sQ);
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -1126,8 +1199,9 @@ static int launch_bwd_tc_upper_t(const BwdStageArgs &a, cudaStream_t st) {
 
 int launch_bwd_tc_upper(const BwdStageArgs &a, int D, cudaStream_t st) {
     if (a.nb == 0) return HDT_OK;
-    if (a.tok == nullptr || a.own_dq == nullptr || a.own_dk == nullptr || a.own_dv == nullptr)
-        return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_upper: needs a tok map and own-gradient buffers");
+    if (a.tok == nullptr || (!a.final_merge && (a.own_dq == nullptr || a.own_dk == nullptr || a.own_dv == nullptr)) ||
+        (a.final_merge && (a.carry_dq == nullptr || a.carry_dk == nullptr || a.carry_dv == nullptr)))
+        return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_upper: needs a tok map and own-gradient (or carry) buffers");
     if (D == 64) return launch_bwd_tc_upper_t<64>(a, st);
     if (D == 128) return launch_bwd_tc_upper_t<128>(a, st);
     return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);

@@ -156,6 +156,12 @@ struct FwdStageArgs {
     int dirs;           // direction bits kept (7 = full rule), see dir_ok
     const int *tok_rows;  // SIMT kernels: token map of the block rows (nullptr: identity); `tok` maps the keys
     int part;             // launch_fwd_tc: 0 = all blocks, 1 = only the self-contained ones (looping kernel), 2 = only the others
+    // Gathering kernel, stage 1 run after stage 0 (final_merge = 1): instead of leaving its own
+    // partial result it completes every element of the stage: its own result, stage 0's partial
+    // (carry_*) and, for elements that live on in stage 2, that stage's own partial (next_own_*,
+    // at up[e]; nullptr without a stage 2) are merged and written to o / lse at the element's token.
+    int final_merge;
+    const float *next_own_o, *next_own_lse;
     const DevHeader *hdr; // set: the index build is still in flight; the looping kernel reads n_fused and stage 1's size here
     size_t ws_bytes;      // with hdr: bytes behind part_o (the caller's workspace)
 };
@@ -182,6 +188,11 @@ struct BwdStageArgs {
     int dirs;                                     // direction bits kept (7 = full rule), see dir_ok
     const int *tok_rows;                          // SIMT kernel: token map of the block rows (nullptr: identity); `tok` maps the walked span
     int phases;                                   // 0 = both, 1 = rows as queries only (dQ), 2 = rows as keys only (dK, dV); SIMT and gathering kernels
+    // Gathering kernel, stage 1 run after stage 0 (final_merge = 1): the element's gradients are its
+    // own plus stage 0's partials (carry_*) plus, for elements that live on in stage 2, that stage's
+    // own (next_own_*, at up[e]; nullptr without a stage 2); they go to dq / dk / dv at its token.
+    int final_merge;
+    const float *next_own_dq, *next_own_dk, *next_own_dv;
     int gather_end_q, gather_end_k;               // gathering kernel: elements at or beyond these read as zero rows on the Q/dO and the K/V side (0: n)
 };
 
