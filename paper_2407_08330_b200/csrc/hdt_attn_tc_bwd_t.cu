@@ -177,6 +177,14 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
                     }
                 }
             }
+            // the next item's tiles start their way from HBM to L2 now; the loads into shared memory
+            // (requested once this item's output MMAs have released the tiles) then find them there
+            if (tid == 0 && d1.valid) {
+                tma_prefetch_3d(&tm_k, 0, d1.h, d1.r0);
+                tma_prefetch_3d(&tm_q, 0, d1.h, d1.r0);
+                tma_prefetch_3d(&tm_v, 0, d1.h, d1.r0);
+                tma_prefetch_3d(&tm_do, 0, d1.h, d1.r0);
+            }
             HDT_TSTAMP(0);
             ok = mbar_wait(bar_in, it & 1, abort_flag, WAIT_CYCLES) && ok;
             HDT_TSTAMP(1);
