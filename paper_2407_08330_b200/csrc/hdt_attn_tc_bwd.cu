@@ -555,6 +555,16 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
             const RowStat rn = load_stat(d1);                          // row statistics one item ahead
             const int r0 = d0.r0, r1 = d0.r1, h = d0.h, nrows = r1 - r0;
             const int Nc = (nrows + 15) & ~15;
+            // the next item's tiles start their way from HBM to L2 now; the loads into shared memory
+            // (requested once this item's output MMAs have released the tiles) then find them there
+            if (tid == 0 && d1.valid) {
+                for (int s = 0; s < NSUB; ++s) {
+                    tma_prefetch_3d(&tm_q, 64 * s, d1.h, d1.r0);
+                    tma_prefetch_3d(&tm_do, 64 * s, d1.h, d1.r0);
+                    tma_prefetch_3d(&tm_k, 64 * s, d1.h, d1.r0);
+                    tma_prefetch_3d(&tm_v, 64 * s, d1.h, d1.r0);
+                }
+            }
             ok = mbar_wait(bar_in, it & 1, abort_flag, WAIT_CYCLES) && ok;
             if (issuer && warp < 2 && !*abort_flag) {      // warp 0: S = Q K^T, warp 1: dP = dO V^T
                 tc_fence_after();
