@@ -1,12 +1,14 @@
-"""Diagnostic: cycles per phase of the persistent stage-0 kernels, from their own clock stamps.
+"""Diagnostic: where the looping stage-0 backward kernel spends its time, from its own clock stamps.
 
     python -m paper_2407_08330_b200.phase_cycles [config]
 
-Thread 0 of CTA 0 of `k_fwd_tc_p` (forward, option no_persistent = 2) and of `k_bwd_tc_p`
-(backward, the default at head_dim 64) accumulates clock64() differences between fixed points of
-its item loop; `hdt_debug_fwd_phase_cycles` / `hdt_debug_bwd_phase_cycles` read and reset the
-counters.  The numbers are one thread's view of a lockstep loop: a phase that ends in a CTA
-barrier includes the wait for the slowest warp.
+With option "phase_stamps" the transposed looping backward (head_dim 64) runs an instrumented
+instantiation: thread 0 of CTA 0 adds clock64() differences between fixed points of its item loop
+(`hdt_debug_bwd_phase_cycles` reads and resets them) and every CTA records the global timer at its
+entry, when its first input tiles had arrived and at the end of its loop (`hdt_debug_bwd_timeline`).
+The cycle numbers are one thread's view of a lockstep loop: a phase that ends in a CTA barrier
+includes the wait for the slowest warp.  With "no_persistent" = 4 the persistent 512-thread kernel
+runs instead and reports its own twelve phases through the same call.
 """
 import ctypes as C
 import sys
@@ -17,10 +19,10 @@ import torch
 import gen
 import paper_2407_08330_b200 as P
 
-BWD_PHASES = ["loop top (row statistics of the next item)", "wait for S, dP (+ staged tiles gone)", "P, dS arithmetic",
-              "barrier", "issue S, dP of the next item", "wait for the output MMAs", "input request + drain of dQ, dK, dV",
-              "barrier", "TMA store requests", "item bookkeeping (next item)", "issue of the output MMAs",
-              "wait for the next item's inputs"]
+BWD_PHASES = ["loop top (O / dO row loads, L2 prefetch of the next tiles)", "wait for the input tiles",
+              "issue of S^T, dP^T", "wait for them, dO.O reduction, barrier", "P^T, dS^T arithmetic", "barrier",
+              "issue of the output MMAs", "wait for dV, dK, dQ", "drain", "barrier", "TMA store requests", "loop end"]
+EXTRA = {13: "  (record prefetch, inside the wait for the output MMAs)", 14: "  (row statistics prefetch, same place)"}
 
 
 def main(c=3):
@@ -35,18 +37,36 @@ def main(c=3):
     o, lse = P.hdt_attn_fwd(idx, q, k, v)
     L = P.lib()
     out = (C.c_int64 * 16)()
-    for _ in range(3):
-        P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
-    L.hdt_debug_bwd_phase_cycles(out)           # reset after the warm-up calls
-    for _ in range(5):
-        P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
-    torch.cuda.synchronize()
-    L.hdt_debug_bwd_phase_cycles(out)
-    v_ = np.array(list(out), float)
-    n = max(v_[12], 1.0)
-    print(f"backward, {cfg.name}: {int(n)} items of CTA 0, {v_[:12].sum() / n:.0f} cycles per item")
-    for name, x in zip(BWD_PHASES, v_[:12] / n):
-        print(f"  {name:44s} {x:7.0f}")
+    P.hdt_set_option("phase_stamps", 1)
+    try:
+        for _ in range(3):
+            P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
+        L.hdt_debug_bwd_phase_cycles(out)           # reset after the warm-up calls
+        for i in range(16):
+            out[i] = 0
+        for _ in range(5):
+            P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
+        torch.cuda.synchronize()
+        L.hdt_debug_bwd_phase_cycles(out)
+        v_ = np.array(list(out), float)
+        n = max(v_[12], 1.0)
+        print(f"backward, {cfg.name}: {int(n)} items of CTA 0, {(v_[:12].sum() + v_[13] + v_[14]) / n:.0f} cycles per item")
+        for name, x in zip(BWD_PHASES, v_[:12] / n):
+            print(f"  {name:60s} {x:7.0f}")
+        for i, name in EXTRA.items():
+            print(f"  {name:60s} {v_[i] / n:7.0f}")
+        tl = (C.c_int64 * 2048)()
+        L.hdt_debug_bwd_timeline(tl)
+        a = np.array(list(tl), dtype=np.int64).reshape(512, 4)
+        a = a[a[:, 2] > 0]
+        if len(a):
+            t0 = a[:, 0].min()
+            st, first, end = (a[:, 0] - t0) / 1e3, (a[:, 1] - t0) / 1e3, (a[:, 2] - t0) / 1e3
+            print(f"last launch, {len(a)} CTAs on {len(set(a[:, 3].tolist()))} SMs (us after the first CTA's entry): "
+                  f"entry median {np.median(st):.1f} max {st.max():.1f}; first tiles in median {np.median(first):.1f}; "
+                  f"end min {end.min():.1f} median {np.median(end):.1f} max {end.max():.1f}")
+    finally:
+        P.hdt_set_option("phase_stamps", 0)
 
 
 if __name__ == "__main__":
