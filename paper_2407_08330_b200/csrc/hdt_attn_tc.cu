@@ -121,6 +121,19 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
     float m = NEG, l = 0.f;
     uint32_t ph_tma = 0, ph_mma = 0;
     bool ok = true;
+    // final_merge (gathering kernel): what the epilogue needs from the other stages is requested now
+    float fm_lb = NEG, fm_lu = NEG;
+    int fm_tk = 0, fm_e2 = -1;
+    if constexpr (GATHER) {
+        if (a.final_merge && inb) {
+            fm_tk = a.tok[row];
+            fm_lb = a.carry_lse[(size_t)row * H + h];
+            if (a.next_own_o != nullptr) {
+                fm_e2 = a.up[row];
+                if (fm_e2 >= 0) fm_lu = a.next_own_lse[(size_t)fm_e2 * H + h];
+            }
+        }
+    }
     const bool empty = (fl & HDT_BLK_EMPTY) != 0;
     const bool dead = (*abort_flag != 0);   // same value in every thread: read after the barrier
 
@@ -130,14 +143,20 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             const int Nc = (nvalid + 15) & ~15;
             const bool first = (c0 == ka);
             if constexpr (GATHER) {
-                if (first) {
-                    uint8_t *const dq_[1] = {sQ};
-                    const void *const sq_[1] = {a.q};
-                    gather_tiles<D, 128, 1>(dq_, sq_, a.tok, r0, r1, H, h, tid);
+                if (first && ka == r0 && kb == r1) {     // keys = the block's own rows: one round of loads for all three
+                    uint8_t *const d3[3] = {sQ, sK, sV};
+                    const void *const s3[3] = {a.q, a.k, a.v};
+                    gather_tiles<D, 128, 3>(d3, s3, a.tok, r0, r1, H, h, tid);
+                } else {
+                    if (first) {
+                        uint8_t *const dq_[1] = {sQ};
+                        const void *const sq_[1] = {a.q};
+                        gather_tiles<D, 128, 1>(dq_, sq_, a.tok, r0, r1, H, h, tid);
+                    }
+                    uint8_t *const dkv[2] = {sK, sV};
+                    const void *const skv[2] = {a.k, a.v};
+                    gather_tiles<D, 128, 2>(dkv, skv, a.tok, c0, kb, H, h, tid);
                 }
-                uint8_t *const dkv[2] = {sK, sV};
-                const void *const skv[2] = {a.k, a.v};
-                gather_tiles<D, 128, 2>(dkv, skv, a.tok, c0, kb, H, h, tid);
                 fence_proxy_async_smem();     // generic-proxy writes, read by the MMA
                 __syncthreads();
             } else if constexpr (PIPE) {
@@ -294,20 +313,12 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
         if (a.final_merge) {
             // log-sum-exp merge of the three partial results of the element: this stage's (in TMEM,
             // unnormalised), stage 0's, stage 2's; straight to the token's row
-            float lb = NEG, lu = NEG;
+            const float lb = fm_lb, lu = fm_lu;
             const float *pb = nullptr, *pu = nullptr;
-            int tk = 0;
+            const int tk = fm_tk;
             if (inb) {
-                tk = a.tok[row];
-                lb = a.carry_lse[(size_t)row * H + h];
                 pb = a.carry_o + ((size_t)row * H + h) * D;
-                if (a.next_own_o != nullptr) {
-                    const int e2 = a.up[row];
-                    if (e2 >= 0) {
-                        lu = a.next_own_lse[(size_t)e2 * H + h];
-                        pu = a.next_own_o + ((size_t)e2 * H + h) * D;
-                    }
-                }
+                if (fm_e2 >= 0) pu = a.next_own_o + ((size_t)fm_e2 * H + h) * D;
             }
             const float mx = fmaxf(fmaxf(lse, lb), lu);
             float wo = 0.f, wb = 0.f, wu = 0.f, lse_f = NEG;
