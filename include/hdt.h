@@ -82,7 +82,9 @@ typedef struct {
                            positional-encoding calls) waits instead and returns the structure error,
                            if any; every later call on that index returns it too.  hdt_attn_fwd on a
                            bf16 index still in flight queues its stage-0 kernel first (the kernel
-                           reads the counts on the device) and waits only then                 */
+                           reads the counts on the device) and waits only then.  The structure
+                           arrays and the workspace must stay allocated until the stream has
+                           passed the build (as for any asynchronous call)                      */
     int32_t reserved[3];
 } hdt_index_params_t;
 
