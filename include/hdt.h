@@ -336,7 +336,10 @@ int hdt_debug_bwd_phase_cycles(int64_t *out16);
  * barriers (max exchange), P arithmetic and stores, barrier, MMA issue, wait for O, drain, loop top,
  * barrier, output stores; out16[12] = items processed. */
 int hdt_debug_fwd_phase_cycles(int64_t *out16);
-/* With option "phase_stamps" = 1 the transposed looping backward (head_dim 64) runs an instrumented
+/* With option "phase_stamps" = 1 the looping forward (head_dim 64) runs an instrumented instantiation
+ * too and hdt_debug_fwd_phase_cycles reports its phases (out16[0..10]: loop top, wait for Q/K, S,
+ * row maximum, exponentials with P into TMEM, barrier, V and the P V MMA, drain, barrier, stores, loop
+ * end).  With the same option the transposed looping backward (head_dim 64) runs an instrumented
  * instantiation: hdt_debug_bwd_phase_cycles then reports its phases (out16[0..11]: loop top, wait for
  * the input tiles, issue of S^T/dP^T, wait for them, P^T/dS^T arithmetic, barrier, issue of the output
  * MMAs, prefetch and wait for dV/dK/dQ, drain, barrier, store requests, loop end), and

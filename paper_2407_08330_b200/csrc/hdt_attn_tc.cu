@@ -463,16 +463,31 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 // K of the next item are fetched as soon as P V of the current one has finished (P, which lives
 // in the Q/K tiles, is dead then), V of the next item once the staged O has left the V tile.
 // ---------------------------------------------------------------------------------------------
-template <int D, bool DIRS = false>
+// Cycle counts per phase, accumulated by thread 0 of CTA 0 (diagnostics): of the looping kernel's
+// instrumented instantiation (STAMP), or of the persistent kernel further down.
+__device__ long long g_fwd_phase_cycles[16];
+#define HDT_LSTAMP(i)                                                              \
+    do {                                                                           \
+        if constexpr (STAMP) {                                                     \
+            if (tid == 0 && blockIdx.x == 0) {                                     \
+                const long long now_ = clock64();                                  \
+                atomicAdd((unsigned long long *)&g_fwd_phase_cycles[i], (unsigned long long)(now_ - t_last)); \
+                t_last = now_;                                                     \
+            }                                                                      \
+        }                                                                          \
+    } while (0)
+
+template <int D, bool DIRS = false, bool STAMP = false>
 __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
                                                      const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
     constexpr int NSUB = D / 64;
-    constexpr uint32_t TM_COLS = 128;   // S, then O over it
+    // S (N <= 128 columns); P (bf16, two per column) is written over its first half as the rows are
+    // exponentiated and is the A operand of O = P V; O lies beside it
+    constexpr uint32_t TM_O = (D == 64) ? 64 : 128, TM_COLS = (D == 64) ? 128 : 256;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t *sQ = sm, *sK = sQ + NSUB * SUB, *sV = sK + NSUB * SUB;
-    uint8_t *sP = sQ;                   // P (2 sub-tiles) over Q (and K at D = 64)
     uint64_t *bar_qk = (uint64_t *)(sV + NSUB * SUB);
     uint64_t *bar_v = bar_qk + 1, *bar_mma = bar_qk + 2;
     uint32_t *slot = (uint32_t *)(bar_qk + 3);
@@ -544,6 +559,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
         if (tid == 0) { issue_qk(dc); issue_v(dc); }
         uint32_t ph = 0;           // phase of bar_qk and bar_v (one completion of each per item)
         uint32_t ph_mma = 0;
+        long long t_last = STAMP ? clock64() : 0;
         for (int item = (int)blockIdx.x; item < n_items; item += G) {
             const Desc dn2 = load_desc(item + 2 * G);   // needed two iterations from now
             const int r0 = dc.r0, r1 = dc.r1, ka = dc.ka, kb = dc.kb, h = dc.h;
@@ -569,7 +585,9 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             }
             const int nvalid = min(128, kb - ka), Nc = (nvalid + 15) & ~15;
 
+            HDT_LSTAMP(0);
             ok = mbar_wait(bar_qk, ph, abort_flag, WAIT_CYCLES) && ok;
+            HDT_LSTAMP(1);
             if (tid == 0 && !*abort_flag) {
                 tc_fence_after();
                 const uint32_t idesc = idesc_bf16(Nc, false, false);
@@ -583,6 +601,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
             ph_mma ^= 1;
             tc_fence_after();
+            HDT_LSTAMP(2);
+            if (tid == 0 && have_next && !*abort_flag) issue_qk(dn);   // S is there: Q, K of the next item
 
             // ---- masked softmax of this row (one chunk: no running maximum needed) ----
             const int jl = max(lo - ka, 0), jh = min(hi - ka, nvalid);
@@ -607,6 +627,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
                     }
                 }
             }
+            HDT_LSTAMP(3);
             const float m = mx * a.scale_log2;
             float l = 0.f;
             for (int k = 0; k < nsl; ++k) {
@@ -632,30 +653,28 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
                         }
                     }
                 }
-                uint8_t *dst = sP + (k >> 1) * SUB;
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    *reinterpret_cast<uint4 *>(dst + swz(tid, (k & 1) * 4 + c)) =
-                        make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                // keys s0..s0+31 are K indices s0..s0+31 of the P V MMA: 16 packed columns, over S columns
+                // this thread has already read
+                tmem_st16(tmem + lane_base + 16 * k, pk);
             }
-            fence_proxy_async_smem();
+            tmem_wait_st();
             tc_fence_before();
+            HDT_LSTAMP(4);
             __syncthreads();
+            HDT_LSTAMP(5);
             ok = mbar_wait(bar_v, ph, abort_flag, WAIT_CYCLES) && ok;
             ph ^= 1;
             if (tid == 0 && !*abort_flag) {
                 tc_fence_after();
                 const uint32_t idesc = idesc_bf16(D, false, true);
                 for (int kk = 0; kk < Nc / 16; ++kk)
-                    mma_ss(tmem, smem_desc(smem_u32(sP) + (kk / 4) * SUB + (kk % 4) * 32, 0, 1024),
-                           smem_desc(smem_u32(sV) + kk * 2048, SUB, 1024), idesc, kk > 0);
+                    mma_ts(tmem + TM_O, tmem + 8 * kk, smem_desc(smem_u32(sV) + kk * 2048, SUB, 1024), idesc, kk > 0);
                 mma_commit(bar_mma);
             }
             ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
             ph_mma ^= 1;
             tc_fence_after();
-            if (tid == 0 && have_next && !*abort_flag) issue_qk(dn);   // P is dead: Q, K of the next item
-
+            HDT_LSTAMP(6);
             // ---- drain O, stage it (bf16) in the V tile, store ----
             float lse = NEG, w0 = 0.f;
             if (l > 0.f) { w0 = 1.f / l; lse = (m + log2f(l)) * LN2; }
@@ -667,7 +686,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
 #pragma unroll
             for (int k = 0; k < D / 32; ++k) {
                 uint32_t r[32];
-                tmem_ld32(tmem + lane_base + 32 * k, r);
+                tmem_ld32(tmem + TM_O + lane_base + 32 * k, r);
                 tmem_wait_ld();
                 float x[32];
 #pragma unroll
@@ -688,7 +707,9 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             }
             if (inb) a.lse[(size_t)h * a.T + row] = lse;
             tc_fence_before();
+            HDT_LSTAMP(7);
             __syncthreads();
+            HDT_LSTAMP(8);
             {
                 __nv_bfloat16 *og = reinterpret_cast<__nv_bfloat16 *>(a.o);
                 const int nrows = r1 - r0;
@@ -700,7 +721,10 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
                     }
                 }
             }
+            HDT_LSTAMP(9);
             __syncthreads();   // the staged O has been read: the V tile may be overwritten
+            HDT_LSTAMP(10);
+            if constexpr (STAMP) { if (tid == 0 && blockIdx.x == 0) atomicAdd((unsigned long long *)&g_fwd_phase_cycles[12], 1ull); }
             if (tid == 0 && have_next && !*abort_flag) issue_v(dn);
             dc = dn; dn = dn2;
         }
@@ -712,7 +736,6 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
 }
 
 // Cycle counts per phase of k_fwd_tc_p, accumulated by thread 0 of CTA 0 (diagnostics).
-__device__ long long g_fwd_phase_cycles[16];
 #define HDT_STAMP(i)                                        \
     do {                                                    \
         if (stamp) {                                        \
@@ -1037,7 +1060,14 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
             const long long items = (long long)a.n_fused * a.H;
             const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
             if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
-            else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
+            else if (g_phase_stamps && D == 64) {
+                static bool attr_s = false;
+                if (!attr_s) {
+                    HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
+                    attr_s = true;
+                }
+                k_fwd_tc_loop<64, false, true><<<(int)(items < slots ? items : slots), 128, 3 * SUB + 1024 + 64, st>>>(tq, tk, tv, a);
+            } else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
         }
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());

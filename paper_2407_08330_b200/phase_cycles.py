@@ -2,9 +2,9 @@
 
     python -m paper_2407_08330_b200.phase_cycles [config]
 
-With option "phase_stamps" the transposed looping backward (head_dim 64) runs an instrumented
-instantiation: thread 0 of CTA 0 adds clock64() differences between fixed points of its item loop
-(`hdt_debug_bwd_phase_cycles` reads and resets them) and every CTA records the global timer at its
+With option "phase_stamps" the looping forward and the transposed looping backward (head_dim 64) run
+instrumented instantiations: thread 0 of CTA 0 adds clock64() differences between fixed points of
+its item loop (`hdt_debug_fwd_phase_cycles` / `hdt_debug_bwd_phase_cycles` read and reset them) and every CTA records the global timer at its
 entry, when its first input tiles had arrived and at the end of its loop (`hdt_debug_bwd_timeline`).
 The cycle numbers are one thread's view of a lockstep loop: a phase that ends in a CTA barrier
 includes the wait for the slowest warp.  With "no_persistent" = 4 the persistent 512-thread kernel
@@ -19,6 +19,8 @@ import torch
 import gen
 import paper_2407_08330_b200 as P
 
+FWD_PHASES = ["loop top (records, ranges)", "wait for Q, K", "issue of S, wait for it", "row maximum", "exponentials, P into TMEM",
+              "barrier", "wait for V, issue of P V, wait for it", "drain of O, staging", "barrier", "stores", "barrier (loop end)"]
 BWD_PHASES = ["loop top (O / dO row loads, L2 prefetch of the next tiles)", "wait for the input tiles",
               "issue of S^T, dP^T", "wait for them, dO.O reduction, barrier", "P^T, dS^T arithmetic", "barrier",
               "issue of the output MMAs", "wait for dV, dK, dQ", "drain", "barrier", "TMA store requests", "loop end"]
@@ -39,6 +41,15 @@ def main(c=3):
     out = (C.c_int64 * 16)()
     P.hdt_set_option("phase_stamps", 1)
     try:
+        L.hdt_debug_fwd_phase_cycles(out)
+        for _ in range(5):
+            P.hdt_attn_fwd(idx, q, k, v)
+        L.hdt_debug_fwd_phase_cycles(out)
+        f_ = np.array(list(out), float)
+        nf = max(f_[12], 1.0)
+        print(f"forward, {cfg.name}: {int(nf)} items of CTA 0, {f_[:11].sum() / nf:.0f} cycles per item")
+        for name, x in zip(FWD_PHASES, f_[:11] / nf):
+            print(f"  {name:60s} {x:7.0f}")
         for _ in range(3):
             P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
         L.hdt_debug_bwd_phase_cycles(out)           # reset after the warm-up calls
