@@ -346,6 +346,8 @@ int hdt_debug_fwd_phase_cycles(int64_t *out16);
  * hdt_debug_bwd_timeline the last such launch per CTA (up to 512): out2048[4 c + 0..3] = global timer
  * (ns) at entry, when the first input tiles had arrived, at the end of the item loop, and the SM. */
 int hdt_debug_bwd_timeline(int64_t *out2048);
+/* The same for the last instrumented launch of the looping forward, up to 1024 CTAs. */
+int hdt_debug_fwd_timeline(int64_t *out4096);
 
 #ifdef __cplusplus
 }

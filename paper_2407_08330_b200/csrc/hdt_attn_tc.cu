@@ -466,6 +466,8 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
 // Cycle counts per phase, accumulated by thread 0 of CTA 0 (diagnostics): of the looping kernel's
 // instrumented instantiation (STAMP), or of the persistent kernel further down.
 __device__ long long g_fwd_phase_cycles[16];
+__device__ long long g_fwd_timeline[1024][4];   // STAMP: per CTA: global timer at entry, first tiles in, loop end; SM id
+__device__ __forceinline__ long long gtime_f() { long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
 #define HDT_LSTAMP(i)                                                              \
     do {                                                                           \
         if constexpr (STAMP) {                                                     \
@@ -495,6 +497,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
 
     const int tid = threadIdx.x, warp = tid >> 5;
     const int H = a.H, G = gridDim.x;
+    if constexpr (STAMP) { if (tid == 0 && blockIdx.x < 1024) { g_fwd_timeline[blockIdx.x][0] = gtime_f(); unsigned sm_; asm("mov.u32 %0, %%smid;" : "=r"(sm_)); g_fwd_timeline[blockIdx.x][3] = sm_; g_fwd_timeline[blockIdx.x][1] = 0; g_fwd_timeline[blockIdx.x][2] = 0; } }
     // Counts not yet known to the host (the index build is still in flight when this kernel is
     // queued): they are read from the index header, and the partial buffers of stage 1 are laid
     // out from its element count the way the host does it (results, then LSE, 256-byte aligned).
@@ -517,22 +520,6 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
     const int n_items = n_fused * H;
     const float NEG = -INFINITY, LN2 = 0.6931471805599453f;
 
-    if (tid == 0) {
-        mbar_init(bar_qk, 1);
-        mbar_init(bar_v, 1);
-        mbar_init(bar_mma, 1);
-        *abort_flag = (*a.status != 0);
-        fence_mbar_init();
-    }
-    if (warp == 0) tmem_alloc(slot, TM_COLS);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *slot;
-    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
-    const bool dead = (*abort_flag != 0);
-    bool ok = true;
-
     struct Desc { int r0, r1, ka, kb, h; };
     auto load_desc = [&](int item) {
         Desc d{0, 0, 0, 0, 0};
@@ -554,9 +541,30 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
         for (int s = 0; s < NSUB; ++s) tma_load_3d(sV + s * SUB, &tm_v, 64 * s, d.h, d.ka, bar_v);
     };
 
+    if (tid == 0) {
+        mbar_init(bar_qk, 1);
+        mbar_init(bar_v, 1);
+        mbar_init(bar_mma, 1);
+        fence_mbar_init();
+        // the first item's tiles are requested before anything else is set up
+        if ((int)blockIdx.x < n_items) {
+            const Desc d = load_desc((int)blockIdx.x);
+            issue_qk(d);
+            issue_v(d);
+        }
+        *abort_flag = (*a.status != 0);
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)(warp * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    bool ok = true;
+
     if (!dead && (int)blockIdx.x < n_items) {
         Desc dc = load_desc((int)blockIdx.x), dn = load_desc((int)blockIdx.x + G);
-        if (tid == 0) { issue_qk(dc); issue_v(dc); }
         uint32_t ph = 0;           // phase of bar_qk and bar_v (one completion of each per item)
         uint32_t ph_mma = 0;
         long long t_last = STAMP ? clock64() : 0;
@@ -588,6 +596,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             HDT_LSTAMP(0);
             ok = mbar_wait(bar_qk, ph, abort_flag, WAIT_CYCLES) && ok;
             HDT_LSTAMP(1);
+            if constexpr (STAMP) { if (tid == 0 && item == (int)blockIdx.x && blockIdx.x < 1024) g_fwd_timeline[blockIdx.x][1] = gtime_f(); }
             if (tid == 0 && !*abort_flag) {
                 tc_fence_after();
                 const uint32_t idesc = idesc_bf16(Nc, false, false);
@@ -729,6 +738,12 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             dc = dn; dn = dn2;
         }
     }
+    if (dead && (int)blockIdx.x < n_items) {     // an earlier failure: only let the tiles requested above land
+        volatile int none = 0;
+        (void)mbar_wait(bar_qk, 0, &none, WAIT_CYCLES);
+        (void)mbar_wait(bar_v, 0, &none, WAIT_CYCLES);
+    }
+    if constexpr (STAMP) { if (tid == 0 && blockIdx.x < 1024) g_fwd_timeline[blockIdx.x][2] = gtime_f(); }
     if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
     tc_fence_before();
     __syncthreads();
@@ -989,6 +1004,11 @@ __global__ void __launch_bounds__(512, 1) k_fwd_tc_p(const __grid_constant__ CUt
 }
 
 // Diagnostics: cycles CTA 0 of the persistent forward spent per phase since the last call.
+int read_fwd_timeline(long long *out4096) {
+    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out4096, g_fwd_timeline, sizeof(long long) * 4096));
+    return HDT_OK;
+}
+
 int read_fwd_phase_cycles(long long *out16) {
     HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out16, g_fwd_phase_cycles, sizeof(long long) * 16));
     long long zero[16] = {0};

@@ -82,24 +82,6 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
         if (tid == 0) atomicCAS(a.status, 0, HDT_ERR_CUDA);
         return;
     }
-    if (tid == 0) {
-        mbar_init(bar_in, 1);
-        mbar_init(bar_a, 2);
-        mbar_init(bar_b, 3);
-        *abort_flag = (*a.status != 0);
-        fence_mbar_init();
-    }
-    if (warp == 0) tmem_alloc(slot, TM_COLS);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem = *slot;
-    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
-    const bool dead = (*abort_flag != 0);
-    bool ok = true;
-    const bool issuer = ((tid & 31) == 0) && warp < 3;
-    const bool store_thread = ((tid & 31) == 0) && warp >= 2;     // six threads: two boxes per gradient tensor
-
     // Item i of this CTA is entry blockIdx.x + i * G of queue_split x heads.  Its block number is
     // read three items ahead and its record two items ahead, so that no load in the loop waits for
     // another one.
@@ -120,6 +102,26 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
         tma_load_3d(sV, &tm_v, 0, d.h, d.r0, bar_in);
         tma_load_3d(sDO, &tm_do, 0, d.h, d.r0, bar_in);
     };
+    if (tid == 0) {
+        mbar_init(bar_in, 1);
+        mbar_init(bar_a, 2);
+        mbar_init(bar_b, 3);
+        fence_mbar_init();
+        // the first item's tiles are requested before anything else is set up
+        if ((int)blockIdx.x < n_items) issue_loads(fetch((int)blockIdx.x, block_of((int)blockIdx.x)));
+        *abort_flag = (*a.status != 0);
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    bool ok = true;
+    const bool issuer = ((tid & 31) == 0) && warp < 3;
+    const bool store_thread = ((tid & 31) == 0) && warp >= 2;     // six threads: two boxes per gradient tensor
+
     struct RowStat { int lo, hi, up; float lse, dl; };
     auto load_stat = [&](const It &d) {
         RowStat r{0, 0, -1, 0.f, 0.f};
@@ -139,7 +141,6 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
         It d0 = fetch(i0, block_of(i0)), d1 = fetch(i0 + G, block_of(i0 + G));
         int b2 = block_of(i0 + 2 * G);
         RowStat rc = load_stat(d0);
-        if (tid == 0 && d0.valid) issue_loads(d0);
         long long t_last = STAMP ? clock64() : 0;
         for (int it = 0; d0.valid && !*abort_flag; ++it) {
             const int r0 = d0.r0, r1 = d0.r1, h = d0.h, nrows = r1 - r0;
@@ -341,6 +342,10 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
             if constexpr (STAMP) { if (tid == 0 && blockIdx.x == 0) atomicAdd((unsigned long long *)&g_bwd_t_phase_cycles[12], 1ull); }
             d0 = d1; d1 = d2; rc = rn; b2 = b3;
         }
+    }
+    if (dead && (int)blockIdx.x < n_items) {     // an earlier failure: only let the tiles requested above land
+        volatile int none = 0;
+        (void)mbar_wait(bar_in, 0, &none, WAIT_CYCLES);
     }
     if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
     if (store_thread) bulk_wait_read();

@@ -124,3 +124,10 @@ extern "C" int hdt_debug_bwd_timeline(int64_t *out2048) {
     HDT_CUDA_CHECK(cudaDeviceSynchronize());
     return hdt::read_bwd_t_timeline((long long *)out2048);
 }
+
+// The same for the looping forward (up to 1024 CTAs).
+extern "C" int hdt_debug_fwd_timeline(int64_t *out4096) {
+    if (!out4096) return hdt::set_error(HDT_ERR_INVALID_ARG, "hdt_debug_fwd_timeline: null pointer");
+    HDT_CUDA_CHECK(cudaDeviceSynchronize());
+    return hdt::read_fwd_timeline((long long *)out4096);
+}

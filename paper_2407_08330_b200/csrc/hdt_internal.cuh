@@ -207,6 +207,7 @@ int read_bwd_phase_cycles(long long *out16);
 int read_bwd_t_phase_cycles(long long *out16);   // adds to out16
 int read_bwd_t_timeline(long long *out2048);     // per CTA of the last instrumented launch: entry, first tiles in, end (ns), SM
 int read_fwd_phase_cycles(long long *out16);
+int read_fwd_timeline(long long *out4096);       // per CTA of the last instrumented looping forward: entry, first tiles in, end (ns), SM
 int launch_bwd_simt(const BwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 int launch_delta(const void *o, const void *d_o, float *delta, int T, int H, int head_dim, int dtype,
                  cudaStream_t st);
