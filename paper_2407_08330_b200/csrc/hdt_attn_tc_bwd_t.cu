@@ -29,6 +29,12 @@ constexpr int SUB = 16384;
 constexpr long long WAIT_CYCLES = 400000000LL;
 __device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
 
+// 16 bytes read once: not kept in L1 (which shares its storage with the tiles in shared memory)
+__device__ __forceinline__ uint4 ld_stream(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
 }  // namespace
 
 // TMEM columns.  S^T occupies 0..127 and dP^T 128..255 until the keys have turned them into P^T and
@@ -52,8 +58,8 @@ __device__ __forceinline__ long long gtime() { long long t; asm volatile("mov.u6
     } while (0)
 
 // FD (fused delta): a.delta is not read; delta[query] = dO[query] . O[query] is computed here: eight
-// lanes per token row, 16 bytes each of O and dO, requested at the top of the item and reduced once
-// S^T and dP^T are there.
+// lanes per token row, 16 bytes each of O and dO, requested at the top of the item (past L1) and
+// reduced once S^T and dP^T are there.  (dO from its tile in shared memory instead: 8 % slower.)
 template <bool DIRS, bool STAMP = false, bool FD = false>
 __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
@@ -154,8 +160,8 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
                     xg[k] = make_uint4(0u, 0u, 0u, 0u);
                     if (r < nrows) {
                         const size_t off = ((size_t)(r0 + r) * H + h) * D + (tid & 7) * 8;
-                        xo[k] = *reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.o) + off);
-                        xg[k] = *reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.d_o) + off);
+                        xo[k] = ld_stream(reinterpret_cast<const __nv_bfloat16 *>(a.o) + off);
+                        xg[k] = ld_stream(reinterpret_cast<const __nv_bfloat16 *>(a.d_o) + off);
                     }
                 }
             }
