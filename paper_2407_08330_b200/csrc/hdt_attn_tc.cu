@@ -482,7 +482,8 @@ __device__ __forceinline__ long long gtime_f() { long long t; asm volatile("mov.
 template <int D, bool DIRS = false, bool STAMP = false>
 __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
-                                                     const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
+                                                     const __grid_constant__ CUtensorMap tm_v,
+                                                     const __grid_constant__ OutMaps om, const FwdStageArgs a) {
     constexpr int NSUB = D / 64;
     // S (N <= 128 columns); P (bf16, two per column) is written over its first half as the rows are
     // exponentiated and is the A operand of O = P V; O lies beside it
@@ -595,6 +596,10 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
 
             HDT_LSTAMP(0);
             ok = mbar_wait(bar_qk, ph, abort_flag, WAIT_CYCLES) && ok;
+            if (tid == 32 && item != (int)blockIdx.x) {      // V of this item, into the tile the previous item's stores read
+                bulk_wait_read();
+                if (!*abort_flag) issue_v(dc);
+            }
             HDT_LSTAMP(1);
             if constexpr (STAMP) { if (tid == 0 && item == (int)blockIdx.x && blockIdx.x < 1024) g_fwd_timeline[blockIdx.x][1] = gtime_f(); }
             if (tid == 0 && !*abort_flag) {
@@ -715,29 +720,34 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
                         make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
             }
             if (inb) a.lse[(size_t)h * a.T + row] = lse;
+            fence_proxy_async_smem();
             tc_fence_before();
             HDT_LSTAMP(7);
             __syncthreads();
             HDT_LSTAMP(8);
-            {
-                __nv_bfloat16 *og = reinterpret_cast<__nv_bfloat16 *>(a.o);
+            // The staged rows leave through TMA stores: rows [0, nrows) as at most two boxes of b rows, b
+            // the largest power of two <= min(nrows, 64) (where the two overlap the same values are
+            // written twice).  One thread of warp 1 requests them; at the top of the next item, once it
+            // has seen that item's Q and K arrive, it waits until the stores have read the tile and
+            // requests V into it.  (Not here: a thread that lags behind the others by that wait could
+            // miss a phase of the Q / K barrier, which thread 0 re-arms as soon as S is there.)
+            if (tid == 32 && !*abort_flag) {
                 const int nrows = r1 - r0;
-                for (int idx = tid; idx < NSUB * 128 * 8; idx += 128) {
-                    const int t = idx >> 10, rem = idx & 1023, r = rem >> 3, c = rem & 7;
-                    if (r < nrows) {
-                        const uint4 v = *reinterpret_cast<const uint4 *>(sV + t * SUB + swz(r, c));
-                        *reinterpret_cast<uint4 *>(og + ((size_t)(r0 + r) * H + h) * D + t * 64 + c * 8) = v;
-                    }
+                const int bx = max(__clz(nrows) - 25, 0);          // box of 64 >> bx rows: 64 for nrows >= 64
+                const int b = 64 >> bx;
+                for (int s2 = 0; s2 < NSUB; ++s2) {
+                    tma_store_3d(&om.m[bx], 64 * s2, h, r0, sV + s2 * SUB);
+                    if (nrows > b) tma_store_3d(&om.m[bx], 64 * s2, h, r0 + nrows - b, sV + s2 * SUB + (nrows - b) * 128);
                 }
+                bulk_commit();
             }
             HDT_LSTAMP(9);
-            __syncthreads();   // the staged O has been read: the V tile may be overwritten
             HDT_LSTAMP(10);
             if constexpr (STAMP) { if (tid == 0 && blockIdx.x == 0) atomicAdd((unsigned long long *)&g_fwd_phase_cycles[12], 1ull); }
-            if (tid == 0 && have_next && !*abort_flag) issue_v(dn);
             dc = dn; dn = dn2;
         }
     }
+    if (tid == 32) bulk_wait_read();       // the last item's stores have read the tile
     if (dead && (int)blockIdx.x < n_items) {     // an earlier failure: only let the tiles requested above land
         volatile int none = 0;
         (void)mbar_wait(bar_qk, 0, &none, WAIT_CYCLES);
@@ -1025,6 +1035,11 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     if (rc) return rc;
     rc = make_tmap_bf16(&tv, a.v, D, a.H, a.T, 128);
     if (rc) return rc;
+    OutMaps om;      // the looping kernel's output tiles leave through TMA stores (boxes of 64 .. 1 rows)
+    for (int bx = 0; bx < 7; ++bx) {
+        rc = make_tmap_bf16(&om.m[bx], a.o, D, a.H, a.T, 64 >> bx);
+        if (rc) return rc;
+    }
     constexpr int smem = (4 * (D / 64) + 2) * SUB + 1024 + 64;     // general kernel: Q, two K tiles, V, P
     constexpr int smem_1 = 3 * (D / 64) * SUB + 1024 + 64;
     static bool attr = false;
@@ -1047,8 +1062,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
             HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm_e, cudaDevAttrMultiProcessorCount, dev));
         }
         const int grid = n_sm_e * (D == 64 ? 4 : 2);
-        if (dirs) k_fwd_tc_loop<D, true><<<grid, 128, smem_1, st>>>(tq, tk, tv, a);
-        else k_fwd_tc_loop<D><<<grid, 128, smem_1, st>>>(tq, tk, tv, a);
+        if (dirs) k_fwd_tc_loop<D, true><<<grid, 128, smem_1, st>>>(tq, tk, tv, om, a);
+        else k_fwd_tc_loop<D><<<grid, 128, smem_1, st>>>(tq, tk, tv, om, a);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
         return HDT_OK;
@@ -1079,15 +1094,15 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
             }
             const long long items = (long long)a.n_fused * a.H;
             const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
-            if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
+            if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
             else if (g_phase_stamps && D == 64) {
                 static bool attr_s = false;
                 if (!attr_s) {
                     HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
                     attr_s = true;
                 }
-                k_fwd_tc_loop<64, false, true><<<(int)(items < slots ? items : slots), 128, 3 * SUB + 1024 + 64, st>>>(tq, tk, tv, a);
-            } else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, a);
+                k_fwd_tc_loop<64, false, true><<<(int)(items < slots ? items : slots), 128, 3 * SUB + 1024 + 64, st>>>(tq, tk, tv, om, a);
+            } else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
         }
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());

@@ -45,6 +45,7 @@ inline int make_tmap_bf16(CUtensorMap *tm, const void *base, int D, int H, long 
 // with boxes of 64, 32, ..., 1 rows and a tile is stored as two (possibly overlapping) boxes of the
 // largest size that fits.
 struct StoreMaps { CUtensorMap m[3][7]; };
+struct OutMaps { CUtensorMap m[7]; };     // the same for one tensor (the forward's O)
 
 // Self-contained (SELF, non-EMPTY) blocks of stage 0 at head_dim 64 through the transposed looping
 // backward (hdt_attn_tc_bwd_t.cu); the maps are those of q, k, v, dO with boxes of 128 rows.

@@ -166,3 +166,31 @@ def test_deferred_full_size_sampled(P):
     for x in (o, dq, dk, dv):
         assert torch.isfinite(x.float()).all()
     P.hdt_device_status()
+
+
+def test_many_steps_no_expired_wait_and_same_bytes(P):
+    """300 steps of the benchmark's forward configuration (deferred build, caller workspace, L2 flushed
+    in between): no bounded wait of a kernel runs out (a thread of the looping forward that lags behind
+    the others by more than an item would miss a phase of a re-armed barrier) and every step writes the
+    same bytes."""
+    c = 3
+    cfg = gen.CONFIGS[c]
+    b = gen.make_hierarchy(c)
+    T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
+    t = gen.make_tensors(cfg.tensor_seed, T, H, d, cfg.dtype)
+    q, k, v = (dev_tensor(t[n], cfg.dtype) for n in ("q", "k", "v"))
+    ws = attn_ws(P, b, H, d, cfg.dtype, 0)
+    st = dev_struct(b)
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda")
+    o0 = lse0 = None
+    for i in range(300):
+        flush.zero_()
+        idx = P.hdt_build_index(*st, max_stages=4, deferred=True)
+        o, lse = P.hdt_attn_fwd(idx, q, k, v, workspace=ws)
+        if i % 50 == 0:
+            P.hdt_device_status()
+            if o0 is None:
+                o0, lse0 = o.clone(), lse.clone()
+            else:
+                assert torch.equal(o, o0) and torch.equal(lse, lse0)
+    P.hdt_device_status()
