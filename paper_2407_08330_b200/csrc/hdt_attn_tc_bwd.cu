@@ -478,7 +478,8 @@ template <int D>
 __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ CUtensorMap tm_q,
                                                         const __grid_constant__ CUtensorMap tm_k,
                                                         const __grid_constant__ CUtensorMap tm_v,
-                                                        const __grid_constant__ CUtensorMap tm_do, const BwdStageArgs a) {
+                                                        const __grid_constant__ CUtensorMap tm_do,
+                                                        const __grid_constant__ StoreMaps sm_out, const BwdStageArgs a) {
     constexpr int NSUB = D / 64;
     constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DV = 0, TM_DK = 128, TM_DQ = 256, TM_COLS = 512;
     extern __shared__ uint8_t smem_raw[];
@@ -513,6 +514,7 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
     bool ok = true;
     // MMAs are issued by lane 0 of warps 0, 1, 2 side by side (a thread needs about 100 cycles per MMA)
     const bool issuer = ((tid & 31) == 0) && warp < 3;
+    const bool store_thread = ((tid & 31) == 0) && warp >= 2;     // six threads: two boxes per gradient tensor
 
     struct It { int valid, r0, r1, h; };
     auto fetch = [&](int i) {
@@ -582,6 +584,9 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
             const int jl = max(rc.lo - r0, 0), jh = min(rc.hi - r0, nrows);
             const bool has = inq && jh > jl;
             ok = mbar_wait(bar_a, it & 1, abort_flag, WAIT_CYCLES) && ok;
+            // the previous item's staged gradients have left shared memory before P and dS overwrite them
+            if (store_thread) bulk_wait_read();
+            __syncthreads();
             tc_fence_after();
 #pragma unroll
             for (int sl = 0; sl < 2; ++sl) {
@@ -677,26 +682,28 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
                     }
                 }
             }
+            fence_proxy_async_smem();
             tc_fence_before();
             __syncthreads();
-            {
-                __nv_bfloat16 *g[3] = {(__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv};
-                const uint8_t *srcs[3] = {sP, sDS, sStg};
-#pragma unroll
-                for (int t = 0; t < 3; ++t)
-                    for (int idx = tid; idx < NSUB * 128 * 8; idx += 256) {
-                        const int u = idx >> 10, rem = idx & 1023, r = rem >> 3, c = rem & 7;
-                        if (r < nrows) {
-                            const uint4 v = *reinterpret_cast<const uint4 *>(srcs[t] + u * SUB + swz(r, c));
-                            *reinterpret_cast<uint4 *>(g[t] + ((size_t)(r0 + r) * H + h) * D + u * 64 + c * 8) = v;
-                        }
-                    }
+            // TMA stores: rows [0, nrows) of each staged tile as at most two boxes of b rows, b the largest
+            // power of two <= min(nrows, 64): [0, b) and [nrows - b, nrows); where the two overlap the same
+            // values are written twice.  They read shared memory until the next item's arithmetic is
+            // about to overwrite it.
+            if (store_thread && !*abort_flag) {
+                const int t = (warp - 2) >> 1, second = (warp - 2) & 1;
+                const int bx = max(__clz(nrows) - 25, 0);          // box of 64 >> bx rows: 64 for nrows >= 64
+                const int b = 64 >> bx;
+                const int off = second ? nrows - b : 0;
+                const uint8_t *src = (t == 0) ? sP : (t == 1) ? sDS : sStg;
+                if (!second || nrows > b)
+                    for (int u = 0; u < NSUB; ++u) tma_store_3d(&sm_out.m[t][bx], 64 * u, h, r0 + off, src + u * SUB + off * 128);
+                bulk_commit();
             }
-            __syncthreads();     // the staged tiles are read before the next item's P and dS overwrite them
             d0 = d1; d1 = d2; rc = rn;
         }
     }
     if (!ok && tid == 0) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+    if (store_thread) bulk_wait_read();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
@@ -1099,6 +1106,15 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     b.rest_only = 0;
     int n_general = a.nb;
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
+    StoreMaps outs;                  // the looping and persistent kernels store through TMA
+    {
+        void *outp[3] = {a.dq, a.dk, a.dv};
+        for (int t = 0; t < 3; ++t)
+            for (int bx = 0; bx < 7; ++bx) {
+                rc = make_tmap_bf16(&outs.m[t][bx], outp[t], D, a.H, a.T, 64 >> bx);
+                if (rc) return rc;
+            }
+    }
     if (D == 64 && a.nb > 0 && (!a.no_persistent || a.no_persistent == 4 || a.no_persistent == 6)) {   // (no_persistent == 5: the looping kernel below instead)
         // the persistent kernel takes everything: first the blocks of split families (longest first),
         // then the self-contained blocks
@@ -1115,13 +1131,6 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
             HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
             attr_p = true;
         }
-        StoreMaps outs;
-        void *outp[3] = {a.dq, a.dk, a.dv};
-        for (int t = 0; t < 3; ++t)
-            for (int bx = 0; bx < 7; ++bx) {
-                rc = make_tmap_bf16(&outs.m[t][bx], outp[t], D, a.H, a.T, 64 >> bx);
-                if (rc) return rc;
-            }
         for (int mode = 1; mode >= 0; --mode) {
             const long long units = (long long)(mode ? a.nb - a.n_fused : a.n_fused) * a.H;
             if (units == 0) continue;
@@ -1156,7 +1165,7 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
             attr_l = true;
         }
         const long long items = (long long)a.n_fused * a.H;
-        k_bwd_tc_loop<D><<<(int)(items < n_sm_l ? items : n_sm_l), 256, smem_l, st>>>(tq, tk, tv, tdo, a);
+        k_bwd_tc_loop<D><<<(int)(items < n_sm_l ? items : n_sm_l), 256, smem_l, st>>>(tq, tk, tv, tdo, outs, a);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
         b.rest_only = 1;
