@@ -921,7 +921,18 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     ix->max_stages = ms;
     ix->pending = 1;
     {
-        const cudaError_t e_ = cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, st);
+        // A deferred build leaves the caller's stream free for the attention kernel that follows: the
+        // copy goes to the side stream, behind an event (the fallback wait of index_ready is then on
+        // that stream).  Compute -> copy -> compute on one stream costs the kernel behind the copy a
+        // few microseconds.
+        cudaStream_t cs = st;
+        Side *sdc = nullptr;
+        if (params && params->deferred && !g_no_overlap && get_side(&sdc) == HDT_OK && sdc != nullptr &&
+            cudaEventRecord(sdc->fork, st) == cudaSuccess && cudaStreamWaitEvent(sdc->s, sdc->fork, 0) == cudaSuccess) {
+            cs = sdc->s;
+            ix->stream = cs;
+        }
+        const cudaError_t e_ = cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, cs);
         if (e_ != cudaSuccess) {
             pinned_release(h_pinned);
             delete ix;
