@@ -48,7 +48,7 @@ ProfScope::~ProfScope() {
 }
 
 // ---- device-side failure word -------------------------------------------------------------------
-__device__ int g_device_status = 0;  // first failure recorded by a kernel (hdt_status_t), 0 = none
+__device__ int g_device_status[4] = {0, 0, 0, 0};  // [0] first failure recorded by a kernel (hdt_status_t), 0 = none; [1] where (kernel << 8 | wait site), [2] its loop count
 
 int *device_status_ptr() {
     int *p = nullptr;
@@ -153,12 +153,13 @@ extern "C" int64_t hdt_launch_count(void) { return (int64_t)g_launches.load(); }
 // Waits for `stream`, then returns and clears the first failure recorded by a kernel.
 extern "C" int hdt_device_status(void *stream) {
     HDT_CUDA_CHECK(cudaStreamSynchronize((cudaStream_t)stream));
-    int h = 0;
-    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(&h, g_device_status, sizeof(int)));
-    if (h != 0) {
-        const int zero = 0;
-        HDT_CUDA_CHECK(cudaMemcpyToSymbol(g_device_status, &zero, sizeof(int)));
-        return set_error(h, "a kernel recorded device-side failure %d (a bounded wait ran out)", h);
+    int h[4] = {0, 0, 0, 0};
+    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(h, g_device_status, sizeof(h)));
+    if (h[0] != 0) {
+        const int zero[4] = {0, 0, 0, 0};
+        HDT_CUDA_CHECK(cudaMemcpyToSymbol(g_device_status, zero, sizeof(zero)));
+        return set_error(h[0], "a kernel recorded device-side failure %d (a bounded wait ran out; kernel %d, wait %d, loop count %d)",
+                         h[0], h[1] >> 8, h[1] & 255, h[2]);
     }
     return HDT_OK;
 }

@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                         for (int s = 0; s < NSUB; ++s) tma_load_3d(kn + s * SUB, &tm_k, 64 * s, h, c0 + 128, bn);
                     }
                 }
-                ok = mbar_wait((ci & 1) ? bar_k1 : bar_tma, (ci >> 1) & 1, abort_flag, WAIT_CYCLES) && ok;
+                if (!mbar_wait((ci & 1) ? bar_k1 : bar_tma, (ci >> 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (1 << 8) | 1; }
             } else {
                 if (tid == 0 && !*abort_flag) {   // after a failed wait nothing new is issued
                     mbar_expect_tx(bar_tma, (uint32_t)((first ? NSUB : 0) + 2 * NSUB) * SUB);
@@ -188,7 +188,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                         tma_load_3d(sV + s * SUB, &tm_v, 64 * s, h, c0, bar_tma);
                     }
                 }
-                ok = mbar_wait(bar_tma, ph_tma, abort_flag, WAIT_CYCLES) && ok;
+                if (!mbar_wait(bar_tma, ph_tma, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (1 << 8) | 2; }
                 ph_tma ^= 1;
             }
             if (tid == 0 && !*abort_flag) {
@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                 }
                 mma_commit(bar_mma);
             }
-            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            if (!mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (1 << 8) | 3; }
             ph_mma ^= 1;
             tc_fence_after();
 
@@ -292,7 +292,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
                 }
                 mma_commit(bar_mma);
             }
-            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            if (!mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (1 << 8) | 4; }
             ph_mma ^= 1;
             tc_fence_after();
             if constexpr (PIPE) {
@@ -595,7 +595,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             const int nvalid = min(128, kb - ka), Nc = (nvalid + 15) & ~15;
 
             HDT_LSTAMP(0);
-            ok = mbar_wait(bar_qk, ph, abort_flag, WAIT_CYCLES) && ok;
+            if (!mbar_wait(bar_qk, ph, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) { a.status[1] = (2 << 8) | 1; a.status[2] = item; } }
             if (tid == 32 && item != (int)blockIdx.x) {      // V of this item, into the tile the previous item's stores read
                 bulk_wait_read();
                 if (!*abort_flag) issue_v(dc);
@@ -612,11 +612,10 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
                 }
                 mma_commit(bar_mma);
             }
-            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            if (!mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) { a.status[1] = (2 << 8) | 2; a.status[2] = item; } }
             ph_mma ^= 1;
             tc_fence_after();
             HDT_LSTAMP(2);
-            if (tid == 0 && have_next && !*abort_flag) issue_qk(dn);   // S is there: Q, K of the next item
 
             // ---- masked softmax of this row (one chunk: no running maximum needed) ----
             const int jl = max(lo - ka, 0), jh = min(hi - ka, nvalid);
@@ -676,7 +675,10 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             HDT_LSTAMP(4);
             __syncthreads();
             HDT_LSTAMP(5);
-            ok = mbar_wait(bar_v, ph, abort_flag, WAIT_CYCLES) && ok;
+            // Q, K of the next item (S has consumed the tiles; only after this barrier has every thread
+            // seen the current phase of their barrier, so that re-arming it cannot overtake anybody)
+            if (tid == 0 && have_next && !*abort_flag) issue_qk(dn);
+            if (!mbar_wait(bar_v, ph, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) { a.status[1] = (2 << 8) | 3; a.status[2] = item; } }
             ph ^= 1;
             if (tid == 0 && !*abort_flag) {
                 tc_fence_after();
@@ -685,7 +687,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
                     mma_ts(tmem + TM_O, tmem + 8 * kk, smem_desc(smem_u32(sV) + kk * 2048, SUB, 1024), idesc, kk > 0);
                 mma_commit(bar_mma);
             }
-            ok = mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES) && ok;
+            if (!mbar_wait(bar_mma, ph_mma, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) { a.status[1] = (2 << 8) | 4; a.status[2] = item; } }
             ph_mma ^= 1;
             tc_fence_after();
             HDT_LSTAMP(6);
