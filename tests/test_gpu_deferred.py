@@ -169,28 +169,31 @@ def test_deferred_full_size_sampled(P):
 
 
 def test_many_steps_no_expired_wait_and_same_bytes(P):
-    """300 steps of the benchmark's forward configuration (deferred build, caller workspace, L2 flushed
-    in between): no bounded wait of a kernel runs out (a thread of the looping forward that lags behind
-    the others by more than an item would miss a phase of a re-armed barrier) and every step writes the
-    same bytes."""
+    """800 steps of the benchmark's configuration (deferred build, caller workspaces, forward and backward,
+    L2 flushed in between): no bounded wait of a kernel runs out (a thread of a looping kernel that
+    reaches its wait on a barrier after the barrier has been re-armed twice waits for a phase that has
+    passed; seen once in fifteen and once in a thousand steps while the looping forward was rebuilt)
+    and every step writes the same bytes."""
     c = 3
     cfg = gen.CONFIGS[c]
     b = gen.make_hierarchy(c)
     T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
     t = gen.make_tensors(cfg.tensor_seed, T, H, d, cfg.dtype)
-    q, k, v = (dev_tensor(t[n], cfg.dtype) for n in ("q", "k", "v"))
-    ws = attn_ws(P, b, H, d, cfg.dtype, 0)
+    q, k, v, do = (dev_tensor(t[n], cfg.dtype) for n in ("q", "k", "v", "do"))
+    ws_f, ws_b = attn_ws(P, b, H, d, cfg.dtype, 0), attn_ws(P, b, H, d, cfg.dtype, 1)
     st = dev_struct(b)
     flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda")
-    o0 = lse0 = None
-    for i in range(300):
+    first = None
+    for i in range(800):
         flush.zero_()
         idx = P.hdt_build_index(*st, max_stages=4, deferred=True)
-        o, lse = P.hdt_attn_fwd(idx, q, k, v, workspace=ws)
-        if i % 50 == 0:
+        o, lse = P.hdt_attn_fwd(idx, q, k, v, workspace=ws_f)
+        dq, dk, dv = P.hdt_attn_bwd(idx, q, k, v, o, lse, do, workspace=ws_b)
+        if i % 100 == 0:
             P.hdt_device_status()
-            if o0 is None:
-                o0, lse0 = o.clone(), lse.clone()
+            if first is None:
+                first = [x.clone() for x in (o, lse, dq, dk, dv)]
             else:
-                assert torch.equal(o, o0) and torch.equal(lse, lse0)
+                for x, y in zip((o, lse, dq, dk, dv), first):
+                    assert torch.equal(x, y)
     P.hdt_device_status()
