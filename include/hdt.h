@@ -301,7 +301,8 @@ int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const i
  * = 6 gives the latter one CTA per SM; "no_fused_delta" = 1 runs the delta pass even where every
  * backward kernel of the call could compute dO . O itself; "no_fold" bit 0 = 1 lets a merge
  * kernel complete the elements of stage 1 in the forward instead of the stage-1 kernel itself, bit 2
- * = 1 makes the backward's stage-1 kernel do it (off by default); "phase_stamps" = 1 selects the
+ * = 1 makes the backward's stage-1 kernel do it (off by default); "no_pdl" = 1 launches the kernels of hdt_build_index as ordinary stream
+ * successors instead of programmatic dependents; "phase_stamps" = 1 selects the
  * instrumented instantiation of the transposed looping backward (see hdt_debug_bwd_timeline).
  */
 int hdt_set_option(const char *name, int32_t value);

@@ -120,6 +120,8 @@ __global__ void k_init(const int8_t *__restrict__ level, const int32_t *__restri
 }
 
 __global__ void k_count(const DevHeader *hdr, int s, const int *__restrict__ par, int *cnt) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
         const int p = par[e];
@@ -129,6 +131,8 @@ __global__ void k_count(const DevHeader *hdr, int s, const int *__restrict__ par
 
 __global__ void k_nlc(const DevHeader *hdr, int s, const int *__restrict__ par,
                       const int *__restrict__ cnt, int *nlc) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
         const int p = par[e];
@@ -151,6 +155,8 @@ __global__ void __launch_bounds__(CHUNK)
 k_ranges(DevHeader *hdr, int s, const int8_t *__restrict__ level /* stage 0 only */,
          const int *__restrict__ par, const int *__restrict__ cnt, const int *__restrict__ nlc,
          int *rng, uint8_t *keep, uint8_t *fpos, int *blocksum, int dirs) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
     const int e = blockIdx.x * CHUNK + threadIdx.x;
     int kp = 0;
@@ -210,6 +216,8 @@ k_ranges(DevHeader *hdr, int s, const int8_t *__restrict__ level /* stage 0 only
 __global__ void __launch_bounds__(CHUNK)
 k_scan(DevHeader *hdr, int s, int nchunk_cap, const uint8_t *__restrict__ keep,
        const int *__restrict__ blocksum, const int *__restrict__ tok, int *pre, int *up, int *tok2) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
     const int nchunk = (n + CHUNK - 1) / CHUNK;
     if ((int)blockIdx.x >= nchunk && blockIdx.x != 0) return;
@@ -273,6 +281,8 @@ k_scan(DevHeader *hdr, int s, int nchunk_cap, const uint8_t *__restrict__ keep,
 __global__ void k_compact(const DevHeader *hdr, int s, int B, const int *__restrict__ par,
                           const int *__restrict__ up, const int *__restrict__ pre,
                           const int *__restrict__ scu, int *par2, int *scu2, int *cnt, int *nlc) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n, n2 = hdr->st[s + 1].n;
     const int gtid = blockIdx.x * blockDim.x + threadIdx.x, gsz = gridDim.x * blockDim.x;
     for (int e = gtid; e < n; e += gsz) {
@@ -293,6 +303,8 @@ __global__ void k_compact(const DevHeader *hdr, int s, int B, const int *__restr
 // (0 for heads and for elements in no family, capped at 255 >= block_m).
 __global__ void k_walk(const DevHeader *hdr, int s, int bm, const int *__restrict__ scu,
                        const uint8_t *__restrict__ fpos, int *bstart, int *seqcount, int smem_cap) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     extern __shared__ __align__(16) uint8_t s_fp[];
     const int n = hdr->st[s].n;
     const int b = blockIdx.x;
@@ -343,6 +355,8 @@ __global__ void k_blocks(DevHeader *hdr, int s, int bm, int B, const int *__rest
                          const int *__restrict__ bstart, const int *__restrict__ seqcount,
                          const int *__restrict__ rng, const int *__restrict__ up, int *blocks,
                          long long *cost) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
     const int b = blockIdx.x;
     if (s > 0 && n == 0) return;
@@ -417,6 +431,8 @@ __global__ void k_blocks(DevHeader *hdr, int s, int bm, int B, const int *__rest
 __global__ void __launch_bounds__(256)
 k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost, const int *__restrict__ blocks, int *queue,
         int *queue_split) {
+    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
+    pdl_wait();                   // the kernel before this one has completed
     const int nb = hdr->st[s].nb;
     const int lane = threadIdx.x & 31;
     const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nw = (gridDim.x * blockDim.x) >> 5;
@@ -709,6 +725,24 @@ extern "C" size_t hdt_index_workspace_bytes(int32_t batch, int32_t total_tokens,
     return make_layout(batch, total_tokens, min(bm, bmu), ms).total;
 }
 
+// Launch as a programmatic dependent of the kernel before it on the stream (its CTAs are scheduled
+// while that kernel ends and wait for it with pdl_wait): the dozen tiny kernels of a build are a
+// chain, and most of each link is launch latency.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = g_no_pdl ? 0 : 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Pinned landing buffers for index headers: a small pool shared by all host threads (a deferred
 // index keeps its buffer until the header has been read).
 static const int kUnset = 0x7fffffff;
@@ -834,16 +868,16 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             // the last possible stage writes its (unused) next-stage arrays into its own up/pre scratch
             const StagePtrs &N = ix->st[(s + 1 < ms) ? s + 1 : s];
             const bool last = (s + 1 == ms);
-            if (s >= 1) { k_count<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt); ++n_launched; }
-            k_nlc<<<g_stride, 256, 0, st>>>(hdr, s, P.par, cnt, nlc);
-            k_ranges<<<g_chunk, CHUNK, 0, st>>>(hdr, s, s == 0 ? level : nullptr, P.par, cnt, nlc, P.rng, keep,
-                                                fpos, blocksum, dirs);
+            if (s >= 1) { HDT_ENQ(launch_chain(k_count, dim3(g_stride), dim3(256), 0, st, hdr, s, P.par, cnt)); ++n_launched; }
+            HDT_ENQ(launch_chain(k_nlc, dim3(g_stride), dim3(256), 0, st, hdr, s, P.par, cnt, nlc));
+            HDT_ENQ(launch_chain(k_ranges, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, s == 0 ? level : (const int8_t *)nullptr, P.par, cnt, nlc,
+                                 P.rng, keep, fpos, blocksum, dirs));
             // tok2 of the last possible stage is never read: point it at scratch (pre is rewritten first)
-            k_scan<<<g_chunk, CHUNK, 0, st>>>(hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
-                                              last ? cnt : N.tok);
+            HDT_ENQ(launch_chain(k_scan, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
+                                 last ? cnt : N.tok));
             n_launched += 3;
             if (!last) {
-                k_compact<<<g_stride, 256, 0, st>>>(hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc);
+                HDT_ENQ(launch_chain(k_compact, dim3(g_stride), dim3(256), 0, st, hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc));
                 ++n_launched;
                 if (s == 0 && sd) {   // fork: the upper stages start now
                     HDT_ENQ(cudaEventRecord(sd->fork, st));
@@ -855,10 +889,10 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             if (B > 0) {
                 int maxlen_smem = kSmemCap;  // sequences longer than this walk through global memory
                 const int bms = (s == 0) ? bm : bmu;
-                k_walk<<<B, 256, kSmemCap, st>>>(hdr, s, bms, P.scu, fpos, bstart, seqcount, maxlen_smem);
+                HDT_ENQ(launch_chain(k_walk, dim3(B), dim3(256), (size_t)kSmemCap, st, hdr, s, bms, P.scu, fpos, bstart, seqcount, maxlen_smem));
                 const int gy = max(1, min(64, 2048 / max(B, 1)));   // enough CTAs to spread a few long sequences
-                k_blocks<<<dim3(B, gy), 256, 0, st>>>(hdr, s, bms, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost);
-                k_queue<<<max(1, min(L.capnb / 8 + 1, 148 * 4)), 256, 0, st>>>(hdr, s, cost, P.blocks, P.queue, P.queue_split);
+                HDT_ENQ(launch_chain(k_blocks, dim3(B, gy), dim3(256), 0, st, hdr, s, bms, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost));
+                HDT_ENQ(launch_chain(k_queue, dim3(max(1, min(L.capnb / 8 + 1, 148 * 4))), dim3(256), 0, st, hdr, s, cost, P.blocks, P.queue, P.queue_split));
                 n_launched += 3;
             }
         }

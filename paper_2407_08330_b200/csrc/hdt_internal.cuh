@@ -87,6 +87,14 @@ extern int g_force_simt;   // option "force_simt"
 extern int g_no_graph;     // option "no_graph"
 extern int g_phase_stamps; // option "phase_stamps": the transposed backward runs its instrumented instantiation
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
+// be scheduled while the kernel before it on the stream still runs (once every CTA of that kernel
+// has called pdl_launch_dependents or has exited); pdl_wait then blocks until that kernel has
+// completed and its writes are visible.  Both are no-ops in a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+extern int g_no_pdl;       // option "no_pdl"
+
 // Direction bits inside a row range (paper, "Mathematical Reasoning Tasks": the ListOps attention
 // patterns).  Row e of a stage has the key range [lo, hi).  If the range starts at or after e, e is
 // the head of the family and the keys after it are its children; otherwise lo is e's parent and
