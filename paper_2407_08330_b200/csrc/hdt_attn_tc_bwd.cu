@@ -60,6 +60,65 @@ __device__ __forceinline__ void gather_tiles(uint8_t *const (&dst)[NTEN], const 
     }
 }
 
+// The same with delta = dO . O of every gathered row computed on the way (no delta pass ran): src[IDO]
+// is dO; the eight lanes that hold a row's chunks also fetch the chunks of its O row, multiply and
+// reduce, and lane 0 of the eight leaves the sum in s_delta[row - row0] (0 for rows at or beyond end).
+template <int D, int NT, int NTEN, int IDO>
+__device__ __forceinline__ void gather_tiles_delta(uint8_t *const (&dst)[NTEN], const void *const (&src)[NTEN], const void *o_rows,
+                                                   float *s_delta, const int *__restrict__ tok, int row0, int end, int H, int h,
+                                                   int tid) {
+    constexpr int RPP = NT / 8, NP = 128 / RPP, NSUB = D / 64;
+    const int c = tid & 7, rr = tid >> 3;
+    int tk[NP];
+    float acc[NP];
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        const int e = row0 + rr + p * RPP;
+        tk[p] = e < end ? tok[e] : -1;
+        acc[p] = 0.f;
+    }
+#pragma unroll
+    for (int t = 0; t < NSUB; ++t) {
+        uint4 v[NTEN][NP], vo[NP];
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            vo[p] = make_uint4(0u, 0u, 0u, 0u);
+            if (tk[p] >= 0)
+                vo[p] = *reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(o_rows) + ((size_t)tk[p] * H + h) * D + t * 64 + c * 8);
+        }
+#pragma unroll
+        for (int x = 0; x < NTEN; ++x) {
+            const __nv_bfloat16 *g = reinterpret_cast<const __nv_bfloat16 *>(src[x]);
+#pragma unroll
+            for (int p = 0; p < NP; ++p) {
+                v[x][p] = make_uint4(0u, 0u, 0u, 0u);
+                if (tk[p] >= 0) v[x][p] = *reinterpret_cast<const uint4 *>(g + ((size_t)tk[p] * H + h) * D + t * 64 + c * 8);
+            }
+        }
+#pragma unroll
+        for (int x = 0; x < NTEN; ++x)
+#pragma unroll
+            for (int p = 0; p < NP; ++p) *reinterpret_cast<uint4 *>(dst[x] + t * SUB + swz(rr + p * RPP, c)) = v[x][p];
+#pragma unroll
+        for (int p = 0; p < NP; ++p) {
+            const uint32_t xs[4] = {vo[p].x, vo[p].y, vo[p].z, vo[p].w}, ys[4] = {v[IDO][p].x, v[IDO][p].y, v[IDO][p].z, v[IDO][p].w};
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                acc[p] = fmaf(__uint_as_float(xs[w] << 16), __uint_as_float(ys[w] << 16), acc[p]);
+                acc[p] = fmaf(__uint_as_float(xs[w] & 0xffff0000u), __uint_as_float(ys[w] & 0xffff0000u), acc[p]);
+            }
+        }
+    }
+#pragma unroll
+    for (int p = 0; p < NP; ++p) {
+        float x = acc[p];
+        x += __shfl_xor_sync(0xffffffffu, x, 1);
+        x += __shfl_xor_sync(0xffffffffu, x, 2);
+        x += __shfl_xor_sync(0xffffffffu, x, 4);
+        if (c == 0) s_delta[rr + p * RPP] = x;
+    }
+}
+
 // GATHER = true: a stage above 0 computed beside stage 0.  Rows (and their LSE / delta) are fetched
 // through the stage's tok map by the threads instead of TMA, and the kernel leaves only the stage's
 // own gradients per element (fp32, indexed by element) for the chain merge.
@@ -84,6 +143,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     uint64_t *bar_mma = bar_tma + 1;
     uint32_t *slot = (uint32_t *)(bar_mma + 1);
     volatile int *abort_flag = (volatile int *)(slot + 1);
+    float *s_delta = (float *)(bar_tma + 8);     // gathering kernel without a delta pass: dO . O of the query-side rows
 
     const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, hf = tid >> 7;
     // rest_only: take the blocks after the first n_fused entries of queue_split
@@ -150,20 +210,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
                 const int tk = GATHER ? a.tok[e] : e;
                 lse2 = a.lse[(size_t)h * a.T + tk] * LOG2E;
                 if (a.delta != nullptr) dl = a.delta[(size_t)h * a.T + tk];
-                else {      // no delta pass ran: dO . O of the row, here
-                    const uint4 *po = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.o) + ((size_t)tk * H + h) * D);
-                    const uint4 *pg = reinterpret_cast<const uint4 *>(reinterpret_cast<const __nv_bfloat16 *>(a.d_o) + ((size_t)tk * H + h) * D);
-#pragma unroll
-                    for (int c = 0; c < D / 8; ++c) {
-                        const uint4 x = po[c], y = pg[c];
-                        const uint32_t xs[4] = {x.x, x.y, x.z, x.w}, ys[4] = {y.x, y.y, y.z, y.w};
-#pragma unroll
-                        for (int w = 0; w < 4; ++w) {
-                            dl = fmaf(__uint_as_float(xs[w] << 16), __uint_as_float(ys[w] << 16), dl);
-                            dl = fmaf(__uint_as_float(xs[w] & 0xffff0000u), __uint_as_float(ys[w] & 0xffff0000u), dl);
-                        }
-                    }
-                }
+                else dl = s_delta[rl];      // no delta pass ran: left by the gather of the query-side rows
             }
         }
         const int jl = max(lo - k_row0, 0), jh = min(hi - k_row0, nk);
@@ -249,15 +296,18 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
     auto load = [&](bool q_side, int row0_q, bool k_side, int row0_k) {
         if constexpr (GATHER) {
             const int end_q = a.gather_end_q ? a.gather_end_q : a.n, end_k = a.gather_end_k ? a.gather_end_k : a.n;
+            const bool need_delta = a.delta == nullptr;
             if (q_side && k_side && row0_q == row0_k && end_q == end_k) {
                 uint8_t *const d4[4] = {sQ, sDO, sK, sV};
                 const void *const s4[4] = {a.q, a.d_o, a.k, a.v};
-                gather_tiles<D, 256, 4>(d4, s4, a.tok, row0_q, end_q, H, h, tid);
+                if (need_delta) gather_tiles_delta<D, 256, 4, 1>(d4, s4, a.o, s_delta, a.tok, row0_q, end_q, H, h, tid);
+                else gather_tiles<D, 256, 4>(d4, s4, a.tok, row0_q, end_q, H, h, tid);
             } else {
                 if (q_side) {
                     uint8_t *const d2[2] = {sQ, sDO};
                     const void *const s2[2] = {a.q, a.d_o};
-                    gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_q, end_q, H, h, tid);
+                    if (need_delta) gather_tiles_delta<D, 256, 2, 1>(d2, s2, a.o, s_delta, a.tok, row0_q, end_q, H, h, tid);
+                    else gather_tiles<D, 256, 2>(d2, s2, a.tok, row0_q, end_q, H, h, tid);
                 }
                 if (k_side) {
                     uint8_t *const d2[2] = {sK, sV};
@@ -303,10 +353,12 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
             }
             uint32_t pk[16];
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
+            for (int j = 0; j < 32; j += 4) {
                 const float x0 = __uint_as_float(r[j]) * scale, x1 = __uint_as_float(r[j + 1]) * scale;
-                if (part != nullptr) *reinterpret_cast<float2 *>(part + c0 + j) = make_float2(x0, x1);
+                const float x2 = __uint_as_float(r[j + 2]) * scale, x3 = __uint_as_float(r[j + 3]) * scale;
+                if (part != nullptr) *reinterpret_cast<float4 *>(part + c0 + j) = make_float4(x0, x1, x2, x3);
                 pk[j >> 1] = pack_bf16(x0, x1);
+                pk[(j >> 1) + 1] = pack_bf16(x2, x3);
             }
             uint8_t *d = dst + (c0 >> 6) * SUB;
 #pragma unroll
@@ -1096,7 +1148,7 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     if (rc) return rc;
     rc = make_tmap_bf16(&tdo, a.d_o, D, a.H, a.T, 128);
     if (rc) return rc;
-    constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64;
+    constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64 + 512;
     static bool attr = false;
     if (!attr) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -1202,7 +1254,7 @@ static int launch_bwd_tc_upper_t(const BwdStageArgs &a, cudaStream_t st) {
     CUtensorMap tq;     // the gathering kernel takes no tensor map; the parameter slots get a valid one
     int rc = make_tmap_bf16(&tq, a.q, D, a.H, a.T, 128);
     if (rc) return rc;
-    constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64;
+    constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64 + 512;
     static bool attr = false;
     if (!attr) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
