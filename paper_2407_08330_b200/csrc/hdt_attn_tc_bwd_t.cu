@@ -315,10 +315,12 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
                     tmem_wait_ld();
                     uint32_t pk[16];
 #pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
+                    for (int j = 0; j < 32; j += 4) {
                         const float x0 = __uint_as_float(r[j]) * sc, x1 = __uint_as_float(r[j + 1]) * sc;
-                        if (part != nullptr) *reinterpret_cast<float2 *>(part + c0 + j) = make_float2(x0, x1);
+                        const float x2 = __uint_as_float(r[j + 2]) * sc, x3 = __uint_as_float(r[j + 3]) * sc;
+                        if (part != nullptr) *reinterpret_cast<float4 *>(part + c0 + j) = make_float4(x0, x1, x2, x3);
                         pk[j >> 1] = pack_bf16(x0, x1);
+                        pk[(j >> 1) + 1] = pack_bf16(x2, x3);
                     }
 #pragma unroll
                     for (int c = 0; c < 4; ++c)
