@@ -67,6 +67,7 @@ static thread_local Side g_side[64];
 int g_no_overlap = 0;
 int g_no_graph = 0;
 int g_phase_stamps = 0;
+int g_no_fwd_mc = 0;
 int g_no_pdl = 0;
 static int g_no_fused_delta = 0;
 static int g_no_fold = 0;
@@ -146,6 +147,7 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "no_fused_delta") == 0) { g_no_fused_delta = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_fold") == 0) { g_no_fold = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_pdl") == 0) { g_no_pdl = value; return HDT_OK; }
+    if (name && std::strcmp(name, "no_fwd_mc") == 0) { g_no_fwd_mc = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 

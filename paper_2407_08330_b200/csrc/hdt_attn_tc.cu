@@ -1028,6 +1028,299 @@ int read_fwd_phase_cycles(long long *out16) {
     return HDT_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Multi-chunk forward at D = 64 for the blocks that are not self-contained (a family longer than
+// one block: every block of it walks the whole family's keys in chunks of 128) and for EMPTY
+// blocks.  One CTA of 256 threads per (block, head), two CTAs per SM.  Two threads share a query
+// row (TMEM lane): thread t and t + 128 take the lower and the upper 64 columns of S, exchange
+// their partial row maximum through shared memory and keep partial row sums until the epilogue.
+// P goes to TMEM (A operand of the P V MMA), so S of chunk i + 1 is issued together with P V of
+// chunk i as soon as every thread has S of chunk i in registers; K and V tiles are double-buffered
+// and only thread 0 waits for them.  The running maximum is only raised when the chunk's maximum
+// exceeds it by more than 8 (in the exponent of 2): O and the row sum then need no rescale on
+// most chunks, and both use the same reference, so the result is the exact softmax.
+// TMEM: S columns [0, 128), O [128, 192), P (bf16 pairs) [192, 256).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CUtensorMap tm_q,
+                                                      const __grid_constant__ CUtensorMap tm_k,
+                                                      const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
+    constexpr int D = 64;
+    constexpr uint32_t TM_S = 0, TM_O = 128, TM_P = 192, TM_COLS = 256;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *sm = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t *sQ = sm;                       // reused to stage O
+    uint8_t *sK = sm + SUB;                 // two tiles
+    uint8_t *sV = sm + 3 * SUB;             // two tiles
+    float *s_x = (float *)(sm + 5 * SUB);   // [2][128]: partial row maxima, at the end partial row sums
+    uint64_t *bar_k = (uint64_t *)(s_x + 256);   // [2]; bar_k[0] also carries Q
+    uint64_t *bar_v = bar_k + 2;                 // [2]
+    uint64_t *bar_mma = bar_k + 4;
+    uint32_t *slot = (uint32_t *)(bar_k + 5);
+    volatile int *abort_flag = (volatile int *)(slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, half = tid >> 7, rl = tid & 127;
+    const int blk = a.rest_only ? a.queue_split[a.n_fused + blockIdx.x] : a.queue[blockIdx.x];
+    const int h = blockIdx.y, H = a.H;
+    const int *rec = a.blocks + 5 * (size_t)blk;
+    const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3], fl = rec[4];
+    const float NEG = -INFINITY, LN2 = 0.6931471805599453f;
+
+    if (tid == 0) {
+        for (int i = 0; i < 5; ++i) mbar_init(bar_k + i, 1);
+        *abort_flag = (*a.status != 0);     // an earlier failure: do not wait for anything
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+
+    const int row = r0 + rl;
+    const bool inb = row < r1;
+    int lo = 0, hi = 0;
+    if (inb) { lo = a.rng[2 * row]; hi = a.rng[2 * row + 1]; }
+    float m = NEG, l = 0.f;
+    bool ok = true;
+    const bool empty = (fl & HDT_BLK_EMPTY) != 0;
+    const bool dead = (*abort_flag != 0);   // same value in every thread: read after the barrier
+    const int n_chunks = (empty || dead) ? 0 : (kb - ka + 127) >> 7;
+    const float sc = a.scale_log2;
+
+    // S of chunk i: Q K_i^T into TMEM columns [0, 128); thread 0 only
+    auto issue_s = [&](int i) {
+        const int Nc = (min(128, kb - (ka + 128 * i)) + 15) & ~15;
+        const uint32_t idesc = idesc_bf16(Nc, false, false);
+        const uint32_t kt = smem_u32(sK + (i & 1) * SUB);
+#pragma unroll
+        for (int kk = 0; kk < D / 16; ++kk)
+            mma_ss(tmem + TM_S, smem_desc(smem_u32(sQ) + kk * 32, 0, 1024), smem_desc(kt + kk * 32, 0, 1024), idesc, kk > 0);
+    };
+
+    if (n_chunks > 0 && tid == 0) {
+        mbar_expect_tx(bar_k, 2u * SUB);
+        tma_load_3d(sQ, &tm_q, 0, h, r0, bar_k);
+        tma_load_3d(sK, &tm_k, 0, h, ka, bar_k);
+        mbar_expect_tx(bar_v, (uint32_t)SUB);
+        tma_load_3d(sV, &tm_v, 0, h, ka, bar_v);
+        if (n_chunks > 1) {
+            mbar_expect_tx(bar_k + 1, (uint32_t)SUB);
+            tma_load_3d(sK + SUB, &tm_k, 0, h, ka + 128, bar_k + 1);
+            mbar_expect_tx(bar_v + 1, (uint32_t)SUB);
+            tma_load_3d(sV + SUB, &tm_v, 0, h, ka + 128, bar_v + 1);
+        }
+        if (!mbar_wait(bar_k, 0, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 1; }
+        if (!*abort_flag) {
+            tc_fence_after();
+            issue_s(0);
+            mma_commit(bar_mma);
+        }
+    }
+
+    for (int i = 0; i < n_chunks; ++i) {
+        const int c0 = ka + 128 * i;
+        const int nvalid = min(128, kb - c0);
+        const int Nc = (nvalid + 15) & ~15;
+        // S of this chunk is there, and P V of the previous chunk is done
+        if (!mbar_wait(bar_mma, i & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 2; }
+        tc_fence_after();
+        if (tid == 0 && !*abort_flag) {
+            if (i + 2 < n_chunks) {          // the K tile that S of this chunk has left
+                mbar_expect_tx(bar_k + (i & 1), (uint32_t)SUB);
+                tma_load_3d(sK + (i & 1) * SUB, &tm_k, 0, h, c0 + 256, bar_k + (i & 1));
+            }
+            if (i >= 1 && i + 1 < n_chunks) {   // the V tile that P V of the previous chunk has left
+                mbar_expect_tx(bar_v + ((i + 1) & 1), (uint32_t)SUB);
+                tma_load_3d(sV + ((i + 1) & 1) * SUB, &tm_v, 0, h, c0 + 128, bar_v + ((i + 1) & 1));
+            }
+        }
+
+        // ---- this thread's 64 columns of S: two slices of 32, all in registers ----
+        const int jl = max(lo - c0, 0), jh = min(hi - c0, nvalid);
+        const bool has = inb && jh > jl;
+        const int cb = 64 * half;
+        const bool act0 = cb < Nc, act1 = cb + 32 < Nc;      // uniform in the warp
+        uint32_t x0[32], x1[32];
+        if (act0) tmem_ld32(tmem + TM_S + lane_base + cb, x0);
+        if (act1) tmem_ld32(tmem + TM_S + lane_base + cb + 32, x1);
+        if (act0) tmem_wait_ld();
+        const uint32_t km0 = (has && act0) ? keep_mask<false>(cb, 32, jl, jh, 0, 0, false, false) : 0u;
+        const uint32_t km1 = (has && act1) ? keep_mask<false>(cb + 32, 32, jl, jh, 0, 0, false, false) : 0u;
+        const bool full0 = __all_sync(0xffffffffu, km0 == 0xffffffffu);
+        const bool full1 = __all_sync(0xffffffffu, km1 == 0xffffffffu);
+        float mx = NEG;
+        {
+            float t0 = NEG, t1 = NEG, t2 = NEG, t3 = NEG;
+            if (full0) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    t0 = fmaxf(t0, __uint_as_float(x0[j])); t1 = fmaxf(t1, __uint_as_float(x0[j + 1]));
+                    t2 = fmaxf(t2, __uint_as_float(x0[j + 2])); t3 = fmaxf(t3, __uint_as_float(x0[j + 3]));
+                }
+            } else if (km0 != 0u) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    t0 = fmaxf(t0, (km0 & (1u << j)) ? __uint_as_float(x0[j]) : NEG);
+                    t1 = fmaxf(t1, (km0 & (2u << j)) ? __uint_as_float(x0[j + 1]) : NEG);
+                }
+            }
+            if (full1) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    t0 = fmaxf(t0, __uint_as_float(x1[j])); t1 = fmaxf(t1, __uint_as_float(x1[j + 1]));
+                    t2 = fmaxf(t2, __uint_as_float(x1[j + 2])); t3 = fmaxf(t3, __uint_as_float(x1[j + 3]));
+                }
+            } else if (km1 != 0u) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    t2 = fmaxf(t2, (km1 & (1u << j)) ? __uint_as_float(x1[j]) : NEG);
+                    t3 = fmaxf(t3, (km1 & (2u << j)) ? __uint_as_float(x1[j + 1]) : NEG);
+                }
+            }
+            mx = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
+        }
+        s_x[half * 128 + rl] = mx;
+        __syncthreads();
+        mx = fmaxf(mx, s_x[(half ^ 1) * 128 + rl]);
+        // the reference maximum moves only when the chunk's maximum is well above it
+        const float mc = mx * sc;
+        float alpha = 1.f;
+        if (mc > m + 8.f) { alpha = exp2f(m - mc); m = mc; }
+        if (i > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {    // rescale this thread's half of the running O
+            uint32_t r[32];
+            tmem_ld32(tmem + TM_O + lane_base + 32 * half, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
+            tmem_st32(tmem + TM_O + lane_base + 32 * half, r);
+        }
+        // ---- P = exp2(S scale - m), bf16 pairs into TMEM; partial row sum ----
+        float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+        if (act0) {
+            uint32_t pk[16];
+            if (full0) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float p0 = exp2f(fmaf(__uint_as_float(x0[j]), sc, -m)), p1 = exp2f(fmaf(__uint_as_float(x0[j + 1]), sc, -m));
+                    const float p2 = exp2f(fmaf(__uint_as_float(x0[j + 2]), sc, -m)), p3 = exp2f(fmaf(__uint_as_float(x0[j + 3]), sc, -m));
+                    q0 += p0; q1 += p1; q2 += p2; q3 += p3;
+                    pk[j >> 1] = pack_bf16(p0, p1); pk[(j >> 1) + 1] = pack_bf16(p2, p3);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    const float p0 = (km0 & (1u << j)) ? exp2f(fmaf(__uint_as_float(x0[j]), sc, -m)) : 0.f;
+                    const float p1 = (km0 & (2u << j)) ? exp2f(fmaf(__uint_as_float(x0[j + 1]), sc, -m)) : 0.f;
+                    q0 += p0; q1 += p1;
+                    pk[j >> 1] = pack_bf16(p0, p1);
+                }
+            }
+            tmem_st16(tmem + TM_P + lane_base + 32 * half, pk);
+        }
+        if (act1) {
+            uint32_t pk[16];
+            if (full1) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4) {
+                    const float p0 = exp2f(fmaf(__uint_as_float(x1[j]), sc, -m)), p1 = exp2f(fmaf(__uint_as_float(x1[j + 1]), sc, -m));
+                    const float p2 = exp2f(fmaf(__uint_as_float(x1[j + 2]), sc, -m)), p3 = exp2f(fmaf(__uint_as_float(x1[j + 3]), sc, -m));
+                    q0 += p0; q1 += p1; q2 += p2; q3 += p3;
+                    pk[j >> 1] = pack_bf16(p0, p1); pk[(j >> 1) + 1] = pack_bf16(p2, p3);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 32; j += 2) {
+                    const float p0 = (km1 & (1u << j)) ? exp2f(fmaf(__uint_as_float(x1[j]), sc, -m)) : 0.f;
+                    const float p1 = (km1 & (2u << j)) ? exp2f(fmaf(__uint_as_float(x1[j + 1]), sc, -m)) : 0.f;
+                    q2 += p0; q3 += p1;
+                    pk[j >> 1] = pack_bf16(p0, p1);
+                }
+            }
+            tmem_st16(tmem + TM_P + lane_base + 32 * half + 16, pk);
+        }
+        l = l * alpha + ((q0 + q1) + (q2 + q3));
+        tmem_wait_st();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0 && !*abort_flag) {
+            tc_fence_after();
+            if (i + 1 < n_chunks) {          // S of the next chunk: every thread holds this chunk's S in registers
+                if (!mbar_wait(bar_k + ((i + 1) & 1), ((i + 1) >> 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 3; }
+                else issue_s(i + 1);
+            }
+            if (!mbar_wait(bar_v + (i & 1), (i >> 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 4; }
+            else {
+                const uint32_t idesc = idesc_bf16(D, false, true);
+                const uint32_t vt = smem_u32(sV + (i & 1) * SUB);
+                for (int kk = 0; kk < Nc / 16; ++kk)
+                    mma_ts(tmem + TM_O, tmem + TM_P + 8 * kk, smem_desc(vt + kk * 2048, SUB, 1024), idesc, (i > 0) || kk > 0);
+                mma_commit(bar_mma);
+            }
+        }
+    }
+    if (n_chunks > 0) {
+        if (!mbar_wait(bar_mma, n_chunks & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 5; }
+        tc_fence_after();
+    }
+    if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
+
+    // ---- epilogue: the row sum is the sum of the two threads' parts; normalise; rows that live on
+    // in the next stage also leave their fp32 partial result (O, LSE) there; stage O, store ----
+    __syncthreads();                 // the last chunk's maxima have been read
+    s_x[half * 128 + rl] = l;
+    __syncthreads();
+    l = s_x[rl] + s_x[128 + rl];
+    float lse = NEG, w0 = 0.f;
+    if (l > 0.f) { w0 = 1.f / l; lse = (m + log2f(l)) * LN2; }
+    float *po = nullptr;
+    if (inb && a.part_o != nullptr) {
+        const int u = a.up[row];
+        if (u >= 0) {
+            po = a.part_o + ((size_t)u * H + h) * D;
+            if (half == 0) a.part_lse[(size_t)u * H + h] = lse;
+        }
+    }
+    {
+        uint32_t r[32];
+        if (n_chunks > 0) {
+            tmem_ld32(tmem + TM_O + lane_base + 32 * half, r);
+            tmem_wait_ld();
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) r[j] = 0u;
+        }
+        float x[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) x[j] = (w0 > 0.f) ? __uint_as_float(r[j]) * w0 : 0.f;
+        if (po != nullptr) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4 *>(po + 32 * half + j) = make_float4(x[j], x[j + 1], x[j + 2], x[j + 3]);
+        }
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+            *reinterpret_cast<uint4 *>(sQ + swz(rl, half * 4 + c)) =
+                make_uint4(pack_bf16(x[8 * c], x[8 * c + 1]), pack_bf16(x[8 * c + 2], x[8 * c + 3]),
+                           pack_bf16(x[8 * c + 4], x[8 * c + 5]), pack_bf16(x[8 * c + 6], x[8 * c + 7]));
+    }
+    if (inb && half == 0) a.lse[(size_t)h * a.T + row] = lse;
+    tc_fence_before();
+    __syncthreads();
+    {
+        __nv_bfloat16 *og = reinterpret_cast<__nv_bfloat16 *>(a.o);
+        const int nrows = r1 - r0;
+        for (int idx = tid; idx < 128 * 8; idx += 256) {
+            const int r = idx >> 3, c = idx & 7;
+            if (r < nrows) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(sQ + swz(r, c));
+                *reinterpret_cast<uint4 *>(og + ((size_t)(r0 + r) * H + h) * D + c * 8) = v;
+            }
+        }
+    }
+    if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
 template <int D>
 static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     CUtensorMap tq, tk, tv;
@@ -1044,6 +1337,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     }
     constexpr int smem = (4 * (D / 64) + 2) * SUB + 1024 + 64;     // general kernel: Q, two K tiles, V, P
     constexpr int smem_1 = 3 * (D / 64) * SUB + 1024 + 64;
+    constexpr int smem_mc = 5 * SUB + 2 * 128 * 4 + 1024 + 64;     // multi-chunk kernel: Q, two K, two V tiles
     static bool attr = false;
     if (!attr) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
@@ -1053,6 +1347,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             8 * SUB + 4 * 128 * 4 + 1024 + 64));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
         attr = true;
     }
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
@@ -1115,6 +1410,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
         if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);
+        else if (D == 64 && !g_no_fwd_mc) k_fwd_tc_mc<<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
         else k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());

@@ -86,6 +86,7 @@ extern int g_no_overlap;   // option "no_overlap"
 extern int g_force_simt;   // option "force_simt"
 extern int g_no_graph;     // option "no_graph"
 extern int g_phase_stamps; // option "phase_stamps": the transposed backward runs its instrumented instantiation
+extern int g_no_fwd_mc;    // option "no_fwd_mc": blocks that are not self-contained stay on the 128-thread general forward kernel
 
 // Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute may
 // be scheduled while the kernel before it on the stream still runs (once every CTA of that kernel
