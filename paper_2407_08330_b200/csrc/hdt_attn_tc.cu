@@ -1034,13 +1034,27 @@ int read_fwd_phase_cycles(long long *out16) {
 // blocks.  One CTA of 256 threads per (block, head), two CTAs per SM.  Two threads share a query
 // row (TMEM lane): thread t and t + 128 take the lower and the upper 64 columns of S, exchange
 // their partial row maximum through shared memory and keep partial row sums until the epilogue.
-// P goes to TMEM (A operand of the P V MMA), so S of chunk i + 1 is issued together with P V of
-// chunk i as soon as every thread has S of chunk i in registers; K and V tiles are double-buffered
-// and only thread 0 waits for them.  The running maximum is only raised when the chunk's maximum
+// P goes to TMEM (A operand of the P V MMA); S of chunk i + 1 is issued as soon as every thread
+// has S of chunk i in registers (at the barrier of the maximum exchange) and runs beside the
+// exponentials, P V of chunk i beside the maximum pass of chunk i + 1; K and V tiles are
+// double-buffered and only thread 0 waits for them.  The running maximum is only raised when the chunk's maximum
 // exceeds it by more than 8 (in the exponent of 2): O and the row sum then need no rescale on
 // most chunks, and both use the same reference, so the result is the exact softmax.
 // TMEM: S columns [0, 128), O [128, 192), P (bf16 pairs) [192, 256).
 // ---------------------------------------------------------------------------------------------
+// Cycle counts per phase of k_fwd_tc_mc's chunk loop (STAMP instantiation): thread 64 of the eight
+// longest blocks of head 0 adds clock64() differences between fixed points of the loop.
+#define HDT_MSTAMP(i)                                                              \
+    do {                                                                           \
+        if constexpr (STAMP) {                                                     \
+            if (stamper) {                                                         \
+                const long long now_ = clock64();                                  \
+                atomicAdd((unsigned long long *)&g_fwd_phase_cycles[i], (unsigned long long)(now_ - t_last)); \
+                t_last = now_;                                                     \
+            }                                                                      \
+        }                                                                          \
+    } while (0)
+template <bool STAMP = false>
 __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CUtensorMap tm_q,
                                                       const __grid_constant__ CUtensorMap tm_k,
                                                       const __grid_constant__ CUtensorMap tm_v, const FwdStageArgs a) {
@@ -1054,8 +1068,8 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
     float *s_x = (float *)(sm + 5 * SUB);   // [2][128]: partial row maxima, at the end partial row sums
     uint64_t *bar_k = (uint64_t *)(s_x + 256);   // [2]; bar_k[0] also carries Q
     uint64_t *bar_v = bar_k + 2;                 // [2]
-    uint64_t *bar_mma = bar_k + 4;
-    uint32_t *slot = (uint32_t *)(bar_k + 5);
+    uint64_t *bar_s = bar_k + 4, *bar_o = bar_k + 5;   // S of a chunk has arrived; P V of a chunk is done
+    uint32_t *slot = (uint32_t *)(bar_k + 6);
     volatile int *abort_flag = (volatile int *)(slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, half = tid >> 7, rl = tid & 127;
@@ -1066,7 +1080,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
     const float NEG = -INFINITY, LN2 = 0.6931471805599453f;
 
     if (tid == 0) {
-        for (int i = 0; i < 5; ++i) mbar_init(bar_k + i, 1);
+        for (int i = 0; i < 6; ++i) mbar_init(bar_k + i, 1);
         *abort_flag = (*a.status != 0);     // an earlier failure: do not wait for anything
         fence_mbar_init();
     }
@@ -1114,26 +1128,25 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         if (!*abort_flag) {
             tc_fence_after();
             issue_s(0);
-            mma_commit(bar_mma);
+            mma_commit(bar_s);
         }
     }
 
+    long long t_last = 0;
+    const bool stamper = STAMP && tid == 64 && blockIdx.y == 0 && blockIdx.x < 8;
+    const bool stamp0 = STAMP && tid == 0 && blockIdx.y == 0 && blockIdx.x < 8;
+    if constexpr (STAMP) { if (stamper) t_last = clock64(); }
     for (int i = 0; i < n_chunks; ++i) {
         const int c0 = ka + 128 * i;
         const int nvalid = min(128, kb - c0);
         const int Nc = (nvalid + 15) & ~15;
-        // S of this chunk is there, and P V of the previous chunk is done
-        if (!mbar_wait(bar_mma, i & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 2; }
+        // S of this chunk is there
+        if (!mbar_wait(bar_s, i & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 2; }
         tc_fence_after();
-        if (tid == 0 && !*abort_flag) {
-            if (i + 2 < n_chunks) {          // the K tile that S of this chunk has left
-                mbar_expect_tx(bar_k + (i & 1), (uint32_t)SUB);
-                tma_load_3d(sK + (i & 1) * SUB, &tm_k, 0, h, c0 + 256, bar_k + (i & 1));
-            }
-            if (i >= 1 && i + 1 < n_chunks) {   // the V tile that P V of the previous chunk has left
-                mbar_expect_tx(bar_v + ((i + 1) & 1), (uint32_t)SUB);
-                tma_load_3d(sV + ((i + 1) & 1) * SUB, &tm_v, 0, h, c0 + 128, bar_v + ((i + 1) & 1));
-            }
+        HDT_MSTAMP(0);
+        if (tid == 0 && !*abort_flag && i + 2 < n_chunks) {          // the K tile that S of this chunk has left
+            mbar_expect_tx(bar_k + (i & 1), (uint32_t)SUB);
+            tma_load_3d(sK + (i & 1) * SUB, &tm_k, 0, h, c0 + 256, bar_k + (i & 1));
         }
 
         // ---- this thread's 64 columns of S: two slices of 32, all in registers ----
@@ -1145,6 +1158,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         if (act0) tmem_ld32(tmem + TM_S + lane_base + cb, x0);
         if (act1) tmem_ld32(tmem + TM_S + lane_base + cb + 32, x1);
         if (act0) tmem_wait_ld();
+        HDT_MSTAMP(1);
         const uint32_t km0 = (has && act0) ? keep_mask<false>(cb, 32, jl, jh, 0, 0, false, false) : 0u;
         const uint32_t km1 = (has && act1) ? keep_mask<false>(cb + 32, 32, jl, jh, 0, 0, false, false) : 0u;
         const bool full0 = __all_sync(0xffffffffu, km0 == 0xffffffffu);
@@ -1181,12 +1195,36 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
             mx = fmaxf(fmaxf(t0, t1), fmaxf(t2, t3));
         }
         s_x[half * 128 + rl] = mx;
+        tc_fence_before();
         __syncthreads();
+        HDT_MSTAMP(2);
+        // S of the next chunk: every thread holds this chunk's S in registers, so the MMA runs
+        // beside the exponentials
+        if (tid == 0 && !*abort_flag && i + 1 < n_chunks) {
+            tc_fence_after();
+            long long t0_ = 0;
+            if constexpr (STAMP) t0_ = clock64();
+            if (!mbar_wait(bar_k + ((i + 1) & 1), ((i + 1) >> 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 3; }
+            else {
+                if constexpr (STAMP) { if (stamp0) { const long long n_ = clock64(); atomicAdd((unsigned long long *)&g_fwd_phase_cycles[7], (unsigned long long)(n_ - t0_)); t0_ = n_; } }
+                issue_s(i + 1); mma_commit(bar_s);
+                if constexpr (STAMP) { if (stamp0) atomicAdd((unsigned long long *)&g_fwd_phase_cycles[8], (unsigned long long)(clock64() - t0_)); }
+            }
+        }
         mx = fmaxf(mx, s_x[(half ^ 1) * 128 + rl]);
         // the reference maximum moves only when the chunk's maximum is well above it
         const float mc = mx * sc;
         float alpha = 1.f;
         if (mc > m + 8.f) { alpha = exp2f(m - mc); m = mc; }
+        if (i > 0) {          // P V of the previous chunk is done: O may be rescaled, P overwritten, its V tile reused
+            if (!mbar_wait(bar_o, (i - 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 6; }
+            tc_fence_after();
+            if (tid == 0 && !*abort_flag && i + 1 < n_chunks) {
+                mbar_expect_tx(bar_v + ((i + 1) & 1), (uint32_t)SUB);
+                tma_load_3d(sV + ((i + 1) & 1) * SUB, &tm_v, 0, h, c0 + 128, bar_v + ((i + 1) & 1));
+            }
+        }
+        HDT_MSTAMP(3);
         if (i > 0 && !__all_sync(0xffffffffu, alpha == 1.f)) {    // rescale this thread's half of the running O
             uint32_t r[32];
             tmem_ld32(tmem + TM_O + lane_base + 32 * half, r);
@@ -1195,6 +1233,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
             for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * alpha);
             tmem_st32(tmem + TM_O + lane_base + 32 * half, r);
         }
+        HDT_MSTAMP(4);
         // ---- P = exp2(S scale - m), bf16 pairs into TMEM; partial row sum ----
         float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
         if (act0) {
@@ -1242,25 +1281,28 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         l = l * alpha + ((q0 + q1) + (q2 + q3));
         tmem_wait_st();
         tc_fence_before();
+        HDT_MSTAMP(5);
         __syncthreads();
+        HDT_MSTAMP(6);
+        if constexpr (STAMP) { if (stamper) atomicAdd((unsigned long long *)&g_fwd_phase_cycles[12], 1ull); }
         if (tid == 0 && !*abort_flag) {
             tc_fence_after();
-            if (i + 1 < n_chunks) {          // S of the next chunk: every thread holds this chunk's S in registers
-                if (!mbar_wait(bar_k + ((i + 1) & 1), ((i + 1) >> 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 3; }
-                else issue_s(i + 1);
-            }
+            long long t0_ = 0;
+            if constexpr (STAMP) t0_ = clock64();
             if (!mbar_wait(bar_v + (i & 1), (i >> 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 4; }
             else {
+                if constexpr (STAMP) { if (stamp0) { const long long n_ = clock64(); atomicAdd((unsigned long long *)&g_fwd_phase_cycles[9], (unsigned long long)(n_ - t0_)); t0_ = n_; } }
                 const uint32_t idesc = idesc_bf16(D, false, true);
                 const uint32_t vt = smem_u32(sV + (i & 1) * SUB);
                 for (int kk = 0; kk < Nc / 16; ++kk)
                     mma_ts(tmem + TM_O, tmem + TM_P + 8 * kk, smem_desc(vt + kk * 2048, SUB, 1024), idesc, (i > 0) || kk > 0);
-                mma_commit(bar_mma);
+                mma_commit(bar_o);
+                if constexpr (STAMP) { if (stamp0) atomicAdd((unsigned long long *)&g_fwd_phase_cycles[10], (unsigned long long)(clock64() - t0_)); }
             }
         }
     }
     if (n_chunks > 0) {
-        if (!mbar_wait(bar_mma, n_chunks & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 5; }
+        if (!mbar_wait(bar_o, (n_chunks - 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 5; }
         tc_fence_after();
     }
     if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
@@ -1347,7 +1389,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             8 * SUB + 4 * 128 * 4 + 1024 + 64));
-        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
         attr = true;
     }
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
@@ -1410,7 +1453,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
         if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);
-        else if (D == 64 && !g_no_fwd_mc) k_fwd_tc_mc<<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
+        else if (D == 64 && !g_no_fwd_mc && g_phase_stamps) k_fwd_tc_mc<true><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
+        else if (D == 64 && !g_no_fwd_mc) k_fwd_tc_mc<false><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
         else k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
