@@ -1112,7 +1112,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
             mma_ss(tmem + TM_S, smem_desc(smem_u32(sQ) + kk * 32, 0, 1024), smem_desc(kt + kk * 32, 0, 1024), idesc, kk > 0);
     };
 
-    if (n_chunks > 0 && tid == 0) {
+    if (n_chunks > 0 && warp == 0 && elect_one()) {      // (uniform branch, one lane: the MMA issue is cheaper that way)
         mbar_expect_tx(bar_k, 2u * SUB);
         tma_load_3d(sQ, &tm_q, 0, h, r0, bar_k);
         tma_load_3d(sK, &tm_k, 0, h, ka, bar_k);
@@ -1134,7 +1134,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
 
     long long t_last = 0;
     const bool stamper = STAMP && tid == 64 && blockIdx.y == 0 && blockIdx.x < 8;
-    const bool stamp0 = STAMP && tid == 0 && blockIdx.y == 0 && blockIdx.x < 8;
+    const bool stamp0 = STAMP && blockIdx.y == 0 && blockIdx.x < 8;
     if constexpr (STAMP) { if (stamper) t_last = clock64(); }
     for (int i = 0; i < n_chunks; ++i) {
         const int c0 = ka + 128 * i;
@@ -1144,7 +1144,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         if (!mbar_wait(bar_s, i & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 2; }
         tc_fence_after();
         HDT_MSTAMP(0);
-        if (tid == 0 && !*abort_flag && i + 2 < n_chunks) {          // the K tile that S of this chunk has left
+        if (warp == 0 && !*abort_flag && i + 2 < n_chunks && elect_one()) {          // the K tile that S of this chunk has left
             mbar_expect_tx(bar_k + (i & 1), (uint32_t)SUB);
             tma_load_3d(sK + (i & 1) * SUB, &tm_k, 0, h, c0 + 256, bar_k + (i & 1));
         }
@@ -1200,7 +1200,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         HDT_MSTAMP(2);
         // S of the next chunk: every thread holds this chunk's S in registers, so the MMA runs
         // beside the exponentials
-        if (tid == 0 && !*abort_flag && i + 1 < n_chunks) {
+        if (warp == 0 && !*abort_flag && i + 1 < n_chunks && elect_one()) {
             tc_fence_after();
             long long t0_ = 0;
             if constexpr (STAMP) t0_ = clock64();
@@ -1219,7 +1219,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         if (i > 0) {          // P V of the previous chunk is done: O may be rescaled, P overwritten, its V tile reused
             if (!mbar_wait(bar_o, (i - 1) & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 6; }
             tc_fence_after();
-            if (tid == 0 && !*abort_flag && i + 1 < n_chunks) {
+            if (warp == 0 && !*abort_flag && i + 1 < n_chunks && elect_one()) {
                 mbar_expect_tx(bar_v + ((i + 1) & 1), (uint32_t)SUB);
                 tma_load_3d(sV + ((i + 1) & 1) * SUB, &tm_v, 0, h, c0 + 128, bar_v + ((i + 1) & 1));
             }
@@ -1285,7 +1285,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         __syncthreads();
         HDT_MSTAMP(6);
         if constexpr (STAMP) { if (stamper) atomicAdd((unsigned long long *)&g_fwd_phase_cycles[12], 1ull); }
-        if (tid == 0 && !*abort_flag) {
+        if (warp == 0 && !*abort_flag && elect_one()) {
             tc_fence_after();
             long long t0_ = 0;
             if constexpr (STAMP) t0_ = clock64();
