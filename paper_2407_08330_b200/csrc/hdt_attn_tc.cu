@@ -602,7 +602,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             }
             HDT_LSTAMP(1);
             if constexpr (STAMP) { if (tid == 0 && item == (int)blockIdx.x && blockIdx.x < 1024) g_fwd_timeline[blockIdx.x][1] = gtime_f(); }
-            if (tid == 0 && !*abort_flag) {
+            if (warp == 0 && !*abort_flag && elect_one()) {
                 tc_fence_after();
                 const uint32_t idesc = idesc_bf16(Nc, false, false);
 #pragma unroll
@@ -680,7 +680,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
             if (tid == 0 && have_next && !*abort_flag) issue_qk(dn);
             if (!mbar_wait(bar_v, ph, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) { a.status[1] = (2 << 8) | 3; a.status[2] = item; } }
             ph ^= 1;
-            if (tid == 0 && !*abort_flag) {
+            if (warp == 0 && !*abort_flag && elect_one()) {
                 tc_fence_after();
                 const uint32_t idesc = idesc_bf16(D, false, true);
                 for (int kk = 0; kk < Nc / 16; ++kk)
