@@ -141,7 +141,7 @@ def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
     # (fp32 runs with and without the side-stream overlap of the upper stages)
     # (the upper stages of bf16 runs: gathering tensor-core kernels with 128- and 32-row blocks, SIMT)
     opts = (({}, {"_block_m_upper": 32}, {"simt_upper": 1}, {"no_fold": 1}, {"no_fold": 4}, {"no_fused_delta": 1, "no_persistent": 4}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2},
-             {"no_persistent": 3}, {"no_persistent": 5}, {"force_simt": 1})
+             {"no_persistent": 3}, {"no_persistent": 5}, {"no_fwd_mc": 1}, {"force_simt": 1})
             if dtype == "bf16" else ({}, {"no_overlap": 1}))
     for opt in opts:
         opt = dict(opt)
@@ -199,6 +199,33 @@ def test_ragged_long_families_and_padding(P, dtype):
     run_case(P, b, 2, 64, dtype, 11)
     run_case(P, b, 2, 128, dtype, 12, block_m=32)
     run_case(P, b, 1, 64, dtype, 13, block_m=128, scale=0.2)
+
+
+def test_multi_chunk_forward_with_growing_maxima(P):
+    """Families of up to nine key chunks at head_dim 64 (the multi-chunk forward kernel): keys grow
+    by powers of two along the sequence, so the row maxima rise from chunk to chunk by more and by
+    less than the kernel's threshold for moving its reference maximum; the 128-thread general
+    kernel (option no_fwd_mc) must give the same result within the tolerance."""
+    b = gen.pack([gen.layout([[1024, 3], [700, 129, 0]]), gen.layout([[257], [5, 130]])])
+    H, d = 2, 64
+    t = gen.make_tensors(21, b.total_tokens, H, d, "bf16")
+    grow = (2.0 ** (np.arange(b.total_tokens) * 4 // b.total_tokens)).astype(t["k"].dtype)
+    t["k"] = t["k"] * grow[:, None, None]          # exact in bf16
+    idx = P.hdt_build_index(*dev_struct(b))
+    q, k, v = (dev_tensor(t[n], "bf16") for n in ("q", "k", "v"))
+    o_ref, lse_ref = oracle.forward(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"])
+    outs = []
+    for opt in (0, 1):
+        P.hdt_set_option("no_fwd_mc", opt)
+        try:
+            o, lse = P.hdt_attn_fwd(idx, q, k, v)
+        finally:
+            P.hdt_set_option("no_fwd_mc", 0)
+        check_close(host(o), o_ref, "bf16", f"O (no_fwd_mc={opt})")
+        check_close(host(lse), lse_ref, "bf16", f"LSE (no_fwd_mc={opt})")
+        outs.append(host(o))
+    P.hdt_device_status()
+    assert np.abs(outs[0] - outs[1]).max() <= 2e-2
 
 
 def test_generic_depth_trees(P):
