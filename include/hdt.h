@@ -302,7 +302,9 @@ int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const i
  * backward kernel of the call could compute dO . O itself; "no_fold" bit 0 = 1 lets a merge
  * kernel complete the elements of stage 1 in the forward instead of the stage-1 kernel itself, bit 2
  * = 1 makes the backward's stage-1 kernel do it (off by default); "no_pdl" = 1 launches the kernels of hdt_build_index as ordinary stream
- * successors instead of programmatic dependents; "phase_stamps" = 1 selects the
+ * successors instead of programmatic dependents; "no_fwd_mc" = 1 keeps the blocks of a head_dim 64
+ * forward that are not self-contained on the 128-thread general kernel instead of the 256-thread
+ * multi-chunk one; "phase_stamps" = 1 selects the
  * instrumented instantiation of the transposed looping backward (see hdt_debug_bwd_timeline).
  */
 int hdt_set_option(const char *name, int32_t value);
