@@ -305,7 +305,8 @@ int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const i
  * successors instead of programmatic dependents; "no_fwd_mc" = 1 keeps the blocks of a head_dim 64
  * forward that are not self-contained on the 128-thread general kernel instead of the 256-thread
  * multi-chunk one; "phase_stamps" = 1 selects the
- * instrumented instantiation of the transposed looping backward (see hdt_debug_bwd_timeline).
+ * instrumented instantiations of the looping forward and the transposed looping backward (see
+ * hdt_debug_bwd_timeline), = 2 that of the multi-chunk forward (hdt_debug_fwd_phase_cycles).
  */
 int hdt_set_option(const char *name, int32_t value);
 

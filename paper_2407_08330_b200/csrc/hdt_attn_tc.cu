@@ -1037,13 +1037,17 @@ int read_fwd_phase_cycles(long long *out16) {
 // P goes to TMEM (A operand of the P V MMA); S of chunk i + 1 is issued as soon as every thread
 // has S of chunk i in registers (at the barrier of the maximum exchange) and runs beside the
 // exponentials, P V of chunk i beside the maximum pass of chunk i + 1; K and V tiles are
-// double-buffered and only thread 0 waits for them.  The running maximum is only raised when the chunk's maximum
+// double-buffered; one elected lane of warp 0 requests them, waits for them and issues the MMAs
+// inside warp-uniform branches (an MMA issued under a branch on the thread index costs about twice
+// the cycles: 100 instead of 40).  The running maximum is only raised when the chunk's maximum
 // exceeds it by more than 8 (in the exponent of 2): O and the row sum then need no rescale on
 // most chunks, and both use the same reference, so the result is the exact softmax.
 // TMEM: S columns [0, 128), O [128, 192), P (bf16 pairs) [192, 256).
 // ---------------------------------------------------------------------------------------------
-// Cycle counts per phase of k_fwd_tc_mc's chunk loop (STAMP instantiation): thread 64 of the eight
-// longest blocks of head 0 adds clock64() differences between fixed points of the loop.
+// Cycle counts per phase of k_fwd_tc_mc's chunk loop (STAMP instantiation, option "phase_stamps" =
+// 2; read with hdt_debug_fwd_phase_cycles): thread 64 of the eight longest blocks of head 0 adds
+// clock64() differences between fixed points of the loop (entries 0 to 6 and 11, chunk count in
+// 12), the issuing lane of the same CTAs its waits and issue times (entries 7 to 10).
 #define HDT_MSTAMP(i)                                                              \
     do {                                                                           \
         if constexpr (STAMP) {                                                     \
@@ -1140,6 +1144,7 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
         const int c0 = ka + 128 * i;
         const int nvalid = min(128, kb - c0);
         const int Nc = (nvalid + 15) & ~15;
+        HDT_MSTAMP(11);
         // S of this chunk is there
         if (!mbar_wait(bar_s, i & 1, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 2; }
         tc_fence_after();
@@ -1435,7 +1440,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
             const long long items = (long long)a.n_fused * a.H;
             const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
             if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
-            else if (g_phase_stamps && D == 64) {
+            else if (g_phase_stamps == 1 && D == 64) {
                 static bool attr_s = false;
                 if (!attr_s) {
                     HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
@@ -1453,7 +1458,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
         if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);
-        else if (D == 64 && !g_no_fwd_mc && g_phase_stamps) k_fwd_tc_mc<true><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
+        else if (D == 64 && !g_no_fwd_mc && g_phase_stamps == 2) k_fwd_tc_mc<true><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
         else if (D == 64 && !g_no_fwd_mc) k_fwd_tc_mc<false><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
         else k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);
         count_launch();

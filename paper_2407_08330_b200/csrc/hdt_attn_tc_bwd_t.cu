@@ -388,7 +388,7 @@ int launch_bwd_tc_fused64(const BwdStageArgs &a, const CUtensorMap &tq, const CU
         return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_fused64: the fused-delta kernel needs o and the full rule");
     const long long slots = (a.no_persistent == 6 ? 1LL : 2LL) * n_sm;
     const int grid = (int)(items < slots ? items : slots);
-    if (g_phase_stamps && a.dirs == 7) {
+    if (g_phase_stamps == 1 && a.dirs == 7) {
         if (fd) k_bwd_tc_t<false, true, true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
         else k_bwd_tc_t<false, true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
     } else if (a.dirs != 7) k_bwd_tc_t<true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);

@@ -1,6 +1,7 @@
 """Diagnostic: where the looping stage-0 backward kernel spends its time, from its own clock stamps.
 
     python -m paper_2407_08330_b200.phase_cycles [config]
+    python -m paper_2407_08330_b200.phase_cycles 5 mc      (the multi-chunk forward's chunk loop)
 
 With option "phase_stamps" the looping forward and the transposed looping backward (head_dim 64) run
 instrumented instantiations: thread 0 of CTA 0 adds clock64() differences between fixed points of
@@ -80,5 +81,45 @@ def main(c=3):
         P.hdt_set_option("phase_stamps", 0)
 
 
+MC_PHASES = ["wait for S (the first chunk's includes the first tiles' load)", "S into registers", "row maximum, exchange, barrier",
+             "reference maximum, wait for P V of the previous chunk", "rescale of O", "exponentials, P into TMEM",
+             "barrier", "issuing lane: wait for K", "issuing lane: issue of S", "issuing lane: wait for V",
+             "issuing lane: issue of P V", "loop top"]
+
+
+def main_mc(c=5):
+    """Option "phase_stamps" = 2: thread 64 (and the issuing lane) of the eight longest blocks of head
+    0 of the multi-chunk forward kernel add the cycles between fixed points of their chunk loop."""
+    cfg, b = gen.CONFIGS[c], gen.make_hierarchy(c)
+    T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
+    t = gen.make_tensors(1, T, H, d, "bf16")
+    torch.cuda.set_stream(torch.cuda.Stream())
+    dev = lambda x: torch.from_numpy(x).cuda().to(torch.bfloat16)
+    idx = P.hdt_build_index(torch.from_numpy(b.level).cuda(), torch.from_numpy(b.parent).cuda(),
+                            torch.from_numpy(b.cu_seqlens).cuda())
+    q, k, v = (dev(t[n]) for n in ("q", "k", "v"))
+    P.hdt_attn_fwd(idx, q, k, v)
+    L = P.lib()
+    out = (C.c_int64 * 16)()
+    P.hdt_set_option("phase_stamps", 2)
+    try:
+        L.hdt_debug_fwd_phase_cycles(out)
+        for _ in range(5):
+            P.hdt_attn_fwd(idx, q, k, v)
+        torch.cuda.synchronize()
+        L.hdt_debug_fwd_phase_cycles(out)
+        f_ = np.array(list(out), float)
+        n = max(f_[12], 1.0)
+        print(f"multi-chunk forward, {cfg.name}: {int(n)} chunks, {(f_[:7].sum() + f_[11]) / n:.0f} cycles per chunk")
+        for name, x in zip(MC_PHASES, f_[:12] / n):
+            print(f"  {name:62s} {x:7.0f}")
+    finally:
+        P.hdt_set_option("phase_stamps", 0)
+
+
 if __name__ == "__main__":
-    main(int(sys.argv[1]) if len(sys.argv) > 1 else 3)
+    c_ = int(sys.argv[1]) if len(sys.argv) > 1 else 3
+    if len(sys.argv) > 2 and sys.argv[2] == "mc":
+        main_mc(c_)
+    else:
+        main(c_)
