@@ -34,8 +34,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised under profiles/; keyed by (config, profile id).  None = not captured.
 NCU_TRAFFIC = {
     # profiles/k_bwd_tc_t_and_k_fwd_tc_loop_c3_b4_L8192.md
-    (3, "k_bwd_stage0"): 402.1e6,
-    (3, "k_fwd_stage0"): 192.3e6,
+    (3, "k_bwd_stage0"): 401.6e6,
+    (3, "k_fwd_stage0"): 192.0e6,
 }
 
 
