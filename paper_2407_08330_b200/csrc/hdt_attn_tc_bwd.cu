@@ -823,7 +823,9 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     bool ok = true;
     // MMAs are issued by lane 0 of warps 0, 1, 2 in parallel: a single thread needs about 100 cycles
     // per small MMA (descriptor arithmetic), three chains issued side by side hide that
-    const bool issuer = ((tid & 31) == 0) && warp < 3;
+    // MMAs are issued by one elected lane of warps 0 to 2 inside warp-uniform branches (cheaper than
+    // under a branch on the thread index: C5 backward 1.33 -> 1.29 ms; the same change made the d = 128
+    // looping kernel and the transposed kernel slower, so they keep lane 0)
     // six store threads in six warps: (tensor, first / second box); the MMA-issuing warps 0..2 are left alone
     const bool store_thread = ((tid & 31) == 0) && warp >= 4 && warp < 10;
 
@@ -957,7 +959,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             issue_tma(0, d0);
             if (d1.valid) issue_tma(1, d1);
         }
-        if (issuer && warp < 2 && d0.valid) {
+        if (warp < 2 && d0.valid && elect_one()) {
             ok = mbar_wait(&bar_tma[0], 0, abort_flag, WAIT_CYCLES) && ok;
             if (!*abort_flag) {
                 tc_fence_after();
@@ -1037,7 +1039,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             HDT_STAMP(2);
             __syncthreads();
             HDT_STAMP(3);
-            if (issuer && !*abort_flag) {
+            if (warp < 3 && !*abort_flag && elect_one()) {
                 tc_fence_after();
                 // descriptors differ only in the start address: add (bytes >> 4) to the low word
                 const uint32_t sb = smem_u32(st);
