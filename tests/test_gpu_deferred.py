@@ -197,3 +197,31 @@ def test_many_steps_no_expired_wait_and_same_bytes(P):
                 for x, y in zip((o, lse, dq, dk, dv), first):
                     assert torch.equal(x, y)
     P.hdt_device_status()
+
+
+def test_many_steps_split_families_no_expired_wait(P):
+    """400 forward and backward steps of the skewed configuration (families of up to nine key chunks:
+    the multi-chunk forward and the persistent backward with their tile rings and MMA barriers), L2
+    flushed in between: no bounded wait runs out and the forward writes the same bytes every step."""
+    c = 5
+    cfg = gen.CONFIGS[c]
+    b = gen.make_hierarchy(c)
+    T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
+    t = gen.make_tensors(cfg.tensor_seed, T, H, d, cfg.dtype)
+    q, k, v, do = (dev_tensor(t[n], cfg.dtype) for n in ("q", "k", "v", "do"))
+    st = dev_struct(b)
+    flush = torch.empty(192 << 20, dtype=torch.uint8, device="cuda")
+    first = None
+    for i in range(400):
+        flush.zero_()
+        idx = P.hdt_build_index(*st, max_stages=4, deferred=True)
+        o, lse = P.hdt_attn_fwd(idx, q, k, v)
+        P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
+        if i % 100 == 0:
+            P.hdt_device_status()
+            if first is None:
+                first = [x.clone() for x in (o, lse)]
+            else:
+                for x, y in zip((o, lse), first):
+                    assert torch.equal(x, y)
+    P.hdt_device_status()
