@@ -36,6 +36,9 @@ NCU_TRAFFIC = {
     # profiles/k_bwd_tc_t_and_k_fwd_tc_loop_c3_b4_L8192.md
     (3, "k_bwd_stage0"): 401.6e6,
     (3, "k_fwd_stage0"): 192.0e6,
+    # profiles/k_fwd_tc_mc_and_k_bwd_tc_p_c5_skew_2x32768.md
+    (5, "k_bwd_stage0"): 685.5e6,
+    (5, "k_fwd_stage0"): 300.2e6,
 }
 
 
