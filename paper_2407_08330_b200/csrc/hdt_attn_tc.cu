@@ -1085,8 +1085,23 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
 
     if (tid == 0) {
         for (int i = 0; i < 6; ++i) mbar_init(bar_k + i, 1);
-        *abort_flag = (*a.status != 0);     // an earlier failure: do not wait for anything
+        const int dead0 = (*a.status != 0);
+        *abort_flag = dead0;                // an earlier failure: do not wait for anything
         fence_mbar_init();
+        // the first tiles are requested before the TMEM allocation and the CTA barrier
+        if (!dead0 && !(fl & HDT_BLK_EMPTY) && kb > ka) {
+            mbar_expect_tx(bar_k, 2u * SUB);
+            tma_load_3d(sQ, &tm_q, 0, h, r0, bar_k);
+            tma_load_3d(sK, &tm_k, 0, h, ka, bar_k);
+            mbar_expect_tx(bar_v, (uint32_t)SUB);
+            tma_load_3d(sV, &tm_v, 0, h, ka, bar_v);
+            if (kb - ka > 128) {
+                mbar_expect_tx(bar_k + 1, (uint32_t)SUB);
+                tma_load_3d(sK + SUB, &tm_k, 0, h, ka + 128, bar_k + 1);
+                mbar_expect_tx(bar_v + 1, (uint32_t)SUB);
+                tma_load_3d(sV + SUB, &tm_v, 0, h, ka + 128, bar_v + 1);
+            }
+        }
     }
     if (warp == 0) tmem_alloc(slot, TM_COLS);
     tc_fence_before();
@@ -1117,17 +1132,6 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
     };
 
     if (n_chunks > 0 && warp == 0 && elect_one()) {      // (uniform branch, one lane: the MMA issue is cheaper that way)
-        mbar_expect_tx(bar_k, 2u * SUB);
-        tma_load_3d(sQ, &tm_q, 0, h, r0, bar_k);
-        tma_load_3d(sK, &tm_k, 0, h, ka, bar_k);
-        mbar_expect_tx(bar_v, (uint32_t)SUB);
-        tma_load_3d(sV, &tm_v, 0, h, ka, bar_v);
-        if (n_chunks > 1) {
-            mbar_expect_tx(bar_k + 1, (uint32_t)SUB);
-            tma_load_3d(sK + SUB, &tm_k, 0, h, ka + 128, bar_k + 1);
-            mbar_expect_tx(bar_v + 1, (uint32_t)SUB);
-            tma_load_3d(sV + SUB, &tm_v, 0, h, ka + 128, bar_v + 1);
-        }
         if (!mbar_wait(bar_k, 0, abort_flag, WAIT_CYCLES)) { ok = false; if (a.status[1] == 0) a.status[1] = (5 << 8) | 1; }
         if (!*abort_flag) {
             tc_fence_after();
