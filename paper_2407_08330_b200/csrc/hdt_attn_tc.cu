@@ -1303,8 +1303,11 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
                 if constexpr (STAMP) { if (stamp0) { const long long n_ = clock64(); atomicAdd((unsigned long long *)&g_fwd_phase_cycles[9], (unsigned long long)(n_ - t0_)); t0_ = n_; } }
                 const uint32_t idesc = idesc_bf16(D, false, true);
                 const uint32_t vt = smem_u32(sV + (i & 1) * SUB);
-                for (int kk = 0; kk < Nc / 16; ++kk)
-                    mma_ts(tmem + TM_O, tmem + TM_P + 8 * kk, smem_desc(vt + kk * 2048, SUB, 1024), idesc, (i > 0) || kk > 0);
+                const uint64_t dv0 = smem_desc(vt, SUB, 1024);     // the K steps differ in the start address only (16-byte units)
+                const int nk16 = Nc / 16;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    if (kk < nk16) mma_ts(tmem + TM_O, tmem + TM_P + 8 * kk, dv0 + (uint64_t)(kk * 128), idesc, (i > 0) || kk > 0);
                 mma_commit(bar_o);
                 if constexpr (STAMP) { if (stamp0) atomicAdd((unsigned long long *)&g_fwd_phase_cycles[10], (unsigned long long)(clock64() - t0_)); }
             }
