@@ -265,6 +265,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.tok = s ? P.tok : nullptr;
         a.rng = P.rng; a.up = P.up; a.blocks = P.blocks; a.queue = P.queue;
         a.queue_split = P.queue_split; a.n_fused = ix->desc[s].n_fused;
+        a.n_empty = ix->desc[s].n_empty;
         a.block_rows = s ? ix->block_m_upper : ix->block_m;
         a.q = q; a.k = k; a.v = v;
         a.scale_log2 = scale * 1.4426950408889634f;

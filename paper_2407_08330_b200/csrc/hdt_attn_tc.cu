@@ -1375,6 +1375,36 @@ __global__ void __launch_bounds__(256, 2) k_fwd_tc_mc(const __grid_constant__ CU
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
+// EMPTY blocks (rows without any key in this stage: PAD, lone roots): zero rows of O, LSE = -inf,
+// and the same as partial result of the rows that live on in the next stage.  No shared memory and
+// no TMEM, so its CTAs run beside the resident CTAs of the looping kernel (which hold all of an
+// SM's TMEM and most of its shared memory).  Blocks of the list that are not EMPTY are skipped.
+template <int D>
+__global__ void __launch_bounds__(128) k_fwd_empty(const FwdStageArgs a) {
+    const int blk = a.rest_only ? a.queue_split[a.n_fused + blockIdx.x] : a.queue[blockIdx.x];
+    const int *rec = a.blocks + 5 * (size_t)blk;
+    if (!(rec[4] & HDT_BLK_EMPTY)) return;
+    const int r0 = rec[0], nrows = rec[1] - r0, h = blockIdx.y, H = a.H;
+    __nv_bfloat16 *og = reinterpret_cast<__nv_bfloat16 *>(a.o);
+    const uint4 z4 = make_uint4(0u, 0u, 0u, 0u);
+    for (int idx = threadIdx.x; idx < nrows * (D / 8); idx += 128) {
+        const int r = idx / (D / 8), c = idx % (D / 8);
+        *reinterpret_cast<uint4 *>(og + ((size_t)(r0 + r) * H + h) * D + c * 8) = z4;
+    }
+    for (int r = threadIdx.x; r < nrows; r += 128) {
+        const int row = r0 + r;
+        a.lse[(size_t)h * a.T + row] = -INFINITY;
+        if (a.part_o != nullptr) {
+            const int u = a.up[row];
+            if (u >= 0) {
+                float4 *po = reinterpret_cast<float4 *>(a.part_o + ((size_t)u * H + h) * D);
+                for (int j = 0; j < D / 4; ++j) po[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                a.part_lse[(size_t)u * H + h] = -INFINITY;
+            }
+        }
+    }
+}
+
 template <int D>
 static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     CUtensorMap tq, tk, tv;
@@ -1464,7 +1494,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     if (a.part == 1 && split_launch) n_general = 0;     // the caller launches the other blocks separately
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
-        if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);
+        if (a.n_empty == n_general && !g_no_fwd_mc) k_fwd_empty<D><<<grid, 128, 0, st>>>(b);   // nothing but EMPTY blocks left
+        else if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);
         else if (D == 64 && !g_no_fwd_mc && g_phase_stamps == 2) k_fwd_tc_mc<true><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
         else if (D == 64 && !g_no_fwd_mc) k_fwd_tc_mc<false><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
         else k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);

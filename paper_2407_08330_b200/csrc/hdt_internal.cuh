@@ -173,6 +173,8 @@ struct FwdStageArgs {
     const float *next_own_o, *next_own_lse;
     const DevHeader *hdr; // set: the index build is still in flight; the looping kernel reads n_fused and stage 1's size here
     size_t ws_bytes;      // with hdr: bytes behind part_o (the caller's workspace)
+    int n_empty;          // EMPTY blocks of the stage (0 where the caller does not know): when they are all that is left
+                          // beside the self-contained blocks, a kernel without shared memory and TMEM writes their rows
 };
 
 struct BwdStageArgs {
