@@ -1519,7 +1519,19 @@ static int launch_fwd_tc_upper_t(const FwdStageArgs &a, cudaStream_t st) {
     }
     FwdStageArgs b = a;
     b.rest_only = 0;
-    k_fwd_tc<D, false, true><<<dim3(a.nb, a.H), 128, smem, st>>>(tq, tq, tq, b);
+    // every block self-contained (keys = its own rows, one chunk): the single-chunk layout (P over the
+    // Q / K tiles, O over S) needs 48 KB and 128 TMEM columns at D = 64, so four CTAs share an SM
+    // instead of two and the stage runs in one wave
+    if (a.n_fused == a.nb && a.queue_split != nullptr && !g_no_fwd_mc) {
+        constexpr int smem_1 = 3 * (D / 64) * SUB + 1024 + 64;
+        static bool attr_1 = false;
+        if (!attr_1) {
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
+            attr_1 = true;
+        }
+        k_fwd_tc<D, true, true><<<dim3(a.nb, a.H), 128, smem_1, st>>>(tq, tq, tq, b);
+    } else
+        k_fwd_tc<D, false, true><<<dim3(a.nb, a.H), 128, smem, st>>>(tq, tq, tq, b);
     count_launch();
     HDT_CUDA_CHECK(cudaGetLastError());
     return HDT_OK;
