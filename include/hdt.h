@@ -304,7 +304,9 @@ int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const i
  * = 1 makes the backward's stage-1 kernel do it (off by default); "no_pdl" = 1 launches the kernels of hdt_build_index as ordinary stream
  * successors instead of programmatic dependents; "no_fwd_mc" = 1 keeps the blocks of a head_dim 64
  * forward that are not self-contained on the 128-thread general kernel instead of the 256-thread
- * multi-chunk one; "phase_stamps" = 1 selects the
+ * multi-chunk one (and with it the EMPTY blocks of padded batches, which otherwise have a kernel of
+ * their own, and the stages above 0 whose blocks are all self-contained, which otherwise run in the
+ * single-chunk layout); "phase_stamps" = 1 selects the
  * instrumented instantiations of the looping forward and the transposed looping backward (see
  * hdt_debug_bwd_timeline), = 2 that of the multi-chunk forward (hdt_debug_fwd_phase_cycles).
  */
