@@ -31,7 +31,10 @@
  *    0 <= parent[i] < i (sequence-relative); level[i] = level[parent[i]] + 1; tokens are in
  *    document (pre-)order, i.e. a node whose children are all childless is directly followed
  *    by those children; PAD only as a suffix of a sequence.
- *    PAD rows produce O = 0, LSE = -inf and zero gradients.
+ *    PAD rows produce O = 0, LSE = -inf and zero gradients.  The Q, K, V and dO rows of PAD tokens
+ *    must hold finite numbers: the tensor-core kernels load them with their tile and multiply them
+ *    by exact zeros, and 0 x NaN or 0 x inf would reach real rows of the same tile (zero-fill them,
+ *    as a padded batch normally is; nothing checks this).
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  hdt_attn_fwd/bwd are
  *    asynchronous on it.  hdt_build_index enqueues its kernels on it and then waits for them,
  *    because it returns the sizes the attention calls need.
@@ -289,71 +292,15 @@ int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const i
                        size_t workspace_bytes, void *stream);
 
 /*
- * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
- * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
- * general tensor-core kernels, = 2 the persistent forward kernel, = 3 the forward kernel with one CTA
- * per (block, head), = 5 the looping backward kernel (the default at head_dim 128) at head_dim 64 too; "simt_upper" = 1 computes the stages above 0 of bf16 calls on the fp32 SIMT
- * kernels instead of the gathering tensor-core kernels; "no_overlap" = 1 runs the stages
- * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream;
- * "no_graph" = 1 makes hdt_build_index launch its kernels one by one instead of replaying a cached
- * CUDA graph (A/B comparisons, tests).  "no_persistent" = 4 keeps the self-contained blocks of a
- * head_dim 64 backward on the persistent 512-thread kernel instead of the transposed looping one,
- * = 6 gives the latter one CTA per SM; "no_fused_delta" = 1 runs the delta pass even where every
- * backward kernel of the call could compute dO . O itself; "no_fold" bit 0 = 1 lets a merge
- * kernel complete the elements of stage 1 in the forward instead of the stage-1 kernel itself, bit 2
- * = 1 makes the backward's stage-1 kernel do it (off by default); "no_pdl" = 1 launches the kernels of hdt_build_index as ordinary stream
- * successors instead of programmatic dependents; "no_fwd_mc" = 1 keeps the blocks of a head_dim 64
- * forward that are not self-contained on the 128-thread general kernel instead of the 256-thread
- * multi-chunk one (and with it the EMPTY blocks of padded batches, which otherwise have a kernel of
- * their own, and the stages above 0 whose blocks are all self-contained, which otherwise run in the
- * single-chunk layout); "phase_stamps" = 1 selects the
- * instrumented instantiations of the looping forward and the transposed looping backward (see
- * hdt_debug_bwd_timeline), = 2 that of the multi-chunk forward (hdt_debug_fwd_phase_cycles).
- */
-int hdt_set_option(const char *name, int32_t value);
-
-/*
  * Waits for `stream`, then returns and clears the first failure a kernel of this library
  * recorded on the device: HDT_ERR_TIMEOUT when a bounded wait (on a TMA or tensor-core
  * completion barrier) ran out; results of that call are then undefined.  HDT_OK if none.
- * (No counterpart in the paper.)
+ * While a failure is recorded and not yet cleared, every later tensor-core kernel of the library
+ * sees it at its start and does nothing (its outputs stay unwritten) although hdt_attn_fwd /
+ * hdt_attn_bwd still return HDT_OK, because they do not wait for the device: a caller that needs
+ * to know calls this function after the step.  (No counterpart in the paper.)
  */
 int hdt_device_status(void *stream);
-
-/*
- * Test hook for the tensor-core primitives (no counterpart in the paper): C[128,N] = A * B on
- * one CTA with TMA-staged, 128-byte-swizzled operands and tcgen05.mma.
- *   a  device bf16 [128, K] (a_mn = 0) or [K, 128] (a_mn = 1)
- *   b  device bf16 [N, K] (b_mn = 0, C = A B^T) or [K, N] (b_mn = 1, C = A B)
- *   c  device float [128, N];  N, K multiples of 16 in 16..128.  Waits for the result.
- */
-int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N, int32_t K, int32_t a_mn, int32_t b_mn,
-                   void *stream);
-
-/*
- * Diagnostics (no counterpart in the paper): SM clock cycles that CTA 0 of the persistent backward
- * kernel spent in each of its phases since the last call (out16[0..11]: prefetch issue, wait for
- * S/dP, P/dS arithmetic, barrier, rest of the MMA issue, wait for dQ/dK/dV, drain, barrier, stores,
- * loop end, issue of the output MMAs, wait for the next item's TMA), out16[12] = items processed.
- * Synchronises the device and resets the counters.
- */
-int hdt_debug_bwd_phase_cycles(int64_t *out16);
-/* The same for the persistent forward kernel: out16[0..11] = prefetch issue, wait for S, row maximum,
- * barriers (max exchange), P arithmetic and stores, barrier, MMA issue, wait for O, drain, loop top,
- * barrier, output stores; out16[12] = items processed. */
-int hdt_debug_fwd_phase_cycles(int64_t *out16);
-/* With option "phase_stamps" = 1 the looping forward (head_dim 64) runs an instrumented instantiation
- * too and hdt_debug_fwd_phase_cycles reports its phases (out16[0..10]: loop top, wait for Q/K, S,
- * row maximum, exponentials with P into TMEM, barrier, V and the P V MMA, drain, barrier, stores, loop
- * end).  With the same option the transposed looping backward (head_dim 64) runs an instrumented
- * instantiation: hdt_debug_bwd_phase_cycles then reports its phases (out16[0..11]: loop top, wait for
- * the input tiles, issue of S^T/dP^T, wait for them, P^T/dS^T arithmetic, barrier, issue of the output
- * MMAs, prefetch and wait for dV/dK/dQ, drain, barrier, store requests, loop end), and
- * hdt_debug_bwd_timeline the last such launch per CTA (up to 512): out2048[4 c + 0..3] = global timer
- * (ns) at entry, when the first input tiles had arrived, at the end of the item loop, and the SM. */
-int hdt_debug_bwd_timeline(int64_t *out2048);
-/* The same for the last instrumented launch of the looping forward, up to 1024 CTAs. */
-int hdt_debug_fwd_timeline(int64_t *out4096);
 
 #ifdef __cplusplus
 }

@@ -9,7 +9,7 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIBPATH = os.path.join(_HERE, "libhdt.so")
-_HEADER = os.path.join(_HERE, "..", "include", "hdt.h")
+_HEADERS = [os.path.join(_HERE, "..", "include", h) for h in ("hdt.h", "hdt_debug.h")]
 _lib = None
 
 HDT_F32, HDT_BF16 = 0, 1
@@ -68,8 +68,8 @@ def lib():
 
 
 def declared_symbols():
-    """Names of every function include/hdt.h declares."""
-    txt = open(_HEADER).read()
+    """Names of every function the headers under include/ declare."""
+    txt = "".join(open(h).read() for h in _HEADERS)
     txt = re.sub(r"/\*.*?\*/", "", txt, flags=re.S)
     return sorted(set(re.findall(r"\b(hdt_[a-z0-9_]+)\s*\(", txt)))
 

@@ -32,19 +32,49 @@ def needs_build() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile every .cu of csrc/ to an object file (in parallel; objects whose sources and headers
+    are older are reused unless `force`) and link them into libhdt.so."""
     if not force and not needs_build():
         return LIB
+    from concurrent.futures import ThreadPoolExecutor
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB + f".tmp{os.getpid()}"
-    cmd = [nvcc] + NVCC_FLAGS + ["-o", tmp] + sources() + ["-lcudart"]
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        sys.stderr.write(res.stdout + res.stderr)
-    if res.returncode != 0:
+    objdir = os.path.join(HERE, "build")
+    os.makedirs(objdir, exist_ok=True)
+    hdrs = glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(HERE, "..", "include", "*.h")) + \
+        [os.path.abspath(__file__)]
+    t_hdr = max(os.path.getmtime(h) for h in hdrs)
+    flags = [f for f in NVCC_FLAGS if f != "-shared"]
+
+    def compile_one(src):
+        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
+        log = obj + ".log"
+        if not force and os.path.exists(obj) and os.path.exists(log) and \
+                os.path.getmtime(obj) > max(os.path.getmtime(src), t_hdr):
+            return obj, 0, open(log).read()
+        res = subprocess.run([nvcc] + flags + ["-c", "-o", obj, src], capture_output=True, text=True)
+        out = res.stdout + res.stderr
+        if res.returncode == 0:
+            with open(log, "w") as f:
+                f.write(out)
+        return obj, res.returncode, out
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        results = list(ex.map(compile_one, sources()))
+    info = "".join(out for _, _, out in results)
+    failed = [r for r in results if r[1] != 0]
+    if verbose or failed:
+        sys.stderr.write("".join(out for _, rc, out in results if verbose or rc != 0))
+    if failed:
         raise RuntimeError("nvcc failed building libhdt.so")
+    tmp = LIB + f".tmp{os.getpid()}"
+    res = subprocess.run([nvcc, "-shared", "-o", tmp] + [r[0] for r in results] + ["-lcudart"],
+                         capture_output=True, text=True)
+    if res.returncode != 0:
+        sys.stderr.write(res.stdout + res.stderr)
+        raise RuntimeError("nvcc failed linking libhdt.so")
     os.replace(tmp, LIB)
     with open(os.path.join(HERE, "ptxas_info.txt"), "w") as f:
-        f.write(res.stderr)
+        f.write(info)
     return LIB
 
 

@@ -89,19 +89,45 @@ int get_side(Side **out) {
     return HDT_OK;
 }
 
+int sm_count(int *n_sm) {
+    static std::atomic<int> cache[64];
+    int dev = 0;
+    HDT_CUDA_CHECK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return set_error(HDT_ERR_UNSUPPORTED, "device ordinal %d", dev);
+    int n = cache[dev].load(std::memory_order_relaxed);
+    if (n == 0) {
+        HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+        cache[dev].store(n, std::memory_order_relaxed);
+    }
+    *n_sm = n;
+    return HDT_OK;
+}
+
 static size_t al256(size_t x) { return (x + 255) & ~size_t(255); }
 
 struct AttnLayout {
     size_t delta;                       // bwd only
+    size_t dq_acc;                      // bwd, bf16, head_dim 64, batches with split families: fp32 [T, H, 64] sums of dQ tiles
+    bool has_dq_acc;
     size_t part[HDT_MAX_STAGES][4];     // partials handed from stage s-1 to stage s.  fwd: o, lse;  bwd: dq, dk, dv
     size_t own[HDT_MAX_STAGES][4];      // own partials of stage s when it is computed beside stage 0
     size_t total;
 };
 
-static AttnLayout attn_layout(const hdt_index *ix, int H, int D, int bwd) {
+static int g_bwd_two_walk = 0;          // option "bwd_two_walk"
+
+// Blocks of stage 0 that are neither self-contained nor EMPTY: families longer than a row block.
+static int n_split_blocks(const hdt_index *ix) { return ix->desc[0].nb - ix->desc[0].n_fused - ix->desc[0].n_empty; }
+
+static AttnLayout attn_layout(const hdt_index *ix, int H, int D, int bwd, int dtype = HDT_BF16) {
     AttnLayout L{};
     size_t o = 0;
     if (bwd) { L.delta = o; o += al256(sizeof(float) * (size_t)H * ix->total_tokens); }
+    if (bwd && dtype == HDT_BF16 && D == 64 && n_split_blocks(ix) > 0) {
+        L.has_dq_acc = true;
+        L.dq_acc = o;
+        o += al256(sizeof(float) * (size_t)ix->total_tokens * H * 64);
+    }
     for (int s = 1; s < ix->n_stages; ++s) {
         const size_t n = (size_t)ix->desc[s].n;
         const int cnt = bwd ? 3 : 1;
@@ -148,6 +174,7 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "no_fold") == 0) { g_no_fold = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_pdl") == 0) { g_no_pdl = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_fwd_mc") == 0) { g_no_fwd_mc = value; return HDT_OK; }
+    if (name && std::strcmp(name, "bwd_two_walk") == 0) { g_bwd_two_walk = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 
@@ -203,7 +230,7 @@ extern "C" size_t hdt_attn_workspace_bytes(const hdt_index_t *ix, int32_t heads,
     (void)dtype;
     if (!ix || heads <= 0 || head_dim <= 0) return 0;
     if (index_ready(ix)) return 0;
-    return attn_layout(ix, heads, head_dim, bwd).total;
+    return attn_layout(ix, heads, head_dim, bwd, dtype).total;
 }
 
 extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k, const void *v, void *o,
@@ -381,7 +408,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
                             size_t workspace_bytes, void *stream) {
     if (!ix) return set_error(HDT_ERR_INVALID_ARG, "hdt_attn_bwd: null index");
     if (const int rc0 = index_ready(ix)) return rc0;
-    const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 1);
+    const AttnLayout L = attn_layout(ix, heads > 0 ? heads : 1, head_dim > 0 ? head_dim : 64, 1, dtype);
     int rc = check_common(ix, heads, head_dim, dtype, workspace, workspace_bytes, L.total, "hdt_attn_bwd");
     if (rc) return rc;
     if (ix->total_tokens == 0) return HDT_OK;
@@ -407,6 +434,15 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     const bool fused_delta = dtype == HDT_BF16 && !g_force_simt && head_dim == 64 && g_no_persistent == 0 &&
                              !g_no_fused_delta && ix->directions == 7 && ix->desc[0].n_fused == ix->desc[0].nb &&
                              ix->desc[0].nb > 0 && (ix->n_stages == 1 || (overlap && tc_upper));
+    // Families longer than a row block (head_dim 64): one walk over their tile pairs, dQ tiles summed
+    // in an fp32 buffer that starts at zero (option "bwd_two_walk" = 1: two walks, no buffer).
+    float *dq_acc = nullptr;
+    if (L.has_dq_acc && !g_force_simt && !g_bwd_two_walk &&
+        (g_no_persistent == 0 || g_no_persistent == 4 || g_no_persistent == 6)) {
+        dq_acc = (float *)(ws + L.dq_acc);
+        ProfScope ps(PROF_BWD_STAGE0, st);
+        HDT_CUDA_CHECK(cudaMemsetAsync(dq_acc, 0, sizeof(float) * (size_t)ix->total_tokens * heads * 64, st));
+    }
     if (!fused_delta) {
         ProfScope ps(PROF_DELTA, st);
         rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
@@ -438,6 +474,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.no_persistent = g_no_persistent;
         a.dirs = ix->directions;
         a.tok_rows = a.tok;
+        if (s == 0) a.dq_acc = dq_acc;
         return a;
     };
     if (overlap) {   // delta is ready: the upper stages' own gradients are computed beside stage 0

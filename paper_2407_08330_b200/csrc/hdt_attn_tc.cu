@@ -1422,8 +1422,8 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     constexpr int smem = (4 * (D / 64) + 2) * SUB + 1024 + 64;     // general kernel: Q, two K tiles, V, P
     constexpr int smem_1 = 3 * (D / 64) * SUB + 1024 + 64;
     constexpr int smem_mc = 5 * SUB + 2 * 128 * 4 + 1024 + 64;     // multi-chunk kernel: Q, two K, two V tiles
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
@@ -1433,16 +1433,12 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
                                             8 * SUB + 4 * 128 * 4 + 1024 + 64));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
-        attr = true;
+        attr.set();
     }
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
     if (a.hdr != nullptr) {          // counts on the device only: the looping kernel with all its CTAs
-        static int n_sm_e = 0;
-        if (n_sm_e == 0) {
-            int dev = 0;
-            HDT_CUDA_CHECK(cudaGetDevice(&dev));
-            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm_e, cudaDevAttrMultiProcessorCount, dev));
-        }
+        int n_sm_e = 0;
+        if (const int rc_ = sm_count(&n_sm_e)) return rc_;
         const int grid = n_sm_e * (D == 64 ? 4 : 2);
         if (dirs) k_fwd_tc_loop<D, true><<<grid, 128, smem_1, st>>>(tq, tk, tv, om, a);
         else k_fwd_tc_loop<D><<<grid, 128, smem_1, st>>>(tq, tk, tv, om, a);
@@ -1460,28 +1456,23 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
     } else if (a.n_fused > 0 && split_launch) {
         if (D == 64 && a.no_persistent == 2 && !dirs) {   // option: the persistent single-CTA-per-SM kernel
             constexpr int smem_p = 8 * SUB + 4 * 128 * 4 + 1024 + 64;
-            int dev = 0, n_sm = 0;
-            HDT_CUDA_CHECK(cudaGetDevice(&dev));
-            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
+            int n_sm = 0;
+            if (const int rc_ = sm_count(&n_sm)) return rc_;
             const long long items = (long long)a.n_fused * a.H;
             k_fwd_tc_p<<<(int)(items < n_sm ? items : n_sm), 512, smem_p, st>>>(tq, tk, tv, a);
         } else if (a.no_persistent == 3 && !dirs) {       // option: one CTA per (block, head), no loop
             k_fwd_tc<D, true><<<dim3(a.n_fused, a.H), 128, smem_1, st>>>(tq, tk, tv, a);
         } else {
-            static int n_sm = 0;      // once per process (one process per GPU)
-            if (n_sm == 0) {
-                int dev = 0;
-                HDT_CUDA_CHECK(cudaGetDevice(&dev));
-                HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-            }
+            int n_sm = 0;
+            if (const int rc_ = sm_count(&n_sm)) return rc_;
             const long long items = (long long)a.n_fused * a.H;
             const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
             if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
             else if (g_phase_stamps == 1 && D == 64) {
-                static bool attr_s = false;
-                if (!attr_s) {
+                static DevOnce attr_s;
+                if (!attr_s.done()) {
                     HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<64, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
-                    attr_s = true;
+                    attr_s.set();
                 }
                 k_fwd_tc_loop<64, false, true><<<(int)(items < slots ? items : slots), 128, 3 * SUB + 1024 + 64, st>>>(tq, tk, tv, om, a);
             } else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
@@ -1512,10 +1503,10 @@ static int launch_fwd_tc_upper_t(const FwdStageArgs &a, cudaStream_t st) {
     int rc = make_tmap_bf16(&tq, a.q, D, a.H, a.T, 128);
     if (rc) return rc;
     constexpr int smem = (3 * (D / 64) + 2) * SUB + 1024 + 64;
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr = true;
+        attr.set();
     }
     FwdStageArgs b = a;
     b.rest_only = 0;
@@ -1524,10 +1515,10 @@ static int launch_fwd_tc_upper_t(const FwdStageArgs &a, cudaStream_t st) {
     // instead of two and the stage runs in one wave
     if (a.n_fused == a.nb && a.queue_split != nullptr && !g_no_fwd_mc) {
         constexpr int smem_1 = 3 * (D / 64) * SUB + 1024 + 64;
-        static bool attr_1 = false;
-        if (!attr_1) {
+        static DevOnce attr_1;
+        if (!attr_1.done()) {
             HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
-            attr_1 = true;
+            attr_1.set();
         }
         k_fwd_tc<D, true, true><<<dim3(a.nb, a.H), 128, smem_1, st>>>(tq, tq, tq, b);
     } else

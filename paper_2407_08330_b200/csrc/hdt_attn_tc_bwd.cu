@@ -782,12 +782,22 @@ __device__ long long g_bwd_phase_cycles[16];
 // Thread t: row t % 128 (TMEM lane), column quarter t / 128.
 // ---------------------------------------------------------------------------------------------
 
-template <bool SPLIT, bool DIRS = false>
+// SPLIT = 0: self-contained blocks.  SPLIT = 1: the other blocks, split families in two walks (first
+// every block as query rows over its key span for dQ, then as keys over the same span taken as query
+// rows for dK, dV; S, dP, P, dS of every tile pair are computed twice; no atomics, deterministic).
+// SPLIT = 2: the other blocks in ONE walk: every block is taken as keys only and walks its span as
+// query tiles; dK and dV accumulate in TMEM as before, and the tile's dQ contribution dS K (a fresh
+// accumulator per tile pair) is drained as fp32 into a swizzled staging tile and added to the
+// fp32 buffer a.dq_acc [T, H, 64] by two TMA reduce-add copies (the L2 does the additions; the
+// order in which the CTAs reach a row is not fixed, so dQ of those rows is reproducible only up to
+// fp32 rounding of the sum).  k_dq_finish then scales and converts the sums.
+template <int SPLIT, bool DIRS = false>
 __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
                                                      const __grid_constant__ CUtensorMap tm_v,
                                                      const __grid_constant__ CUtensorMap tm_do,
-                                                     const __grid_constant__ StoreMaps sm_out, const BwdStageArgs a) {
+                                                     const __grid_constant__ StoreMaps sm_out,
+                                                     const __grid_constant__ CUtensorMap tm_acc, const BwdStageArgs a) {
     constexpr int D = 64;
     constexpr uint32_t TM_S = 0, TM_DP = 128, TM_DQ = 256, TM_DK = 320, TM_DV = 384, TM_COLS = 512;
     constexpr int STG = SUB;              // one staged output tile: [128 x 64] bf16, swizzled like the inputs
@@ -796,7 +806,9 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     uint8_t *sIn = sm;                    // 2 stages x {Q, dO, K, V}
     uint8_t *sP = sm + 8 * SUB;           // 2 sub-tiles; later staging of dQ (sub-tile 0), dK (sub-tile 1)
     uint8_t *sDS = sP + 2 * SUB;          // 2 sub-tiles; later staging of dV (sub-tile 0)
-    uint64_t *bar_tma = (uint64_t *)(sDS + 2 * SUB);   // [2]
+    constexpr bool onewalk = SPLIT == 2;
+    uint8_t *sAcc = sDS + 2 * SUB;        // one walk: a tile's dQ contribution as fp32, two swizzled sub-tiles of [128 x 32]
+    uint64_t *bar_tma = (uint64_t *)(sAcc + (onewalk ? 2 * SUB : 0));   // [2]
     uint64_t *bar_a = bar_tma + 2, *bar_b = bar_tma + 3;
     uint32_t *slot = (uint32_t *)(bar_tma + 4);
     volatile int *abort_flag = (volatile int *)(slot + 1);
@@ -837,7 +849,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
     // then as keys over the same span taken as query rows (dK, dV accumulate).  EMPTY blocks are
     // written as zeros on the spot.  Block ids are fetched two units ahead, records one unit ahead,
     // items two ahead and row statistics one ahead: no global-memory latency between two items.
-    constexpr bool split = SPLIT;
+    constexpr bool split = SPLIT != 0;
     const int unit_base = split ? a.n_fused : 0;
     const int n_units = (split ? (a.nb - a.n_fused) : a.n_fused) * H;
     struct UB { int blk, h; };
@@ -904,6 +916,12 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                     role = 2;
                 } else {
                     const int nch = (cur.kb - cur.ka + 127) >> 7, c0 = cur.ka + 128 * chunk;
+                    if constexpr (onewalk) {   // keys = the block, query tile = chunk of its span; all three products
+                        x.q0 = c0; x.qe = cur.kb; x.k0 = cur.r0; x.ke = cur.r1;
+                        x.flags = F_DQ | F_DKDV | (chunk > 0 ? F_ACC : 0) | (chunk == nch - 1 ? F_LAST : 0);
+                        if (++chunk == nch) { chunk = 0; role = 2; }
+                        return x;
+                    }
                     if (role == 0) { x.q0 = cur.r0; x.qe = cur.r1; x.k0 = c0; x.ke = cur.kb; }
                     else { x.q0 = c0; x.qe = cur.kb; x.k0 = cur.r0; x.ke = cur.r1; }
                     x.flags = (role == 0 ? F_DQ : F_DKDV) | (chunk > 0 ? F_ACC : 0) | (chunk == nch - 1 ? F_LAST : 0);
@@ -966,6 +984,9 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                 issue_sdp(0, keys16(d0));
             }
         }
+        // one walk: the thread that requests the reduce-add copies of a staged dQ tile, and the tile's place
+        const bool red_thread = onewalk && tid == 96;
+        int red_q0 = -1, red_h = 0;
         const bool stamp = (tid == 0 && blockIdx.x == 0);
         long long ph_acc[12] = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
         long long t_last = clock64();
@@ -984,7 +1005,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             const int e_row = d0.q0 + rl;
             const int c_self = e_row - k0, c_head = (rc.lo < e_row) ? rc.lo - k0 : -0x40000000;
             const bool keep_head = (a.dirs & 1) != 0, keep_rest = (a.dirs & ((rc.lo >= e_row) ? 4 : 2)) != 0;
-            const int flags = SPLIT ? d0.flags : (F_DQ | F_DKDV | F_LAST);   // constant for self-contained blocks
+            const int flags = split ? d0.flags : (F_DQ | F_DKDV | F_LAST);   // constant for self-contained blocks
             uint8_t *st = sIn + (it & 1) * 4 * SUB;
 
             HDT_STAMP(0);
@@ -993,6 +1014,15 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             if (store_thread) bulk_wait_read();   // the previous item's staged gradients have left shared memory
             __syncthreads();
             tc_fence_after();
+            if constexpr (onewalk) {
+                // the previous item's dQ tile is staged (all threads have passed the barrier): add it to the buffer
+                if (red_thread && red_q0 >= 0 && !*abort_flag) {
+                    tma_reduce_add_3d(&tm_acc, 0, red_h, red_q0, sAcc);
+                    tma_reduce_add_3d(&tm_acc, 32, red_h, red_q0, sAcc + SUB);
+                    bulk_commit();
+                    red_q0 = -1;
+                }
+            }
             HDT_STAMP(1);
             // ---- P and dS of this thread's 32 columns, in two halves of 16 ----
             if (32 * qt < Nc) {
@@ -1057,9 +1087,10 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                 } else if (warp == 2 && (flags & F_DQ)) {     // dQ (+)= dS K, contraction over the keys
                     const uint32_t idesc = idesc_bf16(D, false, true);
                     const uint64_t da = smem_desc(smem_u32(sDS), 0, 1024), db = smem_desc(sb + 2 * SUB, SUB, 1024);
+                    const uint32_t acc_q = onewalk ? 0u : acc;     // one walk: a fresh dQ contribution per tile pair
                     for (int kk = 0; kk < Nc / 16; ++kk)
                         mma_ss(tmem + TM_DQ, da + (uint64_t)((kk / 4) * (SUB >> 4) + (kk % 4) * 2),
-                               db + (uint64_t)(kk * 128), idesc, acc | (kk > 0));
+                               db + (uint64_t)(kk * 128), idesc, acc_q | (kk > 0));
                 }
                 mma_commit(bar_b);   // every issuer arrives, with or without MMAs of its own
                 HDT_STAMP(10);
@@ -1074,16 +1105,32 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             }
             HDT_STAMP(4);
             if (warp == 0) ok = mbar_wait(bar_b, it & 1, abort_flag, WAIT_CYCLES) && ok;   // this item's output MMAs
+            if (red_thread) bulk_wait_read();      // the reduce-add copies have read the staging tile
             __syncthreads();
             tc_fence_after();
             HDT_STAMP(5);
             if (tid == 0 && d2.valid && !*abort_flag) issue_tma(it + 2, d2);   // this stage is free again
+            if constexpr (onewalk) {
+                // this tile pair's dQ contribution: 16 fp32 columns of this thread's query row into the
+                // staging tile (sub-tile = column half, 128-byte rows, swizzled); the additions are requested
+                // behind the next CTA barrier.  Rows beyond the span's end hold exact zeros (their dS is 0).
+                uint32_t r[16];
+                tmem_ld16(tmem + TM_DQ + lane_base + 16 * qt, r);
+                tmem_wait_ld();
+                uint8_t *dst = sAcc + (qt >> 1) * SUB;
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    *reinterpret_cast<uint4 *>(dst + swz(rl, (qt & 1) * 4 + j)) = make_uint4(r[4 * j], r[4 * j + 1], r[4 * j + 2], r[4 * j + 3]);
+                fence_proxy_async_smem();
+                red_q0 = d0.q0; red_h = h;
+            }
             if (flags & F_LAST) {
                 // ---- drain: 16 columns of each finished gradient per thread, staged as bf16 ----
                 const int r0 = d0.r0, nrows = d0.nrows;
 #pragma unroll
                 for (int t = 0; t < 3; ++t) {
                     if (!(flags & (t == 0 ? F_DQ : F_DKDV))) continue;   // same in every thread
+                    if (onewalk && t == 0) continue;                     // dQ went to the fp32 buffer tile by tile
                     const uint32_t col = (t == 0) ? TM_DQ : (t == 1) ? TM_DK : TM_DV;
                     const float sc = (t == 2) ? 1.f : a.scale;
                     uint8_t *dst = sP + t * STG;    // staging: one swizzled [128 x 64] tile per tensor
@@ -1119,7 +1166,7 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
                     const int bx = max(__clz(nrows) - 25, 0);          // box of 64 >> bx rows: 64 for nrows >= 64
                     const int b = 64 >> bx;
                     const int off = second ? nrows - b : 0;
-                    const bool use = (flags & (t == 0 ? F_DQ : F_DKDV)) && (!second || nrows > b);
+                    const bool use = (flags & (t == 0 ? F_DQ : F_DKDV)) && (!second || nrows > b) && !(onewalk && t == 0);
                     if (use) tma_store_3d(&sm_out.m[t][bx], 0, h, r0 + off, sP + t * STG + off * 128);
                     bulk_commit();
                 }
@@ -1131,12 +1178,43 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
             for (int i = 0; i < 12; ++i) g_bwd_phase_cycles[i] += ph_acc[i];
             g_bwd_phase_cycles[12] += it;
         }
+        if constexpr (onewalk) {       // the last item's dQ tile
+            __syncthreads();
+            if (red_thread && red_q0 >= 0 && !*abort_flag) {
+                tma_reduce_add_3d(&tm_acc, 0, red_h, red_q0, sAcc);
+                tma_reduce_add_3d(&tm_acc, 32, red_h, red_q0, sAcc + SUB);
+                bulk_commit();
+            }
+            if (red_thread) bulk_wait_read();
+        }
     }
     if (!ok) atomicCAS(a.status, 0, HDT_ERR_TIMEOUT);
     if (store_thread) bulk_wait_read();
     tc_fence_before();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
+// After the one-walk kernel: dQ of the rows of every block that is neither self-contained nor EMPTY
+// is the sum in a.dq_acc times the softmax scale; it goes to dq as bf16 and, for rows that live on in
+// the next stage, as fp32 to that stage's buffer.  One CTA per (block after the first n_fused of
+// queue_split, head); thread t: 16-byte pieces t, t + 256, ... of the block's [rows x 64] fp32 tile.
+__global__ void __launch_bounds__(256) k_dq_finish(const BwdStageArgs a) {
+    const int *rec = a.blocks + 5 * (size_t)a.queue_split[a.n_fused + blockIdx.x];
+    const int r0 = rec[0], nrows = rec[1] - r0, h = blockIdx.y, H = a.H;
+    if (rec[4] & HDT_BLK_EMPTY) return;          // written as zeros by the one-walk kernel
+    for (int i = threadIdx.x; i < nrows * 16; i += 256) {
+        const int r = i >> 4, c = i & 15;
+        const size_t row = (size_t)(r0 + r);
+        const float4 x = *reinterpret_cast<const float4 *>(a.dq_acc + (row * H + h) * 64 + 4 * c);
+        const float4 y = make_float4(x.x * a.scale, x.y * a.scale, x.z * a.scale, x.w * a.scale);
+        *reinterpret_cast<uint2 *>(reinterpret_cast<__nv_bfloat16 *>(a.dq) + (row * H + h) * 64 + 4 * c) =
+            make_uint2(pack_bf16(y.x, y.y), pack_bf16(y.z, y.w));
+        if (a.part_dq != nullptr) {
+            const int u = a.up[row];
+            if (u >= 0) *reinterpret_cast<float4 *>(a.part_dq + ((size_t)u * H + h) * 64 + 4 * c) = y;
+        }
+    }
 }
 
 template <int D>
@@ -1151,10 +1229,10 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     rc = make_tmap_bf16(&tdo, a.d_o, D, a.H, a.T, 128);
     if (rc) return rc;
     constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64 + 512;
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr = true;
+        attr.set();
     }
     BwdStageArgs b = a;
     b.rest_only = 0;
@@ -1172,18 +1250,26 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     if (D == 64 && a.nb > 0 && (!a.no_persistent || a.no_persistent == 4 || a.no_persistent == 6)) {   // (no_persistent == 5: the looping kernel below instead)
         // the persistent kernel takes everything: first the blocks of split families (longest first),
         // then the self-contained blocks
-        constexpr int smem_p = 12 * SUB + 1024 + 64;
-        static bool attr_p = false;
-        static int n_sm = 0;
-        if (!attr_p) {
-            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
-            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
-            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
-            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
-            int dev = 0;
-            HDT_CUDA_CHECK(cudaGetDevice(&dev));
-            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-            attr_p = true;
+        constexpr int smem_p = 12 * SUB + 1024 + 64, smem_w = 14 * SUB + 1024 + 64;
+        static DevOnce attr_p;
+        int n_sm = 0;
+        if (const int rc_ = sm_count(&n_sm)) return rc_;
+        if (!attr_p.done()) {
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_p));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_w));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_p<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_w));
+            attr_p.set();
+        }
+        // split families in one walk when the caller supplied the fp32 dQ buffer (zeroed): dQ tiles are
+        // added to it and k_dq_finish scales and converts the sums afterwards
+        const bool onewalk = a.dq_acc != nullptr && a.nb > a.n_fused;
+        CUtensorMap tacc = tq;       // (a valid map in the parameter slot of the kernels that do not use it)
+        if (onewalk) {
+            rc = make_tmap_f32_acc(&tacc, a.dq_acc, a.H, a.T, 128);
+            if (rc) return rc;
         }
         for (int mode = 1; mode >= 0; --mode) {
             const long long units = (long long)(mode ? a.nb - a.n_fused : a.n_fused) * a.H;
@@ -1196,11 +1282,18 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
             BwdStageArgs c = a;
             c.rest_only = mode;
             const int grid_p = (int)(units < n_sm ? units : n_sm);
-            if (dirs) {
-                if (mode) k_bwd_tc_p<true, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
-                else k_bwd_tc_p<false, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
-            } else if (mode) k_bwd_tc_p<true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
-            else k_bwd_tc_p<false><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, c);
+            if (mode && onewalk) {
+                if (dirs) k_bwd_tc_p<2, true><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);
+                else k_bwd_tc_p<2><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);
+                count_launch();
+                HDT_CUDA_CHECK(cudaGetLastError());
+                const int n_rest = a.nb - a.n_fused;
+                k_dq_finish<<<dim3(n_rest, a.H), 256, 0, st>>>(c);
+            } else if (dirs) {
+                if (mode) k_bwd_tc_p<1, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, tacc, c);
+                else k_bwd_tc_p<0, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, tacc, c);
+            } else if (mode) k_bwd_tc_p<1><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, tacc, c);
+            else k_bwd_tc_p<0><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, tacc, c);
             count_launch();
             HDT_CUDA_CHECK(cudaGetLastError());
         }
@@ -1209,14 +1302,12 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     if (((D == 128 && !a.no_persistent) || (D == 64 && a.no_persistent == 5)) && a.n_fused > 0 && !dirs) {
         // self-contained blocks through the looping kernel, the rest through the general one
         constexpr int smem_l = (4 * (D / 64) + 4 + (D / 64)) * SUB + 1024 + 64;
-        static bool attr_l = false;
-        static int n_sm_l = 0;
-        if (!attr_l) {
+        static DevOnce attr_l;
+        int n_sm_l = 0;
+        if (const int rc_ = sm_count(&n_sm_l)) return rc_;
+        if (!attr_l.done()) {
             HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_loop<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_l));
-            int dev = 0;
-            HDT_CUDA_CHECK(cudaGetDevice(&dev));
-            HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm_l, cudaDevAttrMultiProcessorCount, dev));
-            attr_l = true;
+            attr_l.set();
         }
         const long long items = (long long)a.n_fused * a.H;
         k_bwd_tc_loop<D><<<(int)(items < n_sm_l ? items : n_sm_l), 256, smem_l, st>>>(tq, tk, tv, tdo, outs, a);
@@ -1228,10 +1319,10 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     if (n_general > 0) {
         dim3 grid(n_general, a.H);
         if (dirs) {
-            static bool attr_d = false;
-            if (!attr_d) {
+            static DevOnce attr_d;
+            if (!attr_d.done()) {
                 HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-                attr_d = true;
+                attr_d.set();
             }
             k_bwd_tc<D, false, true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, b);
         } else k_bwd_tc<D><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, b);
@@ -1257,10 +1348,10 @@ static int launch_bwd_tc_upper_t(const BwdStageArgs &a, cudaStream_t st) {
     int rc = make_tmap_bf16(&tq, a.q, D, a.H, a.T, 128);
     if (rc) return rc;
     constexpr int smem = (4 * (D / 64) + 4) * SUB + 1024 + 64 + 512;
-    static bool attr = false;
-    if (!attr) {
+    static DevOnce attr;
+    if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr = true;
+        attr.set();
     }
     BwdStageArgs b = a;
     b.rest_only = 0;

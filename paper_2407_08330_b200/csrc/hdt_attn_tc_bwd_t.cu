@@ -366,9 +366,10 @@ __global__ void __maxnreg__(120) k_bwd_tc_t(const __grid_constant__ CUtensorMap 
 int launch_bwd_tc_fused64(const BwdStageArgs &a, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                           const CUtensorMap &tdo, const StoreMaps &outs, cudaStream_t st) {
     constexpr int smem = 7 * SUB + 64;
-    static bool attr = false;
-    static int n_sm = 0;
-    if (!attr) {
+    static DevOnce attr;
+    int n_sm = 0;
+    if (const int rc_ = sm_count(&n_sm)) return rc_;
+    if (!attr.done()) {
         const void *fns[6] = {(const void *)k_bwd_tc_t<false>,       (const void *)k_bwd_tc_t<true>,
                               (const void *)k_bwd_tc_t<false, true>, (const void *)k_bwd_tc_t<false, false, true>,
                               (const void *)k_bwd_tc_t<false, true, true>, nullptr};
@@ -376,10 +377,7 @@ int launch_bwd_tc_fused64(const BwdStageArgs &a, const CUtensorMap &tq, const CU
             HDT_CUDA_CHECK(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             HDT_CUDA_CHECK(cudaFuncSetAttribute(fns[i], cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
         }
-        int dev = 0;
-        HDT_CUDA_CHECK(cudaGetDevice(&dev));
-        HDT_CUDA_CHECK(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, dev));
-        attr = true;
+        attr.set();
     }
     const long long items = (long long)a.n_fused * a.H;
     if (items == 0) return HDT_OK;

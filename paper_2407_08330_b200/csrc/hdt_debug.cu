@@ -100,6 +100,64 @@ extern "C" int hdt_debug_gemm(const void *a, const void *b, float *c, int32_t N,
 }
 
 
+namespace hdt {
+// One CTA that sets up what the attention kernels set up (an mbarrier, TMEM columns) and then waits on
+// a barrier nobody ever arrives on: no TMA copy and no MMA is issued, so nothing is in flight when the
+// bounded wait gives up.  It then takes the failure path of the attention kernels: abort flag,
+// HDT_ERR_TIMEOUT with kernel id 15 / wait site 1 / the wait limit's low bits in the status word, TMEM
+// released, normal exit.  second[0] counts the threads that saw the abort flag and left their own wait early.
+__global__ void __launch_bounds__(128) k_debug_wait(long long limit_cycles, int *status, int *second) {
+    __shared__ uint64_t bar;
+    __shared__ uint32_t slot;
+    __shared__ int abort_flag_s;
+    volatile int *abort_flag = &abort_flag_s;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    if (tid == 0) {
+        mbar_init(&bar, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(&slot, 32);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = slot;
+    const long long t0 = clock64();
+    const bool ok = mbar_wait(&bar, 0, abort_flag, limit_cycles);
+    if (!ok) {
+        if (clock64() - t0 <= limit_cycles) atomicAdd(second, 1);       // left early through the abort flag
+        if (tid == 0) {
+            if (atomicCAS(status, 0, HDT_ERR_TIMEOUT) == 0) {
+                status[1] = (15 << 8) | 1;
+                status[2] = (int)(limit_cycles & 0x7fffffff);
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 32);
+}
+}  // namespace hdt
+
+// Test hook for the failure path of the bounded device-side waits (no counterpart in the paper): see
+// k_debug_wait.  Returns what hdt_device_status returns afterwards (HDT_ERR_TIMEOUT when the path
+// works) and, in *left_early, how many of the 128 threads stopped waiting because of the abort flag.
+extern "C" int hdt_debug_wait_timeout(int64_t limit_cycles, int32_t *left_early, void *stream) {
+    if (limit_cycles < 1000 || limit_cycles > 2000000000LL)
+        return set_error(HDT_ERR_INVALID_ARG, "hdt_debug_wait_timeout: limit_cycles must be 1e3..2e9");
+    cudaStream_t st = (cudaStream_t)stream;
+    int *status = device_status_ptr();
+    if (!status) return HDT_ERR_CUDA;
+    k_debug_wait<<<1, 128, 0, st>>>((long long)limit_cycles, status, status + 3);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    HDT_CUDA_CHECK(cudaStreamSynchronize(st));
+    int h[4] = {0, 0, 0, 0};
+    HDT_CUDA_CHECK(cudaMemcpy(h, status, sizeof(h), cudaMemcpyDeviceToHost));
+    if (left_early) *left_early = h[3];
+    return hdt_device_status(stream);
+}
+
 // Diagnostics (no counterpart in the paper): SM cycles that CTA 0 of the persistent backward kernel
 // spent in each of its phases since the last call (out16[0..11]) and the items it processed (out16[12]).
 // Waits for the device.

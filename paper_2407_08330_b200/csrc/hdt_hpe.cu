@@ -413,11 +413,11 @@ extern "C" int hdt_hpe(const hdt_index_t *ix, const int8_t *level, const int32_t
             const int per_sm = (int)max((size_t)1, min((size_t)2, (size_t)(220 * 1024) / (smem + 1024)));
             const int nb = min(n_tiles, 148 * per_sm);
             int *status = device_status_ptr();
-            static bool attr_done = false;
-            if (!attr_done) {
+            static DevOnce attr_done;
+            if (!attr_done.done()) {
                 HDT_CUDA_CHECK(cudaFuncSetAttribute(k_hpe_acc_bulk<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
                 HDT_CUDA_CHECK(cudaFuncSetAttribute(k_hpe_acc_bulk<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-                attr_done = true;
+                attr_done.set();
             }
             if (dtype == HDT_BF16) k_hpe_acc_bulk<true><<<nb, dim3(tx, 4), smem, st>>>(level, pvec, n_tiles, d_model, ns, x, status);
             else k_hpe_acc_bulk<false><<<nb, dim3(tx, 4), smem, st>>>(level, pvec, n_tiles, d_model, ns, x, status);

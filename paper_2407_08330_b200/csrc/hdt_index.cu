@@ -747,24 +747,32 @@ static cudaError_t launch_chain(void (*kern)(KArgs...), dim3 grid, dim3 block, s
 // index keeps its buffer until the header has been read).
 static const int kUnset = 0x7fffffff;
 static std::mutex g_pinned_mu;
-static std::vector<DevHeader *> g_pinned_free;
-static DevHeader *pinned_acquire() {
+// A landing buffer for the header with the event that marks the end of its copy.
+struct PinnedSlot { DevHeader *p; cudaEvent_t ev; };
+static std::vector<PinnedSlot> g_pinned_free;
+static bool pinned_acquire(PinnedSlot *out) {
     {
         std::lock_guard<std::mutex> lk(g_pinned_mu);
         if (!g_pinned_free.empty()) {
-            DevHeader *p = g_pinned_free.back();
+            *out = g_pinned_free.back();
             g_pinned_free.pop_back();
-            return p;
+            return true;
         }
     }
-    DevHeader *p = nullptr;
-    if (cudaMallocHost((void **)&p, sizeof(DevHeader)) != cudaSuccess) { (void)cudaGetLastError(); return nullptr; }
-    return p;
+    PinnedSlot s{nullptr, nullptr};
+    if (cudaMallocHost((void **)&s.p, sizeof(DevHeader)) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    if (cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cudaFreeHost(s.p);
+        return false;
+    }
+    *out = s;
+    return true;
 }
-static void pinned_release(DevHeader *p) {
+static void pinned_release(DevHeader *p, cudaEvent_t ev) {
     if (!p) return;
     std::lock_guard<std::mutex> lk(g_pinned_mu);
-    g_pinned_free.push_back(p);
+    g_pinned_free.push_back(PinnedSlot{p, ev});
 }
 
 extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const int32_t *cu_seqlens,
@@ -822,11 +830,11 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     const int g_chunk = max(1, (T + CHUNK - 1) / CHUNK);
     const int g_stride = max(1, min((T + 255) / 256, 148 * 8));
     static const int kSmemCap = 200 * 1024;
-    static bool attr_done = false;     // once per process (one process per GPU)
-    if (!attr_done) {
+    static DevOnce attr_done;
+    if (!attr_done.done()) {
         HDT_BUILD_CHECK(cudaFuncSetAttribute(k_walk, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemCap));
         HDT_BUILD_CHECK(cudaFuncSetAttribute(k_upper_stages, cudaFuncAttributeMaxDynamicSharedMemorySize, USMEM));
-        attr_done = true;
+        attr_done.set();
     }
     // One CTA builds all stages above 0 when they are small (documents: a few percent of the
     // tokens, up to 3-4 stages).  A caller that allows many stages expects deep trees, whose upper
@@ -942,14 +950,16 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     // by the driver).  First and last word of the buffer are set to a value the device never writes
     // (status is 0 or negative, tail is 0) so that the host can watch the copy land: it is the last
     // operation of the build on the stream, and its words arrive in order.
-    DevHeader *h_pinned = pinned_acquire();
+    PinnedSlot slot_{nullptr, nullptr};
+    DevHeader *h_pinned = pinned_acquire(&slot_) ? slot_.p : nullptr;
     if (!h_pinned) {
         delete ix;
         return set_error(HDT_ERR_CUDA, "hdt_build_index: no pinned host memory for the index header");
     }
-    h_pinned->status = kUnset;
-    h_pinned->tail = kUnset;
+    // every word of the (reused) landing buffer is poisoned, not only the two the host watches
+    for (size_t w = 0; w < sizeof(DevHeader) / sizeof(int); ++w) reinterpret_cast<int *>(h_pinned)[w] = kUnset;
     ix->h_pinned = h_pinned;
+    ix->hdr_ev = slot_.ev;
     ix->hdr_dev = hdr;
     ix->stream = st;
     ix->max_stages = ms;
@@ -966,11 +976,13 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             cs = sdc->s;
             ix->stream = cs;
         }
-        const cudaError_t e_ = cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, cs);
+        cudaError_t e_ = cudaMemcpyAsync(h_pinned, hdr, sizeof(DevHeader), cudaMemcpyDeviceToHost, cs);
+        if (e_ == cudaSuccess) e_ = cudaEventRecord(slot_.ev, cs);      // the end of the copy, as the runtime sees it
         if (e_ != cudaSuccess) {
-            pinned_release(h_pinned);
+            (void)cudaStreamSynchronize(cs);                              // the copy may be queued: let it land first
+            pinned_release(h_pinned, slot_.ev);
             delete ix;
-            return set_error(HDT_ERR_CUDA, "cudaMemcpyAsync of the index header failed: %s", cudaGetErrorString(e_));
+            return set_error(HDT_ERR_CUDA, "queueing the copy of the index header failed: %s", cudaGetErrorString(e_));
         }
     }
 #undef HDT_BUILD_CHECK
@@ -989,25 +1001,30 @@ namespace hdt {
 int index_ready(const hdt_index *cix) {
     hdt_index *ix = const_cast<hdt_index *>(cix);
     if (ix->pending) {
-        // The host watches the copy land instead of waiting in the driver; after a bounded number
-        // of polls the ordinary wait takes over.
+        // The host watches the copy land instead of sleeping in the driver: the first and the last
+        // word of the buffer change when (parts of) the copy have arrived.  That is only a hint — the
+        // bytes of one copy need not reach host memory in address order — so the event recorded
+        // behind the copy decides: it is polled (about a microsecond per query) and, after a bounded
+        // number of polls, waited for.
         DevHeader *hp = ix->h_pinned;
         volatile int *p_status = &hp->status, *p_tail = &hp->tail;
         bool landed = false;
         for (long long spin = 0; spin < 20000000LL && !landed; ++spin) landed = (*p_tail != kUnset && *p_status != kUnset);
-        if (!landed) {
-            const cudaError_t e_ = cudaStreamSynchronize(ix->stream);
-            if (e_ != cudaSuccess) {
-                ix->pending = 0;
-                ix->failed = HDT_ERR_CUDA;
-                pinned_release(hp);
-                ix->h_pinned = nullptr;
-                return set_error(HDT_ERR_CUDA, "waiting for the index build failed: %s", cudaGetErrorString(e_));
-            }
+        cudaError_t e_ = cudaErrorNotReady;
+        for (int poll = 0; poll < 200000 && e_ == cudaErrorNotReady; ++poll) e_ = cudaEventQuery(ix->hdr_ev);
+        if (e_ == cudaErrorNotReady) e_ = cudaEventSynchronize(ix->hdr_ev);
+        if (e_ != cudaSuccess) {
+            (void)cudaGetLastError();
+            (void)cudaStreamSynchronize(ix->stream);
+            ix->pending = 0;
+            ix->failed = HDT_ERR_CUDA;
+            pinned_release(hp, ix->hdr_ev);
+            ix->h_pinned = nullptr;
+            return set_error(HDT_ERR_CUDA, "waiting for the index build failed: %s", cudaGetErrorString(e_));
         }
         std::atomic_thread_fence(std::memory_order_acquire);
         const DevHeader h = *hp;
-        pinned_release(hp);
+        pinned_release(hp, ix->hdr_ev);
         ix->h_pinned = nullptr;
         ix->pending = 0;
         ix->failed = h.status;

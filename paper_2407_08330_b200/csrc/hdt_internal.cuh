@@ -5,6 +5,7 @@
 #include <atomic>
 
 #include "../../include/hdt.h"
+#include "../../include/hdt_debug.h"
 
 namespace hdt {
 
@@ -47,6 +48,7 @@ struct hdt_index {
     int failed;                       // hdt_status_t found in the header (or by its check), 0 = fine
     int err_pos, max_stages;
     hdt::DevHeader *h_pinned;         // pinned landing buffer (from a pool), nullptr once released
+    cudaEvent_t hdr_ev;               // recorded behind the copy of the header into h_pinned
     const hdt::DevHeader *hdr_dev;    // the header in the index workspace
     cudaStream_t stream;              // stream of the build
 };
@@ -77,6 +79,23 @@ struct ProfScope {
         if (e_ != cudaSuccess)                                                                \
             return hdt::set_error(HDT_ERR_CUDA, "%s failed: %s", #expr, cudaGetErrorString(e_)); \
     } while (0)
+
+// State that is set up once per device (function attributes such as the dynamic shared-memory
+// limit belong to a device's copy of the kernel, not to the process): one flag per device ordinal,
+// read and set for the current device.  Two host threads that race on the first call both do the
+// set-up, which is idempotent.
+struct DevOnce {
+    std::atomic<bool> f[64];
+    static int cur() {
+        int d = 0;
+        if (cudaGetDevice(&d) != cudaSuccess || d < 0 || d >= 64) d = 0;
+        return d;
+    }
+    bool done() const { return f[cur()].load(std::memory_order_acquire); }
+    void set() { f[cur()].store(true, std::memory_order_release); }
+};
+// Number of SMs of the current device (cached per device ordinal).
+int sm_count(int *n_sm);
 
 // Side stream (one per host thread and device, created on first use): work that does not depend
 // on the main kernel of a call runs beside it.  fork / join are events for the two hand-overs.
@@ -204,6 +223,8 @@ struct BwdStageArgs {
     // own (next_own_*, at up[e]; nullptr without a stage 2); they go to dq / dk / dv at its token.
     int final_merge;
     const float *next_own_dq, *next_own_dk, *next_own_dv;
+    float *dq_acc;                                // stage 0, head_dim 64: fp32 [T,H,64] buffer, zero on entry, that the one-walk kernel of the
+                                                  // split families adds its dQ tiles to (nullptr: they are walked twice instead)
     int gather_end_q, gather_end_k;               // gathering kernel: elements at or beyond these read as zero rows on the Q/dO and the K/V side (0: n)
 };
 

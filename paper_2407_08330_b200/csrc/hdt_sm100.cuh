@@ -87,6 +87,16 @@ __device__ __forceinline__ void tma_store_3d(const CUtensorMap *tm, int x, int y
                  : "memory");
 }
 
+// 3-D tiled reduction: the shared-memory box (same format as the map's loads) is ADDED, element by
+// element, to the global tensor (the map's data type decides the arithmetic: fp32 here); the
+// additions are performed by the memory system, atomically per element.  x * element size must be a
+// multiple of 16 bytes and no coordinate may be negative.  Completion as for tma_store_3d.
+__device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap *tm, int x, int y, int z, const void *src) {
+    asm volatile("cp.reduce.async.bulk.tensor.3d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2, %3}], [%4];" ::"l"(tm),
+                 "r"(x), "r"(y), "r"(z), "r"(smem_u32(src))
+                 : "memory");
+}
+
 // Bulk copy of `bytes` (multiple of 16, both addresses 16-byte aligned) from shared to global
 // memory; completion is tracked per thread in bulk groups.
 __device__ __forceinline__ void bulk_store(void *gdst, const void *ssrc, uint32_t bytes) {

@@ -40,6 +40,22 @@ inline int make_tmap_bf16(CUtensorMap *tm, const void *base, int D, int H, long 
     return HDT_OK;
 }
 
+// fp32 accumulation buffer [T, H, 64] for reduce-add copies: box = (32 floats, 1, box_rows), i.e.
+// 128-byte rows with the 128-byte swizzle; a [rows x 64] tile is two such boxes (x = 0 and x = 32).
+inline int make_tmap_f32_acc(CUtensorMap *tm, const void *base, int H, long long T, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return set_error(HDT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    cuuint64_t dims[3] = {64, (cuuint64_t)H, (cuuint64_t)(T > 0 ? T : 1)};
+    cuuint64_t strides[2] = {64 * 4, 64 * 4 * (cuuint64_t)H};
+    cuuint32_t box[3] = {32, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void *>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return set_error(HDT_ERR_CUDA, "cuTensorMapEncodeTiled (fp32) failed with CUresult %d", (int)r);
+    return HDT_OK;
+}
+
 // Output tiles of the persistent backward kernels leave through TMA stores.  A block has 1..128 rows
 // and a store box has a fixed number of rows, so each gradient tensor (dq, dk, dv) gets seven maps
 // with boxes of 64, 32, ..., 1 rows and a tile is stored as two (possibly overlapping) boxes of the

@@ -1,5 +1,8 @@
 """GPU parity of hdt_cross_attn_fwd / hdt_cross_attn_bwd (decoder rows attending to a level subset of
-the encoder tokens) against the fp64 oracle: fp32 <= 1e-4, bf16 max <= 2e-2 and mean <= 2e-3."""
+the encoder tokens) against the fp64 oracle: fp32 <= 1e-4, bf16 max <= 2e-2 and mean <= 2e-3, with
+dO ~ N(0,1).  A chosen encoder row collects gradient from every decoder row of its document, so dK and
+dV pass 4, where the bf16 grid is coarser than 2e-2: gradients may exceed the maximum by half a bf16
+ulp of the expected value (the rounding of the stored result), element by element."""
 import numpy as np
 import pytest
 import torch
@@ -20,8 +23,6 @@ def case(b, nq, H, d, dtype, seed):
     f = gen.round_bf16 if dtype == "bf16" else (lambda x: x)
     qd, do = (f(rng.standard_normal((Tq, H, d)).astype(np.float32)) for _ in range(2))
     k, v = (f(rng.standard_normal((b.total_tokens, H, d)).astype(np.float32)) for _ in range(2))
-    if dtype == "bf16":
-        do = do * 0.125      # gradients of order one: the absolute bf16 tolerance is stated for that range
     return cu_q, qd, k, v, do
 
 
@@ -38,9 +39,9 @@ def run(P, b, nq, mask, H, d, dtype, seed):
     dq = torch.full_like(tq, float("nan")); dk = torch.full_like(tk, float("nan")); dv = torch.full_like(tv, float("nan"))
     P.hdt_cross_attn_bwd(lv, cuk, cuq, mask, tq, tk, tv, o, lse, tdo, dq=dq, dk=dk, dv=dv)
     dq_r, dk_r, dv_r = co.backward(b.level, b.cu_seqlens, mask, cu_q, qd, k, v, do)
-    check_close(host(dq), dq_r, dtype, "dQ")
-    check_close(host(dk), dk_r, dtype, "dK")
-    check_close(host(dv), dv_r, dtype, "dV")
+    check_close(host(dq), dq_r, dtype, "dQ", out_rounding=True)
+    check_close(host(dk), dk_r, dtype, "dK", out_rounding=True)
+    check_close(host(dv), dv_r, dtype, "dV", out_rounding=True)
     P.hdt_device_status()
 
 
@@ -90,8 +91,8 @@ def test_cross_attention_config3_anchor_subsets():
     dq_r, dk_r, dv_r = co.backward(b.level, b.cu_seqlens, SEC | SENT, cu_q, qd, k, v, do)
     check_close(host(o), o_r, "bf16", "O")
     check_close(host(lse), lse_r, "bf16", "LSE")
-    check_close(host(dq), dq_r, "bf16", "dQ")
-    check_close(host(dk), dk_r, "bf16", "dK")
-    check_close(host(dv), dv_r, "bf16", "dV")
+    check_close(host(dq), dq_r, "bf16", "dQ", out_rounding=True)
+    check_close(host(dk), dk_r, "bf16", "dK", out_rounding=True)
+    check_close(host(dv), dv_r, "bf16", "dV", out_rounding=True)
     regular = torch.from_numpy(b.level == 3).cuda()
     assert (dk[regular] == 0).all() and (dv[regular] == 0).all()

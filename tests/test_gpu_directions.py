@@ -40,11 +40,10 @@ def test_index_totals_with_directions(P, d):
 
 def run(P, b, H, dim, dtype, d, seed):
     t = gen.make_tensors(seed, b.total_tokens, H, dim, dtype)
-    if dtype == "bf16":
-        # Without the sibling group an anchor collects the whole probability mass of its children:
-        # gradients reach 20 and more, where the spacing of bf16 outputs alone (0.125) exceeds the
-        # absolute tolerance.  A power-of-two scale on dO (exact in bf16) keeps them of order one.
-        t["do"] = t["do"] * 0.125
+    # Without the sibling group an anchor collects the whole probability mass of its children and
+    # gradients reach 20 and more, where the spacing of bf16 outputs alone (0.125) exceeds the
+    # absolute tolerance: gradients may exceed the maximum by half a bf16 ulp of the expected value
+    # (the rounding of the stored result), element by element; dO stays N(0,1).
     idx = P.hdt_build_index(*dev_struct(b), max_stages=12, directions=d)
     q, k, v, do = (dev_tensor(t[n], dtype) for n in ("q", "k", "v", "do"))
     o, lse = P.hdt_attn_fwd(idx, q, k, v)
@@ -53,9 +52,10 @@ def run(P, b, H, dim, dtype, d, seed):
     check_close(host(lse), lse_r, "f32" if dtype == "f32" else "bf16", "LSE")
     dq, dk, dv = P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
     dq_r, dk_r, dv_r = oracle.backward(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], t["do"], directions=d)
-    check_close(host(dq), dq_r, dtype, "dQ")
-    check_close(host(dk), dk_r, dtype, "dK")
-    check_close(host(dv), dv_r, dtype, "dV")
+    # (row_rel: the bf16 rounding of P and dS inside the kernels, 2^-9 relative per term, grows with them)
+    check_close(host(dq), dq_r, dtype, "dQ", out_rounding=True, row_rel=2.0 ** -8)
+    check_close(host(dk), dk_r, dtype, "dK", out_rounding=True, row_rel=2.0 ** -8)
+    check_close(host(dv), dv_r, dtype, "dV", out_rounding=True, row_rel=2.0 ** -8)
     P.hdt_device_status()
 
 

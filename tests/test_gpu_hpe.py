@@ -4,7 +4,7 @@ import pytest
 import torch
 
 import gen
-from gpu_util import dev_struct
+from gpu_util import check_close, dev_struct
 from oracle import hpe_oracle as ho
 
 pytestmark = pytest.mark.gpu
@@ -23,8 +23,10 @@ def run(P, b, d_model, n_levels, dtype, max_stages=8):
     P.hdt_hpe(idx, lv, pa, cu, d_model, n_levels, x=x, accumulate=True)
     pad = torch.from_numpy(b.level < 0).cuda()
     assert torch.equal(x[pad], x0[pad])
-    err = np.abs(x.float().cpu().numpy() - (x0.float().cpu().numpy() + want))
-    assert err.max() <= (1e-4 if dtype == torch.float32 else 6e-2)
+    # bf16: x0 + HPE reaches 4 and more, where the bf16 grid is coarser than 2e-2: half an ulp of the
+    # expected sum (the rounding of the stored result) is allowed on top, element by element
+    check_close(x.float().cpu().numpy(), x0.float().cpu().numpy().astype(np.float64) + want,
+                "f32" if dtype == torch.float32 else "bf16", "x + HPE", out_rounding=True)
     P.hdt_device_status()
 
 

@@ -308,3 +308,121 @@ def test_full_size_config_sampled(P, c):
         tot_dv = dv.float().sum(0)
         tot_do = do.float()[~pad].sum(0)
         assert torch.allclose(tot_dv, tot_do, atol=2.0 if cfg.dtype == "bf16" else 1e-2, rtol=2e-2)
+
+
+# ------------------------------------------------------------------------------------------
+# full-size configurations: every entry against the oracle
+# ------------------------------------------------------------------------------------------
+# (sequences, heads) the oracle computes: all of configurations 2, 3 and 6; two sequences x 4 heads of
+# configuration 4 and one sequence x 2 heads of configuration 5 (the dense n x n mask of a 32768-token
+# sequence is 1 GiB and the fp64 loops take tens of seconds); the sampled test above covers the
+# other heads and sequences of those two.
+FULL_COMPARE = {2: (None, None), 3: (None, None), 6: (None, None), 4: ([0, 1], 4), 5: ([0], 2)}
+
+
+@pytest.mark.parametrize("c", [2, 3, 6, 4, 5])
+def test_full_size_config_every_entry(P, c):
+    cfg = gen.CONFIGS[c]
+    b = gen.make_hierarchy(c)
+    T, H, d = b.total_tokens, cfg.heads, cfg.head_dim
+    t = gen.make_tensors(cfg.tensor_seed, T, H, d, cfg.dtype)
+    # the launch configuration the benchmark times: deferred build, caller workspaces
+    idx = P.hdt_build_index(*dev_struct(b), max_stages=4, deferred=True)
+    q, k, v, do = (dev_tensor(t[n], cfg.dtype) for n in ("q", "k", "v", "do"))
+    o, lse = P.hdt_attn_fwd(idx, q, k, v)
+    if cfg.backward:
+        dq, dk, dv = P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
+    P.hdt_device_status()
+    seqs, heads = FULL_COMPARE[c]
+    seqs = list(range(b.batch)) if seqs is None else seqs
+    hs = H if heads is None else heads
+    for s in seqs:
+        lo, hi = int(b.cu_seqlens[s]), int(b.cu_seqlens[s + 1])
+        sub = gen.pack([(b.level[lo:hi], b.parent[lo:hi])])
+        tq, tk, tv, tdo = (np.ascontiguousarray(t[n][lo:hi, :hs]) for n in ("q", "k", "v", "do"))
+        o_r, lse_r = oracle.forward(sub.level, sub.parent, sub.cu_seqlens, tq, tk, tv)
+        check_close(host(o[lo:hi, :hs]), o_r, cfg.dtype, f"O seq {s}")
+        check_close(host(lse[:hs, lo:hi]), lse_r, cfg.dtype, f"LSE seq {s}")
+        if cfg.backward:
+            dq_r, dk_r, dv_r = oracle.backward(sub.level, sub.parent, sub.cu_seqlens, tq, tk, tv, tdo)
+            check_close(host(dq[lo:hi, :hs]), dq_r, cfg.dtype, f"dQ seq {s}")
+            check_close(host(dk[lo:hi, :hs]), dk_r, cfg.dtype, f"dK seq {s}")
+            check_close(host(dv[lo:hi, :hs]), dv_r, cfg.dtype, f"dV seq {s}")
+
+
+# ------------------------------------------------------------------------------------------
+# the mask the kernels apply, read out bit by bit
+# ------------------------------------------------------------------------------------------
+def _mask_readout(P, b, dtype, directions, opts=()):
+    """Q = 0 makes every kept entry of a row equally likely and V = the leading columns of the identity
+    turns the row of O into the row of the mask divided by its degree: round(O * degree) must equal the
+    oracle's dense mask exactly, which checks every bit of the predicate the kernel evaluated."""
+    T = b.total_tokens
+    assert b.batch == 1 and T <= 64
+    H, d = 2, 64
+    q = np.zeros((T, H, d), np.float32)
+    k = gen.make_tensors(3, T, H, d, dtype)["k"]
+    v = np.zeros((T, H, d), np.float32)
+    for h in range(H):
+        v[np.arange(T), h, np.arange(T)] = 1.0
+    M = oracle.mask(b.level, b.parent, b.cu_seqlens, 0, directions=directions).astype(np.int64)
+    deg = M.sum(1)
+    for name, val in opts:
+        P.hdt_set_option(name, val)
+    try:
+        idx = P.hdt_build_index(*dev_struct(b), max_stages=12, directions=directions)
+        o, lse = P.hdt_attn_fwd(idx, dev_tensor(q, dtype), dev_tensor(k, dtype), dev_tensor(v, dtype))
+        P.hdt_device_status()
+    finally:
+        for name, _ in opts:
+            P.hdt_set_option(name, 0)
+    got = host(o)
+    real = b.level >= 0
+    for h in range(H):
+        read = np.rint(got[:, h, :T] * deg[:, None]).astype(np.int64)
+        assert np.array_equal(read[real], M[real]), (dtype, directions, opts, h)
+        assert np.all(got[:, h, T:] == 0)
+        # 1/deg is stored in bf16 with relative error 2^-9 at most: deg * O stays within 0.2 % of 0 or 1
+        assert np.abs(got[:, h, :T] * deg[:, None] - M)[real].max() < 4e-3
+        np.testing.assert_allclose(host(lse)[h][real], np.log(deg[real]), atol=1e-4)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_mask_readout_config1_and_directed(P, dtype):
+    b1 = gen.make_hierarchy(1)                                       # 57 tokens
+    rng = np.random.default_rng(8)
+    tree = gen.pack([gen.layout_tree(gen.random_tree(rng, 4, 5, p_leaf=0.4))[:2]])
+    small = [b1, gen.pack([gen.layout([[9, 3, 0], [12], [2, 2, 2, 2]])])]
+    if tree.total_tokens <= 64:
+        small.append(tree)
+    paths = ((), (("force_simt", 1),), (("no_persistent", 1),)) if dtype == "bf16" else ((),)
+    for b in small:
+        for directions in (7, 6, 4, 3, 5, 0):
+            for opts in paths:
+                _mask_readout(P, b, dtype, directions, opts)
+
+
+def test_backward_is_deterministic_and_guard_bands_untouched(P):
+    """Two backward calls on the same inputs give the same bits (self-contained blocks: no atomics; split
+    families: see the header on the order of the dQ additions), and nothing is written outside the
+    gradient tensors."""
+    for b in (gen.small_random_batch(56, n_seqs=3, max_len=300),
+              gen.pack([gen.layout([[300, 2], [1, 131, 0]]), gen.layout([[7] * 40])])):
+        T, H, d = b.total_tokens, 2, 64
+        t = gen.make_tensors(6, T, H, d, "bf16")
+        idx = P.hdt_build_index(*dev_struct(b))
+        q, k, v, do = (dev_tensor(t[n], "bf16") for n in ("q", "k", "v", "do"))
+        o, lse = P.hdt_attn_fwd(idx, q, k, v)
+        bigs = [torch.full((T + 2, H, d), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+        g1 = P.hdt_attn_bwd(idx, q, k, v, o, lse, do, dq=bigs[0][1:T + 1], dk=bigs[1][1:T + 1], dv=bigs[2][1:T + 1])
+        g2 = P.hdt_attn_bwd(idx, q, k, v, o, lse, do)
+        P.hdt_device_status()
+        split = idx.export(0)["n_fused"] < idx.export(0)["n_blocks"]
+        for name, x, y in zip(("dQ", "dK", "dV"), g1, g2):
+            if name == "dQ" and split:
+                # the dQ tiles of a split family are added in the order the CTAs reach them
+                assert float((x.float() - y.float()).abs().max()) <= 2e-2
+            else:
+                assert torch.equal(x, y), name
+        for big in bigs:
+            assert torch.isnan(big[0]).all() and torch.isnan(big[T + 1]).all()

@@ -1,17 +1,18 @@
 """Randomised GPU parity: seeded random batches (1-6 sequences, 60-1500 tokens, sentence and section
 counts drawn anew, PAD tails), 1-4 heads, head_dim 64 / 128, row blocks of 7 / 32 / 64 / 128 rows,
 waiting and deferred builds, default and custom softmax scale, bf16, forward and backward against
-the fp64 oracle.  A custom scale of 0.2 sharpens the softmax and lets gradients reach 10: there the
-spacing of bf16 outputs alone (2^-4) exceeds the absolute tolerance, and the bf16 rounding of P and
-dS (relative 2^-9 each) grows with them.  The maximum error of a tensor (the maximum over up to
-millions of entries here, not over sampled rows) is therefore held to 2.5e-2 times max(1, largest
-expected magnitude / 4), the mean error to 2e-3 as everywhere."""
+the fp64 oracle, every entry, at the stated tolerance: max 2e-2, mean 2e-3.  Where an expected
+value passes 4 the bf16 grid itself is coarser than 2e-2, so an element may exceed the maximum by
+half a bf16 ulp of its expected value (the rounding of the stored result), nothing more.  The custom
+scale is 0.1, between the defaults of the two head sizes (0.125 and 0.088): much sharper softmaxes
+(0.2, say) make dS reach 30 and the bf16 rounding of P and dS inside the kernels (2^-9 relative per
+term, part of the prescribed bf16 arithmetic) alone passes 2e-2 in the gradients."""
 import numpy as np
 import pytest
 
 import gen
 import oracle
-from gpu_util import dev_struct, dev_tensor, host
+from gpu_util import check_close, dev_struct, dev_tensor, host
 
 pytestmark = pytest.mark.gpu
 
@@ -35,7 +36,7 @@ def test_random_batches(P, seed):
         H, d = int(rng.integers(1, 5)), int(rng.choice([64, 128]))
         bm = int(rng.choice([128, 128, 64, 32, 7]))
         deferred = bool(rng.integers(2))
-        scale = float(rng.choice([0.0, 0.0, 0.2]))
+        scale = float(rng.choice([0.0, 0.0, 0.1]))
         what = dict(seed=seed, case=case, n_seqs=n_seqs, max_len=max_len, K=K, H=H, d=d, block_m=bm, deferred=deferred,
                     scale=scale, T=b.total_tokens)
         t = gen.make_tensors(int(rng.integers(1 << 30)), b.total_tokens, H, d, "bf16")
@@ -48,13 +49,4 @@ def test_random_batches(P, seed):
         o_r, lse_r = oracle.forward(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], scale=sc)
         dq_r, dk_r, dv_r = oracle.backward(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], t["do"], scale=sc)
         for name, got, want in (("O", o, o_r), ("LSE", lse, lse_r), ("dQ", dq, dq_r), ("dK", dk, dk_r), ("dV", dv, dv_r)):
-            g = host(got)
-            fin = np.isfinite(want)
-            assert np.array_equal(np.isfinite(g), fin), (name, what)
-            assert np.array_equal(g[~fin], want[~fin]), (name, what)
-            err = np.abs(g[fin] - want[fin])
-            if err.size == 0:
-                continue
-            tol = 2.5e-2 * max(1.0, float(np.abs(want[fin]).max()) / 4.0)
-            assert err.max() <= tol, (name, float(err.max()), tol, what)
-            assert err.mean() <= 2e-3, (name, float(err.mean()), what)
+            check_close(host(got), want, "bf16", f"{name} {what}", out_rounding=True)
