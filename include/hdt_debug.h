@@ -84,6 +84,29 @@ int hdt_debug_bwd_timeline(int64_t *out2048);
 /* The same for the last instrumented launch of the looping forward, up to 1024 CTAs. */
 int hdt_debug_fwd_timeline(int64_t *out4096);
 
+/* With option "bwd_walk" = 86: the SM clock at fixed points of tiles 20 and 21 of CTA 0 of the last launch of the
+ * warp-specialised one-walk backward (families longer than a row block, head_dim 64), out128[16 role + 8 (tile - 20) + mark]; roles 0 / 1 the compute groups (marks: loop top, S^T / dP^T
+ * there, other waits passed, arrived), 2 the drain group (loop top, dQ there, reduce requested), 3 the load warp
+ * (before / after the wait for the ring stage), 4 the MMA warp (loop top, group a arrived, other waits passed,
+ * step a issued, group b arrived, dQ accumulator free, step b issued). */
+int hdt_debug_bwd_w_marks(int64_t *out128);
+/* The same run: out512[t] = (SM clock << 8 | unit number mod 256) at the MMA warp's loop top of tile t of CTA 0. */
+int hdt_debug_bwd_w_tiles(int64_t *out512);
+
+/* Timing probe of the tensor pipe (allocates 16 bytes of device memory for its result and waits for the
+ * device): one thread of one CTA issues `reps` groups of `per_group` MMAs (M = 128, N = n <= 128 (the probe holds two 64-column operand groups), K = 16 each; A from
+ * shared memory or, a_tmem = 1, from TMEM; B K-major or, b_mn = 1, MN-major) and commits once.  out2[0] = SM
+ * clock cycles from the first issue until the last MMA had completed, out2[1] = cycles of the issue loop.
+ * mode bit 0: A from TMEM; bit 1: consecutive MMAs alternate between two accumulators (none depends on the one before); bit 2: two warps issue
+ * the same sequence side by side (n <= 64), out2 holds the first warp's figures. */
+int hdt_debug_mma_rate(int32_t n, int32_t reps, int32_t per_group, int32_t mode, int32_t b_mn, int64_t *out2);
+
+/* Timing probe of TMEM loads (allocates 256 bytes of device memory for its result and waits for the device):
+ * `warps` (1..28) warps of one CTA each run `reps` rounds of `per_round` (1..4) loads of 32 lanes x 16 columns
+ * followed by one wait; with mma != 0 another warp keeps the tensor pipe busy meanwhile.  out32[w] = SM clock
+ * cycles of warp w's loop. */
+int hdt_debug_tmem_ld(int32_t warps, int32_t reps, int32_t per_round, int32_t mma, int64_t *out32);
+
 #ifdef __cplusplus
 }
 #endif

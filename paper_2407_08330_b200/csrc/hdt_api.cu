@@ -114,7 +114,7 @@ struct AttnLayout {
     size_t total;
 };
 
-static int g_bwd_two_walk = 0;          // option "bwd_two_walk"
+int g_bwd_walk = 0;                     // option "bwd_walk"
 
 // Blocks of stage 0 that are neither self-contained nor EMPTY: families longer than a row block.
 static int n_split_blocks(const hdt_index *ix) { return ix->desc[0].nb - ix->desc[0].n_fused - ix->desc[0].n_empty; }
@@ -174,7 +174,7 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "no_fold") == 0) { g_no_fold = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_pdl") == 0) { g_no_pdl = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_fwd_mc") == 0) { g_no_fwd_mc = value; return HDT_OK; }
-    if (name && std::strcmp(name, "bwd_two_walk") == 0) { g_bwd_two_walk = value; return HDT_OK; }
+    if (name && std::strcmp(name, "bwd_walk") == 0) { g_bwd_walk = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 
@@ -435,9 +435,9 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
                              !g_no_fused_delta && ix->directions == 7 && ix->desc[0].n_fused == ix->desc[0].nb &&
                              ix->desc[0].nb > 0 && (ix->n_stages == 1 || (overlap && tc_upper));
     // Families longer than a row block (head_dim 64): one walk over their tile pairs, dQ tiles summed
-    // in an fp32 buffer that starts at zero (option "bwd_two_walk" = 1: two walks, no buffer).
+    // in an fp32 buffer that starts at zero (option "bwd_walk" = 1: two walks, no buffer).
     float *dq_acc = nullptr;
-    if (L.has_dq_acc && !g_force_simt && !g_bwd_two_walk &&
+    if (L.has_dq_acc && !g_force_simt && g_bwd_walk != 1 &&
         (g_no_persistent == 0 || g_no_persistent == 4 || g_no_persistent == 6)) {
         dq_acc = (float *)(ws + L.dq_acc);
         ProfScope ps(PROF_BWD_STAGE0, st);
@@ -475,6 +475,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         a.dirs = ix->directions;
         a.tok_rows = a.tok;
         if (s == 0) a.dq_acc = dq_acc;
+        a.n_empty = ix->desc[s].n_empty;
         return a;
     };
     if (overlap) {   // delta is ready: the upper stages' own gradients are computed beside stage 0

@@ -1282,7 +1282,13 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
             BwdStageArgs c = a;
             c.rest_only = mode;
             const int grid_p = (int)(units < n_sm ? units : n_sm);
-            if (mode && onewalk) {
+            if (g_bwd_walk == 86 || g_bwd_walk == 85) c.phases = g_bwd_walk;                // (clock marks: hdt_debug_bwd_w_marks)
+            if (mode && onewalk && (g_bwd_walk == 0 || g_bwd_walk == 86 || g_bwd_walk == 85)) {
+                // the warp-specialised one-walk kernel (hdt_attn_tc_bwd_w.cu), then the sums become dQ rows
+                rc = launch_bwd_tc_onewalk64(c, tq, tk, tv, tdo, outs, tacc, a.n_empty, st);
+                if (rc) return rc;
+                k_dq_finish<<<dim3(a.nb - a.n_fused, a.H), 256, 0, st>>>(c);
+            } else if (mode && onewalk) {
                 if (dirs) k_bwd_tc_p<2, true><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);
                 else k_bwd_tc_p<2><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);
                 count_launch();

@@ -1,0 +1,646 @@
+// Warp-specialised one-walk backward for stage 0 in bf16 at D = 64: the row blocks that are neither
+// self-contained nor EMPTY, i.e. the pieces of families longer than a row block.
+//
+// A unit is (row block, head).  The block is taken as KEYS only (K, V of its 128 token rows stay in
+// shared memory) and walks its key span [ka, kb) — which, the family ranges being symmetric, holds
+// every query that attends one of its keys — in query tiles of 128 rows, each in two steps of 64
+// queries.  With the keys in the TMEM lanes (the transposed pass of hdt_attn_tc_bwd_t.cu):
+//   MMA      S^T = K Q^T, dP^T = V dO^T for the step's 64 queries            -> TMEM (lane = key)
+//   compute  P^T = exp2(S^T c - LSE[query]) inside the key's range, dS^T = P^T o (dP^T - delta[query]);
+//            P^T (bf16) stays in TMEM over the S^T columns it came from, dS^T -> shared memory
+//   MMA      dV += P^T dO (A operand from TMEM), dK += dS^T Q: accumulated in TMEM over the whole walk;
+//            after both steps dQ_tile = dS K (M = the tile's 128 queries, A = dS^T read MN-major), a
+//            fresh accumulator per tile
+//   drain    the dQ tile as fp32, in two halves of 32 columns, through a swizzled staging tile and a TMA
+//            reduce-add copy each into the buffer a.dq_acc [T, H, 64] (k_dq_finish scales and converts
+//            the sums afterwards); at the end of the unit dK, dV -> bf16 rows through TMA stores
+// Every tile pair is visited once (the two-walk kernels compute S, dP, P, dS of each pair twice).
+//
+// One CTA of 736 threads per SM.  Warps 0-7 compute step a (queries 0..63 of each tile: warp = TMEM lane
+// quarter x half of the step's queries), warps 8-15 step b, warps 16-19 drain, warp 20 requests the
+// tiles (TMA) and fetches the queries' LSE and delta, warp 21 issues the MMAs, warp 22 requests the
+// reduce-add copies of the staged dQ tiles.  The roles meet only at
+// mbarriers, so the tensor pipe, the exponentials of the two compute groups and the drains overlap;
+// S^T / dP^T are double buffered by step, dS^T and the dQ accumulator by tile, Q / dO in a ring of
+// three tiles; K / V have one buffer (the next unit's are requested into L2 ahead of time).
+// TMEM columns: S^T a 0..63 (P^T a over 0..15 and 32..47: each warp writes inside the columns it alone
+// reads), dP^T a 64..127, step b the same from 128; dK 256..319, dV 320..383, dQ 384..447 and 448..511.
+// Measured on this part (one thread issuing back to back): an MMA of M = 128, K = 16 takes about 75
+// cycles at N = 64 with both operands in shared memory, 47 with A in TMEM, 106 / 70 at N = 128 — the
+// operand reads, not the arithmetic, set the pace at these shapes — which makes a tile pair cost the
+// tensor pipe about 2800 cycles here (16 x 75 for S^T / dP^T, 8 x 47 for dV, 16 x 75 for dK and dQ).
+// What a compute group waits for between two of its steps is dV of the step (its P^T lies over the
+// S^T columns) and the next S^T / dP^T; dK and dQ, which read dS^T from shared memory, are issued
+// behind them.  Clock stamps of an earlier form with four warps per compute group showed a step's
+// arithmetic (64 entries per thread) taking 3500 cycles, an issue rate of one instruction in eight
+// cycles per warp: the groups have eight warps each since.
+#include <cuda_bf16.h>
+
+#include "hdt_internal.cuh"
+#include "hdt_sm100.cuh"
+#include "hdt_tmap.cuh"
+
+namespace hdt {
+using namespace sm100;
+
+namespace {
+constexpr int SUB = 16384;
+constexpr long long WAIT_CYCLES = 400000000LL;
+constexpr int KID = 7;     // kernel id in the device status word
+__device__ __forceinline__ uint32_t swz(int r, int c) { return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4)); }
+
+// Barrier `id` over `n` threads (a warp group) that also tells every thread whether ALL of them
+// passed `pred`: the group leaves its loop together when a bounded wait of one thread ran out.
+__device__ __forceinline__ bool group_all(bool pred, int id, int n) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, %2, %3, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)pred), "r"(id), "r"(n)
+        : "memory");
+    return r != 0;
+}
+
+// Timeline of two tiles of CTA 0 (option "bwd_walk" = 86): absolute SM clock at fixed points of each role.
+__device__ long long g_bwd_w_marks[128];
+__device__ long long g_bwd_w_tiles[512];      // (instrumented run) CTA 0: SM clock at the MMA warp's loop top of every tile, unit number in the low 8 bits
+#define W_MARK(role, tt, id)                                                                    \
+    do {                                                                                        \
+        if (marks && (tt) >= 7 && (tt) < 9) {                                                 \
+            const long long now_ = clock64();                                                   \
+            if (lane == 0) s_marks[(role) * 16 + ((tt) - 7) * 8 + (id)] = now_;                \
+        }                                                                                       \
+    } while (0)
+
+struct WUnit { int valid, r0, r1, ka, kb, h, nt; };
+// Position of a role in this CTA's sequence of query tiles: unit slot k, unit U (its uc-th non-empty
+// unit), tile j of it, t-th tile overall, which lies in stage qs of the Q / dO ring on that stage's
+// use of parity qph; N: the record of the unit after U, requested a unit ahead.
+struct Walk { int k, j, t, uc, valid, qs, qph; WUnit U, N; };
+}  // namespace
+
+template <bool DIRS>
+__global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUtensorMap tm_q,
+                                                     const __grid_constant__ CUtensorMap tm_k,
+                                                     const __grid_constant__ CUtensorMap tm_v,
+                                                     const __grid_constant__ CUtensorMap tm_do,
+                                                     const __grid_constant__ StoreMaps sm_out,
+                                                     const __grid_constant__ CUtensorMap tm_acc, const BwdStageArgs a) {
+    constexpr int D = 64;
+    constexpr uint32_t TM_DK = 256, TM_DV = 320, TM_DQ = 384, TM_COLS = 512;
+    constexpr int W_DRAIN = 16, W_LOAD = 20, W_MMA = 21, W_RED = 22;      // first warp of each role
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    uint8_t *sKV = smem_raw;                 // [2 units] x {K, V}
+    uint8_t *sQD = sKV + 4 * SUB;            // [3 tiles] x {Q, dO}
+    uint8_t *sDS = sQD + 6 * SUB;            // [2 tiles] x {dS^T of step a, of step b}: row = key, 64 queries per row; once dQ of
+                                             // the tile has read it, the same 32 KB stage the dQ tile as fp32 (two swizzled [128 x 32] halves)
+    float2 *sStat = (float2 *)(sDS + 4 * SUB);   // [2 tiles][128]: LSE * log2(e) and delta of the tile's queries
+    uint64_t *bars = (uint64_t *)(sStat + 2 * 128);
+    uint64_t *qdo_full = bars, *qdo_empty = bars + 3, *sdp_full = bars + 6, *pds_ready = bars + 8;
+    uint64_t *dq_full = bars + 10, *dq_free = bars + 12, *kv_full = bars + 14, *kv_empty = bars + 16;
+    uint64_t *acc_full = bars + 18, *acc_free = bars + 19, *stat_full = bars + 20, *stg_free = bars + 22, *stg_full = bars + 24, *kv_reuse = bars + 26;
+    uint32_t *slot = (uint32_t *)(bars + 28);
+    volatile int *abort_flag = (volatile int *)(slot + 1);
+    long long *s_marks = (long long *)(bars + 30);      // [5 roles][2 tiles][8 marks] of the instrumented run (only then allocated)
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int H = a.H, G = gridDim.x;
+    const float LOG2E = 1.4426950408889634f;
+    const bool marks = (a.phases == 86 || a.phases == 85) && blockIdx.x == 0 && (warp == 0 || warp == 8 || warp == W_DRAIN || warp >= W_LOAD);
+    if ((a.phases == 86 || a.phases == 85) && tid < 80) s_marks[tid] = 0;
+    // EMPTY blocks cost nothing in the queue's order, so they are the tail of queue_split and are left
+    // out here (k_bwd_zero_empty writes their rows)
+    const int n_units = (a.nb - a.n_fused - a.n_empty) * H;
+
+    if ((smem_u32(smem_raw) & 1023u) != 0u) {      // the swizzled tiles need 1024-byte alignment
+        if (tid == 0) atomicCAS(a.status, 0, HDT_ERR_CUDA);
+        return;
+    }
+    if (tid == 0) {
+        for (int i = 0; i < 3; ++i) {
+            mbar_init(&qdo_full[i], 1);
+            mbar_init(&qdo_empty[i], 1);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&sdp_full[i], 1);
+            mbar_init(&pds_ready[i], 256);
+            mbar_init(&dq_full[i], 1);
+            mbar_init(&dq_free[i], 128);
+        }
+        for (int i = 0; i < 2; ++i) {
+            mbar_init(&kv_full[i], 1);
+            mbar_init(&kv_empty[i], 1);
+            mbar_init(&stat_full[i], 1);
+            mbar_init(&stg_free[i], 1);
+            mbar_init(&stg_full[i], 128);
+            mbar_init(&kv_reuse[i], 1);
+        }
+        mbar_init(acc_full, 1);
+        mbar_init(acc_free, 128);
+        *abort_flag = (*a.status != 0);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(slot, TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *slot;
+    const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+    const bool dead = (*abort_flag != 0);
+    bool ok = true;
+    int fail_site = 0;
+    // (the warp-wide instructions of every role need all lanes to take the same way: after its waits a
+    // warp agrees on whether all of them ended well)
+#define HDT_AGREE() (ok = __all_sync(0xffffffffu, ok))
+#define HDT_WAIT(bar, parity, site)                                                   \
+    do {                                                                              \
+        if (ok && !mbar_wait((bar), (uint32_t)(parity), abort_flag, WAIT_CYCLES)) {   \
+            ok = false;                                                               \
+            fail_site = (site);                                                       \
+        }                                                                             \
+    } while (0)
+
+    // ---- this CTA's sequence of units and tiles (every role walks it on its own) -------------------
+    auto get_unit = [&](int k) {
+        WUnit u{0, 0, 0, 0, 0, 0, 0};
+        const int i = (int)blockIdx.x + k * G;
+        if (i < n_units) {
+            const int bi = i / H;
+            const int *rec = a.blocks + 5 * (size_t)a.queue_split[a.n_fused + bi];
+            u.valid = 1; u.r0 = rec[0]; u.r1 = rec[1]; u.ka = rec[2]; u.kb = rec[3]; u.h = i - bi * H;
+            u.nt = (u.kb - u.ka + 127) >> 7;      // (>= 1: EMPTY blocks are not among these units)
+        }
+        return u;
+    };
+    // The record of the unit after the current one is requested a whole unit ahead (w.N): its loads
+    // are in flight while the current unit is walked and no role waits for them at a unit boundary.
+    auto step = [&](Walk &w) {      // to the next tile
+        ++w.t;
+        if (++w.qs == 3) { w.qs = 0; w.qph ^= 1; }
+        if (w.uc >= 0 && w.j + 1 < w.U.nt) { ++w.j; return; }
+        while (true) {
+            const WUnit u = w.N;
+            w.N = get_unit(w.k++);
+            if (!u.valid) { w.valid = 0; return; }
+            if (u.nt > 0) { w.U = u; w.j = 0; ++w.uc; w.valid = 1; return; }
+        }
+    };
+    auto begin = [&]() {
+        Walk w;
+        w.k = 0; w.j = 0; w.t = -1; w.uc = -1; w.valid = 0; w.qs = 2; w.qph = 1; w.U = WUnit{0, 0, 0, 0, 0, 0, 0};
+        w.N = get_unit(w.k++);
+        step(w);
+        return w;
+    };
+
+    if (!dead && n_units > 0) {
+        if (warp == W_LOAD) {
+            // ================= load warp: K / V per unit, Q / dO and the queries' statistics per tile =================
+            for (Walk w = begin(); w.valid && ok; step(w)) {
+                const WUnit &U = w.U;
+                const int q0 = U.ka + 128 * w.j, qs = w.qs;
+                // before the wait for the ring stage: the tile starts its way into L2 and the queries'
+                // statistics into registers
+                if (lane == 0) {
+                    tma_prefetch_3d(&tm_q, 0, U.h, q0);
+                    tma_prefetch_3d(&tm_do, 0, U.h, q0);
+                }
+                float2 st4[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = q0 + lane + 32 * i;
+                    st4[i] = make_float2(0.f, 0.f);
+                    if (row < U.kb) st4[i] = make_float2(a.lse[(size_t)U.h * a.T + row] * LOG2E, a.delta[(size_t)U.h * a.T + row]);
+                }
+                W_MARK(3, w.t, 0);
+                if (w.j == 0) {      // the unit's K, V into the buffer the unit before the last one has left
+                    if (w.uc >= 2) {      // every MMA of unit uc - 2 has read the buffer, and its dK, dV rows, staged there afterwards, have left
+                        HDT_WAIT(&kv_empty[w.uc & 1], ((w.uc >> 1) + 1) & 1, 1);
+                        HDT_WAIT(&kv_reuse[w.uc & 1], ((w.uc >> 1) + 1) & 1, 19);
+                    }
+                    if (!HDT_AGREE()) break;
+                    if (lane == 0) {
+                        uint8_t *kv = sKV + (w.uc & 1) * 2 * SUB;
+                        mbar_expect_tx(&kv_full[w.uc & 1], 2u * SUB);
+                        tma_load_3d(kv, &tm_k, 0, U.h, U.r0, &kv_full[w.uc & 1]);
+                        tma_load_3d(kv + SUB, &tm_v, 0, U.h, U.r0, &kv_full[w.uc & 1]);
+                    }
+                }
+                if (w.t >= 3) HDT_WAIT(&qdo_empty[qs], w.qph ^ 1, 2);
+                if (!HDT_AGREE()) break;
+                W_MARK(3, w.t, 1);
+                if (lane == 0) {
+                    uint8_t *qd = sQD + qs * 2 * SUB;
+                    mbar_expect_tx(&qdo_full[qs], 2u * SUB);
+                    tma_load_3d(qd, &tm_q, 0, U.h, q0, &qdo_full[qs]);
+                    tma_load_3d(qd + SUB, &tm_do, 0, U.h, q0, &qdo_full[qs]);
+                }
+                // the statistics have two buffers only: tile t - 2 must be through (the tile loads above did not wait for that)
+                if (w.t >= 2) {
+                    const int q2 = qs == 0 ? 1 : qs == 1 ? 2 : 0;          // ring stage of tile t - 2
+                    HDT_WAIT(&qdo_empty[q2], qs == 2 ? w.qph : (w.qph ^ 1), 17);
+                }
+                if (!HDT_AGREE()) break;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) sStat[(w.t & 1) * 128 + lane + 32 * i] = st4[i];
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&stat_full[w.t & 1]);
+                if (w.j == min(1, U.nt - 1) && w.N.valid && lane == 0) {      // the next unit's K, V on their way into L2
+                    tma_prefetch_3d(&tm_k, 0, w.N.h, w.N.r0);
+                    tma_prefetch_3d(&tm_v, 0, w.N.h, w.N.r0);
+                }
+            }
+        } else if (warp == W_RED) {
+            // ================= reduce warp: the TMA reduce-add copies of every staged dQ tile =================
+            for (Walk w = begin(); w.valid && ok; step(w)) {
+                const int t = w.t, db = t & 1;
+                HDT_WAIT(&stg_full[db], (t >> 1) & 1, 18);
+                if (!HDT_AGREE()) break;
+                if (lane == 0) {
+                    const uint8_t *stg = sDS + db * 2 * SUB;
+                    const int q0 = w.U.ka + 128 * w.j;      // the tile's first query row
+                    tma_reduce_add_3d(&tm_acc, 0, w.U.h, q0, stg);
+                    tma_reduce_add_3d(&tm_acc, 32, w.U.h, q0, stg + SUB);
+                    bulk_commit();
+                    bulk_wait_read();                 // the copies have read the tile:
+                    mbar_arrive(&stg_free[db]);       // the compute groups may write dS^T of tile t + 2 there
+                }
+                __syncwarp();
+            }
+        } else if (warp == W_MMA) {
+            // ================= MMA warp =================
+            const uint32_t id_sdp = idesc_bf16(64, false, false);   // A = K / V (K-major), B = Q / dO rows of the step (K-major)
+            const uint32_t id_kv = idesc_bf16(D, false, true);      // A = P^T (TMEM) / dS^T (K-major), B = dO / Q (MN-major)
+            const uint32_t id_q = idesc_bf16(D, true, true);        // A = dS (MN-major: stored as dS^T), B = K (MN-major)
+            // base descriptors (two 32-bit words each) of every operand form; an MMA adds (byte offset >> 4)
+            // to the low word.  K-major: sbo 1024; MN-major: lbo = SUB between 64-element groups, sbo 1024.
+            const uint64_t d_kv_k = smem_desc(smem_u32(sKV), 0, 1024), d_kv_mn = smem_desc(smem_u32(sKV), SUB, 1024);
+            const uint64_t d_qd_k = smem_desc(smem_u32(sQD), 0, 1024), d_qd_mn = smem_desc(smem_u32(sQD), SUB, 1024);
+            const uint64_t d_ds_k = smem_desc(smem_u32(sDS), 0, 1024), d_ds_mn = smem_desc(smem_u32(sDS), SUB, 1024);
+            const uint32_t kvk_lo = (uint32_t)d_kv_k, kvk_hi = (uint32_t)(d_kv_k >> 32), kvm_lo = (uint32_t)d_kv_mn, kvm_hi = (uint32_t)(d_kv_mn >> 32);
+            const uint32_t qdk_lo = (uint32_t)d_qd_k, qdk_hi = (uint32_t)(d_qd_k >> 32), qdm_lo = (uint32_t)d_qd_mn, qdm_hi = (uint32_t)(d_qd_mn >> 32);
+            const uint32_t dsk_lo = (uint32_t)d_ds_k, dsk_hi = (uint32_t)(d_ds_k >> 32), dsm_lo = (uint32_t)d_ds_mn, dsm_hi = (uint32_t)(d_ds_mn >> 32);
+            constexpr uint32_t S16 = SUB >> 4;      // one sub-tile in descriptor address units
+            auto issue_sdp = [&](int x, int qs, int kvb) {
+                const uint32_t q_lo = qdk_lo + qs * 2 * S16 + x * (8192 >> 4), k_lo = kvk_lo + kvb * 2 * S16;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ss_w(tmem + 128u * x, k_lo + 2 * kk, kvk_hi, q_lo + 2 * kk, qdk_hi, id_sdp, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ss_w(tmem + 128u * x + 64u, k_lo + S16 + 2 * kk, kvk_hi, q_lo + S16 + 2 * kk, qdk_hi, id_sdp, kk > 0);
+                mma_commit(&sdp_full[x]);
+            };
+            auto issue_dv = [&](int x, int qs, uint32_t acc) {      // P^T: queries 0..31 of the step in columns 0..15, 32..63 in 32..47
+                const uint32_t do_lo = qdm_lo + qs * 2 * S16 + x * (8192 >> 4) + S16;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts_w(tmem + TM_DV, tmem + 128u * x + (kk < 2 ? 8u * kk : 32u + 8u * (kk - 2)), do_lo + 128 * kk, qdm_hi, id_kv, acc | (kk > 0));
+            };
+            auto issue_dk = [&](int x, int qs, int dsb, uint32_t acc) {
+                const uint32_t q_lo = qdm_lo + qs * 2 * S16 + x * (8192 >> 4);
+                const uint32_t d_lo = dsk_lo + dsb * 2 * S16 + x * S16;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ss_w(tmem + TM_DK, d_lo + 2 * kk, dsk_hi, q_lo + 128 * kk, qdm_hi, id_kv, acc | (kk > 0));
+            };
+            auto issue_dq = [&](int dsb, int kvb) {
+                const uint32_t d_lo = dsm_lo + dsb * 2 * S16, k_lo = kvm_lo + kvb * 2 * S16;
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    mma_ss_w(tmem + TM_DQ + 64u * dsb, d_lo + 128 * kk, dsm_hi, k_lo + 128 * kk, kvm_hi, id_q, kk > 0);
+            };
+            Walk w = begin();
+            if (w.valid) {      // S^T, dP^T of both steps of the first tile
+                HDT_WAIT(&kv_full[0], 0, 3);
+                HDT_WAIT(&qdo_full[0], 0, 4);
+                if (HDT_AGREE() && elect_one()) {
+                    tc_fence_after();
+                    issue_sdp(0, 0, 0);
+                    issue_sdp(1, 0, 0);
+                }
+                __syncwarp();
+            }
+            while (w.valid && ok) {
+                // the next tile, without walking there: same unit or the next one (units here are never EMPTY)
+                const int t = w.t, db = t & 1;
+                const bool first = w.j == 0, last = w.j == w.U.nt - 1;
+                struct { int valid, qs, qph, uc; } n;
+                n.valid = !last || w.N.valid;
+                n.qs = w.qs == 2 ? 0 : w.qs + 1;
+                n.qph = w.qs == 2 ? (w.qph ^ 1) : w.qph;
+                n.uc = w.uc + (last ? 1 : 0);
+                const int kvb = w.uc & 1;
+                const uint32_t acc = first ? 0u : 1u;
+                // ---- step a: dV; S^T, dP^T of the next tile's step a; dK ----
+                W_MARK(4, t, 0);
+                if ((a.phases == 86 || a.phases == 85) && blockIdx.x == 0 && lane == 0 && t < 512) g_bwd_w_tiles[t] = (clock64() << 8) | (long long)(w.uc & 255);
+                HDT_WAIT(&pds_ready[0], t & 1, 5);
+                W_MARK(4, t, 1);
+                if (first && w.uc >= 1) HDT_WAIT(acc_free, (w.uc - 1) & 1, 6);      // the previous unit's dK, dV have been read
+                if (n.valid) {
+                    HDT_WAIT(&qdo_full[n.qs], n.qph, 7);
+                    if (last) HDT_WAIT(&kv_full[n.uc & 1], (n.uc >> 1) & 1, 8);      // the next tile opens a unit (the other K / V buffer)
+                }
+                if (!HDT_AGREE()) break;
+                W_MARK(4, t, 2);
+                if (elect_one()) {
+                    tc_fence_after();
+                    issue_dv(0, w.qs, acc);
+                    if (n.valid) issue_sdp(0, n.qs, n.uc & 1);
+                    issue_dk(0, w.qs, db, acc);
+                }
+                __syncwarp();
+                W_MARK(4, t, 3);
+                // ---- step b: dV; S^T, dP^T of the next tile's step b; dK; the tile's dQ ----
+                HDT_WAIT(&pds_ready[1], t & 1, 9);
+                W_MARK(4, t, 4);
+                if (t >= 2) HDT_WAIT(&dq_free[db], ((t >> 1) + 1) & 1, 10);
+                if (!HDT_AGREE()) break;
+                W_MARK(4, t, 5);
+                if (elect_one()) {
+                    tc_fence_after();
+                    issue_dv(1, w.qs, 1u);
+                    if (n.valid) issue_sdp(1, n.qs, n.uc & 1);
+                    issue_dk(1, w.qs, db, 1u);
+                    mma_commit(&qdo_empty[w.qs]);        // every MMA that reads this tile's Q / dO has been issued
+                    if (last) mma_commit(acc_full);
+                    issue_dq(db, kvb);
+                    mma_commit(&dq_full[db]);
+                    if (last) mma_commit(&kv_empty[kvb]);
+                }
+                __syncwarp();
+                W_MARK(4, t, 6);
+                step(w);
+            }
+        } else if (warp < W_DRAIN) {
+            // ================= compute groups: x = 0 (warps 0-7) step a, x = 1 (warps 8-15) step b;
+            // a warp: TMEM lane quarter warp % 4, queries 32 qh .. 32 qh + 31 of the step =================
+            const int x = warp >> 3, qh = (warp >> 2) & 1, kl = (warp & 3) * 32 + lane;
+            const uint32_t tm_s = tmem + 128u * x + 32u * qh + lane_base, tm_dp = tm_s + 64u;
+            int lo = 0, hi = 0, row = 0, lo_n = 0, hi_n = 0, r0_n = -1;      // *_n: the range of this lane's key row in the block that starts at r0_n
+            bool inb = false;
+            auto fetch_range = [&](const WUnit &u) {
+                const int r = u.r0 + kl;
+                r0_n = u.r0; lo_n = 0; hi_n = 0;
+                if (r < u.r1) { lo_n = a.rng[2 * r]; hi_n = a.rng[2 * r + 1]; }
+            };
+            Walk w = begin();
+            if (w.valid) fetch_range(w.U);
+            for (; w.valid && ok; step(w)) {
+                const WUnit &U = w.U;
+                if (w.j == 0) {
+                    if (r0_n != U.r0) fetch_range(U);      // (only when a unit was skipped in between)
+                    row = U.r0 + kl;
+                    inb = row < U.r1;
+                    lo = lo_n; hi = hi_n;
+                }
+                // the next unit's range a unit ahead (its record, requested at this unit's start, has arrived by the second tile)
+                if (w.j == min(1, U.nt - 1) && w.N.valid) fetch_range(w.N);
+                const int t = w.t, db = t & 1;
+                const int q0 = U.ka + 128 * w.j, nq = min(128, U.kb - q0);
+                // this key row over the tile's queries: the queries that attend it are its own family range
+                const int jl = max(lo - q0, 0), jh = min(hi - q0, nq);
+                const bool has = inb && jh > jl;
+                const int c_self = row - q0, c_head = (lo < row) ? lo - q0 : -0x40000000;
+                const bool keep_head = (a.dirs & 4) != 0, keep_rest = (a.dirs & ((lo >= row) ? 1 : 2)) != 0;
+                uint8_t *ds = sDS + db * 2 * SUB + x * SUB;
+                const float2 *stat = sStat + db * 128 + 64 * x + 32 * qh;
+                // keep masks of the two 16-query pieces, and what the warp as a whole needs of them
+                uint32_t km[2];
+                bool any[2], all[2];
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    km[i] = has ? keep_mask<DIRS>(64 * x + 32 * qh + 16 * i, 16, jl, jh, c_self, c_head, keep_head, keep_rest) : 0u;
+                    any[i] = __any_sync(0xffffffffu, km[i] != 0u);
+                    all[i] = __all_sync(0xffffffffu, km[i] == 0xffffu);
+                }
+                W_MARK(x, t, 0);
+                HDT_WAIT(&sdp_full[x], t & 1, 11);
+                W_MARK(x, t, 1);
+                HDT_WAIT(&stat_full[db], (t >> 1) & 1, 12);                      // the queries' statistics are there
+                if (t >= 2) HDT_WAIT(&stg_free[db], ((t >> 1) + 1) & 1, 13);    // dQ of tile t - 2 has left this buffer (read as dS^T, then staged in it)
+                if (!HDT_AGREE()) break;
+                tc_fence_after();
+                W_MARK(x, t, 2);
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    uint32_t s_[16], d_[16], pp[8], pd[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) { pp[j] = 0u; pd[j] = 0u; }
+                    if (any[i]) {
+                        tmem_ld16(tm_s + 16u * i, s_);
+                        tmem_ld16(tm_dp + 16u * i, d_);
+                        tmem_wait_ld();
+                    }
+                    if (all[i]) {
+                        // every key of the warp keeps all 16 queries of the piece: no predicates
+#pragma unroll
+                        for (int j = 0; j < 16; j += 2) {
+                            const float4 st = *reinterpret_cast<const float4 *>(&stat[16 * i + j]);
+                            const float p0 = exp2f(fmaf(__uint_as_float(s_[j]), a.scale_log2, -st.x));
+                            const float p1 = exp2f(fmaf(__uint_as_float(s_[j + 1]), a.scale_log2, -st.z));
+                            pp[j >> 1] = pack_bf16(p0, p1);
+                            pd[j >> 1] = pack_bf16(p0 * (__uint_as_float(d_[j]) - st.y), p1 * (__uint_as_float(d_[j + 1]) - st.w));
+                        }
+                    } else if (any[i] && km[i] != 0u) {
+#pragma unroll
+                        for (int j = 0; j < 16; j += 2) {
+                            const float4 st = *reinterpret_cast<const float4 *>(&stat[16 * i + j]);
+                            float p0 = 0.f, p1 = 0.f, e0 = 0.f, e1 = 0.f;
+                            if (km[i] & (1u << j)) {
+                                p0 = exp2f(fmaf(__uint_as_float(s_[j]), a.scale_log2, -st.x));
+                                e0 = p0 * (__uint_as_float(d_[j]) - st.y);
+                            }
+                            if (km[i] & (2u << j)) {
+                                p1 = exp2f(fmaf(__uint_as_float(s_[j + 1]), a.scale_log2, -st.z));
+                                e1 = p1 * (__uint_as_float(d_[j + 1]) - st.w);
+                            }
+                            pp[j >> 1] = pack_bf16(p0, p1);
+                            pd[j >> 1] = pack_bf16(e0, e1);
+                        }
+                    }
+                    // P^T: the piece's 16 queries are 8 packed columns, inside the S^T columns this warp has read
+                    tmem_st8(tm_s + 8u * i, pp);
+                    *reinterpret_cast<uint4 *>(ds + swz(kl, 4 * qh + 2 * i)) = make_uint4(pd[0], pd[1], pd[2], pd[3]);
+                    *reinterpret_cast<uint4 *>(ds + swz(kl, 4 * qh + 2 * i + 1)) = make_uint4(pd[4], pd[5], pd[6], pd[7]);
+                }
+                tmem_wait_st();
+                fence_proxy_async_smem();
+                tc_fence_before();
+                mbar_arrive(&pds_ready[x]);
+                W_MARK(x, t, 3);
+            }
+        } else if (warp < W_LOAD) {
+            // ================= drain group: the dQ tile of every tile pair, added to the fp32 buffer =================
+            const int rl = tid & 127;
+            bool go = true;
+            for (Walk w = begin(); w.valid && go; step(w)) {
+                const WUnit &U = w.U;
+                const int t = w.t, db = t & 1;
+                W_MARK(2, t, 0);
+                HDT_WAIT(&dq_full[db], (t >> 1) & 1, 14);
+                W_MARK(2, t, 1);
+                uint8_t *stg = sDS + db * 2 * SUB;
+                // fp32 staging in the tile's dS^T buffer (dQ, the last MMA to read it, is complete): row = query, one
+                // swizzled [128 x 32] sub-tile per column half, a TMA reduce-add copy each.  Rows beyond the span's end
+                // hold exact zeros (their dS is zero).  The compute groups take the buffer back for tile t + 2 once the
+                // copies have read it.
+                if (!HDT_AGREE()) break;
+                tc_fence_after();
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {      // 32 columns per round of TMEM loads
+                    uint32_t r[32];
+                    tmem_ld32(tmem + TM_DQ + 64u * db + lane_base + 32u * half, r);
+                    tmem_wait_ld();
+                    if (half == 1) {          // the accumulator has been read: dQ of tile t + 2 may overwrite it
+                        tc_fence_before();
+                        mbar_arrive(&dq_free[db]);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4 *>(stg + half * SUB + swz(rl, c)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(&stg_full[db]);      // the reduce warp requests the copies and tells the compute groups when they have read the tile
+                if (w.j == U.nt - 1) {
+                    // ---- end of the unit: dK and dV of this thread's key row.  bf16 rows staged in the unit's K / V
+                    // buffer (every MMA of the unit is complete), one swizzled [128 x 64] tile per tensor, TMA stores;
+                    // the load warp takes the buffer for the unit after the next once the stores have read it. ----
+                    const int nrows = U.r1 - U.r0, kvb = w.uc & 1;
+                    uint8_t *skv = sKV + kvb * 2 * SUB;
+                    int up = -1;
+                    if (rl < nrows && a.part_dk != nullptr) up = a.up[U.r0 + rl];
+                    const int bx = max(__clz(nrows) - 25, 0);
+                    const int bbox = 64 >> bx;
+                    HDT_WAIT(acc_full, w.uc & 1, 15);
+                    if (HDT_AGREE()) {
+                        tc_fence_after();
+#pragma unroll
+                        for (int pc = 0; pc < 4; ++pc) {      // dK columns 0..31, 32..63, then dV
+                            const int tt = pc >> 1, c0 = 32 * (pc & 1);
+                            uint32_t r[32];
+                            tmem_ld32(tmem + (tt ? TM_DV : TM_DK) + lane_base + c0, r);
+                            tmem_wait_ld();
+                            if (pc == 3) {        // both accumulators have been read: the next unit may overwrite them
+                                tc_fence_before();
+                                mbar_arrive(acc_free);
+                            }
+                            const float sc = tt ? 1.f : a.scale;
+#pragma unroll
+                            for (int j = 0; j < 32; j += 8) {
+                                float v[8];
+#pragma unroll
+                                for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[j + e]) * sc;
+                                if (up >= 0) {      // this row lives on in the next stage: its fp32 gradients go there too
+                                    float4 *pt = reinterpret_cast<float4 *>((tt ? a.part_dv : a.part_dk) + ((size_t)up * H + U.h) * D + c0 + j);
+                                    pt[0] = make_float4(v[0], v[1], v[2], v[3]);
+                                    pt[1] = make_float4(v[4], v[5], v[6], v[7]);
+                                }
+                                *reinterpret_cast<uint4 *>(skv + tt * SUB + swz(rl, (c0 + j) >> 3)) =
+                                    make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+                            }
+                        }
+                    }
+                    fence_proxy_async_smem();
+                    go = group_all(ok, 1, 128);
+                    if (!go) break;
+                    // rows [0, nrows) of each staged tile as at most two boxes of b rows, b the largest power of two
+                    // <= min(nrows, 64): [0, b) and [nrows - b, nrows); where the two overlap the same values are written twice
+                    if (rl == 0) {
+#pragma unroll
+                        for (int tt = 0; tt < 2; ++tt) {
+                            tma_store_3d(&sm_out.m[1 + tt][bx], 0, U.h, U.r0, skv + tt * SUB);
+                            if (nrows > bbox) tma_store_3d(&sm_out.m[1 + tt][bx], 0, U.h, U.r0 + nrows - bbox, skv + tt * SUB + (nrows - bbox) * 128);
+                        }
+                        bulk_commit();
+                        bulk_wait_read();
+                        mbar_arrive(&kv_reuse[kvb]);
+                    }
+                }
+                W_MARK(2, t, 2);
+            }
+        }
+    }
+    if (!ok) {
+        if (atomicCAS(a.status, 0, HDT_ERR_TIMEOUT) == 0) {
+            a.status[1] = (KID << 8) | fail_site;
+            a.status[2] = (int)blockIdx.x;
+        }
+    }
+#undef HDT_WAIT
+#undef HDT_AGREE
+    tc_fence_before();
+    __syncthreads();
+    if (blockIdx.x == 0 && tid < 80 && (a.phases == 86 || a.phases == 85)) g_bwd_w_marks[tid] = s_marks[tid];
+    if (warp == 0) tmem_dealloc(tmem, TM_COLS);
+}
+
+// EMPTY blocks among those after the first n_fused of queue_split (rows without any key in this
+// stage: PAD, lone roots): zero gradients, also in the next stage's buffers for rows that live on.
+// One CTA of 128 threads per (block, head) over the last blocks of queue_split, from entry n_fused + first; thread t: row t.
+__global__ void __launch_bounds__(128) k_bwd_zero_empty(const BwdStageArgs a, int first) {
+    const int *rec = a.blocks + 5 * (size_t)a.queue_split[a.n_fused + first + blockIdx.x];
+    if (!(rec[4] & HDT_BLK_EMPTY)) return;
+    const int row = rec[0] + (int)threadIdx.x, h = blockIdx.y, H = a.H;
+    if (row >= rec[1]) return;
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    __nv_bfloat16 *g[3] = {(__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv};
+    float *pt[3] = {a.part_dq, a.part_dk, a.part_dv};
+    const int up = a.part_dq != nullptr ? a.up[row] : -1;
+#pragma unroll
+    for (int t = 0; t < 3; ++t) {
+        uint4 *o = reinterpret_cast<uint4 *>(g[t] + ((size_t)row * H + h) * 64);
+#pragma unroll
+        for (int c = 0; c < 8; ++c) o[c] = z;
+        if (up >= 0) {
+            float4 *c4 = reinterpret_cast<float4 *>(pt[t] + ((size_t)up * H + h) * 64);
+#pragma unroll
+            for (int c = 0; c < 16; ++c) c4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+}
+
+int read_bwd_w_marks(long long *out128) {
+    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out128, g_bwd_w_marks, sizeof(long long) * 128));
+    return HDT_OK;
+}
+int read_bwd_w_tiles(long long *out512) {
+    HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out512, g_bwd_w_tiles, sizeof(long long) * 512));
+    return HDT_OK;
+}
+
+int launch_bwd_tc_onewalk64(const BwdStageArgs &a, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+                            const CUtensorMap &tdo, const StoreMaps &outs, const CUtensorMap &tacc, int n_empty, cudaStream_t st) {
+    constexpr int smem_max = 14 * SUB + 2 * 1024 + 256 + 640;
+    const int smem = smem_max - ((a.phases == 86 || a.phases == 85) ? 0 : 640);      // (the clock marks of an instrumented run)
+    static DevOnce attr;
+    if (!attr.done()) {
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_w<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_w<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+        attr.set();
+    }
+    int n_sm = 0;
+    if (const int rc = sm_count(&n_sm)) return rc;
+    const int n_rest = a.nb - a.n_fused;
+    if (n_rest <= 0) return HDT_OK;
+    if (a.delta == nullptr || a.dq_acc == nullptr || n_empty < 0 || n_empty != a.n_empty)
+        return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_onewalk64: needs delta, the fp32 dQ buffer and the number of EMPTY blocks");
+    const long long units = (long long)n_rest * a.H;
+    const int grid = (int)(units < n_sm ? units : n_sm);
+    if (a.dirs != 7) k_bwd_tc_w<true><<<grid, 736, smem, st>>>(tq, tk, tv, tdo, outs, tacc, a);
+    else k_bwd_tc_w<false><<<grid, 736, smem, st>>>(tq, tk, tv, tdo, outs, tacc, a);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    if (n_empty > 0) {       // (EMPTY blocks cost nothing in the queue's order: they are the last n_empty of queue_split)
+        k_bwd_zero_empty<<<dim3(n_empty, a.H), 128, 0, st>>>(a, n_rest - n_empty);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+    }
+    return HDT_OK;
+}
+
+}  // namespace hdt

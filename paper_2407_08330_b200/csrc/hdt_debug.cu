@@ -189,3 +189,193 @@ extern "C" int hdt_debug_fwd_timeline(int64_t *out4096) {
     HDT_CUDA_CHECK(cudaDeviceSynchronize());
     return hdt::read_fwd_timeline((long long *)out4096);
 }
+
+extern "C" int hdt_debug_bwd_w_tiles(int64_t *out512) {
+    if (!out512) return hdt::set_error(HDT_ERR_INVALID_ARG, "hdt_debug_bwd_w_tiles: null pointer");
+    HDT_CUDA_CHECK(cudaDeviceSynchronize());
+    return hdt::read_bwd_w_tiles((long long *)out512);
+}
+
+extern "C" int hdt_debug_bwd_w_marks(int64_t *out128) {
+    if (!out128) return hdt::set_error(HDT_ERR_INVALID_ARG, "hdt_debug_bwd_w_marks: null pointer");
+    HDT_CUDA_CHECK(cudaDeviceSynchronize());
+    return hdt::read_bwd_w_marks((long long *)out128);
+}
+
+namespace hdt {
+// Timing probe of the tensor pipe: one CTA, one thread issues `reps` groups of `per_group` MMAs
+// (M = 128, N = n, K = 16 each, operands = whatever the shared memory / TMEM holds: only the time
+// matters), commits once, and the SM clock cycles from the first issue to the completion of the last
+// MMA go to out[0], those of the issue loop alone to out[1].  mode bit 0: A from TMEM; bit 1: consecutive
+// MMAs alternate between two accumulators, so that none depends on the one before it.
+__global__ void __launch_bounds__(128) k_debug_mma_rate(int n, int reps, int per_group, int mode, int b_mn, long long *out) {
+    extern __shared__ __align__(1024) uint8_t sm[];
+    __shared__ uint64_t bars2[2];
+    __shared__ uint32_t slot;
+    __shared__ int abort_s;
+    volatile int *abort_flag = &abort_s;
+    const int tid = threadIdx.x, warp = tid >> 5;
+    for (int i = tid; i < 4 * 16384 / 4; i += 128) ((uint32_t *)sm)[i] = 0x3c003c00u;     // finite bf16 values
+    if (tid == 0) { mbar_init(&bars2[0], 1); mbar_init(&bars2[1], 1); *abort_flag = 0; fence_mbar_init(); }
+    const int n_issuers = (mode & 4) ? 2 : 1;      // mode bit 2: warps 0 and 1 both issue (accumulators 64 columns apart)
+    uint64_t &bar = bars2[warp & 1];
+    fence_proxy_async_smem();
+    if (warp == 0) tmem_alloc(&slot, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = slot;
+    if (warp < n_issuers) {
+        long long t0 = 0, t1 = 0;
+        if (elect_one()) {
+            const uint32_t idesc = idesc_bf16(n > 64 && n_issuers == 2 ? 64 : n, false, b_mn != 0);
+            const uint64_t da = smem_desc(smem_u32(sm), 0, 1024);
+            const uint64_t db = b_mn ? smem_desc(smem_u32(sm) + 2 * 16384, 16384, 1024) : smem_desc(smem_u32(sm) + 2 * 16384, 0, 1024);
+            const int alt = (mode >> 1) & 1, at = mode & 1;
+            t0 = clock64();
+            for (int r = 0; r < reps; ++r) {
+                const uint32_t d = tmem + 256u * (r & 1) + 64u * warp;
+                for (int g = 0; g < per_group; ++g) {
+                    const uint32_t dd = d + (alt ? 128u * (g & 1) : 0u);
+                    const uint32_t acc = alt ? (g > 1) : (g > 0);
+                    if (at) mma_ts(dd, tmem + 448u + 8u * (g & 3), db + (uint64_t)((g & 3) * (b_mn ? 128 : 2)), idesc, acc);
+                    else mma_ss(dd, da + (uint64_t)(2 * (g & 3)), db + (uint64_t)((g & 3) * (b_mn ? 128 : 2)), idesc, acc);
+                }
+            }
+            t1 = clock64();
+            mma_commit(&bar);
+        }
+        __syncwarp();
+        const bool ok = mbar_wait(&bar, 0, abort_flag, 400000000LL);
+        const long long t2 = clock64();
+        if (tid == 0) { out[0] = ok ? t2 - t0 : -1; out[1] = t1 - t0; }
+        if (tid == 32) { out[2] = ok ? t2 - t0 : -1; out[3] = t1 - t0; }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+}  // namespace hdt
+
+// Diagnostics: see k_debug_mma_rate.  out2 (host): cycles until the last MMA completed, cycles of the issue loop.
+extern "C" int hdt_debug_mma_rate(int32_t n, int32_t reps, int32_t per_group, int32_t mode, int32_t b_mn, int64_t *out2) {
+    if (!out2 || n < 16 || n > 128 || n % 16 || reps < 1 || reps > 100000 || per_group < 1 || per_group > 64 || mode < 0 || mode > 7)
+        return hdt::set_error(HDT_ERR_INVALID_ARG, "hdt_debug_mma_rate: bad arguments");
+    long long *d = nullptr;
+    HDT_CUDA_CHECK(cudaMalloc(&d, 32));
+    const int smem = 4 * 16384;
+    HDT_CUDA_CHECK(cudaFuncSetAttribute(hdt::k_debug_mma_rate, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    hdt::k_debug_mma_rate<<<1, 128, smem>>>(n, reps, per_group, mode, b_mn, d);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(out2, d, 16, cudaMemcpyDeviceToHost);
+    cudaFree(d);
+    if (e != cudaSuccess) return hdt::set_error(HDT_ERR_CUDA, "hdt_debug_mma_rate: %s", cudaGetErrorString(e));
+    return HDT_OK;
+}
+
+namespace hdt {
+// Timing probe of TMEM loads: `warps` warps (lane quarter = warp % 4) each do `reps` rounds of `per_round`
+// tcgen05.ld (32 lanes x 16 columns) followed by one tcgen05.wait::ld, while (mma != 0) warp 31 keeps the
+// tensor pipe busy with N = 64 MMAs accumulating into other TMEM columns.  out[w] = cycles of warp w's loop.
+__global__ void __launch_bounds__(1024) k_debug_tmem_ld(int warps, int reps, int per_round, int mma, long long *out) {
+    extern __shared__ __align__(1024) uint8_t sm[];
+    __shared__ uint64_t bar;
+    __shared__ uint32_t slot;
+    __shared__ int abort_s, stop_s;
+    volatile int *abort_flag = &abort_s;
+    volatile int *stop = &stop_s;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    for (int i = tid; i < 4 * 16384 / 4; i += blockDim.x) ((uint32_t *)sm)[i] = 0x3c003c00u;
+    if (tid == 0) { mbar_init(&bar, 1); *abort_flag = 0; *stop = 0; fence_mbar_init(); }
+    fence_proxy_async_smem();
+    if (warp == 0) tmem_alloc(&slot, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = slot;
+    if (warp < warps && mma >= 2) {
+        // mma = 2 + n: warp 31 issues n MMAs into columns 256..383 and commits; the loading warps wait for the
+        // commit's barrier and then time `reps` rounds of loads FROM THOSE COLUMNS (out[w] = cycles of the rounds,
+        // out[16 + w] = cycles the wait for the barrier took after the loop's start)
+        const uint32_t base = tmem + 256u + ((uint32_t)((warp & 3) * 32) << 16) + 16u * ((warp >> 2) & 7);
+        uint32_t acc = 0;
+        const long long ta = clock64();
+        (void)mbar_wait(&bar, 0, abort_flag, 400000000LL);
+        tc_fence_after();
+        const long long t0 = clock64();
+        for (int r = 0; r < reps; ++r) {
+            uint32_t v[4][16];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k < per_round) tmem_ld16(base + 64u * (k & 1), v[k]);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k < per_round) acc ^= v[k][0] ^ v[k][15];
+        }
+        const long long t1 = clock64();
+        if (lane == 0) { out[warp] = t1 - t0 + (acc == 0x12345678u ? 1 : 0); if (warp < 16) out[16 + warp] = t0 - ta; }
+    } else if (warp == 31 && mma >= 2) {
+        if (elect_one()) {
+            const uint32_t idesc = idesc_bf16(64, false, true);
+            const uint64_t da = smem_desc(smem_u32(sm), 0, 1024);
+            const uint64_t db = smem_desc(smem_u32(sm) + 2 * 16384, 16384, 1024);
+            for (int g = 0; g < mma - 2; ++g) mma_ss(tmem + 256u + 64u * (g & 1), da + (uint64_t)(2 * (g & 3)), db + (uint64_t)((g & 3) * 128), idesc, g > 1);
+            mma_commit(&bar);
+        }
+        __syncwarp();
+    } else if (warp < warps) {
+        const uint32_t base = tmem + ((uint32_t)((warp & 3) * 32) << 16) + 16u * ((warp >> 2) & 7);
+        uint32_t acc = 0;
+        const long long t0 = clock64();
+        for (int r = 0; r < reps; ++r) {
+            uint32_t v[4][16];
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k < per_round) tmem_ld16(base + 128u * (k & 1), v[k]);
+            tmem_wait_ld();
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (k < per_round) acc ^= v[k][0] ^ v[k][15];
+        }
+        const long long t1 = clock64();
+        if (lane == 0) out[warp] = t1 - t0 + (acc == 0x12345678u ? 1 : 0);
+        __syncwarp();
+        if (warp == 0 && lane == 0) *stop = 1;
+    } else if (warp == 31 && mma == 1) {
+        if (elect_one()) {
+            const uint32_t idesc = idesc_bf16(64, false, true);
+            const uint64_t da = smem_desc(smem_u32(sm), 0, 1024);
+            const uint64_t db = smem_desc(smem_u32(sm) + 2 * 16384, 16384, 1024);
+            int n = 0;
+            while (!*stop && n < 20000) {
+                for (int g = 0; g < 8; ++g) mma_ss(tmem + 256u + 64u * (g & 1), da + (uint64_t)(2 * (g & 3)), db + (uint64_t)((g & 3) * 128), idesc, 1);
+                n += 8;
+            }
+            mma_commit(&bar);
+        }
+        __syncwarp();
+        (void)mbar_wait(&bar, 0, abort_flag, 400000000LL);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+}  // namespace hdt
+
+// Diagnostics: see k_debug_tmem_ld.  out32 (host): cycles of each loading warp's loop.
+extern "C" int hdt_debug_tmem_ld(int32_t warps, int32_t reps, int32_t per_round, int32_t mma, int64_t *out32) {
+    if (!out32 || warps < 1 || warps > 28 || reps < 1 || reps > 100000 || per_round < 1 || per_round > 4)
+        return hdt::set_error(HDT_ERR_INVALID_ARG, "hdt_debug_tmem_ld: bad arguments");
+    long long *d = nullptr;
+    HDT_CUDA_CHECK(cudaMalloc(&d, 256));
+    HDT_CUDA_CHECK(cudaMemset(d, 0, 256));
+    const int smem = 4 * 16384;
+    HDT_CUDA_CHECK(cudaFuncSetAttribute(hdt::k_debug_tmem_ld, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    hdt::k_debug_tmem_ld<<<1, 1024, smem>>>(warps, reps, per_round, mma, d);
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e == cudaSuccess) e = cudaMemcpy(out32, d, 256, cudaMemcpyDeviceToHost);
+    cudaFree(d);
+    if (e != cudaSuccess) return hdt::set_error(HDT_ERR_CUDA, "hdt_debug_tmem_ld: %s", cudaGetErrorString(e));
+    return HDT_OK;
+}

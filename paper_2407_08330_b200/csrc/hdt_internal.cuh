@@ -114,6 +114,8 @@ extern int g_no_fwd_mc;    // option "no_fwd_mc": blocks that are not self-conta
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 extern int g_no_pdl;       // option "no_pdl"
+extern int g_bwd_walk;     // option "bwd_walk": families longer than a row block in the head_dim 64 backward: 0 = one walk on the
+                           // warp-specialised kernel, 1 = two walks (no dQ buffer, deterministic), 2 = one walk on the lockstep kernel
 
 // Direction bits inside a row range (paper, "Mathematical Reasoning Tasks": the ListOps attention
 // patterns).  Row e of a stage has the key range [lo, hi).  If the range starts at or after e, e is
@@ -225,6 +227,7 @@ struct BwdStageArgs {
     const float *next_own_dq, *next_own_dk, *next_own_dv;
     float *dq_acc;                                // stage 0, head_dim 64: fp32 [T,H,64] buffer, zero on entry, that the one-walk kernel of the
                                                   // split families adds its dQ tiles to (nullptr: they are walked twice instead)
+    int n_empty;                                  // EMPTY blocks of the stage (-1: unknown)
     int gather_end_q, gather_end_k;               // gathering kernel: elements at or beyond these read as zero rows on the Q/dO and the K/V side (0: n)
 };
 
@@ -236,6 +239,8 @@ int launch_bwd_tc(const BwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_fwd_tc_upper(const FwdStageArgs &a, int head_dim, cudaStream_t st);
 int launch_bwd_tc_upper(const BwdStageArgs &a, int head_dim, cudaStream_t st);
 int read_bwd_phase_cycles(long long *out16);
+int read_bwd_w_marks(long long *out128);
+int read_bwd_w_tiles(long long *out512);          // the warp-specialised one-walk backward: see hdt_debug_bwd_w_cycles
 int read_bwd_t_phase_cycles(long long *out16);   // adds to out16
 int read_bwd_t_timeline(long long *out2048);     // per CTA of the last instrumented launch: entry, first tiles in, end (ns), SM
 int read_fwd_phase_cycles(long long *out16);

@@ -68,4 +68,11 @@ struct OutMaps { CUtensorMap m[7]; };     // the same for one tensor (the forwar
 int launch_bwd_tc_fused64(const BwdStageArgs &a, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                           const CUtensorMap &tdo, const StoreMaps &outs, cudaStream_t st);
 
+// The blocks after the first n_fused of queue_split (pieces of families longer than a row block, and
+// EMPTY blocks) at head_dim 64 through the warp-specialised one-walk backward (hdt_attn_tc_bwd_w.cu):
+// dK, dV rows are written, dQ tiles are added to a.dq_acc through `tacc` (the caller converts the sums).
+// n_empty: EMPTY blocks among them (-1: unknown).
+int launch_bwd_tc_onewalk64(const BwdStageArgs &a, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
+                            const CUtensorMap &tdo, const StoreMaps &outs, const CUtensorMap &tacc, int n_empty, cudaStream_t st);
+
 }  // namespace hdt
