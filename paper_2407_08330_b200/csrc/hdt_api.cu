@@ -429,9 +429,9 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
     const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3 && ix->directions == 7;
     // No delta pass when every kernel of this call computes dO . O of its rows itself: stage 0
-    // entirely on the transposed looping kernel (head_dim 64, every block self-contained), the
-    // stages above it on the gathering tensor-core kernels.
-    const bool fused_delta = dtype == HDT_BF16 && !g_force_simt && head_dim == 64 && g_no_persistent == 0 &&
+    // entirely on the looping kernels (the transposed one at head_dim 64, the fused five-MMA one at
+    // head_dim 128; every block self-contained), the stages above it on the gathering tensor-core kernels.
+    const bool fused_delta = dtype == HDT_BF16 && !g_force_simt && (head_dim == 64 || head_dim == 128) && g_no_persistent == 0 &&
                              !g_no_fused_delta && ix->directions == 7 && ix->desc[0].n_fused == ix->desc[0].nb &&
                              ix->desc[0].nb > 0 && (ix->n_stages == 1 || (overlap && tc_upper));
     // Families longer than a row block (head_dim 64): one walk over their tile pairs, dQ tiles summed

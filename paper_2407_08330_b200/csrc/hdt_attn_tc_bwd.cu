@@ -526,7 +526,10 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
 // next item as soon as the output MMAs of the current one have finished — the gradients are
 // staged in tiles of their own, so the loads fly while the CTA drains, stages and stores.
 // ---------------------------------------------------------------------------------------------
-template <int D>
+// FD (fused delta): a.delta is not read; delta[row] = dO[row] . O[row] is computed here: the 2 D / 16 lanes that
+// share a token row fetch 16 bytes each of its O and dO rows at the top of the item (past L1) and reduce them
+// while S and dP are computed; the sums reach the row's two threads through shared memory.
+template <int D, bool FD = false>
 __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ CUtensorMap tm_q,
                                                         const __grid_constant__ CUtensorMap tm_k,
                                                         const __grid_constant__ CUtensorMap tm_v,
@@ -543,11 +546,13 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
     uint64_t *bar_a = bar_in + 1, *bar_b = bar_in + 2;      // S and dP (two issuing threads); dV, dK, dQ (three)
     uint32_t *slot = (uint32_t *)(bar_in + 3);
     volatile int *abort_flag = (volatile int *)(slot + 1);
+    float *s_delta = (float *)(bar_in + 8);                 // FD: dO . O of the item's 128 rows
 
     const int tid = threadIdx.x, warp = tid >> 5, rl = tid & 127, hf = tid >> 7;
     const int H = a.H, G = gridDim.x;
     const float LOG2E = 1.4426950408889634f;
     const int n_items = a.n_fused * H;
+    constexpr int LPR = D / 8, RPP = 256 / LPR, NPASS = 128 / RPP;      // FD: lanes per row, rows per pass, passes
 
     if (tid == 0) {
         mbar_init(bar_in, 1);
@@ -594,7 +599,7 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
             r.lo = a.rng[2 * row];
             r.hi = a.rng[2 * row + 1];
             r.lse = a.lse[(size_t)d.h * a.T + row];      // natural log; scaled where it is used
-            r.dl = a.delta[(size_t)d.h * a.T + row];
+            if constexpr (!FD) r.dl = a.delta[(size_t)d.h * a.T + row];
             if (a.part_dq != nullptr) r.up = a.up[row];
         }
         return r;
@@ -609,6 +614,20 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
             const RowStat rn = load_stat(d1);                          // row statistics one item ahead
             const int r0 = d0.r0, r1 = d0.r1, h = d0.h, nrows = r1 - r0;
             const int Nc = (nrows + 15) & ~15;
+            uint4 xo[NPASS], xg[NPASS];      // FD: chunk tid % LPR of rows tid / LPR + RPP k of O and dO
+            if constexpr (FD) {
+#pragma unroll
+                for (int k = 0; k < NPASS; ++k) {
+                    const int r = tid / LPR + RPP * k;
+                    xo[k] = make_uint4(0u, 0u, 0u, 0u);
+                    xg[k] = make_uint4(0u, 0u, 0u, 0u);
+                    if (r < nrows) {
+                        const size_t off = ((size_t)(r0 + r) * H + h) * D + (tid % LPR) * 8;
+                        xo[k] = ld_stream16(reinterpret_cast<const __nv_bfloat16 *>(a.o) + off);
+                        xg[k] = ld_stream16(reinterpret_cast<const __nv_bfloat16 *>(a.d_o) + off);
+                    }
+                }
+            }
             // the next item's tiles start their way from HBM to L2 now; the loads into shared memory
             // (requested once this item's output MMAs have released the tiles) then find them there
             if (tid == 0 && d1.valid) {
@@ -632,14 +651,31 @@ __global__ void __launch_bounds__(256, 1) k_bwd_tc_loop(const __grid_constant__ 
                 mma_commit(bar_a);
             }
             const bool inq = rl < nrows;
-            const float lse2 = rc.lse * LOG2E, dl = rc.dl;
+            const float lse2 = rc.lse * LOG2E;
+            float dl = rc.dl;
             const int jl = max(rc.lo - r0, 0), jh = min(rc.hi - r0, nrows);
             const bool has = inq && jh > jl;
+            if constexpr (FD) {      // dO . O of the rows this thread fetched: products, then a sum over the LPR lanes of a row
+#pragma unroll
+                for (int k = 0; k < NPASS; ++k) {
+                    const uint32_t xs[4] = {xo[k].x, xo[k].y, xo[k].z, xo[k].w}, ys[4] = {xg[k].x, xg[k].y, xg[k].z, xg[k].w};
+                    float acc = 0.f;
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        acc = fmaf(__uint_as_float(xs[w] << 16), __uint_as_float(ys[w] << 16), acc);
+                        acc = fmaf(__uint_as_float(xs[w] & 0xffff0000u), __uint_as_float(ys[w] & 0xffff0000u), acc);
+                    }
+#pragma unroll
+                    for (int m = 1; m < LPR; m <<= 1) acc += __shfl_xor_sync(0xffffffffu, acc, m);
+                    if (tid % LPR == 0) s_delta[tid / LPR + RPP * k] = acc;
+                }
+            }
             ok = mbar_wait(bar_a, it & 1, abort_flag, WAIT_CYCLES) && ok;
             // the previous item's staged gradients have left shared memory before P and dS overwrite them
             if (store_thread) bulk_wait_read();
             __syncthreads();
             tc_fence_after();
+            if constexpr (FD) dl = s_delta[rl];
 #pragma unroll
             for (int sl = 0; sl < 2; ++sl) {
                 const int s0 = 64 * hf + 32 * sl;
@@ -1307,16 +1343,20 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
     }
     if (((D == 128 && !a.no_persistent) || (D == 64 && a.no_persistent == 5)) && a.n_fused > 0 && !dirs) {
         // self-contained blocks through the looping kernel, the rest through the general one
-        constexpr int smem_l = (4 * (D / 64) + 4 + (D / 64)) * SUB + 1024 + 64;
+        constexpr int smem_l = (4 * (D / 64) + 4 + (D / 64)) * SUB + 1024 + 64 + 512;
         static DevOnce attr_l;
         int n_sm_l = 0;
         if (const int rc_ = sm_count(&n_sm_l)) return rc_;
         if (!attr_l.done()) {
             HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_loop<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_l));
+            HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_loop<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_l));
             attr_l.set();
         }
         const long long items = (long long)a.n_fused * a.H;
-        k_bwd_tc_loop<D><<<(int)(items < n_sm_l ? items : n_sm_l), 256, smem_l, st>>>(tq, tk, tv, tdo, outs, a);
+        if (a.delta == nullptr) {      // no delta pass ran: the kernel computes dO . O of its rows itself
+            if (a.o == nullptr) return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc: the fused-delta kernel needs o");
+            k_bwd_tc_loop<D, true><<<(int)(items < n_sm_l ? items : n_sm_l), 256, smem_l, st>>>(tq, tk, tv, tdo, outs, a);
+        } else k_bwd_tc_loop<D><<<(int)(items < n_sm_l ? items : n_sm_l), 256, smem_l, st>>>(tq, tk, tv, tdo, outs, a);
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
         b.rest_only = 1;

@@ -11,29 +11,41 @@
 //   MMA      dV += P^T dO (A operand from TMEM), dK += dS^T Q: accumulated in TMEM over the whole walk;
 //            after both steps dQ_tile = dS K (M = the tile's 128 queries, A = dS^T read MN-major), a
 //            fresh accumulator per tile
-//   drain    the dQ tile as fp32, in two halves of 32 columns, through a swizzled staging tile and a TMA
-//            reduce-add copy each into the buffer a.dq_acc [T, H, 64] (k_dq_finish scales and converts
-//            the sums afterwards); at the end of the unit dK, dV -> bf16 rows through TMA stores
+//   drain    the dQ tile as fp32 through a swizzled staging tile and two TMA reduce-add copies into the
+//            buffer a.dq_acc [T, H, 64] (k_dq_finish scales and converts the sums afterwards); at the
+//            end of the unit dK, dV -> bf16 rows, staged in the unit's K / V buffer, TMA stores
 // Every tile pair is visited once (the two-walk kernels compute S, dP, P, dS of each pair twice).
 //
 // One CTA of 736 threads per SM.  Warps 0-7 compute step a (queries 0..63 of each tile: warp = TMEM lane
 // quarter x half of the step's queries), warps 8-15 step b, warps 16-19 drain, warp 20 requests the
 // tiles (TMA) and fetches the queries' LSE and delta, warp 21 issues the MMAs, warp 22 requests the
-// reduce-add copies of the staged dQ tiles.  The roles meet only at
-// mbarriers, so the tensor pipe, the exponentials of the two compute groups and the drains overlap;
-// S^T / dP^T are double buffered by step, dS^T and the dQ accumulator by tile, Q / dO in a ring of
-// three tiles; K / V have one buffer (the next unit's are requested into L2 ahead of time).
+// reduce-add copies of the staged dQ tiles.  The roles meet only at mbarriers, so the tensor pipe, the
+// exponentials of the two compute groups, the drains and the copies overlap; S^T / dP^T are double
+// buffered by step, dS^T and the dQ accumulator by tile, Q / dO by tile, K / V by unit.
 // TMEM columns: S^T a 0..63 (P^T a over 0..15 and 32..47: each warp writes inside the columns it alone
 // reads), dP^T a 64..127, step b the same from 128; dK 256..319, dV 320..383, dQ 384..447 and 448..511.
-// Measured on this part (one thread issuing back to back): an MMA of M = 128, K = 16 takes about 75
-// cycles at N = 64 with both operands in shared memory, 47 with A in TMEM, 106 / 70 at N = 128 — the
-// operand reads, not the arithmetic, set the pace at these shapes — which makes a tile pair cost the
-// tensor pipe about 2800 cycles here (16 x 75 for S^T / dP^T, 8 x 47 for dV, 16 x 75 for dK and dQ).
-// What a compute group waits for between two of its steps is dV of the step (its P^T lies over the
-// S^T columns) and the next S^T / dP^T; dK and dQ, which read dS^T from shared memory, are issued
-// behind them.  Clock stamps of an earlier form with four warps per compute group showed a step's
-// arithmetic (64 entries per thread) taking 3500 cycles, an issue rate of one instruction in eight
-// cycles per warp: the groups have eight warps each since.
+//
+// What was measured on the way (cycles of the SM clock, one CTA per SM, config 5):
+//  - one thread issuing back to back: an MMA of M = 128, K = 16 takes about 75 cycles at N = 64 with both
+//    operands in shared memory (63 with two issuing warps: the pipe's own pace), 39..47 with A in TMEM,
+//    106 / 70 at N = 128: the operand reads, not the arithmetic, set the pace at these shapes.  A tile
+//    pair costs the tensor pipe about 2500 cycles here (32 MMAs from shared memory, 8 with A in TMEM).
+//  - a round of tcgen05.ld + wait costs a warp 150 cycles alone and about 100 cycles per warp that shares
+//    its TMEM lane quarter at the same time, whether the round loads 16 or 64 columns: few, wide rounds.
+//  - what a compute group waits for between two of its steps is dV of the step (its P^T lies over the
+//    S^T columns) and the next S^T / dP^T; dK and dQ, which read dS^T from shared memory, are issued
+//    behind them.  With four warps per compute group a step's arithmetic (64 entries per thread) took
+//    3500 cycles, one instruction issued in eight cycles per warp: the groups have eight warps each.
+//  - units end often (4.7 tiles per unit on config 5): one K / V buffer cost 13000 cycles per unit
+//    (the pipeline drains and refills around the reload), draining dK / dV by the compute groups with
+//    plain stores 7000 (32 rows per store instruction); with the second buffer, the drain group taking
+//    the accumulators first and staging them in the finished unit's K / V buffer, a unit's first tile
+//    takes 4000..5000 cycles against 3500 inside a unit.
+//  - the reduce-add copies of a 32 KB dQ tile take about 2500 cycles to read their staging tile; with
+//    the staging in the tile's dS^T buffer every other tile waited for them (a third of the ring of
+//    Q / dO tiles went to a staging area of its own instead), requested by a warp of their own because
+//    the requesting thread waits for the read.  Adding the tile from registers with red.global.v4.f32
+//    was much slower (the step time rose from 0.75 to 0.98 ms).
 #include <cuda_bf16.h>
 
 #include "hdt_internal.cuh"
@@ -69,9 +81,9 @@ __device__ long long g_bwd_w_marks[128];
 __device__ long long g_bwd_w_tiles[512];      // (instrumented run) CTA 0: SM clock at the MMA warp's loop top of every tile, unit number in the low 8 bits
 #define W_MARK(role, tt, id)                                                                    \
     do {                                                                                        \
-        if (marks && (tt) >= 7 && (tt) < 9) {                                                 \
+        if (marks && (tt) >= 4 && (tt) < 6) {                                                 \
             const long long now_ = clock64();                                                   \
-            if (lane == 0) s_marks[(role) * 16 + ((tt) - 7) * 8 + (id)] = now_;                \
+            if (lane == 0) s_marks[(role) * 16 + ((tt) - 4) * 8 + (id)] = now_;                \
         }                                                                                       \
     } while (0)
 
@@ -94,10 +106,10 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     constexpr int W_DRAIN = 16, W_LOAD = 20, W_MMA = 21, W_RED = 22;      // first warp of each role
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t *sKV = smem_raw;                 // [2 units] x {K, V}
-    uint8_t *sQD = sKV + 4 * SUB;            // [3 tiles] x {Q, dO}
-    uint8_t *sDS = sQD + 6 * SUB;            // [2 tiles] x {dS^T of step a, of step b}: row = key, 64 queries per row; once dQ of
-                                             // the tile has read it, the same 32 KB stage the dQ tile as fp32 (two swizzled [128 x 32] halves)
-    float2 *sStat = (float2 *)(sDS + 4 * SUB);   // [2 tiles][128]: LSE * log2(e) and delta of the tile's queries
+    uint8_t *sQD = sKV + 4 * SUB;            // [2 tiles] x {Q, dO}
+    uint8_t *sDS = sQD + 4 * SUB;            // [2 tiles] x {dS^T of step a, of step b}: row = key, 64 queries per row
+    uint8_t *sStg = sDS + 4 * SUB;           // staging of a dQ tile as fp32: two swizzled [128 rows x 32 columns] halves
+    float2 *sStat = (float2 *)(sStg + 2 * SUB);   // [2 tiles][128]: LSE * log2(e) and delta of the tile's queries
     uint64_t *bars = (uint64_t *)(sStat + 2 * 128);
     uint64_t *qdo_full = bars, *qdo_empty = bars + 3, *sdp_full = bars + 6, *pds_ready = bars + 8;
     uint64_t *dq_full = bars + 10, *dq_free = bars + 12, *kv_full = bars + 14, *kv_empty = bars + 16;
@@ -109,8 +121,8 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int H = a.H, G = gridDim.x;
     const float LOG2E = 1.4426950408889634f;
-    const bool marks = (a.phases == 86 || a.phases == 85) && blockIdx.x == 0 && (warp == 0 || warp == 8 || warp == W_DRAIN || warp >= W_LOAD);
-    if ((a.phases == 86 || a.phases == 85) && tid < 80) s_marks[tid] = 0;
+    const bool marks = (a.phases == 86) && blockIdx.x == 0 && (warp == 0 || warp == 8 || warp == W_DRAIN || warp >= W_LOAD);
+    if ((a.phases == 86) && tid < 80) s_marks[tid] = 0;
     // EMPTY blocks cost nothing in the queue's order, so they are the tail of queue_split and are left
     // out here (k_bwd_zero_empty writes their rows)
     const int n_units = (a.nb - a.n_fused - a.n_empty) * H;
@@ -179,7 +191,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     // are in flight while the current unit is walked and no role waits for them at a unit boundary.
     auto step = [&](Walk &w) {      // to the next tile
         ++w.t;
-        if (++w.qs == 3) { w.qs = 0; w.qph ^= 1; }
+        if (++w.qs == 2) { w.qs = 0; w.qph ^= 1; }
         if (w.uc >= 0 && w.j + 1 < w.U.nt) { ++w.j; return; }
         while (true) {
             const WUnit u = w.N;
@@ -190,7 +202,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     };
     auto begin = [&]() {
         Walk w;
-        w.k = 0; w.j = 0; w.t = -1; w.uc = -1; w.valid = 0; w.qs = 2; w.qph = 1; w.U = WUnit{0, 0, 0, 0, 0, 0, 0};
+        w.k = 0; w.j = 0; w.t = -1; w.uc = -1; w.valid = 0; w.qs = 1; w.qph = 1; w.U = WUnit{0, 0, 0, 0, 0, 0, 0};
         w.N = get_unit(w.k++);
         step(w);
         return w;
@@ -229,7 +241,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                         tma_load_3d(kv + SUB, &tm_v, 0, U.h, U.r0, &kv_full[w.uc & 1]);
                     }
                 }
-                if (w.t >= 3) HDT_WAIT(&qdo_empty[qs], w.qph ^ 1, 2);
+                if (w.t >= 2) HDT_WAIT(&qdo_empty[qs], w.qph ^ 1, 2);
                 if (!HDT_AGREE()) break;
                 W_MARK(3, w.t, 1);
                 if (lane == 0) {
@@ -237,11 +249,6 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                     mbar_expect_tx(&qdo_full[qs], 2u * SUB);
                     tma_load_3d(qd, &tm_q, 0, U.h, q0, &qdo_full[qs]);
                     tma_load_3d(qd + SUB, &tm_do, 0, U.h, q0, &qdo_full[qs]);
-                }
-                // the statistics have two buffers only: tile t - 2 must be through (the tile loads above did not wait for that)
-                if (w.t >= 2) {
-                    const int q2 = qs == 0 ? 1 : qs == 1 ? 2 : 0;          // ring stage of tile t - 2
-                    HDT_WAIT(&qdo_empty[q2], qs == 2 ? w.qph : (w.qph ^ 1), 17);
                 }
                 if (!HDT_AGREE()) break;
 #pragma unroll
@@ -256,17 +263,17 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
         } else if (warp == W_RED) {
             // ================= reduce warp: the TMA reduce-add copies of every staged dQ tile =================
             for (Walk w = begin(); w.valid && ok; step(w)) {
-                const int t = w.t, db = t & 1;
-                HDT_WAIT(&stg_full[db], (t >> 1) & 1, 18);
+                const int t = w.t;
+                HDT_WAIT(&stg_full[0], t & 1, 18);
                 if (!HDT_AGREE()) break;
                 if (lane == 0) {
-                    const uint8_t *stg = sDS + db * 2 * SUB;
+                    const uint8_t *stg = sStg;
                     const int q0 = w.U.ka + 128 * w.j;      // the tile's first query row
                     tma_reduce_add_3d(&tm_acc, 0, w.U.h, q0, stg);
                     tma_reduce_add_3d(&tm_acc, 32, w.U.h, q0, stg + SUB);
                     bulk_commit();
                     bulk_wait_read();                 // the copies have read the tile:
-                    mbar_arrive(&stg_free[db]);       // the compute groups may write dS^T of tile t + 2 there
+                    mbar_arrive(&stg_free[0]);        // the drain group may stage the next tile
                 }
                 __syncwarp();
             }
@@ -330,21 +337,22 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 const bool first = w.j == 0, last = w.j == w.U.nt - 1;
                 struct { int valid, qs, qph, uc; } n;
                 n.valid = !last || w.N.valid;
-                n.qs = w.qs == 2 ? 0 : w.qs + 1;
-                n.qph = w.qs == 2 ? (w.qph ^ 1) : w.qph;
+                n.qs = w.qs ^ 1;
+                n.qph = w.qs == 1 ? (w.qph ^ 1) : w.qph;
                 n.uc = w.uc + (last ? 1 : 0);
                 const int kvb = w.uc & 1;
                 const uint32_t acc = first ? 0u : 1u;
                 // ---- step a: dV; S^T, dP^T of the next tile's step a; dK ----
                 W_MARK(4, t, 0);
-                if ((a.phases == 86 || a.phases == 85) && blockIdx.x == 0 && lane == 0 && t < 512) g_bwd_w_tiles[t] = (clock64() << 8) | (long long)(w.uc & 255);
-                HDT_WAIT(&pds_ready[0], t & 1, 5);
-                W_MARK(4, t, 1);
+                if ((a.phases == 86) && blockIdx.x == 0 && lane == 0 && t < 512) g_bwd_w_tiles[t] = (clock64() << 8) | (long long)(w.uc & 255);
+                // (what is normally there already first, the wait for the compute group last: it ends the chain)
                 if (first && w.uc >= 1) HDT_WAIT(acc_free, (w.uc - 1) & 1, 6);      // the previous unit's dK, dV have been read
                 if (n.valid) {
                     HDT_WAIT(&qdo_full[n.qs], n.qph, 7);
                     if (last) HDT_WAIT(&kv_full[n.uc & 1], (n.uc >> 1) & 1, 8);      // the next tile opens a unit (the other K / V buffer)
                 }
+                W_MARK(4, t, 1);
+                HDT_WAIT(&pds_ready[0], t & 1, 5);
                 if (!HDT_AGREE()) break;
                 W_MARK(4, t, 2);
                 if (elect_one()) {
@@ -356,9 +364,9 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 __syncwarp();
                 W_MARK(4, t, 3);
                 // ---- step b: dV; S^T, dP^T of the next tile's step b; dK; the tile's dQ ----
-                HDT_WAIT(&pds_ready[1], t & 1, 9);
-                W_MARK(4, t, 4);
                 if (t >= 2) HDT_WAIT(&dq_free[db], ((t >> 1) + 1) & 1, 10);
+                W_MARK(4, t, 4);
+                HDT_WAIT(&pds_ready[1], t & 1, 9);
                 if (!HDT_AGREE()) break;
                 W_MARK(4, t, 5);
                 if (elect_one()) {
@@ -419,10 +427,10 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                     all[i] = __all_sync(0xffffffffu, km[i] == 0xffffu);
                 }
                 W_MARK(x, t, 0);
-                HDT_WAIT(&sdp_full[x], t & 1, 11);
-                W_MARK(x, t, 1);
                 HDT_WAIT(&stat_full[db], (t >> 1) & 1, 12);                      // the queries' statistics are there
-                if (t >= 2) HDT_WAIT(&stg_free[db], ((t >> 1) + 1) & 1, 13);    // dQ of tile t - 2 has left this buffer (read as dS^T, then staged in it)
+                if (t >= 2) HDT_WAIT(&dq_full[db], ((t >> 1) + 1) & 1, 13);     // dQ of tile t - 2 has read this dS^T buffer
+                W_MARK(x, t, 1);
+                HDT_WAIT(&sdp_full[x], t & 1, 11);                               // (last: this one ends the chain)
                 if (!HDT_AGREE()) break;
                 tc_fence_after();
                 W_MARK(x, t, 2);
@@ -484,30 +492,9 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 W_MARK(2, t, 0);
                 HDT_WAIT(&dq_full[db], (t >> 1) & 1, 14);
                 W_MARK(2, t, 1);
-                uint8_t *stg = sDS + db * 2 * SUB;
-                // fp32 staging in the tile's dS^T buffer (dQ, the last MMA to read it, is complete): row = query, one
-                // swizzled [128 x 32] sub-tile per column half, a TMA reduce-add copy each.  Rows beyond the span's end
-                // hold exact zeros (their dS is zero).  The compute groups take the buffer back for tile t + 2 once the
-                // copies have read it.
-                if (!HDT_AGREE()) break;
-                tc_fence_after();
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {      // 32 columns per round of TMEM loads
-                    uint32_t r[32];
-                    tmem_ld32(tmem + TM_DQ + 64u * db + lane_base + 32u * half, r);
-                    tmem_wait_ld();
-                    if (half == 1) {          // the accumulator has been read: dQ of tile t + 2 may overwrite it
-                        tc_fence_before();
-                        mbar_arrive(&dq_free[db]);
-                    }
-#pragma unroll
-                    for (int c = 0; c < 8; ++c)
-                        *reinterpret_cast<uint4 *>(stg + half * SUB + swz(rl, c)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
-                }
-                fence_proxy_async_smem();
-                mbar_arrive(&stg_full[db]);      // the reduce warp requests the copies and tells the compute groups when they have read the tile
                 if (w.j == U.nt - 1) {
-                    // ---- end of the unit: dK and dV of this thread's key row.  bf16 rows staged in the unit's K / V
+                    // ---- end of the unit, before the tile's dQ (the next unit's MMAs wait for the accumulators): dK and dV of this
+                    // thread's key row.  bf16 rows staged in the unit's K / V
                     // buffer (every MMA of the unit is complete), one swizzled [128 x 64] tile per tensor, TMA stores;
                     // the load warp takes the buffer for the unit after the next once the stores have read it. ----
                     const int nrows = U.r1 - U.r0, kvb = w.uc & 1;
@@ -561,6 +548,27 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                         mbar_arrive(&kv_reuse[kvb]);
                     }
                 }
+                uint8_t *stg = sStg;
+                // fp32 staging: row = query, one swizzled [128 x 32] sub-tile per column half, a TMA reduce-add copy
+                // each (requested by the reduce warp).  Rows beyond the span's end hold exact zeros (their dS is zero).
+                if (t >= 1) HDT_WAIT(&stg_free[0], (t - 1) & 1, 20);      // the copies of tile t - 1 have read the staging area
+                if (!HDT_AGREE()) break;
+                tc_fence_after();
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {      // 32 columns per round of TMEM loads
+                    uint32_t r[32];
+                    tmem_ld32(tmem + TM_DQ + 64u * db + lane_base + 32u * half, r);
+                    tmem_wait_ld();
+                    if (half == 1) {          // the accumulator has been read: dQ of tile t + 2 may overwrite it
+                        tc_fence_before();
+                        mbar_arrive(&dq_free[db]);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 8; ++c)
+                        *reinterpret_cast<uint4 *>(stg + half * SUB + swz(rl, c)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
+                }
+                fence_proxy_async_smem();
+                mbar_arrive(&stg_full[0]);       // the reduce warp requests the copies
                 W_MARK(2, t, 2);
             }
         }
@@ -575,7 +583,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
 #undef HDT_AGREE
     tc_fence_before();
     __syncthreads();
-    if (blockIdx.x == 0 && tid < 80 && (a.phases == 86 || a.phases == 85)) g_bwd_w_marks[tid] = s_marks[tid];
+    if (blockIdx.x == 0 && tid < 80 && (a.phases == 86)) g_bwd_w_marks[tid] = s_marks[tid];
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
@@ -616,7 +624,7 @@ int read_bwd_w_tiles(long long *out512) {
 int launch_bwd_tc_onewalk64(const BwdStageArgs &a, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                             const CUtensorMap &tdo, const StoreMaps &outs, const CUtensorMap &tacc, int n_empty, cudaStream_t st) {
     constexpr int smem_max = 14 * SUB + 2 * 1024 + 256 + 640;
-    const int smem = smem_max - ((a.phases == 86 || a.phases == 85) ? 0 : 640);      // (the clock marks of an instrumented run)
+    const int smem = smem_max - (a.phases == 86 ? 0 : 640);      // (the clock marks of an instrumented run)
     static DevOnce attr;
     if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_w<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
