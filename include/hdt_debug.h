@@ -12,26 +12,45 @@ extern "C" {
 #endif
 
 /*
- * Library options (no counterpart in the paper).  "force_simt" = 1 routes bf16 stage-0 work
- * through the fp32 SIMT kernels instead of the tensor-core kernels; "no_persistent" = 1 uses only the
- * general tensor-core kernels, = 2 the persistent forward kernel, = 3 the forward kernel with one CTA
- * per (block, head), = 5 the looping backward kernel (the default at head_dim 128) at head_dim 64 too; "simt_upper" = 1 computes the stages above 0 of bf16 calls on the fp32 SIMT
- * kernels instead of the gathering tensor-core kernels; "no_overlap" = 1 runs the stages
- * above 0 after stage 0 on the caller's stream instead of beside it on an internal stream;
- * "no_graph" = 1 makes hdt_build_index launch its kernels one by one instead of replaying a cached
- * CUDA graph (A/B comparisons, tests).  "no_persistent" = 4 keeps the self-contained blocks of a
- * head_dim 64 backward on the persistent 512-thread kernel instead of the transposed looping one,
- * = 6 gives the latter one CTA per SM; "no_fused_delta" = 1 runs the delta pass even where every
- * backward kernel of the call could compute dO . O itself; "no_fold" bit 0 = 1 lets a merge
- * kernel complete the elements of stage 1 in the forward instead of the stage-1 kernel itself, bit 2
- * = 1 makes the backward's stage-1 kernel do it (off by default); "no_pdl" = 1 launches the kernels of hdt_build_index as ordinary stream
- * successors instead of programmatic dependents; "no_fwd_mc" = 1 keeps the blocks of a head_dim 64
- * forward that are not self-contained on the 128-thread general kernel instead of the 256-thread
- * multi-chunk one (and with it the EMPTY blocks of padded batches, which otherwise have a kernel of
- * their own, and the stages above 0 whose blocks are all self-contained, which otherwise run in the
- * single-chunk layout); "phase_stamps" = 1 selects the
- * instrumented instantiations of the looping forward and the transposed looping backward (see
- * hdt_debug_bwd_timeline), = 2 that of the multi-chunk forward (hdt_debug_fwd_phase_cycles).
+ * Library options (no counterpart in the paper).  Every option is 0 by default; an unknown name
+ * returns HDT_ERR_INVALID_ARG.  They exist for A/B comparisons and for tests that must reach a kernel the
+ * default routing would not choose; results agree with the oracle under every setting.
+ *
+ *   "force_simt"     1: bf16 stage-0 work runs on the fp32 SIMT kernels, not the tensor-core ones.
+ *   "simt_upper"     1: the stages above 0 of bf16 calls run on the fp32 SIMT kernels instead of the
+ *                    gathering tensor-core kernels.
+ *   "no_persistent"  1: only the general tensor-core kernels; 2: the persistent forward kernel;
+ *                    3: the forward kernel with one CTA per (block, head); 4: the self-contained
+ *                    blocks of a head_dim 64 backward stay on the persistent 512-thread kernel
+ *                    instead of the transposed looping one; 5: the looping backward kernel (the
+ *                    default at head_dim 128) at head_dim 64 too; 6: one CTA per SM for the
+ *                    transposed looping backward.
+ *   "no_fwd_mc"      1: the blocks of a head_dim 64 forward that are not self-contained stay on the
+ *                    128-thread general kernel instead of the 256-thread multi-chunk one (and with
+ *                    it the EMPTY blocks of padded batches, which otherwise have a kernel of their
+ *                    own, and the stages above 0 whose blocks are all self-contained, which
+ *                    otherwise run in the single-chunk layout).
+ *   "bwd_walk"       how a bf16 head_dim 64 backward treats the stage-0 blocks whose key range
+ *                    leaves the block.  0: one walk over each block's range by the warp-specialised
+ *                    kernel (dK and dV kept in tensor memory, dQ tiles summed in an fp32 buffer of
+ *                    the workspace by TMA reduce-add, then scaled and rounded by a finishing pass);
+ *                    1: two walks (one for dQ, one for dK and dV), no fp32 buffer; 2: the one walk
+ *                    in the lock-step form of the two-walk kernel; 86: as 0, with the clock marks
+ *                    that hdt_debug_bwd_w_marks and hdt_debug_bwd_w_tiles read back.
+ *   "no_fused_delta" 1: the delta pass (rowsum(dO . O)) runs even where every backward kernel of the
+ *                    call could compute it itself.
+ *   "no_fold"        bit 0: a merge kernel completes the elements of stage 1 in the forward instead
+ *                    of the stage-1 kernel itself; bit 2: the backward's stage-1 kernel does the
+ *                    completion (off by default).
+ *   "no_overlap"     1: the stages above 0 run after stage 0 on the caller's stream instead of
+ *                    beside it on an internal stream.
+ *   "no_graph"       1: hdt_build_index launches its kernels one by one instead of replaying a
+ *                    cached CUDA graph.
+ *   "no_pdl"         1: the kernels of hdt_build_index are ordinary stream successors instead of
+ *                    programmatic dependents.
+ *   "phase_stamps"   1: the instrumented instantiations of the looping forward and the transposed
+ *                    looping backward (see hdt_debug_bwd_timeline); 2: that of the multi-chunk
+ *                    forward (hdt_debug_fwd_phase_cycles).
  */
 int hdt_set_option(const char *name, int32_t value);
 
