@@ -19,7 +19,8 @@ extern "C" {
  *   "force_simt"     1: bf16 stage-0 work runs on the fp32 SIMT kernels, not the tensor-core ones.
  *   "simt_upper"     1: the stages above 0 of bf16 calls run on the fp32 SIMT kernels instead of the
  *                    gathering tensor-core kernels.
- *   "no_persistent"  1: only the general tensor-core kernels; 2: the persistent forward kernel;
+ *   "no_persistent"  1: only the general tensor-core kernels; 2: the persistent forward kernel (only
+ *                    in a library built with HDT_WORKBENCH defined; otherwise as 0);
  *                    3: the forward kernel with one CTA per (block, head); 4: the self-contained
  *                    blocks of a head_dim 64 backward stay on the persistent 512-thread kernel
  *                    instead of the transposed looping one; 5: the looping backward kernel (the
@@ -48,7 +49,8 @@ extern "C" {
  *                    cached CUDA graph.
  *   "no_pdl"         1: the kernels of hdt_build_index are ordinary stream successors instead of
  *                    programmatic dependents.
- *   "phase_stamps"   1: the instrumented instantiations of the looping forward and the transposed
+ *   "phase_stamps"   (only in a library built with HDT_WORKBENCH defined; otherwise ignored)
+ *                    1: the instrumented instantiations of the looping forward and the transposed
  *                    looping backward (see hdt_debug_bwd_timeline); 2: that of the multi-chunk
  *                    forward (hdt_debug_fwd_phase_cycles).
  */

@@ -14,6 +14,11 @@ NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--use_fast_math", "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v",
 ]
+# HDT_WORKBENCH=1 in the environment also compiles the instrumented instantiations (option
+# "phase_stamps") and the persistent forward kept for comparisons (option "no_persistent" = 2); a
+# default build leaves them out and those option values fall back to the default kernels.
+if os.environ.get("HDT_WORKBENCH", "0") not in ("", "0"):
+    NVCC_FLAGS.append("-DHDT_WORKBENCH")
 # --use_fast_math is limited to the intrinsics it maps (exp2f/log2f/division in the kernels are
 # already the approximate forms the tolerances were derived for); host code is unaffected.
 

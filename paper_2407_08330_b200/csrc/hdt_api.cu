@@ -331,7 +331,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
         // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
         // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
-        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3 && ix->directions == 7;
+        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3;
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 1;
         c.tok1 = ix->st[1].tok;
@@ -427,7 +427,7 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
     // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
     // tensor cores adds a bf16 rounding of P and dS to the elements it touches.
-    const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3 && ix->directions == 7;
+    const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && ix->n_stages <= 3;
     // No delta pass when every kernel of this call computes dO . O of its rows itself: stage 0
     // entirely on the looping kernels (the transposed one at head_dim 64, the fused five-MMA one at
     // head_dim 128; every block self-contained), the stages above it on the gathering tensor-core kernels.

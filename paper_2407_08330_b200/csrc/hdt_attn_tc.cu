@@ -763,6 +763,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc_loop(const __grid_constant__ CUt
 }
 
 // Cycle counts per phase of k_fwd_tc_p, accumulated by thread 0 of CTA 0 (diagnostics).
+#ifdef HDT_WORKBENCH      // (the persistent single-CTA-per-SM forward: kept for comparisons, option "no_persistent" = 2)
 #define HDT_STAMP(i)                                        \
     do {                                                    \
         if (stamp) {                                        \
@@ -1014,8 +1015,9 @@ __global__ void __launch_bounds__(512, 1) k_fwd_tc_p(const __grid_constant__ CUt
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
+#endif  // HDT_WORKBENCH
 
-// Diagnostics: cycles CTA 0 of the persistent forward spent per phase since the last call.
+// Diagnostics: cycles per phase since the last call; per-CTA timeline of the last instrumented launch.
 int read_fwd_timeline(long long *out4096) {
     HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out4096, g_fwd_timeline, sizeof(long long) * 4096));
     return HDT_OK;
@@ -1429,10 +1431,12 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_loop<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_1));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
+#ifdef HDT_WORKBENCH
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_p, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                             8 * SUB + 4 * 128 * 4 + 1024 + 64));
-        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc_mc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_mc));
+#endif
         attr.set();
     }
     const bool dirs = a.dirs != 7;   // direction bits: the instantiations that apply them
@@ -1454,13 +1458,16 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         b.rest_only = 1;
         n_general = a.nb - a.n_fused;
     } else if (a.n_fused > 0 && split_launch) {
+#ifdef HDT_WORKBENCH
         if (D == 64 && a.no_persistent == 2 && !dirs) {   // option: the persistent single-CTA-per-SM kernel
             constexpr int smem_p = 8 * SUB + 4 * 128 * 4 + 1024 + 64;
             int n_sm = 0;
             if (const int rc_ = sm_count(&n_sm)) return rc_;
             const long long items = (long long)a.n_fused * a.H;
             k_fwd_tc_p<<<(int)(items < n_sm ? items : n_sm), 512, smem_p, st>>>(tq, tk, tv, a);
-        } else if (a.no_persistent == 3 && !dirs) {       // option: one CTA per (block, head), no loop
+        } else
+#endif
+        if (a.no_persistent == 3 && !dirs) {       // option: one CTA per (block, head), no loop
             k_fwd_tc<D, true><<<dim3(a.n_fused, a.H), 128, smem_1, st>>>(tq, tk, tv, a);
         } else {
             int n_sm = 0;
@@ -1468,6 +1475,7 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
             const long long items = (long long)a.n_fused * a.H;
             const long long slots = (long long)n_sm * (D == 64 ? 4 : 2);
             if (dirs) k_fwd_tc_loop<D, true><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
+#ifdef HDT_WORKBENCH
             else if (g_phase_stamps == 1 && D == 64) {
                 static DevOnce attr_s;
                 if (!attr_s.done()) {
@@ -1475,7 +1483,9 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
                     attr_s.set();
                 }
                 k_fwd_tc_loop<64, false, true><<<(int)(items < slots ? items : slots), 128, 3 * SUB + 1024 + 64, st>>>(tq, tk, tv, om, a);
-            } else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
+            }
+#endif
+            else k_fwd_tc_loop<D><<<(int)(items < slots ? items : slots), 128, smem_1, st>>>(tq, tk, tv, om, a);
         }
         count_launch();
         HDT_CUDA_CHECK(cudaGetLastError());
@@ -1487,7 +1497,9 @@ static int launch_fwd_tc_t(const FwdStageArgs &a, cudaStream_t st) {
         dim3 grid(n_general, a.H);
         if (a.n_empty == n_general && !g_no_fwd_mc) k_fwd_empty<D><<<grid, 128, 0, st>>>(b);   // nothing but EMPTY blocks left
         else if (dirs) k_fwd_tc<D, false, false, true><<<grid, 128, smem, st>>>(tq, tk, tv, b);
+#ifdef HDT_WORKBENCH
         else if (D == 64 && !g_no_fwd_mc && g_phase_stamps == 2) k_fwd_tc_mc<true><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
+#endif
         else if (D == 64 && !g_no_fwd_mc) k_fwd_tc_mc<false><<<grid, 256, smem_mc, st>>>(tq, tk, tv, b);
         else k_fwd_tc<D, false><<<grid, 128, smem, st>>>(tq, tk, tv, b);
         count_launch();
@@ -1506,10 +1518,17 @@ static int launch_fwd_tc_upper_t(const FwdStageArgs &a, cudaStream_t st) {
     static DevOnce attr;
     if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_fwd_tc<D, false, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attr.set();
     }
     FwdStageArgs b = a;
     b.rest_only = 0;
+    if (a.dirs != 7) {      // direction bits: the general layout's instantiation that applies them
+        k_fwd_tc<D, false, true, true><<<dim3(a.nb, a.H), 128, smem, st>>>(tq, tq, tq, b);
+        count_launch();
+        HDT_CUDA_CHECK(cudaGetLastError());
+        return HDT_OK;
+    }
     // every block self-contained (keys = its own rows, one chunk): the single-chunk layout (P over the
     // Q / K tiles, O over S) needs 48 KB and 128 TMEM columns at D = 64, so four CTAs share an SM
     // instead of two and the stage runs in one wave

@@ -1397,11 +1397,13 @@ static int launch_bwd_tc_upper_t(const BwdStageArgs &a, cudaStream_t st) {
     static DevOnce attr;
     if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc<D, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attr.set();
     }
     BwdStageArgs b = a;
     b.rest_only = 0;
-    k_bwd_tc<D, true><<<dim3(a.nb, a.H), 256, smem, st>>>(tq, tq, tq, tq, b);
+    if (a.dirs != 7) k_bwd_tc<D, true, true><<<dim3(a.nb, a.H), 256, smem, st>>>(tq, tq, tq, tq, b);      // direction bits
+    else k_bwd_tc<D, true><<<dim3(a.nb, a.H), 256, smem, st>>>(tq, tq, tq, tq, b);
     count_launch();
     HDT_CUDA_CHECK(cudaGetLastError());
     return HDT_OK;

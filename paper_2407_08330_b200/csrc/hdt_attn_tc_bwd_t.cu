@@ -371,8 +371,11 @@ int launch_bwd_tc_fused64(const BwdStageArgs &a, const CUtensorMap &tq, const CU
     if (const int rc_ = sm_count(&n_sm)) return rc_;
     if (!attr.done()) {
         const void *fns[6] = {(const void *)k_bwd_tc_t<false>,       (const void *)k_bwd_tc_t<true>,
-                              (const void *)k_bwd_tc_t<false, true>, (const void *)k_bwd_tc_t<false, false, true>,
-                              (const void *)k_bwd_tc_t<false, true, true>, nullptr};
+                              (const void *)k_bwd_tc_t<false, false, true>,
+#ifdef HDT_WORKBENCH      // the instrumented instantiations (option "phase_stamps" = 1)
+                              (const void *)k_bwd_tc_t<false, true>, (const void *)k_bwd_tc_t<false, true, true>,
+#endif
+                              nullptr};
         for (int i = 0; fns[i]; ++i) {
             HDT_CUDA_CHECK(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
             HDT_CUDA_CHECK(cudaFuncSetAttribute(fns[i], cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
@@ -386,10 +389,13 @@ int launch_bwd_tc_fused64(const BwdStageArgs &a, const CUtensorMap &tq, const CU
         return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_fused64: the fused-delta kernel needs o and the full rule");
     const long long slots = (a.no_persistent == 6 ? 1LL : 2LL) * n_sm;
     const int grid = (int)(items < slots ? items : slots);
+#ifdef HDT_WORKBENCH
     if (g_phase_stamps == 1 && a.dirs == 7) {
         if (fd) k_bwd_tc_t<false, true, true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
         else k_bwd_tc_t<false, true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
-    } else if (a.dirs != 7) k_bwd_tc_t<true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
+    } else
+#endif
+    if (a.dirs != 7) k_bwd_tc_t<true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
     else if (fd) k_bwd_tc_t<false, false, true><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
     else k_bwd_tc_t<false><<<grid, 256, smem, st>>>(tq, tk, tv, tdo, outs, a);
     count_launch();

@@ -25,8 +25,30 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
+// A tensor map is a function of (address, extents, box) only, and a training loop comes back with the
+// same tensors step after step: each host thread keeps the maps it made in a small direct-mapped
+// table (a call of the attention makes some thirty of them).
+struct TmapEntry {
+    alignas(64) CUtensorMap map;
+    const void *base;
+    long long T;
+    int D, H, box_rows, kind;      // kind: 1 = bf16 [T, H, D], 2 = fp32 accumulation buffer; 0 = empty
+};
+inline TmapEntry *tmap_slot(const void *base, int D, int H, long long T, int box_rows, int kind, bool *hit) {
+    static thread_local TmapEntry table[128];
+    const uintptr_t a = (uintptr_t)base;
+    const unsigned h = (unsigned)((a >> 8) * 0x9E3779B1u) ^ ((unsigned)box_rows * 0x85EBCA6Bu) ^ ((unsigned)kind << 5) ^ (unsigned)D;
+    TmapEntry *e = &table[(h ^ (h >> 15)) & 127u];
+    *hit = e->kind == kind && e->base == base && e->T == T && e->D == D && e->H == H && e->box_rows == box_rows;
+    return e;
+}
+
 // base: device pointer, 16-byte aligned; D: inner extent (elements, D * 2 bytes a multiple of 16).
 inline int make_tmap_bf16(CUtensorMap *tm, const void *base, int D, int H, long long T, int box_rows) {
+    bool hit = false;
+    TmapEntry *slot = tmap_slot(base, D, H, T, box_rows, 1, &hit);
+    if (hit) { *tm = slot->map; return HDT_OK; }
+    const int rc = [&]() -> int {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return set_error(HDT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
     cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)(T > 0 ? T : 1)};
@@ -38,6 +60,9 @@ inline int make_tmap_bf16(CUtensorMap *tm, const void *base, int D, int H, long 
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return set_error(HDT_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
     return HDT_OK;
+    }();
+    if (rc == HDT_OK) { slot->map = *tm; slot->base = base; slot->T = T; slot->D = D; slot->H = H; slot->box_rows = box_rows; slot->kind = 1; }
+    return rc;
 }
 
 // fp32 accumulation buffer [T, H, 64] for reduce-add copies: box = (32 floats, 1, box_rows), i.e.
