@@ -912,10 +912,13 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         ProfScope ps(PROF_INDEX, st);
         // The build is a dozen tiny kernels: launching them one by one is slower than running them.
         // They are captured once into a CUDA graph, which is replayed while the same buffers, sizes
-        // and parameters come back (one cached graph per host thread).
+        // and parameters come back (a few cached graphs per host thread).
         struct GraphKey { const void *a, *b, *c, *w; int B, T, bm, ms, bmu, ov, dirs, pad; };   // no padding bytes: compared with memcmp
-        struct GraphCache { GraphKey key; cudaGraphExec_t exec; int launches; bool valid; };
-        static thread_local GraphCache cache{};
+        struct GraphCache { GraphKey key; cudaGraphExec_t exec; int launches; bool valid; unsigned long long used; };
+        // (a few entries, least recently used replaced: a loop that alternates between buffer sets replays instead of capturing again)
+        constexpr int kGraphs = 4;
+        static thread_local GraphCache cache[kGraphs]{};
+        static thread_local unsigned long long tick = 0;
         const GraphKey key{level, parent, cu_seqlens, workspace, B, T, bm, ms, bmu, sd ? 1 : 0, dirs, 0};
         static_assert(sizeof(GraphKey) == 4 * sizeof(void *) + 8 * sizeof(int), "GraphKey must not contain padding");
         bool done = false;
@@ -924,16 +927,22 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         const bool capturable = st != nullptr && st != cudaStreamLegacy && st != cudaStreamPerThread;
         if (!g_no_graph && capturable && cudaStreamIsCapturing(st, &cap) == cudaSuccess &&
             cap == cudaStreamCaptureStatusNone) {
-            if (cache.valid && std::memcmp(&cache.key, &key, sizeof(key)) == 0) {
-                if (cudaGraphLaunch(cache.exec, st) == cudaSuccess) { done = true; count_launch(cache.launches); }
+            GraphCache *hit = nullptr, *victim = &cache[0];
+            for (int i = 0; i < kGraphs; ++i) {
+                if (cache[i].valid && std::memcmp(&cache[i].key, &key, sizeof(key)) == 0) hit = &cache[i];
+                if (!cache[i].valid || (victim->valid && cache[i].used < victim->used)) victim = &cache[i];
+            }
+            if (hit) {
+                hit->used = ++tick;
+                if (cudaGraphLaunch(hit->exec, st) == cudaSuccess) { done = true; count_launch(hit->launches); }
             } else if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
                 const cudaError_t e = enqueue_all();
                 cudaGraph_t g = nullptr;
                 const cudaError_t e2 = cudaStreamEndCapture(st, &g);
                 cudaGraphExec_t exec = nullptr;
                 if (e == cudaSuccess && e2 == cudaSuccess && g && cudaGraphInstantiate(&exec, g, 0) == cudaSuccess) {
-                    if (cache.valid) cudaGraphExecDestroy(cache.exec);
-                    cache = GraphCache{key, exec, n_launched, true};
+                    if (victim->valid) cudaGraphExecDestroy(victim->exec);
+                    *victim = GraphCache{key, exec, n_launched, true, ++tick};
                     if (cudaGraphLaunch(exec, st) == cudaSuccess) { done = true; count_launch(n_launched); }
                 }
                 if (g) cudaGraphDestroy(g);

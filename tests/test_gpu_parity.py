@@ -86,6 +86,30 @@ def test_index_graph_replay_with_new_contents(P):
             P.hdt_set_option("no_graph", 0)
 
 
+def test_index_graph_cache_with_alternating_buffer_sets(P):
+    """Six buffer sets (structure arrays and workspace of their own) visited round-robin three times:
+    the build's graph cache holds fewer entries than that, so graphs are replayed, replaced and
+    captured again, and every build must still equal the oracle's index."""
+    rng = np.random.default_rng(5)
+    sets = []
+    for i in range(6):
+        b = gen.pack([gen.gen_fill(rng, 500 + 40 * i, (2, 5), (2, 8), (3, 25)) for _ in range(2)])
+        ws = torch.empty(P.hdt_index_workspace_bytes(2, b.total_tokens, 0, 4), dtype=torch.uint8, device="cuda")
+        sets.append((b, dev_struct(b), ws, ix.build(b.level, b.parent, b.cu_seqlens, 128)))
+    with torch.cuda.stream(torch.cuda.Stream()):
+        for order in (range(6), (0, 1, 0, 1, 2, 3), reversed(range(6))):
+            for i in order:
+                b, (lv, pa, cu), ws, want = sets[i]
+                idx = P.hdt_build_index(lv, pa, cu, max_stages=4, workspace=ws)
+                assert idx.nnz == want.nnz and idx.n_stages == len(want.stages)
+                for s_, st in enumerate(want.stages):
+                    got = idx.export(s_)
+                    for name in ("rng", "up", "blocks", "queue", "queue_split"):
+                        assert np.array_equal(got[name], getattr(st, name)), (i, s_, name)
+        torch.cuda.current_stream().synchronize()
+    P.hdt_device_status()
+
+
 def test_index_many_sequences(P):
     """More sequences than the single-CTA upper-stage builder takes: the per-stage kernels run."""
     rng = np.random.default_rng(12)
