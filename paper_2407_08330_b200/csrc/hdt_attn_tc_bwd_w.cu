@@ -81,7 +81,7 @@ __device__ long long g_bwd_w_marks[128];
 __device__ long long g_bwd_w_tiles[512];      // (instrumented run) CTA 0: SM clock at the MMA warp's loop top of every tile, unit number in the low 8 bits
 #define W_MARK(role, tt, id)                                                                    \
     do {                                                                                        \
-        if (marks && (tt) >= 4 && (tt) < 6) {                                                 \
+        if (MARKS && marks && (tt) >= 4 && (tt) < 6) {                                        \
             const long long now_ = clock64();                                                   \
             if (lane == 0) s_marks[(role) * 16 + ((tt) - 4) * 8 + (id)] = now_;                \
         }                                                                                       \
@@ -94,7 +94,8 @@ struct WUnit { int valid, r0, r1, ka, kb, h, nt; };
 struct Walk { int k, j, t, uc, valid, qs, qph; WUnit U, N; };
 }  // namespace
 
-template <bool DIRS>
+// MARKS: the instantiation that leaves the clock marks and the tile log (option "bwd_walk" = 86).
+template <bool DIRS, bool MARKS = false>
 __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUtensorMap tm_q,
                                                      const __grid_constant__ CUtensorMap tm_k,
                                                      const __grid_constant__ CUtensorMap tm_v,
@@ -121,8 +122,8 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int H = a.H, G = gridDim.x;
     const float LOG2E = 1.4426950408889634f;
-    const bool marks = (a.phases == 86) && blockIdx.x == 0 && (warp == 0 || warp == 8 || warp == W_DRAIN || warp >= W_LOAD);
-    if ((a.phases == 86) && tid < 80) s_marks[tid] = 0;
+    const bool marks = MARKS && blockIdx.x == 0 && (warp == 0 || warp == 8 || warp == W_DRAIN || warp >= W_LOAD);
+    if (MARKS && tid < 80) s_marks[tid] = 0;
     // EMPTY blocks cost nothing in the queue's order, so they are the tail of queue_split and are left
     // out here (k_bwd_zero_empty writes their rows)
     const int n_units = (a.nb - a.n_fused - a.n_empty) * H;
@@ -320,8 +321,17 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 for (int kk = 0; kk < 8; ++kk)
                     mma_ss_w(tmem + TM_DQ + 64u * dsb, d_lo + 128 * kk, dsm_hi, k_lo + 128 * kk, kvm_hi, id_q, kk > 0);
             };
-            Walk w = begin();
-            if (w.valid) {      // S^T, dP^T of both steps of the first tile
+            // (a walk of its own with the little this warp needs: tiles per unit, requested a unit ahead; the ring
+            // stage and its parity follow from the tile count.  Every instruction here is on the kernel's
+            // critical chain: the warp shares its scheduler with five others.)
+            auto unit_nt = [&](int k) {
+                const int i = (int)blockIdx.x + k * G;
+                if (i >= n_units) return 0;
+                const int *rec = a.blocks + 5 * (size_t)a.queue_split[a.n_fused + i / H];
+                return (rec[3] - rec[2] + 127) >> 7;      // (>= 1: EMPTY blocks are not among these units)
+            };
+            int nt = unit_nt(0), nt_n = unit_nt(1), k = 2, j = 0, t = 0, uc = 0;
+            if (nt > 0) {      // S^T, dP^T of both steps of the first tile
                 HDT_WAIT(&kv_full[0], 0, 3);
                 HDT_WAIT(&qdo_full[0], 0, 4);
                 if (HDT_AGREE() && elect_one()) {
@@ -331,25 +341,22 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 }
                 __syncwarp();
             }
-            while (w.valid && ok) {
-                // the next tile, without walking there: same unit or the next one (units here are never EMPTY)
-                const int t = w.t, db = t & 1;
-                const bool first = w.j == 0, last = w.j == w.U.nt - 1;
-                struct { int valid, qs, qph, uc; } n;
-                n.valid = !last || w.N.valid;
-                n.qs = w.qs ^ 1;
-                n.qph = w.qs == 1 ? (w.qph ^ 1) : w.qph;
-                n.uc = w.uc + (last ? 1 : 0);
-                const int kvb = w.uc & 1;
+            while (nt > 0 && ok) {
+                // the next tile: same unit or the next one (units here are never EMPTY)
+                const int db = t & 1, qs = t & 1, n_qs = qs ^ 1;
+                const bool first = j == 0, last = j == nt - 1;
+                const bool n_valid = !last || nt_n > 0;
+                const int n_qph = ((t + 1) >> 1) & 1, n_uc = uc + (last ? 1 : 0);
+                const int kvb = uc & 1;
                 const uint32_t acc = first ? 0u : 1u;
                 // ---- step a: dV; S^T, dP^T of the next tile's step a; dK ----
                 W_MARK(4, t, 0);
-                if ((a.phases == 86) && blockIdx.x == 0 && lane == 0 && t < 512) g_bwd_w_tiles[t] = (clock64() << 8) | (long long)(w.uc & 255);
+                if (MARKS && blockIdx.x == 0 && lane == 0 && t < 512) g_bwd_w_tiles[t] = (clock64() << 8) | (long long)(uc & 255);
                 // (what is normally there already first, the wait for the compute group last: it ends the chain)
-                if (first && w.uc >= 1) HDT_WAIT(acc_free, (w.uc - 1) & 1, 6);      // the previous unit's dK, dV have been read
-                if (n.valid) {
-                    HDT_WAIT(&qdo_full[n.qs], n.qph, 7);
-                    if (last) HDT_WAIT(&kv_full[n.uc & 1], (n.uc >> 1) & 1, 8);      // the next tile opens a unit (the other K / V buffer)
+                if (first && uc >= 1) HDT_WAIT(acc_free, (uc - 1) & 1, 6);      // the previous unit's dK, dV have been read
+                if (n_valid) {
+                    HDT_WAIT(&qdo_full[n_qs], n_qph, 7);
+                    if (last) HDT_WAIT(&kv_full[n_uc & 1], (n_uc >> 1) & 1, 8);      // the next tile opens a unit (the other K / V buffer)
                 }
                 W_MARK(4, t, 1);
                 HDT_WAIT(&pds_ready[0], t & 1, 5);
@@ -357,9 +364,9 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 W_MARK(4, t, 2);
                 if (elect_one()) {
                     tc_fence_after();
-                    issue_dv(0, w.qs, acc);
-                    if (n.valid) issue_sdp(0, n.qs, n.uc & 1);
-                    issue_dk(0, w.qs, db, acc);
+                    issue_dv(0, qs, acc);
+                    if (n_valid) issue_sdp(0, n_qs, n_uc & 1);
+                    issue_dk(0, qs, db, acc);
                 }
                 __syncwarp();
                 W_MARK(4, t, 3);
@@ -371,10 +378,10 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 W_MARK(4, t, 5);
                 if (elect_one()) {
                     tc_fence_after();
-                    issue_dv(1, w.qs, 1u);
-                    if (n.valid) issue_sdp(1, n.qs, n.uc & 1);
-                    issue_dk(1, w.qs, db, 1u);
-                    mma_commit(&qdo_empty[w.qs]);        // every MMA that reads this tile's Q / dO has been issued
+                    issue_dv(1, qs, 1u);
+                    if (n_valid) issue_sdp(1, n_qs, n_uc & 1);
+                    issue_dk(1, qs, db, 1u);
+                    mma_commit(&qdo_empty[qs]);        // every MMA that reads this tile's Q / dO has been issued
                     if (last) mma_commit(acc_full);
                     issue_dq(db, kvb);
                     mma_commit(&dq_full[db]);
@@ -382,7 +389,9 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 }
                 __syncwarp();
                 W_MARK(4, t, 6);
-                step(w);
+                ++t;
+                if (!last) ++j;
+                else { nt = nt_n; nt_n = unit_nt(k++); j = 0; ++uc; }
             }
         } else if (warp < W_DRAIN) {
             // ================= compute groups: x = 0 (warps 0-7) step a, x = 1 (warps 8-15) step b;
@@ -583,7 +592,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
 #undef HDT_AGREE
     tc_fence_before();
     __syncthreads();
-    if (blockIdx.x == 0 && tid < 80 && (a.phases == 86)) g_bwd_w_marks[tid] = s_marks[tid];
+    if (MARKS && blockIdx.x == 0 && tid < 80) g_bwd_w_marks[tid] = s_marks[tid];
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
@@ -624,11 +633,12 @@ int read_bwd_w_tiles(long long *out512) {
 int launch_bwd_tc_onewalk64(const BwdStageArgs &a, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv,
                             const CUtensorMap &tdo, const StoreMaps &outs, const CUtensorMap &tacc, int n_empty, cudaStream_t st) {
     constexpr int smem_max = 14 * SUB + 2 * 1024 + 256 + 640;
-    const int smem = smem_max - (a.phases == 86 ? 0 : 640);      // (the clock marks of an instrumented run)
+    const int smem = smem_max - ((a.phases == 86 && a.dirs == 7) ? 0 : 640);      // (the clock marks of an instrumented run)
     static DevOnce attr;
     if (!attr.done()) {
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_w<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
         HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_w<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
+        HDT_CUDA_CHECK(cudaFuncSetAttribute(k_bwd_tc_w<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_max));
         attr.set();
     }
     int n_sm = 0;
@@ -639,7 +649,8 @@ int launch_bwd_tc_onewalk64(const BwdStageArgs &a, const CUtensorMap &tq, const 
         return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_onewalk64: needs delta, the fp32 dQ buffer and the number of EMPTY blocks");
     const long long units = (long long)n_rest * a.H;
     const int grid = (int)(units < n_sm ? units : n_sm);
-    if (a.dirs != 7) k_bwd_tc_w<true><<<grid, 736, smem, st>>>(tq, tk, tv, tdo, outs, tacc, a);
+    if (a.phases == 86 && a.dirs == 7) k_bwd_tc_w<false, true><<<grid, 736, smem, st>>>(tq, tk, tv, tdo, outs, tacc, a);
+    else if (a.dirs != 7) k_bwd_tc_w<true><<<grid, 736, smem, st>>>(tq, tk, tv, tdo, outs, tacc, a);
     else k_bwd_tc_w<false><<<grid, 736, smem, st>>>(tq, tk, tv, tdo, outs, tacc, a);
     count_launch();
     HDT_CUDA_CHECK(cudaGetLastError());
