@@ -1323,7 +1323,9 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
                 // the warp-specialised one-walk kernel (hdt_attn_tc_bwd_w.cu), then the sums become dQ rows
                 rc = launch_bwd_tc_onewalk64(c, tq, tk, tv, tdo, outs, tacc, a.n_empty, st);
                 if (rc) return rc;
-                k_dq_finish<<<dim3(a.nb - a.n_fused, a.H), 256, 0, st>>>(c);
+                BwdStageArgs f = c;
+                f.scale = 1.f;      // (this kernel's sums carry softmax_scale already: it is in dS)
+                k_dq_finish<<<dim3(a.nb - a.n_fused, a.H), 256, 0, st>>>(f);
             } else if (mode && onewalk) {
                 if (dirs) k_bwd_tc_p<2, true><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);
                 else k_bwd_tc_p<2><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);

@@ -6,7 +6,8 @@
 // every query that attends one of its keys — in query tiles of 128 rows, each in two steps of 64
 // queries.  With the keys in the TMEM lanes (the transposed pass of hdt_attn_tc_bwd_t.cu):
 //   MMA      S^T = K Q^T, dP^T = V dO^T for the step's 64 queries            -> TMEM (lane = key)
-//   compute  P^T = exp2(S^T c - LSE[query]) inside the key's range, dS^T = P^T o (dP^T - delta[query]);
+//   compute  P^T = exp2(S^T c - LSE[query]) inside the key's range, dS^T = softmax_scale P^T o (dP^T - delta[query])
+//            (the factor here, in the fma that subtracts delta, so that dK and dQ need none afterwards);
 //            P^T (bf16) stays in TMEM over the S^T columns it came from, dS^T -> shared memory
 //   MMA      dV += P^T dO (A operand from TMEM), dK += dS^T Q: accumulated in TMEM over the whole walk;
 //            after both steps dQ_tile = dS K (M = the tile's 128 queries, A = dS^T read MN-major), a
@@ -36,6 +37,14 @@
 //    S^T columns) and the next S^T / dP^T; dK and dQ, which read dS^T from shared memory, are issued
 //    behind them.  With four warps per compute group a step's arithmetic (64 entries per thread) took
 //    3500 cycles, one instruction issued in eight cycles per warp: the groups have eight warps each.
+//  - the warps of an SM quarter share one instruction issue slot a cycle, and the sixteen compute warps fill most
+//    of them: the MMA warp gets an instruction out every five or six cycles, so its waits, its walk and the
+//    forty MMAs of a tile are a chain of 3500 cycles by themselves.  It walks tile counts only (ring stage and
+//    parity from the tile number), the compute warps a record of four integers; that took the scope on config 5
+//    from 0.625 to 0.589 ms together with: the drain group reads dV before dK at a unit's end and frees each with
+//    a barrier of its own, so that dV and the next S^T / dP^T are issued while dK is still being read.
+//    Tried and not kept: two MMA warps taking turns, the Q / dO ring in half tiles, the loop unrolled by tile
+//    parity (more spills), sleeping between barrier tests in the other warps.
 //  - units end often (4.7 tiles per unit on config 5): one K / V buffer cost 13000 cycles per unit
 //    (the pipeline drains and refills around the reload), draining dK / dV by the compute groups with
 //    plain stores 7000 (32 rows per store instruction); with the second buffer, the drain group taking
@@ -114,8 +123,9 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     uint64_t *bars = (uint64_t *)(sStat + 2 * 128);
     uint64_t *qdo_full = bars, *qdo_empty = bars + 3, *sdp_full = bars + 6, *pds_ready = bars + 8;
     uint64_t *dq_full = bars + 10, *dq_free = bars + 12, *kv_full = bars + 14, *kv_empty = bars + 16;
-    uint64_t *acc_full = bars + 18, *acc_free = bars + 19, *stat_full = bars + 20, *stg_free = bars + 22, *stg_full = bars + 24, *kv_reuse = bars + 26;
-    uint32_t *slot = (uint32_t *)(bars + 28);
+    uint64_t *acc_full = bars + 18, *dv_free = bars + 19, *stat_full = bars + 20, *stg_free = bars + 22, *stg_full = bars + 24, *kv_reuse = bars + 26;
+    uint64_t *dk_free = bars + 28;
+    uint32_t *slot = (uint32_t *)(bars + 29);
     volatile int *abort_flag = (volatile int *)(slot + 1);
     long long *s_marks = (long long *)(bars + 30);      // [5 roles][2 tiles][8 marks] of the instrumented run (only then allocated)
 
@@ -152,7 +162,8 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
             mbar_init(&kv_reuse[i], 1);
         }
         mbar_init(acc_full, 1);
-        mbar_init(acc_free, 128);
+        mbar_init(dv_free, 128);
+        mbar_init(dk_free, 128);
         *abort_flag = (*a.status != 0);
         fence_mbar_init();
     }
@@ -226,7 +237,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 for (int i = 0; i < 4; ++i) {
                     const int row = q0 + lane + 32 * i;
                     st4[i] = make_float2(0.f, 0.f);
-                    if (row < U.kb) st4[i] = make_float2(a.lse[(size_t)U.h * a.T + row] * LOG2E, a.delta[(size_t)U.h * a.T + row]);
+                    if (row < U.kb) st4[i] = make_float2(a.lse[(size_t)U.h * a.T + row] * LOG2E, a.delta[(size_t)U.h * a.T + row] * a.scale);
                 }
                 W_MARK(3, w.t, 0);
                 if (w.j == 0) {      // the unit's K, V into the buffer the unit before the last one has left
@@ -353,7 +364,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 W_MARK(4, t, 0);
                 if (MARKS && blockIdx.x == 0 && lane == 0 && t < 512) g_bwd_w_tiles[t] = (clock64() << 8) | (long long)(uc & 255);
                 // (what is normally there already first, the wait for the compute group last: it ends the chain)
-                if (first && uc >= 1) HDT_WAIT(acc_free, (uc - 1) & 1, 6);      // the previous unit's dK, dV have been read
+                if (first && uc >= 1) HDT_WAIT(dv_free, (uc - 1) & 1, 6);      // the previous unit's dV has been read (dK: below)
                 if (n_valid) {
                     HDT_WAIT(&qdo_full[n_qs], n_qph, 7);
                     if (last) HDT_WAIT(&kv_full[n_uc & 1], (n_uc >> 1) & 1, 8);      // the next tile opens a unit (the other K / V buffer)
@@ -366,9 +377,17 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                     tc_fence_after();
                     issue_dv(0, qs, acc);
                     if (n_valid) issue_sdp(0, n_qs, n_uc & 1);
-                    issue_dk(0, qs, db, acc);
+                    if (!(first && uc >= 1)) issue_dk(0, qs, db, acc);
                 }
                 __syncwarp();
+                if (first && uc >= 1) {
+                    // (the drain group reads dV first: dV and the next S^T / dP^T, which the compute group waits for, have
+                    // gone ahead while it still reads the previous unit's dK)
+                    HDT_WAIT(dk_free, (uc - 1) & 1, 24);
+                    if (!HDT_AGREE()) break;
+                    if (elect_one()) issue_dk(0, qs, db, acc);
+                    __syncwarp();
+                }
                 W_MARK(4, t, 3);
                 // ---- step b: dV; S^T, dP^T of the next tile's step b; dK; the tile's dQ ----
                 if (t >= 2) HDT_WAIT(&dq_free[db], ((t >> 1) + 1) & 1, 10);
@@ -398,27 +417,33 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
             // a warp: TMEM lane quarter warp % 4, queries 32 qh .. 32 qh + 31 of the step =================
             const int x = warp >> 3, qh = (warp >> 2) & 1, kl = (warp & 3) * 32 + lane;
             const uint32_t tm_s = tmem + 128u * x + 32u * qh + lane_base, tm_dp = tm_s + 64u;
-            int lo = 0, hi = 0, row = 0, lo_n = 0, hi_n = 0, r0_n = -1;      // *_n: the range of this lane's key row in the block that starts at r0_n
-            bool inb = false;
-            auto fetch_range = [&](const WUnit &u) {
-                const int r = u.r0 + kl;
-                r0_n = u.r0; lo_n = 0; hi_n = 0;
-                if (r < u.r1) { lo_n = a.rng[2 * r]; hi_n = a.rng[2 * r + 1]; }
-            };
-            Walk w = begin();
-            if (w.valid) fetch_range(w.U);
-            for (; w.valid && ok; step(w)) {
-                const WUnit &U = w.U;
-                if (w.j == 0) {
-                    if (r0_n != U.r0) fetch_range(U);      // (only when a unit was skipped in between)
-                    row = U.r0 + kl;
-                    inb = row < U.r1;
-                    lo = lo_n; hi = hi_n;
+            // (a walk of its own with what a compute warp needs: the unit's rows and span, this lane's key range;
+            // the next unit's are requested a unit ahead, at the unit's second tile)
+            struct CU { int r0, r1, ka, kb; };
+            auto unit_rec = [&](int k) {
+                CU u{0, 0, 0, 0};      // (kb == ka: no such unit)
+                const int i = (int)blockIdx.x + k * G;
+                if (i < n_units) {
+                    const int *rec = a.blocks + 5 * (size_t)a.queue_split[a.n_fused + i / H];
+                    u.r0 = rec[0]; u.r1 = rec[1]; u.ka = rec[2]; u.kb = rec[3];
                 }
-                // the next unit's range a unit ahead (its record, requested at this unit's start, has arrived by the second tile)
-                if (w.j == min(1, U.nt - 1) && w.N.valid) fetch_range(w.N);
-                const int t = w.t, db = t & 1;
-                const int q0 = U.ka + 128 * w.j, nq = min(128, U.kb - q0);
+                return u;
+            };
+            auto range_of = [&](const CU &u, int &lo_, int &hi_) {
+                const int r = u.r0 + kl;
+                lo_ = 0; hi_ = 0;
+                if (u.kb > u.ka && r < u.r1) { lo_ = a.rng[2 * r]; hi_ = a.rng[2 * r + 1]; }
+            };
+            CU U = unit_rec(0), N = unit_rec(1);
+            int k = 2, j = 0, t = 0, lo, hi, lo_n = 0, hi_n = 0;
+            range_of(U, lo, hi);
+            while (U.kb > U.ka && ok) {
+                const int nt = (U.kb - U.ka + 127) >> 7;
+                const int row = U.r0 + kl;
+                const bool inb = row < U.r1;
+                if (j == min(1, nt - 1)) range_of(N, lo_n, hi_n);
+                const int db = t & 1;
+                const int q0 = U.ka + 128 * j, nq = min(128, U.kb - q0);
                 // this key row over the tile's queries: the queries that attend it are its own family range
                 const int jl = max(lo - q0, 0), jh = min(hi - q0, nq);
                 const bool has = inb && jh > jl;
@@ -461,7 +486,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                             const float p0 = exp2f(fmaf(__uint_as_float(s_[j]), a.scale_log2, -st.x));
                             const float p1 = exp2f(fmaf(__uint_as_float(s_[j + 1]), a.scale_log2, -st.z));
                             pp[j >> 1] = pack_bf16(p0, p1);
-                            pd[j >> 1] = pack_bf16(p0 * (__uint_as_float(d_[j]) - st.y), p1 * (__uint_as_float(d_[j + 1]) - st.w));
+                            pd[j >> 1] = pack_bf16(p0 * fmaf(__uint_as_float(d_[j]), a.scale, -st.y), p1 * fmaf(__uint_as_float(d_[j + 1]), a.scale, -st.w));
                         }
                     } else if (any[i] && km[i] != 0u) {
 #pragma unroll
@@ -470,11 +495,11 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                             float p0 = 0.f, p1 = 0.f, e0 = 0.f, e1 = 0.f;
                             if (km[i] & (1u << j)) {
                                 p0 = exp2f(fmaf(__uint_as_float(s_[j]), a.scale_log2, -st.x));
-                                e0 = p0 * (__uint_as_float(d_[j]) - st.y);
+                                e0 = p0 * fmaf(__uint_as_float(d_[j]), a.scale, -st.y);
                             }
                             if (km[i] & (2u << j)) {
                                 p1 = exp2f(fmaf(__uint_as_float(s_[j + 1]), a.scale_log2, -st.z));
-                                e1 = p1 * (__uint_as_float(d_[j + 1]) - st.w);
+                                e1 = p1 * fmaf(__uint_as_float(d_[j + 1]), a.scale, -st.w);
                             }
                             pp[j >> 1] = pack_bf16(p0, p1);
                             pd[j >> 1] = pack_bf16(e0, e1);
@@ -490,6 +515,9 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 tc_fence_before();
                 mbar_arrive(&pds_ready[x]);
                 W_MARK(x, t, 3);
+                ++t;
+                if (j + 1 < nt) ++j;
+                else { U = N; N = unit_rec(k++); lo = lo_n; hi = hi_n; j = 0; }
             }
         } else if (warp < W_LOAD) {
             // ================= drain group: the dQ tile of every tile pair, added to the fp32 buffer =================
@@ -515,31 +543,32 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                     HDT_WAIT(acc_full, w.uc & 1, 15);
                     if (HDT_AGREE()) {
                         tc_fence_after();
-#pragma unroll
-                        for (int pc = 0; pc < 4; ++pc) {      // dK columns 0..31, 32..63, then dV
-                            const int tt = pc >> 1, c0 = 32 * (pc & 1);
+                        // dV first (the next unit's MMAs need its accumulator first), then dK; 32 columns a round.
+                        // (no factor: the compute warps put softmax_scale into dS)
+                        auto round = [&](uint32_t tm_acc, float *part, uint8_t *stage, int c0, uint64_t *read_bar) {
                             uint32_t r[32];
-                            tmem_ld32(tmem + (tt ? TM_DV : TM_DK) + lane_base + c0, r);
+                            tmem_ld32(tm_acc + lane_base + c0, r);
                             tmem_wait_ld();
-                            if (pc == 3) {        // both accumulators have been read: the next unit may overwrite them
+                            if (read_bar != nullptr) {      // the accumulator has been read: the next unit may overwrite it
                                 tc_fence_before();
-                                mbar_arrive(acc_free);
+                                mbar_arrive(read_bar);
                             }
-                            const float sc = tt ? 1.f : a.scale;
 #pragma unroll
                             for (int j = 0; j < 32; j += 8) {
-                                float v[8];
-#pragma unroll
-                                for (int e = 0; e < 8; ++e) v[e] = __uint_as_float(r[j + e]) * sc;
                                 if (up >= 0) {      // this row lives on in the next stage: its fp32 gradients go there too
-                                    float4 *pt = reinterpret_cast<float4 *>((tt ? a.part_dv : a.part_dk) + ((size_t)up * H + U.h) * D + c0 + j);
-                                    pt[0] = make_float4(v[0], v[1], v[2], v[3]);
-                                    pt[1] = make_float4(v[4], v[5], v[6], v[7]);
+                                    float4 *pt = reinterpret_cast<float4 *>(part + ((size_t)up * H + U.h) * D + c0 + j);
+                                    pt[0] = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                                    pt[1] = make_float4(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]), __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
                                 }
-                                *reinterpret_cast<uint4 *>(skv + tt * SUB + swz(rl, (c0 + j) >> 3)) =
-                                    make_uint4(pack_bf16(v[0], v[1]), pack_bf16(v[2], v[3]), pack_bf16(v[4], v[5]), pack_bf16(v[6], v[7]));
+                                *reinterpret_cast<uint4 *>(stage + swz(rl, (c0 + j) >> 3)) =
+                                    make_uint4(pack_bf16(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), pack_bf16(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])),
+                                               pack_bf16(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])), pack_bf16(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
                             }
-                        }
+                        };
+                        round(tmem + TM_DV, a.part_dv, skv + SUB, 0, nullptr);
+                        round(tmem + TM_DV, a.part_dv, skv + SUB, 32, dv_free);
+                        round(tmem + TM_DK, a.part_dk, skv, 0, nullptr);
+                        round(tmem + TM_DK, a.part_dk, skv, 32, dk_free);
                     }
                     fence_proxy_async_smem();
                     go = group_all(ok, 1, 128);
