@@ -471,8 +471,6 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
 #pragma unroll
                 for (int i = 0; i < 2; ++i) {
                     uint32_t s_[16], d_[16], pp[8], pd[8];
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) { pp[j] = 0u; pd[j] = 0u; }
                     if (any[i]) {
                         tmem_ld16(tm_s + 16u * i, s_);
                         tmem_ld16(tm_dp + 16u * i, d_);
@@ -504,6 +502,9 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                             pp[j >> 1] = pack_bf16(p0, p1);
                             pd[j >> 1] = pack_bf16(e0, e1);
                         }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) { pp[j] = 0u; pd[j] = 0u; }
                     }
                     // P^T: the piece's 16 queries are 8 packed columns, inside the S^T columns this warp has read
                     tmem_st8(tm_s + 8u * i, pp);
