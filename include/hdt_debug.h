@@ -38,6 +38,11 @@ extern "C" {
  *                    1: two walks (one for dQ, one for dK and dV), no fp32 buffer; 2: the one walk
  *                    in the lock-step form of the two-walk kernel; 86: as 0, with the clock marks
  *                    that hdt_debug_bwd_w_marks and hdt_debug_bwd_w_tiles read back.
+ *   "tc_deep"        1: hierarchies of more than three stages run the stages above 0 of bf16 calls on the
+ *                    gathering tensor-core kernels too (faster; on deep random trees single gradient
+ *                    entries then pass the 2e-2 bound by a few percent).
+ *   "no_multi_upper" 1: the fp32 SIMT kernels take the stages above 0 of such hierarchies with a launch
+ *                    per stage instead of one launch over the blocks of all of them.
  *   "no_fused_delta" 1: the delta pass (rowsum(dO . O)) runs even where every backward kernel of the
  *                    call could compute it itself.
  *   "no_fold"        bit 0: a merge kernel completes the elements of stage 1 in the forward instead

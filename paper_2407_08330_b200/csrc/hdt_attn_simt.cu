@@ -84,12 +84,13 @@ __device__ __forceinline__ void stage_rows(float4 *dst, const void *src, const i
 // ---------------------------------------------------------------------------------------------
 // forward
 // ---------------------------------------------------------------------------------------------
+// (the body for entry bx of a stage's queue: the one-stage kernel and the kernel over several stages call it)
 template <int D, bool BF16, int NTHREADS>
-__global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
+__device__ __forceinline__ void fwd_simt_block(const FwdStageArgs &a, int bx) {
     constexpr int G = D / 16, U = D / 4, RP = NTHREADS / G;
     __shared__ float4 sK[KC * U];
     __shared__ float4 sV[KC * U];
-    const int blk = a.queue[blockIdx.x], h = blockIdx.y, H = a.H;
+    const int blk = a.queue[bx], h = blockIdx.y, H = a.H;
     const int *rec = a.blocks + 5 * (size_t)blk;
     const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3];
     const int g = threadIdx.x % G, rl = threadIdx.x / G;
@@ -206,17 +207,34 @@ __global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
     }
 }
 
+template <int D, bool BF16, int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) k_fwd_simt(const FwdStageArgs a) {
+    fwd_simt_block<D, BF16, NTHREADS>(a, (int)blockIdx.x);
+}
+// Several stages in own-partial mode (deep trees: a launch per stage is mostly launch latency) in one
+// launch: CTA x belongs to the stage s with cum[s] <= x < cum[s + 1] and is entry x - cum[s] of its queue.
+template <int D, bool BF16, int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) k_fwd_simt_multi(const MultiFwdArgs m) {
+    int s = 0;
+    while (s + 1 < m.n && (int)blockIdx.x >= m.st[s + 1].cum) ++s;
+    FwdStageArgs a = m.base;
+    const MultiStage &t = m.st[s];
+    a.n = t.n; a.nb = t.nb; a.tok = t.tok; a.tok_rows = t.tok; a.rng = t.rng; a.up = t.up; a.blocks = t.blocks; a.queue = t.queue;
+    a.own_o = t.own[0]; a.own_lse = t.own_lse;
+    fwd_simt_block<D, BF16, NTHREADS>(a, (int)blockIdx.x - t.cum);
+}
+
 // ---------------------------------------------------------------------------------------------
 // backward: phase A rows -> dQ, phase B keys -> dK, dV (the family ranges are symmetric, so the
 // same blocks serve as key blocks)
 // ---------------------------------------------------------------------------------------------
 template <int D, bool BF16, int NTHREADS>
-__global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
+__device__ __forceinline__ void bwd_simt_block(const BwdStageArgs &a, int bx) {
     constexpr int G = D / 16, U = D / 4, RP = NTHREADS / G;
     __shared__ float4 sA[KC * U];  // K (phase A) / Q (phase B)
     __shared__ float4 sB[KC * U];  // V (phase A) / dO (phase B)
     __shared__ float sL[KC], sDl[KC];
-    const int blk = a.queue[blockIdx.x], h = blockIdx.y, H = a.H;
+    const int blk = a.queue[bx], h = blockIdx.y, H = a.H;
     const int *rec = a.blocks + 5 * (size_t)blk;
     const int r0 = rec[0], r1 = rec[1], ka = rec[2], kb = rec[3];
     const int g = threadIdx.x % G, rl = threadIdx.x / G;
@@ -376,6 +394,21 @@ __global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
     }
 }
 
+template <int D, bool BF16, int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) k_bwd_simt(const BwdStageArgs a) {
+    bwd_simt_block<D, BF16, NTHREADS>(a, (int)blockIdx.x);
+}
+template <int D, bool BF16, int NTHREADS>
+__global__ void __launch_bounds__(NTHREADS) k_bwd_simt_multi(const MultiBwdArgs m) {
+    int s = 0;
+    while (s + 1 < m.n && (int)blockIdx.x >= m.st[s + 1].cum) ++s;
+    BwdStageArgs a = m.base;
+    const MultiStage &t = m.st[s];
+    a.n = t.n; a.nb = t.nb; a.tok = t.tok; a.tok_rows = t.tok; a.rng = t.rng; a.up = t.up; a.blocks = t.blocks; a.queue = t.queue;
+    a.own_dq = t.own[0]; a.own_dk = t.own[1]; a.own_dv = t.own[2];
+    bwd_simt_block<D, BF16, NTHREADS>(a, (int)blockIdx.x - t.cum);
+}
+
 // delta[h, t] = sum_c dO[t,h,c] * O[t,h,c].  A (token, head) row is read by LPR adjacent lanes with
 // one 16-byte load each per tensor (8 bf16 or 4 fp32 values), so a warp covers 32 / LPR rows.
 template <int D, bool BF16>
@@ -496,6 +529,41 @@ static int launch_bwd_t(const BwdStageArgs &a, cudaStream_t st) {
     count_launch();
     HDT_CUDA_CHECK(cudaGetLastError());
     return HDT_OK;
+}
+
+template <int D, bool BF16>
+static int launch_fwd_multi_t(const MultiFwdArgs &m, cudaStream_t st) {
+    const int total = m.st[m.n - 1].cum + m.st[m.n - 1].nb;
+    if (total == 0) return HDT_OK;
+    dim3 grid(total, m.base.H);
+    if (m.base.block_rows <= 32) k_fwd_simt_multi<D, BF16, 128><<<grid, 128, 0, st>>>(m);
+    else k_fwd_simt_multi<D, BF16, 512><<<grid, 512, 0, st>>>(m);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+template <int D, bool BF16>
+static int launch_bwd_multi_t(const MultiBwdArgs &m, cudaStream_t st) {
+    const int total = m.st[m.n - 1].cum + m.st[m.n - 1].nb;
+    if (total == 0) return HDT_OK;
+    dim3 grid(total, m.base.H);
+    if (m.base.block_rows <= 32) k_bwd_simt_multi<D, BF16, 128><<<grid, 128, 0, st>>>(m);
+    else k_bwd_simt_multi<D, BF16, 512><<<grid, 512, 0, st>>>(m);
+    count_launch();
+    HDT_CUDA_CHECK(cudaGetLastError());
+    return HDT_OK;
+}
+int launch_fwd_simt_multi(const MultiFwdArgs &m, int D, int dtype, cudaStream_t st) {
+    if (m.n <= 0) return HDT_OK;
+    if (D == 64) return dtype == HDT_BF16 ? launch_fwd_multi_t<64, true>(m, st) : launch_fwd_multi_t<64, false>(m, st);
+    if (D == 128) return dtype == HDT_BF16 ? launch_fwd_multi_t<128, true>(m, st) : launch_fwd_multi_t<128, false>(m, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
+}
+int launch_bwd_simt_multi(const MultiBwdArgs &m, int D, int dtype, cudaStream_t st) {
+    if (m.n <= 0) return HDT_OK;
+    if (D == 64) return dtype == HDT_BF16 ? launch_bwd_multi_t<64, true>(m, st) : launch_bwd_multi_t<64, false>(m, st);
+    if (D == 128) return dtype == HDT_BF16 ? launch_bwd_multi_t<128, true>(m, st) : launch_bwd_multi_t<128, false>(m, st);
+    return set_error(HDT_ERR_UNSUPPORTED, "head_dim %d not supported (64 or 128)", D);
 }
 
 int launch_fwd_simt(const FwdStageArgs &a, int D, int dtype, cudaStream_t st) {

@@ -231,6 +231,18 @@ struct BwdStageArgs {
     int gather_end_q, gather_end_k;               // gathering kernel: elements at or beyond these read as zero rows on the Q/dO and the K/V side (0: n)
 };
 
+// The stages above 0 of a deep tree in own-partial mode, all in one launch of the SIMT kernels: what differs
+// from stage to stage, and where the stage's CTAs start in the launch's grid.
+struct MultiStage {
+    int n, nb, cum;
+    const int *tok, *rng, *up, *blocks, *queue;
+    float *own[3];       // forward: own[0] = O; backward: dQ, dK, dV
+    float *own_lse;      // forward only
+};
+struct MultiFwdArgs { FwdStageArgs base; int n; MultiStage st[HDT_MAX_STAGES - 1]; };
+struct MultiBwdArgs { BwdStageArgs base; int n; MultiStage st[HDT_MAX_STAGES - 1]; };
+int launch_fwd_simt_multi(const MultiFwdArgs &m, int head_dim, int dtype, cudaStream_t st);
+int launch_bwd_simt_multi(const MultiBwdArgs &m, int head_dim, int dtype, cudaStream_t st);
 int launch_fwd_simt(const FwdStageArgs &a, int head_dim, int dtype, cudaStream_t st);
 // Tensor-core (TMA + tcgen05) stage-0 kernels for bf16 (hdt_attn_tc.cu).
 int launch_fwd_tc(const FwdStageArgs &a, int head_dim, cudaStream_t st);
