@@ -258,6 +258,13 @@ def test_generic_depth_trees(P):
     b = gen.pack(seqs)
     run_case(P, b, 2, 64, "f32", 21)
     run_case(P, b, 2, 64, "bf16", 22)
+    # (more than three stages: the stages above 0 run in one launch; here with a launch per stage as well)
+    P.hdt_set_option("no_multi_upper", 1)
+    try:
+        _run_case(P, b, 2, 64, "f32", 21, True, 128, 0.0)
+        _run_case(P, b, 2, 64, "bf16", 22, True, 128, 0.0)
+    finally:
+        P.hdt_set_option("no_multi_upper", 0)
 
 
 def test_forward_is_deterministic_and_guard_bands_untouched(P):
