@@ -124,10 +124,10 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     uint64_t *qdo_full = bars, *qdo_empty = bars + 3, *sdp_full = bars + 6, *pds_ready = bars + 8;
     uint64_t *dq_full = bars + 10, *dq_free = bars + 12, *kv_full = bars + 14, *kv_empty = bars + 16;
     uint64_t *acc_full = bars + 18, *dv_free = bars + 19, *stat_full = bars + 20, *stg_free = bars + 22, *stg_full = bars + 24, *kv_reuse = bars + 26;
-    uint64_t *dk_free = bars + 28;
-    uint32_t *slot = (uint32_t *)(bars + 29);
+    uint64_t *dk_free = bars + 28, *dvacc_full = bars + 29;
+    uint32_t *slot = (uint32_t *)(bars + 30);
     volatile int *abort_flag = (volatile int *)(slot + 1);
-    long long *s_marks = (long long *)(bars + 30);      // [5 roles][2 tiles][8 marks] of the instrumented run (only then allocated)
+    long long *s_marks = (long long *)(bars + 31);      // [5 roles][2 tiles][8 marks] of the instrumented run (only then allocated)
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int H = a.H, G = gridDim.x;
@@ -164,6 +164,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
         mbar_init(acc_full, 1);
         mbar_init(dv_free, 128);
         mbar_init(dk_free, 128);
+        mbar_init(dvacc_full, 1);
         *abort_flag = (*a.status != 0);
         fence_mbar_init();
     }
@@ -363,12 +364,10 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 // ---- step a: dV; S^T, dP^T of the next tile's step a; dK ----
                 W_MARK(4, t, 0);
                 if (MARKS && blockIdx.x == 0 && lane == 0 && t < 512) g_bwd_w_tiles[t] = (clock64() << 8) | (long long)(uc & 255);
-                // (what is normally there already first, the wait for the compute group last: it ends the chain)
+                // dV of the step first: it needs nothing of the next tile.  S^T / dP^T of the next tile's step a behind
+                // it (P^T lies over the S^T columns), once that tile's Q / dO are there, then dK: the pipe has dV to
+                // work on while this warp waits for the load.
                 if (first && uc >= 1) HDT_WAIT(dv_free, (uc - 1) & 1, 6);      // the previous unit's dV has been read (dK: below)
-                if (n_valid) {
-                    HDT_WAIT(&qdo_full[n_qs], n_qph, 7);
-                    if (last) HDT_WAIT(&kv_full[n_uc & 1], (n_uc >> 1) & 1, 8);      // the next tile opens a unit (the other K / V buffer)
-                }
                 W_MARK(4, t, 1);
                 HDT_WAIT(&pds_ready[0], t & 1, 5);
                 if (!HDT_AGREE()) break;
@@ -376,6 +375,15 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 if (elect_one()) {
                     tc_fence_after();
                     issue_dv(0, qs, acc);
+                }
+                __syncwarp();
+                if (n_valid) {
+                    HDT_WAIT(&qdo_full[n_qs], n_qph, 7);
+                    if (last) HDT_WAIT(&kv_full[n_uc & 1], (n_uc >> 1) & 1, 8);      // the next tile opens a unit (the other K / V buffer)
+                    if (!HDT_AGREE()) break;
+                }
+                if (elect_one()) {
+                    tc_fence_after();
                     if (n_valid) issue_sdp(0, n_qs, n_uc & 1);
                     if (!(first && uc >= 1)) issue_dk(0, qs, db, acc);
                 }
@@ -398,6 +406,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 if (elect_one()) {
                     tc_fence_after();
                     issue_dv(1, qs, 1u);
+                    if (last) mma_commit(dvacc_full);        // dV of the unit is complete: the drain group may start on it
                     if (n_valid) issue_sdp(1, n_qs, n_uc & 1);
                     issue_dk(1, qs, db, 1u);
                     mma_commit(&qdo_empty[qs]);        // every MMA that reads this tile's Q / dO has been issued
@@ -528,46 +537,54 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 const WUnit &U = w.U;
                 const int t = w.t, db = t & 1;
                 W_MARK(2, t, 0);
+                // ---- end of a unit: dK and dV of this thread's key row (the next unit's MMAs wait for the
+                // accumulators).  bf16 rows staged in the unit's K / V buffer, one swizzled [128 x 64] tile per
+                // tensor, TMA stores; the load warp takes the buffer for the unit after the next once the stores have
+                // read it.  dV first: its last MMA is the first of the tile's step b, and V's last reader (S^T / dP^T of
+                // this tile) was issued a tile ago, so the V half of the buffer is free before the tile's dQ is done;
+                // dK, whose half dQ = dS K still reads, after the wait for dQ.  32 columns a round; no factor: the
+                // compute warps put softmax_scale into dS. ----
+                const bool last = w.j == U.nt - 1;
+                const int nrows = U.r1 - U.r0, kvb = w.uc & 1;
+                uint8_t *skv = sKV + kvb * 2 * SUB;
+                int up = -1;
+                if (last && rl < nrows && a.part_dk != nullptr) up = a.up[U.r0 + rl];
+                auto round = [&](uint32_t tm_acc, float *part, uint8_t *stage, int c0, uint64_t *read_bar) {
+                    uint32_t r[32];
+                    tmem_ld32(tm_acc + lane_base + c0, r);
+                    tmem_wait_ld();
+                    if (read_bar != nullptr) {      // the accumulator has been read: the next unit may overwrite it
+                        tc_fence_before();
+                        mbar_arrive(read_bar);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 32; j += 8) {
+                        if (up >= 0) {      // this row lives on in the next stage: its fp32 gradients go there too
+                            float4 *pt = reinterpret_cast<float4 *>(part + ((size_t)up * H + U.h) * D + c0 + j);
+                            pt[0] = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+                            pt[1] = make_float4(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]), __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+                        }
+                        *reinterpret_cast<uint4 *>(stage + swz(rl, (c0 + j) >> 3)) =
+                            make_uint4(pack_bf16(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), pack_bf16(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])),
+                                       pack_bf16(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])), pack_bf16(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
+                    }
+                };
+                if (last) {
+                    HDT_WAIT(dvacc_full, w.uc & 1, 26);
+                    if (HDT_AGREE()) {
+                        tc_fence_after();
+                        round(tmem + TM_DV, a.part_dv, skv + SUB, 0, nullptr);
+                        round(tmem + TM_DV, a.part_dv, skv + SUB, 32, dv_free);
+                    }
+                }
                 HDT_WAIT(&dq_full[db], (t >> 1) & 1, 14);
                 W_MARK(2, t, 1);
-                if (w.j == U.nt - 1) {
-                    // ---- end of the unit, before the tile's dQ (the next unit's MMAs wait for the accumulators): dK and dV of this
-                    // thread's key row.  bf16 rows staged in the unit's K / V
-                    // buffer (every MMA of the unit is complete), one swizzled [128 x 64] tile per tensor, TMA stores;
-                    // the load warp takes the buffer for the unit after the next once the stores have read it. ----
-                    const int nrows = U.r1 - U.r0, kvb = w.uc & 1;
-                    uint8_t *skv = sKV + kvb * 2 * SUB;
-                    int up = -1;
-                    if (rl < nrows && a.part_dk != nullptr) up = a.up[U.r0 + rl];
+                if (last) {
                     const int bx = max(__clz(nrows) - 25, 0);
                     const int bbox = 64 >> bx;
                     HDT_WAIT(acc_full, w.uc & 1, 15);
                     if (HDT_AGREE()) {
                         tc_fence_after();
-                        // dV first (the next unit's MMAs need its accumulator first), then dK; 32 columns a round.
-                        // (no factor: the compute warps put softmax_scale into dS)
-                        auto round = [&](uint32_t tm_acc, float *part, uint8_t *stage, int c0, uint64_t *read_bar) {
-                            uint32_t r[32];
-                            tmem_ld32(tm_acc + lane_base + c0, r);
-                            tmem_wait_ld();
-                            if (read_bar != nullptr) {      // the accumulator has been read: the next unit may overwrite it
-                                tc_fence_before();
-                                mbar_arrive(read_bar);
-                            }
-#pragma unroll
-                            for (int j = 0; j < 32; j += 8) {
-                                if (up >= 0) {      // this row lives on in the next stage: its fp32 gradients go there too
-                                    float4 *pt = reinterpret_cast<float4 *>(part + ((size_t)up * H + U.h) * D + c0 + j);
-                                    pt[0] = make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-                                    pt[1] = make_float4(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]), __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
-                                }
-                                *reinterpret_cast<uint4 *>(stage + swz(rl, (c0 + j) >> 3)) =
-                                    make_uint4(pack_bf16(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), pack_bf16(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])),
-                                               pack_bf16(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])), pack_bf16(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
-                            }
-                        };
-                        round(tmem + TM_DV, a.part_dv, skv + SUB, 0, nullptr);
-                        round(tmem + TM_DV, a.part_dv, skv + SUB, 32, dv_free);
                         round(tmem + TM_DK, a.part_dk, skv, 0, nullptr);
                         round(tmem + TM_DK, a.part_dk, skv, 32, dk_free);
                     }
