@@ -85,6 +85,8 @@ int get_side(Side **out) {
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.fork, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join2, cudaEventDisableTiming));
+        HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.fork0, cudaEventDisableTiming));
+        HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join0, cudaEventDisableTiming));
         sd.ready = true;
     }
     *out = &sd;
@@ -462,14 +464,29 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     if (L.has_dq_acc && !g_force_simt && g_bwd_walk != 1 &&
         (g_no_persistent == 0 || g_no_persistent == 4 || g_no_persistent == 6)) {
         dq_acc = (float *)(ws + L.dq_acc);
-        ProfScope ps(PROF_BWD_STAGE0, st);
-        HDT_CUDA_CHECK(cudaMemsetAsync(dq_acc, 0, sizeof(float) * (size_t)ix->total_tokens * heads * 64, st));
+    }
+    // The buffer is cleared (writes) beside the delta pass (reads), on the second side stream: both are
+    // HBM-bound, one in each direction.  Stage 0 waits for it (join0).
+    Side *sd0 = nullptr;
+    const bool clear_beside = dq_acc != nullptr && !fused_delta && !g_no_overlap && get_side(&sd0) == HDT_OK && sd0 != nullptr;
+    if (dq_acc != nullptr) {
+        const size_t bytes = sizeof(float) * (size_t)ix->total_tokens * heads * 64;
+        if (clear_beside) {
+            HDT_CUDA_CHECK(cudaEventRecord(sd0->fork0, st));
+            HDT_CUDA_CHECK(cudaStreamWaitEvent(sd0->s2, sd0->fork0, 0));
+            HDT_CUDA_CHECK(cudaMemsetAsync(dq_acc, 0, bytes, sd0->s2));
+            HDT_CUDA_CHECK(cudaEventRecord(sd0->join0, sd0->s2));
+        } else {
+            ProfScope ps(PROF_BWD_STAGE0, st);
+            HDT_CUDA_CHECK(cudaMemsetAsync(dq_acc, 0, bytes, st));
+        }
     }
     if (!fused_delta) {
         ProfScope ps(PROF_DELTA, st);
         rc = launch_delta(o, d_o, delta, ix->total_tokens, heads, head_dim, dtype, st);
     }
     if (rc) return rc;
+    if (clear_beside) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd0->join0, 0));
     auto stage_args = [&](int s) {
         const StagePtrs &P = ix->st[s];
         BwdStageArgs a{};
