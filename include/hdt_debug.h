@@ -43,6 +43,8 @@ extern "C" {
  *                    entries then pass the 2e-2 bound by a few percent).
  *   "no_multi_upper" 1: the fp32 SIMT kernels take the stages above 0 of such hierarchies with a launch
  *                    per stage instead of one launch over the blocks of all of them.
+ *   "no_self_beside" 1: in a backward with the one-walk kernel, the kernel of the self-contained stage-0 blocks
+ *                    runs behind it on the caller's stream instead of beside it on an internal stream.
  *   "no_fused_delta" 1: the delta pass (rowsum(dO . O)) runs even where every backward kernel of the
  *                    call could compute it itself.
  *   "no_fold"        bit 0: a merge kernel completes the elements of stage 1 in the forward instead

@@ -70,6 +70,7 @@ int g_phase_stamps = 0;
 int g_no_fwd_mc = 0;
 int g_no_pdl = 0;
 static int g_no_multi_upper = 0;
+static int g_no_self_beside = 0;
 static int g_tc_deep = 0;
 static int g_no_fused_delta = 0;
 static int g_no_fold = 0;
@@ -181,6 +182,7 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "bwd_walk") == 0) { g_bwd_walk = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_multi_upper") == 0) { g_no_multi_upper = value; return HDT_OK; }
     if (name && std::strcmp(name, "tc_deep") == 0) { g_tc_deep = value; return HDT_OK; }
+    if (name && std::strcmp(name, "no_self_beside") == 0) { g_no_self_beside = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
 
@@ -523,7 +525,10 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
         if (rc) return rc;
         HDT_CUDA_CHECK(cudaEventRecord(sd->fork, st));
         HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s, sd->fork, 0));
-        const bool two = ix->n_stages > 2;
+        // (with the one-walk kernel the self-contained blocks' kernel goes to the second side stream: its CTAs take
+        // the SMs that the one-walk kernel's CTAs leave first, and it shares HBM with the pass that converts dQ)
+        const bool self_beside = dq_acc != nullptr && ix->desc[0].n_fused > 0 && !g_no_self_beside;
+        const bool two = ix->n_stages > 2 || self_beside;
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 3;
@@ -564,16 +569,21 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
-        if (two) HDT_CUDA_CHECK(cudaEventRecord(sd->join2, sd->s2));
+        if (two && !self_beside) HDT_CUDA_CHECK(cudaEventRecord(sd->join2, sd->s2));
         {
             BwdStageArgs a = stage_args(0);
+            if (self_beside) a.self_stream = (void *)sd->s2;
             ProfScope ps(PROF_BWD_STAGE0, st);
             if (dtype == HDT_BF16 && !g_force_simt) rc = launch_bwd_tc(a, head_dim, st);
             else rc = launch_bwd_simt(a, head_dim, dtype, st);
             if (rc) return rc;
+            if (self_beside) {       // (inside the scope: stage 0 ends when both streams have)
+                HDT_CUDA_CHECK(cudaEventRecord(sd->join2, sd->s2));
+                HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
+            }
         }
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
-        if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
+        if (two && !self_beside) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
         ProfScope ps(PROF_BWD_UPPER, st);
         if (fold) {
             a1.final_merge = 1;

@@ -1311,7 +1311,7 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
             const long long units = (long long)(mode ? a.nb - a.n_fused : a.n_fused) * a.H;
             if (units == 0) continue;
             if (mode == 0 && a.no_persistent != 4) {     // (4: the persistent kernel takes these too)
-                rc = launch_bwd_tc_fused64(a, tq, tk, tv, tdo, outs, st);
+                rc = launch_bwd_tc_fused64(a, tq, tk, tv, tdo, outs, (onewalk && a.self_stream) ? (cudaStream_t)a.self_stream : st);
                 if (rc) return rc;
                 continue;
             }

@@ -228,6 +228,8 @@ struct BwdStageArgs {
     float *dq_acc;                                // stage 0, head_dim 64: fp32 [T,H,64] buffer, zero on entry, that the one-walk kernel of the
                                                   // split families adds its dQ tiles to (nullptr: they are walked twice instead)
     int n_empty;                                  // EMPTY blocks of the stage (-1: unknown)
+    void *self_stream;                            // stage 0 with dq_acc: stream (cudaStream_t, already forked from the caller's) for the kernel of the
+                                                  // self-contained blocks, which then runs beside the one-walk kernel of the others (nullptr: behind it)
     int gather_end_q, gather_end_k;               // gathering kernel: elements at or beyond these read as zero rows on the Q/dO and the K/V side (0: n)
 };
 
