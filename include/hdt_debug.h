@@ -48,8 +48,9 @@ extern "C" {
  *   "no_fused_delta" 1: the delta pass (rowsum(dO . O)) runs even where every backward kernel of the
  *                    call could compute it itself.
  *   "no_fold"        bit 0: a merge kernel completes the elements of stage 1 in the forward instead
- *                    of the stage-1 kernel itself; bit 2: the backward's stage-1 kernel does the
- *                    completion (off by default).
+ *                    of the stage-1 kernel itself (the default where a family of stage 1 is longer than
+ *                    a block); bit 1: the stage-1 kernel does it there too; bit 2: the backward's
+ *                    stage-1 kernel does the completion (off by default).
  *   "no_overlap"     1: the stages above 0 run after stage 0 on the caller's stream instead of
  *                    beside it on an internal stream.
  *   "no_graph"       1: hdt_build_index launches its kernels one by one instead of replaying a

@@ -348,8 +348,16 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         c.tok1 = ix->st[1].tok;
         // On the gathering kernels stage 1 runs after stage 0 and completes its elements itself
         // (its own result merged with stage 0's partial and stage 2's own); only stage 2 runs beside
-        // stage 0, and there is no merge kernel.
-        const bool fold = tc_upper && !(g_no_fold & 1) && ix->n_stages > 1 && ix->n_stages <= 3;
+        // stage 0, and there is no merge kernel.  That pays while the stage-1 kernel is shorter than
+        // the merge it saves (about 10 us): no family of stage 1 longer than a block, and its CTAs
+        // resident at once.  Otherwise (skewed documents with long sections: 47 us against 13; large
+        // batches at head_dim 128: 59 against 23) stage 1 runs beside stage 0 like the others and the
+        // merge kernel follows.
+        int n_sm1 = 0;
+        if (const int rc_ = sm_count(&n_sm1)) return rc_;
+        const bool short1 = ix->n_stages > 1 && ix->desc[1].n_fused + ix->desc[1].n_empty == ix->desc[1].nb &&
+                            (long long)ix->desc[1].nb * heads <= 2LL * n_sm1;
+        const bool fold = tc_upper && !(g_no_fold & 1) && (short1 || (g_no_fold & 2)) && ix->n_stages > 1 && ix->n_stages <= 3;
         FwdStageArgs a1{};
         // (deep trees: the stages above 0 are independent in own-partial mode and small, and a launch per stage is
         // mostly launch latency: one launch over the blocks of all of them)

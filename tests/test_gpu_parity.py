@@ -164,7 +164,7 @@ def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
     # default kernels; general tensor-core kernels only; persistent forward; SIMT everywhere
     # (fp32 runs with and without the side-stream overlap of the upper stages)
     # (the upper stages of bf16 runs: gathering tensor-core kernels with 128- and 32-row blocks, SIMT)
-    opts = (({}, {"_block_m_upper": 32}, {"simt_upper": 1}, {"no_fold": 1}, {"no_fold": 4}, {"no_fused_delta": 1, "no_persistent": 4}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2},
+    opts = (({}, {"_block_m_upper": 32}, {"simt_upper": 1}, {"no_fold": 1}, {"no_fold": 2}, {"no_fold": 4}, {"no_fused_delta": 1, "no_persistent": 4}, {"no_persistent": 1, "no_overlap": 1}, {"no_persistent": 2},
              {"no_persistent": 3}, {"no_persistent": 5}, {"no_fwd_mc": 1}, {"no_self_beside": 1}, {"force_simt": 1})
             if dtype == "bf16" else ({}, {"no_overlap": 1}))
     for opt in opts:
