@@ -75,7 +75,7 @@ __device__ __forceinline__ void dev_fail(DevHeader *h, int code, int pos) {
 // ---------------------------------------------------------------------------------------------
 __global__ void k_init(const int8_t *__restrict__ level, const int32_t *__restrict__ parent,
                        const int32_t *__restrict__ cu, int B, int T, int max_level, DevHeader *hdr,
-                       int *tok, int *par, int *scu, int *cnt) {
+                       int *tok, int *par, int *scu, int *cnt, int *nlc) {
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i <= B) {
         const int c = cu[i];
@@ -116,27 +116,26 @@ __global__ void k_init(const int8_t *__restrict__ level, const int32_t *__restri
     if (!ok) { dev_fail(hdr, HDT_ERR_BAD_HIERARCHY, i); gp = -1; }
     tok[i] = i;
     par[i] = gp;
-    if (gp >= 0) atomicAdd(&cnt[gp], 1);   // cnt and nlc were zeroed with the header
-}
-
-__global__ void k_count(const DevHeader *hdr, int s, const int *__restrict__ par, int *cnt) {
-    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
-    pdl_wait();                   // the kernel before this one has completed
-    const int n = hdr->st[s].n;
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
-        const int p = par[e];
-        if (p >= 0) atomicAdd(&cnt[p], 1);
+    // cnt and nlc were zeroed with the header.  nlc[x] = children of x that have children: the first
+    // child to register with its parent reports that parent to the grandparent, once per parent
+    // (no second pass over the elements after the counts are complete).
+    if (gp >= 0 && atomicAdd(&cnt[gp], 1) == 0) {
+        const int pg = parent[gp];
+        if (pg >= 0 && pg < gp - s0) atomicAdd(&nlc[s0 + pg], 1);   // (gp's own thread reports a bad entry)
     }
 }
 
-__global__ void k_nlc(const DevHeader *hdr, int s, const int *__restrict__ par,
-                      const int *__restrict__ cnt, int *nlc) {
+// Child counts of a stage above 0, and nlc as in k_init (first child to register reports its parent).
+__global__ void k_count(const DevHeader *hdr, int s, const int *__restrict__ par, int *cnt, int *nlc) {
     pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
     pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
     for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
         const int p = par[e];
-        if (p >= 0 && cnt[e] > 0) atomicAdd(&nlc[p], 1);
+        if (p >= 0 && atomicAdd(&cnt[p], 1) == 0) {
+            const int pp = par[p];
+            if (pp >= 0) atomicAdd(&nlc[pp], 1);
+        }
     }
 }
 
@@ -480,24 +479,30 @@ struct UpperArgs {
 static constexpr int UT = 1024;      // threads of the fused kernel
 static constexpr int UMAXB = 1024;   // sequences it handles (per-sequence offsets live in shared memory)
 static constexpr int UCAP = 4096;    // elements of a stage whose scratch fits in shared memory
-static constexpr int USMEM = UCAP * (7 * 4 + 2);   // bytes of that scratch
+static constexpr int USB = 2048;     // block slots of a stage whose block starts, costs and flags stay in shared memory
+static constexpr int USMEM = UCAP * (8 * 4 + 2) + USB * (4 + 8 + 1);   // bytes of that scratch
 
 __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const UpperArgs u) {
-    // Stages of at most UCAP elements keep their per-element scratch (parents, child counts, keep
-    // flags, prefix sums, ranges, next-stage indices) in shared memory: a dozen barrier-separated
-    // steps per stage would otherwise each pay a round trip to global memory.
+    // Stages of at most UCAP elements keep their per-element scratch (tokens, parents, child counts,
+    // keep flags, prefix sums, ranges, next-stage indices) in shared memory, and with at most USB
+    // block slots the block starts, costs and flags too: a dozen barrier-separated steps per stage
+    // would otherwise each pay a round trip to global memory (after the loads at a stage's start
+    // such a stage only writes to it).
     extern __shared__ __align__(16) int s_dyn[];
     int *s_par = s_dyn, *s_cnt = s_par + UCAP, *s_nlc = s_cnt + UCAP, *s_pre = s_nlc + UCAP, *s_up = s_pre + UCAP;
     int *s_rng = s_up + UCAP;                                   // 2 * UCAP
-    uint8_t *s_keep = reinterpret_cast<uint8_t *>(s_rng + 2 * UCAP), *s_fpos = s_keep + UCAP;
+    int *s_tok = s_rng + 2 * UCAP;
+    long long *s_cst = reinterpret_cast<long long *>(s_tok + UCAP);   // (8-byte aligned: the arrays before it are multiples of 16 KB)
+    int *s_bst = reinterpret_cast<int *>(s_cst + USB);
+    uint8_t *s_keep = reinterpret_cast<uint8_t *>(s_bst + USB), *s_fpos = s_keep + UCAP, *s_bfl = s_fpos + UCAP;
     __shared__ int s_off[UMAXB], s_base[UMAXB + 1], s_nbs[UMAXB], s_scu[UMAXB + 1];   // per sequence: block slots, first block, block count, offsets
     __shared__ int s_w[32];
-    __shared__ int s_carry, s_flag;
+    __shared__ int s_carry, s_flag, s_cap;
     __shared__ long long s_ll[32];
     const int t = threadIdx.x, lane = t & 31, w = t >> 5;
     const int B = u.B, bm = u.bm;
+    int n = hdr->st[1].n;                // (stage 0's kernels wrote it; the later ones are computed here)
     for (int s = 1; s < u.max_stages; ++s) {
-        const int n = hdr->st[s].n;      // written by the previous stage, same value in every thread
         if (n == 0) break;
         const StagePtrs P = u.st[s];
         const bool last = (s + 1 == u.max_stages);
@@ -505,11 +510,11 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         const bool small = n <= UCAP;
         int *cnt = small ? s_cnt : u.cnt, *nlc = small ? s_nlc : u.nlc, *pre = small ? s_pre : u.pre;
         uint8_t *keep = small ? s_keep : u.keep, *fpos = small ? s_fpos : u.fpos;
-        const int *par = small ? s_par : P.par;
+        const int *par = small ? s_par : P.par, *tokr = small ? s_tok : P.tok;
         const int *rngr = small ? s_rng : P.rng, *upr = small ? s_up : P.up;    // read-back of this stage's results
         for (int b = t; b <= B; b += UT) s_scu[b] = P.scu[b];
         if (small)
-            for (int e = t; e < n; e += UT) { s_par[e] = P.par[e]; s_cnt[e] = 0; s_nlc[e] = 0; }
+            for (int e = t; e < n; e += UT) { s_par[e] = P.par[e]; s_tok[e] = P.tok[e]; s_cnt[e] = 0; s_nlc[e] = 0; }
         __syncthreads();
         // children counts (cnt, nlc are zero for [0, n))
         for (int e = t; e < n; e += UT) { const int p = par[e]; if (p >= 0) atomicAdd(&cnt[p], 1); }
@@ -571,7 +576,7 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                 const int up = (kp && has_next) ? excl : -1;
                 P.up[e] = up;
                 if (small) s_up[e] = up;
-                if (up >= 0 && !last) N.tok[up] = P.tok[e];
+                if (up >= 0 && !last) N.tok[up] = tokr[e];
             }
             __syncthreads();
             if (t == 0) s_carry += s_w[31];
@@ -598,8 +603,12 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
             int off = 0;
             for (int c = 0; c < b; ++c) off += 2 * ((s_scu[c + 1] - s_scu[c] + bm - 1) / bm) + 2;
             s_off[b] = off;
+            if (b == B - 1) s_cap = off + 2 * ((s_scu[b + 1] - s_scu[b] + bm - 1) / bm) + 2;
         }
         __syncthreads();
+        const bool few = B > 0 && s_cap <= USB;        // block slots of this stage fit in shared memory
+        int *bst = few ? s_bst : u.bstart;
+        long long *cst = few ? s_cst : u.cost;
         for (int b = w; b < B; b += UT / 32) {
             if (lane == 0) {
                 const int s0 = s_scu[b], len = s_scu[b + 1] - s0, off = s_off[b];
@@ -610,7 +619,7 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                         const int f = fpos[s0 + end];
                         if (f >= 1 && f < end - pos) end -= f;
                     }
-                    u.bstart[off + cntb] = s0 + pos;
+                    bst[off + cntb] = s0 + pos;
                     ++cntb;
                     pos = end;
                 }
@@ -636,8 +645,8 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                 // (the largest b with s_base[b] <= gb always owns blocks: an empty sequence has the base of its successor)
                 const int b = lo_b, i = gb - s_base[b];
                 const int nb_seq = s_nbs[b], off = s_off[b], base = s_base[b], s1 = s_scu[b + 1];
-                const int r0 = u.bstart[off + i];
-                const int r1 = (i + 1 < nb_seq) ? u.bstart[off + i + 1] : s1;
+                const int r0 = bst[off + i];
+                const int r1 = (i + 1 < nb_seq) ? bst[off + i + 1] : s1;
                 int a = 0x7fffffff, bb = (int)0x80000000, carry = 0;
                 for (int e = r0 + lane; e < r1; e += 32) {
                     const int lo = rngr[2 * e], hi = rngr[2 * e + 1];
@@ -664,7 +673,8 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                     int *rec = P.blocks + 5 * (size_t)(base + i);
                     rec[0] = r0; rec[1] = r1; rec[2] = a; rec[3] = bb; rec[4] = fl;
                     const long long c = (long long)(r1 - r0) * (long long)(bb - a);
-                    u.cost[base + i] = c;
+                    cst[base + i] = c;
+                    if (few) s_bfl[base + i] = (uint8_t)fl;
                     vis += c;
                 }
             }
@@ -675,13 +685,13 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         const int nb = (B > 0) ? s_base[B] : 0;
         int mine = 0, mine_empty = 0;
         for (int i = w; i < nb; i += UT / 32) {      // one warp per block, lanes share the scan
-            const long long ci = u.cost[i];
-            const int fi = P.blocks[5 * i + 4];
+            const long long ci = cst[i];
+            const int fi = few ? (int)s_bfl[i] : P.blocks[5 * i + 4];
             const int ei = ((fi & HDT_BLK_SELF) && !(fi & HDT_BLK_EMPTY)) ? 1 : 0;
             int rank = 0, rank2 = 0;
             for (int j = lane; j < nb; j += 32) {
-                const long long cj = u.cost[j];
-                const int fj = P.blocks[5 * j + 4];
+                const long long cj = cst[j];
+                const int fj = few ? (int)s_bfl[j] : P.blocks[5 * j + 4];
                 const int ej = ((fj & HDT_BLK_SELF) && !(fj & HDT_BLK_EMPTY)) ? 1 : 0;
                 const int before = (cj > ci) || (cj == ci && j < i);
                 rank += before;
@@ -700,7 +710,8 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
         }
         if (mine) atomicAdd(&hdr->st[s].n_fused, mine);
         if (mine_empty) atomicAdd(&hdr->st[s].n_empty, mine_empty);
-        __syncthreads();   // hdr->st[s+1].n and everything else is visible before the next stage reads it
+        __syncthreads();   // every read of this stage's scratch is done before the next stage overwrites it
+        n = n2;
     }
 }
 
@@ -854,7 +865,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
         // header, cnt and nlc are adjacent in the workspace: one memset clears all three
         HDT_ENQ(cudaMemsetAsync(ws + L.header, 0, L.pre - L.header, st));
         k_init<<<g_el, 256, 0, st>>>(level, parent, cu_seqlens, B, T, HDT_MAX_STAGES * 8, hdr, ix->st[0].tok,
-                                     ix->st[0].par, ix->st[0].scu, cnt);
+                                     ix->st[0].par, ix->st[0].scu, cnt, nlc);
         ++n_launched;
         auto launch_upper = [&](cudaStream_t s_) {
             UpperArgs u;
@@ -876,14 +887,13 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             // the last possible stage writes its (unused) next-stage arrays into its own up/pre scratch
             const StagePtrs &N = ix->st[(s + 1 < ms) ? s + 1 : s];
             const bool last = (s + 1 == ms);
-            if (s >= 1) { HDT_ENQ(launch_chain(k_count, dim3(g_stride), dim3(256), 0, st, hdr, s, P.par, cnt)); ++n_launched; }
-            HDT_ENQ(launch_chain(k_nlc, dim3(g_stride), dim3(256), 0, st, hdr, s, P.par, cnt, nlc));
+            if (s >= 1) { HDT_ENQ(launch_chain(k_count, dim3(g_stride), dim3(256), 0, st, hdr, s, P.par, cnt, nlc)); ++n_launched; }
             HDT_ENQ(launch_chain(k_ranges, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, s == 0 ? level : (const int8_t *)nullptr, P.par, cnt, nlc,
                                  P.rng, keep, fpos, blocksum, dirs));
             // tok2 of the last possible stage is never read: point it at scratch (pre is rewritten first)
             HDT_ENQ(launch_chain(k_scan, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
                                  last ? cnt : N.tok));
-            n_launched += 3;
+            n_launched += 2;
             if (!last) {
                 HDT_ENQ(launch_chain(k_compact, dim3(g_stride), dim3(256), 0, st, hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc));
                 ++n_launched;
