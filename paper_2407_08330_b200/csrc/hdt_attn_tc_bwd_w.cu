@@ -327,6 +327,14 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 for (int kk = 0; kk < 4; ++kk)
                     mma_ss_w(tmem + TM_DK, d_lo + 2 * kk, dsk_hi, q_lo + 128 * kk, qdm_hi, id_kv, acc | (kk > 0));
             };
+            // (dS^T also lies packed over the dP^T columns, like P^T over S^T: dK takes it from there, which spares
+            // the shared-memory pipe the 4 KB operand of each of these MMAs and is the faster form besides)
+            auto issue_dk_t = [&](int x, int qs, uint32_t acc) {
+                const uint32_t q_lo = qdm_lo + qs * 2 * S16 + x * (8192 >> 4);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk)
+                    mma_ts_w(tmem + TM_DK, tmem + 128u * x + 64u + (kk < 2 ? 8u * kk : 32u + 8u * (kk - 2)), q_lo + 128 * kk, qdm_hi, id_kv, acc | (kk > 0));
+            };
             auto issue_dq = [&](int dsb, int kvb) {
                 const uint32_t d_lo = dsm_lo + dsb * 2 * S16, k_lo = kvm_lo + kvb * 2 * S16;
 #pragma unroll
@@ -375,6 +383,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 if (elect_one()) {
                     tc_fence_after();
                     issue_dv(0, qs, acc);
+                    if (!(first && uc >= 1)) issue_dk_t(0, qs, acc);      // (before the next dP^T overwrites its operand)
                 }
                 __syncwarp();
                 if (n_valid) {
@@ -385,12 +394,12 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                 if (elect_one()) {
                     tc_fence_after();
                     if (n_valid) issue_sdp(0, n_qs, n_uc & 1);
-                    if (!(first && uc >= 1)) issue_dk(0, qs, db, acc);
                 }
                 __syncwarp();
                 if (first && uc >= 1) {
                     // (the drain group reads dV first: dV and the next S^T / dP^T, which the compute group waits for, have
-                    // gone ahead while it still reads the previous unit's dK)
+                    // gone ahead while it still reads the previous unit's dK; this dK takes dS^T from shared memory, the
+                    // copy in TMEM is gone by now)
                     HDT_WAIT(dk_free, (uc - 1) & 1, 24);
                     if (!HDT_AGREE()) break;
                     if (elect_one()) issue_dk(0, qs, db, acc);
@@ -407,8 +416,8 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                     tc_fence_after();
                     issue_dv(1, qs, 1u);
                     if (last) mma_commit(dvacc_full);        // dV of the unit is complete: the drain group may start on it
+                    issue_dk_t(1, qs, 1u);
                     if (n_valid) issue_sdp(1, n_qs, n_uc & 1);
-                    issue_dk(1, qs, db, 1u);
                     mma_commit(&qdo_empty[qs]);        // every MMA that reads this tile's Q / dO has been issued
                     if (last) mma_commit(acc_full);
                     issue_dq(db, kvb);
@@ -517,6 +526,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
                     }
                     // P^T: the piece's 16 queries are 8 packed columns, inside the S^T columns this warp has read
                     tmem_st8(tm_s + 8u * i, pp);
+                    tmem_st8(tm_dp + 8u * i, pd);      // dS^T for dK, inside the dP^T columns this warp has read
                     *reinterpret_cast<uint4 *>(ds + swz(kl, 4 * qh + 2 * i)) = make_uint4(pd[0], pd[1], pd[2], pd[3]);
                     *reinterpret_cast<uint4 *>(ds + swz(kl, 4 * qh + 2 * i + 1)) = make_uint4(pd[4], pd[5], pd[6], pd[7]);
                 }
