@@ -273,9 +273,8 @@ int hdt_hpe(const hdt_index_t *index, const int8_t *level, const int32_t *parent
  *                      row (zero outside the subset)
  *   lse                device float [heads, total_q]
  *   workspace          device, >= hdt_cross_workspace_bytes(batch, total_tokens, total_q, heads,
- *                      head_dim, dtype, bwd), 256-byte aligned; holds the list of chosen tokens,
- *                      rebuilt by every call, and (bf16) fp32 results per element before they are
- *                      converted
+ *                      head_dim, dtype, bwd), 256-byte aligned; holds the list of chosen tokens and
+ *                      their block records, rebuilt by every call (and delta in the backward)
  * head_dim 64 or 128; softmax_scale <= 0 means 1/sqrt(head_dim).  Asynchronous on `stream`, no
  * host wait.  The chosen rows are read in place through the list (no gathered copy of K, V).
  */

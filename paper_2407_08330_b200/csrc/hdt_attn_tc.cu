@@ -127,7 +127,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
     if constexpr (GATHER) {
         if (a.final_merge && inb) {
             fm_tk = a.tok[row];
-            fm_lb = a.carry_lse[(size_t)row * H + h];
+            if (a.carry_lse != nullptr) fm_lb = a.carry_lse[(size_t)row * H + h];
             if (a.next_own_o != nullptr) {
                 fm_e2 = a.up[row];
                 if (fm_e2 >= 0) fm_lu = a.next_own_lse[(size_t)fm_e2 * H + h];
@@ -317,7 +317,7 @@ __global__ void __launch_bounds__(128) k_fwd_tc(const __grid_constant__ CUtensor
             const float *pb = nullptr, *pu = nullptr;
             const int tk = fm_tk;
             if (inb) {
-                pb = a.carry_o + ((size_t)row * H + h) * D;
+                if (a.carry_o != nullptr) pb = a.carry_o + ((size_t)row * H + h) * D;
                 if (fm_e2 >= 0) pu = a.next_own_o + ((size_t)fm_e2 * H + h) * D;
             }
             const float mx = fmaxf(fmaxf(lse, lb), lu);
@@ -1550,7 +1550,8 @@ static int launch_fwd_tc_upper_t(const FwdStageArgs &a, cudaStream_t st) {
 int launch_fwd_tc_upper(const FwdStageArgs &a, int D, cudaStream_t st) {
     if (a.nb == 0) return HDT_OK;
     if (a.tok == nullptr || (!a.final_merge && (a.own_o == nullptr || a.own_lse == nullptr)) ||
-        (a.final_merge && (a.carry_o == nullptr || a.carry_lse == nullptr)))
+        (a.final_merge == 1 && (a.carry_o == nullptr || a.carry_lse == nullptr)) ||
+        (a.final_merge == 2 && (a.carry_o != nullptr || a.next_own_o != nullptr || a.o == nullptr || a.lse == nullptr)))
         return set_error(HDT_ERR_INVALID_ARG, "launch_fwd_tc_upper: needs a tok map and own-partial (or carry) buffers");
     if (D == 64) return launch_fwd_tc_upper_t<64>(a, st);
     if (D == 128) return launch_fwd_tc_upper_t<128>(a, st);

@@ -386,7 +386,7 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
             float x[32];
 #pragma unroll
             for (int j = 0; j < 32; j += 4) {
-                const float4 y = *reinterpret_cast<const float4 *>(base + c0 + j);
+                const float4 y = base != nullptr ? *reinterpret_cast<const float4 *>(base + c0 + j) : make_float4(0.f, 0.f, 0.f, 0.f);
                 x[j] = fmaf(__uint_as_float(r[j]), scale, y.x);
                 x[j + 1] = fmaf(__uint_as_float(r[j + 1]), scale, y.y);
                 x[j + 2] = fmaf(__uint_as_float(r[j + 2]), scale, y.z);
@@ -446,10 +446,13 @@ __global__ void __launch_bounds__(256) k_bwd_tc(const __grid_constant__ CUtensor
         if (fin && inb) {
             const size_t tk = (size_t)a.tok[row];
             const size_t ob = ((size_t)row * H + h) * D;
-            fb[0] = a.carry_dq + ob; fb[1] = a.carry_dk + ob; fb[2] = a.carry_dv + ob;
-            fo[0] = reinterpret_cast<__nv_bfloat16 *>(a.dq) + (tk * H + h) * D;
-            fo[1] = reinterpret_cast<__nv_bfloat16 *>(a.dk) + (tk * H + h) * D;
-            fo[2] = reinterpret_cast<__nv_bfloat16 *>(a.dv) + (tk * H + h) * D;
+            if (a.final_merge == 1) { fb[0] = a.carry_dq + ob; fb[1] = a.carry_dk + ob; fb[2] = a.carry_dv + ob; }
+            // (final_merge = 2: nothing to add; a launch that walks one side only writes that side's gradients only)
+            if (a.final_merge == 1 || a.phases != 2) fo[0] = reinterpret_cast<__nv_bfloat16 *>(a.dq) + (tk * H + h) * D;
+            if (a.final_merge == 1 || a.phases != 1) {
+                fo[1] = reinterpret_cast<__nv_bfloat16 *>(a.dk) + (tk * H + h) * D;
+                fo[2] = reinterpret_cast<__nv_bfloat16 *>(a.dv) + (tk * H + h) * D;
+            }
             if (a.next_own_dq != nullptr) {
                 const int e2 = a.up[row];
                 if (e2 >= 0) {
@@ -1414,7 +1417,8 @@ static int launch_bwd_tc_upper_t(const BwdStageArgs &a, cudaStream_t st) {
 int launch_bwd_tc_upper(const BwdStageArgs &a, int D, cudaStream_t st) {
     if (a.nb == 0) return HDT_OK;
     if (a.tok == nullptr || (!a.final_merge && (a.own_dq == nullptr || a.own_dk == nullptr || a.own_dv == nullptr)) ||
-        (a.final_merge && (a.carry_dq == nullptr || a.carry_dk == nullptr || a.carry_dv == nullptr)))
+        (a.final_merge == 1 && (a.carry_dq == nullptr || a.carry_dk == nullptr || a.carry_dv == nullptr)) ||
+        (a.final_merge == 2 && (a.next_own_dq != nullptr || a.dq == nullptr || a.dk == nullptr || a.dv == nullptr)))
         return set_error(HDT_ERR_INVALID_ARG, "launch_bwd_tc_upper: needs a tok map and own-gradient (or carry) buffers");
     if (D == 64) return launch_bwd_tc_upper_t<64>(a, st);
     if (D == 128) return launch_bwd_tc_upper_t<128>(a, st);

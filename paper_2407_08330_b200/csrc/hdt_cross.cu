@@ -13,8 +13,8 @@
 // description, so they serve as they are:
 //   bf16  the gathering tcgen05 kernels (128-row blocks): forward over the decoder-row blocks;
 //         backward once over the decoder-row blocks (dQ) and once over the blocks of chosen
-//         tokens (dK, dV); they leave fp32 results per element, which small kernels convert and
-//         scatter to the caller's tensors;
+//         tokens (dK, dV); their epilogues round to bf16 and write each element's rows at its token in
+//         the caller's tensors (no fp32 buffers, no convert pass);
 //   fp32  the SIMT kernels (32-row blocks), which write the caller's tensors directly.
 // Encoder rows outside the subset get zero dK, dV (cleared first).  Block slots are assigned
 // without a scan: document b owns the slots from start / rows_per_block + b on, unused slots stay
@@ -28,14 +28,14 @@ namespace hdt {
 constexpr int XC = 32;      // CTAs (contiguous chunks) per document in the selection kernels
 
 struct CrossLayout {
-    size_t cnt, cntc, cu_sel, tokx, rngx, blocks_q, blocks_k, queue, delta, own[5], total;
+    size_t cnt, cntc, cu_sel, tokx, rngx, blocks_q, blocks_k, queue, delta, total;
     int nbq, nbk, xr;
     size_t zero_bytes;      // cnt .. tokx is cleared at the start of every call
 };
 
 static size_t al256c(size_t v) { return (v + 255) & ~size_t(255); }
 
-// tc: bf16 on the tensor-core kernels (fp32 per-element results in the workspace)
+// tc: bf16 on the tensor-core kernels (128-row blocks)
 static CrossLayout cross_layout(int B, int T, int Tq, int H, int D, bool tc, int bwd) {
     CrossLayout L{};
     L.xr = tc ? 128 : 32;
@@ -53,17 +53,6 @@ static CrossLayout cross_layout(int B, int T, int Tq, int H, int D, bool tc, int
     L.rngx = o; o += al256c(sizeof(int) * 2 * max(n, (size_t)1));
     L.queue = o; o += al256c(sizeof(int) * (size_t)max(L.nbq, L.nbk));
     L.delta = o; if (bwd) o += al256c(sizeof(float) * (size_t)H * max(Tq, 1));
-    if (tc) {
-        const size_t rq = sizeof(float) * (size_t)max(Tq, 1) * H, rk = sizeof(float) * (size_t)max(T, 1) * H;
-        if (!bwd) {
-            L.own[0] = o; o += al256c(rq * D);      // O
-            L.own[1] = o; o += al256c(rq);          // LSE
-        } else {
-            L.own[2] = o; o += al256c(rq * D);      // dQ
-            L.own[3] = o; o += al256c(rk * D);      // dK
-            L.own[4] = o; o += al256c(rk * D);      // dV
-        }
-    }
     L.total = o + 256;
     return L;
 }
@@ -175,42 +164,6 @@ __global__ void __launch_bounds__(256) k_cross_fill(const int8_t *__restrict__ l
     }
 }
 
-// fp32 per-element results [n, H, D] of the tensor-core kernels -> bf16 rows of the caller's tensor:
-// element e goes to row map[e] (e itself without a map); count: device counter of the elements, or
-// null for n.  One thread per 8 values.  lse_src [n, H] -> lse_dst [H, n_rows] on the side.
-template <int D>
-__global__ void k_cross_cvt(const float *__restrict__ src, __nv_bfloat16 *dst, const int *__restrict__ map, int n,
-                            const int *__restrict__ count, int H, const float *__restrict__ lse_src, float *lse_dst,
-                            int lse_rows) {
-    constexpr int G = D / 8;
-    const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const int m = count ? min(n, *count) : n;
-    const long long e = gid / ((long long)H * G);
-    if (e >= m) return;
-    const int h = (int)((gid / G) % H), g = (int)(gid % G);
-    const float4 *p = reinterpret_cast<const float4 *>(src + ((size_t)e * H + h) * D + 8 * g);
-    const float4 x = p[0], y = p[1];
-    const int row = map ? map[e] : (int)e;
-    uint4 out;
-    __nv_bfloat162 *o2 = reinterpret_cast<__nv_bfloat162 *>(&out);
-    o2[0] = __floats2bfloat162_rn(x.x, x.y); o2[1] = __floats2bfloat162_rn(x.z, x.w);
-    o2[2] = __floats2bfloat162_rn(y.x, y.y); o2[3] = __floats2bfloat162_rn(y.z, y.w);
-    *reinterpret_cast<uint4 *>(dst + ((size_t)row * H + h) * D + 8 * g) = out;
-    if (lse_src != nullptr && g == 0) lse_dst[(size_t)h * lse_rows + row] = lse_src[(size_t)e * H + h];
-}
-
-static int cross_cvt(const float *src, void *dst, const int *map, int n, const int *count, int H, int D,
-                     const float *lse_src, float *lse_dst, int lse_rows, cudaStream_t st) {
-    if (n == 0) return HDT_OK;
-    const long long threads = (long long)n * H * (D / 8);
-    const unsigned grid = (unsigned)((threads + 255) / 256);
-    if (D == 64) k_cross_cvt<64><<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, map, n, count, H, lse_src, lse_dst, lse_rows);
-    else k_cross_cvt<128><<<grid, 256, 0, st>>>(src, (__nv_bfloat16 *)dst, map, n, count, H, lse_src, lse_dst, lse_rows);
-    count_launch();
-    HDT_CUDA_CHECK(cudaGetLastError());
-    return HDT_OK;
-}
-
 static int cross_build(const CrossLayout &L, char *ws, const int8_t *level, const int32_t *cu_k, const int32_t *cu_q,
                        int B, int Tq, int level_mask, cudaStream_t st) {
     // the token map is cleared as a whole: tiles of the gathering kernels reach past the elements
@@ -285,11 +238,8 @@ extern "C" int hdt_cross_attn_fwd(const int8_t *level, const int32_t *cu_seqlens
     a.status = device_status_ptr();
     a.block_rows = L.xr; a.dirs = 7;
     if (!tc) return launch_fwd_simt(a, head_dim, dtype, st);
-    a.own_o = (float *)(ws + L.own[0]);
-    a.own_lse = (float *)(ws + L.own[1]);
-    rc = launch_fwd_tc_upper(a, head_dim, st);
-    if (rc) return rc;
-    return cross_cvt(a.own_o, o, nullptr, total_q, nullptr, heads, head_dim, a.own_lse, lse, total_q, st);
+    a.final_merge = 2;       // the kernel's epilogue writes the bf16 rows and the LSE of the decoder rows itself
+    return launch_fwd_tc_upper(a, head_dim, st);
 }
 
 extern "C" int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens_k, const int32_t *cu_seqlens_q,
@@ -322,7 +272,6 @@ extern "C" int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens
     rc = launch_delta(o, d_o, delta, total_q, heads, head_dim, dtype, st);
     if (rc) return rc;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / sqrtf((float)head_dim);
-    const int KO = total_q;
     BwdStageArgs a{};
     a.n = total_q + total_tokens; a.H = heads; a.T = total_q;
     a.tok = (const int *)(ws + L.tokx); a.tok_rows = a.tok;
@@ -343,19 +292,10 @@ extern "C" int hdt_cross_attn_bwd(const int8_t *level, const int32_t *cu_seqlens
         if (rc) return rc;
         return launch_bwd_simt(ak, head_dim, dtype, st);
     }
-    float *own_dq = (float *)(ws + L.own[2]), *own_dk = (float *)(ws + L.own[3]), *own_dv = (float *)(ws + L.own[4]);
-    aq.own_dq = own_dq; aq.own_dk = own_dk; aq.own_dv = own_dv;           // only dQ is written (phases = 1)
-    // the chosen tokens are elements KO ..: their results land at position e - KO of the buffers
-    const size_t shift = (size_t)KO * heads * head_dim;
-    ak.own_dq = own_dq; ak.own_dk = own_dk - shift; ak.own_dv = own_dv - shift;
+    // the epilogues write bf16 rows at the element's token: dq from the first launch (decoder rows, token =
+    // row), dk and dv from the second (chosen tokens, token = their encoder row)
+    aq.final_merge = 2; ak.final_merge = 2;
     rc = launch_bwd_tc_upper(aq, head_dim, st);
     if (rc) return rc;
-    rc = launch_bwd_tc_upper(ak, head_dim, st);
-    if (rc) return rc;
-    rc = cross_cvt(own_dq, dq, nullptr, total_q, nullptr, heads, head_dim, nullptr, nullptr, 0, st);
-    if (rc) return rc;
-    const int *sel = (const int *)(ws + L.tokx) + KO, *ns = (const int *)(ws + L.cu_sel) + batch;
-    rc = cross_cvt(own_dk, dk, sel, total_tokens, ns, heads, head_dim, nullptr, nullptr, 0, st);
-    if (rc) return rc;
-    return cross_cvt(own_dv, dv, sel, total_tokens, ns, heads, head_dim, nullptr, nullptr, 0, st);
+    return launch_bwd_tc_upper(ak, head_dim, st);
 }

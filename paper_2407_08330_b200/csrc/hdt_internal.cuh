@@ -190,6 +190,8 @@ struct FwdStageArgs {
     // partial result it completes every element of the stage: its own result, stage 0's partial
     // (carry_*) and, for elements that live on in stage 2, that stage's own partial (next_own_*,
     // at up[e]; nullptr without a stage 2) are merged and written to o / lse at the element's token.
+    // final_merge = 2: the stage's own result is the element's result (nothing to merge; cross-attention):
+    // bf16 rows and LSE straight to the element's token, no partial buffers.
     int final_merge;
     const float *next_own_o, *next_own_lse;
     const DevHeader *hdr; // set: the index build is still in flight; the looping kernel reads n_fused and stage 1's size here
@@ -223,6 +225,8 @@ struct BwdStageArgs {
     // Gathering kernel, stage 1 run after stage 0 (final_merge = 1): the element's gradients are its
     // own plus stage 0's partials (carry_*) plus, for elements that live on in stage 2, that stage's
     // own (next_own_*, at up[e]; nullptr without a stage 2); they go to dq / dk / dv at its token.
+    // final_merge = 2: the element's own gradients alone, straight to its token's rows (cross-attention;
+    // with phases = 1 only dq, with phases = 2 only dk and dv are written).
     int final_merge;
     const float *next_own_dq, *next_own_dk, *next_own_dv;
     float *dq_acc;                                // stage 0, head_dim 64: fp32 [T,H,64] buffer, zero on entry, that the one-walk kernel of the
