@@ -246,8 +246,8 @@ int hdt_attn_fwd_static(const hdt_index_t *index, const void *q, const void *k, 
  * level-l ancestor (or of the token itself) among its siblings, and 0 on levels deeper than the
  * token's own.  The root has p = 0 on every level; PAD tokens get 0 (accumulate = 0) or are left
  * unchanged (accumulate = 1).
- *   index              built from the same level / parent / cu_seqlens (its stages give the
- *                      sibling numbers)
+ *   index              built from the same level / parent / cu_seqlens (the build leaves every
+ *                      token's number among its siblings in the index workspace)
  *   x                  device [total_tokens, d_model] of `dtype`; overwritten (accumulate = 0) or
  *                      incremented (accumulate = 1: token embeddings + HPE, as the encoder input)
  *   workspace          device, >= hdt_hpe_workspace_bytes(index, n_levels), 256-byte aligned

@@ -4,33 +4,14 @@
 // below an anchor's own level and for the root), and
 //     HPE(p, 2k) = sum_l sin(w_k p^l),  HPE(p, 2k+1) = sum_l cos(w_k p^l),  w_k = 10000^(-2k/d_model).
 // The sibling numbers come for free from the staged index: in the stage where a node is handled as
-// a child of its family, its number is its distance from the family head.
+// a child of its family, its number is its distance from the family head; the index build writes it
+// (hdt_index::rank) where it finds the family.
 #include <cuda_bf16.h>
 
 #include "hdt_internal.cuh"
 #include "hdt_sm100.cuh"
 
 namespace hdt {
-
-struct HpeStages {
-    int n_stages;
-    int n[HDT_MAX_STAGES];
-    const int *tok[HDT_MAX_STAGES], *par[HDT_MAX_STAGES], *rng[HDT_MAX_STAGES];
-};
-
-// rank[token] = sibling number (1-based) of every element that is a family child in its stage.
-// Every node below the root is a family child in exactly one stage, so all entries that
-// k_hpe_pvec reads are written here.
-__global__ void k_hpe_rank(HpeStages S, int *rank) {
-    for (int s = 0; s < S.n_stages; ++s) {
-        const int n = S.n[s];
-        const int *__restrict__ tok = S.tok[s], *__restrict__ par = S.par[s], *__restrict__ rng = S.rng[s];
-        for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
-            const int lo = rng[2 * e], hi = rng[2 * e + 1], p = par[e];
-            if (hi > lo && p >= 0 && lo == p) rank[tok[e]] = e - lo;
-        }
-    }
-}
 
 // pvec[token, l-1] = p^l: walk up from the token, one ancestor per level
 __global__ void k_hpe_pvec(const int8_t *__restrict__ level, const int32_t *__restrict__ parent,
@@ -361,7 +342,7 @@ static size_t al256h(size_t v) { return (v + 255) & ~size_t(255); }
 extern "C" size_t hdt_hpe_workspace_bytes(const hdt_index_t *ix, int32_t n_levels) {
     if (!ix || n_levels < 1 || n_levels > 32) return 0;
     const size_t T = (size_t)ix->total_tokens;
-    return al256h(sizeof(int) * T) + al256h(sizeof(int) * T * n_levels) + 256;
+    return al256h(sizeof(int) * T * n_levels) + 256;
 }
 
 extern "C" int hdt_hpe(const hdt_index_t *ix, const int8_t *level, const int32_t *parent, const int32_t *cu_seqlens,
@@ -381,20 +362,8 @@ extern "C" int hdt_hpe(const hdt_index_t *ix, const int8_t *level, const int32_t
     if (((uintptr_t)workspace & 255) || ((uintptr_t)x & 7))
         return set_error(HDT_ERR_INVALID_ARG, "hdt_hpe: workspace must be 256-byte, x 8-byte aligned");
     cudaStream_t st = (cudaStream_t)stream;
-    int *rank = (int *)workspace;
-    int *pvec = (int *)((char *)workspace + al256h(sizeof(int) * (size_t)T));
-    HpeStages S;
-    S.n_stages = ix->n_stages;
-    int n_max = 0;
-    for (int s = 0; s < ix->n_stages; ++s) {
-        S.n[s] = ix->desc[s].n;
-        S.tok[s] = ix->st[s].tok;
-        S.par[s] = ix->st[s].par;
-        S.rng[s] = ix->st[s].rng;
-        n_max = max(n_max, S.n[s]);
-    }
-    k_hpe_rank<<<max(1, min((n_max + 255) / 256, 148 * 8)), 256, 0, st>>>(S, rank);
-    count_launch();
+    const int *rank = ix->rank;
+    int *pvec = (int *)workspace;
     k_hpe_pvec<<<(T + 255) / 256, 256, 0, st>>>(level, parent, cu_seqlens, B, T, n_levels, rank, pvec);
     count_launch();
     const bool x16 = ((uintptr_t)x & 15) == 0;

@@ -25,6 +25,7 @@ static constexpr int CHUNK = 1024;  // elements per CTA in the element-wise kern
 struct Layout {
     size_t header, cnt, nlc, pre, keep, fpos, blocksum, bstart, seqcount, cost, stage0, stage_stride;
     size_t fpos2, bstart2, seqcount2, cost2;   // second set for the upper stages, built beside stage 0's blocks
+    size_t rank;                               // per token: its number among its siblings (written where its family is found)
     size_t s_tok, s_par, s_rng, s_up, s_scu, s_blocks, s_queue, s_queue2;  // offsets inside a stage
     size_t total;
     int capnb, nchunk;
@@ -51,6 +52,7 @@ static Layout make_layout(int B, int T, int bm, int max_stages) {   // bm: the s
     L.bstart2 = o; o += al(sizeof(int) * (size_t)L.capnb);
     L.seqcount2 = o; o += al(sizeof(int) * (size_t)(B + 1));
     L.cost2 = o; o += al(sizeof(long long) * (size_t)L.capnb);
+    L.rank = o; o += al(sizeof(int) * (size_t)T);
     L.stage0 = o;
     size_t s = 0;
     L.s_tok = s; s += al(sizeof(int) * (size_t)T);
@@ -153,7 +155,8 @@ __device__ __forceinline__ int row_pairs(int e, int lo, int hi, int dirs) {
 __global__ void __launch_bounds__(CHUNK)
 k_ranges(DevHeader *hdr, int s, const int8_t *__restrict__ level /* stage 0 only */,
          const int *__restrict__ par, const int *__restrict__ cnt, const int *__restrict__ nlc,
-         int *rng, uint8_t *keep, uint8_t *fpos, int *blocksum, int dirs) {
+         int *rng, uint8_t *keep, uint8_t *fpos, int *blocksum, int dirs, const int *__restrict__ tok /* nullptr: identity */,
+         int *rank) {
     pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
     pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
@@ -177,6 +180,7 @@ k_ranges(DevHeader *hdr, int s, const int8_t *__restrict__ level /* stage 0 only
                 hi = p + 1 + cp;
                 fp = min(e - p, 255);
                 kp = 0;
+                rank[tok ? tok[e] : e] = e - p;     // the token's number among its siblings (hierarchical positions)
             }
         }
         rng[2 * e] = lo;
@@ -471,7 +475,7 @@ k_queue(DevHeader *hdr, int s, const long long *__restrict__ cost, const int *__
 struct UpperArgs {
     StagePtrs st[HDT_MAX_STAGES];
     int max_stages, B, bm, dirs;
-    int *cnt, *nlc, *pre, *bstart, *seqcount;
+    int *cnt, *nlc, *pre, *bstart, *seqcount, *rank;
     uint8_t *keep, *fpos;
     long long *cost;
 };
@@ -536,6 +540,7 @@ __global__ void __launch_bounds__(UT) k_upper_stages(DevHeader *hdr, const Upper
                 if (cp > 0 && nlc[p] == 0) {
                     if (!(p < e && e <= p + cp)) dev_fail(hdr, HDT_ERR_BAD_HIERARCHY, e);
                     lo = p; hi = p + 1 + cp; fp = min(e - p, 255); kp = 0;
+                    u.rank[tokr[e]] = e - p;
                 }
             }
             P.rng[2 * e] = lo;
@@ -821,6 +826,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     ix->batch = B; ix->total_tokens = T; ix->block_m = bm; ix->block_m_upper = bmu; ix->n_stages = 0;
     ix->directions = dirs;
     ix->workspace = workspace; ix->workspace_bytes = workspace_bytes;
+    ix->rank = (const int *)(ws + L.rank);
     for (int s = 0; s < ms; ++s) {
         char *base = ws + L.stage0 + L.stage_stride * (size_t)s;
         ix->st[s] = StagePtrs{(int *)(base + L.s_tok), (int *)(base + L.s_par), (int *)(base + L.s_rng),
@@ -874,6 +880,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             u.cnt = cnt; u.nlc = nlc; u.pre = pre; u.keep = keep;
             u.bstart = (int *)(ws + L.bstart2); u.seqcount = (int *)(ws + L.seqcount2);
             u.fpos = (uint8_t *)(ws + L.fpos2); u.cost = (long long *)(ws + L.cost2);
+            u.rank = (int *)(ws + L.rank);
             k_upper_stages<<<1, UT, USMEM, s_>>>(hdr, u);
             ++n_launched;
         };
@@ -889,7 +896,7 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
             const bool last = (s + 1 == ms);
             if (s >= 1) { HDT_ENQ(launch_chain(k_count, dim3(g_stride), dim3(256), 0, st, hdr, s, P.par, cnt, nlc)); ++n_launched; }
             HDT_ENQ(launch_chain(k_ranges, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, s == 0 ? level : (const int8_t *)nullptr, P.par, cnt, nlc,
-                                 P.rng, keep, fpos, blocksum, dirs));
+                                 P.rng, keep, fpos, blocksum, dirs, s == 0 ? (const int *)nullptr : (const int *)P.tok, (int *)(ws + L.rank)));
             // tok2 of the last possible stage is never read: point it at scratch (pre is rewritten first)
             HDT_ENQ(launch_chain(k_scan, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
                                  last ? cnt : N.tok));

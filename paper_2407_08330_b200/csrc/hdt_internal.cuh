@@ -42,6 +42,7 @@ struct hdt_index {
     hdt::StagePtrs st[HDT_MAX_STAGES];
     void *workspace;
     size_t workspace_bytes;
+    const int *rank;                  // device [total_tokens]: a token's number among its siblings (undefined for roots and PAD)
     // Deferred build: the device header is on its way to h_pinned; hdt::index_ready() waits for it
     // and fills n_stages, nnz, visited and desc.
     int pending;                      // 1 until the header has been read
