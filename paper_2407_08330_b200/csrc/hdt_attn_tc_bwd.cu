@@ -1238,10 +1238,32 @@ __global__ void __launch_bounds__(512, 1) k_bwd_tc_p(const __grid_constant__ CUt
 // is the sum in a.dq_acc times the softmax scale; it goes to dq as bf16 and, for rows that live on in
 // the next stage, as fp32 to that stage's buffer.  One CTA per (block after the first n_fused of
 // queue_split, head); thread t: 16-byte pieces t, t + 256, ... of the block's [rows x 64] fp32 tile.
-__global__ void __launch_bounds__(256) k_dq_finish(const BwdStageArgs a) {
+// zero_empty: the rows of EMPTY blocks (no key in this stage: PAD, lone roots) get their zero gradients here too,
+// also in the next stage's buffers for rows that live on (else the kernel before this one has written them).
+__global__ void __launch_bounds__(256) k_dq_finish(const BwdStageArgs a, int zero_empty) {
     const int *rec = a.blocks + 5 * (size_t)a.queue_split[a.n_fused + blockIdx.x];
     const int r0 = rec[0], nrows = rec[1] - r0, h = blockIdx.y, H = a.H;
-    if (rec[4] & HDT_BLK_EMPTY) return;          // written as zeros by the one-walk kernel
+    if (rec[4] & HDT_BLK_EMPTY) {
+        if (!zero_empty) return;
+        const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+        __nv_bfloat16 *g[3] = {(__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv};
+        float *pt[3] = {a.part_dq, a.part_dk, a.part_dv};
+        for (int i = threadIdx.x; i < nrows * 8; i += 256) {      // 16 bytes of a row and tensor per step
+            const int r = i >> 3, c = i & 7;
+            const size_t row = (size_t)(r0 + r);
+            const int u = a.part_dq != nullptr ? a.up[row] : -1;
+#pragma unroll
+            for (int t = 0; t < 3; ++t) {
+                *reinterpret_cast<uint4 *>(g[t] + (row * H + h) * 64 + 8 * c) = z;
+                if (u >= 0) {
+                    float4 *c4 = reinterpret_cast<float4 *>(pt[t] + ((size_t)u * H + h) * 64 + 8 * c);
+                    c4[0] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    c4[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+        return;
+    }
     for (int i = threadIdx.x; i < nrows * 16; i += 256) {
         const int r = i >> 4, c = i & 15;
         const size_t row = (size_t)(r0 + r);
@@ -1328,14 +1350,14 @@ static int launch_bwd_tc_t(const BwdStageArgs &a, cudaStream_t st) {
                 if (rc) return rc;
                 BwdStageArgs f = c;
                 f.scale = 1.f;      // (this kernel's sums carry softmax_scale already: it is in dS)
-                k_dq_finish<<<dim3(a.nb - a.n_fused, a.H), 256, 0, st>>>(f);
+                k_dq_finish<<<dim3(a.nb - a.n_fused, a.H), 256, 0, st>>>(f, 1);      // (and the EMPTY blocks' zero rows)
             } else if (mode && onewalk) {
                 if (dirs) k_bwd_tc_p<2, true><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);
                 else k_bwd_tc_p<2><<<grid_p, 512, smem_w, st>>>(tq, tk, tv, tdo, outs, tacc, c);
                 count_launch();
                 HDT_CUDA_CHECK(cudaGetLastError());
                 const int n_rest = a.nb - a.n_fused;
-                k_dq_finish<<<dim3(n_rest, a.H), 256, 0, st>>>(c);
+                k_dq_finish<<<dim3(n_rest, a.H), 256, 0, st>>>(c, 0);
             } else if (dirs) {
                 if (mode) k_bwd_tc_p<1, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, tacc, c);
                 else k_bwd_tc_p<0, true><<<grid_p, 512, smem_p, st>>>(tq, tk, tv, tdo, outs, tacc, c);

@@ -135,7 +135,7 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     const bool marks = MARKS && blockIdx.x == 0 && (warp == 0 || warp == 8 || warp == W_DRAIN || warp >= W_LOAD);
     if (MARKS && tid < 80) s_marks[tid] = 0;
     // EMPTY blocks cost nothing in the queue's order, so they are the tail of queue_split and are left
-    // out here (k_bwd_zero_empty writes their rows)
+    // out here (k_dq_finish writes their rows)
     const int n_units = (a.nb - a.n_fused - a.n_empty) * H;
 
     if ((smem_u32(smem_raw) & 1023u) != 0u) {      // the swizzled tiles need 1024-byte alignment
@@ -653,31 +653,6 @@ __global__ void __launch_bounds__(736, 1) k_bwd_tc_w(const __grid_constant__ CUt
     if (warp == 0) tmem_dealloc(tmem, TM_COLS);
 }
 
-// EMPTY blocks among those after the first n_fused of queue_split (rows without any key in this
-// stage: PAD, lone roots): zero gradients, also in the next stage's buffers for rows that live on.
-// One CTA of 128 threads per (block, head) over the last blocks of queue_split, from entry n_fused + first; thread t: row t.
-__global__ void __launch_bounds__(128) k_bwd_zero_empty(const BwdStageArgs a, int first) {
-    const int *rec = a.blocks + 5 * (size_t)a.queue_split[a.n_fused + first + blockIdx.x];
-    if (!(rec[4] & HDT_BLK_EMPTY)) return;
-    const int row = rec[0] + (int)threadIdx.x, h = blockIdx.y, H = a.H;
-    if (row >= rec[1]) return;
-    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
-    __nv_bfloat16 *g[3] = {(__nv_bfloat16 *)a.dq, (__nv_bfloat16 *)a.dk, (__nv_bfloat16 *)a.dv};
-    float *pt[3] = {a.part_dq, a.part_dk, a.part_dv};
-    const int up = a.part_dq != nullptr ? a.up[row] : -1;
-#pragma unroll
-    for (int t = 0; t < 3; ++t) {
-        uint4 *o = reinterpret_cast<uint4 *>(g[t] + ((size_t)row * H + h) * 64);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) o[c] = z;
-        if (up >= 0) {
-            float4 *c4 = reinterpret_cast<float4 *>(pt[t] + ((size_t)up * H + h) * 64);
-#pragma unroll
-            for (int c = 0; c < 16; ++c) c4[c] = make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-    }
-}
-
 int read_bwd_w_marks(long long *out128) {
     HDT_CUDA_CHECK(cudaMemcpyFromSymbol(out128, g_bwd_w_marks, sizeof(long long) * 128));
     return HDT_OK;
@@ -711,12 +686,7 @@ int launch_bwd_tc_onewalk64(const BwdStageArgs &a, const CUtensorMap &tq, const 
     else k_bwd_tc_w<false><<<grid, 736, smem, st>>>(tq, tk, tv, tdo, outs, tacc, a);
     count_launch();
     HDT_CUDA_CHECK(cudaGetLastError());
-    if (n_empty > 0) {       // (EMPTY blocks cost nothing in the queue's order: they are the last n_empty of queue_split)
-        k_bwd_zero_empty<<<dim3(n_empty, a.H), 128, 0, st>>>(a, n_rest - n_empty);
-        count_launch();
-        HDT_CUDA_CHECK(cudaGetLastError());
-    }
-    return HDT_OK;
+    return HDT_OK;      // (the EMPTY blocks, the last n_empty of queue_split, get their zero rows from k_dq_finish)
 }
 
 }  // namespace hdt
