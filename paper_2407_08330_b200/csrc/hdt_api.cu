@@ -3,6 +3,7 @@
 #include <cstdarg>
 #include <cstdio>
 #include <cstring>
+#include <memory>
 #include <mutex>
 #include <vector>
 
@@ -83,6 +84,8 @@ int get_side(Side **out) {
     if (!sd.ready) {
         HDT_CUDA_CHECK(cudaStreamCreateWithFlags(&sd.s, cudaStreamNonBlocking));
         HDT_CUDA_CHECK(cudaStreamCreateWithFlags(&sd.s2, cudaStreamNonBlocking));
+        HDT_CUDA_CHECK(cudaStreamCreateWithFlags(&sd.s3, cudaStreamNonBlocking));
+        HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join3, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.fork, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join2, cudaEventDisableTiming));
@@ -262,6 +265,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
     // from the build straight into the attention.  The stream is forked first: what the host
     // launches on the side streams after its wait still runs beside that kernel, not behind it.
     bool early = false;
+    std::unique_ptr<ProfScope> ps_early;      // stage 0's time when a kernel goes ahead: from its start to the end of the stage's other kernel
     if (ix->pending && ix->total_tokens > 0 && dtype == HDT_BF16 && !g_force_simt && g_no_persistent == 0 &&
         !g_no_overlap && (workspace == nullptr || ((uintptr_t)workspace & 255) == 0)) {
         Side *sd = nullptr;
@@ -282,7 +286,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         a.status = status;
         a.dirs = ix->directions;
         a.part = 1;
-        ProfScope ps(PROF_FWD_STAGE0, st);
+        ps_early.reset(new ProfScope(PROF_FWD_STAGE0, st));
         rc = launch_fwd_tc(a, head_dim, st);
         if (rc) return rc;
         early = true;
@@ -334,7 +338,7 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         // looping kernel (measured: a batch of padded documents gains 7 %); where split families
         // dominate, one kernel after the other is faster (the skewed batch loses 3 % side by side).
         const bool rest_beside = early || (tc0 && 2 * (ix->desc[0].nb - ix->desc[0].n_fused - ix->desc[0].n_empty) <= ix->desc[0].nb);
-        const bool two = ix->n_stages > 2 || rest_beside;
+        const bool two = ix->n_stages > 2;
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
         // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
         // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
@@ -390,13 +394,15 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         if (rest_beside) {
             FwdStageArgs a = stage_args(0);
             a.part = 2;
-            // (profiled with stage 0 when the looping kernel went ahead: the two make up the stage)
-            ProfScope ps(PROF_FWD_STAGE0, sd->s2, early && a.nb > a.n_fused);
-            rc = launch_fwd_tc(a, head_dim, sd->s2);      // behind the (small) even stages, not behind stage 1
+            // On a stream of its own, queued after the stages above 0: their CTAs are dispatched first as SMs
+            // become free, and this kernel does not wait for any of them to finish.
+            HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s3, sd->fork, 0));
+            rc = launch_fwd_tc(a, head_dim, sd->s3);
             if (rc) return rc;
         }
         HDT_CUDA_CHECK(cudaEventRecord(sd->join, sd->s));
         if (two) HDT_CUDA_CHECK(cudaEventRecord(sd->join2, sd->s2));
+        if (rest_beside) HDT_CUDA_CHECK(cudaEventRecord(sd->join3, sd->s3));
         {   // stage 0 after the small side kernels are queued: they take their SM share first (the
             // stage-0 kernel would otherwise fill every SM and push them behind itself)
             FwdStageArgs a = stage_args(0);
@@ -410,8 +416,12 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         }
         if (ix->n_stages == 1) {             // (early only) nothing to merge: wait for the other blocks' kernel
             if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
+            if (rest_beside) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join3, 0));
+            ps_early.reset();
             return HDT_OK;
         }
+        if (rest_beside) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join3, 0));
+        ps_early.reset();                    // (stage 0 ends here: both of its kernels are done)
         HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join, 0));
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(st, sd->join2, 0));
         ProfScope ps(PROF_FWD_UPPER, st);
