@@ -45,3 +45,17 @@ def test_hpe_config_sizes():
     import paper_2407_08330_b200 as P
     run(P, gen.make_hierarchy(1), 768, 3, torch.float32)
     run(P, gen.make_hierarchy(5), 768, 3, torch.float32, max_stages=4)   # sibling numbers up to ~1000
+
+
+def test_hpe_sibling_numbers_from_every_index_path():
+    """The index build writes the sibling numbers that hdt_hpe reads: from the per-stage kernels (a
+    caller that allows more than 8 stages, or more than 1024 sequences) and from the one-CTA builder
+    of the upper stages with a stage in shared memory and with one too large for it."""
+    import paper_2407_08330_b200 as P
+    rng = np.random.default_rng(9)
+    deep = gen.pack([gen.layout_tree(gen.random_tree(rng, int(rng.integers(2, 7)), 5)) for _ in range(12)])
+    run(P, deep, 64, 6, torch.float32, max_stages=24)                   # per-stage kernels on every stage
+    many = gen.pack([gen.gen_fill(rng, int(rng.integers(3, 40)), (1, 3), (1, 3), (0, 6))[:2] for _ in range(1100)])
+    run(P, many, 32, 3, torch.float32, max_stages=4)                    # more sequences than the one-CTA builder takes
+    big = gen.pack([gen.gen_fill(rng, 30000, (4, 24), (3, 20), (2, 6)) for _ in range(2)])
+    run(P, big, 32, 3, torch.float32, max_stages=4)                     # stage 1 of about 10 000 elements: global scratch
