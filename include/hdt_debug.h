@@ -38,11 +38,9 @@ extern "C" {
  *                    1: two walks (one for dQ, one for dK and dV), no fp32 buffer; 2: the one walk
  *                    in the lock-step form of the two-walk kernel; 86: as 0, with the clock marks
  *                    that hdt_debug_bwd_w_marks and hdt_debug_bwd_w_tiles read back.
- *   "tc_deep"        1: hierarchies of more than three stages run the stages above 0 of bf16 calls on the
- *                    gathering tensor-core kernels too (faster; on deep random trees single gradient
- *                    entries then pass the 2e-2 bound by a few percent).
- *   "no_multi_upper" 1: the fp32 SIMT kernels take the stages above 0 of such hierarchies with a launch
- *                    per stage instead of one launch over the blocks of all of them.
+ *   "no_multi_upper" 1: where the fp32 SIMT kernels take the stages above 0 of a hierarchy of more than three
+ *                    stages (fp32 calls; bf16 with "simt_upper"), a launch per stage instead of one launch
+ *                    over the blocks of all of them.
  *   "no_self_beside" 1: in a backward with the one-walk kernel, the kernel of the self-contained stage-0 blocks
  *                    runs behind it on the caller's stream instead of beside it on an internal stream.
  *   "no_fused_delta" 1: the delta pass (rowsum(dO . O)) runs even where every backward kernel of the

@@ -72,7 +72,6 @@ int g_no_fwd_mc = 0;
 int g_no_pdl = 0;
 static int g_no_multi_upper = 0;
 static int g_no_self_beside = 0;
-static int g_tc_deep = 0;
 static int g_no_fused_delta = 0;
 static int g_no_fold = 0;
 
@@ -184,7 +183,6 @@ extern "C" int hdt_set_option(const char *name, int32_t value) {
     if (name && std::strcmp(name, "no_fwd_mc") == 0) { g_no_fwd_mc = value; return HDT_OK; }
     if (name && std::strcmp(name, "bwd_walk") == 0) { g_bwd_walk = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_multi_upper") == 0) { g_no_multi_upper = value; return HDT_OK; }
-    if (name && std::strcmp(name, "tc_deep") == 0) { g_tc_deep = value; return HDT_OK; }
     if (name && std::strcmp(name, "no_self_beside") == 0) { g_no_self_beside = value; return HDT_OK; }
     return set_error(HDT_ERR_INVALID_ARG, "hdt_set_option: unknown option");
 }
@@ -340,13 +338,10 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
         const bool rest_beside = early || (tc0 && 2 * (ix->desc[0].nb - ix->desc[0].n_fused - ix->desc[0].n_empty) <= ix->desc[0].nb);
         const bool two = ix->n_stages > 2;
         if (two) HDT_CUDA_CHECK(cudaStreamWaitEvent(sd->s2, sd->fork, 0));
-        // Stages above 0 of bf16 calls run on the gathering tensor-core kernels for documents (up to
-        // three stages).  Deeper trees keep the fp32 SIMT kernels there: every further stage on the
-        // tensor cores adds a bf16 rounding of P and dS to the elements it touches, and on random trees
-        // of depth 6 one gradient entry then passes the maximum-error bound (2.06e-2 against 2e-2; the
-        // mean error rises by a tenth).  Option "tc_deep" = 1 takes the tensor cores there all the same
-        // (the ListOps-shaped batch: 1.42 -> 1.24 ms a step).
-        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && (ix->n_stages <= 3 || g_tc_deep);
+        // Stages above 0 of bf16 calls run on the gathering tensor-core kernels, whatever the depth of the
+        // hierarchy (option "simt_upper" = 1: on the fp32 SIMT kernels, which take trees of more than three
+        // stages in one launch over the blocks of all those stages).
+        const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper;
         ChainArgs c{};
         c.n1 = ix->desc[1].n; c.H = heads; c.T = ix->total_tokens; c.n_stages = ix->n_stages; c.nt = 1;
         c.tok1 = ix->st[1].tok;
@@ -363,8 +358,10 @@ extern "C" int hdt_attn_fwd(const hdt_index_t *ix, const void *q, const void *k,
                             (long long)ix->desc[1].nb * heads <= 2LL * n_sm1;
         const bool fold = tc_upper && !(g_no_fold & 1) && (short1 || (g_no_fold & 2)) && ix->n_stages > 1 && ix->n_stages <= 3;
         FwdStageArgs a1{};
-        // (deep trees: the stages above 0 are independent in own-partial mode and small, and a launch per stage is
-        // mostly launch latency: one launch over the blocks of all of them)
+        // (deep trees on the SIMT kernels: the stages above 0 are independent in own-partial mode and small, and a
+        // launch per stage is mostly launch latency: one launch over the blocks of all of them.  The tensor-core
+        // kernels keep a launch per stage, odd and even stages on two streams: one launch over all their blocks
+        // takes every SM ahead of stage 0 and was slower, 1.253 against 1.234 ms on the expression trees.)
         const bool multi = !tc_upper && ix->n_stages > 3 && !g_no_multi_upper;
         MultiFwdArgs mf{};
         for (int s = 1; s < ix->n_stages; ++s) {
@@ -470,8 +467,8 @@ extern "C" int hdt_attn_bwd(const hdt_index_t *ix, const void *q, const void *k,
     int *status = device_status_ptr();
     if (!status) return HDT_ERR_CUDA;
     const bool overlap = ix->n_stages > 1 && !g_no_overlap;
-    // Stages above 0 of bf16 calls: gathering tensor-core kernels for up to three stages (see hdt_attn_fwd).
-    const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper && (ix->n_stages <= 3 || g_tc_deep);
+    // Stages above 0 of bf16 calls: the gathering tensor-core kernels (see hdt_attn_fwd).
+    const bool tc_upper = dtype == HDT_BF16 && !g_force_simt && !g_simt_upper;
     // No delta pass when every kernel of this call computes dO . O of its rows itself: stage 0
     // entirely on the looping kernels (the transposed one at head_dim 64, the fused five-MMA one at
     // head_dim 128; every block self-contained), the stages above it on the gathering tensor-core kernels.

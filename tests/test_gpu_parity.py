@@ -158,7 +158,7 @@ def test_index_rejects_bad_hierarchies(P):
 # ------------------------------------------------------------------------------------------
 # attention, small cases compared element by element
 # ------------------------------------------------------------------------------------------
-def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
+def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0, out_rounding=False):
     """bf16 runs three times: persistent + general tensor-core kernels, general tensor-core kernels
     only, SIMT kernels on every stage."""
     # default kernels; general tensor-core kernels only; persistent forward; SIMT everywhere
@@ -173,13 +173,16 @@ def run_case(P, b, H, d, dtype, seed, bwd=True, block_m=128, scale=0.0):
         for k_, v_ in opt.items():
             P.hdt_set_option(k_, v_)
         try:
-            _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale, bmu)
+            _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale, bmu, out_rounding)
         finally:
             for k_ in opt:
                 P.hdt_set_option(k_, 0)
 
 
-def _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale, block_m_upper=0):
+def _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale, block_m_upper=0, out_rounding=False):
+    """out_rounding: gradients beyond 2 in magnitude are expected, where the spacing of bf16 values alone is
+    2^-6 and more: the stored result may be off by half a bf16 ulp of the expected value on top of the
+    2e-2 that bounds the kernels' own error (element by element; tests/gpu_util.py)."""
     t = gen.make_tensors(seed, b.total_tokens, H, d, dtype)
     idx = P.hdt_build_index(*dev_struct(b), block_m=block_m, max_stages=8, block_m_upper=block_m_upper)
     q, k, v, do = (dev_tensor(t[n], dtype) for n in ("q", "k", "v", "do"))
@@ -192,9 +195,9 @@ def _run_case(P, b, H, d, dtype, seed, bwd, block_m, scale, block_m_upper=0):
         dq, dk, dv = P.hdt_attn_bwd(idx, q, k, v, o, lse, do, softmax_scale=scale)
         # the oracle differentiates its own forward; the GPU uses its stored (rounded) O for delta
         dq_r, dk_r, dv_r = oracle.backward(b.level, b.parent, b.cu_seqlens, t["q"], t["k"], t["v"], t["do"], scale=sc)
-        check_close(host(dq), dq_r, dtype, "dQ")
-        check_close(host(dk), dk_r, dtype, "dK")
-        check_close(host(dv), dv_r, dtype, "dV")
+        check_close(host(dq), dq_r, dtype, "dQ", out_rounding=out_rounding)
+        check_close(host(dk), dk_r, dtype, "dK", out_rounding=out_rounding)
+        check_close(host(dv), dv_r, dtype, "dV", out_rounding=out_rounding)
     P.hdt_device_status()
 
 
@@ -257,14 +260,18 @@ def test_generic_depth_trees(P):
     seqs = [gen.layout_tree(gen.random_tree(rng, int(rng.integers(2, 7)), 6, p_leaf=0.4)) for _ in range(12)]
     b = gen.pack(seqs)
     run_case(P, b, 2, 64, "f32", 21)
-    run_case(P, b, 2, 64, "bf16", 22)
-    # (more than three stages: the stages above 0 run in one launch; here with a launch per stage as well)
+    # (gradients reach 3 here: the stored bf16 result's own rounding, half an ulp of the expected value, is allowed
+    # on top of the 2e-2 of the kernels' arithmetic; the run includes the fp32 SIMT kernels above stage 0)
+    run_case(P, b, 2, 64, "bf16", 22, out_rounding=True)
+    # (more than three stages: the SIMT kernels take the stages above 0 in one launch; here with a launch per stage as well)
     P.hdt_set_option("no_multi_upper", 1)
+    P.hdt_set_option("simt_upper", 1)
     try:
         _run_case(P, b, 2, 64, "f32", 21, True, 128, 0.0)
         _run_case(P, b, 2, 64, "bf16", 22, True, 128, 0.0)
     finally:
         P.hdt_set_option("no_multi_upper", 0)
+        P.hdt_set_option("simt_upper", 0)
 
 
 def test_forward_is_deterministic_and_guard_bands_untouched(P):
