@@ -90,6 +90,7 @@ int get_side(Side **out) {
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join2, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.fork0, cudaEventDisableTiming));
         HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.join0, cudaEventDisableTiming));
+        for (int i = 0; i < 2 * HDT_MAX_STAGES; ++i) HDT_CUDA_CHECK(cudaEventCreateWithFlags(&sd.stage_ev[i], cudaEventDisableTiming));
         sd.ready = true;
     }
     *out = &sd;

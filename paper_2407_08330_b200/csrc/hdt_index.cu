@@ -127,20 +127,6 @@ __global__ void k_init(const int8_t *__restrict__ level, const int32_t *__restri
     }
 }
 
-// Child counts of a stage above 0, and nlc as in k_init (first child to register reports its parent).
-__global__ void k_count(const DevHeader *hdr, int s, const int *__restrict__ par, int *cnt, int *nlc) {
-    pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
-    pdl_wait();                   // the kernel before this one has completed
-    const int n = hdr->st[s].n;
-    for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
-        const int p = par[e];
-        if (p >= 0 && atomicAdd(&cnt[p], 1) == 0) {
-            const int pp = par[p];
-            if (pp >= 0) atomicAdd(&nlc[pp], 1);
-        }
-    }
-}
-
 // One CTA per CHUNK elements (needed for the per-chunk keep counts).
 // Keys of row e with range [lo, hi) that the direction bits keep.  A row whose range starts at or
 // after itself is the head of its family (the keys after it are its children); otherwise lo is
@@ -218,7 +204,8 @@ k_ranges(DevHeader *hdr, int s, const int8_t *__restrict__ level /* stage 0 only
 // Exclusive scan of keep[] (per-CTA offset = sum of the chunk counts before it), next-stage tok.
 __global__ void __launch_bounds__(CHUNK)
 k_scan(DevHeader *hdr, int s, int nchunk_cap, const uint8_t *__restrict__ keep,
-       const int *__restrict__ blocksum, const int *__restrict__ tok, int *pre, int *up, int *tok2) {
+       const int *__restrict__ blocksum, const int *__restrict__ tok, int *pre, int *up, int *tok2, int *cnt_clear,
+       int *nlc_clear) {
     pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
     pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n;
@@ -278,12 +265,16 @@ k_scan(DevHeader *hdr, int s, int nchunk_cap, const uint8_t *__restrict__ keep,
         const int u = (kp && has_next) ? excl : -1;
         up[e] = u;
         if (u >= 0) tok2[u] = tok[e];
+        // (this stage's counts are dead: cleared here where k_compact goes on to count the next stage's children)
+        if (cnt_clear != nullptr) { cnt_clear[e] = 0; nlc_clear[e] = 0; }
     }
 }
 
+// count_next: cnt and nlc were cleared by k_scan; the next stage's child counts (and nlc, as in k_init) are taken
+// here, where its parent indices are formed, instead of in a kernel of their own.
 __global__ void k_compact(const DevHeader *hdr, int s, int B, const int *__restrict__ par,
                           const int *__restrict__ up, const int *__restrict__ pre,
-                          const int *__restrict__ scu, int *par2, int *scu2, int *cnt, int *nlc) {
+                          const int *__restrict__ scu, int *par2, int *scu2, int *cnt, int *nlc, int count_next) {
     pdl_launch_dependents();      // the kernel queued behind this one may be scheduled now; it waits likewise
     pdl_wait();                   // the kernel before this one has completed
     const int n = hdr->st[s].n, n2 = hdr->st[s + 1].n;
@@ -292,10 +283,16 @@ __global__ void k_compact(const DevHeader *hdr, int s, int B, const int *__restr
         const int u = up[e];
         if (u >= 0) {
             const int p = par[e];
-            par2[u] = (p >= 0) ? pre[p] : -1;
+            const int q = (p >= 0) ? pre[p] : -1;
+            par2[u] = q;
+            if (count_next && n2 > 0 && q >= 0 && atomicAdd(&cnt[q], 1) == 0) {      // (a kept element's ancestors are kept)
+                const int pp = par[p];
+                if (pp >= 0) atomicAdd(&nlc[pre[pp]], 1);
+            }
         }
     }
-    for (int e = gtid; e < n2; e += gsz) { cnt[e] = 0; nlc[e] = 0; }
+    if (!count_next)
+        for (int e = gtid; e < n2; e += gsz) { cnt[e] = 0; nlc[e] = 0; }
     for (int b = gtid; b <= B; b += gsz) {
         const int x = scu[b];
         scu2[b] = (n2 > 0) ? ((x < n) ? pre[x] : n2) : 0;
@@ -860,7 +857,13 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
     // The upper stages only need stage 0's compaction; with their own scratch they are built on the
     // side stream while stage 0's blocks and queues are built on the caller's stream.
     Side *sd = nullptr;
-    if (fused_upper && ms > 1 && !g_no_overlap && get_side(&sd) != HDT_OK) sd = nullptr;
+    if (ms > 1 && !g_no_overlap && get_side(&sd) != HDT_OK) sd = nullptr;
+    // The per-stage kernels (deep trees, many sequences) as two chains: what the next stage waits for (counts,
+    // ranges, scan, compaction) on the caller's stream, the stage's blocks and queues (walk, block records,
+    // ranking), which nothing but the attention kernels reads, on the side stream behind the stage's compaction.
+    // The two share the family positions and the block scratch, so those alternate between two sets by stage
+    // parity, and stage s + 2 takes a set only when the walk of stage s has read it.
+    const bool piped = !fused_upper && sd != nullptr && ms > 1;
 
     // Everything the build enqueues; returns the first CUDA error.  Called directly or under
     // stream capture (see below).
@@ -890,36 +893,57 @@ extern "C" int hdt_build_index(const int8_t *level, const int32_t *parent, const
                 else launch_upper(st);
                 break;
             }
+            // (piped: the scratch set of this stage's parity)
+            const bool set2 = piped && (s & 1);
+            uint8_t *fpos_s = set2 ? (uint8_t *)(ws + L.fpos2) : fpos;
+            int *bstart_s = set2 ? (int *)(ws + L.bstart2) : bstart, *seqcount_s = set2 ? (int *)(ws + L.seqcount2) : seqcount;
+            long long *cost_s = set2 ? (long long *)(ws + L.cost2) : cost;
+            if (piped && s >= 2) HDT_ENQ(cudaStreamWaitEvent(st, sd->stage_ev[2 * (s - 2) + 1], 0));   // the walk of stage s - 2 has read fpos
             const StagePtrs &P = ix->st[s];
             // the last possible stage writes its (unused) next-stage arrays into its own up/pre scratch
             const StagePtrs &N = ix->st[(s + 1 < ms) ? s + 1 : s];
             const bool last = (s + 1 == ms);
-            if (s >= 1) { HDT_ENQ(launch_chain(k_count, dim3(g_stride), dim3(256), 0, st, hdr, s, P.par, cnt, nlc)); ++n_launched; }
+            // (a kernel chain per stage: the stage before counted this stage's children in its compaction)
             HDT_ENQ(launch_chain(k_ranges, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, s == 0 ? level : (const int8_t *)nullptr, P.par, cnt, nlc,
-                                 P.rng, keep, fpos, blocksum, dirs, s == 0 ? (const int *)nullptr : (const int *)P.tok, (int *)(ws + L.rank)));
+                                 P.rng, keep, fpos_s, blocksum, dirs, s == 0 ? (const int *)nullptr : (const int *)P.tok, (int *)(ws + L.rank)));
             // tok2 of the last possible stage is never read: point it at scratch (pre is rewritten first)
+            const bool chain = !fused_upper;     // (else the one-CTA builder counts for itself and expects cleared arrays)
             HDT_ENQ(launch_chain(k_scan, dim3(g_chunk), dim3(CHUNK), 0, st, hdr, s, L.nchunk, keep, blocksum, P.tok, pre, P.up,
-                                 last ? cnt : N.tok));
+                                 last ? cnt : N.tok, chain ? cnt : (int *)nullptr, chain ? nlc : (int *)nullptr));
             n_launched += 2;
             if (!last) {
-                HDT_ENQ(launch_chain(k_compact, dim3(g_stride), dim3(256), 0, st, hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc));
+                HDT_ENQ(launch_chain(k_compact, dim3(g_stride), dim3(256), 0, st, hdr, s, B, P.par, P.up, pre, P.scu, N.par, N.scu, cnt, nlc,
+                                     chain ? 1 : 0));
                 ++n_launched;
-                if (s == 0 && sd) {   // fork: the upper stages start now
+                if (s == 0 && sd && fused_upper) {   // fork: the upper stages start now
                     HDT_ENQ(cudaEventRecord(sd->fork, st));
                     HDT_ENQ(cudaStreamWaitEvent(sd->s, sd->fork, 0));
                     launch_upper(sd->s);
                     HDT_ENQ(cudaEventRecord(sd->join, sd->s));
                 }
             }
+            cudaStream_t sb = st;        // the stream of the stage's blocks and queues
+            if (piped) {
+                sb = sd->s;
+                HDT_ENQ(cudaEventRecord(sd->stage_ev[2 * s], st));
+                HDT_ENQ(cudaStreamWaitEvent(sb, sd->stage_ev[2 * s], 0));
+            }
             if (B > 0) {
                 int maxlen_smem = kSmemCap;  // sequences longer than this walk through global memory
                 const int bms = (s == 0) ? bm : bmu;
-                HDT_ENQ(launch_chain(k_walk, dim3(B), dim3(256), (size_t)kSmemCap, st, hdr, s, bms, P.scu, fpos, bstart, seqcount, maxlen_smem));
+                HDT_ENQ(launch_chain(k_walk, dim3(B), dim3(256), (size_t)kSmemCap, sb, hdr, s, bms, P.scu, fpos_s, bstart_s, seqcount_s, maxlen_smem));
+                if (piped) HDT_ENQ(cudaEventRecord(sd->stage_ev[2 * s + 1], sb));
                 const int gy = max(1, min(64, 2048 / max(B, 1)));   // enough CTAs to spread a few long sequences
-                HDT_ENQ(launch_chain(k_blocks, dim3(B, gy), dim3(256), 0, st, hdr, s, bms, B, P.scu, bstart, seqcount, P.rng, P.up, P.blocks, cost));
-                HDT_ENQ(launch_chain(k_queue, dim3(max(1, min(L.capnb / 8 + 1, 148 * 4))), dim3(256), 0, st, hdr, s, cost, P.blocks, P.queue, P.queue_split));
+                HDT_ENQ(launch_chain(k_blocks, dim3(B, gy), dim3(256), 0, sb, hdr, s, bms, B, P.scu, bstart_s, seqcount_s, P.rng, P.up, P.blocks, cost_s));
+                HDT_ENQ(launch_chain(k_queue, dim3(max(1, min(L.capnb / 8 + 1, 148 * 4))), dim3(256), 0, sb, hdr, s, cost_s, P.blocks, P.queue, P.queue_split));
                 n_launched += 3;
+            } else if (piped) {
+                HDT_ENQ(cudaEventRecord(sd->stage_ev[2 * s + 1], sb));
             }
+        }
+        if (piped) {      // the side chain joins the caller's stream
+            HDT_ENQ(cudaEventRecord(sd->join, sd->s));
+            HDT_ENQ(cudaStreamWaitEvent(st, sd->join, 0));
         }
         return cudaGetLastError();
 #undef HDT_ENQ

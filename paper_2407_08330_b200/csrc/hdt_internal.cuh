@@ -100,7 +100,12 @@ int sm_count(int *n_sm);
 
 // Side stream (one per host thread and device, created on first use): work that does not depend
 // on the main kernel of a call runs beside it.  fork / join are events for the two hand-overs.
-struct Side { cudaStream_t s, s2, s3; cudaEvent_t fork, join, join2, join3, fork0, join0; bool ready; };      // fork0 / join0: a hand-over of their own for work that starts before `fork`
+struct Side {
+    cudaStream_t s, s2, s3;
+    cudaEvent_t fork, join, join2, join3, fork0, join0;      // fork0 / join0: a hand-over of their own for work that starts before `fork`
+    cudaEvent_t stage_ev[2 * HDT_MAX_STAGES];                // index build with a kernel chain per stage: [2 s] the stage's compaction is queued, [2 s + 1] its walk
+    bool ready;
+};
 int get_side(Side **out);
 extern int g_no_overlap;   // option "no_overlap"
 extern int g_force_simt;   // option "force_simt"
